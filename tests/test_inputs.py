@@ -39,7 +39,7 @@ def test_regression_recipe_structure():
         assert 0.07 < resid.std() < 0.12
     # across a segment boundary one map does not fit
     A, *_ = np.linalg.lstsq(k[0, 0, 0:1024].astype(np.float64), v[0, 0, 0:1024].astype(np.float64), rcond=None)
-    assert (v[0, 0, :1024] - k[0, 0, :1024] @ A).std() > 0.3
+    assert (v[0, 0, :1024] - k[0, 0, :1024] @ A).std() > 0.125   # signal std is 1/sqrt(d) = 0.125
 
 
 def test_decode_workload_and_sharding():
