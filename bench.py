@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the LLA hot path on B200: causal forward (prefill) throughput with its roofline,
+the decode step against HBM bandwidth, the end-to-end host-buffer number and the CPU oracle
+baseline.  Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole forward path (direct early rows + iterative rows) over one batch
+of the bf16 prefill workload B=4, H=8, n=1024, d=dv=64.  With N > 1 every rank runs that batch on
+its own GPU (independent (batch, head) problems, no collective on the data path: weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_01450_b200 import inputs  # noqa: E402
+
+METRIC = "lla_prefill_tokens_per_s"
+UNIT = "tokens/s"
+WORKLOAD = 2          # the bf16 prefill workload the headline metric is quoted on
+ROTATE = 16           # input sets cycled through so no step finds its inputs in L2
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
+# (None until a capture of the current kernel exists).
+NCU_TRAFFIC_BYTES = None
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML while the timed regions run."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def algorithmic_flops(w, iters: np.ndarray) -> float:
+    """N_p (8d + 2dv) + 6d sum_i (i+1) T_i per head, with the CG iterations actually executed
+    (rows solved directly contribute no iteration term)."""
+    n, d, dv = w.n, w.d, w.dv
+    pairs = n * (n + 1) / 2.0
+    it = np.maximum(iters.reshape(-1, n).astype(np.float64), 0.0)
+    vis = np.arange(1, n + 1, dtype=np.float64)
+    return float(it.shape[0] * pairs * (8 * d + 2 * dv) + 6.0 * d * (it * vis).sum())
+
+
+def oracle_sample_rows(w, n_rows: int, seed: int) -> np.ndarray:
+    rng = np.random.default_rng(seed)
+    return np.sort(rng.choice(w.B * w.H * w.n, size=min(n_rows, w.B * w.H * w.n), replace=False)).astype(np.int64)
+
+
+def run_reference(args):
+    """Reference arm: the float64 CPU oracle, as it stands, on a bounded sample of the workload."""
+    rank = env_int("RANK", 0)
+    if rank != 0:
+        return
+    from oracle import lla_oracle
+    w = inputs.CONFIGS[WORKLOAD]
+    q, k, v = inputs.make_prefill(w)
+    total_rows = w.B * w.H * w.n
+    # calibrate: rows are drawn uniformly over (batch, head, position), so the sample's mean cost
+    # per row equals the workload's
+    probe = oracle_sample_rows(w, 512, 1)
+    t0 = time.perf_counter()
+    lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=probe)
+    per_row = (time.perf_counter() - t0) / probe.size
+    budget_s = 120.0
+    rows_per_step = int(max(64, min(total_rows, budget_s / max(per_row, 1e-9) / (args.steps + args.warmup))))
+    for i in range(args.warmup):
+        lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=oracle_sample_rows(w, rows_per_step, 100 + i))
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=oracle_sample_rows(w, rows_per_step, 200 + i))
+    dt = time.perf_counter() - t0
+    value = rows_per_step * args.steps / dt
+    sample = f"{rows_per_step} of {total_rows} rows per step, drawn uniformly over (batch, head, position)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "dv": w.dv, "lambda": w.lam,
+                   "causal": True},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2510_01450_b200 as L
+
+    world = env_int("WORLD_SIZE", 1)
+    rank = env_int("RANK", 0)
+    local = env_int("LOCAL_RANK", 0)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peaks = load_peaks()
+    w = inputs.CONFIGS[WORKLOAD].shrink(seed=inputs.CONFIGS[WORKLOAD].seed + 1000 * rank)
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+
+    # ---- inputs: ROTATE seeded sets resident in HBM (together larger than L2) ----
+    q0, k0, v0 = inputs.make_prefill(w)
+    hq, hk, hv = (torch.from_numpy(x).to(torch.bfloat16) for x in (q0, k0, v0))
+    sets = []
+    for r in range(ROTATE):
+        # every set is the same seeded batch with its (batch, head) order rotated: same work, new addresses
+        sh = r % (w.B * w.H)
+        roll = lambda t: torch.roll(t.reshape(w.B * w.H, w.n, -1), sh, 0).reshape(t.shape).contiguous()
+        sets.append(tuple(roll(t).cuda() for t in (hq, hk, hv)))
+    outs = [torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16, device="cuda") for _ in range(ROTATE)]
+    set_bytes = sum(t.numel() * t.element_size() for t in sets[0]) + outs[0].numel() * 2
+
+    def step(i, phases=L.LLA_PHASE_ALL):
+        q, k, v = sets[i % ROTATE]
+        L.lla_forward_ex(q, k, v, outs[i % ROTATE], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1,
+                         phases=phases, stream=sp)
+
+    # iterations actually executed (for the algorithmic flop count), outside the timed region
+    iters = torch.zeros((w.B, w.H, w.n), dtype=torch.int32, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    L.lla_forward_ex(*sets[0], outs[0], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1, iters=iters,
+                     device_status=status, stream=sp)
+    torch.cuda.synchronize()
+    it_np = iters.cpu().numpy()
+    flops_step = algorithmic_flops(w, it_np)
+    cg_rows = it_np[it_np >= 0]
+    mean_iters = float(cg_rows.mean()) if cg_rows.size else 0.0
+
+    clocks = ClockSampler(local)
+    with clocks:
+        # ---- device-resident throughput ----
+        for i in range(args.warmup):
+            step(i)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            step(args.warmup + i)
+        e1.record(stream)
+        barrier()
+        ms_total = max_over_ranks(e0.elapsed_time(e1))
+
+        # ---- dominant kernel alone (iterative rows), per-launch average, same rotation ----
+        for i in range(3):
+            step(i, L.LLA_PHASE_ITERATIVE)
+        torch.cuda.synchronize()
+        k0e, k1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        k0e.record(stream)
+        for i in range(args.steps):
+            step(3 + i, L.LLA_PHASE_ITERATIVE)
+        k1e.record(stream)
+        torch.cuda.synchronize()
+        ms_kernel = k0e.elapsed_time(k1e) / args.steps
+        d0e, d1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0e.record(stream)
+        for i in range(args.steps):
+            step(i, L.LLA_PHASE_DIRECT)
+        d1e.record(stream)
+        torch.cuda.synchronize()
+        ms_direct = d0e.elapsed_time(d1e) / args.steps
+
+        # ---- end to end through the host-buffer entry point (pinned memory) ----
+        pq, pk, pv = (t.pin_memory() for t in (hq, hk, hv))
+        pout = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16).pin_memory()
+
+        def e2e_step():
+            L.lla_forward_host(pq, pk, pv, pout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_BF16, w.scale,
+                               w.lam, 1, sp)
+
+        for _ in range(max(3, args.warmup // 4)):
+            e2e_step()
+        e2e_steps = max(5, args.steps // 4)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        e2e_s = max_over_ranks(time.perf_counter() - t0)
+        barrier()
+
+        # ---- decode step (64 sequences x 16 heads over a bf16 KV cache), rank 0 only ----
+        decode = None
+        if rank == 0 and not args.no_decode:
+            decode = bench_decode(L, torch, peaks, sp, stream)
+
+    tokens_step = w.B * w.n
+    ms_step = ms_total / args.steps
+    value = world * tokens_step / (ms_step * 1e-3)
+    tflops_kernel = flops_step_iterative(w, it_np) / (ms_kernel * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "dv": w.dv, "lambda": w.lam,
+                   "causal": True, "cg_tol": 1e-4, "cg_mean_iters": mean_iters,
+                   "rows_at_iter_cap": int(status.cpu()[L.STATUS_ROWS_AT_CAP]),
+                   "l2": f"inputs rotate over {ROTATE} sets ({ROTATE * set_bytes / 1e6:.0f} MB > 126 MB L2)"},
+        "tflops": flops_step / (ms_step * 1e-3) / 1e12,
+        "roofline": {"bound": "tensor", "achieved": tflops_kernel, "peak": peak, "unit": "TFLOP/s",
+                     "frac": tflops_kernel / peak, "traffic": NCU_TRAFFIC_BYTES,
+                     "kernel": "iterative-rows forward kernel", "ms_per_launch": ms_kernel,
+                     "peak_source": f"{peaks['source']} burst bf16 (MEASURED_PEAKS.json)",
+                     "direct_rows_ms_per_launch": ms_direct},
+        "e2e": {"value": world * tokens_step * e2e_steps / e2e_s, "unit": UNIT,
+                "h2d_bytes_per_step": int(sum(t.numel() * 2 for t in (hq, hk, hv))),
+                "d2h_bytes_per_step": int(pout.numel() * 2), "steps": e2e_steps},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks.summary(),
+    }
+    if decode is not None:
+        line["decode"] = decode
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(w, q0, k0, v0)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def flops_step_iterative(w, iters):
+    """Algorithmic flops of the rows the iterative kernel computes (rows with iters >= 0)."""
+    n, d, dv = w.n, w.d, w.dv
+    it = iters.reshape(-1, n).astype(np.float64)
+    vis = np.arange(1, n + 1, dtype=np.float64)
+    mask = it >= 0
+    return float(((8 * d + 2 * dv) * (mask * vis).sum()) + 6.0 * d * (np.maximum(it, 0) * vis).sum())
+
+
+def bench_decode(L, torch, peaks, sp, stream, steps=20, warmup=5):
+    wd = inputs.CONFIGS[5]
+    gen = torch.Generator(device="cuda").manual_seed(wd.seed)
+    inv = 1.0 / np.sqrt(wd.d)
+    kc = (torch.randn((wd.B, wd.H, wd.n, wd.d), generator=gen, device="cuda", dtype=torch.float32) * inv).to(torch.bfloat16)
+    vc = torch.randn((wd.B, wd.H, wd.n, wd.dv), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    q = (torch.randn((wd.B, wd.H, wd.d), generator=gen, device="cuda", dtype=torch.float32) * inv).to(torch.bfloat16)
+    lens_np = np.random.default_rng(wd.seed).integers(wd.len_min, wd.len_max + 1, size=wd.B).astype(np.int32)
+    lens = torch.from_numpy(lens_np).cuda()
+    out = torch.empty((wd.B, wd.H, wd.dv), dtype=torch.bfloat16, device="cuda")
+    for _ in range(warmup):
+        L.lla_decode(q, kc, vc, lens, out, wd.B, wd.H, wd.n, wd.d, wd.dv, wd.scale, wd.lam, sp)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        L.lla_decode(q, kc, vc, lens, out, wd.B, wd.H, wd.n, wd.d, wd.dv, wd.scale, wd.lam, sp)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    live_bytes = float(lens_np.astype(np.int64).sum()) * wd.H * (wd.d + wd.dv) * 2
+    gbs = live_bytes / (ms * 1e-3) / 1e9
+    del kc, vc
+    return {"workload": wd.name, "us_per_step": ms * 1e3, "us_per_token": ms * 1e3 / wd.B, "steps": steps,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "algorithmic_bytes": live_bytes,
+                         "frac_of_nominal_8TBs": gbs / 8000.0,
+                         "peak_source": f"{peaks['source']} copy bandwidth (MEASURED_PEAKS.json)"},
+            "l2": "live cache bytes (1.2 GB) exceed L2 (126 MB)"}
+
+
+def cpu_baseline(w, q, k, v):
+    """The oracle, untuned, on this machine's host cores, on a bounded uniform row sample."""
+    from oracle import lla_oracle
+    probe = oracle_sample_rows(w, 256, 7)
+    t0 = time.perf_counter()
+    lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=probe)
+    per_row = (time.perf_counter() - t0) / probe.size
+    total = w.B * w.H * w.n
+    n_rows = int(max(256, min(total, 15.0 / max(per_row, 1e-9))))
+    rows = oracle_sample_rows(w, n_rows, 8)
+    t0 = time.perf_counter()
+    lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows)
+    dt = time.perf_counter() - t0
+    return {"value": rows.size / dt, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
+            "sample": f"{rows.size} of {total} rows of {w.name}, drawn uniformly over (batch, head, position); "
+                      f"{dt:.1f} s"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-decode", action="store_true", help="skip the decode measurement")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,207 @@
+/*
+ * lla.h - C ABI of the B200 (sm_100a) Local Linear Attention library.
+ *
+ * One hot path: the causal LLA forward pass and its single-query decode variant.
+ * For every query i the pass forms kernel weights w_ij = exp(scale * q_i.k_j) over the
+ * visible keys (j <= i when causal), the query-centred moments
+ *     omega_i = sum_j w_ij,  mu_i = sum_j w_ij (k_j - q_i),
+ *     Sigma_i = sum_j w_ij (k_j - q_i)(k_j - q_i)^T + lambda I        (Eq. "query_specific"),
+ * solves Sigma_i rho_i = mu_i without ever storing Sigma_i (matrix-free conjugate gradients,
+ * Section 3.1 / Algorithm 2; rows with very few visible keys are solved directly), and emits
+ *     o_i = sum_j w_ij (1 - (k_j - q_i)^T rho_i) v_j / (omega_i - mu_i^T rho_i)   (Eq. "lla").
+ *
+ * Conventions shared by every entry point
+ *   - All tensor pointers are DEVICE pointers unless a comment says "host".  Tensors are
+ *     contiguous, row-major, innermost index fastest, base address 16-byte aligned.
+ *   - The caller owns every buffer.  The library reads inputs, writes outputs (outputs must
+ *     not alias inputs), and keeps no pointer once the enqueued work has completed.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work
+ *     is enqueued on it; no entry point synchronises the device.
+ *   - Return value: an lla_status as int.  Argument errors are detected on the host before any
+ *     launch.  Nothing throws or aborts.  Conditions that only the device can see (rows that hit
+ *     the iteration cap, a failed pivot in a directly-solved row) are counted in the optional
+ *     `device_status` words, readable after the caller synchronises the stream.
+ *   - The library is CUDA only: there is no host fallback.  On a machine without a usable
+ *     device every launch returns LLA_ERR_CUDA.
+ *   - Supported head sizes: d = dv in {16, 64, 128}; other values return LLA_ERR_UNSUPPORTED.
+ *   - lambda must be >= 0.  With lambda == 0 rows that see fewer than d+1 keys have a singular
+ *     system; their output is unspecified (the paper's definition has no unique answer there).
+ */
+#ifndef LLA_H_
+#define LLA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lla_status {
+    LLA_OK = 0,
+    LLA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, negative lambda, non-finite scale */
+    LLA_ERR_UNSUPPORTED = 2, /* head size or dtype combination not compiled in */
+    LLA_ERR_WORKSPACE = 3,   /* caller workspace missing or too small */
+    LLA_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
+    LLA_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported via device_status) */
+} lla_status;
+
+typedef enum lla_dtype { LLA_BF16 = 0, LLA_F32 = 1 } lla_dtype;
+
+/* Implementation selector for lla_forward_ex. */
+typedef enum lla_impl {
+    LLA_IMPL_AUTO = 0,   /* tensor-core kernel where compiled for the shape, else SIMT */
+    LLA_IMPL_SIMT = 1,   /* fp32 CUDA-core kernel (every supported shape and dtype) */
+    LLA_IMPL_TENSOR = 2  /* tcgen05/TMEM kernel (bf16 inputs, d = dv = 64) */
+} lla_impl;
+
+/* Row groups for lla_forward_params.phases. */
+enum { LLA_PHASE_ALL = 0, LLA_PHASE_DIRECT = 1, LLA_PHASE_ITERATIVE = 2 };
+
+/* Words of the optional device_status array (int[LLA_STATUS_WORDS], zeroed by the call). */
+enum {
+    LLA_STATUS_ROWS_AT_CAP = 0,  /* rows whose CG stopped at max_iters above the tolerance */
+    LLA_STATUS_BAD_PIVOT = 1,    /* directly-solved rows whose Cholesky met a pivot <= 0 */
+    LLA_STATUS_TIMEOUT = 2,      /* bounded waits that expired (0 in a healthy run) */
+    LLA_STATUS_ITER_SUM = 3,     /* low 31 bits of the sum over CG rows of iterations executed */
+    LLA_STATUS_WORDS = 4
+};
+
+/*
+ * Causal LLA forward, bf16 in / bf16 out, fp32 accumulation (Section 3.2, matrix form and
+ * Algorithm 1; solver per Algorithm 2).
+ *   q, k : [B, H, n, d]  bf16      v : [B, H, n, dv] bf16      out : [B, H, n, dv] bf16
+ *   scale  : multiplies q.k inside exp (the paper's 1/h); lambda : ridge, >= 0
+ *   causal : nonzero -> row i sees keys 0..i (diagonal included); zero -> every row sees all n
+ * Uses the default solver settings (see lla_forward_ex) and no caller workspace.
+ */
+int lla_forward(const void *q, const void *k, const void *v, void *out, int B, int H, int n, int d,
+                int dv, float scale, float lambda, int causal, void *stream);
+
+/* Same operation with fp32 inputs and fp32 output (fp32 arithmetic, tighter solver tolerance). */
+int lla_forward_f32(const void *q, const void *k, const void *v, void *out, int B, int H, int n,
+                    int d, int dv, float scale, float lambda, int causal, void *stream);
+
+/*
+ * Single-query decode over a KV cache: Eq. "lla" for one query per (sequence, head).  The paper
+ * only names an inference kernel; the semantics are its definition at one row.
+ *   q      : [B, H, d]                 bf16
+ *   kcache : [B, H, Lmax, d]           bf16     vcache : [B, H, Lmax, dv] bf16
+ *   lens   : [B] int32, DEVICE pointer, 1 <= lens[b] <= Lmax.  lens[b] counts the current token,
+ *            whose key and value are already stored in the cache (this matches j <= i).
+ *            A length outside [1, Lmax] is clamped into that range on the device.
+ *   out    : [B, H, dv]                bf16
+ */
+int lla_decode(const void *q, const void *kcache, const void *vcache, const int *lens, void *out,
+               int B, int H, int Lmax, int d, int dv, float scale, float lambda, void *stream);
+
+/* Decode with fp32 caches, query and output. */
+int lla_decode_f32(const void *q, const void *kcache, const void *vcache, const int *lens,
+                   void *out, int B, int H, int Lmax, int d, int dv, float scale, float lambda,
+                   void *stream);
+
+/*
+ * Full-control forward.  Zero-initialise the struct, then set fields; zero / NULL means default.
+ *   in_dtype / out_dtype : lla_dtype of q,k,v and of out (bf16 inputs may write an fp32 output)
+ *   max_iters : CG iteration cap per row (default 48; Algorithm 2's T)
+ *   tol       : CG stops a row when |residual| <= tol * |right-hand side| (Algorithm 2's
+ *               epsilon; default 1e-4 for bf16 inputs, 1e-6 for fp32 inputs)
+ *   head_rows : rows that see fewer than this many keys are solved directly in fp64 from the
+ *               explicit d x d system instead of by CG (0 = default 2*d; negative disables).  Those early systems are too ill-conditioned for fp32 CG.
+ *   impl      : lla_impl
+ *   phases    : which groups of rows to compute: 0 = all; LLA_PHASE_DIRECT = only the rows
+ *               solved directly; LLA_PHASE_ITERATIVE = only the rows solved by CG (profiling aid:
+ *               the other rows of `out` are left untouched)
+ *   rho       : optional [B, H, n, d] fp32, the solutions Sigma_i^{-1} mu_i (Algorithm 1 keeps
+ *               them for the backward pass)
+ *   stats     : optional [B, H, n, 3] fp32: row maximum m_i of the scaled scores, omega_i and
+ *               delta_i = omega_i - mu_i^T rho_i, the last two for weights exp(score - m_i)
+ *   iters     : optional [B, H, n] int32, CG iterations executed for the row (-1 for rows solved
+ *               directly)
+ *   device_status : optional int[LLA_STATUS_WORDS] on the device
+ *   workspace / workspace_bytes : device scratch of at least lla_forward_workspace_bytes(...)
+ *               bytes, 256-byte aligned; may be NULL when that function returns 0
+ */
+typedef struct lla_forward_params {
+    const void *q, *k, *v;
+    void *out;
+    int B, H, n, d, dv;
+    int in_dtype, out_dtype;
+    float scale, lambda;
+    int causal;
+    int max_iters;
+    float tol;
+    int head_rows;
+    int impl;
+    int phases;
+    float *rho;
+    float *stats;
+    int *iters;
+    int *device_status;
+    void *workspace;
+    size_t workspace_bytes;
+    void *stream;
+} lla_forward_params;
+
+int lla_forward_ex(const lla_forward_params *p);
+
+/*
+ * Full-control decode.  Fields as in lla_decode; additionally
+ *   in_dtype / out_dtype : lla_dtype of q and the caches, and of out
+ *   splits    : number of key-range parts each (sequence, head) is divided into so that long
+ *               caches spread over more thread blocks (0 = chosen from B*H and Lmax; 1 = none).
+ *               With splits > 1 partial moments go through `workspace`.
+ *   workspace : device scratch of at least lla_decode_workspace_bytes(...) bytes, 256-byte
+ *               aligned; required when the effective number of splits exceeds 1
+ */
+typedef struct lla_decode_params {
+    const void *q, *kcache, *vcache;
+    const int *lens;
+    void *out;
+    int B, H, Lmax, d, dv;
+    int in_dtype, out_dtype;
+    float scale, lambda;
+    int splits;
+    int impl;
+    int *device_status;
+    void *workspace;
+    size_t workspace_bytes;
+    void *stream;
+} lla_decode_params;
+
+int lla_decode_ex(const lla_decode_params *p);
+
+/*
+ * Host-buffer convenience forms of the two operations above (same mathematics, Eq. "lla").
+ * q, k, v, lens and out are HOST pointers (pinned memory gives the fastest copies; pageable
+ * memory works).  The call allocates device buffers from the stream-ordered pool, copies the
+ * inputs up, runs the device path on `stream`, copies the result back and SYNCHRONISES the
+ * stream before returning, so `out` is valid on return.  dtypes are lla_dtype values.
+ * lla_decode_host reads lens[] on the host and uploads only the first lens[b] rows of every
+ * (sequence, head) cache.
+ */
+int lla_forward_host(const void *q, const void *k, const void *v, void *out, int B, int H, int n,
+                     int d, int dv, int in_dtype, int out_dtype, float scale, float lambda,
+                     int causal, void *stream);
+int lla_decode_host(const void *q, const void *kcache, const void *vcache, const int *lens,
+                    void *out, int B, int H, int Lmax, int d, int dv, int in_dtype, int out_dtype,
+                    float scale, float lambda, void *stream);
+
+/* Scratch bytes lla_forward_ex needs for this problem (0 when none). Host-only arithmetic. */
+size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl);
+
+/* Scratch bytes lla_decode_ex needs for this problem and split count (0 when splits <= 1). */
+size_t lla_decode_workspace_bytes(int B, int H, int Lmax, int d, int dv, int in_dtype, int splits);
+
+/* Number of key-range parts lla_decode / lla_decode_ex(splits = 0) would use. */
+int lla_decode_default_splits(int B, int H, int Lmax);
+
+/* Static, NUL-terminated description of a status code. */
+const char *lla_status_string(int status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int lla_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLA_H_ */

@@ -1,0 +1,186 @@
+"""ctypes binding of ``liblla.so``: the same names as ``include/lla.h``, argument marshalling only.
+
+Every function takes device tensors (anything with ``data_ptr()``; torch is used by callers for
+memory and streams only) or raw integer addresses, and returns nothing; a non-zero status from the
+library raises ``LlaError``.  There is no CPU fallback: if the shared library is missing the first
+call raises, telling how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "liblla.so"
+_lib = None
+
+LLA_BF16, LLA_F32 = 0, 1
+LLA_IMPL_AUTO, LLA_IMPL_SIMT, LLA_IMPL_TENSOR = 0, 1, 2
+LLA_STATUS_WORDS = 4
+LLA_PHASE_ALL, LLA_PHASE_DIRECT, LLA_PHASE_ITERATIVE = 0, 1, 2
+STATUS_ROWS_AT_CAP, STATUS_BAD_PIVOT, STATUS_TIMEOUT, STATUS_ITER_SUM = 0, 1, 2, 3
+
+EXPORTS = (
+    "lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex", "lla_decode_ex",
+    "lla_forward_host", "lla_decode_host", "lla_forward_workspace_bytes", "lla_decode_workspace_bytes",
+    "lla_decode_default_splits", "lla_status_string", "lla_version",
+)
+
+
+class LlaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+class ForwardParams(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
+        ("B", ctypes.c_int), ("H", ctypes.c_int), ("n", ctypes.c_int), ("d", ctypes.c_int), ("dv", ctypes.c_int),
+        ("in_dtype", ctypes.c_int), ("out_dtype", ctypes.c_int),
+        ("scale", ctypes.c_float), ("lambda_", ctypes.c_float),
+        ("causal", ctypes.c_int), ("max_iters", ctypes.c_int), ("tol", ctypes.c_float),
+        ("head_rows", ctypes.c_int), ("impl", ctypes.c_int), ("phases", ctypes.c_int),
+        ("rho", ctypes.c_void_p), ("stats", ctypes.c_void_p), ("iters", ctypes.c_void_p),
+        ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
+class DecodeParams(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("kcache", ctypes.c_void_p), ("vcache", ctypes.c_void_p),
+        ("lens", ctypes.c_void_p), ("out", ctypes.c_void_p),
+        ("B", ctypes.c_int), ("H", ctypes.c_int), ("Lmax", ctypes.c_int), ("d", ctypes.c_int), ("dv", ctypes.c_int),
+        ("in_dtype", ctypes.c_int), ("out_dtype", ctypes.c_int),
+        ("scale", ctypes.c_float), ("lambda_", ctypes.c_float),
+        ("splits", ctypes.c_int), ("impl", ctypes.c_int),
+        ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
+def load():
+    """Load ``liblla.so`` and declare the prototypes.  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2510_01450_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    fwd = [vp, vp, vp, vp, i, i, i, i, i, f, f, i, vp]
+    dec = [vp, vp, vp, vp, vp, i, i, i, i, i, f, f, vp]
+    lib.lla_forward.argtypes = fwd
+    lib.lla_forward_f32.argtypes = fwd
+    lib.lla_decode.argtypes = dec
+    lib.lla_decode_f32.argtypes = dec
+    lib.lla_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, f, i, vp]
+    lib.lla_decode_host.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, f, vp]
+    lib.lla_forward_ex.argtypes = [ctypes.POINTER(ForwardParams)]
+    lib.lla_decode_ex.argtypes = [ctypes.POINTER(DecodeParams)]
+    for name in ("lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex",
+                 "lla_decode_ex", "lla_forward_host", "lla_decode_host", "lla_version",
+                 "lla_decode_default_splits"):
+        getattr(lib, name).restype = i
+    lib.lla_decode_default_splits.argtypes = [i, i, i]
+    lib.lla_forward_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
+    lib.lla_forward_workspace_bytes.restype = sz
+    lib.lla_decode_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
+    lib.lla_decode_workspace_bytes.restype = sz
+    lib.lla_status_string.argtypes = [i]
+    lib.lla_status_string.restype = ctypes.c_char_p
+    lib.lla_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _p(x):
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        return ctypes.c_void_p(x.data_ptr())
+    return ctypes.c_void_p(int(x))
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise LlaError(rc, where)
+
+
+def status_string(status: int) -> str:
+    return load().lla_status_string(int(status)).decode()
+
+
+def lla_version() -> int:
+    return int(load().lla_version())
+
+
+def lla_forward(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, stream=0):
+    _check(load().lla_forward(_p(q), _p(k), _p(v), _p(out), B, H, n, d, dv, scale, lam, int(causal), _p(stream)),
+           "lla_forward")
+
+
+def lla_forward_f32(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, stream=0):
+    _check(load().lla_forward_f32(_p(q), _p(k), _p(v), _p(out), B, H, n, d, dv, scale, lam, int(causal),
+                                  _p(stream)), "lla_forward_f32")
+
+
+def lla_decode(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, stream=0):
+    _check(load().lla_decode(_p(q), _p(kcache), _p(vcache), _p(lens), _p(out), B, H, Lmax, d, dv, scale, lam,
+                             _p(stream)), "lla_decode")
+
+
+def lla_decode_f32(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, stream=0):
+    _check(load().lla_decode_f32(_p(q), _p(kcache), _p(vcache), _p(lens), _p(out), B, H, Lmax, d, dv, scale, lam,
+                                 _p(stream)), "lla_decode_f32")
+
+
+def lla_forward_host(q, k, v, out, B, H, n, d, dv, in_dtype, out_dtype, scale, lam, causal=1, stream=0):
+    """Host-buffer form: q, k, v, out are host tensors/addresses; synchronises ``stream``."""
+    _check(load().lla_forward_host(_p(q), _p(k), _p(v), _p(out), B, H, n, d, dv, in_dtype, out_dtype, scale, lam,
+                                   int(causal), _p(stream)), "lla_forward_host")
+
+
+def lla_decode_host(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, in_dtype, out_dtype, scale, lam, stream=0):
+    _check(load().lla_decode_host(_p(q), _p(kcache), _p(vcache), _p(lens), _p(out), B, H, Lmax, d, dv, in_dtype,
+                                  out_dtype, scale, lam, _p(stream)), "lla_decode_host")
+
+
+def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=LLA_BF16, out_dtype=LLA_BF16,
+                   max_iters=0, tol=0.0, head_rows=0, impl=LLA_IMPL_AUTO, phases=0, rho=None, stats=None, iters=None,
+                   device_status=None, workspace=None, workspace_bytes=0, stream=0):
+    p = ForwardParams()
+    p.q, p.k, p.v, p.out = _p(q), _p(k), _p(v), _p(out)
+    p.B, p.H, p.n, p.d, p.dv = B, H, n, d, dv
+    p.in_dtype, p.out_dtype = in_dtype, out_dtype
+    p.scale, p.lambda_, p.causal = scale, lam, int(causal)
+    p.max_iters, p.tol, p.head_rows, p.impl, p.phases = max_iters, tol, head_rows, impl, phases
+    p.rho, p.stats, p.iters, p.device_status = _p(rho), _p(stats), _p(iters), _p(device_status)
+    p.workspace, p.workspace_bytes, p.stream = _p(workspace), workspace_bytes, _p(stream)
+    _check(load().lla_forward_ex(ctypes.byref(p)), "lla_forward_ex")
+
+
+def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, in_dtype=LLA_BF16,
+                  out_dtype=LLA_BF16, splits=0, impl=LLA_IMPL_AUTO, device_status=None, workspace=None,
+                  workspace_bytes=0, stream=0):
+    p = DecodeParams()
+    p.q, p.kcache, p.vcache, p.lens, p.out = _p(q), _p(kcache), _p(vcache), _p(lens), _p(out)
+    p.B, p.H, p.Lmax, p.d, p.dv = B, H, Lmax, d, dv
+    p.in_dtype, p.out_dtype = in_dtype, out_dtype
+    p.scale, p.lambda_, p.splits, p.impl = scale, lam, splits, impl
+    p.device_status, p.workspace, p.workspace_bytes, p.stream = _p(device_status), _p(workspace), workspace_bytes, _p(stream)
+    _check(load().lla_decode_ex(ctypes.byref(p)), "lla_decode_ex")
+
+
+def lla_forward_workspace_bytes(B, H, n, d, dv, in_dtype=LLA_BF16, impl=LLA_IMPL_AUTO) -> int:
+    return int(load().lla_forward_workspace_bytes(B, H, n, d, dv, in_dtype, impl))
+
+
+def lla_decode_workspace_bytes(B, H, Lmax, d, dv, in_dtype=LLA_BF16, splits=1) -> int:
+    return int(load().lla_decode_workspace_bytes(B, H, Lmax, d, dv, in_dtype, splits))
+
+
+def lla_decode_default_splits(B, H, Lmax) -> int:
+    return int(load().lla_decode_default_splits(B, H, Lmax))

@@ -1,0 +1,297 @@
+// C-ABI entry points: argument validation, defaults, dispatch.  See include/lla.h for the contract.
+#include <math.h>
+
+#include "lla_common.cuh"
+
+namespace {
+
+using lla::DecodeArgs;
+using lla::ForwardArgs;
+
+bool head_size_ok(int d, int dv) { return d == dv && (d == 16 || d == 64 || d == 128); }
+
+int check_forward(const lla_forward_params* p) {
+    if (!p) return LLA_ERR_INVALID_ARG;
+    if (!p->q || !p->k || !p->v || !p->out) return LLA_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->n < 1 || p->d < 1 || p->dv < 1) return LLA_ERR_INVALID_ARG;
+    if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
+    if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
+    if ((long long)p->B * p->H > 65535) return LLA_ERR_UNSUPPORTED;
+    if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
+    const bool dt_ok = (p->in_dtype == LLA_BF16 && (p->out_dtype == LLA_BF16 || p->out_dtype == LLA_F32)) ||
+                       (p->in_dtype == LLA_F32 && p->out_dtype == LLA_F32);
+    if (!dt_ok) return LLA_ERR_UNSUPPORTED;
+    if (p->impl != LLA_IMPL_AUTO && p->impl != LLA_IMPL_SIMT && p->impl != LLA_IMPL_TENSOR)
+        return LLA_ERR_INVALID_ARG;
+    if (p->phases < LLA_PHASE_ALL || p->phases > LLA_PHASE_ITERATIVE) return LLA_ERR_INVALID_ARG;
+    const uintptr_t align = (uintptr_t)p->q | (uintptr_t)p->k | (uintptr_t)p->v | (uintptr_t)p->out;
+    if (align & 15u) return LLA_ERR_INVALID_ARG;
+    return LLA_OK;
+}
+
+ForwardArgs to_args(const lla_forward_params* p) {
+    ForwardArgs a;
+    a.q = p->q; a.k = p->k; a.v = p->v; a.out = p->out;
+    a.B = p->B; a.H = p->H; a.n = p->n; a.d = p->d; a.dv = p->dv;
+    a.in_dtype = p->in_dtype; a.out_dtype = p->out_dtype;
+    a.scale = p->scale; a.lambda = p->lambda; a.causal = p->causal ? 1 : 0;
+    a.max_iters = p->max_iters > 0 ? p->max_iters : 48;
+    a.tol = p->tol > 0.f ? p->tol : (p->in_dtype == LLA_F32 ? 1e-6f : 1e-4f);
+    a.head_rows = p->head_rows == 0 ? 2 * p->d : (p->head_rows < 0 ? 0 : p->head_rows);
+    a.rho = p->rho; a.stats = p->stats; a.iters = p->iters; a.status = p->device_status;
+    a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
+    a.stream = (cudaStream_t)p->stream;
+    return a;
+}
+
+int check_decode(const lla_decode_params* p) {
+    if (!p) return LLA_ERR_INVALID_ARG;
+    if (!p->q || !p->kcache || !p->vcache || !p->lens || !p->out) return LLA_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->Lmax < 1 || p->d < 1 || p->dv < 1 || p->splits < 0) return LLA_ERR_INVALID_ARG;
+    if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
+    if ((long long)p->B * p->H > 65535) return LLA_ERR_UNSUPPORTED;
+    if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
+    const bool dt_ok = (p->in_dtype == LLA_BF16 && (p->out_dtype == LLA_BF16 || p->out_dtype == LLA_F32)) ||
+                       (p->in_dtype == LLA_F32 && p->out_dtype == LLA_F32);
+    if (!dt_ok) return LLA_ERR_UNSUPPORTED;
+    const uintptr_t align = (uintptr_t)p->q | (uintptr_t)p->kcache | (uintptr_t)p->vcache | (uintptr_t)p->out;
+    if (align & 15u) return LLA_ERR_INVALID_ARG;
+    return LLA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lla_forward_ex(const lla_forward_params* p) {
+    const int rc = check_forward(p);
+    if (rc != LLA_OK) return rc;
+    ForwardArgs a = to_args(p);
+    const bool tensor_ok = lla::forward_tensor_supported(a);
+    if (p->impl == LLA_IMPL_TENSOR && !tensor_ok) return LLA_ERR_UNSUPPORTED;
+    const bool use_tensor = tensor_ok && p->impl != LLA_IMPL_SIMT;
+    const size_t need = lla_forward_workspace_bytes(a.B, a.H, a.n, a.d, a.dv, a.in_dtype,
+                                                    use_tensor ? LLA_IMPL_TENSOR : LLA_IMPL_SIMT);
+    if (need > 0 && (!a.workspace || a.workspace_bytes < need || ((uintptr_t)a.workspace & 255u)))
+        return LLA_ERR_WORKSPACE;
+    if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
+    if (p->phases != LLA_PHASE_ITERATIVE) {
+        const int st = lla::launch_head_rows(a);
+        if (st != LLA_OK) return st;
+    }
+    if (p->phases == LLA_PHASE_DIRECT) return LLA_OK;
+    return use_tensor ? lla::launch_forward_tensor(a) : lla::launch_forward_simt(a);
+}
+
+int lla_forward(const void* q, const void* k, const void* v, void* out, int B, int H, int n, int d, int dv,
+                float scale, float lambda, int causal, void* stream) {
+    lla_forward_params p = {};
+    p.q = q; p.k = k; p.v = v; p.out = out;
+    p.B = B; p.H = H; p.n = n; p.d = d; p.dv = dv;
+    p.in_dtype = LLA_BF16; p.out_dtype = LLA_BF16;
+    p.scale = scale; p.lambda = lambda; p.causal = causal;
+    p.stream = stream;
+    return lla_forward_ex(&p);
+}
+
+int lla_forward_f32(const void* q, const void* k, const void* v, void* out, int B, int H, int n, int d,
+                    int dv, float scale, float lambda, int causal, void* stream) {
+    lla_forward_params p = {};
+    p.q = q; p.k = k; p.v = v; p.out = out;
+    p.B = B; p.H = H; p.n = n; p.d = d; p.dv = dv;
+    p.in_dtype = LLA_F32; p.out_dtype = LLA_F32;
+    p.scale = scale; p.lambda = lambda; p.causal = causal;
+    p.stream = stream;
+    return lla_forward_ex(&p);
+}
+
+int lla_decode_default_splits(int B, int H, int Lmax) {
+    // enough thread blocks to fill 148 SMs twice over, but no part shorter than 512 keys
+    const long long bh = (long long)B * H;
+    if (bh <= 0 || Lmax <= 0) return 1;
+    long long s = (2 * 148 + bh - 1) / bh;
+    const long long cap = Lmax / 512 > 1 ? Lmax / 512 : 1;
+    if (s > cap) s = cap;
+    if (s > 32) s = 32;
+    return s < 1 ? 1 : (int)s;
+}
+
+int lla_decode_ex(const lla_decode_params* p) {
+    const int rc = check_decode(p);
+    if (rc != LLA_OK) return rc;
+    DecodeArgs a;
+    a.q = p->q; a.kcache = p->kcache; a.vcache = p->vcache; a.lens = p->lens; a.out = p->out;
+    a.B = p->B; a.H = p->H; a.Lmax = p->Lmax; a.d = p->d; a.dv = p->dv;
+    a.in_dtype = p->in_dtype; a.out_dtype = p->out_dtype;
+    a.scale = p->scale; a.lambda = p->lambda;
+    a.splits = p->splits > 0 ? p->splits : lla_decode_default_splits(p->B, p->H, p->Lmax);
+    if (p->splits == 0 && a.splits > 1) {
+        // default split count, but the caller gave no (or too small a) workspace: run unsplit
+        const size_t need = lla::decode_workspace_bytes(a.B, a.H, a.d, a.dv, a.splits);
+        if (!p->workspace || p->workspace_bytes < need) a.splits = 1;
+    }
+    if (a.splits > 1 && ((uintptr_t)p->workspace & 255u)) return LLA_ERR_WORKSPACE;
+    a.status = p->device_status;
+    a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
+    a.stream = (cudaStream_t)p->stream;
+    if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
+    return lla::launch_decode(a);
+}
+
+int lla_decode(const void* q, const void* kcache, const void* vcache, const int* lens, void* out, int B,
+               int H, int Lmax, int d, int dv, float scale, float lambda, void* stream) {
+    lla_decode_params p = {};
+    p.q = q; p.kcache = kcache; p.vcache = vcache; p.lens = lens; p.out = out;
+    p.B = B; p.H = H; p.Lmax = Lmax; p.d = d; p.dv = dv;
+    p.in_dtype = LLA_BF16; p.out_dtype = LLA_BF16;
+    p.scale = scale; p.lambda = lambda;
+    p.stream = stream;
+    return lla_decode_ex(&p);
+}
+
+int lla_decode_f32(const void* q, const void* kcache, const void* vcache, const int* lens, void* out,
+                   int B, int H, int Lmax, int d, int dv, float scale, float lambda, void* stream) {
+    lla_decode_params p = {};
+    p.q = q; p.kcache = kcache; p.vcache = vcache; p.lens = lens; p.out = out;
+    p.B = B; p.H = H; p.Lmax = Lmax; p.d = d; p.dv = dv;
+    p.in_dtype = LLA_F32; p.out_dtype = LLA_F32;
+    p.scale = scale; p.lambda = lambda;
+    p.stream = stream;
+    return lla_decode_ex(&p);
+}
+
+size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl) {
+    (void)B; (void)H; (void)n; (void)d; (void)dv; (void)in_dtype; (void)impl;
+    return 0;
+}
+
+size_t lla_decode_workspace_bytes(int B, int H, int Lmax, int d, int dv, int in_dtype, int splits) {
+    (void)Lmax; (void)in_dtype;
+    if (B < 1 || H < 1 || d < 1 || dv < 1) return 0;
+    return lla::decode_workspace_bytes(B, H, d, dv, splits);
+}
+
+const char* lla_status_string(int status) {
+    switch (status) {
+        case LLA_OK: return "ok";
+        case LLA_ERR_INVALID_ARG: return "invalid argument";
+        case LLA_ERR_UNSUPPORTED: return "unsupported head size or dtype";
+        case LLA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case LLA_ERR_CUDA: return "CUDA runtime error";
+        case LLA_ERR_TIMEOUT: return "bounded device wait expired";
+        default: return "unknown status";
+    }
+}
+
+int lla_version(void) { return 100; }
+
+}  // extern "C"
+
+// ---- host-buffer convenience entry points --------------------------------------------------
+namespace {
+
+struct DeviceScratch {   // stream-ordered allocations released on scope exit
+    cudaStream_t stream;
+    void* ptrs[8];
+    int count = 0;
+    explicit DeviceScratch(cudaStream_t s) : stream(s) {}
+    void* get(size_t bytes) {
+        void* p = nullptr;
+        if (count >= 8 || cudaMallocAsync(&p, bytes ? bytes : 16, stream) != cudaSuccess) return nullptr;
+        ptrs[count++] = p;
+        return p;
+    }
+    ~DeviceScratch() {
+        for (int i = 0; i < count; ++i) cudaFreeAsync(ptrs[i], stream);
+    }
+};
+
+void keep_pool_memory() {
+    // let the stream-ordered pool keep freed blocks so repeated host-buffer calls do not re-allocate
+    static bool done = false;
+    if (done) return;
+    int dev = 0;
+    cudaMemPool_t pool;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+        unsigned long long keep = ~0ull;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    }
+    done = true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lla_forward_host(const void* q, const void* k, const void* v, void* out, int B, int H, int n, int d,
+                     int dv, int in_dtype, int out_dtype, float scale, float lambda, int causal, void* stream) {
+    lla_forward_params p = {};
+    p.q = q; p.k = k; p.v = v; p.out = out;   // host pointers: only checked for null / alignment here
+    p.B = B; p.H = H; p.n = n; p.d = d; p.dv = dv;
+    p.in_dtype = in_dtype; p.out_dtype = out_dtype;
+    p.scale = scale; p.lambda = lambda; p.causal = causal;
+    p.stream = stream;
+    const int rc = check_forward(&p);
+    if (rc != LLA_OK) return rc;
+    keep_pool_memory();
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t esz_in = in_dtype == LLA_F32 ? 4 : 2, esz_out = out_dtype == LLA_F32 ? 4 : 2;
+    const size_t nq = (size_t)B * H * n * d * esz_in, nv = (size_t)B * H * n * dv * esz_in;
+    const size_t no = (size_t)B * H * n * dv * esz_out;
+    DeviceScratch mem(st);
+    void* dq = mem.get(nq); void* dk = mem.get(nq); void* dvv = mem.get(nv); void* dout = mem.get(no);
+    if (!dq || !dk || !dvv || !dout) return LLA_ERR_CUDA;
+    LLA_CUDA_TRY(cudaMemcpyAsync(dq, q, nq, cudaMemcpyHostToDevice, st));
+    LLA_CUDA_TRY(cudaMemcpyAsync(dk, k, nq, cudaMemcpyHostToDevice, st));
+    LLA_CUDA_TRY(cudaMemcpyAsync(dvv, v, nv, cudaMemcpyHostToDevice, st));
+    p.q = dq; p.k = dk; p.v = dvv; p.out = dout;
+    const int st_rc = lla_forward_ex(&p);
+    if (st_rc != LLA_OK) return st_rc;
+    LLA_CUDA_TRY(cudaMemcpyAsync(out, dout, no, cudaMemcpyDeviceToHost, st));
+    LLA_CUDA_TRY(cudaStreamSynchronize(st));
+    return LLA_OK;
+}
+
+int lla_decode_host(const void* q, const void* kcache, const void* vcache, const int* lens, void* out, int B,
+                    int H, int Lmax, int d, int dv, int in_dtype, int out_dtype, float scale, float lambda,
+                    void* stream) {
+    lla_decode_params p = {};
+    p.q = q; p.kcache = kcache; p.vcache = vcache; p.lens = lens; p.out = out;
+    p.B = B; p.H = H; p.Lmax = Lmax; p.d = d; p.dv = dv;
+    p.in_dtype = in_dtype; p.out_dtype = out_dtype;
+    p.scale = scale; p.lambda = lambda;
+    p.splits = 1;
+    p.stream = stream;
+    const int rc = check_decode(&p);
+    if (rc != LLA_OK) return rc;
+    keep_pool_memory();
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t esz_in = in_dtype == LLA_F32 ? 4 : 2, esz_out = out_dtype == LLA_F32 ? 4 : 2;
+    const size_t nq = (size_t)B * H * d * esz_in, no = (size_t)B * H * dv * esz_out;
+    const size_t nk = (size_t)B * H * Lmax * d * esz_in, nv = (size_t)B * H * Lmax * dv * esz_in;
+    DeviceScratch mem(st);
+    void* dq = mem.get(nq); void* dk = mem.get(nk); void* dvv = mem.get(nv);
+    void* dl = mem.get(sizeof(int) * (size_t)B); void* dout = mem.get(no);
+    if (!dq || !dk || !dvv || !dl || !dout) return LLA_ERR_CUDA;
+    LLA_CUDA_TRY(cudaMemcpyAsync(dq, q, nq, cudaMemcpyHostToDevice, st));
+    LLA_CUDA_TRY(cudaMemcpyAsync(dl, lens, sizeof(int) * (size_t)B, cudaMemcpyHostToDevice, st));
+    // only the live prefix of every (sequence, head) cache crosses the bus
+    for (int b = 0; b < B; ++b) {
+        int L = lens[b] < 1 ? 1 : (lens[b] > Lmax ? Lmax : lens[b]);
+        for (int h = 0; h < H; ++h) {
+            const size_t off = ((size_t)b * H + h) * Lmax;
+            LLA_CUDA_TRY(cudaMemcpyAsync((char*)dk + off * d * esz_in, (const char*)kcache + off * d * esz_in,
+                                         (size_t)L * d * esz_in, cudaMemcpyHostToDevice, st));
+            LLA_CUDA_TRY(cudaMemcpyAsync((char*)dvv + off * dv * esz_in, (const char*)vcache + off * dv * esz_in,
+                                         (size_t)L * dv * esz_in, cudaMemcpyHostToDevice, st));
+        }
+    }
+    p.q = dq; p.kcache = dk; p.vcache = dvv; p.lens = (const int*)dl; p.out = dout;
+    const int st_rc = lla_decode_ex(&p);
+    if (st_rc != LLA_OK) return st_rc;
+    LLA_CUDA_TRY(cudaMemcpyAsync(out, dout, no, cudaMemcpyDeviceToHost, st));
+    LLA_CUDA_TRY(cudaStreamSynchronize(st));
+    return LLA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,241 @@
+// Direct fp64 solve for the rows that see only a few keys.
+//
+// For a row with L visible keys and L < head_rows (default 2d) the system Sigma_i rho_i = mu_i of
+// Eq. "query_specific" has condition numbers of 1e4..1e5 at the paper's ridge sizes (Sigma_i is
+// low rank plus lambda*I while L < d).  fp32 conjugate gradients cannot resolve that, so these few
+// rows are computed exactly as Section 2.3 writes them: explicit moments, an LDL^T factorisation
+// of the d x d matrix in shared memory, and the intercept of Eq. "lla".  They are 2d/n of the
+// rows and about (2d/n)^2 of the pair work.
+//
+// One thread block per (batch*head, row).  All arithmetic is double precision.
+#include "lla_common.cuh"
+
+namespace lla {
+namespace {
+
+constexpr int HR_THREADS = 256;
+constexpr int HR_CHUNK = 16;  // keys staged per step of the moment build
+
+template <int D>
+struct HrCfg {
+    static constexpr int TILES_1D = D / 4;                           // 4x4 register tiles
+    static constexpr int TILES = TILES_1D * (TILES_1D + 1) / 2;      // lower triangle incl. diagonal
+    static constexpr int TILES_PER_THREAD = (TILES + HR_THREADS - 1) / HR_THREADS;
+    static constexpr int LDS = D + 1;                                // padded row stride (doubles)
+};
+
+__device__ __forceinline__ double block_reduce(double x, bool is_max, double* scratch) {
+    // scratch: HR_THREADS/32 + 1 doubles
+    for (int off = 16; off > 0; off >>= 1) {
+        const double y = __shfl_xor_sync(0xffffffffu, x, off);
+        x = is_max ? fmax(x, y) : x + y;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) scratch[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+        double t = lane < HR_THREADS / 32 ? scratch[lane] : (is_max ? -INFINITY : 0.0);
+        for (int off = 16; off > 0; off >>= 1) {
+            const double y = __shfl_xor_sync(0xffffffffu, t, off);
+            t = is_max ? fmax(t, y) : t + y;
+        }
+        if (lane == 0) scratch[HR_THREADS / 32] = t;
+    }
+    __syncthreads();
+    return scratch[HR_THREADS / 32];
+}
+
+template <int D, int DV, typename TIn, typename TOut>
+__global__ void __launch_bounds__(HR_THREADS)
+head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
+                 TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
+                 double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
+                 int* __restrict__ iters, int* __restrict__ status) {
+    using C = HrCfg<D>;
+    extern __shared__ double smem[];
+    double* S = smem;                       // D * LDS
+    double* qd = S + D * C::LDS;            // D
+    double* rhs = qd + D;                   // D  (mu, then rho)
+    double* w = rhs + D;                    // lcap (scores -> weights -> coefficients)
+    double* zc = w + lcap;                  // HR_CHUNK * D  centred keys of the current chunk
+    double* red = zc + HR_CHUNK * D;        // HR_THREADS/32 + 1
+
+    const int tid = threadIdx.x;
+    const int bh = blockIdx.y;
+    const int i = blockIdx.x;               // row index inside the head
+    if (i >= rows_per_head) return;
+    const int L = causal ? i + 1 : n;
+    const TIn* qrow = q + ((size_t)bh * n + i) * D;
+    const TIn* kb = k + (size_t)bh * n * D;
+    const TIn* vb = v + (size_t)bh * n * DV;
+
+    for (int c = tid; c < D; c += HR_THREADS) qd[c] = (double)to_f32(qrow[c]);
+    __syncthreads();
+
+    // scores, their maximum, weights exp(s - m), ridge lambda * exp(-m)
+    double lmax = -INFINITY;
+    for (int j = tid; j < L; j += HR_THREADS) {
+        const TIn* kr = kb + (size_t)j * D;
+        double s = 0.0;
+        for (int c = 0; c < D; ++c) s += qd[c] * (double)to_f32(kr[c]);
+        s *= scale;
+        w[j] = s;
+        lmax = fmax(lmax, s);
+    }
+    const double m = block_reduce(lmax, true, red);
+    double lsum = 0.0;
+    for (int j = tid; j < L; j += HR_THREADS) {
+        const double e = exp(w[j] - m);
+        w[j] = e;
+        lsum += e;
+    }
+    const double omega = block_reduce(lsum, false, red);
+    const double lambda_m = lambda * exp(-m);
+
+    // moments: Sigma (lower 4x4 tiles in registers) and mu
+    double acc[C::TILES_PER_THREAD][4][4];
+    int tr[C::TILES_PER_THREAD], tc[C::TILES_PER_THREAD];
+#pragma unroll
+    for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
+        const int tile = tid + t * HR_THREADS;
+        // tile index -> (row tile, col tile) in the lower triangle
+        int r = 0;
+        if (tile < C::TILES) {
+            r = (int)((sqrt(8.0 * tile + 1.0) - 1.0) * 0.5);
+            while ((r + 1) * (r + 2) / 2 <= tile) ++r;
+            while (r * (r + 1) / 2 > tile) --r;
+        }
+        tr[t] = tile < C::TILES ? r : -1;
+        tc[t] = tile < C::TILES ? tile - r * (r + 1) / 2 : 0;
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[t][a][b] = 0.0;
+    }
+    double mu_acc = 0.0;  // thread tid < D owns mu[tid]
+    for (int j0 = 0; j0 < L; j0 += HR_CHUNK) {
+        const int jn = min(HR_CHUNK, L - j0);
+        __syncthreads();
+        for (int e = tid; e < jn * D; e += HR_THREADS) {
+            const int jj = e / D, c = e - jj * D;
+            zc[jj * D + c] = (double)to_f32(kb[(size_t)(j0 + jj) * D + c]) - qd[c];
+        }
+        __syncthreads();
+        if (tid < D)
+            for (int jj = 0; jj < jn; ++jj) mu_acc += w[j0 + jj] * zc[jj * D + tid];
+#pragma unroll
+        for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
+            if (tr[t] < 0) continue;
+            const int r0 = tr[t] * 4, c0 = tc[t] * 4;
+            for (int jj = 0; jj < jn; ++jj) {
+                const double wj = w[j0 + jj];
+                double zr[4], zcv[4];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    zr[a] = wj * zc[jj * D + r0 + a];
+                    zcv[a] = zc[jj * D + c0 + a];
+                }
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) acc[t][a][b] += zr[a] * zcv[b];
+            }
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
+        if (tr[t] < 0) continue;
+        const int r0 = tr[t] * 4, c0 = tc[t] * 4;
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int r = r0 + a, c = c0 + b;
+                if (c <= r) S[r * C::LDS + c] = acc[t][a][b] + (r == c ? lambda_m : 0.0);
+            }
+    }
+    if (tid < D) rhs[tid] = mu_acc;
+    __syncthreads();
+
+    // rhs <- Sigma^{-1} mu (LDL^T in shared memory)
+    const bool bad = !block_ldlt_solve(S, C::LDS, rhs, D);
+
+    // coefficients c_j = w_j (1 - z_j . rho) and their sum (= omega - mu . rho)
+    double csum = 0.0;
+    for (int j = tid; j < L; j += HR_THREADS) {
+        const TIn* kr = kb + (size_t)j * D;
+        double t = 0.0;
+        for (int c = 0; c < D; ++c) t += ((double)to_f32(kr[c]) - qd[c]) * rhs[c];
+        const double cj = w[j] * (1.0 - t);
+        w[j] = cj;
+        csum += cj;
+    }
+    const double denom = block_reduce(csum, false, red);
+    for (int c = tid; c < DV; c += HR_THREADS) {
+        double o = 0.0;
+        for (int j = 0; j < L; ++j) o += w[j] * (double)to_f32(vb[(size_t)j * DV + c]);
+        store_out(out + ((size_t)bh * n + i) * DV + c, (float)(o / denom));
+    }
+    const size_t row = (size_t)bh * n + i;
+    if (rho_out && tid < D) rho_out[row * D + tid] = (float)rhs[tid];
+    if (tid == 0) {
+        if (stats) {
+            stats[row * 3 + 0] = (float)m;
+            stats[row * 3 + 1] = (float)omega;
+            stats[row * 3 + 2] = (float)denom;
+        }
+        if (iters) iters[row] = -1;
+        if (bad && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
+    }
+}
+
+template <int D, typename TIn, typename TOut>
+int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
+    using C = HrCfg<D>;
+    const size_t smem = sizeof(double) *
+        ((size_t)D * C::LDS + 2 * D + lcap + (size_t)HR_CHUNK * D + HR_THREADS / 32 + 1);
+    auto kern = head_rows_kernel<D, D, TIn, TOut>;
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid(rows_per_head, a.B * a.H);
+    kern<<<grid, HR_THREADS, smem, a.stream>>>(
+        (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
+        (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status);
+    LLA_CUDA_TRY(cudaGetLastError());
+    return LLA_OK;
+}
+
+template <int D>
+int launch_d(const ForwardArgs& a, int rows_per_head, int lcap) {
+    if (a.in_dtype == LLA_BF16 && a.out_dtype == LLA_BF16)
+        return launch_t<D, __nv_bfloat16, __nv_bfloat16>(a, rows_per_head, lcap);
+    if (a.in_dtype == LLA_BF16 && a.out_dtype == LLA_F32)
+        return launch_t<D, __nv_bfloat16, float>(a, rows_per_head, lcap);
+    if (a.in_dtype == LLA_F32 && a.out_dtype == LLA_F32)
+        return launch_t<D, float, float>(a, rows_per_head, lcap);
+    return LLA_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+// Number of leading rows per head handled directly (causal), or n / 0 (non-causal).
+int head_rows_count(const ForwardArgs& a) {
+    if (a.head_rows <= 0) return 0;
+    if (a.causal) return a.n < a.head_rows - 1 ? a.n : a.head_rows - 1;
+    return a.n < a.head_rows ? a.n : 0;
+}
+
+int launch_head_rows(const ForwardArgs& a) {
+    const int rows = head_rows_count(a);
+    if (rows <= 0) return LLA_OK;
+    const int lcap = a.causal ? rows : a.n;
+    if (a.d != a.dv) return LLA_ERR_UNSUPPORTED;
+    switch (a.d) {
+        case 16: return launch_d<16>(a, rows, lcap);
+        case 64: return launch_d<64>(a, rows, lcap);
+        case 128: return launch_d<128>(a, rows, lcap);
+        default: return LLA_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace lla

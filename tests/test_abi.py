@@ -1,0 +1,90 @@
+"""Host-only checks of the C ABI: the library loads, exports every symbol the header declares, and
+rejects bad arguments before touching a device."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2510_01450_b200 import binding, build
+
+ROOT = Path(__file__).resolve().parents[1]
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def _declared_functions():
+    text = (ROOT / "include" / "lla.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lla_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_exports_match_header(lib):
+    declared = _declared_functions()
+    assert set(declared) == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_version_and_status_strings(lib):
+    assert binding.lla_version() >= 100
+    assert binding.status_string(0) == "ok"
+    for code in range(1, 6):
+        assert binding.status_string(code) not in ("ok", "unknown status")
+    assert binding.status_string(99) == "unknown status"
+
+
+def test_struct_sizes_match_c_layout():
+    # 4 pointers, 5+2 ints, 2 floats, 2 ints, 1 float, 2 ints, 4 pointers, pointer, size_t, pointer
+    assert ctypes.sizeof(binding.ForwardParams) == 4 * 8 + 15 * 4 + 4 + 7 * 8
+    assert ctypes.sizeof(binding.DecodeParams) == 5 * 8 + 11 * 4 + 4 + 4 * 8
+
+
+def test_argument_validation_without_device(lib):
+    ok_ptr = 0x1000
+    args = dict(B=1, H=1, n=8, d=64, dv=64, scale=0.125, lam=1e-3)
+
+    def fwd(**kw):
+        a = {**args, **kw}
+        q = kw.get("q", ok_ptr)
+        return lib.lla_forward(q, ok_ptr, ok_ptr, ok_ptr, a["B"], a["H"], a["n"], a["d"], a["dv"],
+                               a["scale"], a["lam"], 1, None)
+
+    assert fwd(q=None) == 1
+    assert fwd(n=0) == 1
+    assert fwd(lam=-1.0) == 1
+    assert fwd(scale=float("nan")) == 1
+    assert fwd(q=0x1004) == 1            # misaligned
+    assert fwd(d=32, dv=32) == 2
+    assert fwd(d=64, dv=16) == 2
+    assert lib.lla_decode(ok_ptr, ok_ptr, ok_ptr, None, ok_ptr, 1, 1, 8, 64, 64, 0.125, 1e-3, None) == 1
+    assert lib.lla_decode(ok_ptr, ok_ptr, ok_ptr, ok_ptr, ok_ptr, 1, 1, 0, 64, 64, 0.125, 1e-3, None) == 1
+    assert lib.lla_decode(ok_ptr, ok_ptr, ok_ptr, ok_ptr, ok_ptr, 1, 1, 8, 48, 48, 0.125, 1e-3, None) == 2
+    assert lib.lla_forward_ex(None) == 1
+    p = binding.DecodeParams()
+    p.q = p.kcache = p.vcache = p.lens = p.out = ok_ptr
+    p.B, p.H, p.Lmax, p.d, p.dv, p.scale, p.lambda_ = 1, 1, 4096, 64, 64, 0.125, 1e-3
+    p.splits = 4                          # explicit split without workspace
+    assert lib.lla_decode_ex(ctypes.byref(p)) == 3
+    with pytest.raises(binding.LlaError):
+        binding.lla_forward(None, ok_ptr, ok_ptr, ok_ptr, 1, 1, 8, 64, 64, 0.125, 1e-3)
+
+
+def test_workspace_and_split_arithmetic(lib):
+    assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == 0
+    assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=1) == 0
+    assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=3) == 4 * 2 * 4 * 3 * (2 * 64 * 64 + 130)
+    assert binding.lla_decode_default_splits(64, 16, 8192) == 1          # 1024 blocks already fill the chip
+    assert binding.lla_decode_default_splits(1, 16, 8192) == 16          # 512-key floor
+    assert binding.lla_decode_default_splits(1, 1, 100) == 1
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "liblla.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.load()

@@ -1,0 +1,237 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle on the
+same seeded inputs.
+
+Gate (written here, as the workloads state it): row-wise relative L2 error
+    E_row = max_i |o_i - oracle_i|_2 / |oracle_i|_2
+<= 1e-5 for the fp32 path and <= 2e-3 for bf16 inputs with fp32 accumulation.  For bf16 inputs the
+gate is taken on an fp32 output buffer: rounding the exact answer to bf16 alone costs up to 2^-9 =
+1.95e-3 per element, so the bf16-output result is additionally checked to be within one bf16 step
+(relative 2^-7 of the row's largest element) of the oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_01450_b200 import binding as L
+from paper_2510_01450_b200 import inputs
+from tests.gpu_util import LLA_DT, dev, forward, row_err, stream_ptr
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-5
+TOL_BF16 = 2e-3
+
+
+def _check_bf16_output(got_bf16, ref):
+    ref2 = ref.reshape(-1, ref.shape[-1])
+    got2 = got_bf16.reshape(-1, ref.shape[-1])
+    step = np.abs(ref2).max(axis=1, keepdims=True) * 2.0 ** -7
+    assert (np.abs(got2 - ref2) <= step).all()
+
+
+def test_config1_fp32_full(oracle):
+    w = inputs.CONFIGS[1]
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    dq, dk, dv_ = dev(q, "f32"), dev(k, "f32"), dev(v, "f32")
+    out = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.float32, device="cuda")
+    L.lla_forward_f32(dq, dk, dv_, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, 1, stream_ptr())
+    torch.cuda.synchronize()
+    err = row_err(out.cpu().numpy(), ref)
+    assert err.max() <= TOL_F32, err.max()
+
+
+@pytest.mark.parametrize("impl", [L.LLA_IMPL_SIMT, L.LLA_IMPL_AUTO])
+def test_config2_bf16_full(oracle, impl):
+    w = inputs.CONFIGS[2]
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    got = forward(w, q, k, v, out_dtype="f32", impl=impl, device_status=status)
+    err = row_err(got, ref)
+    assert err.max() <= TOL_BF16, err.max()
+    st = status.cpu().numpy()
+    assert st[L.STATUS_ROWS_AT_CAP] == 0 and st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
+    # the plain entry point (bf16 output)
+    dq, dk, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
+    out = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16, device="cuda")
+    L.lla_forward(dq, dk, dv_, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, 1, stream_ptr())
+    torch.cuda.synchronize()
+    _check_bf16_output(out.float().cpu().numpy().astype(np.float64), ref)
+
+
+def test_config3_regression_reduced_full_rows(oracle):
+    w = inputs.CONFIGS[3].shrink(B=1, H=2, n=1300)       # two segment boundaries, ragged tail
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    err = row_err(forward(w, q, k, v, out_dtype="f32"), ref)
+    assert err.max() <= TOL_BF16, err.max()
+
+
+def test_config3_full_size_sampled_rows(oracle):
+    w = inputs.CONFIGS[3]
+    q, k, v = inputs.make_prefill(w)
+    rows = inputs.sample_rows(w, per_head=96, heads=3, dense_below=4 * w.d)
+    ref = oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows)
+    got = forward(w, q, k, v, out_dtype="f32").reshape(-1, w.dv)[rows]
+    err = row_err(got, ref)
+    assert err.max() <= TOL_BF16, err.max()
+
+
+def test_config4_reduced_full_rows(oracle):
+    w = inputs.CONFIGS[4].shrink(H=2, n=1100)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    err = row_err(forward(w, q, k, v, out_dtype="f32"), ref)
+    assert err.max() <= TOL_BF16, err.max()
+
+
+def test_config4_full_size_sampled_rows(oracle):
+    w = inputs.CONFIGS[4]
+    q, k, v = inputs.make_prefill(w)
+    rows = inputs.sample_rows(w, per_head=48, heads=2, dense_below=2 * w.d + 16)
+    ref = oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows)
+    got = forward(w, q, k, v, out_dtype="f32").reshape(-1, w.dv)[rows]
+    err = row_err(got, ref)
+    assert err.max() <= TOL_BF16, err.max()
+
+
+def test_config5_decode_full(oracle):
+    w = inputs.CONFIGS[5]
+    q, kc, vc, lens = inputs.make_decode(w)
+    ref = oracle.decode(q, kc, vc, lens, w.scale, w.lam)
+    dq, dk, dv_ = dev(q, "bf16"), dev(kc, "bf16"), dev(vc, "bf16")
+    dl = torch.from_numpy(lens).cuda()
+    out32 = torch.empty((w.B, w.H, w.dv), dtype=torch.float32, device="cuda")
+    L.lla_decode_ex(dq, dk, dv_, dl, out32, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam,
+                    out_dtype=L.LLA_F32, stream=stream_ptr())
+    out16 = torch.empty((w.B, w.H, w.dv), dtype=torch.bfloat16, device="cuda")
+    L.lla_decode(dq, dk, dv_, dl, out16, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, stream_ptr())
+    torch.cuda.synchronize()
+    err = row_err(out32.cpu().numpy(), ref)
+    assert err.max() <= TOL_BF16, err.max()
+    _check_bf16_output(out16.float().cpu().numpy().astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 16), ("bf16", 16), ("bf16", 128), ("f32", 64)])
+def test_decode_matches_oracle_and_splits_agree(oracle, dtype, d):
+    w = inputs.CONFIGS[5].shrink(B=3, H=2, n=1500, d=d, dv=d, dtype=dtype, len_min=1, len_max=1500, seed=50 + d)
+    q, kc, vc, lens = inputs.make_decode(w)
+    lens[0], lens[1] = 1, 1500                 # one cached pair; a full cache
+    ref = oracle.decode(q, kc, vc, lens, w.scale, w.lam)
+    dq, dk, dv_ = dev(q, dtype), dev(kc, dtype), dev(vc, dtype)
+    dl = torch.from_numpy(lens).cuda()
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    for splits in (1, 3, 8):
+        nbytes = L.lla_decode_workspace_bytes(w.B, w.H, w.n, d, d, LLA_DT[dtype], splits)
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        out = torch.full((w.B, w.H, d), float("nan"), dtype=torch.float32, device="cuda")
+        L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, w.H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                        out_dtype=L.LLA_F32, splits=splits, workspace=ws, workspace_bytes=nbytes,
+                        stream=stream_ptr())
+        torch.cuda.synchronize()
+        err = row_err(out.cpu().numpy(), ref)
+        assert err.max() <= tol, (splits, err.max())
+    # decode of the last token equals the last prefill row on the same data
+    np.testing.assert_allclose(out.cpu().numpy()[0], vc[0, :, 0], rtol=1e-5, atol=1e-6)
+
+
+@pytest.mark.parametrize("n", [1, 2, 31, 127, 128, 129, 300])
+def test_ragged_and_tiny_lengths(oracle, n):
+    w = inputs.CONFIGS[2].shrink(B=2, H=1, n=n, seed=100 + n)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    err = row_err(forward(w, q, k, v, out_dtype="f32"), ref)
+    assert err.max() <= TOL_BF16, err.max()
+
+
+@pytest.mark.parametrize("dtype,d,n", [("f32", 16, 200), ("bf16", 16, 200), ("f32", 64, 400), ("f32", 128, 300)])
+def test_other_shapes_and_dtypes(oracle, dtype, d, n):
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=n, d=d, dv=d, dtype=dtype, seed=7 + d)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    err = row_err(forward(w, q, k, v, out_dtype="f32"), ref)
+    assert err.max() <= (TOL_F32 if dtype == "f32" else TOL_BF16), err.max()
+
+
+def test_noncausal(oracle):
+    for n in (40, 333):                                   # below and above the direct-solve threshold
+        w = inputs.CONFIGS[2].shrink(B=1, H=2, n=n, seed=11)
+        q, k, v = inputs.make_prefill(w)
+        ref = oracle.forward(q, k, v, w.scale, w.lam, causal=False)
+        err = row_err(forward(w, q, k, v, out_dtype="f32", causal=False), ref)
+        assert err.max() <= TOL_BF16, (n, err.max())
+
+
+def test_large_scores_and_ridge_rescale(oracle):
+    # scale 8x the usual: row maxima of several units, so the ridge lambda*exp(-m) matters
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=512, seed=12)
+    q, k, v = inputs.make_prefill(w)
+    scale = 8.0 * w.scale
+    ref = oracle.forward(q, k, v, scale, w.lam)
+    dq, dk, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
+    out = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.float32, device="cuda")
+    L.lla_forward_ex(dq, dk, dv_, out, w.B, w.H, w.n, w.d, w.dv, scale, w.lam, out_dtype=L.LLA_F32,
+                     max_iters=96, stream=stream_ptr())
+    torch.cuda.synchronize()
+    err = row_err(out.cpu().numpy(), ref)
+    assert err.max() <= TOL_BF16, err.max()
+
+
+def test_softmax_limit_on_device():
+    # lambda -> infinity: the output tends to softmax attention (Eq. "local_constant")
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=384, lam=1e7, seed=13)
+    q, k, v = inputs.make_prefill(w)
+    got = forward(w, q, k, v, out_dtype="f32")
+    tq, tk, tv = (torch.from_numpy(x).double() for x in (q, k, v))
+    s = (tq @ tk.transpose(-1, -2)) * w.scale
+    s = s.masked_fill(~torch.tril(torch.ones(w.n, w.n, dtype=torch.bool)), float("-inf"))
+    ref = (torch.softmax(s, dim=-1) @ tv).numpy()
+    assert row_err(got, ref).max() <= 1e-4
+
+
+def test_saved_tensors_match_oracle(oracle):
+    # rho and (m, omega, delta) as Algorithm 1 stores them for the backward pass
+    w = inputs.CONFIGS[2].shrink(B=1, H=1, n=400, seed=14)
+    q, k, v = inputs.make_prefill(w)
+    ref, rho_ref, aux_ref, _ = oracle.forward_rows(q, k, v, w.scale, w.lam, want_aux=True)
+    rho = torch.zeros((1, 1, w.n, w.d), dtype=torch.float32, device="cuda")
+    stats = torch.zeros((1, 1, w.n, 3), dtype=torch.float32, device="cuda")
+    iters = torch.zeros((1, 1, w.n), dtype=torch.int32, device="cuda")
+    got = forward(w, q, k, v, out_dtype="f32", rho=rho, stats=stats, iters=iters)
+    assert row_err(got, ref).max() <= TOL_BF16
+    assert row_err(rho.cpu().numpy(), rho_ref).max() <= 2e-3
+    np.testing.assert_allclose(stats.cpu().numpy().reshape(-1, 3), aux_ref, rtol=2e-3, atol=1e-6)
+    it = iters.cpu().numpy().ravel()
+    assert (it[:2 * w.d - 1] == -1).all() and (it[2 * w.d - 1:] > 0).all()
+
+
+def test_head_rows_disabled_still_converges_for_late_rows(oracle):
+    # with the direct path off, CG handles every row; late rows must still meet the gate
+    w = inputs.CONFIGS[2].shrink(B=1, H=1, n=512, seed=15)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    got = forward(w, q, k, v, out_dtype="f32", head_rows=-1, max_iters=64)
+    err = row_err(got, ref)
+    assert err[4 * w.d:].max() <= TOL_BF16
+
+
+def test_host_buffer_entry_points(oracle):
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=300, seed=16)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    hq, hk, hv = (torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in (q, k, v))
+    hout = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        L.lla_forward_host(hq, hk, hv, hout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_F32, w.scale, w.lam, 1,
+                           stream_ptr())
+        assert row_err(hout.numpy(), ref).max() <= TOL_BF16
+    wd = inputs.CONFIGS[5].shrink(B=3, H=2, n=700, len_min=5, len_max=700, seed=17)
+    dq, kc, vc, lens = inputs.make_decode(wd)
+    dref = oracle.decode(dq, kc, vc, lens, wd.scale, wd.lam)
+    hq, hk, hv = (torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in (dq, kc, vc))
+    hl = torch.from_numpy(lens)
+    hout = torch.empty((wd.B, wd.H, wd.dv), dtype=torch.float32).pin_memory()
+    L.lla_decode_host(hq, hk, hv, hl, hout, wd.B, wd.H, wd.n, wd.d, wd.dv, L.LLA_BF16, L.LLA_F32, wd.scale,
+                      wd.lam, stream_ptr())
+    assert row_err(hout.numpy(), dref).max() <= TOL_BF16
