@@ -144,8 +144,9 @@ def run_reference(args):
     for i in range(args.steps):
         lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=oracle_sample_rows(w, rows_per_step, 200 + i))
     dt = time.perf_counter() - t0
-    value = rows_per_step * args.steps / dt
-    sample = f"{rows_per_step} of {total_rows} rows per step, drawn uniformly over (batch, head, position)"
+    value = rows_per_step / w.H * args.steps / dt      # a token is one position with all H heads
+    sample = (f"{rows_per_step} of {total_rows} (head, position) rows per step, drawn uniformly over "
+              "(batch, head, position); tokens = rows / H")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
@@ -364,9 +365,9 @@ def cpu_baseline(w, q, k, v):
     t0 = time.perf_counter()
     lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows)
     dt = time.perf_counter() - t0
-    return {"value": rows.size / dt, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
+    return {"value": rows.size / w.H / dt, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
             "sample": f"{rows.size} of {total} rows of {w.name}, drawn uniformly over (batch, head, position); "
-                      f"{dt:.1f} s"}
+                      f"{dt:.1f} s; tokens = rows / H"}
 
 
 def main():
