@@ -131,11 +131,14 @@ int lla_decode_ex(const lla_decode_params* p) {
         if (!p->workspace || p->workspace_bytes < need) a.splits = 1;
     }
     if (a.splits > 1 && ((uintptr_t)p->workspace & 255u)) return LLA_ERR_WORKSPACE;
+    a.head_rows = 2 * p->d;
     a.status = p->device_status;
     a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
     a.stream = (cudaStream_t)p->stream;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
-    return lla::launch_decode(a);
+    const int st = lla::launch_decode(a);
+    if (st != LLA_OK) return st;
+    return lla::launch_head_rows_decode(a);
 }
 
 int lla_decode(const void* q, const void* kcache, const void* vcache, const int* lens, void* out, int B,

@@ -43,6 +43,7 @@ struct DecodeArgs {
     int in_dtype, out_dtype;
     float scale, lambda;
     int splits;
+    int head_rows;   // caches shorter than this are solved directly (fp64)
     int* status;
     void* workspace;
     size_t workspace_bytes;
@@ -56,6 +57,7 @@ int launch_forward_simt(const ForwardArgs& a);
 int launch_forward_tensor(const ForwardArgs& a);
 bool forward_tensor_supported(const ForwardArgs& a);
 int launch_decode(const DecodeArgs& a);
+int launch_head_rows_decode(const DecodeArgs& a);
 size_t decode_workspace_bytes(int B, int H, int d, int dv, int splits);
 
 // ---------------------------------------------------------------------------------------------

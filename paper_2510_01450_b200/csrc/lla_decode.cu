@@ -23,14 +23,14 @@ template <int D>
 struct DcCfg {
     static constexpr int T1 = D / 4;                                  // 4x4 tiles per side
     static constexpr int TPT = (T1 * T1 + DC_THREADS - 1) / DC_THREADS;  // tiles per thread per matrix
-    static constexpr int PART_FLOATS = 2 * D * D + 2 * D + 2;         // M, N, a, c, omega, m
+    static constexpr int PART_FLOATS = 2 * D * D + 2 * D + 4;         // M, N, a, c, omega, m, 2 pad (16-byte rows)
 };
 
 // Solve and emit one output row from moments held in shared memory (doubles).
-//   Md: M (becomes C), lower triangle used, row stride D+1;  Nd: N, row stride D
+//   Md: M (becomes C), lower triangle used, row stride D+1;  Nd: N as float, row stride D
 //   a, c: first moments; returns through out[dv]
 template <int D, typename TOut>
-__device__ void finalize_row(double* Md, const double* Nd, double* a, double* c, double omega, double m,
+__device__ void finalize_row(double* Md, const float* Nd, double* a, double* c, double omega, double m,
                              const double* qd, double lambda, TOut* out, int* status) {
     const int tid = threadIdx.x;
     constexpr int LDS = D + 1;
@@ -52,7 +52,7 @@ __device__ void finalize_row(double* Md, const double* Nd, double* a, double* c,
     const bool ok = block_ldlt_solve(Md, LDS, rhs, D);
     for (int e = tid; e < D; e += DC_THREADS) {   // dv == d
         double o = c[e];
-        for (int f = 0; f < D; ++f) o += (Nd[e * D + f] * inv - c[e] * a[f]) * rhs[f];
+        for (int f = 0; f < D; ++f) o += ((double)Nd[e * D + f] * inv - c[e] * a[f]) * rhs[f];
         store_out(out + e, (float)o);
     }
     if (!ok && tid == 0 && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
@@ -62,7 +62,7 @@ template <int D, typename TIn, typename TOut>
 __global__ void __launch_bounds__(DC_THREADS)
 decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache, const TIn* __restrict__ vcache,
                       const int* __restrict__ lens, TOut* __restrict__ out, int H, int Lmax, float scale,
-                      float lambda, int splits, float* __restrict__ parts, int* __restrict__ status) {
+                      float lambda, int splits, int head_rows, float* __restrict__ parts, int* __restrict__ status) {
     using C = DcCfg<D>;
     constexpr bool ACCURATE = sizeof(TIn) == 4;
     extern __shared__ double smem_d[];
@@ -77,6 +77,7 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     const int b = bh / H;
     int L = lens[b];
     L = max(1, min(L, Lmax));
+    if (L < head_rows) return;   // short caches are solved directly by the fp64 kernel
     const int chunk = ((L + splits - 1) / splits + DC_BK - 1) / DC_BK * DC_BK;
     const int jbeg = part * chunk, jend = min(L, jbeg + chunk);
     const TIn* kb = kcache + (size_t)bh * Lmax * D;
@@ -190,9 +191,9 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     for (int e = tid; e < D; e += DC_THREADS) qd_s[e] = (double)qs[e];
     __syncthreads();
     double* Md = smem_d;                 // D * (D+1)
-    double* Nd = Md + D * (D + 1);       // D * D
-    double* a = Nd + D * D;              // D
+    double* a = Md + D * (D + 1);        // D
     double* c = a + D;                   // D, followed by rhs (D)
+    float* Nd = reinterpret_cast<float*>(c + 2 * D);   // D * D
 #pragma unroll
     for (int t = 0; t < C::TPT; ++t) {
         const int tile = tid + t * DC_THREADS;
@@ -203,7 +204,7 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
 #pragma unroll
                 for (int y = 0; y < 4; ++y) {
                     Md[(r0 + x) * (D + 1) + c0 + y] = (double)accM[t][x][y];
-                    Nd[(r0 + x) * D + c0 + y] = (double)accN[t][x][y];
+                    Nd[(r0 + x) * D + c0 + y] = accN[t][x][y];
                 }
         }
     }
@@ -215,15 +216,17 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
 template <int D, typename TIn, typename TOut>
 __global__ void __launch_bounds__(DC_THREADS)
 decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts, TOut* __restrict__ out,
-                      float lambda, int splits, int* __restrict__ status) {
+                      const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
+                      int* __restrict__ status) {
     using C = DcCfg<D>;
     extern __shared__ double smem_d[];
     double* Md = smem_d;
-    double* Nd = Md + D * (D + 1);
-    double* a = Nd + D * D;
+    double* a = Md + D * (D + 1);
     double* c = a + D;
+    float* Nd = reinterpret_cast<float*>(c + 2 * D);
     __shared__ double qd_s[D];
     const int tid = threadIdx.x, bh = blockIdx.x;
+    if (max(1, min(lens[bh / H], Lmax)) < head_rows) return;
     const float* src = parts + (size_t)bh * splits * C::PART_FLOATS;
     for (int e = tid; e < D; e += DC_THREADS) qd_s[e] = (double)to_f32(q[(size_t)bh * D + e]);
     float m = -INFINITY;
@@ -239,7 +242,7 @@ decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts
             sn += f * (double)pp[D * D + e];
         }
         Md[r * (D + 1) + cc] = sm;
-        Nd[e] = sn;
+        Nd[e] = (float)sn;
     }
     for (int e = tid; e < 2 * D; e += DC_THREADS) {
         double s1 = 0.0;
@@ -259,7 +262,7 @@ decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts
 template <int D>
 constexpr size_t decode_smem_bytes() {
     const size_t stream = sizeof(float) * (2 * (size_t)DC_BK * D + DC_BK + D);
-    const size_t fin = sizeof(double) * ((size_t)D * (D + 1) + (size_t)D * D + 3 * D);
+    const size_t fin = sizeof(double) * ((size_t)D * (D + 1) + 3 * D) + sizeof(float) * (size_t)D * D;
     return stream > fin ? stream : fin;
 }
 
@@ -276,13 +279,13 @@ int launch_t(const DecodeArgs& a) {
     dim3 grid(splits, a.B * a.H);
     k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
                                              a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
-                                             (float*)a.workspace, a.status);
+                                             a.head_rows, (float*)a.workspace, a.status);
     LLA_CUDA_TRY(cudaGetLastError());
     if (splits > 1) {
         auto k2 = decode_combine_kernel<D, TIn, TOut>;
         LLA_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         k2<<<a.B * a.H, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const float*)a.workspace,
-                                                      (TOut*)a.out, a.lambda, splits, a.status);
+                                                      (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows, a.lambda, splits, a.status);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     return LLA_OK;
@@ -301,7 +304,7 @@ int launch_d(const DecodeArgs& a) {
 size_t decode_workspace_bytes(int B, int H, int d, int dv, int splits) {
     if (splits <= 1) return 0;
     (void)dv;
-    return sizeof(float) * (size_t)B * H * splits * (2 * (size_t)d * d + 2 * d + 2);
+    return sizeof(float) * (size_t)B * H * splits * (2 * (size_t)d * d + 2 * d + 4);
 }
 
 int launch_decode(const DecodeArgs& a) {

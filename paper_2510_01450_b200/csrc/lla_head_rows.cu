@@ -51,7 +51,10 @@ __global__ void __launch_bounds__(HR_THREADS)
 head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
                  TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
-                 int* __restrict__ iters, int* __restrict__ status) {
+                 int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H) {
+    // Prefill (lens == nullptr): block (i, bh) solves row i of head bh; n is the sequence length.
+    // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
+    // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
     using C = HrCfg<D>;
     extern __shared__ double smem[];
     double* S = smem;                       // D * LDS
@@ -65,8 +68,13 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     const int bh = blockIdx.y;
     const int i = blockIdx.x;               // row index inside the head
     if (i >= rows_per_head) return;
-    const int L = causal ? i + 1 : n;
-    const TIn* qrow = q + ((size_t)bh * n + i) * D;
+    int L = causal ? i + 1 : n;
+    if (lens) {
+        L = max(1, min(lens[bh / H], n));
+        if (L > lcap) return;               // long caches go through the moment kernel
+    }
+    const size_t row = lens ? (size_t)bh : (size_t)bh * n + i;
+    const TIn* qrow = q + row * D;
     const TIn* kb = k + (size_t)bh * n * D;
     const TIn* vb = v + (size_t)bh * n * DV;
 
@@ -175,9 +183,8 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     for (int c = tid; c < DV; c += HR_THREADS) {
         double o = 0.0;
         for (int j = 0; j < L; ++j) o += w[j] * (double)to_f32(vb[(size_t)j * DV + c]);
-        store_out(out + ((size_t)bh * n + i) * DV + c, (float)(o / denom));
+        store_out(out + row * DV + c, (float)(o / denom));
     }
-    const size_t row = (size_t)bh * n + i;
     if (rho_out && tid < D) rho_out[row * D + tid] = (float)rhs[tid];
     if (tid == 0) {
         if (stats) {
@@ -200,9 +207,35 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     dim3 grid(rows_per_head, a.B * a.H);
     kern<<<grid, HR_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
-        (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status);
+        (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
+}
+
+template <int D, typename TIn, typename TOut>
+int launch_decode_t(const DecodeArgs& a, int lcap) {
+    using C = HrCfg<D>;
+    const size_t smem = sizeof(double) *
+        ((size_t)D * C::LDS + 2 * D + lcap + (size_t)HR_CHUNK * D + HR_THREADS / 32 + 1);
+    auto kern = head_rows_kernel<D, D, TIn, TOut>;
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid(1, a.B * a.H);
+    kern<<<grid, HR_THREADS, smem, a.stream>>>(
+        (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
+        (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H);
+    LLA_CUDA_TRY(cudaGetLastError());
+    return LLA_OK;
+}
+
+template <int D>
+int launch_decode_d(const DecodeArgs& a, int lcap) {
+    if (a.in_dtype == LLA_BF16 && a.out_dtype == LLA_BF16)
+        return launch_decode_t<D, __nv_bfloat16, __nv_bfloat16>(a, lcap);
+    if (a.in_dtype == LLA_BF16 && a.out_dtype == LLA_F32)
+        return launch_decode_t<D, __nv_bfloat16, float>(a, lcap);
+    if (a.in_dtype == LLA_F32 && a.out_dtype == LLA_F32)
+        return launch_decode_t<D, float, float>(a, lcap);
+    return LLA_ERR_UNSUPPORTED;
 }
 
 template <int D>
@@ -234,6 +267,18 @@ int launch_head_rows(const ForwardArgs& a) {
         case 16: return launch_d<16>(a, rows, lcap);
         case 64: return launch_d<64>(a, rows, lcap);
         case 128: return launch_d<128>(a, rows, lcap);
+        default: return LLA_ERR_UNSUPPORTED;
+    }
+}
+
+// Decode: (sequence, head) pairs whose cache holds at most head_rows - 1 keys.
+int launch_head_rows_decode(const DecodeArgs& a) {
+    if (a.head_rows <= 1) return LLA_OK;
+    const int lcap = a.head_rows - 1;
+    switch (a.d) {
+        case 16: return launch_decode_d<16>(a, lcap);
+        case 64: return launch_decode_d<64>(a, lcap);
+        case 128: return launch_decode_d<128>(a, lcap);
         default: return LLA_ERR_UNSUPPORTED;
     }
 }
