@@ -186,6 +186,37 @@ int lla_decode_host(const void *q, const void *kcache, const void *vcache, const
                     void *out, int B, int H, int Lmax, int d, int dv, int in_dtype, int out_dtype,
                     float scale, float lambda, void *stream);
 
+/*
+ * Decode for callers that must not allocate.  (The paper has no counterpart; this is a packaging
+ * variant of the split-key decode, same arithmetic as lla_decode_ex with `splits` parts.)
+ *
+ * Who needs it: code that runs where the CUDA allocator is off limits - inside a serving loop
+ * whose memory is fully pre-planned, under a framework that forbids cudaMalloc after start-up
+ * (a synchronising allocation would stall every stream of the process), or in a plug-in that is
+ * handed device buffers but owns no allocator.  Such callers cannot provide the partial-moment
+ * workspace that a split decode needs, and the library may not allocate it for them either.
+ *
+ * Instead the partial moments go to a fixed array of LLA_NOALLOC_SCRATCH_BYTES that is part of the
+ * library image: every GPU that loads the library holds those bytes until the library is unloaded.
+ * The call performs no cudaMalloc, cudaFree or other allocating call.  Its first use on a device
+ * looks up the array's device address (with that device current); make that first call outside
+ * any stream capture.
+ *
+ * Arguments are those of lla_decode plus the dtypes and `splits` (0 = the default of
+ * lla_decode_default_splits; 1 = no split, which uses no scratch at all).  All tensor pointers are
+ * device pointers owned by the caller.
+ * Errors: LLA_ERR_WORKSPACE if B*H*splits partial records do not fit in the fixed array
+ * (lla_decode_workspace_bytes(...) > LLA_NOALLOC_SCRATCH_BYTES): use fewer splits or lla_decode_ex
+ * with a caller workspace.  Other codes as for lla_decode_ex.
+ * Sharing: all calls on a device use the same array.  Each call overwrites every record it later
+ * reads, so nothing needs clearing between calls, but two calls whose kernels may run at the same
+ * time (different streams, or different host threads) race on it: serialise them.
+ */
+#define LLA_NOALLOC_SCRATCH_BYTES (32u << 20)
+int lla_decode_noalloc(const void *q, const void *kcache, const void *vcache, const int *lens,
+                       void *out, int B, int H, int Lmax, int d, int dv, int in_dtype,
+                       int out_dtype, float scale, float lambda, int splits, void *stream);
+
 /* Scratch bytes lla_forward_ex needs for this problem (0 when none). Host-only arithmetic. */
 size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl);
 

@@ -22,7 +22,7 @@ STATUS_ROWS_AT_CAP, STATUS_BAD_PIVOT, STATUS_TIMEOUT, STATUS_ITER_SUM = 0, 1, 2,
 
 EXPORTS = (
     "lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex", "lla_decode_ex",
-    "lla_forward_host", "lla_decode_host", "lla_forward_workspace_bytes", "lla_decode_workspace_bytes",
+    "lla_forward_host", "lla_decode_host", "lla_decode_noalloc", "lla_forward_workspace_bytes", "lla_decode_workspace_bytes",
     "lla_decode_default_splits", "lla_status_string", "lla_version",
 )
 
@@ -78,10 +78,12 @@ def load():
     lib.lla_decode_f32.argtypes = dec
     lib.lla_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, f, f, i, vp]
     lib.lla_decode_host.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, f, vp]
+    lib.lla_decode_noalloc.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, f, i, vp]
+    lib.lla_decode_noalloc.restype = i
     lib.lla_forward_ex.argtypes = [ctypes.POINTER(ForwardParams)]
     lib.lla_decode_ex.argtypes = [ctypes.POINTER(DecodeParams)]
     for name in ("lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex",
-                 "lla_decode_ex", "lla_forward_host", "lla_decode_host", "lla_version",
+                 "lla_decode_ex", "lla_forward_host", "lla_decode_host", "lla_decode_noalloc", "lla_version",
                  "lla_decode_default_splits"):
         getattr(lib, name).restype = i
     lib.lla_decode_default_splits.argtypes = [i, i, i]
@@ -172,6 +174,19 @@ def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, i
     p.scale, p.lambda_, p.splits, p.impl = scale, lam, splits, impl
     p.device_status, p.workspace, p.workspace_bytes, p.stream = _p(device_status), _p(workspace), workspace_bytes, _p(stream)
     _check(load().lla_decode_ex(ctypes.byref(p)), "lla_decode_ex")
+
+
+NOALLOC_SCRATCH_BYTES = 32 << 20
+
+
+def lla_decode_noalloc(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, in_dtype=LLA_BF16,
+                       out_dtype=LLA_BF16, splits=0, stream=0):
+    """Split-key decode for callers that may not allocate device memory (a pre-planned serving loop,
+    a host framework that forbids cudaMalloc after start-up): the partial moments live in a fixed
+    32 MiB array inside the library instead of a workspace.  Raises LlaError(status 3) when
+    B*H*splits records do not fit.  Calls that may overlap on the GPU race on that array."""
+    _check(load().lla_decode_noalloc(_p(q), _p(kcache), _p(vcache), _p(lens), _p(out), B, H, Lmax, d, dv,
+                                     in_dtype, out_dtype, scale, lam, splits, _p(stream)), "lla_decode_noalloc")
 
 
 def lla_forward_workspace_bytes(B, H, n, d, dv, in_dtype=LLA_BF16, impl=LLA_IMPL_AUTO) -> int:

@@ -317,4 +317,66 @@ int launch_decode(const DecodeArgs& a) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Decode without any allocation: the split-key decode above, with the partial-moment records kept
+// in a fixed device array that is part of the library image.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch shared by every lla_decode_noalloc call on a device.  It lives in each device's copy of
+// the module for as long as the library stays loaded.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[LLA_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+// The array's name is only a host-side handle in host code; kernels need its device address.
+int noalloc_scratch_ptr(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LLA_ERR_CUDA;
+    void* p = __atomic_load_n(&g_noalloc_ptr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return LLA_ERR_CUDA;
+        __atomic_store_n(&g_noalloc_ptr[dev], p, __ATOMIC_RELEASE);   // same value from any thread
+    }
+    *out = p;
+    return LLA_OK;
+}
+
+}  // namespace
 }  // namespace lla
+
+extern "C" int lla_decode_noalloc(const void* q, const void* kcache, const void* vcache, const int* lens,
+                                  void* out, int B, int H, int Lmax, int d, int dv, int in_dtype, int out_dtype,
+                                  float scale, float lambda, int splits, void* stream) {
+    if (!q || !kcache || !vcache || !lens || !out) return LLA_ERR_INVALID_ARG;
+    if (B < 1 || H < 1 || Lmax < 1 || d < 1 || dv < 1 || splits < 0) return LLA_ERR_INVALID_ARG;
+    if (!(lambda >= 0.f) || !isfinite(lambda) || !isfinite(scale)) return LLA_ERR_INVALID_ARG;
+    if (((uintptr_t)q | (uintptr_t)kcache | (uintptr_t)vcache | (uintptr_t)out) & 15u) return LLA_ERR_INVALID_ARG;
+    if (d != dv || !(d == 16 || d == 64 || d == 128) || (long long)B * H > 65535) return LLA_ERR_UNSUPPORTED;
+    const bool dt_ok = (in_dtype == LLA_BF16 && (out_dtype == LLA_BF16 || out_dtype == LLA_F32)) ||
+                       (in_dtype == LLA_F32 && out_dtype == LLA_F32);
+    if (!dt_ok) return LLA_ERR_UNSUPPORTED;
+    lla::DecodeArgs a;
+    a.q = q; a.kcache = kcache; a.vcache = vcache; a.lens = lens; a.out = out;
+    a.B = B; a.H = H; a.Lmax = Lmax; a.d = d; a.dv = dv;
+    a.in_dtype = in_dtype; a.out_dtype = out_dtype;
+    a.scale = scale; a.lambda = lambda;
+    a.splits = splits > 0 ? splits : lla_decode_default_splits(B, H, Lmax);
+    a.head_rows = 2 * d;
+    a.status = nullptr;
+    a.workspace = nullptr; a.workspace_bytes = 0;
+    a.stream = (cudaStream_t)stream;
+    if (a.splits > 1) {
+        const size_t need = lla::decode_workspace_bytes(B, H, d, dv, a.splits);
+        if (need > (size_t)LLA_NOALLOC_SCRATCH_BYTES) return LLA_ERR_WORKSPACE;   // beyond the fixed array
+        void* scratch = nullptr;
+        const int rc = lla::noalloc_scratch_ptr(&scratch);
+        if (rc != LLA_OK) return rc;
+        a.workspace = scratch;
+        a.workspace_bytes = LLA_NOALLOC_SCRATCH_BYTES;
+    }
+    const int st = lla::launch_decode(a);
+    if (st != LLA_OK) return st;
+    return lla::launch_head_rows_decode(a);
+}
