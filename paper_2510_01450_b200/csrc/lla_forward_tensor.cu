@@ -1,7 +1,697 @@
-// Placeholder translation unit for the tcgen05 forward kernel (filled in by the tensor-core path).
+// LLA forward on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 inputs, d = dv = 64.
+//
+// One thread block per (batch*head, 128-row query tile).  The three loops of Algorithm 1 and the
+// per-iteration loop of Algorithm 2 are all "sweeps" over 64-key blocks with the same skeleton:
+//
+//   TMA            K block (and V block in the last sweep) -> 128B-swizzled shared memory
+//   MMA 1 (SS)     S = Q K^T                     [128 x 64] fp32 in TMEM
+//                  A = P_hi K^T + P_lo K^T       [128 x 64] fp32 in TMEM   (CG and output sweeps)
+//   CUDA cores     one thread pair per query row reads S, A from TMEM, forms
+//                      max sweep     running row maximum m_i
+//                      stats sweep   w = exp(s - m),                 omega += w
+//                      CG sweep      u = w (a - kbar.p)              (Algorithm 2's W .* (P K^T))
+//                      output sweep  c = w (1 - (a - kbar.y)),       den += c
+//                  splits the result into bf16 hi + lo and stores both back into the TMEM columns S
+//                  came from (two 16-bit values per column)
+//   MMA 2 (TS)     ACC += U_hi B + U_lo B, A operand straight from TMEM, B = the same K block read
+//                  MN-major (or the V block in the output sweep)
+//
+// S/A/U are double buffered in TMEM (2 x 128 columns) and ACC takes 64 more; K/V blocks go through a
+// 4-stage ring.  Roles: warps 0-7 compute (warp w owns TMEM lanes 32*(w%4).. and key half w/4 of each
+// block; two threads share a row and exchange partial sums through shared memory), warp 8 issues TMA,
+// warp 9 issues MMAs.  Every on-the-fly MMA operand (P, y, U) is carried as a bf16 pair hi + lo so
+// the products keep ~16 mantissa bits: a single bf16 rounding of those operands would leave a
+// 2e-3..5e-3 error in the output, above the 2e-3 gate.  Q, K, V are exact bf16 inputs.
+//
+// The mathematics is the centred form described in lla_forward_simt.cu (same CG, same freeze rule).
+// All waits on mbarriers are bounded; a wait that expires sets LLA_STATUS_TIMEOUT and the block
+// leaves through the common exit (TMEM is released there).
+#include <cuda.h>
+
 #include "lla_common.cuh"
 
 namespace lla {
-bool forward_tensor_supported(const ForwardArgs&) { return false; }
-int launch_forward_tensor(const ForwardArgs&) { return LLA_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int TC_D = 64;             // head size handled here
+constexpr int TC_BR = 128;           // query rows per block (TMEM lanes)
+constexpr int TC_BC = 64;            // keys per block
+constexpr int TC_NST = 4;            // K/V ring stages
+constexpr int TC_COMPUTE = 256;      // compute threads (warps 0..7)
+constexpr int TC_THREADS = 320;      // + TMA warp + MMA warp
+constexpr int TC_TMEM_COLS = 512;
+constexpr int TC_ACC_COL = 256;      // ACC columns [256, 320)
+
+enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4 };
+
+// shared-memory carve-up (bytes, from a 1024-byte aligned base)
+constexpr int SM_Q = 0;                                  // 128 x 64 bf16, swizzled            16384
+constexpr int SM_PHI = SM_Q + 16384;                     // P / y hi                            16384
+constexpr int SM_PLO = SM_PHI + 16384;                   // P / y lo                            16384
+constexpr int SM_KV = SM_PLO + 16384;                    // TC_NST x (K 8192 + V 8192)          65536
+constexpr int SM_X = SM_KV + TC_NST * 16384;             // x   fp32 [64][128]                  32768
+constexpr int SM_KBAR = SM_X + 32768;                    // kbar fp32 [64][128]                 32768
+constexpr int SM_RED = SM_KBAR + 32768;                  // pair reduction buffers 2 x 2 x 128   2048
+constexpr int SM_FLAGS = SM_RED + 2048;                  // 2 x 8 ints                             64
+constexpr int SM_BAR = SM_FLAGS + 64;                    // mbarriers (8 bytes each)              256
+constexpr int SM_MISC = SM_BAR + 256;                    // tmem base, ctl kind, abort              64
+constexpr int SM_TOTAL = SM_MISC + 64;
+constexpr int SM_ALLOC = SM_TOTAL + 1024;                // slack for manual 1024-byte alignment
+
+// mbarrier indices
+enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST, B_SAFULL = B_KVEMPTY + TC_NST,
+       B_UFULL = B_SAFULL + 2, B_BUFFREE = B_UFULL + 2, B_ACCFULL = B_BUFFREE + 2, B_CTL = B_ACCFULL + 1,
+       B_COUNT = B_CTL + 1 };
+static_assert(B_COUNT * 8 <= 256, "barrier area too small");
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2^31 clock ticks or as soon as another thread flagged an abort.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > (1ll << 31)) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void named_sync_compute() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+
+// 32 consecutive TMEM columns of this thread's lane -> registers (and back)
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// {hi16: bf16(a), lo16: bf16(b)}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(a), "f"(b));
+    return r;
+}
+
+// Shared-memory matrix descriptors (128-byte swizzle, tile base 1024-byte aligned).
+//   K-major:  rows of 128 bytes, 8-row groups 1024 bytes apart; a 16-element K step is +32 bytes.
+//   MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements; 8-row groups
+//             1024 bytes apart; a 16-element K step is +2048 bytes.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);         // start address
+    d |= (uint64_t)1 << 16;                              // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset
+    d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
+    return d;
+}
+
+constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+constexpr uint32_t IDESC_SS = make_idesc(TC_BR, TC_BC, 0, 0);   // S/A: A, B K-major
+constexpr uint32_t IDESC_TS = make_idesc(TC_BR, TC_D, 0, 1);    // ACC: A from TMEM, B MN-major
+
+// byte offset of the 16-byte chunk `chunk` (8 bf16) of row `row` in a swizzled 128 x 64 bf16 tile
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+struct TcParams {
+    int n, causal, head_rows, max_iters, first_tile;
+    float scale, lambda, tol;
+    float* rho;
+    float* stats;
+    int* iters;
+    int* status;
+};
+
+template <typename TOut>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, TOut* __restrict__ out, const TcParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + SM_BAR;
+    auto bar = [&](int i) { return bars + 8u * i; };
+    volatile int* misc = reinterpret_cast<volatile int*>(smem + SM_MISC);   // [0] tmem base, [1] kind, [2] abort
+    volatile int* abort_flag = misc + 2;
+    float* xs = reinterpret_cast<float*>(smem + SM_X);
+    float* kbs = reinterpret_cast<float*>(smem + SM_KBAR);
+    float* red = reinterpret_cast<float*>(smem + SM_RED);
+    volatile int* flags = reinterpret_cast<volatile int*>(smem + SM_FLAGS);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.y;
+    const int tile = prm.first_tile + (gridDim.x - 1 - blockIdx.x);      // heaviest tiles first
+    const int r0 = tile * TC_BR;
+    const int n = prm.n;
+    const int nblk_all = (n + TC_BC - 1) / TC_BC;
+    const int nblk = prm.causal ? min(nblk_all, (r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
+
+    if (tid == 0) {
+        mbar_init(bar(B_QFULL), 1);
+        for (int s = 0; s < TC_NST; ++s) { mbar_init(bar(B_KVFULL + s), 1); mbar_init(bar(B_KVEMPTY + s), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(B_SAFULL + b), 1);
+            mbar_init(bar(B_UFULL + b), TC_COMPUTE);
+            mbar_init(bar(B_BUFFREE + b), 1);
+        }
+        mbar_init(bar(B_ACCFULL), 1);
+        mbar_init(bar(B_CTL), TC_COMPUTE);
+        misc[1] = SW_MAX;
+        misc[2] = 0;
+        fence_barrier_init();
+    }
+    if (warp == 8) {   // TMEM allocation by one full warp; the base address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(sbase + SM_MISC), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)misc[0];
+
+    if (warp == 8) {
+        // ================================ TMA producer ================================
+        if (lane == 0) {
+            mbar_expect_tx(bar(B_QFULL), TC_BR * TC_D * 2);
+            tma_load_3d(sbase + SM_Q, &tmQ, bar(B_QFULL), 0, r0, bh);
+            uint32_t it = 0;
+            for (uint32_t sweep = 0;; ++sweep) {
+                if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+                const int kind = misc[1];
+                if (kind == SW_DONE) break;
+                bool ok = true;
+                for (int c = 0; c < nblk; ++c, ++it) {
+                    const uint32_t s = it % TC_NST, use = it / TC_NST;
+                    if (!mbar_wait(bar(B_KVEMPTY + s), (use & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = sbase + SM_KV + s * 16384;
+                    mbar_expect_tx(bar(B_KVFULL + s), kind == SW_OUT ? 16384 : 8192);
+                    tma_load_3d(dst, &tmK, bar(B_KVFULL + s), 0, c * TC_BC, bh);
+                    if (kind == SW_OUT) tma_load_3d(dst + 8192, &tmV, bar(B_KVFULL + s), 0, c * TC_BC, bh);
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp == 9) {
+        // ================================ MMA issuer ================================
+        if (lane == 0) {
+            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
+            const uint64_t qdesc = make_desc(sbase + SM_Q);
+            const uint64_t phdesc = make_desc(sbase + SM_PHI);
+            const uint64_t pldesc = make_desc(sbase + SM_PLO);
+            uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it & 1)
+            for (uint32_t sweep = 0; ok; ++sweep) {
+                if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+                const int kind = misc[1];
+                if (kind == SW_DONE) break;
+                tc_fence_after();
+                const uint32_t it0 = it;
+                for (int c = 0; c <= nblk && ok; ++c) {
+                    if (c < nblk) {
+                        const uint32_t g = it0 + c, s = g % TC_NST, b = g & 1;
+                        if (!mbar_wait(bar(B_KVFULL + s), (g / TC_NST) & 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(bar(B_BUFFREE + b), ((g >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t kdesc = make_desc(sbase + SM_KV + s * 16384);
+                        const uint32_t s_tm = tmem + b * 128, a_tm = s_tm + 64;
+#pragma unroll
+                        for (int ks = 0; ks < TC_D / 16; ++ks)
+                            mma_ss(s_tm, qdesc + 2 * ks, kdesc + 2 * ks, IDESC_SS, ks > 0);
+                        if (kind == SW_CG || kind == SW_OUT) {
+#pragma unroll
+                            for (int ks = 0; ks < TC_D / 16; ++ks)
+                                mma_ss(a_tm, phdesc + 2 * ks, kdesc + 2 * ks, IDESC_SS, ks > 0);
+#pragma unroll
+                            for (int ks = 0; ks < TC_D / 16; ++ks)
+                                mma_ss(a_tm, pldesc + 2 * ks, kdesc + 2 * ks, IDESC_SS, 1);
+                        }
+                        tc_commit(bar(B_SAFULL + b));
+                    }
+                    if (c >= 1) {
+                        const uint32_t g = it0 + c - 1, s = g % TC_NST, b = g & 1;
+                        if (!mbar_wait(bar(B_UFULL + b), (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        if (kind != SW_MAX) {
+                            const uint32_t bsm = sbase + SM_KV + s * 16384 + (kind == SW_OUT ? 8192 : 0);
+                            const uint64_t bdesc = make_desc(bsm);
+                            const uint32_t u_tm = tmem + b * 128;
+#pragma unroll
+                            for (int ks = 0; ks < TC_BC / 16; ++ks) {
+                                // 16 keys = two 8-row groups = 2048 bytes = 128 descriptor units
+                                mma_ts(tmem + TC_ACC_COL, u_tm + 16 * ks, bdesc + 128 * ks, IDESC_TS, (c > 1 || ks > 0));
+                                mma_ts(tmem + TC_ACC_COL, u_tm + 16 * ks + 8, bdesc + 128 * ks, IDESC_TS, 1);
+                            }
+                            tc_commit(bar(B_KVEMPTY + s));
+                            tc_commit(bar(B_BUFFREE + b));
+                            if (c == nblk) tc_commit(bar(B_ACCFULL));
+                        } else {
+                            mbar_arrive(bar(B_KVEMPTY + s));
+                            mbar_arrive(bar(B_BUFFREE + b));
+                        }
+                    }
+                }
+                it = it0 + nblk;
+            }
+        }
+    } else {
+        // ================================ compute warps ================================
+        const int quad = warp & 3, half = warp >> 2;
+        const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
+        const int row = r0 + lrow;
+        const int L = prm.causal ? row + 1 : n;
+        const bool row_ok = row < n && L >= prm.head_rows;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const int c0 = half * 32;                          // first column / first key (inside a block) owned
+        int red_sel = 0;
+        auto pair_sum = [&](float v) {
+            float* buf = red + red_sel * 256;
+            red_sel ^= 1;
+            buf[half * 128 + lrow] = v;
+            named_sync_compute();
+            return buf[lrow] + buf[128 + lrow];
+        };
+        auto pair_max = [&](float v) {
+            float* buf = red + red_sel * 256;
+            red_sel ^= 1;
+            buf[half * 128 + lrow] = v;
+            named_sync_compute();
+            return fmaxf(buf[lrow], buf[128 + lrow]);
+        };
+        int flag_sel = 0;
+        auto group_any = [&](bool v) {
+            volatile int* f = flags + flag_sel * 8;
+            flag_sel ^= 1;
+            const int any = __any_sync(0xffffffffu, v);
+            if (lane == 0) f[warp] = any;
+            named_sync_compute();
+            int r = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) r |= f[i];
+            return r != 0;
+        };
+        // store 32 fp32 values of this row as bf16 hi/lo into the swizzled operand tiles
+        auto write_operand = [&](const float* vec) {
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float a = vec[ch * 8 + 2 * e], b = vec[ch * 8 + 2 * e + 1];
+                    hi[e] = pack_bf16(b, a);
+                    const float ra = a - __uint_as_float(hi[e] << 16), rb = b - __uint_as_float(hi[e] & 0xFFFF0000u);
+                    lo[e] = pack_bf16(rb, ra);
+                }
+                const uint32_t off = swz(lrow, half * 4 + ch);
+                *reinterpret_cast<uint4*>(smem + SM_PHI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(smem + SM_PLO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+        };
+
+        const float c1 = prm.scale * 1.4426950408889634f;    // scores in log2 units
+        float mx2 = -INFINITY, omega = 0.f, inv_omega = 0.f, ridge = 0.f, den = 0.f;
+        float abar = 0.f;                                     // kbar.p (CG) or kbar.y (output)
+        uint32_t blk = 0;                                     // global block counter (buffer = blk & 1)
+        bool ok = true;
+
+        // One sweep over the key blocks.  kind is uniform over the block.
+        auto sweep = [&](int kind) {
+            float part = 0.f;                                 // omega / den partial, or max
+            if (kind == SW_MAX) part = -INFINITY;
+            for (int c = 0; c < nblk; ++c, ++blk) {
+                const uint32_t b = blk & 1;
+                if (!mbar_wait(bar(B_SAFULL + b), (blk >> 1) & 1, abort_flag)) { ok = false; return part; }
+                tc_fence_after();
+                const uint32_t s_addr = tmem + lane_addr + b * 128 + c0;
+                uint32_t sv[32], av[32];
+                tmem_ld32(s_addr, sv);
+                if (kind == SW_CG || kind == SW_OUT) tmem_ld32(s_addr + 64, av);
+                tc_wait_ld();
+                const int j0 = c * TC_BC + c0;                // first key of this thread's 32
+                const int jlim = min(L, n) - j0;              // keys e < jlim are visible
+                if (kind == SW_MAX) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (e < jlim) part = fmaxf(part, __uint_as_float(sv[e]) * c1);
+                } else {
+                    float u[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        float w = ex2f(fmaf(__uint_as_float(sv[e]), c1, -mx2));
+                        if (kind == SW_CG) w *= (__uint_as_float(av[e]) - abar);
+                        if (kind == SW_OUT) w *= (1.f - (__uint_as_float(av[e]) - abar));
+                        u[e] = e < jlim ? w : 0.f;
+                    }
+                    if (kind != SW_CG) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) part += u[e];
+                    }
+                    // two k-steps of 16 keys; per k-step 8 columns of hi then 8 columns of lo
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float a = u[ks * 16 + 2 * e], bq = u[ks * 16 + 2 * e + 1];
+                            const uint32_t hi = pack_bf16(bq, a);
+                            const float ra = a - __uint_as_float(hi << 16), rb = bq - __uint_as_float(hi & 0xFFFF0000u);
+                            pk[ks * 16 + e] = hi;
+                            pk[ks * 16 + 8 + e] = pack_bf16(rb, ra);
+                        }
+                    tmem_st32(s_addr, pk);
+                    tc_wait_st();
+                }
+                tc_fence_before();
+                mbar_arrive(bar(B_UFULL + b));
+            }
+            return part;
+        };
+        // read this thread's 32 ACC columns after the sweep's last MMA
+        uint32_t acc_uses = 0;
+        auto read_acc = [&](float* dst) {
+            if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag)) { ok = false; return; }
+            ++acc_uses;
+            tc_fence_after();
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_addr + TC_ACC_COL + c0, v);
+            tc_wait_ld();
+            tc_fence_before();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) dst[e] = __uint_as_float(v[e]);
+        };
+        auto start_sweep = [&](int kind) {
+            if (tid == 0) misc[1] = kind;
+            fence_proxy_async();       // operand tiles written with ordinary stores -> visible to the MMA
+            mbar_arrive(bar(B_CTL));
+        };
+
+        float r[32], p[32];
+        float rr = 0.f, stop = 0.f;
+        int its = 0;
+        bool active = false;
+
+        // ---- sweep 0: row maxima ----
+        start_sweep(SW_MAX);
+        {
+            const float part = sweep(SW_MAX);
+            if (ok) mx2 = pair_max(part);
+        }
+        // ---- sweep 1: omega and kbar ----
+        if (ok) {
+            start_sweep(SW_STATS);
+            const float part = sweep(SW_STATS);
+            float acc[32];
+            if (ok) read_acc(acc);
+            if (ok) {
+                omega = pair_sum(part);
+                inv_omega = 1.f / omega;
+                ridge = prm.lambda * ex2f(-mx2) * inv_omega;
+                float rr_p = 0.f, ab_p = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    const uint4 qraw = *reinterpret_cast<const uint4*>(smem + SM_Q + swz(lrow, half * 4 + ch));
+                    const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float qv = (e & 1) ? __uint_as_float(qw[e >> 1] & 0xFFFF0000u) : __uint_as_float(qw[e >> 1] << 16);
+                        const int col = ch * 8 + e;
+                        const float kb = acc[col] * inv_omega;
+                        kbs[(c0 + col) * TC_BR + lrow] = kb;
+                        xs[(c0 + col) * TC_BR + lrow] = 0.f;
+                        const float bv = row_ok ? kb - qv : 0.f;
+                        r[col] = bv;
+                        p[col] = bv;
+                        rr_p += bv * bv;
+                        ab_p += kb * bv;
+                    }
+                }
+                rr = pair_sum(rr_p);
+                abar = pair_sum(ab_p);
+                stop = prm.tol * prm.tol * rr;
+                active = row_ok && rr > 0.f;
+                write_operand(p);
+            }
+        }
+        // ---- conjugate gradients (Algorithm 2) ----
+        for (int t = 0; ok && t < prm.max_iters; ++t) {
+            active = active && rr > stop;
+            if (!group_any(active)) break;
+            start_sweep(SW_CG);
+            sweep(SW_CG);
+            float ap[32];
+            if (ok) read_acc(ap);
+            if (!ok) break;
+            float pap_p = 0.f;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                ap[e] = fmaf(ap[e], inv_omega, ridge * p[e]);
+                pap_p += p[e] * ap[e];
+            }
+            const float pap = pair_sum(pap_p);
+            if (active && !(pap > 0.f)) active = false;
+            const float alpha = active ? rr / pap : 0.f;
+            float rr2_p = 0.f;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                xs[(c0 + e) * TC_BR + lrow] += alpha * p[e];
+                r[e] -= alpha * ap[e];
+                rr2_p += r[e] * r[e];
+            }
+            const float rr2 = pair_sum(rr2_p);
+            float ab_p = 0.f;
+            if (active) {
+                const float beta = rr2 / rr;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) p[e] = fmaf(beta, p[e], r[e]);
+                rr = rr2;
+                ++its;
+            }
+#pragma unroll
+            for (int e = 0; e < 32; ++e) ab_p += kbs[(c0 + e) * TC_BR + lrow] * p[e];
+            abar = pair_sum(ab_p);
+            write_operand(p);
+        }
+        const bool at_cap = active && rr > stop;
+        // ---- output sweep ----
+        float gfac = 1.f;
+        if (ok) {
+            float y[32];
+            float yb_p = 0.f, g_p = 0.f;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                const uint4 qraw = *reinterpret_cast<const uint4*>(smem + SM_Q + swz(lrow, half * 4 + ch));
+                const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float qv = (e & 1) ? __uint_as_float(qw[e >> 1] & 0xFFFF0000u) : __uint_as_float(qw[e >> 1] << 16);
+                    const int col = ch * 8 + e;
+                    const float kb = kbs[(c0 + col) * TC_BR + lrow];
+                    y[col] = xs[(c0 + col) * TC_BR + lrow];
+                    yb_p += kb * y[col];
+                    g_p += (kb - qv) * y[col];
+                }
+            }
+            abar = pair_sum(yb_p);
+            gfac = 1.f + pair_sum(g_p);
+            write_operand(y);
+            start_sweep(SW_OUT);
+            const float part = sweep(SW_OUT);
+            float o[32];
+            if (ok) read_acc(o);
+            if (ok) {
+                den = pair_sum(part);
+                if (row_ok) {
+                    const float inv_den = 1.f / den;
+                    const size_t rowi = (size_t)bh * n + row;
+                    TOut* orow = out + rowi * TC_D + c0;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) store_out(orow + e, o[e] * inv_den);
+                    if (prm.rho) {
+                        const float ig = 1.f / gfac;
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) prm.rho[rowi * TC_D + c0 + e] = y[e] * ig;
+                    }
+                    if (half == 0) {
+                        if (prm.stats) {
+                            prm.stats[rowi * 3 + 0] = mx2 * 0.6931471805599453f;
+                            prm.stats[rowi * 3 + 1] = omega;
+                            prm.stats[rowi * 3 + 2] = omega / gfac;
+                        }
+                        if (prm.iters) prm.iters[rowi] = its;
+                        if (prm.status) {
+                            if (at_cap) atomicAdd(prm.status + LLA_STATUS_ROWS_AT_CAP, 1);
+                            atomicAdd(prm.status + LLA_STATUS_ITER_SUM, its);
+                        }
+                    }
+                }
+            }
+        }
+        if (ok) start_sweep(SW_DONE);
+    }
+
+    // ================================ common exit ================================
+    if (*abort_flag) {
+        // let copies that are still in flight land before the block's shared memory goes away
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && *abort_flag && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [BH, n, 64] bf16 tensor viewed as 3-D, box = 64 columns x box_rows rows x 1
+bool make_map(CUtensorMap* map, const void* base, int BH, int n, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)TC_D, (cuuint64_t)n, (cuuint64_t)BH};
+    const cuuint64_t strides[2] = {(cuuint64_t)TC_D * 2, (cuuint64_t)n * TC_D * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)TC_D, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename TOut>
+int launch_t(const ForwardArgs& a) {
+    const int hr = head_rows_count(a);
+    if (!a.causal && hr >= a.n) return LLA_OK;
+    const int first_tile = a.causal ? hr / TC_BR : 0;
+    const int tiles = (a.n + TC_BR - 1) / TC_BR - first_tile;
+    if (tiles <= 0) return LLA_OK;
+    CUtensorMap mq, mk, mv;
+    const int BH = a.B * a.H;
+    if (!make_map(&mq, a.q, BH, a.n, TC_BR) || !make_map(&mk, a.k, BH, a.n, TC_BC) ||
+        !make_map(&mv, a.v, BH, a.n, TC_BC))
+        return LLA_ERR_CUDA;
+    TcParams prm;
+    prm.n = a.n; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
+    prm.max_iters = a.max_iters; prm.first_tile = first_tile;
+    prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
+    prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
+    auto kern = forward_tc_kernel<TOut>;
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
+    dim3 grid(tiles, BH);
+    kern<<<grid, TC_THREADS, SM_ALLOC, a.stream>>>(mq, mk, mv, (TOut*)a.out, prm);
+    LLA_CUDA_TRY(cudaGetLastError());
+    return LLA_OK;
+}
+
+}  // namespace
+
+bool forward_tensor_supported(const ForwardArgs& a) {
+    return a.in_dtype == LLA_BF16 && a.d == TC_D && a.dv == TC_D && get_encode() != nullptr;
+}
+
+int launch_forward_tensor(const ForwardArgs& a) {
+    if (!forward_tensor_supported(a)) return LLA_ERR_UNSUPPORTED;
+    if (a.out_dtype == LLA_BF16) return launch_t<__nv_bfloat16>(a);
+    if (a.out_dtype == LLA_F32) return launch_t<float>(a);
+    return LLA_ERR_UNSUPPORTED;
+}
+
 }  // namespace lla
