@@ -102,11 +102,12 @@ int lla_decode_f32(const void *q, const void *kcache, const void *vcache, const 
 /*
  * Full-control forward.  Zero-initialise the struct, then set fields; zero / NULL means default.
  *   in_dtype / out_dtype : lla_dtype of q,k,v and of out (bf16 inputs may write an fp32 output)
- *   max_iters : CG iteration cap per row (default 48; Algorithm 2's T)
+ *   max_iters : CG iteration cap per row (default 64; Algorithm 2's T)
  *   tol       : CG stops a row when |residual| <= tol * |right-hand side| (Algorithm 2's
  *               epsilon; default 1e-4 for bf16 inputs, 1e-6 for fp32 inputs)
  *   head_rows : rows that see fewer than this many keys are solved directly in fp64 from the
- *               explicit d x d system instead of by CG (0 = default 2*d; negative disables).  Those early systems are too ill-conditioned for fp32 CG.
+ *               explicit d x d system instead of by CG (0 = default: 1.5*d for bf16 inputs, 2*d for
+ *               fp32 inputs; negative disables).  Those early systems are too ill-conditioned for fp32 CG.
  *   impl      : lla_impl
  *   phases    : which groups of rows to compute: 0 = all; LLA_PHASE_DIRECT = only the rows
  *               solved directly; LLA_PHASE_ITERATIVE = only the rows solved by CG (profiling aid:

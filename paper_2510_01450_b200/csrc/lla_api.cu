@@ -1,12 +1,37 @@
 // C-ABI entry points: argument validation, defaults, dispatch.  See include/lla.h for the contract.
 #include <math.h>
 
+#include <mutex>
+
 #include "lla_common.cuh"
 
 namespace {
 
 using lla::DecodeArgs;
 using lla::ForwardArgs;
+
+// Side stream on which the directly-solved rows run next to the iterative kernel (fork/join with
+// events, so the caller's stream semantics are unchanged).  One per device, created on first use.
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool ok = false;
+};
+SideStream* side_stream() {
+    static std::mutex mu;
+    static SideStream per_dev[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    SideStream& s = per_dev[dev];
+    if (!s.ok) {
+        if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        s.ok = true;
+    }
+    return &s;
+}
 
 bool head_size_ok(int d, int dv) { return d == dv && (d == 16 || d == 64 || d == 128); }
 
@@ -16,7 +41,7 @@ int check_forward(const lla_forward_params* p) {
     if (p->B < 1 || p->H < 1 || p->n < 1 || p->d < 1 || p->dv < 1) return LLA_ERR_INVALID_ARG;
     if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
     if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
-    if ((long long)p->B * p->H > 65535) return LLA_ERR_UNSUPPORTED;
+    if ((long long)p->B * p->H > 65535 || (p->n + 127) / 128 > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
     const bool dt_ok = (p->in_dtype == LLA_BF16 && (p->out_dtype == LLA_BF16 || p->out_dtype == LLA_F32)) ||
                        (p->in_dtype == LLA_F32 && p->out_dtype == LLA_F32);
@@ -35,9 +60,10 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.B = p->B; a.H = p->H; a.n = p->n; a.d = p->d; a.dv = p->dv;
     a.in_dtype = p->in_dtype; a.out_dtype = p->out_dtype;
     a.scale = p->scale; a.lambda = p->lambda; a.causal = p->causal ? 1 : 0;
-    a.max_iters = p->max_iters > 0 ? p->max_iters : 48;
+    a.max_iters = p->max_iters > 0 ? p->max_iters : 64;
     a.tol = p->tol > 0.f ? p->tol : (p->in_dtype == LLA_F32 ? 1e-6f : 1e-4f);
-    a.head_rows = p->head_rows == 0 ? 2 * p->d : (p->head_rows < 0 ? 0 : p->head_rows);
+    a.head_rows = p->head_rows == 0 ? (p->in_dtype == LLA_F32 ? 2 * p->d : p->d + p->d / 2)
+                                   : (p->head_rows < 0 ? 0 : p->head_rows);
     a.rho = p->rho; a.stats = p->stats; a.iters = p->iters; a.status = p->device_status;
     a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
     a.stream = (cudaStream_t)p->stream;
@@ -75,6 +101,21 @@ int lla_forward_ex(const lla_forward_params* p) {
     if (need > 0 && (!a.workspace || a.workspace_bytes < need || ((uintptr_t)a.workspace & 255u)))
         return LLA_ERR_WORKSPACE;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
+    // The two row groups write disjoint rows of `out`; when both run, the direct rows go to a side
+    // stream so they fill the SMs the iterative kernel's last wave leaves idle.
+    const bool both = p->phases == LLA_PHASE_ALL && lla::head_rows_count(a) > 0;
+    SideStream* side = both ? side_stream() : nullptr;
+    if (side) {
+        LLA_CUDA_TRY(cudaEventRecord(side->fork, a.stream));
+        LLA_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+        const int rc_main = use_tensor ? lla::launch_forward_tensor(a) : lla::launch_forward_simt(a);
+        ForwardArgs h = a;
+        h.stream = side->stream;
+        const int rc_head = lla::launch_head_rows(h);
+        LLA_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+        LLA_CUDA_TRY(cudaStreamWaitEvent(a.stream, side->join, 0));
+        return rc_main != LLA_OK ? rc_main : rc_head;
+    }
     if (p->phases != LLA_PHASE_ITERATIVE) {
         const int st = lla::launch_head_rows(a);
         if (st != LLA_OK) return st;

@@ -103,43 +103,84 @@ __device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __fl
 
 // ---------------------------------------------------------------------------------------------
 // Dense symmetric positive-definite solve in shared memory, double precision, by a whole block.
-//   S   : d x d, row stride lds doubles, lower triangle filled; destroyed (LDL^T in place)
-//   rhs : d doubles; replaced by the solution
-// Returns false if a pivot was not positive.  Every thread of the block must call it.
+//   S   : D x D, row stride lds doubles, lower triangle filled; destroyed (LDL^T in place)
+//   rhs : D doubles; replaced by the solution
+// Returns false if a pivot was not positive.  Every thread of the block must call it; blockDim.x
+// must be a multiple of 32 with at least two warps.
+//
+// The right-hand side rides along as an extra matrix row, so the forward substitution happens
+// inside the elimination; the backward substitution is a column sweep by warp 0 with the partial
+// sums of each unknown held in registers.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs, int d) {
+__device__ __forceinline__ double fast_rcp(double x) {
+    double r;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+    r = r * (2.0 - x * r);
+    r = r * (2.0 - x * r);
+    return r;
+}
+
+template <int D>
+__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs) {
     const int tid = threadIdx.x, nt = blockDim.x;
+    const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
     bool ok = true;
     __syncthreads();
-    // after step c, column c holds L[r][c] * D_c (left unscaled), diagonal holds D_c
-    for (int c = 0; c < d - 1; ++c) {
+    // After step c, column c holds L[r][c] * D_c (left unscaled) and the diagonal holds D_c.
+    // Warp ny-1 also carries the right-hand side as row D.
+    for (int c = 0; c < D - 1; ++c) {
         const double piv = S[c * lds + c];
         if (!(piv > 0.0)) ok = false;
-        const double inv = 1.0 / piv;
-        const int rem = d - 1 - c;
-        for (int e = tid; e < rem * rem; e += nt) {
-            const int rr = e / rem, cc = e - rr * rem;
-            if (cc <= rr) {
-                const int r = c + 1 + rr, c2 = c + 1 + cc;
-                S[r * lds + c2] -= S[r * lds + c] * S[c2 * lds + c] * inv;
+        const double inv = fast_rcp(piv);
+        for (int rb = c + 1 + ty; rb < D; rb += 4 * ny) {
+            // four rows of this warp at a time for instruction-level parallelism
+            double l[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int r = rb + u * ny;
+                l[u] = r < D ? S[r * lds + c] * inv : 0.0;
             }
+            const int rmax = min(D - 1, rb + 3 * ny);
+            for (int c2 = c + 1 + tx; c2 <= rmax; c2 += 32) {
+                const double sc = S[c2 * lds + c];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int r = rb + u * ny;
+                    if (r < D && c2 <= r) S[r * lds + c2] -= l[u] * sc;
+                }
+            }
+        }
+        if (ty == ny - 1) {
+            const double lr = rhs[c] * inv;
+            for (int c2 = c + 1 + tx; c2 < D; c2 += 32) rhs[c2] -= lr * S[c2 * lds + c];
         }
         __syncthreads();
     }
-    if (!(S[(d - 1) * lds + (d - 1)] > 0.0)) ok = false;
+    if (!(S[(D - 1) * lds + (D - 1)] > 0.0)) ok = false;
+    // rhs now holds y with L y = b.  Backward: x_r = (y_r - sum_{t>r} S[t][r] x_t) / D_r.
     if (tid < 32) {
-        const int lane = tid;
-        for (int r = 0; r < d; ++r) {   // forward with the unit lower factor L[t][r] = S[t][r] / S[r][r]
-            const double yr = rhs[r] / S[r * lds + r];
-            for (int t = r + 1 + lane; t < d; t += 32) rhs[t] -= S[t * lds + r] * yr;
-            __syncwarp();
+        constexpr int PER = (D + 31) / 32;
+        double part[PER], dinv[PER], yv[PER];
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            const int t = tx + 32 * u;
+            part[u] = 0.0;
+            dinv[u] = t < D ? fast_rcp(S[t * lds + t]) : 0.0;
+            yv[u] = t < D ? rhs[t] : 0.0;
         }
-        for (int r = lane; r < d; r += 32) rhs[r] /= S[r * lds + r];
-        __syncwarp();
-        for (int r = d - 1; r > 0; --r) {   // backward with L^T
-            const double xr = rhs[r];
-            for (int t = lane; t < r; t += 32) rhs[t] -= S[r * lds + t] / S[t * lds + t] * xr;
-            __syncwarp();
+        for (int r = D - 1; r >= 0; --r) {
+            const int owner = r & 31, slot = r >> 5;
+            double xr = 0.0;
+#pragma unroll
+            for (int u = 0; u < PER; ++u)
+                if (u == slot) xr = (yv[u] - part[u]) * dinv[u];
+            xr = __shfl_sync(0xffffffffu, xr, owner);
+            if (tx == owner) rhs[r] = xr;
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int t = tx + 32 * u;
+                if (t < r) part[u] += S[r * lds + t] * xr;
+            }
         }
     }
     __syncthreads();

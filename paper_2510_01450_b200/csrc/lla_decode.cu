@@ -49,7 +49,7 @@ __device__ void finalize_row(double* Md, const float* Nd, double* a, double* c, 
         c[e] *= inv;
         rhs[e] = qd[e] - a[e];
     }
-    const bool ok = block_ldlt_solve(Md, LDS, rhs, D);
+    const bool ok = block_ldlt_solve<D>(Md, LDS, rhs);
     for (int e = tid; e < D; e += DC_THREADS) {   // dv == d
         double o = c[e];
         for (int f = 0; f < D; ++f) o += ((double)Nd[e * D + f] * inv - c[e] * a[f]) * rhs[f];

@@ -219,8 +219,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     volatile int* flags = reinterpret_cast<volatile int*>(smem + SM_FLAGS);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.y;
-    const int tile = prm.first_tile + (gridDim.x - 1 - blockIdx.x);      // heaviest tiles first
+    // blockIdx.x runs fastest in launch order: all heads of the heaviest (last) query tile come first
+    const int bh = blockIdx.x;
+    const int tile = prm.first_tile + (gridDim.y - 1 - blockIdx.y);
     const int r0 = tile * TC_BR;
     const int n = prm.n;
     const int nblk_all = (n + TC_BC - 1) / TC_BC;
@@ -675,7 +676,7 @@ int launch_t(const ForwardArgs& a) {
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     auto kern = forward_tc_kernel<TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
-    dim3 grid(tiles, BH);
+    dim3 grid(BH, tiles);
     kern<<<grid, TC_THREADS, SM_ALLOC, a.stream>>>(mq, mk, mv, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;

@@ -46,8 +46,32 @@ __device__ __forceinline__ double block_reduce(double x, bool is_max, double* sc
     return scratch[HR_THREADS / 32];
 }
 
+// dot product of a double vector in shared memory with one row of keys (vector loads, 8 at a time)
+template <int D>
+__device__ __forceinline__ double dot_row(const double* __restrict__ a, const __nv_bfloat16* __restrict__ kr) {
+    double s = 0.0;
+#pragma unroll 1
+    for (int c = 0; c < D; c += 8) {
+        float f[8];
+        load8(kr + c, f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s += a[c + e] * (double)f[e];
+    }
+    return s;
+}
+template <int D>
+__device__ __forceinline__ double dot_row(const double* __restrict__ a, const float* __restrict__ kr) {
+    double s = 0.0;
+#pragma unroll 1
+    for (int c = 0; c < D; c += 4) {
+        const float4 f = load4(kr + c);
+        s += a[c] * (double)f.x + a[c + 1] * (double)f.y + a[c + 2] * (double)f.z + a[c + 3] * (double)f.w;
+    }
+    return s;
+}
+
 template <int D, int DV, typename TIn, typename TOut>
-__global__ void __launch_bounds__(HR_THREADS)
+__global__ void __launch_bounds__(HR_THREADS, (D <= 64 ? 4 : 1))
 head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
                  TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
@@ -84,10 +108,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     // scores, their maximum, weights exp(s - m), ridge lambda * exp(-m)
     double lmax = -INFINITY;
     for (int j = tid; j < L; j += HR_THREADS) {
-        const TIn* kr = kb + (size_t)j * D;
-        double s = 0.0;
-        for (int c = 0; c < D; ++c) s += qd[c] * (double)to_f32(kr[c]);
-        s *= scale;
+        const double s = dot_row<D>(qd, kb + (size_t)j * D) * scale;
         w[j] = s;
         lmax = fmax(lmax, s);
     }
@@ -135,14 +156,16 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
 #pragma unroll
         for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
             if (tr[t] < 0) continue;
-            const int r0 = tr[t] * 4, c0 = tc[t] * 4;
+            // interleaved 4x4 tile: rows tr + T1*a, columns tc + T1*b, so that neighbouring threads
+            // read neighbouring doubles (no shared-memory bank conflicts)
+            const int r0 = tr[t], c0 = tc[t];
             for (int jj = 0; jj < jn; ++jj) {
                 const double wj = w[j0 + jj];
                 double zr[4], zcv[4];
 #pragma unroll
                 for (int a = 0; a < 4; ++a) {
-                    zr[a] = wj * zc[jj * D + r0 + a];
-                    zcv[a] = zc[jj * D + c0 + a];
+                    zr[a] = wj * zc[jj * D + r0 + C::TILES_1D * a];
+                    zcv[a] = zc[jj * D + c0 + C::TILES_1D * a];
                 }
 #pragma unroll
                 for (int a = 0; a < 4; ++a)
@@ -154,27 +177,27 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
 #pragma unroll
     for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
         if (tr[t] < 0) continue;
-        const int r0 = tr[t] * 4, c0 = tc[t] * 4;
 #pragma unroll
         for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-                const int r = r0 + a, c = c0 + b;
+                const int r = tr[t] + C::TILES_1D * a, c = tc[t] + C::TILES_1D * b;
                 if (c <= r) S[r * C::LDS + c] = acc[t][a][b] + (r == c ? lambda_m : 0.0);
+                else if (tr[t] != tc[t]) S[c * C::LDS + r] = acc[t][a][b];   // mirror of tile (tc, tr)
             }
     }
     if (tid < D) rhs[tid] = mu_acc;
     __syncthreads();
 
     // rhs <- Sigma^{-1} mu (LDL^T in shared memory)
-    const bool bad = !block_ldlt_solve(S, C::LDS, rhs, D);
+    const bool bad = !block_ldlt_solve<D>(S, C::LDS, rhs);
 
     // coefficients c_j = w_j (1 - z_j . rho) and their sum (= omega - mu . rho)
+    double qrho = 0.0;
+    for (int c = 0; c < D; ++c) qrho += qd[c] * rhs[c];
     double csum = 0.0;
     for (int j = tid; j < L; j += HR_THREADS) {
-        const TIn* kr = kb + (size_t)j * D;
-        double t = 0.0;
-        for (int c = 0; c < D; ++c) t += ((double)to_f32(kr[c]) - qd[c]) * rhs[c];
+        const double t = dot_row<D>(rhs, kb + (size_t)j * D) - qrho;
         const double cj = w[j] * (1.0 - t);
         w[j] = cj;
         csum += cj;

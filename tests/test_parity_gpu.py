@@ -203,7 +203,8 @@ def test_saved_tensors_match_oracle(oracle):
     assert row_err(rho.cpu().numpy(), rho_ref).max() <= 2e-3
     np.testing.assert_allclose(stats.cpu().numpy().reshape(-1, 3), aux_ref, rtol=2e-3, atol=1e-6)
     it = iters.cpu().numpy().ravel()
-    assert (it[:2 * w.d - 1] == -1).all() and (it[2 * w.d - 1:] > 0).all()
+    direct = w.d + w.d // 2 - 1            # bf16 inputs: rows seeing fewer than 1.5 d keys are solved directly
+    assert (it[:direct] == -1).all() and (it[direct:] > 0).all()
 
 
 def test_head_rows_disabled_still_converges_for_late_rows(oracle):
