@@ -59,7 +59,8 @@ constexpr int SM_TOTAL = SM_MISC + 64;
 constexpr int SM_ALLOC = SM_TOTAL + 1024;                // slack for manual 1024-byte alignment
 
 // mbarrier indices
-enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST, B_SAFULL = B_KVEMPTY + TC_NST,
+enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST, B_VFULL = B_KVEMPTY + TC_NST,
+       B_SAFULL = B_VFULL + TC_NST,
        B_UFULL = B_SAFULL + 2, B_BUFFREE = B_UFULL + 2, B_ACCFULL = B_BUFFREE + 2, B_CTL = B_ACCFULL + 1,
        B_COUNT = B_CTL + 1 };
 static_assert(B_COUNT * 8 <= 256, "barrier area too small");
@@ -107,9 +108,6 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void named_sync_compute() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
@@ -118,19 +116,54 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
 }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+// MMA issue.  The whole MMA warp runs these convergently and the instructions are predicated on the
+// elected lane (el != 0): issuing from a divergent single-thread branch instead costs ~100 clocks
+// per instruction (operands have to be moved into uniform registers one by one), three times the
+// execution time of a 128x64x16 MMA.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P1;\n\telect.sync _|P1, 0xffffffff;\n\tselp.u32 %0, 1, 0, P1;\n\t}" : "=r"(pred));
+    return pred;
 }
-// D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+// D[tmem] (+)= A[smem] * B[smem] over 64 elements of K (4 instructions, both operands K-major:
+// +32 bytes = 2 descriptor units per step).  acc0 = 0 overwrites D with the first product.
+__device__ __forceinline__ void mma_ss_k64(uint32_t el, uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u64 a1, %2, 2; add.u64 a2, %2, 4; add.u64 a3, %2, 6;\n\t"
+        "add.u64 b1, %3, 2; add.u64 b2, %3, 4; add.u64 b3, %3, 6;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// D[tmem] (+)= (U_hi + U_lo)[tmem] * B[smem] over 64 keys: per 16-key step the hi operand sits at
+// a + 16*step and the lo operand 8 columns further; B is MN-major (+2048 bytes = 128 units per step).
+__device__ __forceinline__ void mma_ts_hilo_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a0l, a1, a1l, a2, a2l, a3, a3l;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a0l, %2, 8; add.u32 a1, %2, 16; add.u32 a1l, %2, 24; add.u32 a2, %2, 32;\n\t"
+        "add.u32 a2l, %2, 40; add.u32 a3, %2, 48; add.u32 a3l, %2, 56;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a0l], %3, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1l], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2l], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3l], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+__device__ __forceinline__ void tc_commit_el(uint32_t el, uint32_t bar) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %0, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
+                 ::"r"(el), "r"(bar) : "memory");
 }
 
 // 32 consecutive TMEM columns of this thread's lane -> registers (and back)
@@ -162,6 +195,13 @@ __device__ __forceinline__ float ex2f(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// two fp32 lanes in one 64-bit register (sm_100 packed fp32 arithmetic)
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 // {hi16: bf16(a), lo16: bf16(b)}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     uint32_t r;
@@ -193,7 +233,17 @@ constexpr uint32_t IDESC_TS = make_idesc(TC_BR, TC_D, 0, 1);    // ACC: A from T
 // byte offset of the 16-byte chunk `chunk` (8 bf16) of row `row` in a swizzled 128 x 64 bf16 tile
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
+// Optional phase timing for tuning (compile with -DLLA_TC_TIMING; totals are added to prm.dbg).
+#ifdef LLA_TC_TIMING
+#define TC_T0(var) const long long var = clock64()
+#define TC_ACC(slot, var) do { if (prm.dbg) atomicAdd(prm.dbg + (slot), (unsigned long long)(clock64() - (var))); } while (0)
+#else
+#define TC_T0(var)
+#define TC_ACC(slot, var)
+#endif
+
 struct TcParams {
+    unsigned long long* dbg;
     int n, causal, head_rows, max_iters, first_tile;
     float scale, lambda, tol;
     float* rho;
@@ -229,10 +279,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
-        for (int s = 0; s < TC_NST; ++s) { mbar_init(bar(B_KVFULL + s), 1); mbar_init(bar(B_KVEMPTY + s), 1); }
+        for (int s = 0; s < TC_NST; ++s) {
+            mbar_init(bar(B_KVFULL + s), 1);
+            mbar_init(bar(B_KVEMPTY + s), 1);
+            mbar_init(bar(B_VFULL + s), 1);
+        }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(B_SAFULL + b), 1);
-            mbar_init(bar(B_UFULL + b), TC_COMPUTE);
+            mbar_init(bar(B_UFULL + b), TC_COMPUTE / 2);
             mbar_init(bar(B_BUFFREE + b), 1);
         }
         mbar_init(bar(B_ACCFULL), 1);
@@ -253,89 +307,111 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     if (warp == 8) {
         // ================================ TMA producer ================================
+        // K blocks stream through the ring continuously: once a sweep's blocks are issued the first
+        // blocks of the next sweep are prefetched without waiting to learn what kind of sweep it is
+        // (every kind needs K).  V blocks are added, on their own barriers, once the output sweep
+        // is announced.
         if (lane == 0) {
             mbar_expect_tx(bar(B_QFULL), TC_BR * TC_D * 2);
             tma_load_3d(sbase + SM_Q, &tmQ, bar(B_QFULL), 0, r0, bh);
-            uint32_t it = 0;
-            for (uint32_t sweep = 0;; ++sweep) {
+            uint32_t kit = 0;      // K blocks issued so far
+            int pre = 0;           // blocks of the coming sweep already issued
+            bool ok = true;
+            auto issue_k = [&](int c) {
+                const uint32_t s = kit % TC_NST;
+                if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                mbar_expect_tx(bar(B_KVFULL + s), 8192);
+                tma_load_3d(sbase + SM_KV + s * 16384, &tmK, bar(B_KVFULL + s), 0, c * TC_BC, bh);
+                ++kit;
+            };
+            auto issue_v = [&](int c, uint32_t g) {
+                const uint32_t s = g % TC_NST;
+                mbar_expect_tx(bar(B_VFULL + s), 8192);
+                tma_load_3d(sbase + SM_KV + s * 16384 + 8192, &tmV, bar(B_VFULL + s), 0, c * TC_BC, bh);
+            };
+            for (uint32_t sweep = 0; ok; ++sweep) {
                 if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
                 const int kind = misc[1];
-                if (kind == SW_DONE) break;
-                bool ok = true;
-                for (int c = 0; c < nblk; ++c, ++it) {
-                    const uint32_t s = it % TC_NST, use = it / TC_NST;
-                    if (!mbar_wait(bar(B_KVEMPTY + s), (use & 1) ^ 1, abort_flag)) { ok = false; break; }
-                    const uint32_t dst = sbase + SM_KV + s * 16384;
-                    mbar_expect_tx(bar(B_KVFULL + s), kind == SW_OUT ? 16384 : 8192);
-                    tma_load_3d(dst, &tmK, bar(B_KVFULL + s), 0, c * TC_BC, bh);
-                    if (kind == SW_OUT) tma_load_3d(dst + 8192, &tmV, bar(B_KVFULL + s), 0, c * TC_BC, bh);
+                if (kind == SW_DONE) {
+                    // prefetched blocks nobody will consume: wait until they have landed
+                    for (int i = 0; i < pre; ++i) {
+                        const uint32_t g = kit - pre + i;
+                        if (!mbar_wait(bar(B_KVFULL + g % TC_NST), (g / TC_NST) & 1, abort_flag)) break;
+                    }
+                    break;
                 }
-                if (!ok) break;
+                const uint32_t g0 = kit - pre;
+                if (kind == SW_OUT)
+                    for (int c = 0; c < pre; ++c) issue_v(c, g0 + c);
+                for (int c = pre; c < nblk && ok; ++c) {
+                    issue_k(c);
+                    if (ok && kind == SW_OUT) issue_v(c, g0 + c);
+                }
+                pre = 0;
+                if (kind != SW_OUT)
+                    for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c); ++pre; }
             }
         }
     } else if (warp == 9) {
         // ================================ MMA issuer ================================
-        if (lane == 0) {
-            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
-            const uint64_t qdesc = make_desc(sbase + SM_Q);
-            const uint64_t phdesc = make_desc(sbase + SM_PHI);
-            const uint64_t pldesc = make_desc(sbase + SM_PLO);
-            uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it & 1)
-            for (uint32_t sweep = 0; ok; ++sweep) {
-                if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
-                const int kind = misc[1];
-                if (kind == SW_DONE) break;
-                tc_fence_after();
-                const uint32_t it0 = it;
-                for (int c = 0; c <= nblk && ok; ++c) {
-                    if (c < nblk) {
-                        const uint32_t g = it0 + c, s = g % TC_NST, b = g & 1;
-                        if (!mbar_wait(bar(B_KVFULL + s), (g / TC_NST) & 1, abort_flag)) { ok = false; break; }
-                        if (!mbar_wait(bar(B_BUFFREE + b), ((g >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint64_t kdesc = make_desc(sbase + SM_KV + s * 16384);
-                        const uint32_t s_tm = tmem + b * 128, a_tm = s_tm + 64;
-#pragma unroll
-                        for (int ks = 0; ks < TC_D / 16; ++ks)
-                            mma_ss(s_tm, qdesc + 2 * ks, kdesc + 2 * ks, IDESC_SS, ks > 0);
-                        if (kind == SW_CG || kind == SW_OUT) {
-#pragma unroll
-                            for (int ks = 0; ks < TC_D / 16; ++ks)
-                                mma_ss(a_tm, phdesc + 2 * ks, kdesc + 2 * ks, IDESC_SS, ks > 0);
-#pragma unroll
-                            for (int ks = 0; ks < TC_D / 16; ++ks)
-                                mma_ss(a_tm, pldesc + 2 * ks, kdesc + 2 * ks, IDESC_SS, 1);
-                        }
-                        tc_commit(bar(B_SAFULL + b));
+        // All 32 lanes run this loop convergently; the MMAs and commits are predicated on one lane.
+        const uint32_t el = elect_one();
+        bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
+        const uint64_t qdesc = make_desc(sbase + SM_Q);
+        const uint64_t phdesc = make_desc(sbase + SM_PHI);
+        const uint64_t pldesc = make_desc(sbase + SM_PLO);
+        uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it & 1)
+        for (uint32_t sweep = 0; ok; ++sweep) {
+            TC_T0(t_c);
+            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+            if (lane == 0) TC_ACC(11, t_c);
+            const int kind = misc[1];
+            if (kind == SW_DONE) break;
+            tc_fence_after();
+            const uint32_t it0 = it;
+            for (int c = 0; c <= nblk && ok; ++c) {
+                if (c < nblk) {
+                    const uint32_t g = it0 + c, s = g % TC_NST, b = g & 1;
+                    TC_T0(t_k);
+                    if (!mbar_wait(bar(B_KVFULL + s), (g / TC_NST) & 1, abort_flag)) { ok = false; break; }
+                    if (lane == 0) TC_ACC(8, t_k);
+                    TC_T0(t_b);
+                    if (!mbar_wait(bar(B_BUFFREE + b), ((g >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (lane == 0) TC_ACC(9, t_b);
+                    tc_fence_after();
+                    const uint64_t kdesc = make_desc(sbase + SM_KV + s * 16384);
+                    const uint32_t s_tm = tmem + b * 128, a_tm = s_tm + 64;
+                    mma_ss_k64(el, s_tm, qdesc, kdesc, IDESC_SS, 0);
+                    if (kind == SW_CG || kind == SW_OUT) {
+                        mma_ss_k64(el, a_tm, phdesc, kdesc, IDESC_SS, 0);
+                        mma_ss_k64(el, a_tm, pldesc, kdesc, IDESC_SS, 1);
                     }
-                    if (c >= 1) {
-                        const uint32_t g = it0 + c - 1, s = g % TC_NST, b = g & 1;
-                        if (!mbar_wait(bar(B_UFULL + b), (g >> 1) & 1, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                        if (kind != SW_MAX) {
-                            const uint32_t bsm = sbase + SM_KV + s * 16384 + (kind == SW_OUT ? 8192 : 0);
-                            const uint64_t bdesc = make_desc(bsm);
-                            const uint32_t u_tm = tmem + b * 128;
-#pragma unroll
-                            for (int ks = 0; ks < TC_BC / 16; ++ks) {
-                                // 16 keys = two 8-row groups = 2048 bytes = 128 descriptor units
-                                mma_ts(tmem + TC_ACC_COL, u_tm + 16 * ks, bdesc + 128 * ks, IDESC_TS, (c > 1 || ks > 0));
-                                mma_ts(tmem + TC_ACC_COL, u_tm + 16 * ks + 8, bdesc + 128 * ks, IDESC_TS, 1);
-                            }
-                            tc_commit(bar(B_KVEMPTY + s));
-                            tc_commit(bar(B_BUFFREE + b));
-                            if (c == nblk) tc_commit(bar(B_ACCFULL));
-                        } else {
-                            mbar_arrive(bar(B_KVEMPTY + s));
-                            mbar_arrive(bar(B_BUFFREE + b));
-                        }
+                    tc_commit_el(el, bar(B_SAFULL + b));
+                }
+                if (c >= 1) {
+                    const uint32_t g = it0 + c - 1, s = g % TC_NST, b = g & 1;
+                    TC_T0(t_u);
+                    if (!mbar_wait(bar(B_UFULL + b), (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (lane == 0) TC_ACC(10, t_u);
+                    tc_fence_after();
+                    if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), ((c - 1) / TC_NST) & 1, abort_flag)) { ok = false; break; }
+                    if (kind != SW_MAX) {
+                        const uint32_t bsm = sbase + SM_KV + s * 16384 + (kind == SW_OUT ? 8192 : 0);
+                        mma_ts_hilo_k64(el, tmem + TC_ACC_COL, tmem + b * 128, make_desc(bsm), IDESC_TS, c > 1);
+                        tc_commit_el(el, bar(B_KVEMPTY + s));
+                        tc_commit_el(el, bar(B_BUFFREE + b));
+                        if (c == nblk) tc_commit_el(el, bar(B_ACCFULL));
+                    } else if (el) {
+                        mbar_arrive(bar(B_KVEMPTY + s));
+                        mbar_arrive(bar(B_BUFFREE + b));
                     }
                 }
-                it = it0 + nblk;
             }
+            it = it0 + nblk;
         }
     } else {
         // ================================ compute warps ================================
+        TC_T0(t_all);
         const int quad = warp & 3, half = warp >> 2;
         const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
         const int row = r0 + lrow;
@@ -395,61 +471,89 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         bool ok = true;
 
         // One sweep over the key blocks.  kind is uniform over the block.
+        // Warps 0-3 (group 0) take the even blocks, warps 4-7 (group 1) the odd ones, each thread all
+        // 64 keys of its row in two passes of 32: the two warps that share a scheduler are then in
+        // different phases of the load -> math -> store chain and hide each other's latency.
         auto sweep = [&](int kind) {
             float part = 0.f;                                 // omega / den partial, or max
             if (kind == SW_MAX) part = -INFINITY;
+            const uint64_t c1c1 = pk2(c1, c1), nmx = pk2(-mx2, -mx2);
+            const uint64_t nab = pk2(-abar, -abar), oab = pk2(1.f + abar, 1.f + abar), neg1 = pk2(-1.f, -1.f);
+            uint64_t part2 = pk2(0.f, 0.f);
             for (int c = 0; c < nblk; ++c, ++blk) {
+                if ((int)(blk & 1) != half) continue;
                 const uint32_t b = blk & 1;
+                TC_T0(t_w);
                 if (!mbar_wait(bar(B_SAFULL + b), (blk >> 1) & 1, abort_flag)) { ok = false; return part; }
+                if (tid == 0) TC_ACC(0, t_w);
                 tc_fence_after();
-                const uint32_t s_addr = tmem + lane_addr + b * 128 + c0;
-                uint32_t sv[32], av[32];
-                tmem_ld32(s_addr, sv);
-                if (kind == SW_CG || kind == SW_OUT) tmem_ld32(s_addr + 64, av);
-                tc_wait_ld();
-                const int j0 = c * TC_BC + c0;                // first key of this thread's 32
-                const int jlim = min(L, n) - j0;              // keys e < jlim are visible
-                if (kind == SW_MAX) {
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    TC_T0(t_l);
+                    const uint32_t s_addr = tmem + lane_addr + b * 128 + 32 * h;
+                    uint32_t sv[32], av[32];
+                    tmem_ld32(s_addr, sv);
+                    if (kind == SW_CG || kind == SW_OUT) tmem_ld32(s_addr + 64, av);
+                    tc_wait_ld();
+                    if (tid == 0) TC_ACC(1, t_l);
+                    TC_T0(t_m);
+                    const int jlim = min(L, n) - (c * TC_BC + 32 * h);   // keys e < jlim are visible
+                    if (kind == SW_MAX) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (e < jlim) part = fmaxf(part, __uint_as_float(sv[e]) * c1);
-                } else {
-                    float u[32];
+                        for (int e = 0; e < 32; ++e)
+                            if (e < jlim) part = fmaxf(part, __uint_as_float(sv[e]) * c1);
+                    } else {
+                        uint32_t pk[32];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        float w = ex2f(fmaf(__uint_as_float(sv[e]), c1, -mx2));
-                        if (kind == SW_CG) w *= (__uint_as_float(av[e]) - abar);
-                        if (kind == SW_OUT) w *= (1.f - (__uint_as_float(av[e]) - abar));
-                        u[e] = e < jlim ? w : 0.f;
-                    }
-                    if (kind != SW_CG) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) part += u[e];
-                    }
-                    // two k-steps of 16 keys; per k-step 8 columns of hi then 8 columns of lo
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const float a = u[ks * 16 + 2 * e], bq = u[ks * 16 + 2 * e + 1];
-                            const uint32_t hi = pack_bf16(bq, a);
-                            const float ra = a - __uint_as_float(hi << 16), rb = bq - __uint_as_float(hi & 0xFFFF0000u);
+                        for (int e2 = 0; e2 < 16; ++e2) {
+                            const uint64_t t2 = fma2(pk2(__uint_as_float(sv[2 * e2]), __uint_as_float(sv[2 * e2 + 1])), c1c1, nmx);
+                            float t0, t1;
+                            upk2(t2, t0, t1);
+                            uint64_t u2 = pk2(ex2f(t0), ex2f(t1));
+                            if (kind == SW_CG)
+                                u2 = mul2(u2, add2(pk2(__uint_as_float(av[2 * e2]), __uint_as_float(av[2 * e2 + 1])), nab));
+                            if (kind == SW_OUT)
+                                u2 = mul2(u2, fma2(pk2(__uint_as_float(av[2 * e2]), __uint_as_float(av[2 * e2 + 1])), neg1, oab));
+                            float u0, u1;
+                            upk2(u2, u0, u1);
+                            if (jlim < 32) {                       // only the diagonal blocks mask
+                                u0 = 2 * e2 < jlim ? u0 : 0.f;
+                                u1 = 2 * e2 + 1 < jlim ? u1 : 0.f;
+                                u2 = pk2(u0, u1);
+                            }
+                            if (kind != SW_CG) part2 = add2(part2, u2);
+                            // 16 keys per k-step: 8 columns of hi, then 8 columns of lo
+                            const uint32_t hi = pack_bf16(u1, u0);
+                            const uint64_t res = sub2(u2, pk2(__uint_as_float(hi << 16), __uint_as_float(hi & 0xFFFF0000u)));
+                            float ra, rb;
+                            upk2(res, ra, rb);
+                            const int ks = e2 >> 3, e = e2 & 7;
                             pk[ks * 16 + e] = hi;
                             pk[ks * 16 + 8 + e] = pack_bf16(rb, ra);
                         }
-                    tmem_st32(s_addr, pk);
-                    tc_wait_st();
+                        if (tid == 0) TC_ACC(2, t_m);
+                        TC_T0(t_s);
+                        tmem_st32(s_addr, pk);
+                        if (tid == 0) TC_ACC(3, t_s);
+                    }
                 }
+                if (kind != SW_MAX) tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(B_UFULL + b));
+            }
+            if (kind != SW_MAX) {
+                float p0, p1;
+                upk2(part2, p0, p1);
+                part = p0 + p1;
             }
             return part;
         };
         // read this thread's 32 ACC columns after the sweep's last MMA
         uint32_t acc_uses = 0;
         auto read_acc = [&](float* dst) {
+            TC_T0(t_a);
             if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag)) { ok = false; return; }
+            if (tid == 0) TC_ACC(4, t_a);
             ++acc_uses;
             tc_fence_after();
             uint32_t v[32];
@@ -607,6 +711,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
         if (ok) start_sweep(SW_DONE);
+        if (tid == 0) TC_ACC(5, t_all);
+        if (tid == 0) { TC_T0(t_one); TC_ACC(6, t_one - 1); (void)nblk; }
     }
 
     // ================================ common exit ================================
@@ -674,6 +780,10 @@ int launch_t(const ForwardArgs& a) {
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
+    prm.dbg = nullptr;
+#ifdef LLA_TC_TIMING
+    prm.dbg = (unsigned long long*)a.workspace;   // tuning builds only: caller passes a zeroed buffer
+#endif
     auto kern = forward_tc_kernel<TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
     dim3 grid(BH, tiles);
