@@ -74,6 +74,7 @@ int check_decode(const lla_decode_params* p) {
     if (!p) return LLA_ERR_INVALID_ARG;
     if (!p->q || !p->kcache || !p->vcache || !p->lens || !p->out) return LLA_ERR_INVALID_ARG;
     if (p->B < 1 || p->H < 1 || p->Lmax < 1 || p->d < 1 || p->dv < 1 || p->splits < 0) return LLA_ERR_INVALID_ARG;
+    if (p->impl != LLA_IMPL_AUTO && p->impl != LLA_IMPL_SIMT && p->impl != LLA_IMPL_TENSOR) return LLA_ERR_INVALID_ARG;
     if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
@@ -173,6 +174,7 @@ int lla_decode_ex(const lla_decode_params* p) {
     }
     if (a.splits > 1 && ((uintptr_t)p->workspace & 255u)) return LLA_ERR_WORKSPACE;
     a.head_rows = 2 * p->d;
+    a.impl = p->impl;
     a.status = p->device_status;
     a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
     a.stream = (cudaStream_t)p->stream;

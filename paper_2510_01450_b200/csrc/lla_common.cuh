@@ -44,6 +44,7 @@ struct DecodeArgs {
     float scale, lambda;
     int splits;
     int head_rows;   // caches shorter than this are solved directly (fp64)
+    int impl;        // lla_impl
     int* status;
     void* workspace;
     size_t workspace_bytes;
@@ -58,6 +59,8 @@ int launch_forward_tensor(const ForwardArgs& a);
 bool forward_tensor_supported(const ForwardArgs& a);
 int launch_decode(const DecodeArgs& a);
 int launch_head_rows_decode(const DecodeArgs& a);
+bool decode_tensor_supported(const DecodeArgs& a);
+int launch_decode_tensor_moments(const DecodeArgs& a);
 size_t decode_workspace_bytes(int B, int H, int d, int dv, int splits);
 
 // ---------------------------------------------------------------------------------------------

@@ -274,13 +274,20 @@ int launch_t(const DecodeArgs& a) {
         const size_t need = decode_workspace_bytes(a.B, a.H, a.d, a.dv, splits);
         if (!a.workspace || a.workspace_bytes < need) return LLA_ERR_WORKSPACE;
     }
-    auto k1 = decode_moments_kernel<D, TIn, TOut>;
-    LLA_CUDA_TRY(cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    dim3 grid(splits, a.B * a.H);
-    k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
-                                             a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
-                                             a.head_rows, (float*)a.workspace, a.status);
-    LLA_CUDA_TRY(cudaGetLastError());
+    if (a.impl != LLA_IMPL_SIMT && decode_tensor_supported(a)) {
+        // moment pass on tensor cores (writes the same partial records when splits > 1)
+        const int st = launch_decode_tensor_moments(a);
+        if (st != LLA_OK) return st;
+    } else {
+        if (a.impl == LLA_IMPL_TENSOR) return LLA_ERR_UNSUPPORTED;
+        auto k1 = decode_moments_kernel<D, TIn, TOut>;
+        LLA_CUDA_TRY(cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        dim3 grid(splits, a.B * a.H);
+        k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
+                                                 a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
+                                                 a.head_rows, (float*)a.workspace, a.status);
+        LLA_CUDA_TRY(cudaGetLastError());
+    }
     if (splits > 1) {
         auto k2 = decode_combine_kernel<D, TIn, TOut>;
         LLA_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -364,6 +371,7 @@ extern "C" int lla_decode_noalloc(const void* q, const void* kcache, const void*
     a.scale = scale; a.lambda = lambda;
     a.splits = splits > 0 ? splits : lla_decode_default_splits(B, H, Lmax);
     a.head_rows = 2 * d;
+    a.impl = LLA_IMPL_AUTO;
     a.status = nullptr;
     a.workspace = nullptr; a.workspace_bytes = 0;
     a.stream = (cudaStream_t)stream;

@@ -1,0 +1,412 @@
+// LLA decode on tensor cores (bf16 caches, d = dv = 64): one pass over the KV cache at HBM speed.
+//
+// Decode is bound by reading K and V once, so the cache is streamed a single time and folded into
+// the weighted moments about the origin that the centred form of Eq. "lla_decomp" needs:
+//     D = [K^T ; V^T] diag(w) [K | 1]      (128 x 80, fp32 in TMEM)
+//       rows 0..63   : M = sum_j w_j k_j k_j^T   and, in column 64, a = sum_j w_j k_j
+//       rows 64..127 : N = sum_j w_j v_j k_j^T   and, in column 64, c = sum_j w_j v_j
+// Per 64-key tile:
+//   TMA         K and V tiles -> 128B-swizzled shared memory (3-stage ring).  The two tiles sit back
+//               to back and together form the MN-major A operand [K^T ; V^T] of one M = 128 MMA.
+//   CUDA cores  two lanes per key: score s_j = scale q.k_j, weight w_j = exp(s_j - m_ref), then the
+//               row w_j [k_j | 1] split into bf16 hi + lo is written to the B operand tiles
+//               (canonical MN-major layout without swizzle, 80 columns); omega += w_j.
+//   MMA (SS)    D += A B_hi + A B_lo, four 16-key steps each.
+// m_ref is the maximum of the first tile; if a later tile's maximum exceeds it by more than 2^40 the
+// accumulator is rescaled in TMEM (never triggered by bounded scores, covered by a test).  After
+// the last tile the moments are copied to shared memory and either solved on the spot (d x d LDL^T
+// in double precision, as in lla_decode.cu) or written as a partial record for the split-key merge.
+#include "lla_sm100.cuh"
+
+namespace lla {
+namespace {
+
+using namespace sm100;
+
+constexpr int DT_D = 64;
+constexpr int DT_BK = 64;             // keys per tile
+constexpr int DT_NST = 3;             // K/V ring stages
+constexpr int DT_COMPUTE = 128;       // warps 0..3
+constexpr int DT_THREADS = 192;       // + TMA warp (4) + MMA warp (5)
+constexpr int DT_TMEM_COLS = 128;
+constexpr int DT_N = 80;              // MMA N: 64 key features + the ones column (padded to 16)
+constexpr int DT_BTILE = 10240;       // one B tile: 10 column blocks x 8 key blocks x 128 bytes
+
+constexpr int SMD_KV = 0;                                   // DT_NST x (K 8192 + V 8192)
+constexpr int SMD_B = SMD_KV + DT_NST * 16384;              // 2 buffers x (hi, lo) x DT_BTILE
+constexpr int SMD_BAR = SMD_B + 4 * DT_BTILE;               // mbarriers
+constexpr int SMD_MISC = SMD_BAR + 128;                     // tmem base, abort, tile maxima
+constexpr int SMD_TOTAL = SMD_MISC + 128;
+// the epilogue reuses everything from offset 0: M (64 x 65 doubles), a, c, rhs (3 x 64 doubles), N (64 x 64 floats)
+constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 64;
+constexpr int SMD_ALLOC = (SMD_TOTAL > SMD_FIN ? SMD_TOTAL : SMD_FIN) + 1024;
+
+enum { DB_KVFULL = 0, DB_KVEMPTY = DB_KVFULL + DT_NST, DB_BFULL = DB_KVEMPTY + DT_NST, DB_BFREE = DB_BFULL + 2,
+       DB_DFULL = DB_BFREE + 2, DB_COUNT = DB_DFULL + 1 };
+static_assert(DB_COUNT * 8 <= 128, "barrier area too small");
+
+// A = [K^T ; V^T]: MN-major, 128B swizzle; the V tile (second group of 64 rows of M) lies 8192 bytes
+// after the K tile (leading byte offset), 8-key groups are 1024 bytes apart (stride byte offset).
+__device__ __forceinline__ uint64_t make_desc_a(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(8192 >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;      // SWIZZLE_128B
+    return d;
+}
+// B: MN-major without swizzle: 8 x 8 core matrices of 128 bytes; key groups are 128 bytes apart
+// (leading byte offset), column groups 1024 bytes apart (stride byte offset).
+__device__ __forceinline__ uint64_t make_desc_b(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(128 >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;                    // layout type 0: no swizzle
+}
+constexpr uint32_t IDESC_DEC = make_idesc(128, DT_N, 1, 1);
+
+// D += A B_hi + A B_lo over 64 keys.  A steps 2048 bytes (128 units) per 16 keys, B 256 bytes (16 units).
+__device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, uint64_t bhi, uint64_t blo, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, h1, h2, h3, l1, l2, l3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "add.u64 a1, %2, 128; add.u64 a2, %2, 256; add.u64 a3, %2, 384;\n\t"
+        "add.u64 h1, %3, 16; add.u64 h2, %3, 32; add.u64 h3, %3, 48;\n\t"
+        "add.u64 l1, %4, 16; add.u64 l2, %4, 32; add.u64 l3, %4, 48;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %5, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %4, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, h1, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, l1, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, h2, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, l2, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, h3, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, l3, %5, p;\n\t}"
+        ::"r"(el), "r"(d), "l"(a), "l"(bhi), "l"(blo), "r"(IDESC_DEC), "r"(acc0) : "memory");
+}
+
+__device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+struct DtParams {
+    int H, Lmax, splits, head_rows;
+    float scale, lambda;
+    const int* lens;
+    float* parts;
+    int* status;
+};
+
+template <typename TOut>
+__global__ void __launch_bounds__(DT_THREADS, 2)
+decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                 const __nv_bfloat16* __restrict__ q, TOut* __restrict__ out, const DtParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + SMD_BAR;
+    auto bar = [&](int i) { return bars + 8u * i; };
+    volatile int* misc = reinterpret_cast<volatile int*>(smem + SMD_MISC);   // [0] tmem base, [1] abort
+    volatile int* abort_flag = misc + 1;
+    volatile float* tmax = reinterpret_cast<volatile float*>(smem + SMD_MISC + 16);   // 2 x 4 warp maxima
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.y, part = blockIdx.x;
+    int L = prm.lens[bh / prm.H];
+    L = max(1, min(L, prm.Lmax));
+    if (L < prm.head_rows) return;                      // short caches: solved by the direct fp64 kernel
+    const int chunk = ((L + prm.splits - 1) / prm.splits + DT_BK - 1) / DT_BK * DT_BK;
+    const int jbeg = part * chunk, jend = min(L, jbeg + chunk);
+    const int ntile = jend > jbeg ? (jend - jbeg + DT_BK - 1) / DT_BK : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < DT_NST; ++s) { mbar_init(bar(DB_KVFULL + s), 1); mbar_init(bar(DB_KVEMPTY + s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(DB_BFULL + b), DT_COMPUTE); mbar_init(bar(DB_BFREE + b), 1); }
+        mbar_init(bar(DB_DFULL), 1);
+        misc[1] = 0;
+        fence_barrier_init();
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(sbase + SMD_MISC), "r"(DT_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)misc[0];
+
+    float omega = 0.f, m_ref = -INFINITY;     // compute threads; m_ref in log2 units
+
+    if (warp == 4) {
+        // ================================ TMA producer ================================
+        if (lane == 0) {
+            for (int t = 0; t < ntile; ++t) {
+                const uint32_t s = t % DT_NST;
+                if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
+                const uint32_t dst = sbase + SMD_KV + s * 16384;
+                mbar_expect_tx(bar(DB_KVFULL + s), 16384);
+                tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, bh);
+                tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, bh);
+            }
+        }
+    } else if (warp == 5) {
+        // ================================ MMA issuer (whole warp, predicated) ================================
+        const uint32_t el = elect_one();
+        for (int t = 0; t < ntile; ++t) {
+            const uint32_t s = t % DT_NST, b = t & 1;
+            if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(DB_BFULL + b), (t >> 1) & 1, abort_flag)) break;
+            tc_fence_after();
+            const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
+            mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), make_desc_b(bsm + DT_BTILE), t > 0);
+            tc_commit_el(el, bar(DB_KVEMPTY + s));
+            tc_commit_el(el, bar(DB_BFREE + b));
+            if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
+        }
+    } else {
+        // ================================ compute warps ================================
+        const int jl = tid >> 1, h = tid & 1;            // key inside the tile, feature half
+        const float c1 = prm.scale * 1.4426950408889634f;
+        float qv[32];
+        {
+            const __nv_bfloat16* qp = q + (size_t)bh * DT_D + 32 * h;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) load8(qp + 8 * i, qv + 8 * i);
+        }
+        bool ok = true;
+        for (int t = 0; t < ntile && ok; ++t) {
+            const uint32_t s = t % DT_NST, b = t & 1;
+            if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) { ok = false; break; }
+            uint8_t* ktile = smem + SMD_KV + s * 16384;
+            const int jglob = jbeg + t * DT_BK + jl;
+            const bool valid = jglob < jend;
+            // this lane's 32 features of key jl (swizzled 16-byte chunks 4h .. 4h+3)
+            float kf[32];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(ktile + jl * 128 + (((4 * h + i) ^ (jl & 7)) << 4));
+                const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    kf[8 * i + 2 * e] = __uint_as_float(wds[e] << 16);
+                    kf[8 * i + 2 * e + 1] = __uint_as_float(wds[e] & 0xFFFF0000u);
+                }
+            }
+            if (!valid) {
+                // ragged last tile: rows past the end may hold anything (unused cache slots).  They are
+                // part of the A operand, so clear them (0 x NaN would poison the accumulator).
+#pragma unroll
+                for (int e = 0; e < 32; ++e) kf[e] = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t off = jl * 128 + (((4 * h + i) ^ (jl & 7)) << 4);
+                    *reinterpret_cast<uint4*>(ktile + off) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(ktile + 8192 + off) = make_uint4(0, 0, 0, 0);
+                }
+            }
+            float sdot = 0.f;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) sdot = fmaf(qv[e], kf[e], sdot);
+            sdot += __shfl_xor_sync(0xffffffffu, sdot, 1);
+            const float s2 = valid ? sdot * c1 : -INFINITY;
+            // tile maximum (uniform over the 128 compute threads)
+            float wm = s2;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
+            volatile float* tm = tmax + (t & 1) * 4;
+            if (lane == 0) tm[warp] = wm;
+            named_sync_128();
+            const float tile_max = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
+            if (t == 0) {
+                m_ref = tile_max;
+            } else if (tile_max > m_ref + 40.f) {
+                // rare: rescale the accumulator (all MMAs of earlier tiles must have finished)
+                const float f = ex2f(m_ref - tile_max);
+                if (!mbar_wait(bar(DB_BFREE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+                for (int cb = 0; cb < 96; cb += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(lane_addr + cb, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+                    tmem_st32(lane_addr + cb, v);
+                    tc_wait_st();
+                }
+                tc_fence_before();
+                omega *= f;
+                m_ref = tile_max;
+                named_sync_128();
+            }
+            const float w = valid ? ex2f(s2 - m_ref) : 0.f;
+            if (h == 0) omega += w;
+            // B rows: w * [k | 1] as bf16 hi + lo.  Wait until the MMA of tile t-2 has released the buffer.
+            if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
+            uint8_t* blo = bhi + DT_BTILE;
+            const uint32_t rowoff = (jl >> 3) * 128 + (jl & 7) * 16;      // key group, row inside the core matrix
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float a = w * kf[8 * i + 2 * e], bq = w * kf[8 * i + 2 * e + 1];
+                    hi[e] = pack_bf16(bq, a);
+                    lo[e] = pack_bf16(bq - __uint_as_float(hi[e] & 0xFFFF0000u), a - __uint_as_float(hi[e] << 16));
+                }
+                const uint32_t off = (4 * h + i) * 1024 + rowoff;          // column block 4h+i
+                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+            {   // column blocks 8 (ones column first) and 9 (zero padding)
+                const uint32_t whi = pack_bf16(0.f, w);
+                const uint32_t wlo = pack_bf16(0.f, w - __uint_as_float(whi << 16));
+                const uint32_t off = (8 + h) * 1024 + rowoff;
+                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
+                *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
+            }
+            fence_proxy_async();
+            mbar_arrive(bar(DB_BFULL + b));
+        }
+        // total weight of this part
+        if (ok) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) omega += __shfl_xor_sync(0xffffffffu, omega, off);
+        }
+    }
+
+    // ================================ epilogue ================================
+    // All 192 threads take part (the solve below is a block-wide routine).
+    __shared__ float s_omega[4];
+    __shared__ float s_mref;
+    if (warp < 4 && lane == 0) s_omega[warp] = omega;
+    if (tid == 0) s_mref = m_ref;
+    bool d_ok = true;
+    if (warp < 4 && ntile > 0) {
+        d_ok = mbar_wait(bar(DB_DFULL), 0, abort_flag);
+        tc_fence_after();
+    }
+    // moments -> registers (lane f: row f of M plus a[f]; lane 64+f: row f of N plus c[f])
+    float dv[96];
+    if (warp < 4) {
+        if (ntile > 0 && d_ok) {
+            const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+            for (int cb = 0; cb < 96; cb += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + cb, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) dv[cb + e] = __uint_as_float(v[e]);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 96; ++e) dv[e] = 0.f;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();       // every pipeline stage is drained: shared memory can be re-carved
+    if (warp == 4) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(DT_TMEM_COLS) : "memory");
+    }
+    const bool aborted = *abort_flag != 0;
+    if (aborted) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+        return;
+    }
+    const float omega_tot = s_omega[0] + s_omega[1] + s_omega[2] + s_omega[3];
+    const float mref_ln = s_mref * 0.6931471805599453f;          // back to natural-log units
+
+    if (prm.splits > 1) {
+        // partial record for the merge kernel: M, N, a, c, omega, m (same layout as the SIMT path)
+        float* dst = prm.parts + ((size_t)bh * prm.splits + part) * (2 * 64 * 64 + 2 * 64 + 4);
+        if (warp < 4) {
+            float* rowp = dst + (size_t)tid * 64;                 // tid < 64: M rows; 64..127: N rows
+#pragma unroll
+            for (int e = 0; e < 64; e += 4)
+                *reinterpret_cast<float4*>(rowp + e) = make_float4(dv[e], dv[e + 1], dv[e + 2], dv[e + 3]);
+            dst[2 * 64 * 64 + tid] = dv[64];                      // a then c
+        }
+        if (tid == 0) {
+            dst[2 * 64 * 64 + 128] = omega_tot;
+            dst[2 * 64 * 64 + 129] = ntile > 0 ? mref_ln : -INFINITY;
+        }
+        return;
+    }
+
+    // single part: centre, solve and emit the output row here
+    double* Md = reinterpret_cast<double*>(smem);              // 64 x 65
+    double* av = Md + 64 * 65;                                  // a -> kbar
+    double* cv = av + 64;                                       // c -> vbar
+    double* rhs = cv + 64;
+    float* Nd = reinterpret_cast<float*>(rhs + 64);             // 64 x 64
+    const double inv = 1.0 / (double)omega_tot;
+    const double ridge = (double)prm.lambda * exp(-(double)mref_ln) * inv;
+    if (warp < 4) {
+        if (tid < 64) av[tid] = (double)dv[64] * inv;
+        else cv[tid - 64] = (double)dv[64] * inv;
+    }
+    __syncthreads();
+    if (warp < 4) {
+        if (tid < 64) {
+            for (int e = 0; e <= tid; ++e)
+                Md[tid * 65 + e] = (double)dv[e] * inv - av[tid] * av[e] + (e == tid ? ridge : 0.0);
+            rhs[tid] = (double)to_f32(q[(size_t)bh * DT_D + tid]) - av[tid];
+        } else {
+#pragma unroll
+            for (int e = 0; e < 64; ++e) Nd[(tid - 64) * 64 + e] = dv[e];
+        }
+    }
+    const bool solved = block_ldlt_solve<64>(Md, 65, rhs);
+    if (tid < 64) {
+        double o = cv[tid];
+        for (int f = 0; f < 64; ++f) o += ((double)Nd[tid * 64 + f] * inv - cv[tid] * av[f]) * rhs[f];
+        store_out(out + (size_t)bh * DT_D + tid, (float)o);
+    }
+    if (!solved && tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_BAD_PIVOT, 1);
+}
+
+template <typename TOut>
+int launch_t(const DecodeArgs& a) {
+    const int splits = a.splits < 1 ? 1 : a.splits;
+    if (splits > 1) {
+        const size_t need = decode_workspace_bytes(a.B, a.H, a.d, a.dv, splits);
+        if (!a.workspace || a.workspace_bytes < need) return LLA_ERR_WORKSPACE;
+    }
+    CUtensorMap mk, mv;
+    const int BH = a.B * a.H;
+    if (!make_map_bf16_64(&mk, a.kcache, BH, a.Lmax, DT_BK) || !make_map_bf16_64(&mv, a.vcache, BH, a.Lmax, DT_BK))
+        return LLA_ERR_CUDA;
+    DtParams prm;
+    prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
+    prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
+    prm.parts = (float*)a.workspace; prm.status = a.status;
+    auto kern = decode_tc_kernel<TOut>;
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMD_ALLOC));
+    dim3 grid(splits, BH);
+    kern<<<grid, DT_THREADS, SMD_ALLOC, a.stream>>>(mk, mv, (const __nv_bfloat16*)a.q, (TOut*)a.out, prm);
+    LLA_CUDA_TRY(cudaGetLastError());
+    return LLA_OK;
+}
+
+}  // namespace
+
+bool decode_tensor_supported(const DecodeArgs& a) {
+    return a.in_dtype == LLA_BF16 && a.d == DT_D && a.dv == DT_D && sm100::get_encode() != nullptr;
+}
+
+// Moment pass on tensor cores; with splits > 1 the caller still runs the merge kernel afterwards.
+int launch_decode_tensor_moments(const DecodeArgs& a) {
+    if (!decode_tensor_supported(a)) return LLA_ERR_UNSUPPORTED;
+    if (a.out_dtype == LLA_BF16) return launch_t<__nv_bfloat16>(a);
+    if (a.out_dtype == LLA_F32) return launch_t<float>(a);
+    return LLA_ERR_UNSUPPORTED;
+}
+
+}  // namespace lla

@@ -136,6 +136,38 @@ def test_decode_matches_oracle_and_splits_agree(oracle, dtype, d):
     np.testing.assert_allclose(out.cpu().numpy()[0], vc[0, :, 0], rtol=1e-5, atol=1e-6)
 
 
+@pytest.mark.parametrize("impl", [L.LLA_IMPL_SIMT, L.LLA_IMPL_AUTO])
+def test_decode_unused_slots_and_late_maximum(oracle, impl):
+    """Slots past lens[b] may hold anything (here NaN) and must not leak into the result; and a cache
+    whose first 64 keys score ~70 units below the rest forces the tensor path to rescale its running
+    accumulator when the later, larger scores arrive."""
+    w = inputs.CONFIGS[5].shrink(B=2, H=2, n=1200, len_min=300, len_max=1200, seed=61)
+    q, kc, vc, lens = inputs.make_decode(w)
+    lens[:] = [1111, 333]
+    qn = q / (np.linalg.norm(q, axis=-1, keepdims=True) ** 2)           # q.qn = 1
+    kc[:, :, :64] += (-70.0 / w.scale) * qn[:, :, None, :]             # scaled score of the first tile ~ -70
+    kc = inputs.round_to_bf16(kc)
+    ref = oracle.decode(q, kc, vc, lens, w.scale, w.lam)
+    for b in range(w.B):
+        kc[b, :, lens[b]:] = np.nan
+        vc[b, :, lens[b]:] = np.nan
+    dq, dk, dv_ = dev(q, "bf16"), dev(kc, "bf16"), dev(vc, "bf16")
+    dl = torch.from_numpy(lens).cuda()
+    for splits in (1, 2):
+        nbytes = L.lla_decode_workspace_bytes(w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, splits)
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+        out = torch.full((w.B, w.H, w.dv), float("nan"), dtype=torch.float32, device="cuda")
+        L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, out_dtype=L.LLA_F32,
+                        splits=splits, impl=impl, device_status=status, workspace=ws, workspace_bytes=nbytes,
+                        stream=stream_ptr())
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        assert np.isfinite(got).all(), splits
+        assert row_err(got, ref).max() <= TOL_BF16, (splits, row_err(got, ref).max())
+        assert status.cpu().numpy()[L.STATUS_TIMEOUT] == 0
+
+
 @pytest.mark.parametrize("n", [1, 2, 31, 127, 128, 129, 300])
 def test_ragged_and_tiny_lengths(oracle, n):
     w = inputs.CONFIGS[2].shrink(B=2, H=1, n=n, seed=100 + n)
