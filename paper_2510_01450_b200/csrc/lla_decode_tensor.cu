@@ -6,7 +6,7 @@
 //       rows 0..63   : M = sum_j w_j k_j k_j^T   and, in column 64, a = sum_j w_j k_j
 //       rows 64..127 : N = sum_j w_j v_j k_j^T   and, in column 64, c = sum_j w_j v_j
 // Per 64-key tile:
-//   TMA         K and V tiles -> 128B-swizzled shared memory (3-stage ring).  The two tiles sit back
+//   TMA         K and V tiles -> 128B-swizzled shared memory (4-stage ring).  The two tiles sit back
 //               to back and together form the MN-major A operand [K^T ; V^T] of one M = 128 MMA.
 //   CUDA cores  two lanes per key: score s_j = scale q.k_j, weight w_j = exp(s_j - m_ref), then the
 //               row w_j [k_j | 1] split into bf16 hi + lo is written to the B operand tiles
@@ -25,11 +25,12 @@ using namespace sm100;
 
 constexpr int DT_D = 64;
 constexpr int DT_BK = 64;             // keys per tile
-constexpr int DT_NST = 3;             // K/V ring stages
+constexpr int DT_NST = 4;             // K/V ring stages
 constexpr int DT_COMPUTE = 128;       // warps 0..3
 constexpr int DT_THREADS = 192;       // + TMA warp (4) + MMA warp (5)
 constexpr int DT_TMEM_COLS = 128;
 constexpr int DT_N = 80;              // MMA N: 64 key features + the ones column (padded to 16)
+constexpr int DT_MAX_RANKED = 1024;   // batches up to this size are processed longest-first
 constexpr int DT_BTILE = 10240;       // one B tile: 10 column blocks x 8 key blocks x 128 bytes
 
 constexpr int SMD_KV = 0;                                   // DT_NST x (K 8192 + V 8192)
@@ -38,7 +39,7 @@ constexpr int SMD_BAR = SMD_B + 4 * DT_BTILE;               // mbarriers
 constexpr int SMD_MISC = SMD_BAR + 128;                     // tmem base, abort, tile maxima
 constexpr int SMD_TOTAL = SMD_MISC + 128;
 // the epilogue reuses everything from offset 0: M (64 x 65 doubles), a, c, rhs (3 x 64 doubles), N (64 x 64 floats)
-constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 64;
+constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 65;
 constexpr int SMD_ALLOC = (SMD_TOTAL > SMD_FIN ? SMD_TOTAL : SMD_FIN) + 1024;
 
 enum { DB_KVFULL = 0, DB_KVEMPTY = DB_KVFULL + DT_NST, DB_BFULL = DB_KVEMPTY + DT_NST, DB_BFREE = DB_BFULL + 2,
@@ -91,7 +92,7 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
 __device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 struct DtParams {
-    int H, Lmax, splits, head_rows;
+    int B, H, Lmax, splits, head_rows;
     float scale, lambda;
     const int* lens;
     float* parts;
@@ -112,7 +113,25 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     volatile float* tmax = reinterpret_cast<volatile float*>(smem + SMD_MISC + 16);   // 2 x 4 warp maxima
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.y, part = blockIdx.x;
+    const int part = blockIdx.x;
+    // Longest caches first: blocks launch in blockIdx order, so block y takes head (y % H) of the
+    // sequence whose length has rank (y / H).  Every block ranks the (few) sequence lengths itself.
+    int bh = blockIdx.y;
+    if (prm.B <= DT_MAX_RANKED) {
+        __shared__ int s_len[DT_MAX_RANKED];
+        __shared__ int s_pick;
+        for (int b = tid; b < prm.B; b += DT_THREADS) s_len[b] = max(1, min(prm.lens[b], prm.Lmax));
+        __syncthreads();
+        const int want = blockIdx.y / prm.H;
+        for (int b = tid; b < prm.B; b += DT_THREADS) {
+            const int lb = s_len[b];
+            int rank = 0;
+            for (int o = 0; o < prm.B; ++o) rank += (s_len[o] > lb) || (s_len[o] == lb && o < b);
+            if (rank == want) s_pick = b;
+        }
+        __syncthreads();
+        bh = s_pick * prm.H + blockIdx.y % prm.H;
+    }
     int L = prm.lens[bh / prm.H];
     L = max(1, min(L, prm.Lmax));
     if (L < prm.head_rows) return;                      // short caches: solved by the direct fp64 kernel
@@ -206,9 +225,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     *reinterpret_cast<uint4*>(ktile + 8192 + off) = make_uint4(0, 0, 0, 0);
                 }
             }
-            float sdot = 0.f;
+            float sd[4] = {0.f, 0.f, 0.f, 0.f};          // four independent chains
 #pragma unroll
-            for (int e = 0; e < 32; ++e) sdot = fmaf(qv[e], kf[e], sdot);
+            for (int e = 0; e < 32; ++e) sd[e & 3] = fmaf(qv[e], kf[e], sd[e & 3]);
+            float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
             sdot += __shfl_xor_sync(0xffffffffu, sdot, 1);
             const float s2 = valid ? sdot * c1 : -INFINITY;
             // tile maximum (uniform over the 128 compute threads)
@@ -345,7 +365,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     double* av = Md + 64 * 65;                                  // a -> kbar
     double* cv = av + 64;                                       // c -> vbar
     double* rhs = cv + 64;
-    float* Nd = reinterpret_cast<float*>(rhs + 64);             // 64 x 64
+    float* Nd = reinterpret_cast<float*>(rhs + 64);             // 64 x 65 (padded rows)
     const double inv = 1.0 / (double)omega_tot;
     const double ridge = (double)prm.lambda * exp(-(double)mref_ln) * inv;
     if (warp < 4) {
@@ -360,13 +380,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             rhs[tid] = (double)to_f32(q[(size_t)bh * DT_D + tid]) - av[tid];
         } else {
 #pragma unroll
-            for (int e = 0; e < 64; ++e) Nd[(tid - 64) * 64 + e] = dv[e];
+            for (int e = 0; e < 64; ++e) Nd[(tid - 64) * 65 + e] = dv[e];
         }
     }
     const bool solved = block_ldlt_solve<64>(Md, 65, rhs);
     if (tid < 64) {
         double o = cv[tid];
-        for (int f = 0; f < 64; ++f) o += ((double)Nd[tid * 64 + f] * inv - cv[tid] * av[f]) * rhs[f];
+        for (int f = 0; f < 64; ++f) o += ((double)Nd[tid * 65 + f] * inv - cv[tid] * av[f]) * rhs[f];
         store_out(out + (size_t)bh * DT_D + tid, (float)o);
     }
     if (!solved && tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_BAD_PIVOT, 1);
@@ -384,11 +404,13 @@ int launch_t(const DecodeArgs& a) {
     if (!make_map_bf16_64(&mk, a.kcache, BH, a.Lmax, DT_BK) || !make_map_bf16_64(&mv, a.vcache, BH, a.Lmax, DT_BK))
         return LLA_ERR_CUDA;
     DtParams prm;
-    prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
+    prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
     prm.parts = (float*)a.workspace; prm.status = a.status;
     auto kern = decode_tc_kernel<TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMD_ALLOC));
+    // two blocks per SM need the largest shared-memory carve-out
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     dim3 grid(splits, BH);
     kern<<<grid, DT_THREADS, SMD_ALLOC, a.stream>>>(mk, mv, (const __nv_bfloat16*)a.q, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());

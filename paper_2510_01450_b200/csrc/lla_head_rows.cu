@@ -227,6 +227,7 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
         ((size_t)D * C::LDS + 2 * D + lcap + (size_t)HR_CHUNK * D + HR_THREADS / 32 + 1);
     auto kern = head_rows_kernel<D, D, TIn, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     dim3 grid(rows_per_head, a.B * a.H);
     kern<<<grid, HR_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
@@ -242,6 +243,7 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
         ((size_t)D * C::LDS + 2 * D + lcap + (size_t)HR_CHUNK * D + HR_THREADS / 32 + 1);
     auto kern = head_rows_kernel<D, D, TIn, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     dim3 grid(1, a.B * a.H);
     kern<<<grid, HR_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
