@@ -29,9 +29,10 @@ METRIC = "lla_prefill_tokens_per_s"
 UNIT = "tokens/s"
 WORKLOAD = 2          # the bf16 prefill workload the headline metric is quoted on
 ROTATE = 16           # input sets cycled through so no step finds its inputs in L2
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
-# (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/
+# (forward_tc_kernel_cfg2.md and decode_tc_kernel_cfg5.md).
+NCU_TRAFFIC_BYTES = 12.68e6
+NCU_DECODE_TRAFFIC_BYTES = 1.189e9 + 35.6e6
 
 
 def env_int(name, default):
@@ -293,7 +294,9 @@ def run_ours(args):
         "tflops": flops_step / (ms_step * 1e-3) / 1e12,
         "roofline": {"bound": "tensor", "achieved": tflops_kernel, "peak": peak, "unit": "TFLOP/s",
                      "frac": tflops_kernel / peak, "traffic": NCU_TRAFFIC_BYTES,
-                     "kernel": "iterative-rows forward kernel", "ms_per_launch": ms_kernel,
+                     "kernel": "iterative-rows forward kernel (forward_tc_kernel)", "ms_per_launch": ms_kernel,
+                     "algorithmic_flops_per_launch": flops_step_iterative(w, it_np),
+                     "algorithmic_bytes_per_launch": int(set_bytes),
                      "peak_source": f"{peaks['source']} burst bf16 (MEASURED_PEAKS.json)",
                      "direct_rows_ms_per_launch": ms_direct},
         "e2e": {"value": world * tokens_step * e2e_steps / e2e_s, "unit": UNIT,
@@ -346,7 +349,7 @@ def bench_decode(L, torch, peaks, sp, stream, steps=20, warmup=5):
     del kc, vc
     return {"workload": wd.name, "us_per_step": ms * 1e3, "us_per_token": ms * 1e3 / wd.B, "steps": steps,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "algorithmic_bytes": live_bytes,
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_DECODE_TRAFFIC_BYTES, "algorithmic_bytes": live_bytes,
                          "frac_of_nominal_8TBs": gbs / 8000.0,
                          "peak_source": f"{peaks['source']} copy bandwidth (MEASURED_PEAKS.json)"},
             "l2": "live cache bytes (1.2 GB) exceed L2 (126 MB)"}
