@@ -16,10 +16,10 @@
 //   MMA 2 (TS)     ACC += U_hi B + U_lo B, A operand straight from TMEM, B = the same K block read
 //                  MN-major (or the V block in the output sweep)
 //
-// S/A/U are double buffered in TMEM (2 x 128 columns) and ACC takes 64 more; K/V blocks go through a
+// S/A/U cycle through three TMEM buffers (3 x 128 columns) and ACC takes 64 more; K/V blocks go through a
 // 4-stage ring.  Roles: warps 0-7 compute (warp w owns TMEM lanes 32*(w%4).. and key half w/4 of each
 // block; two threads share a row and exchange partial sums through shared memory), warp 8 issues TMA,
-// warp 9 issues MMAs.  Every on-the-fly MMA operand (P, y, U) is carried as a bf16 pair hi + lo so
+// warps 9 and 10 issue the two MMA streams.  Every on-the-fly MMA operand (P, y, U) is carried as a bf16 pair hi + lo so
 // the products keep ~16 mantissa bits: a single bf16 rounding of those operands would leave a
 // 2e-3..5e-3 error in the output, above the 2e-3 gate.  Q, K, V are exact bf16 inputs.
 //
@@ -38,9 +38,10 @@ constexpr int TC_BR = 128;           // query rows per block (TMEM lanes)
 constexpr int TC_BC = 64;            // keys per block
 constexpr int TC_NST = 4;            // K/V ring stages
 constexpr int TC_COMPUTE = 256;      // compute threads (warps 0..7)
-constexpr int TC_THREADS = 320;      // + TMA warp + MMA warp
+constexpr int TC_THREADS = 352;      // + TMA warp + two MMA warps
 constexpr int TC_TMEM_COLS = 512;
-constexpr int TC_ACC_COL = 256;      // ACC columns [256, 320)
+constexpr int TC_NBUF = 3;           // S/A/U buffers in TMEM (128 columns each)
+constexpr int TC_ACC_COL = TC_NBUF * 128;   // ACC columns [384, 448)
 
 enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4 };
 
@@ -61,7 +62,7 @@ constexpr int SM_ALLOC = SM_TOTAL + 1024;                // slack for manual 102
 // mbarrier indices
 enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST, B_VFULL = B_KVEMPTY + TC_NST,
        B_SAFULL = B_VFULL + TC_NST,
-       B_UFULL = B_SAFULL + 2, B_BUFFREE = B_UFULL + 2, B_ACCFULL = B_BUFFREE + 2, B_CTL = B_ACCFULL + 1,
+       B_UFULL = B_SAFULL + TC_NBUF, B_BUFFREE = B_UFULL + TC_NBUF, B_ACCFULL = B_BUFFREE + TC_NBUF, B_CTL = B_ACCFULL + 1,
        B_COUNT = B_CTL + 1 };
 static_assert(B_COUNT * 8 <= 256, "barrier area too small");
 
@@ -133,6 +134,16 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(
 #define TC_ACC(slot, var)
 #endif
 
+// Optional event trace of one block for tuning (-DLLA_TC_TRACE; (tag, block, clock) triples in prm.dbg).
+#ifdef LLA_TC_TRACE
+// each traced thread appends to its own region (role r: entries [r*4000, (r+1)*4000)), no atomics
+#define TC_EV_DECL(role) unsigned long long* ev_p_ = (prm.dbg && blockIdx.x == 0 && blockIdx.y == gridDim.y - 1 - LLA_TC_TRACE) ? prm.dbg + 1 + 3ull * 4000 * (role) : nullptr; int ev_n_ = 0
+#define TC_EV(tag, c) do { if (ev_p_ && ev_n_ < 4000) { ev_p_[3 * ev_n_] = (tag); ev_p_[3 * ev_n_ + 1] = (unsigned long long)(c); ev_p_[3 * ev_n_ + 2] = (unsigned long long)clock64(); ++ev_n_; } } while (0)
+#else
+#define TC_EV_DECL(role)
+#define TC_EV(tag, c)
+#endif
+
 struct TcParams {
     unsigned long long* dbg;
     int n, causal, head_rows, max_iters, first_tile;
@@ -175,7 +186,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mbar_init(bar(B_KVEMPTY + s), 1);
             mbar_init(bar(B_VFULL + s), 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < TC_NBUF; ++b) {
             mbar_init(bar(B_SAFULL + b), 1);
             mbar_init(bar(B_UFULL + b), TC_COMPUTE / 2);
             mbar_init(bar(B_BUFFREE + b), 1);
@@ -244,14 +255,22 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
     } else if (warp == 9) {
-        // ================================ MMA issuer ================================
-        // All 32 lanes run this loop convergently; the MMAs and commits are predicated on one lane.
+        // ================================ MMA issuer 1: S = Q K^T, A = P K^T ================================
+        // All 32 lanes run the loop convergently; the MMAs and commits are predicated on one lane.
+        // tcgen05.mma issue is throttled to the execution rate, so the time an issuing warp spends
+        // in barrier waits is tensor-pipe idle time: two warps (this one and warp 10) feed the pipe
+        // and each one's waits hide behind the other's instructions.
+        TC_EV_DECL(0);
         const uint32_t el = elect_one();
+        // broadcast through a shuffle so the compiler treats these as warp-uniform values and keeps
+        // the MMA operands in uniform registers (otherwise every operand is moved there one by one)
+        const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
+        const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
         bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
-        const uint64_t qdesc = make_desc(sbase + SM_Q);
-        const uint64_t phdesc = make_desc(sbase + SM_PHI);
-        const uint64_t pldesc = make_desc(sbase + SM_PLO);
-        uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it & 1)
+        const uint64_t qdesc = make_desc(sb_u + SM_Q);
+        const uint64_t phdesc = make_desc(sb_u + SM_PHI);
+        const uint64_t pldesc = make_desc(sb_u + SM_PLO);
+        uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it % NBUF)
         for (uint32_t sweep = 0; ok; ++sweep) {
             TC_T0(t_c);
             if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
@@ -259,70 +278,86 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const int kind = misc[1];
             if (kind == SW_DONE) break;
             tc_fence_after();
-            const uint32_t it0 = it;
-            for (int c = 0; c <= nblk && ok; ++c) {
-                if (c < nblk) {
-                    const uint32_t g = it0 + c, s = g % TC_NST, b = g & 1;
-                    TC_T0(t_k);
-                    if (!mbar_wait(bar(B_KVFULL + s), (g / TC_NST) & 1, abort_flag)) { ok = false; break; }
-                    if (lane == 0) TC_ACC(8, t_k);
-                    TC_T0(t_b);
-                    if (!mbar_wait(bar(B_BUFFREE + b), ((g >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                    if (lane == 0) TC_ACC(9, t_b);
-                    tc_fence_after();
-                    const uint64_t kdesc = make_desc(sbase + SM_KV + s * 16384);
-                    const uint32_t s_tm = tmem + b * 128, a_tm = s_tm + 64;
-                    mma_ss_k64(el, s_tm, qdesc, kdesc, IDESC_SS, 0);
-                    if (kind == SW_CG || kind == SW_OUT) {
-                        mma_ss_k64(el, a_tm, phdesc, kdesc, IDESC_SS, 0);
-                        mma_ss_k64(el, a_tm, pldesc, kdesc, IDESC_SS, 1);
-                    }
-                    tc_commit_el(el, bar(B_SAFULL + b));
+            for (int c = 0; c < nblk && ok; ++c, ++it) {
+                const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
+                TC_T0(t_k);
+                if (!mbar_wait(bar(B_KVFULL + s), (it / TC_NST) & 1, abort_flag)) { ok = false; break; }
+                if (lane == 0) TC_ACC(8, t_k);
+                TC_T0(t_b);
+                if (!mbar_wait(bar(B_BUFFREE + b), (bu & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (lane == 0) TC_ACC(9, t_b);
+                tc_fence_after();
+                const uint64_t kdesc = make_desc(sb_u + SM_KV + s * 16384);
+                const uint32_t s_tm = tm_u + b * 128, a_tm = s_tm + 64;
+                mma_ss_k64(el, s_tm, qdesc, kdesc, IDESC_SS, 0);
+                if (kind == SW_CG || kind == SW_OUT) {
+                    mma_ss_k64(el, a_tm, phdesc, kdesc, IDESC_SS, 0);
+                    mma_ss_k64(el, a_tm, pldesc, kdesc, IDESC_SS, 1);
                 }
-                if (c >= 1) {
-                    const uint32_t g = it0 + c - 1, s = g % TC_NST, b = g & 1;
-                    TC_T0(t_u);
-                    if (!mbar_wait(bar(B_UFULL + b), (g >> 1) & 1, abort_flag)) { ok = false; break; }
-                    if (lane == 0) TC_ACC(10, t_u);
-                    tc_fence_after();
-                    if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), ((c - 1) / TC_NST) & 1, abort_flag)) { ok = false; break; }
-                    if (kind != SW_MAX) {
-                        const uint32_t bsm = sbase + SM_KV + s * 16384 + (kind == SW_OUT ? 8192 : 0);
-                        mma_ts_hilo_k64(el, tmem + TC_ACC_COL, tmem + b * 128, make_desc(bsm), IDESC_TS, c > 1);
-                        tc_commit_el(el, bar(B_KVEMPTY + s));
-                        tc_commit_el(el, bar(B_BUFFREE + b));
-                        if (c == nblk) tc_commit_el(el, bar(B_ACCFULL));
-                    } else if (el) {
-                        mbar_arrive(bar(B_KVEMPTY + s));
-                        mbar_arrive(bar(B_BUFFREE + b));
-                    }
+                tc_commit_el(el, bar(B_SAFULL + b));
+                if (lane == 0) TC_EV(11, it);
+            }
+        }
+    } else if (warp == 10) {
+        // ================================ MMA issuer 2: ACC += U B ================================
+        TC_EV_DECL(1);
+        const uint32_t el = elect_one();
+        const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
+        const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
+        bool ok = true;
+        uint32_t it = 0;
+        for (uint32_t sweep = 0; ok; ++sweep) {
+            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+            const int kind = misc[1];
+            if (kind == SW_DONE) break;
+            for (int c = 0; c < nblk && ok; ++c, ++it) {
+                const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
+                TC_T0(t_u);
+                if (!mbar_wait(bar(B_UFULL + b), bu & 1, abort_flag)) { ok = false; break; }
+                if (lane == 0) TC_ACC(10, t_u);
+                if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), (c / TC_NST) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                if (lane == 0) TC_EV(20, it);
+                if (kind != SW_MAX) {
+                    const uint32_t bsm = sb_u + SM_KV + s * 16384 + (kind == SW_OUT ? 8192 : 0);
+                    mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm), IDESC_TS, c > 0);
+                    tc_commit_el(el, bar(B_KVEMPTY + s));
+                    tc_commit_el(el, bar(B_BUFFREE + b));
+                    if (c == nblk - 1) tc_commit_el(el, bar(B_ACCFULL));
+                    if (lane == 0) TC_EV(21, it);
+                } else if (el) {
+                    mbar_arrive(bar(B_KVEMPTY + s));
+                    mbar_arrive(bar(B_BUFFREE + b));
                 }
             }
-            it = it0 + nblk;
         }
     } else {
         // ================================ compute warps ================================
         TC_T0(t_all);
         const int quad = warp & 3, half = warp >> 2;
+        TC_EV_DECL(2 + half);
         const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
         const int row = r0 + lrow;
         const int L = prm.causal ? row + 1 : n;
         const bool row_ok = row < n && L >= prm.head_rows;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const int c0 = half * 32;                          // first column / first key (inside a block) owned
+        // The two threads of a row sit in warps w and w+4; only those two warps need to meet, so
+        // each lane quadrant has its own 64-thread named barrier (ids 2..5).
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + quad) : "memory"); };
         int red_sel = 0;
         auto pair_sum = [&](float v) {
             float* buf = red + red_sel * 256;
             red_sel ^= 1;
             buf[half * 128 + lrow] = v;
-            named_sync_compute();
+            pair_sync();
             return buf[lrow] + buf[128 + lrow];
         };
         auto pair_max = [&](float v) {
             float* buf = red + red_sel * 256;
             red_sel ^= 1;
             buf[half * 128 + lrow] = v;
-            named_sync_compute();
+            pair_sync();
             return fmaxf(buf[lrow], buf[128 + lrow]);
         };
         int flag_sel = 0;
@@ -373,9 +408,11 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             uint64_t part2 = pk2(0.f, 0.f);
             for (int c = 0; c < nblk; ++c, ++blk) {
                 if ((int)(blk & 1) != half) continue;
-                const uint32_t b = blk & 1;
+                const uint32_t b = blk % TC_NBUF;
                 TC_T0(t_w);
-                if (!mbar_wait(bar(B_SAFULL + b), (blk >> 1) & 1, abort_flag)) { ok = false; return part; }
+                if (lane == 0 && quad == 0) TC_EV(30 + half, blk);
+                if (!mbar_wait(bar(B_SAFULL + b), (blk / TC_NBUF) & 1, abort_flag)) { ok = false; return part; }
+                if (lane == 0 && quad == 0) TC_EV(32 + half, blk);
                 if (tid == 0) TC_ACC(0, t_w);
                 tc_fence_after();
 #pragma unroll 1
@@ -397,6 +434,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         uint32_t pk[32];
 #pragma unroll
                         for (int e2 = 0; e2 < 16; ++e2) {
+#ifdef LLA_EXP_NO_MATH
+                            pk[e2] = sv[2 * e2]; pk[16 + e2] = sv[2 * e2 + 1];
+                            continue;
+#endif
                             const uint64_t t2 = fma2(pk2(__uint_as_float(sv[2 * e2]), __uint_as_float(sv[2 * e2 + 1])), c1c1, nmx);
                             float t0, t1;
                             upk2(t2, t0, t1);
@@ -431,6 +472,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (kind != SW_MAX) tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(B_UFULL + b));
+                if (lane == 0 && quad == 0) TC_EV(34 + half, blk);
             }
             if (kind != SW_MAX) {
                 float p0, p1;
@@ -510,7 +552,11 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // ---- conjugate gradients (Algorithm 2) ----
         for (int t = 0; ok && t < prm.max_iters; ++t) {
             active = active && rr > stop;
+#ifdef LLA_EXP_FIXED
+            (void)group_any(active);     // tuning builds: always run max_iters sweeps
+#else
             if (!group_any(active)) break;
+#endif
             start_sweep(SW_CG);
             sweep(SW_CG);
             float ap[32];
@@ -641,7 +687,7 @@ int launch_t(const ForwardArgs& a) {
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     prm.dbg = nullptr;
-#ifdef LLA_TC_TIMING
+#if defined(LLA_TC_TIMING) || defined(LLA_TC_TRACE)
     prm.dbg = (unsigned long long*)a.workspace;   // tuning builds only: caller passes a zeroed buffer
 #endif
     auto kern = forward_tc_kernel<TOut>;
