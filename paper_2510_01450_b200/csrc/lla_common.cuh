@@ -129,35 +129,46 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
     const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
     bool ok = true;
     __syncthreads();
-    // After step c, column c holds L[r][c] * D_c (left unscaled) and the diagonal holds D_c.
-    // Warp ny-1 also carries the right-hand side as row D.
-    for (int c = 0; c < D - 1; ++c) {
-        const double piv = S[c * lds + c];
-        if (!(piv > 0.0)) ok = false;
-        const double inv = fast_rcp(piv);
-        for (int rb = c + 1 + ty; rb < D; rb += 4 * ny) {
-            // four rows of this warp at a time for instruction-level parallelism
-            double l[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int r = rb + u * ny;
-                l[u] = r < D ? S[r * lds + c] * inv : 0.0;
+    // Blocked right-looking LDL^T, panels of NB columns.  After a column is eliminated it holds
+    // L[r][c] * D_c (left unscaled) and the diagonal holds D_c.  The right-hand side is carried as
+    // row index D.  Per panel: (a) eliminate inside the panel, one thread per row; (b) one rank-NB
+    // update of everything to the right (4 multiply-adds per element loaded and stored).
+    constexpr int NB = 8;
+    static_assert(D % NB == 0, "head size must be a multiple of the panel width");
+    for (int c0 = 0; c0 < D; c0 += NB) {
+        for (int k = 0; k < NB; ++k) {
+            const int c = c0 + k;
+            const double piv = S[c * lds + c];
+            if (!(piv > 0.0)) ok = false;
+            const double inv = fast_rcp(piv);
+            for (int r = c + 1 + tid; r <= D; r += nt) {
+                double* rowp = r < D ? S + r * lds : rhs;
+                const double l = rowp[c] * inv;
+                for (int c2 = c + 1; c2 < c0 + NB; ++c2)
+                    if (r == D || c2 <= r) rowp[c2] -= l * S[c2 * lds + c];
             }
-            const int rmax = min(D - 1, rb + 3 * ny);
-            for (int c2 = c + 1 + tx; c2 <= rmax; c2 += 32) {
-                const double sc = S[c2 * lds + c];
+            __syncthreads();
+        }
+        if (c0 + NB < D) {
+            double dinv[NB];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int r = rb + u * ny;
-                    if (r < D && c2 <= r) S[r * lds + c2] -= l[u] * sc;
+            for (int k = 0; k < NB; ++k) dinv[k] = fast_rcp(S[(c0 + k) * lds + c0 + k]);
+            for (int r = c0 + NB + ty; r <= D; r += ny) {
+                double* rowp = r < D ? S + r * lds : rhs;
+                double ls[NB];
+#pragma unroll
+                for (int k = 0; k < NB; ++k) ls[k] = rowp[c0 + k] * dinv[k];
+                const int cmax = r < D ? r : D - 1;
+                for (int c2 = c0 + NB + tx; c2 <= cmax; c2 += 32) {
+                    const double* u = S + c2 * lds + c0;
+                    double acc = 0.0;
+#pragma unroll
+                    for (int k = 0; k < NB; ++k) acc += ls[k] * u[k];
+                    rowp[c2] -= acc;
                 }
             }
+            __syncthreads();
         }
-        if (ty == ny - 1) {
-            const double lr = rhs[c] * inv;
-            for (int c2 = c + 1 + tx; c2 < D; c2 += 32) rhs[c2] -= lr * S[c2 * lds + c];
-        }
-        __syncthreads();
     }
     if (!(S[(D - 1) * lds + (D - 1)] > 0.0)) ok = false;
     // rhs now holds y with L y = b.  Backward: x_r = (y_r - sum_{t>r} S[t][r] x_t) / D_r.
