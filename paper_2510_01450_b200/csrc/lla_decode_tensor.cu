@@ -275,16 +275,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const float a = w * kf[8 * i + 2 * e], bq = w * kf[8 * i + 2 * e + 1];
-                    hi[e] = pack_bf16(bq, a);
-                    lo[e] = pack_bf16(bq - __uint_as_float(hi[e] & 0xFFFF0000u), a - __uint_as_float(hi[e] << 16));
+                    hi[e] = split_bf16x2(a, bq, lo[e]);
                 }
                 const uint32_t off = (4 * h + i) * 1024 + rowoff;          // column block 4h+i
                 *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
             {   // column blocks 8 (ones column first) and 9 (zero padding)
-                const uint32_t whi = pack_bf16(0.f, w);
-                const uint32_t wlo = pack_bf16(0.f, w - __uint_as_float(whi << 16));
+                uint32_t wlo;
+                const uint32_t whi = split_bf16x2(w, 0.f, wlo);
                 const uint32_t off = (8 + h) * 1024 + rowoff;
                 *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
                 *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);

@@ -379,10 +379,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 uint32_t hi[4], lo[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float a = vec[ch * 8 + 2 * e], b = vec[ch * 8 + 2 * e + 1];
-                    hi[e] = pack_bf16(b, a);
-                    const float ra = a - __uint_as_float(hi[e] << 16), rb = b - __uint_as_float(hi[e] & 0xFFFF0000u);
-                    lo[e] = pack_bf16(rb, ra);
+                    hi[e] = split_bf16x2(vec[ch * 8 + 2 * e], vec[ch * 8 + 2 * e + 1], lo[e]);
                 }
                 const uint32_t off = swz(lrow, half * 4 + ch);
                 *reinterpret_cast<uint4*>(smem + SM_PHI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -455,13 +452,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             }
                             if (kind != SW_CG) part2 = add2(part2, u2);
                             // 16 keys per k-step: 8 columns of hi, then 8 columns of lo
-                            const uint32_t hi = pack_bf16(u1, u0);
-                            const uint64_t res = sub2(u2, pk2(__uint_as_float(hi << 16), __uint_as_float(hi & 0xFFFF0000u)));
-                            float ra, rb;
-                            upk2(res, ra, rb);
                             const int ks = e2 >> 3, e = e2 & 7;
-                            pk[ks * 16 + e] = hi;
-                            pk[ks * 16 + 8 + e] = pack_bf16(rb, ra);
+                            pk[ks * 16 + e] = split_bf16x2(u0, u1, pk[ks * 16 + 8 + e]);
                         }
                         if (tid == 0) TC_ACC(2, t_m);
                         TC_T0(t_s);

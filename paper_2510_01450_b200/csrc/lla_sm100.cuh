@@ -130,6 +130,17 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { u
 __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+// Split two fp32 values into bf16 hi + lo pairs without touching the conversion unit (which shares
+// the transcendental pipe with exp2): hi is the value truncated to its top 16 bits, lo the
+// truncated exact remainder, so hi + lo keeps 16 mantissa bits.  Returns the packed hi pair and
+// writes the packed lo pair; element `a` goes to the low half-word.
+__device__ __forceinline__ uint32_t split_bf16x2(float a, float b, uint32_t& lo) {
+    const uint32_t ua = __float_as_uint(a), ub = __float_as_uint(b);
+    const uint32_t hi = __byte_perm(ua, ub, 0x7632);
+    const float ra = a - __uint_as_float(ua & 0xFFFF0000u), rb = b - __uint_as_float(ub & 0xFFFF0000u);
+    lo = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
+    return hi;
+}
 // {hi16: bf16(a), lo16: bf16(b)}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     uint32_t r;
