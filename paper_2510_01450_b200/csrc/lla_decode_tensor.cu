@@ -39,7 +39,7 @@ constexpr int SMD_BAR = SMD_B + 4 * DT_BTILE;               // mbarriers
 constexpr int SMD_MISC = SMD_BAR + 128;                     // tmem base, abort, tile maxima
 constexpr int SMD_TOTAL = SMD_MISC + 128;
 // the epilogue reuses everything from offset 0: M (64 x 65 doubles), a, c, rhs (3 x 64 doubles), N (64 x 64 floats)
-constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 65;
+constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 65 + 8 * (128 + 24);
 constexpr int SMD_ALLOC = (SMD_TOTAL > SMD_FIN ? SMD_TOTAL : SMD_FIN) + 1024;
 
 enum { DB_KVFULL = 0, DB_KVEMPTY = DB_KVFULL + DT_NST, DB_BFULL = DB_KVEMPTY + DT_NST, DB_BFREE = DB_BFULL + 2,
@@ -87,6 +87,63 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
         "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, h3, %5, p;\n\t"
         "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, l3, %5, p;\n\t}"
         ::"r"(el), "r"(d), "l"(a), "l"(bhi), "l"(blo), "r"(IDESC_DEC), "r"(acc0) : "memory");
+}
+
+// Solve C x = b for an explicit symmetric positive-definite 64 x 64 matrix in shared memory (row
+// stride 65 doubles, both triangles filled) with conjugate gradients in double precision, run by
+// the 128 threads of warps 0..3 (two threads per row, 32 columns each).  A dense factorisation is a
+// chain of 64 dependent column steps, each with block barriers; here an iteration is one short
+// matrix-vector product and three 128-thread barriers, and the decode systems (>= 2d keys) need a
+// few dozen iterations.  x lands in xs[]; returns false if the residual did not reach 1e-11 |b|
+// within the iteration cap (the caller then falls back to the factorisation).  C is not modified.
+__device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, double* xs, double* pbuf, double* redbuf, int& iters) {
+    const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+    const int r = tid >> 1, hh = tid & 1;
+    auto sync128 = [&]() { asm volatile("bar.sync 2, 128;" ::: "memory"); };
+    auto block_sum = [&](double v, int slot) {       // v is counted once per row (hh == 0 lanes)
+        v = hh == 0 ? v : 0.0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (lane == 0) redbuf[slot * 4 + wp] = v;
+        sync128();
+        return (redbuf[slot * 4] + redbuf[slot * 4 + 1]) + (redbuf[slot * 4 + 2] + redbuf[slot * 4 + 3]);
+    };
+    double x = 0.0, res = b[r], pv = res;
+    if (hh == 0) pbuf[r] = pv;
+    double rr = block_sum(res * res, 0);
+    const double stop = rr * 1e-22;
+    bool done = !(rr > 0.0);
+    int slot = 1;
+    iters = 0;
+    for (int it = 0; it < 192 && !done; ++it) {
+        ++iters;
+        const double* crow = C + r * 65 + 32 * hh;
+        const double* pp = pbuf + 32 * hh;
+        double a0 = 0.0, a1 = 0.0;
+#pragma unroll 8
+        for (int c = 0; c < 32; c += 2) {
+            a0 += crow[c] * pp[c];
+            a1 += crow[c + 1] * pp[c + 1];
+        }
+        double ap = a0 + a1;
+        ap += __shfl_xor_sync(0xffffffffu, ap, 1);
+        const double pap = block_sum(pv * ap, slot);
+        slot = slot % 5 + 1;
+        if (!(pap > 0.0)) break;
+        const double alpha = rr / pap;
+        x += alpha * pv;
+        res -= alpha * ap;
+        const double rr2 = block_sum(res * res, slot);
+        slot = slot % 5 + 1;
+        pv = res + (rr2 / rr) * pv;
+        rr = rr2;
+        done = rr <= stop;
+        if (hh == 0) pbuf[r] = pv;
+        sync128();
+    }
+    if (hh == 0) xs[r] = x;
+    sync128();
+    return done;
 }
 
 __device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -195,18 +252,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             for (int i = 0; i < 4; ++i) load8(qp + 8 * i, qv + 8 * i);
         }
         bool ok = true;
-        for (int t = 0; t < ntile && ok; ++t) {
-            const uint32_t s = t % DT_NST, b = t & 1;
-            if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) { ok = false; break; }
+        const uint32_t rowoff = (jl >> 3) * 128 + (jl & 7) * 16;      // key group, row inside the core matrix
+        // Software pipeline over tiles: the shared-memory loads of tile t+1 are issued before the
+        // scale-and-store phase of tile t, and its score follows right after, so the two phases'
+        // latencies overlap.  stage_load fetches this lane's 32 features of key jl (swizzled 16-byte
+        // chunks 4h .. 4h+3) as raw bf16 pairs; stage_score turns them into kf[], the score and the weight.
+        uint4 raw[4];
+        float kf[32];
+        float w = 0.f;
+        auto stage_load = [&](int t) -> bool {
+            const uint32_t s = t % DT_NST;
+            if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) return false;
             uint8_t* ktile = smem + SMD_KV + s * 16384;
-            const int jglob = jbeg + t * DT_BK + jl;
-            const bool valid = jglob < jend;
-            // this lane's 32 features of key jl (swizzled 16-byte chunks 4h .. 4h+3)
-            float kf[32];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                raw[i] = *reinterpret_cast<const uint4*>(ktile + jl * 128 + (((4 * h + i) ^ (jl & 7)) << 4));
+            return true;
+        };
+        auto stage_score = [&](int t) -> bool {
+            const uint32_t s = t % DT_NST;
+            uint8_t* ktile = smem + SMD_KV + s * 16384;
+            const bool valid = jbeg + t * DT_BK + jl < jend;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint4 raw = *reinterpret_cast<const uint4*>(ktile + jl * 128 + (((4 * h + i) ^ (jl & 7)) << 4));
-                const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
+                const uint32_t wds[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     kf[8 * i + 2 * e] = __uint_as_float(wds[e] << 16);
@@ -242,9 +311,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (t == 0) {
                 m_ref = tile_max;
             } else if (tile_max > m_ref + 40.f) {
-                // rare: rescale the accumulator (all MMAs of earlier tiles must have finished)
+                // rare: rescale the accumulator (all MMAs of earlier tiles must have finished; this
+                // thread's B rows of tile t-1 were handed over before this call)
                 const float f = ex2f(m_ref - tile_max);
-                if (!mbar_wait(bar(DB_BFREE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bar(DB_BFREE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
 #pragma unroll 1
@@ -262,34 +332,45 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 m_ref = tile_max;
                 named_sync_128();
             }
-            const float w = valid ? ex2f(s2 - m_ref) : 0.f;
+            w = valid ? ex2f(s2 - m_ref) : 0.f;
             if (h == 0) omega += w;
-            // B rows: w * [k | 1] as bf16 hi + lo.  Wait until the MMA of tile t-2 has released the buffer.
+            return true;
+        };
+        if (ntile > 0) ok = stage_load(0) && stage_score(0);
+        for (int t = 0; t < ntile && ok; ++t) {
+            const uint32_t b = t & 1;
+            const bool more = t + 1 < ntile;
+            // B rows of tile t: w * [k | 1] as bf16 hi + lo, computed into registers first
+            uint32_t hi[16], lo[16];
+            const uint64_t ww = pk2(w, w);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                float a, bq;
+                upk2(mul2(ww, pk2(kf[2 * e], kf[2 * e + 1])), a, bq);
+                hi[e] = split_bf16x2(a, bq, lo[e]);
+            }
+            uint32_t wlo;
+            const uint32_t whi = split_bf16x2(w, 0.f, wlo);
+            // loads of the next tile go out now; they land while the stores below are issued
+            if (more && !stage_load(t + 1)) { ok = false; break; }
+            // wait until the MMA of tile t-2 has released this B buffer
             if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
             uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
             uint8_t* blo = bhi + DT_BTILE;
-            const uint32_t rowoff = (jl >> 3) * 128 + (jl & 7) * 16;      // key group, row inside the core matrix
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                uint32_t hi[4], lo[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float a = w * kf[8 * i + 2 * e], bq = w * kf[8 * i + 2 * e + 1];
-                    hi[e] = split_bf16x2(a, bq, lo[e]);
-                }
                 const uint32_t off = (4 * h + i) * 1024 + rowoff;          // column block 4h+i
-                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+                *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
             }
             {   // column blocks 8 (ones column first) and 9 (zero padding)
-                uint32_t wlo;
-                const uint32_t whi = split_bf16x2(w, 0.f, wlo);
                 const uint32_t off = (8 + h) * 1024 + rowoff;
                 *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
                 *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
             }
             fence_proxy_async();
             mbar_arrive(bar(DB_BFULL + b));
+            if (more && !stage_score(t + 1)) { ok = false; break; }
         }
         // total weight of this part
         if (ok) {
@@ -374,15 +455,37 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     if (warp < 4) {
         if (tid < 64) {
-            for (int e = 0; e <= tid; ++e)
-                Md[tid * 65 + e] = (double)dv[e] * inv - av[tid] * av[e] + (e == tid ? ridge : 0.0);
-            rhs[tid] = (double)to_f32(q[(size_t)bh * DT_D + tid]) - av[tid];
+            // full row of the centred matrix (M is symmetric up to fp32 rounding of the accumulators)
+            const double ar = av[tid];
+#pragma unroll
+            for (int e = 0; e < 64; ++e) Md[tid * 65 + e] = (double)dv[e] * inv - ar * av[e];
+            Md[tid * 65 + tid] += ridge;
+            rhs[tid] = (double)to_f32(q[(size_t)bh * DT_D + tid]) - ar;
         } else {
 #pragma unroll
             for (int e = 0; e < 64; ++e) Nd[(tid - 64) * 65 + e] = dv[e];
         }
     }
-    const bool solved = block_ldlt_solve<64>(Md, 65, rhs);
+    __syncthreads();
+    // conjugate gradients first (fast); the blocked factorisation only if they do not converge
+    double* xs = reinterpret_cast<double*>(Nd + 64 * 65);      // x, p and reduction scratch after N
+    __shared__ int s_cg_ok;
+    if (warp < 4) {
+        int cg_its = 0;
+        const bool okc = cg_solve_64(Md, rhs, xs, xs + 64, xs + 128, cg_its);
+        if (tid == 0) {
+            s_cg_ok = okc ? 1 : 0;
+            if (prm.status) atomicAdd(prm.status + LLA_STATUS_ITER_SUM, cg_its);
+        }
+    }
+    __syncthreads();
+    bool solved = true;
+    if (s_cg_ok) {
+        if (tid < 64) rhs[tid] = xs[tid];
+        __syncthreads();
+    } else {
+        solved = block_ldlt_solve<64>(Md, 65, rhs);
+    }
     if (tid < 64) {
         double o = cv[tid];
         for (int f = 0; f < 64; ++f) o += ((double)Nd[tid * 65 + f] * inv - cv[tid] * av[f]) * rhs[f];
