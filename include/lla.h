@@ -51,7 +51,7 @@ typedef enum lla_dtype { LLA_BF16 = 0, LLA_F32 = 1 } lla_dtype;
 typedef enum lla_impl {
     LLA_IMPL_AUTO = 0,   /* tensor-core kernel where compiled for the shape, else SIMT */
     LLA_IMPL_SIMT = 1,   /* fp32 CUDA-core kernel (every supported shape and dtype) */
-    LLA_IMPL_TENSOR = 2  /* tcgen05/TMEM kernel (bf16 inputs, d = dv = 64) */
+    LLA_IMPL_TENSOR = 2  /* tcgen05/TMEM kernel (bf16 inputs, d = dv = 64 or 128) */
 } lla_impl;
 
 /* Row groups for lla_forward_params.phases. */
@@ -218,7 +218,10 @@ int lla_decode_noalloc(const void *q, const void *kcache, const void *vcache, co
                        void *out, int B, int H, int Lmax, int d, int dv, int in_dtype,
                        int out_dtype, float scale, float lambda, int splits, void *stream);
 
-/* Scratch bytes lla_forward_ex needs for this problem (0 when none). Host-only arithmetic. */
+/* Scratch bytes lla_forward_ex needs for this problem (0 when none). Host-only arithmetic.
+ * The d = 128 tensor-core kernel additionally keeps one library-owned device buffer per GPU
+ * (2 x SM count x 192 KiB, allocated with cudaMalloc by the first such call and reused by all
+ * later ones; blocks address it by SM id, so concurrent calls may share it). */
 size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl);
 
 /* Scratch bytes lla_decode_ex needs for this problem and split count (0 when splits <= 1). */

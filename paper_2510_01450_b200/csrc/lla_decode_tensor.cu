@@ -23,6 +23,9 @@ namespace {
 
 using namespace sm100;
 
+#ifndef LLA_CG_CAP
+#define LLA_CG_CAP 192
+#endif
 constexpr int DT_D = 64;
 constexpr int DT_BK = 64;             // keys per tile
 constexpr int DT_NST = 4;             // K/V ring stages
@@ -115,7 +118,7 @@ __device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, do
     bool done = !(rr > 0.0);
     int slot = 1;
     iters = 0;
-    for (int it = 0; it < 192 && !done; ++it) {
+    for (int it = 0; it < LLA_CG_CAP && !done; ++it) {
         ++iters;
         const double* crow = C + r * 65 + 32 * hh;
         const double* pp = pbuf + 32 * hh;

@@ -1,4 +1,4 @@
-// LLA forward on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 inputs, d = dv = 64.
+// LLA forward on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 inputs, d = dv = 64 or 128.
 //
 // One thread block per (batch*head, 128-row query tile).  The three loops of Algorithm 1 and the
 // per-iteration loop of Algorithm 2 are all "sweeps" over 64-key blocks with the same skeleton:
@@ -16,8 +16,11 @@
 //   MMA 2 (TS)     ACC += U_hi B + U_lo B, A operand straight from TMEM, B = the same K block read
 //                  MN-major (or the V block in the output sweep)
 //
-// S/A/U cycle through three TMEM buffers (3 x 128 columns) and ACC takes 64 more; K/V blocks go through a
-// 4-stage ring.  Roles: warps 0-7 compute (warp w owns TMEM lanes 32*(w%4).. and key half w/4 of each
+// S/A/U cycle through three TMEM buffers (3 x 128 columns) and ACC takes D more (all 512 columns for
+// D = 128); K/V blocks go through a 4-stage ring (3 stages for D = 128).  Operands wider than 64 columns
+// are held as 64-column sub-tiles so every tile keeps the 128-byte swizzled row.  For D = 128 the fp32
+// row vectors x, kbar and r do not fit in shared memory or registers next to the operand tiles; each
+// thread keeps its own entries in a global scratch slot owned by the SM (L2-resident, thread-private).  Roles: warps 0-7 compute (warp w owns TMEM lanes 32*(w%4).. and key half w/4 of each
 // block; two threads share a row and exchange partial sums through shared memory), warp 8 issues TMA,
 // warps 9 and 10 issue the two MMA streams.  Every on-the-fly MMA operand (P, y, U) is carried as a bf16 pair hi + lo so
 // the products keep ~16 mantissa bits: a single bf16 rounding of those operands would leave a
@@ -26,6 +29,8 @@
 // The mathematics is the centred form described in lla_forward_simt.cu (same CG, same freeze rule).
 // All waits on mbarriers are bounded; a wait that expires sets LLA_STATUS_TIMEOUT and the block
 // leaves through the common exit (TMEM is released there).
+#include <mutex>
+
 #include "lla_sm100.cuh"
 
 namespace lla {
@@ -33,35 +38,53 @@ namespace {
 
 using namespace sm100;
 
-constexpr int TC_D = 64;             // head size handled here
 constexpr int TC_BR = 128;           // query rows per block (TMEM lanes)
 constexpr int TC_BC = 64;            // keys per block
-constexpr int TC_NST = 4;            // K/V ring stages
 constexpr int TC_COMPUTE = 256;      // compute threads (warps 0..7)
 constexpr int TC_THREADS = 352;      // + TMA warp + two MMA warps
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_NBUF = 3;           // S/A/U buffers in TMEM (128 columns each)
-constexpr int TC_ACC_COL = TC_NBUF * 128;   // ACC columns [384, 448)
+constexpr int TC_ACC_COL = TC_NBUF * 128;   // ACC columns [384, 384 + D)
+constexpr int TC_NST_MAX = 4;
 
 enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4 };
 
-// shared-memory carve-up (bytes, from a 1024-byte aligned base)
-constexpr int SM_Q = 0;                                  // 128 x 64 bf16, swizzled            16384
-constexpr int SM_PHI = SM_Q + 16384;                     // P / y hi                            16384
-constexpr int SM_PLO = SM_PHI + 16384;                   // P / y lo                            16384
-constexpr int SM_KV = SM_PLO + 16384;                    // TC_NST x (K 8192 + V 8192)          65536
-constexpr int SM_X = SM_KV + TC_NST * 16384;             // x   fp32 [64][128]                  32768
-constexpr int SM_KBAR = SM_X + 32768;                    // kbar fp32 [64][128]                 32768
-constexpr int SM_RED = SM_KBAR + 32768;                  // pair reduction buffers 2 x 2 x 128   2048
-constexpr int SM_FLAGS = SM_RED + 2048;                  // 2 x 8 ints                             64
-constexpr int SM_BAR = SM_FLAGS + 64;                    // mbarriers (8 bytes each)              256
-constexpr int SM_MISC = SM_BAR + 256;                    // tmem base, ctl kind, abort              64
-constexpr int SM_TOTAL = SM_MISC + 64;
-constexpr int SM_ALLOC = SM_TOTAL + 1024;                // slack for manual 1024-byte alignment
+// Shared-memory carve-up (bytes, from a 1024-byte aligned base), per head size D (64 or 128).
+// Operand tiles are stored as D/64 sub-tiles of 64 columns (128-byte rows, 128B swizzle) one after
+// the other.  For D = 64 the row vectors x and kbar live in shared memory as fp32 [D][128]; for
+// D = 128 there is no room for them, so x, kbar and r live in an L2-resident global scratch slot
+// owned by the SM (one block per SM at a time) and the ring has three stages.
+template <int D>
+struct TcCfg {
+    static constexpr int KSUB = D / 64;                         // 64-column sub-tiles per operand row
+    static constexpr int NCOL = D / 2;                          // row-vector columns per thread
+    static constexpr int NST = D == 64 ? 4 : 3;                 // K/V ring stages
+    static constexpr int QSUB_BYTES = TC_BR * 128;              // one sub-tile of a 128-row operand
+    static constexpr int KSUB_BYTES = TC_BC * 128;              // one sub-tile of a 64-key block
+    static constexpr int OPER_BYTES = KSUB * QSUB_BYTES;        // Q, P_hi, P_lo
+    static constexpr int KBLK_BYTES = KSUB * KSUB_BYTES;        // K block (V block follows it)
+    static constexpr int STAGE_BYTES = 2 * KBLK_BYTES;
+    static constexpr bool STATE_IN_SMEM = D == 64;
+    static constexpr int SM_Q = 0;
+    static constexpr int SM_PHI = SM_Q + OPER_BYTES;
+    static constexpr int SM_PLO = SM_PHI + OPER_BYTES;
+    static constexpr int SM_KV = SM_PLO + OPER_BYTES;
+    static constexpr int SM_X = SM_KV + NST * STAGE_BYTES;                        // fp32 [D][128] (D = 64 only)
+    static constexpr int SM_KBAR = SM_X + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);
+    static constexpr int SM_RED = SM_KBAR + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);  // pair reductions 2 x 2 x 128 floats
+    static constexpr int SM_FLAGS = SM_RED + 2048;                                // 2 x 8 ints
+    static constexpr int SM_BAR = SM_FLAGS + 64;                                  // mbarriers
+    static constexpr int SM_MISC = SM_BAR + 256;                                  // tmem base, ctl kind, abort
+    static constexpr int SM_TOTAL = SM_MISC + 64;
+    static constexpr int SM_ALLOC = SM_TOTAL + 1024;                              // slack for 1024-byte alignment
+    static constexpr uint32_t IDESC_TS = sm100::make_idesc(TC_BR, D, 0, 1);   // ACC: A from TMEM, B MN-major, N = D
+    static constexpr size_t SCRATCH_FLOATS_PER_SM = STATE_IN_SMEM ? 0 : 3 * (size_t)D * TC_BR;   // x, kbar, r
+};
+static_assert(TcCfg<64>::SM_ALLOC <= 227 * 1024 && TcCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
 
 // mbarrier indices
-enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST, B_VFULL = B_KVEMPTY + TC_NST,
-       B_SAFULL = B_VFULL + TC_NST,
+enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST_MAX, B_VFULL = B_KVEMPTY + TC_NST_MAX,
+       B_SAFULL = B_VFULL + TC_NST_MAX,
        B_UFULL = B_SAFULL + TC_NBUF, B_BUFFREE = B_UFULL + TC_NBUF, B_ACCFULL = B_BUFFREE + TC_NBUF, B_CTL = B_ACCFULL + 1,
        B_COUNT = B_CTL + 1 };
 static_assert(B_COUNT * 8 <= 256, "barrier area too small");
@@ -109,18 +132,18 @@ __device__ __forceinline__ void mma_ts_hilo_k64(uint32_t el, uint32_t d, uint32_
 //   K-major:  rows of 128 bytes, 8-row groups 1024 bytes apart; a 16-element K step is +32 bytes.
 //   MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements; 8-row groups
 //             1024 bytes apart; a 16-element K step is +2048 bytes.
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_bytes = 16) {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);         // start address
-    d |= (uint64_t)1 << 16;                              // leading byte offset (unused with swizzle)
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;    // leading byte offset: distance between the 64-wide
+                                                         // column groups of an MN-major operand wider than 64
     d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset
     d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
     d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
     return d;
 }
 
-constexpr uint32_t IDESC_SS = make_idesc(TC_BR, TC_BC, 0, 0);   // S/A: A, B K-major
-constexpr uint32_t IDESC_TS = make_idesc(TC_BR, TC_D, 0, 1);    // ACC: A from TMEM, B MN-major
+constexpr uint32_t IDESC_SS = make_idesc(TC_BR, TC_BC, 0, 0);   // S/A: A, B K-major; ACC uses make_idesc(128, D, 0, 1)
 
 // byte offset of the 16-byte chunk `chunk` (8 bf16) of row `row` in a swizzled 128 x 64 bf16 tile
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
@@ -152,21 +175,45 @@ struct TcParams {
     float* stats;
     int* iters;
     int* status;
+    float* scratch;      // D = 128: per-SM slots for x, kbar, r (TcCfg::SCRATCH_FLOATS_PER_SM each)
+    int scratch_slots;
 };
 
-template <typename TOut>
+template <int D, typename TOut>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, TOut* __restrict__ out, const TcParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    using Cfg = TcCfg<D>;
+    constexpr int TC_NST = Cfg::NST, NCOL = Cfg::NCOL, KSUB = Cfg::KSUB;
+    constexpr int SM_Q = Cfg::SM_Q, SM_PHI = Cfg::SM_PHI, SM_PLO = Cfg::SM_PLO, SM_KV = Cfg::SM_KV;
+    constexpr int SM_RED = Cfg::SM_RED, SM_FLAGS = Cfg::SM_FLAGS, SM_BAR = Cfg::SM_BAR, SM_MISC = Cfg::SM_MISC;
+    constexpr int STAGE = Cfg::STAGE_BYTES, KBLK = Cfg::KBLK_BYTES;
+    constexpr uint32_t IDESC_TS = Cfg::IDESC_TS;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bars = sbase + SM_BAR;
     auto bar = [&](int i) { return bars + 8u * i; };
     volatile int* misc = reinterpret_cast<volatile int*>(smem + SM_MISC);   // [0] tmem base, [1] kind, [2] abort
     volatile int* abort_flag = misc + 2;
-    float* xs = reinterpret_cast<float*>(smem + SM_X);
-    float* kbs = reinterpret_cast<float*>(smem + SM_KBAR);
+    // row-vector state: shared memory (D = 64) or this SM's slot of the global scratch (D = 128)
+    float* xs;
+    float* kbs;
+    float* rs = nullptr;
+    if constexpr (Cfg::STATE_IN_SMEM) {
+        xs = reinterpret_cast<float*>(smem + Cfg::SM_X);
+        kbs = reinterpret_cast<float*>(smem + Cfg::SM_KBAR);
+    } else {
+        uint32_t smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        if (smid >= (uint32_t)prm.scratch_slots) {     // never expected: SM ids are dense on this part
+            if (threadIdx.x == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+            return;
+        }
+        xs = prm.scratch + (size_t)smid * Cfg::SCRATCH_FLOATS_PER_SM;
+        kbs = xs + (size_t)D * TC_BR;
+        rs = kbs + (size_t)D * TC_BR;
+    }
     float* red = reinterpret_cast<float*>(smem + SM_RED);
     volatile int* flags = reinterpret_cast<volatile int*>(smem + SM_FLAGS);
 
@@ -214,22 +261,25 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // (every kind needs K).  V blocks are added, on their own barriers, once the output sweep
         // is announced.
         if (lane == 0) {
-            mbar_expect_tx(bar(B_QFULL), TC_BR * TC_D * 2);
-            tma_load_3d(sbase + SM_Q, &tmQ, bar(B_QFULL), 0, r0, bh);
+            mbar_expect_tx(bar(B_QFULL), Cfg::OPER_BYTES);
+            for (int sub = 0; sub < KSUB; ++sub)
+                tma_load_3d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, bh);
             uint32_t kit = 0;      // K blocks issued so far
             int pre = 0;           // blocks of the coming sweep already issued
             bool ok = true;
             auto issue_k = [&](int c) {
                 const uint32_t s = kit % TC_NST;
                 if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag)) { ok = false; return; }
-                mbar_expect_tx(bar(B_KVFULL + s), 8192);
-                tma_load_3d(sbase + SM_KV + s * 16384, &tmK, bar(B_KVFULL + s), 0, c * TC_BC, bh);
+                mbar_expect_tx(bar(B_KVFULL + s), KBLK);
+                for (int sub = 0; sub < KSUB; ++sub)
+                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, &tmK, bar(B_KVFULL + s), 64 * sub, c * TC_BC, bh);
                 ++kit;
             };
             auto issue_v = [&](int c, uint32_t g) {
                 const uint32_t s = g % TC_NST;
-                mbar_expect_tx(bar(B_VFULL + s), 8192);
-                tma_load_3d(sbase + SM_KV + s * 16384 + 8192, &tmV, bar(B_VFULL + s), 0, c * TC_BC, bh);
+                mbar_expect_tx(bar(B_VFULL + s), KBLK);
+                for (int sub = 0; sub < KSUB; ++sub)
+                    tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, c * TC_BC, bh);
             };
             for (uint32_t sweep = 0; ok; ++sweep) {
                 if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
@@ -287,12 +337,20 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!mbar_wait(bar(B_BUFFREE + b), (bu & 1) ^ 1, abort_flag)) { ok = false; break; }
                 if (lane == 0) TC_ACC(9, t_b);
                 tc_fence_after();
-                const uint64_t kdesc = make_desc(sb_u + SM_KV + s * 16384);
+                const uint64_t kdesc = make_desc(sb_u + SM_KV + s * STAGE);
                 const uint32_t s_tm = tm_u + b * 128, a_tm = s_tm + 64;
-                mma_ss_k64(el, s_tm, qdesc, kdesc, IDESC_SS, 0);
+                // contraction over D: one group of four 16-wide steps per 64-column sub-tile
+                // (sub-tiles are QSUB_BYTES / KSUB_BYTES apart: 1024 / 512 descriptor units)
+#pragma unroll
+                for (int sub = 0; sub < KSUB; ++sub)
+                    mma_ss_k64(el, s_tm, qdesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), IDESC_SS, sub > 0);
                 if (kind == SW_CG || kind == SW_OUT) {
-                    mma_ss_k64(el, a_tm, phdesc, kdesc, IDESC_SS, 0);
-                    mma_ss_k64(el, a_tm, pldesc, kdesc, IDESC_SS, 1);
+#pragma unroll
+                    for (int sub = 0; sub < KSUB; ++sub)
+                        mma_ss_k64(el, a_tm, phdesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), IDESC_SS, sub > 0);
+#pragma unroll
+                    for (int sub = 0; sub < KSUB; ++sub)
+                        mma_ss_k64(el, a_tm, pldesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), IDESC_SS, 1);
                 }
                 tc_commit_el(el, bar(B_SAFULL + b));
                 if (lane == 0) TC_EV(11, it);
@@ -319,8 +377,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tc_fence_after();
                 if (lane == 0) TC_EV(20, it);
                 if (kind != SW_MAX) {
-                    const uint32_t bsm = sb_u + SM_KV + s * 16384 + (kind == SW_OUT ? 8192 : 0);
-                    mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm), IDESC_TS, c > 0);
+                    const uint32_t bsm = sb_u + SM_KV + s * STAGE + (kind == SW_OUT ? KBLK : 0);
+                    // B = the K (or V) block read MN-major, N = D: 64-wide column groups are one sub-tile apart
+                    mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS, c > 0);
                     tc_commit_el(el, bar(B_KVEMPTY + s));
                     tc_commit_el(el, bar(B_BUFFREE + b));
                     if (c == nblk - 1) tc_commit_el(el, bar(B_ACCFULL));
@@ -341,7 +400,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int L = prm.causal ? row + 1 : n;
         const bool row_ok = row < n && L >= prm.head_rows;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        const int c0 = half * 32;                          // first column / first key (inside a block) owned
+        const int c0 = half * NCOL;                        // first row-vector column owned by this thread
+        // byte offset of this thread's chunk ch (8 columns) of row lrow inside a swizzled operand
+        auto oper_off = [&](int ch) {
+            const int col8 = half * (NCOL / 8) + ch;      // 8-column chunk index within the row
+            return (uint32_t)((col8 >> 3) * Cfg::QSUB_BYTES) + swz(lrow, col8 & 7);
+        };
         // The two threads of a row sit in warps w and w+4; only those two warps need to meet, so
         // each lane quadrant has its own 64-thread named barrier (ids 2..5).
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + quad) : "memory"); };
@@ -372,16 +436,16 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int i = 0; i < 8; ++i) r |= f[i];
             return r != 0;
         };
-        // store 32 fp32 values of this row as bf16 hi/lo into the swizzled operand tiles
+        // store this thread's NCOL fp32 values of the row as bf16 hi/lo into the swizzled operand tiles
         auto write_operand = [&](const float* vec) {
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int ch = 0; ch < NCOL / 8; ++ch) {
                 uint32_t hi[4], lo[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     hi[e] = split_bf16x2(vec[ch * 8 + 2 * e], vec[ch * 8 + 2 * e + 1], lo[e]);
                 }
-                const uint32_t off = swz(lrow, half * 4 + ch);
+                const uint32_t off = oper_off(ch);
                 *reinterpret_cast<uint4*>(smem + SM_PHI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<uint4*>(smem + SM_PLO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
@@ -473,7 +537,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             return part;
         };
-        // read this thread's 32 ACC columns after the sweep's last MMA
+        // read this thread's NCOL ACC columns after the sweep's last MMA
         uint32_t acc_uses = 0;
         auto read_acc = [&](float* dst) {
             TC_T0(t_a);
@@ -481,12 +545,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (tid == 0) TC_ACC(4, t_a);
             ++acc_uses;
             tc_fence_after();
-            uint32_t v[32];
-            tmem_ld32(tmem + lane_addr + TC_ACC_COL + c0, v);
-            tc_wait_ld();
-            tc_fence_before();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) dst[e] = __uint_as_float(v[e]);
+            for (int cb = 0; cb < NCOL; cb += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_addr + TC_ACC_COL + c0 + cb, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) dst[cb + e] = __uint_as_float(v[e]);
+            }
+            tc_fence_before();
         };
         auto start_sweep = [&](int kind) {
             if (tid == 0) misc[1] = kind;
@@ -494,7 +561,16 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mbar_arrive(bar(B_CTL));
         };
 
-        float r[32], p[32];
+        // residual r: registers for D = 64, the scratch slot for D = 128 (no registers to spare)
+        float r[Cfg::STATE_IN_SMEM ? NCOL : 1] = {}, p[NCOL];
+        auto r_get = [&](int e) -> float {
+            if constexpr (Cfg::STATE_IN_SMEM) return r[e];
+            else return rs[(c0 + e) * TC_BR + lrow];
+        };
+        auto r_set = [&](int e, float v) {
+            if constexpr (Cfg::STATE_IN_SMEM) r[e] = v;
+            else rs[(c0 + e) * TC_BR + lrow] = v;
+        };
         float rr = 0.f, stop = 0.f;
         int its = 0;
         bool active = false;
@@ -509,7 +585,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (ok) {
             start_sweep(SW_STATS);
             const float part = sweep(SW_STATS);
-            float acc[32];
+            float acc[NCOL];
             if (ok) read_acc(acc);
             if (ok) {
                 omega = pair_sum(part);
@@ -517,8 +593,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 ridge = prm.lambda * ex2f(-mx2) * inv_omega;
                 float rr_p = 0.f, ab_p = 0.f;
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    const uint4 qraw = *reinterpret_cast<const uint4*>(smem + SM_Q + swz(lrow, half * 4 + ch));
+                for (int ch = 0; ch < NCOL / 8; ++ch) {
+                    const uint4 qraw = *reinterpret_cast<const uint4*>(smem + SM_Q + oper_off(ch));
                     const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
@@ -528,7 +604,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         kbs[(c0 + col) * TC_BR + lrow] = kb;
                         xs[(c0 + col) * TC_BR + lrow] = 0.f;
                         const float bv = row_ok ? kb - qv : 0.f;
-                        r[col] = bv;
+                        r_set(col, bv);
                         p[col] = bv;
                         rr_p += bv * bv;
                         ab_p += kb * bv;
@@ -551,12 +627,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #endif
             start_sweep(SW_CG);
             sweep(SW_CG);
-            float ap[32];
+            float ap[NCOL];
             if (ok) read_acc(ap);
             if (!ok) break;
             float pap_p = 0.f;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
+            for (int e = 0; e < NCOL; ++e) {
                 ap[e] = fmaf(ap[e], inv_omega, ridge * p[e]);
                 pap_p += p[e] * ap[e];
             }
@@ -565,22 +641,24 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const float alpha = active ? rr / pap : 0.f;
             float rr2_p = 0.f;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
+            for (int e = 0; e < NCOL; ++e) {
                 xs[(c0 + e) * TC_BR + lrow] += alpha * p[e];
-                r[e] -= alpha * ap[e];
-                rr2_p += r[e] * r[e];
+                const float rn = r_get(e) - alpha * ap[e];
+                r_set(e, rn);
+                ap[e] = rn;                       // ap now holds the new residual
+                rr2_p += rn * rn;
             }
             const float rr2 = pair_sum(rr2_p);
             float ab_p = 0.f;
             if (active) {
                 const float beta = rr2 / rr;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) p[e] = fmaf(beta, p[e], r[e]);
+                for (int e = 0; e < NCOL; ++e) p[e] = fmaf(beta, p[e], ap[e]);
                 rr = rr2;
                 ++its;
             }
 #pragma unroll
-            for (int e = 0; e < 32; ++e) ab_p += kbs[(c0 + e) * TC_BR + lrow] * p[e];
+            for (int e = 0; e < NCOL; ++e) ab_p += kbs[(c0 + e) * TC_BR + lrow] * p[e];
             abar = pair_sum(ab_p);
             write_operand(p);
         }
@@ -588,11 +666,11 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // ---- output sweep ----
         float gfac = 1.f;
         if (ok) {
-            float y[32];
+            float y[NCOL];
             float yb_p = 0.f, g_p = 0.f;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                const uint4 qraw = *reinterpret_cast<const uint4*>(smem + SM_Q + swz(lrow, half * 4 + ch));
+            for (int ch = 0; ch < NCOL / 8; ++ch) {
+                const uint4 qraw = *reinterpret_cast<const uint4*>(smem + SM_Q + oper_off(ch));
                 const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -609,20 +687,20 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             write_operand(y);
             start_sweep(SW_OUT);
             const float part = sweep(SW_OUT);
-            float o[32];
+            float o[NCOL];
             if (ok) read_acc(o);
             if (ok) {
                 den = pair_sum(part);
                 if (row_ok) {
                     const float inv_den = 1.f / den;
                     const size_t rowi = (size_t)bh * n + row;
-                    TOut* orow = out + rowi * TC_D + c0;
+                    TOut* orow = out + rowi * D + c0;
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) store_out(orow + e, o[e] * inv_den);
+                    for (int e = 0; e < NCOL; ++e) store_out(orow + e, o[e] * inv_den);
                     if (prm.rho) {
                         const float ig = 1.f / gfac;
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) prm.rho[rowi * TC_D + c0 + e] = y[e] * ig;
+                        for (int e = 0; e < NCOL; ++e) prm.rho[rowi * D + c0 + e] = y[e] * ig;
                     }
                     if (half == 0) {
                         if (prm.stats) {
@@ -661,8 +739,31 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
-template <typename TOut>
+// Per-device scratch for the D = 128 kernel: one slot per SM id, shared by every launch on the device.
+// A block of this kernel fills an SM (shared memory), so two blocks never use one slot at a time,
+// whichever launches or streams they come from.
+float* scratch_for_device(size_t bytes) {
+    static std::mutex mu;
+    static float* ptr[64] = {};
+    static size_t have[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (have[dev] < bytes) {
+        if (ptr[dev]) cudaFree(ptr[dev]);
+        ptr[dev] = nullptr;
+        have[dev] = 0;
+        void* p = nullptr;
+        if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
+        ptr[dev] = static_cast<float*>(p);
+        have[dev] = bytes;
+    }
+    return ptr[dev];
+}
+
+template <int D, typename TOut>
 int launch_t(const ForwardArgs& a) {
+    using Cfg = TcCfg<D>;
     const int hr = head_rows_count(a);
     if (!a.causal && hr >= a.n) return LLA_OK;
     const int first_tile = a.causal ? hr / TC_BR : 0;
@@ -670,8 +771,8 @@ int launch_t(const ForwardArgs& a) {
     if (tiles <= 0) return LLA_OK;
     CUtensorMap mq, mk, mv;
     const int BH = a.B * a.H;
-    if (!make_map_bf16_64(&mq, a.q, BH, a.n, TC_BR) || !make_map_bf16_64(&mk, a.k, BH, a.n, TC_BC) ||
-        !make_map_bf16_64(&mv, a.v, BH, a.n, TC_BC))
+    if (!make_map_bf16(&mq, a.q, BH, a.n, D, TC_BR) || !make_map_bf16(&mk, a.k, BH, a.n, D, TC_BC) ||
+        !make_map_bf16(&mv, a.v, BH, a.n, D, TC_BC))
         return LLA_ERR_CUDA;
     TcParams prm;
     prm.n = a.n; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
@@ -679,13 +780,23 @@ int launch_t(const ForwardArgs& a) {
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     prm.dbg = nullptr;
+    prm.scratch = nullptr;
+    prm.scratch_slots = 0;
+    if constexpr (!Cfg::STATE_IN_SMEM) {
+        int dev = 0, sms = 0;
+        LLA_CUDA_TRY(cudaGetDevice(&dev));
+        LLA_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        prm.scratch_slots = 2 * sms;     // SM ids are dense in practice; the margin is checked in the kernel
+        prm.scratch = scratch_for_device((size_t)prm.scratch_slots * Cfg::SCRATCH_FLOATS_PER_SM * sizeof(float));
+        if (!prm.scratch) return LLA_ERR_CUDA;
+    }
 #if defined(LLA_TC_TIMING) || defined(LLA_TC_TRACE)
     prm.dbg = (unsigned long long*)a.workspace;   // tuning builds only: caller passes a zeroed buffer
 #endif
-    auto kern = forward_tc_kernel<TOut>;
-    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
+    auto kern = forward_tc_kernel<D, TOut>;
+    LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
     dim3 grid(BH, tiles);
-    kern<<<grid, TC_THREADS, SM_ALLOC, a.stream>>>(mq, mk, mv, (TOut*)a.out, prm);
+    kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -693,13 +804,18 @@ int launch_t(const ForwardArgs& a) {
 }  // namespace
 
 bool forward_tensor_supported(const ForwardArgs& a) {
-    return a.in_dtype == LLA_BF16 && a.d == TC_D && a.dv == TC_D && get_encode() != nullptr;
+    return a.in_dtype == LLA_BF16 && (a.d == 64 || a.d == 128) && a.dv == a.d && get_encode() != nullptr;
 }
 
 int launch_forward_tensor(const ForwardArgs& a) {
     if (!forward_tensor_supported(a)) return LLA_ERR_UNSUPPORTED;
-    if (a.out_dtype == LLA_BF16) return launch_t<__nv_bfloat16>(a);
-    if (a.out_dtype == LLA_F32) return launch_t<float>(a);
+    if (a.d == 64) {
+        if (a.out_dtype == LLA_BF16) return launch_t<64, __nv_bfloat16>(a);
+        if (a.out_dtype == LLA_F32) return launch_t<64, float>(a);
+    } else {
+        if (a.out_dtype == LLA_BF16) return launch_t<128, __nv_bfloat16>(a);
+        if (a.out_dtype == LLA_F32) return launch_t<128, float>(a);
+    }
     return LLA_ERR_UNSUPPORTED;
 }
 

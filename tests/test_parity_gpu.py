@@ -78,12 +78,16 @@ def test_config3_full_size_sampled_rows(oracle):
     assert err.max() <= TOL_BF16, err.max()
 
 
-def test_config4_reduced_full_rows(oracle):
+@pytest.mark.parametrize("impl", [L.LLA_IMPL_SIMT, L.LLA_IMPL_TENSOR])
+def test_config4_reduced_full_rows(oracle, impl):
     w = inputs.CONFIGS[4].shrink(H=2, n=1100)
     q, k, v = inputs.make_prefill(w)
     ref = oracle.forward(q, k, v, w.scale, w.lam)
-    err = row_err(forward(w, q, k, v, out_dtype="f32"), ref)
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    err = row_err(forward(w, q, k, v, out_dtype="f32", impl=impl, device_status=status), ref)
     assert err.max() <= TOL_BF16, err.max()
+    st = status.cpu().tolist()
+    assert st[L.STATUS_ROWS_AT_CAP] == 0 and st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
 
 
 def test_config4_full_size_sampled_rows(oracle):
