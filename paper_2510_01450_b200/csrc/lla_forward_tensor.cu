@@ -29,6 +29,7 @@
 // The mathematics is the centred form described in lla_forward_simt.cu (same CG, same freeze rule).
 // All waits on mbarriers are bounded; a wait that expires sets LLA_STATUS_TIMEOUT and the block
 // leaves through the common exit (TMEM is released there).
+#include <algorithm>
 #include <mutex>
 
 #include "lla_sm100.cuh"
@@ -46,6 +47,8 @@ constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_NBUF = 3;           // S/A/U buffers in TMEM (128 columns each)
 constexpr int TC_ACC_COL = TC_NBUF * 128;   // ACC columns [384, 384 + D)
 constexpr int TC_NST_MAX = 4;
+constexpr int TC_ORDER_MAX = 256;    // launch-order table size (query tiles)
+constexpr int TC_SPLIT_MAX = 4;      // sweeps of at most this many key blocks run in split mode (see the compute role)
 
 enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4 };
 
@@ -71,8 +74,8 @@ struct TcCfg {
     static constexpr int SM_KV = SM_PLO + OPER_BYTES;
     static constexpr int SM_X = SM_KV + NST * STAGE_BYTES;                        // fp32 [D][128] (D = 64 only)
     static constexpr int SM_KBAR = SM_X + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);
-    static constexpr int SM_RED = SM_KBAR + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);  // pair reductions 2 x 2 x 128 floats
-    static constexpr int SM_FLAGS = SM_RED + 2048;                                // 2 x 8 ints
+    static constexpr int SM_RED = SM_KBAR + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);  // pair reductions 2 x 2 x 2 x 128 floats
+    static constexpr int SM_FLAGS = SM_RED + 4096;                                // 2 x 8 ints
     static constexpr int SM_BAR = SM_FLAGS + 64;                                  // mbarriers
     static constexpr int SM_MISC = SM_BAR + 256;                                  // tmem base, ctl kind, abort
     static constexpr int SM_TOTAL = SM_MISC + 64;
@@ -177,6 +180,8 @@ struct TcParams {
     int* status;
     float* scratch;      // D = 128: per-SM slots for x, kbar, r (TcCfg::SCRATCH_FLOATS_PER_SM each)
     int scratch_slots;
+    int use_order;       // 1: blockIdx.y -> tile through order[]; 0: last tile first
+    unsigned short order[TC_ORDER_MAX];
 };
 
 template <int D, typename TOut>
@@ -218,13 +223,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     volatile int* flags = reinterpret_cast<volatile int*>(smem + SM_FLAGS);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // blockIdx.x runs fastest in launch order: all heads of the heaviest (last) query tile come first
+    // blockIdx.x runs fastest in launch order: all heads of one query tile start together, the tiles
+    // in order of decreasing estimated cost (see tile_order on the host side)
     const int bh = blockIdx.x;
-    const int tile = prm.first_tile + (gridDim.y - 1 - blockIdx.y);
+    const int tile = prm.first_tile + (prm.use_order ? (int)prm.order[blockIdx.y] : (int)(gridDim.y - 1 - blockIdx.y));
     const int r0 = tile * TC_BR;
     const int n = prm.n;
     const int nblk_all = (n + TC_BC - 1) / TC_BC;
     const int nblk = prm.causal ? min(nblk_all, (r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
+    const bool split = nblk <= TC_SPLIT_MAX;
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
@@ -235,7 +242,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         for (int b = 0; b < TC_NBUF; ++b) {
             mbar_init(bar(B_SAFULL + b), 1);
-            mbar_init(bar(B_UFULL + b), TC_COMPUTE / 2);
+            mbar_init(bar(B_UFULL + b), split ? TC_COMPUTE : TC_COMPUTE / 2);
             mbar_init(bar(B_BUFFREE + b), 1);
         }
         mbar_init(bar(B_ACCFULL), 1);
@@ -411,14 +418,24 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + quad) : "memory"); };
         int red_sel = 0;
         auto pair_sum = [&](float v) {
-            float* buf = red + red_sel * 256;
+            float* buf = red + red_sel * 512;
             red_sel ^= 1;
             buf[half * 128 + lrow] = v;
             pair_sync();
             return buf[lrow] + buf[128 + lrow];
         };
+        // two sums for one barrier
+        auto pair_sum2 = [&](float& a, float& b) {
+            float* buf = red + red_sel * 512;
+            red_sel ^= 1;
+            buf[half * 128 + lrow] = a;
+            buf[256 + half * 128 + lrow] = b;
+            pair_sync();
+            a = buf[lrow] + buf[128 + lrow];
+            b = buf[256 + lrow] + buf[384 + lrow];
+        };
         auto pair_max = [&](float v) {
-            float* buf = red + red_sel * 256;
+            float* buf = red + red_sel * 512;
             red_sel ^= 1;
             buf[half * 128 + lrow] = v;
             pair_sync();
@@ -458,9 +475,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         bool ok = true;
 
         // One sweep over the key blocks.  kind is uniform over the block.
-        // Warps 0-3 (group 0) take the even blocks, warps 4-7 (group 1) the odd ones, each thread all
-        // 64 keys of its row in two passes of 32: the two warps that share a scheduler are then in
-        // different phases of the load -> math -> store chain and hide each other's latency.
+        // Long sweeps: warps 0-3 (group 0) take the even blocks, warps 4-7 (group 1) the odd ones,
+        // each thread all 64 keys of its row in two passes of 32: the two warps that share a
+        // scheduler are then in different phases of the load -> math -> store chain and hide each
+        // other's latency.  Short sweeps (split mode, the first query tiles) are latency-bound
+        // instead: there both groups work on every block, each thread on its half of the keys, which
+        // halves the time from a block's scores to its contribution.
         auto sweep = [&](int kind) {
             float part = 0.f;                                 // omega / den partial, or max
             if (kind == SW_MAX) part = -INFINITY;
@@ -468,7 +488,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const uint64_t nab = pk2(-abar, -abar), oab = pk2(1.f + abar, 1.f + abar), neg1 = pk2(-1.f, -1.f);
             uint64_t part2 = pk2(0.f, 0.f);
             for (int c = 0; c < nblk; ++c, ++blk) {
-                if ((int)(blk & 1) != half) continue;
+                if (!split && (int)(blk & 1) != half) continue;
                 const uint32_t b = blk % TC_NBUF;
                 TC_T0(t_w);
                 if (lane == 0 && quad == 0) TC_EV(30 + half, blk);
@@ -477,7 +497,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (tid == 0) TC_ACC(0, t_w);
                 tc_fence_after();
 #pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
+                for (int h = split ? half : 0; h < (split ? half + 1 : 2); ++h) {
                     TC_T0(t_l);
                     const uint32_t s_addr = tmem + lane_addr + b * 128 + 32 * h;
                     uint32_t sv[32], av[32];
@@ -625,42 +645,68 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #else
             if (!group_any(active)) break;
 #endif
+            if (lane == 0 && quad == 0) TC_EV(45, t);
             start_sweep(SW_CG);
+            if (lane == 0 && quad == 0) TC_EV(46, t);
             sweep(SW_CG);
+            if (lane == 0 && quad == 0) TC_EV(47, t);
             float ap[NCOL];
             if (ok) read_acc(ap);
             if (!ok) break;
-            float pap_p = 0.f;
+            if (lane == 0 && quad == 0) TC_EV(40, t);
+            // (the loops below keep four independent partial sums and move the row-vector state in
+            //  batches of eight so that the loads overlap: two warps per scheduler hide no latency)
+            float pp[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int e = 0; e < NCOL; ++e) {
                 ap[e] = fmaf(ap[e], inv_omega, ridge * p[e]);
-                pap_p += p[e] * ap[e];
+                pp[e & 3] = fmaf(p[e], ap[e], pp[e & 3]);
             }
-            const float pap = pair_sum(pap_p);
+            const float pap = pair_sum((pp[0] + pp[1]) + (pp[2] + pp[3]));
+            if (lane == 0 && quad == 0) TC_EV(41, t);
             if (active && !(pap > 0.f)) active = false;
             const float alpha = active ? rr / pap : 0.f;
-            float rr2_p = 0.f;
+            if (lane == 0 && quad == 0) TC_EV(48, t);
+            float r2[4] = {0.f, 0.f, 0.f, 0.f}, kr[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int e = 0; e < NCOL; ++e) {
-                xs[(c0 + e) * TC_BR + lrow] += alpha * p[e];
-                const float rn = r_get(e) - alpha * ap[e];
-                r_set(e, rn);
-                ap[e] = rn;                       // ap now holds the new residual
-                rr2_p += rn * rn;
+            for (int e0 = 0; e0 < NCOL; e0 += 8) {
+                float xv[8], kv[8], rv[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    xv[i] = xs[(c0 + e0 + i) * TC_BR + lrow];
+                    kv[i] = kbs[(c0 + e0 + i) * TC_BR + lrow];
+                    rv[i] = r_get(e0 + i);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    xv[i] = fmaf(alpha, p[e0 + i], xv[i]);
+                    rv[i] = fmaf(-alpha, ap[e0 + i], rv[i]);
+                    ap[e0 + i] = rv[i];                       // ap now holds the new residual
+                    r2[i & 3] = fmaf(rv[i], rv[i], r2[i & 3]);
+                    kr[i & 3] = fmaf(kv[i], rv[i], kr[i & 3]);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    xs[(c0 + e0 + i) * TC_BR + lrow] = xv[i];
+                    r_set(e0 + i, rv[i]);
+                }
             }
-            const float rr2 = pair_sum(rr2_p);
-            float ab_p = 0.f;
+            // ||r_new||^2 and kbar . r_new in one exchange; kbar . p_new follows from the recurrence
+            float rr2 = (r2[0] + r2[1]) + (r2[2] + r2[3]), kbr = (kr[0] + kr[1]) + (kr[2] + kr[3]);
+            if (lane == 0 && quad == 0) TC_EV(49, t);
+            pair_sum2(rr2, kbr);
+            if (lane == 0 && quad == 0) TC_EV(42, t);
             if (active) {
                 const float beta = rr2 / rr;
 #pragma unroll
                 for (int e = 0; e < NCOL; ++e) p[e] = fmaf(beta, p[e], ap[e]);
+                abar = fmaf(beta, abar, kbr);
                 rr = rr2;
                 ++its;
             }
-#pragma unroll
-            for (int e = 0; e < NCOL; ++e) ab_p += kbs[(c0 + e) * TC_BR + lrow] * p[e];
-            abar = pair_sum(ab_p);
+            if (lane == 0 && quad == 0) TC_EV(43, t);
             write_operand(p);
+            if (lane == 0 && quad == 0) TC_EV(44, t);
         }
         const bool at_cap = active && rr > stop;
         // ---- output sweep ----
@@ -719,6 +765,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         if (ok) start_sweep(SW_DONE);
         if (tid == 0) TC_ACC(5, t_all);
+#ifdef LLA_TC_TIMING
+        if (tid == 0 && prm.dbg) {   // per-block duration and end time (tuning builds)
+            const size_t idx = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+            unsigned long long gt;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+            prm.dbg[32 + 2 * idx] = (unsigned long long)(clock64() - t_all);
+            prm.dbg[33 + 2 * idx] = gt;
+        }
+#endif
         if (tid == 0) { TC_T0(t_one); TC_ACC(6, t_one - 1); (void)nblk; }
     }
 
@@ -761,6 +816,27 @@ float* scratch_for_device(size_t bytes) {
     return ptr[dev];
 }
 
+// Launch order of the query tiles: longest first, so that the blocks left for the end are short.
+// A tile's cost is (sweeps) x (per-sweep overhead + key blocks).  Sweeps = 3 + CG iterations, and the
+// iteration count falls with the number of visible keys per dimension (the first tiles need several
+// times more than the rest), so at short sequence lengths the first tiles are the longest blocks
+// even though their sweeps are the shortest.  The numbers are a fit to measured runs; they only
+// steer the order, never the result.
+void tile_order(TcParams& prm, int tiles, int first_tile, int n, int d, int causal) {
+    prm.use_order = 0;
+    if (!causal || tiles > TC_ORDER_MAX) return;
+    float cost[TC_ORDER_MAX];
+    for (int t = 0; t < tiles; ++t) {
+        const int r_end = std::min(n, (first_tile + t + 1) * TC_BR);
+        const float its = 6.f + 50.f * (float)d / (float)r_end;
+        const float nblk = (float)((r_end + TC_BC - 1) / TC_BC);
+        cost[t] = (its + 3.f) * (6.f + nblk);
+        prm.order[t] = (unsigned short)t;
+    }
+    std::stable_sort(prm.order, prm.order + tiles, [&](unsigned short x, unsigned short y) { return cost[x] > cost[y]; });
+    prm.use_order = 1;
+}
+
 template <int D, typename TOut>
 int launch_t(const ForwardArgs& a) {
     using Cfg = TcCfg<D>;
@@ -782,6 +858,7 @@ int launch_t(const ForwardArgs& a) {
     prm.dbg = nullptr;
     prm.scratch = nullptr;
     prm.scratch_slots = 0;
+    tile_order(prm, tiles, first_tile, a.n, D, a.causal);
     if constexpr (!Cfg::STATE_IN_SMEM) {
         int dev = 0, sms = 0;
         LLA_CUDA_TRY(cudaGetDevice(&dev));
