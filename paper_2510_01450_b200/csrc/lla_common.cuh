@@ -109,11 +109,18 @@ __device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __fl
 //   S   : D x D, row stride lds doubles, lower triangle filled; destroyed (LDL^T in place)
 //   rhs : D doubles; replaced by the solution
 // Returns false if a pivot was not positive.  Every thread of the block must call it; blockDim.x
-// must be a multiple of 32 with at least two warps.
+// must be a multiple of 32.
 //
-// The right-hand side rides along as an extra matrix row, so the forward substitution happens
-// inside the elimination; the backward substitution is a column sweep by warp 0 with the partial
-// sums of each unknown held in registers.
+// Blocked right-looking LDL^T with panels of NB = 8 columns.  After a column is eliminated it holds
+// L[r][c] * D_c (left unscaled) and the diagonal holds D_c.  The right-hand side rides along as
+// matrix row D, so the forward substitution happens inside the elimination.  Per panel:
+//   (i)   the 8 x 8 diagonal block is factorised by warp 0 in registers (one row per lane, pivot row
+//         and pivot column passed by shuffles: no block barrier inside the eight column steps);
+//   (ii)  every row below it (and the right-hand side) eliminates its eight panel entries against
+//         the finished diagonal block, one thread per row;
+//   (iii) one rank-8 update of everything to the right, all threads.
+// The backward substitution is blocked the same way and runs in warp 0: eight unknowns at a time
+// by shuffles, then their contribution to all earlier unknowns (held in registers, lane-strided).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ double fast_rcp(double x) {
     double r;
@@ -122,82 +129,196 @@ __device__ __forceinline__ double fast_rcp(double x) {
     r = r * (2.0 - x * r);
     return r;
 }
+// One Newton step on the 20-bit seed: relative error ~1e-12, enough for elimination multipliers
+// (the error only perturbs the factorised matrix at that level) and one dependent pair shorter.
+__device__ __forceinline__ double fast_rcp1(double x) {
+    double r;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+    r = r * (2.0 - x * r);
+    return r;
+}
 
-template <int D>
-__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs) {
-    const int tid = threadIdx.x, nt = blockDim.x;
-    const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
-    bool ok = true;
-    __syncthreads();
-    // Blocked right-looking LDL^T, panels of NB columns.  After a column is eliminated it holds
-    // L[r][c] * D_c (left unscaled) and the diagonal holds D_c.  The right-hand side is carried as
-    // row index D.  Per panel: (a) eliminate inside the panel, one thread per row; (b) one rank-NB
-    // update of everything to the right (4 multiply-adds per element loaded and stored).
-    constexpr int NB = 8;
-    static_assert(D % NB == 0, "head size must be a multiple of the panel width");
-    for (int c0 = 0; c0 < D; c0 += NB) {
-        for (int k = 0; k < NB; ++k) {
-            const int c = c0 + k;
-            const double piv = S[c * lds + c];
-            if (!(piv > 0.0)) ok = false;
-            const double inv = fast_rcp(piv);
-            for (int r = c + 1 + tid; r <= D; r += nt) {
-                double* rowp = r < D ? S + r * lds : rhs;
-                const double l = rowp[c] * inv;
-                for (int c2 = c + 1; c2 < c0 + NB; ++c2)
-                    if (r == D || c2 <= r) rowp[c2] -= l * S[c2 * lds + c];
-            }
-            __syncthreads();
-        }
-        if (c0 + NB < D) {
-            double dinv[NB];
+// Optional phase timing for tuning (-DLLA_HR_TIMING): clock totals of thread 0 go to tst[phase].
+#ifdef LLA_HR_TIMING
+#define LDLT_TARG , int* tst = nullptr
+#define LDLT_T0 long long lt_ = clock64()
+#define LDLT_T(ph) do { if (threadIdx.x == 0 && tst) { const long long now_ = clock64(); atomicAdd(tst + (ph), (int)((now_ - lt_) >> 4)); lt_ = now_; } } while (0)
+#else
+#define LDLT_TARG
+#define LDLT_T0
+#define LDLT_T(ph)
+#endif
+
+// (i): factorise the NB x NB diagonal block at c0 (called by one full warp).  The reciprocal of
+// pivot c is left in S[c][c + 1], an element of the unused upper triangle (lds >= D + 1).
+template <int NB>
+__device__ __forceinline__ void ldlt_diag_block(double* S, int lds, int c0) {
+    constexpr unsigned FULL = 0xffffffffu;
+    const int tx = threadIdx.x & 31;
+    const int i = tx & (NB - 1);   // lanes NB..31 mirror lanes 0..NB-1: every shuffle source is live
+    double a[NB];
 #pragma unroll
-            for (int k = 0; k < NB; ++k) dinv[k] = fast_rcp(S[(c0 + k) * lds + c0 + k]);
-            for (int r = c0 + NB + ty; r <= D; r += ny) {
-                double* rowp = r < D ? S + r * lds : rhs;
-                double ls[NB];
+    for (int k = 0; k < NB; ++k) a[k] = k <= i ? S[(c0 + i) * lds + c0 + k] : 0.0;
 #pragma unroll
-                for (int k = 0; k < NB; ++k) ls[k] = rowp[c0 + k] * dinv[k];
-                const int cmax = r < D ? r : D - 1;
-                for (int c2 = c0 + NB + tx; c2 <= cmax; c2 += 32) {
-                    const double* u = S + c2 * lds + c0;
-                    double acc = 0.0;
+    for (int k = 0; k < NB; ++k) {
+        const double piv = __shfl_sync(FULL, a[k], k);
+        const double inv = fast_rcp1(piv);
+        if (tx == 0) S[(c0 + k) * lds + c0 + k + 1] = inv;
+        const double l = a[k] * inv;
 #pragma unroll
-                    for (int k = 0; k < NB; ++k) acc += ls[k] * u[k];
-                    rowp[c2] -= acc;
-                }
-            }
-            __syncthreads();
+        for (int c2 = k + 1; c2 < NB; ++c2) {
+            const double colv = __shfl_sync(FULL, a[k], c2);
+            if (i >= c2) a[c2] -= l * colv;
         }
     }
-    if (!(S[(D - 1) * lds + (D - 1)] > 0.0)) ok = false;
-    // rhs now holds y with L y = b.  Backward: x_r = (y_r - sum_{t>r} S[t][r] x_t) / D_r.
+    if (tx < NB) {
+#pragma unroll
+        for (int k = 1; k < NB; ++k)
+            if (k <= i) S[(c0 + i) * lds + c0 + k] = a[k];
+    }
+}
+
+template <int D>
+__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs LDLT_TARG) {
+    LDLT_T0;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
+    constexpr int NB = 8;
+    constexpr unsigned FULL = 0xffffffffu;
+    constexpr int SLOTS = (D - NB + 31) / 32 > 0 ? (D - NB + 31) / 32 : 1;   // trailing columns per lane
+    static_assert(D % NB == 0, "head size must be a multiple of the panel width");
+    __syncthreads();
+    if (ty == 0) ldlt_diag_block<NB>(S, lds, 0);
+    __syncthreads();
+    LDLT_T(0);
+    for (int c0 = 0; c0 < D; c0 += NB) {
+        double dinv[NB];
+#pragma unroll
+        for (int k = 0; k < NB; ++k) dinv[k] = S[(c0 + k) * lds + c0 + k + 1];
+        // (ii)
+        for (int r = c0 + NB + tid; r <= D; r += nt) {
+            double* rowp = r < D ? S + r * lds : rhs;
+            double x[NB];
+#pragma unroll
+            for (int k = 0; k < NB; ++k) x[k] = rowp[c0 + k];
+#pragma unroll
+            for (int k = 0; k < NB - 1; ++k) {
+                const double l = x[k] * dinv[k];
+#pragma unroll
+                for (int c2 = k + 1; c2 < NB; ++c2) x[c2] -= l * S[(c0 + c2) * lds + c0 + k];
+            }
+#pragma unroll
+            for (int k = 1; k < NB; ++k) rowp[c0 + k] = x[k];
+        }
+        __syncthreads();
+        LDLT_T(1);
+        // (iii) element (r, c2) -= sum_k S[r][c0+k] * S[c2][c0+k] / D_k.  A lane keeps the scaled
+        // panel entries of its columns c2 in registers for the whole update and walks down the rows;
+        // a row's eight panel entries are the same address for every lane (broadcast loads), so
+        // shared-memory traffic is one load and one store per updated element.
+        if (c0 + NB < D) {
+            double u[SLOTS][NB];
+#pragma unroll
+            for (int sl = 0; sl < SLOTS; ++sl) {
+                const int c2 = c0 + NB + tx + 32 * sl;
+#pragma unroll
+                for (int k = 0; k < NB; ++k) u[sl][k] = c2 < D ? S[c2 * lds + c0 + k] * dinv[k] : 0.0;
+            }
+            auto update_row = [&](int r) {
+                double* rowp = r < D ? S + r * lds : rhs;
+                double a[NB];
+#pragma unroll
+                for (int k = 0; k < NB; ++k) a[k] = rowp[c0 + k];
+                const int cmax = r < D ? r : D - 1;
+#pragma unroll
+                for (int sl = 0; sl < SLOTS; ++sl) {
+                    const int c2 = c0 + NB + tx + 32 * sl;
+                    if (c2 <= cmax) {
+                        double acc = 0.0;
+#pragma unroll
+                        for (int k = 0; k < NB; ++k) acc += a[k] * u[sl][k];
+                        rowp[c2] -= acc;
+                    }
+                }
+            };
+            if (ty == 0) {
+                // warp 0 brings the next diagonal block up to date and factorises it at once, while
+                // the other warps update the rows below it
+                // (a lane per element of the block, two passes)
+#pragma unroll
+                for (int pass = 0; pass < NB * NB / 32; ++pass) {
+                    const int e = tx + 32 * pass, ro = e / NB, co = e % NB;
+                    if (co <= ro) {
+                        const double* ra = S + (c0 + NB + ro) * lds + c0;
+                        const double* rb = S + (c0 + NB + co) * lds + c0;
+                        double acc = 0.0;
+#pragma unroll
+                        for (int k = 0; k < NB; ++k) acc += ra[k] * (rb[k] * dinv[k]);
+                        S[(c0 + NB + ro) * lds + c0 + NB + co] -= acc;
+                    }
+                }
+                __syncwarp();
+                ldlt_diag_block<NB>(S, lds, c0 + NB);
+                if (ny == 1)
+                    for (int r = c0 + 2 * NB; r <= D; ++r) update_row(r);
+            } else {
+                for (int r = c0 + 2 * NB + ty - 1; r <= D; r += ny - 1) update_row(r);
+            }
+            __syncthreads();
+            LDLT_T(2);
+        }
+    }
+    bool ok = true;
+    for (int k = 0; k < D; ++k)
+        if (!(S[k * lds + k] > 0.0)) ok = false;
+    LDLT_T(3);
+    // rhs now holds y with L y = b.  Backward: x_t = (y_t - sum_{r>t} S[r][t] x_r) / D_t.
     if (tid < 32) {
         constexpr int PER = (D + 31) / 32;
-        double part[PER], dinv[PER], yv[PER];
+        const int i = tx & 7;
+        double part[PER], yv[PER];
 #pragma unroll
         for (int u = 0; u < PER; ++u) {
             const int t = tx + 32 * u;
             part[u] = 0.0;
-            dinv[u] = t < D ? fast_rcp(S[t * lds + t]) : 0.0;
             yv[u] = t < D ? rhs[t] : 0.0;
         }
-        for (int r = D - 1; r >= 0; --r) {
-            const int owner = r & 31, slot = r >> 5;
-            double xr = 0.0;
+        for (int c0 = D - NB; c0 >= 0; c0 -= NB) {
+            // y - (contributions of later panels) for the eight unknowns c0 + i of this panel
+            double mine = 0.0;
 #pragma unroll
             for (int u = 0; u < PER; ++u)
-                if (u == slot) xr = (yv[u] - part[u]) * dinv[u];
-            xr = __shfl_sync(0xffffffffu, xr, owner);
-            if (tx == owner) rhs[r] = xr;
+                if (u == (c0 >> 5)) mine = yv[u] - part[u];
+            double val = __shfl_sync(FULL, mine, (c0 & 31) + i);
+            double sc[NB];   // column c0 + i of the diagonal block, below the diagonal
+#pragma unroll
+            for (int r = 0; r < NB; ++r) sc[r] = r > i ? S[(c0 + r) * lds + c0 + i] : 0.0;
+            const double di = S[(c0 + i) * lds + c0 + i + 1];
+            double xb[NB];
+#pragma unroll
+            for (int t = NB - 1; t >= 0; --t) {
+                xb[t] = __shfl_sync(FULL, val * di, t);
+                val -= sc[t] * xb[t];
+            }
+            if (tx < NB) {
+                double xm = 0.0;
+#pragma unroll
+                for (int t = 0; t < NB; ++t)
+                    if (t == tx) xm = xb[t];
+                rhs[c0 + tx] = xm;
+            }
 #pragma unroll
             for (int u = 0; u < PER; ++u) {
                 const int t = tx + 32 * u;
-                if (t < r) part[u] += S[r * lds + t] * xr;
+                if (t < c0) {
+#pragma unroll
+                    for (int r = 0; r < NB; ++r) part[u] += S[(c0 + r) * lds + t] * xb[r];
+                }
             }
         }
     }
     __syncthreads();
+    LDLT_T(4);
     return ok;
 }
 

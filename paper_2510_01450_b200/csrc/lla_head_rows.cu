@@ -70,6 +70,15 @@ __device__ __forceinline__ double dot_row(const double* __restrict__ a, const fl
     return s;
 }
 
+// Optional phase timing for tuning (-DLLA_HR_TIMING: clock totals of thread 0 are added to status[8 + phase]).
+#ifdef LLA_HR_TIMING
+#define HR_T(phase) do { if (threadIdx.x == 0 && status) { const long long now_ = clock64(); atomicAdd(status + 8 + (phase), (int)((now_ - hr_t_) >> 4)); hr_t_ = now_; } } while (0)
+#define HR_T0 long long hr_t_ = clock64()
+#else
+#define HR_T(phase)
+#define HR_T0
+#endif
+
 template <int D, int DV, typename TIn, typename TOut>
 __global__ void __launch_bounds__(HR_THREADS, (D <= 64 ? 4 : 1))
 head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
@@ -102,6 +111,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     const TIn* kb = k + (size_t)bh * n * D;
     const TIn* vb = v + (size_t)bh * n * DV;
 
+    HR_T0;
     for (int c = tid; c < D; c += HR_THREADS) qd[c] = (double)to_f32(qrow[c]);
     __syncthreads();
 
@@ -112,6 +122,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         w[j] = s;
         lmax = fmax(lmax, s);
     }
+    HR_T(0);
     const double m = block_reduce(lmax, true, red);
     double lsum = 0.0;
     for (int j = tid; j < L; j += HR_THREADS) {
@@ -121,6 +132,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     }
     const double omega = block_reduce(lsum, false, red);
     const double lambda_m = lambda * exp(-m);
+    HR_T(1);
 
     // moments: Sigma (lower 4x4 tiles in registers) and mu
     double acc[C::TILES_PER_THREAD][4][4];
@@ -174,6 +186,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
             }
         }
     }
+    HR_T(2);
 #pragma unroll
     for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
         if (tr[t] < 0) continue;
@@ -189,8 +202,14 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     if (tid < D) rhs[tid] = mu_acc;
     __syncthreads();
 
+    HR_T(3);
     // rhs <- Sigma^{-1} mu (LDL^T in shared memory)
+#ifdef LLA_HR_TIMING
+    const bool bad = !block_ldlt_solve<D>(S, C::LDS, rhs, status ? status + 16 : nullptr);
+#else
     const bool bad = !block_ldlt_solve<D>(S, C::LDS, rhs);
+#endif
+    HR_T(4);
 
     // coefficients c_j = w_j (1 - z_j . rho) and their sum (= omega - mu . rho)
     double qrho = 0.0;
@@ -203,11 +222,13 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         csum += cj;
     }
     const double denom = block_reduce(csum, false, red);
+    HR_T(5);
     for (int c = tid; c < DV; c += HR_THREADS) {
         double o = 0.0;
         for (int j = 0; j < L; ++j) o += w[j] * (double)to_f32(vb[(size_t)j * DV + c]);
         store_out(out + row * DV + c, (float)(o / denom));
     }
+    HR_T(6);
     if (rho_out && tid < D) rho_out[row * D + tid] = (float)rhs[tid];
     if (tid == 0) {
         if (stats) {
