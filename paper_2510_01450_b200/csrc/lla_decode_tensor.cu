@@ -96,8 +96,10 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
 // stride 65 doubles, both triangles filled) with conjugate gradients in double precision, run by
 // the 128 threads of warps 0..3 (two threads per row, 32 columns each).  A dense factorisation is a
 // chain of 64 dependent column steps, each with block barriers; here an iteration is one short
-// matrix-vector product and three 128-thread barriers, and the decode systems (>= 2d keys) need a
-// few dozen iterations.  x lands in xs[]; returns false if the residual did not reach 1e-11 |b|
+// matrix-vector product and three 128-thread barriers, and the decode systems (>= 2d keys) need one
+// or two dozen iterations.  Each thread keeps its 32 matrix entries in registers for the whole
+// solve: re-reading the matrix from shared memory every iteration costs several times more than
+// the arithmetic while the SM's other block is streaming its cache through the same memory.  x lands in xs[]; returns false if the residual did not reach 1e-9 |b|
 // within the iteration cap (the caller then falls back to the factorisation).  C is not modified.
 __device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, double* xs, double* pbuf, double* redbuf, int& iters) {
     const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
@@ -111,34 +113,42 @@ __device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, do
         sync128();
         return (redbuf[slot * 4] + redbuf[slot * 4 + 1]) + (redbuf[slot * 4 + 2] + redbuf[slot * 4 + 3]);
     };
+    double cr[32];
+    {
+        const double* crow = C + r * 65 + 32 * hh;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) cr[c] = crow[c];
+    }
     double x = 0.0, res = b[r], pv = res;
     if (hh == 0) pbuf[r] = pv;
     double rr = block_sum(res * res, 0);
-    const double stop = rr * 1e-22;
+    const double stop = rr * 1e-18;     // |r| <= 1e-9 |b|: far below what a bf16 or fp32 output resolves
     bool done = !(rr > 0.0);
     int slot = 1;
     iters = 0;
     for (int it = 0; it < LLA_CG_CAP && !done; ++it) {
         ++iters;
-        const double* crow = C + r * 65 + 32 * hh;
-        const double* pp = pbuf + 32 * hh;
-        double a0 = 0.0, a1 = 0.0;
-#pragma unroll 8
-        for (int c = 0; c < 32; c += 2) {
-            a0 += crow[c] * pp[c];
-            a1 += crow[c + 1] * pp[c + 1];
+        const double2* pp = reinterpret_cast<const double2*>(pbuf + 32 * hh);
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+            const double2 p01 = pp[c >> 1], p23 = pp[(c >> 1) + 1];
+            a0 = fma(cr[c], p01.x, a0);
+            a1 = fma(cr[c + 1], p01.y, a1);
+            a2 = fma(cr[c + 2], p23.x, a2);
+            a3 = fma(cr[c + 3], p23.y, a3);
         }
-        double ap = a0 + a1;
+        double ap = (a0 + a1) + (a2 + a3);
         ap += __shfl_xor_sync(0xffffffffu, ap, 1);
         const double pap = block_sum(pv * ap, slot);
         slot = slot % 5 + 1;
         if (!(pap > 0.0)) break;
-        const double alpha = rr / pap;
+        const double alpha = rr * fast_rcp(pap);
         x += alpha * pv;
         res -= alpha * ap;
         const double rr2 = block_sum(res * res, slot);
         slot = slot % 5 + 1;
-        pv = res + (rr2 / rr) * pv;
+        pv = res + (rr2 * fast_rcp(rr)) * pv;
         rr = rr2;
         done = rr <= stop;
         if (hh == 0) pbuf[r] = pv;
@@ -150,6 +160,15 @@ __device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, do
 }
 
 __device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Optional phase timing for tuning (-DLLA_DT_TIMING): clock totals of thread 0 go to status[8 + phase].
+#ifdef LLA_DT_TIMING
+#define DT_T0 long long dt_t_ = clock64()
+#define DT_T(ph) do { if (threadIdx.x == 0 && prm.status) { const long long now_ = clock64(); atomicAdd(prm.status + 8 + (ph), (int)((now_ - dt_t_) >> 4)); dt_t_ = now_; } } while (0)
+#else
+#define DT_T0
+#define DT_T(ph)
+#endif
 
 struct DtParams {
     int B, H, Lmax, splits, head_rows;
@@ -174,6 +193,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int part = blockIdx.x;
+#ifdef LLA_DT_TIMING
+    long long ep_t_ = clock64();
+#define EP_T(ph) do { if (threadIdx.x == 0 && prm.status) { const long long now_ = clock64(); atomicAdd(prm.status + 16 + (ph), (int)((now_ - ep_t_) >> 4)); ep_t_ = now_; } } while (0)
+#else
+#define EP_T(ph)
+#endif
     // Longest caches first: blocks launch in blockIdx order, so block y takes head (y % H) of the
     // sequence whose length has rank (y / H).  Every block ranks the (few) sequence lengths itself.
     int bh = blockIdx.y;
@@ -215,6 +240,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[0];
+    EP_T(0);
 
     float omega = 0.f, m_ref = -INFINITY;     // compute threads; m_ref in log2 units
 
@@ -239,7 +265,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (!mbar_wait(bar(DB_BFULL + b), (t >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
+#ifndef LLA_DEXP_NOMMA
             mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), make_desc_b(bsm + DT_BTILE), t > 0);
+#endif
             tc_commit_el(el, bar(DB_KVEMPTY + s));
             tc_commit_el(el, bar(DB_BFREE + b));
             if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
@@ -303,14 +331,29 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
             sdot += __shfl_xor_sync(0xffffffffu, sdot, 1);
             const float s2 = valid ? sdot * c1 : -INFINITY;
-            // tile maximum (uniform over the 128 compute threads)
-            float wm = s2;
+            // The reference maximum is the first tile's.  Later tiles only need to know whether any
+            // score exceeds it by more than 2^40 (then the accumulator is rescaled): one barrier
+            // that ORs a predicate over the 128 compute threads answers that; the tile maximum
+            // itself is reduced only for the first tile and in the rare rescale.
+            bool need_max = t == 0;
+            if (t > 0) {
+                uint32_t any;
+                asm volatile(
+                    "{\n\t.reg .pred p, q;\n\tsetp.gt.f32 q, %1, %2;\n\t"
+                    "barrier.cta.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                    : "=r"(any) : "f"(s2), "f"(m_ref + 40.f) : "memory");
+                need_max = any != 0;
+            }
+            float tile_max = m_ref;
+            if (need_max) {
+                float wm = s2;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
-            volatile float* tm = tmax + (t & 1) * 4;
-            if (lane == 0) tm[warp] = wm;
-            named_sync_128();
-            const float tile_max = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
+                for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
+                volatile float* tm = tmax + (t & 1) * 4;
+                if (lane == 0) tm[warp] = wm;
+                named_sync_128();
+                tile_max = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
+            }
             if (t == 0) {
                 m_ref = tile_max;
             } else if (tile_max > m_ref + 40.f) {
@@ -340,10 +383,18 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             return true;
         };
         if (ntile > 0) ok = stage_load(0) && stage_score(0);
+        DT_T0;
         for (int t = 0; t < ntile && ok; ++t) {
             const uint32_t b = t & 1;
             const bool more = t + 1 < ntile;
             // B rows of tile t: w * [k | 1] as bf16 hi + lo, computed into registers first
+#ifdef LLA_DEXP_NOSIMT
+            if (more && !stage_load(t + 1)) { ok = false; break; }
+            if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            mbar_arrive(bar(DB_BFULL + b));
+            if (h == 0) omega += kf[0] + __uint_as_float(raw[1].x);
+            continue;
+#endif
             uint32_t hi[16], lo[16];
             const uint64_t ww = pk2(w, w);
 #pragma unroll
@@ -354,10 +405,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             uint32_t wlo;
             const uint32_t whi = split_bf16x2(w, 0.f, wlo);
+            DT_T(0);
             // loads of the next tile go out now; they land while the stores below are issued
             if (more && !stage_load(t + 1)) { ok = false; break; }
+            DT_T(1);
             // wait until the MMA of tile t-2 has released this B buffer
             if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            DT_T(2);
             uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
             uint8_t* blo = bhi + DT_BTILE;
 #pragma unroll
@@ -373,7 +427,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             fence_proxy_async();
             mbar_arrive(bar(DB_BFULL + b));
+            DT_T(3);
             if (more && !stage_score(t + 1)) { ok = false; break; }
+            DT_T(4);
         }
         // total weight of this part
         if (ok) {
@@ -384,6 +440,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     // ================================ epilogue ================================
     // All 192 threads take part (the solve below is a block-wide routine).
+    EP_T(1);
     __shared__ float s_omega[4];
     __shared__ float s_mref;
     if (warp < 4 && lane == 0) s_omega[warp] = omega;
@@ -412,7 +469,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     }
     tc_fence_before();
+    EP_T(2);
     __syncthreads();       // every pipeline stage is drained: shared memory can be re-carved
+    EP_T(3);
     if (warp == 4) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(DT_TMEM_COLS) : "memory");
@@ -443,6 +502,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         return;
     }
 
+#ifdef LLA_DEXP_NOEPI
+    if (tid < 64) store_out(out + (size_t)bh * DT_D + tid, dv[3] + omega_tot);
+    return;
+#endif
     // single part: centre, solve and emit the output row here
     double* Md = reinterpret_cast<double*>(smem);              // 64 x 65
     double* av = Md + 64 * 65;                                  // a -> kbar
@@ -470,6 +533,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     }
     __syncthreads();
+    EP_T(4);
     // conjugate gradients first (fast); the blocked factorisation only if they do not converge
     double* xs = reinterpret_cast<double*>(Nd + 64 * 65);      // x, p and reduction scratch after N
     __shared__ int s_cg_ok;
@@ -482,6 +546,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     }
     __syncthreads();
+    EP_T(5);
     bool solved = true;
     if (s_cg_ok) {
         if (tid < 64) rhs[tid] = xs[tid];
@@ -494,6 +559,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int f = 0; f < 64; ++f) o += ((double)Nd[tid * 65 + f] * inv - cv[tid] * av[f]) * rhs[f];
         store_out(out + (size_t)bh * DT_D + tid, (float)o);
     }
+    EP_T(6);
     if (!solved && tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_BAD_PIVOT, 1);
 }
 

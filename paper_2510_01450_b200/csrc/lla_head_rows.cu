@@ -13,17 +13,26 @@
 namespace lla {
 namespace {
 
-constexpr int HR_THREADS = 256;
-constexpr int HR_CHUNK = 16;  // keys staged per step of the moment build
+constexpr int HR_CHUNK = 32;  // keys staged per step of the moment build
 
 template <int D>
 struct HrCfg {
     static constexpr int TILES_1D = D / 4;                           // 4x4 register tiles
     static constexpr int TILES = TILES_1D * (TILES_1D + 1) / 2;      // lower triangle incl. diagonal
-    static constexpr int TILES_PER_THREAD = (TILES + HR_THREADS - 1) / HR_THREADS;
+    // One thread per tile where that fits (136 tiles for D = 64 -> 5 warps).  The factorisation
+    // that follows has little parallelism, so small blocks, and more of them per SM, is what
+    // keeps the double-precision pipe busy.
+    static constexpr int THREADS = D <= 64 ? 160 : 256;
+    static constexpr int BLOCKS_PER_SM = D <= 64 ? 6 : 1;
+    static constexpr int TILES_PER_THREAD = (TILES + THREADS - 1) / THREADS;
+    // shared memory (doubles): the Sigma matrix; the staged keys of the moment build lie over it
+    // (the matrix is written only after the build)
+    static constexpr int S_DOUBLES = D * (D + 1) > HR_CHUNK * D ? D * (D + 1) : HR_CHUNK * D;
+    static constexpr size_t smem_doubles(int lcap) { return (size_t)S_DOUBLES + 2 * D + ((lcap + 1) & ~1) + THREADS / 32 + 1; }
     static constexpr int LDS = D + 1;                                // padded row stride (doubles)
 };
 
+template <int HR_THREADS>
 __device__ __forceinline__ double block_reduce(double x, bool is_max, double* scratch) {
     // scratch: HR_THREADS/32 + 1 doubles
     for (int off = 16; off > 0; off >>= 1) {
@@ -79,8 +88,20 @@ __device__ __forceinline__ double dot_row(const double* __restrict__ a, const fl
 #define HR_T0
 #endif
 
+// two consecutive elements (4- or 8-byte aligned) as floats
+__device__ __forceinline__ void load2(const __nv_bfloat16* p, float& a, float& b) {
+    const uint32_t raw = *reinterpret_cast<const uint32_t*>(p);
+    a = __uint_as_float(raw << 16);
+    b = __uint_as_float(raw & 0xFFFF0000u);
+}
+__device__ __forceinline__ void load2(const float* p, float& a, float& b) {
+    const float2 f = *reinterpret_cast<const float2*>(p);
+    a = f.x;
+    b = f.y;
+}
+
 template <int D, int DV, typename TIn, typename TOut>
-__global__ void __launch_bounds__(HR_THREADS, (D <= 64 ? 4 : 1))
+__global__ void __launch_bounds__(HrCfg<D>::THREADS, HrCfg<D>::BLOCKS_PER_SM)
 head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
                  TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
@@ -89,13 +110,14 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
     // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
     using C = HrCfg<D>;
-    extern __shared__ double smem[];
-    double* S = smem;                       // D * LDS
-    double* qd = S + D * C::LDS;            // D
+    constexpr int HR_THREADS = C::THREADS;
+    extern __shared__ __align__(16) double smem[];
+    double* S = smem;                       // D * LDS (S_DOUBLES reserved)
+    double* qd = S + C::S_DOUBLES;          // D
     double* rhs = qd + D;                   // D  (mu, then rho)
     double* w = rhs + D;                    // lcap (scores -> weights -> coefficients)
-    double* zc = w + lcap;                  // HR_CHUNK * D  centred keys of the current chunk
-    double* red = zc + HR_CHUNK * D;        // HR_THREADS/32 + 1
+    double* red = w + ((lcap + 1) & ~1);    // HR_THREADS/32 + 1
+    double* zc = S;                         // HR_CHUNK * D  centred keys of the current chunk (over S)
 
     const int tid = threadIdx.x;
     const int bh = blockIdx.y;
@@ -123,14 +145,14 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         lmax = fmax(lmax, s);
     }
     HR_T(0);
-    const double m = block_reduce(lmax, true, red);
+    const double m = block_reduce<HR_THREADS>(lmax, true, red);
     double lsum = 0.0;
     for (int j = tid; j < L; j += HR_THREADS) {
         const double e = exp(w[j] - m);
         w[j] = e;
         lsum += e;
     }
-    const double omega = block_reduce(lsum, false, red);
+    const double omega = block_reduce<HR_THREADS>(lsum, false, red);
     const double lambda_m = lambda * exp(-m);
     HR_T(1);
 
@@ -155,14 +177,32 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
             for (int b = 0; b < 4; ++b) acc[t][a][b] = 0.0;
     }
     double mu_acc = 0.0;  // thread tid < D owns mu[tid]
+    // The keys of a chunk are fetched (element pairs, coalesced) one chunk ahead, so the global-load
+    // latency hides behind the accumulation of the chunk before.
+    constexpr int PAIRS = (HR_CHUNK * D / 2 + HR_THREADS - 1) / HR_THREADS;
+    float pre[PAIRS][2];
+    auto fetch = [&](int j0) {
+        const int np = min(HR_CHUNK, L - j0) * (D / 2);
+#pragma unroll
+        for (int u = 0; u < PAIRS; ++u) {
+            const int pi = tid + HR_THREADS * u;
+            if (pi < np) load2(kb + (size_t)j0 * D + 2 * pi, pre[u][0], pre[u][1]);
+        }
+    };
+    fetch(0);
     for (int j0 = 0; j0 < L; j0 += HR_CHUNK) {
         const int jn = min(HR_CHUNK, L - j0);
         __syncthreads();
-        for (int e = tid; e < jn * D; e += HR_THREADS) {
-            const int jj = e / D, c = e - jj * D;
-            zc[jj * D + c] = (double)to_f32(kb[(size_t)(j0 + jj) * D + c]) - qd[c];
+#pragma unroll
+        for (int u = 0; u < PAIRS; ++u) {
+            const int pi = tid + HR_THREADS * u;
+            if (pi < jn * (D / 2)) {
+                const int c = (2 * pi) % D;
+                *reinterpret_cast<double2*>(zc + 2 * pi) = make_double2((double)pre[u][0] - qd[c], (double)pre[u][1] - qd[c + 1]);
+            }
         }
         __syncthreads();
+        if (j0 + HR_CHUNK < L) fetch(j0 + HR_CHUNK);
         if (tid < D)
             for (int jj = 0; jj < jn; ++jj) mu_acc += w[j0 + jj] * zc[jj * D + tid];
 #pragma unroll
@@ -187,6 +227,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         }
     }
     HR_T(2);
+    __syncthreads();   // the staged keys (lying over S) are no longer read
 #pragma unroll
     for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
         if (tr[t] < 0) continue;
@@ -221,7 +262,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         w[j] = cj;
         csum += cj;
     }
-    const double denom = block_reduce(csum, false, red);
+    const double denom = block_reduce<HR_THREADS>(csum, false, red);
     HR_T(5);
     for (int c = tid; c < DV; c += HR_THREADS) {
         double o = 0.0;
@@ -244,13 +285,12 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
 template <int D, typename TIn, typename TOut>
 int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     using C = HrCfg<D>;
-    const size_t smem = sizeof(double) *
-        ((size_t)D * C::LDS + 2 * D + lcap + (size_t)HR_CHUNK * D + HR_THREADS / 32 + 1);
+    const size_t smem = sizeof(double) * C::smem_doubles(lcap);
     auto kern = head_rows_kernel<D, D, TIn, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     dim3 grid(rows_per_head, a.B * a.H);
-    kern<<<grid, HR_THREADS, smem, a.stream>>>(
+    kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
         (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H);
     LLA_CUDA_TRY(cudaGetLastError());
@@ -260,13 +300,12 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
 template <int D, typename TIn, typename TOut>
 int launch_decode_t(const DecodeArgs& a, int lcap) {
     using C = HrCfg<D>;
-    const size_t smem = sizeof(double) *
-        ((size_t)D * C::LDS + 2 * D + lcap + (size_t)HR_CHUNK * D + HR_THREADS / 32 + 1);
+    const size_t smem = sizeof(double) * C::smem_doubles(lcap);
     auto kern = head_rows_kernel<D, D, TIn, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
     dim3 grid(1, a.B * a.H);
-    kern<<<grid, HR_THREADS, smem, a.stream>>>(
+    kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
         (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H);
     LLA_CUDA_TRY(cudaGetLastError());
