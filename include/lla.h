@@ -152,7 +152,10 @@ int lla_forward_ex(const lla_forward_params *p);
  *               caches spread over more thread blocks (0 = chosen from B*H and Lmax; 1 = none).
  *               With splits > 1 partial moments go through `workspace`.
  *   workspace : device scratch of at least lla_decode_workspace_bytes(...) bytes, 256-byte
- *               aligned; required when the effective number of splits exceeds 1
+ *               aligned; required when the effective number of splits exceeds 1.  Unsplit, it
+ *               is optional: given one, the tensor-core path (bf16, d = dv = 64) writes each
+ *               (sequence, head)'s moments there and solves in a second kernel, which is faster
+ *               than solving at the end of the streaming kernel; the result is the same.
  */
 typedef struct lla_decode_params {
     const void *q, *kcache, *vcache;
@@ -204,7 +207,7 @@ int lla_decode_host(const void *q, const void *kcache, const void *vcache, const
  * any stream capture.
  *
  * Arguments are those of lla_decode plus the dtypes and `splits` (0 = the default of
- * lla_decode_default_splits; 1 = no split, which uses no scratch at all).  All tensor pointers are
+ * lla_decode_default_splits; 1 = no split, which uses the array only if the records fit).  All tensor pointers are
  * device pointers owned by the caller.
  * Errors: LLA_ERR_WORKSPACE if B*H*splits partial records do not fit in the fixed array
  * (lla_decode_workspace_bytes(...) > LLA_NOALLOC_SCRATCH_BYTES): use fewer splits or lla_decode_ex
@@ -213,7 +216,7 @@ int lla_decode_host(const void *q, const void *kcache, const void *vcache, const
  * reads, so nothing needs clearing between calls, but two calls whose kernels may run at the same
  * time (different streams, or different host threads) race on it: serialise them.
  */
-#define LLA_NOALLOC_SCRATCH_BYTES (32u << 20)
+#define LLA_NOALLOC_SCRATCH_BYTES (64u << 20)
 int lla_decode_noalloc(const void *q, const void *kcache, const void *vcache, const int *lens,
                        void *out, int B, int H, int Lmax, int d, int dv, int in_dtype,
                        int out_dtype, float scale, float lambda, int splits, void *stream);
@@ -224,7 +227,8 @@ int lla_decode_noalloc(const void *q, const void *kcache, const void *vcache, co
  * later ones; blocks address it by SM id, so concurrent calls may share it). */
 size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl);
 
-/* Scratch bytes lla_decode_ex needs for this problem and split count (0 when splits <= 1). */
+/* Scratch bytes lla_decode_ex uses for this problem and split count: required when splits > 1,
+ * optional (see lla_decode_params.workspace; 0 where it would not be used) when splits <= 1. */
 size_t lla_decode_workspace_bytes(int B, int H, int Lmax, int d, int dv, int in_dtype, int splits);
 
 /* Number of key-range parts lla_decode / lla_decode_ex(splits = 0) would use. */

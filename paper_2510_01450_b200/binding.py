@@ -176,14 +176,14 @@ def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, i
     _check(load().lla_decode_ex(ctypes.byref(p)), "lla_decode_ex")
 
 
-NOALLOC_SCRATCH_BYTES = 32 << 20
+NOALLOC_SCRATCH_BYTES = 64 << 20
 
 
 def lla_decode_noalloc(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, in_dtype=LLA_BF16,
                        out_dtype=LLA_BF16, splits=0, stream=0):
     """Split-key decode for callers that may not allocate device memory (a pre-planned serving loop,
     a host framework that forbids cudaMalloc after start-up): the partial moments live in a fixed
-    32 MiB array inside the library instead of a workspace.  Raises LlaError(status 3) when
+    64 MiB array inside the library instead of a workspace.  Raises LlaError(status 3) when
     B*H*splits records do not fit.  Calls that may overlap on the GPU race on that array."""
     _check(load().lla_decode_noalloc(_p(q), _p(kcache), _p(vcache), _p(lens), _p(out), B, H, Lmax, d, dv,
                                      in_dtype, out_dtype, scale, lam, splits, _p(stream)), "lla_decode_noalloc")

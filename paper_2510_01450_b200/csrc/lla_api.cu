@@ -86,6 +86,19 @@ int check_decode(const lla_decode_params* p) {
     return LLA_OK;
 }
 
+void keep_pool_memory() {
+    // let the stream-ordered pool keep freed blocks so repeated host-buffer calls do not re-allocate
+    static bool done = false;
+    if (done) return;
+    int dev = 0;
+    cudaMemPool_t pool;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+        unsigned long long keep = ~0ull;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    }
+    done = true;
+}
+
 }  // namespace
 
 extern "C" {
@@ -192,7 +205,22 @@ int lla_decode(const void* q, const void* kcache, const void* vcache, const int*
     p.in_dtype = LLA_BF16; p.out_dtype = LLA_BF16;
     p.scale = scale; p.lambda = lambda;
     p.stream = stream;
-    return lla_decode_ex(&p);
+    // scratch for the moment records comes from the stream-ordered pool (kept warm between calls)
+    p.splits = 1;
+    const size_t ws = lla_decode_workspace_bytes(B, H, Lmax, d, dv, LLA_BF16, 1);
+    void* scratch = nullptr;
+    if (ws > 0 && B > 0 && H > 0) {
+        keep_pool_memory();
+        if (cudaMallocAsync(&scratch, ws, (cudaStream_t)stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            scratch = nullptr;          // fall back to the fused epilogue
+        }
+    }
+    p.workspace = scratch;
+    p.workspace_bytes = scratch ? ws : 0;
+    const int rc = lla_decode_ex(&p);
+    if (scratch) (void)cudaFreeAsync(scratch, (cudaStream_t)stream);
+    return rc;
 }
 
 int lla_decode_f32(const void* q, const void* kcache, const void* vcache, const int* lens, void* out,
@@ -212,9 +240,12 @@ size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dt
 }
 
 size_t lla_decode_workspace_bytes(int B, int H, int Lmax, int d, int dv, int in_dtype, int splits) {
-    (void)Lmax; (void)in_dtype;
+    (void)Lmax;
     if (B < 1 || H < 1 || d < 1 || dv < 1) return 0;
-    return lla::decode_workspace_bytes(B, H, d, dv, splits);
+    if (splits > 1) return lla::decode_workspace_bytes(B, H, d, dv, splits);
+    // unsplit: optional.  The tensor-core path (bf16, d = dv = 64) uses it to run the solve as a
+    // second kernel; without it the call still works (the streaming kernel solves in its epilogue).
+    return (in_dtype == LLA_BF16 && d == 64 && dv == 64) ? lla::decode_record_bytes(B, H, d, dv, 1) : 0;
 }
 
 const char* lla_status_string(int status) {
@@ -251,19 +282,6 @@ struct DeviceScratch {   // stream-ordered allocations released on scope exit
         for (int i = 0; i < count; ++i) cudaFreeAsync(ptrs[i], stream);
     }
 };
-
-void keep_pool_memory() {
-    // let the stream-ordered pool keep freed blocks so repeated host-buffer calls do not re-allocate
-    static bool done = false;
-    if (done) return;
-    int dev = 0;
-    cudaMemPool_t pool;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
-        unsigned long long keep = ~0ull;
-        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
-    }
-    done = true;
-}
 
 }  // namespace
 
@@ -319,6 +337,11 @@ int lla_decode_host(const void* q, const void* kcache, const void* vcache, const
     void* dq = mem.get(nq); void* dk = mem.get(nk); void* dvv = mem.get(nv);
     void* dl = mem.get(sizeof(int) * (size_t)B); void* dout = mem.get(no);
     if (!dq || !dk || !dvv || !dl || !dout) return LLA_ERR_CUDA;
+    const size_t ws = lla_decode_workspace_bytes(B, H, Lmax, d, dv, in_dtype, 1);
+    if (ws > 0) {
+        p.workspace = mem.get(ws);
+        p.workspace_bytes = p.workspace ? ws : 0;
+    }
     LLA_CUDA_TRY(cudaMemcpyAsync(dq, q, nq, cudaMemcpyHostToDevice, st));
     LLA_CUDA_TRY(cudaMemcpyAsync(dl, lens, sizeof(int) * (size_t)B, cudaMemcpyHostToDevice, st));
     // only the live prefix of every (sequence, head) cache crosses the bus

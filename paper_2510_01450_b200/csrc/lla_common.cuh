@@ -61,7 +61,8 @@ int launch_decode(const DecodeArgs& a);
 int launch_head_rows_decode(const DecodeArgs& a);
 bool decode_tensor_supported(const DecodeArgs& a);
 int launch_decode_tensor_moments(const DecodeArgs& a);
-size_t decode_workspace_bytes(int B, int H, int d, int dv, int splits);
+size_t decode_workspace_bytes(int B, int H, int d, int dv, int splits);   // required bytes (0 when unsplit)
+size_t decode_record_bytes(int B, int H, int d, int dv, int splits);      // moment records of all parts
 
 // ---------------------------------------------------------------------------------------------
 // Element access

@@ -275,9 +275,8 @@ int launch_t(const DecodeArgs& a) {
         if (!a.workspace || a.workspace_bytes < need) return LLA_ERR_WORKSPACE;
     }
     if (a.impl != LLA_IMPL_SIMT && decode_tensor_supported(a)) {
-        // moment pass on tensor cores (writes the same partial records when splits > 1)
-        const int st = launch_decode_tensor_moments(a);
-        if (st != LLA_OK) return st;
+        // tensor-core path: streaming kernel plus its own solve kernel (or fused epilogue)
+        return launch_decode_tensor_moments(a);
     } else {
         if (a.impl == LLA_IMPL_TENSOR) return LLA_ERR_UNSUPPORTED;
         auto k1 = decode_moments_kernel<D, TIn, TOut>;
@@ -307,6 +306,11 @@ int launch_d(const DecodeArgs& a) {
 }
 
 }  // namespace
+
+size_t decode_record_bytes(int B, int H, int d, int dv, int splits) {
+    (void)dv;
+    return sizeof(float) * (size_t)B * H * (splits < 1 ? 1 : splits) * (2 * (size_t)d * d + 2 * d + 4);
+}
 
 size_t decode_workspace_bytes(int B, int H, int d, int dv, int splits) {
     if (splits <= 1) return 0;
@@ -375,9 +379,11 @@ extern "C" int lla_decode_noalloc(const void* q, const void* kcache, const void*
     a.status = nullptr;
     a.workspace = nullptr; a.workspace_bytes = 0;
     a.stream = (cudaStream_t)stream;
-    if (a.splits > 1) {
-        const size_t need = lla::decode_workspace_bytes(B, H, d, dv, a.splits);
-        if (need > (size_t)LLA_NOALLOC_SCRATCH_BYTES) return LLA_ERR_WORKSPACE;   // beyond the fixed array
+    // records are required for a split decode and optional otherwise (they let the tensor-core path
+    // run its solve as a separate kernel)
+    const size_t need = lla::decode_record_bytes(B, H, d, dv, a.splits);
+    if (a.splits > 1 && need > (size_t)LLA_NOALLOC_SCRATCH_BYTES) return LLA_ERR_WORKSPACE;   // beyond the fixed array
+    if (need <= (size_t)LLA_NOALLOC_SCRATCH_BYTES) {
         void* scratch = nullptr;
         const int rc = lla::noalloc_scratch_ptr(&scratch);
         if (rc != LLA_OK) return rc;

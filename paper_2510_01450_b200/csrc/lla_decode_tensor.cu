@@ -11,7 +11,9 @@
 //   CUDA cores  two lanes per key: score s_j = scale q.k_j, weight w_j = exp(s_j - m_ref), then the
 //               row w_j [k_j | 1] split into bf16 hi + lo is written to the B operand tiles
 //               (canonical MN-major layout without swizzle, 80 columns); omega += w_j.
-//   MMA (SS)    D += A B_hi + A B_lo, four 16-key steps each.
+//   MMA (SS)    [D_hi | D_lo] += A [B_hi | B_lo]: the two B tiles lie back to back and are read as one
+//               N = 160 operand, so A is fetched once per 16-key step; D = D_hi + D_lo is formed
+//               when the accumulator is read out.
 // m_ref is the maximum of the first tile; if a later tile's maximum exceeds it by more than 2^40 the
 // accumulator is rescaled in TMEM (never triggered by bounded scores, covered by a test).  After
 // the last tile the moments are copied to shared memory and either solved on the spot (d x d LDL^T
@@ -31,7 +33,7 @@ constexpr int DT_BK = 64;             // keys per tile
 constexpr int DT_NST = 4;             // K/V ring stages
 constexpr int DT_COMPUTE = 128;       // warps 0..3
 constexpr int DT_THREADS = 192;       // + TMA warp (4) + MMA warp (5)
-constexpr int DT_TMEM_COLS = 128;
+constexpr int DT_TMEM_COLS = 256;     // 160 accumulator columns (hi | lo), power-of-two allocation
 constexpr int DT_N = 80;              // MMA N: 64 key features + the ones column (padded to 16)
 constexpr int DT_MAX_RANKED = 1024;   // batches up to this size are processed longest-first
 constexpr int DT_BTILE = 10240;       // one B tile: 10 column blocks x 8 key blocks x 128 bytes
@@ -70,38 +72,33 @@ __device__ __forceinline__ uint64_t make_desc_b(uint32_t addr) {
     d |= (uint64_t)1 << 46;
     return d;                    // layout type 0: no swizzle
 }
-constexpr uint32_t IDESC_DEC = make_idesc(128, DT_N, 1, 1);
+constexpr uint32_t IDESC_DEC = make_idesc(128, 2 * DT_N, 1, 1);
 
-// D += A B_hi + A B_lo over 64 keys.  A steps 2048 bytes (128 units) per 16 keys, B 256 bytes (16 units).
-__device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, uint64_t bhi, uint64_t blo, uint32_t acc0) {
+// [D_hi | D_lo] += A [B_hi | B_lo] over 64 keys.  A steps 2048 bytes (128 units) per 16 keys, B 256 bytes (16 units).
+__device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, uint64_t b, uint32_t acc0) {
     asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, h1, h2, h3, l1, l2, l3;\n\t"
-        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, h1, h2, h3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
         "add.u64 a1, %2, 128; add.u64 a2, %2, 256; add.u64 a3, %2, 384;\n\t"
         "add.u64 h1, %3, 16; add.u64 h2, %3, 32; add.u64 h3, %3, 48;\n\t"
-        "add.u64 l1, %4, 16; add.u64 l2, %4, 32; add.u64 l3, %4, 48;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %5, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
         "setp.ne.b32 p, 1, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %4, %5, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, h1, %5, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, l1, %5, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, h2, %5, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, l2, %5, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, h3, %5, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, l3, %5, p;\n\t}"
-        ::"r"(el), "r"(d), "l"(a), "l"(bhi), "l"(blo), "r"(IDESC_DEC), "r"(acc0) : "memory");
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, h1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, h2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, h3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "l"(a), "l"(b), "r"(IDESC_DEC), "r"(acc0) : "memory");
 }
 
-// Solve C x = b for an explicit symmetric positive-definite 64 x 64 matrix in shared memory (row
-// stride 65 doubles, both triangles filled) with conjugate gradients in double precision, run by
-// the 128 threads of warps 0..3 (two threads per row, 32 columns each).  A dense factorisation is a
+// Solve C x = b for an explicit symmetric positive-definite 64 x 64 matrix with conjugate gradients in
+// double precision, run by the 128 threads of warps 0..3: thread 2r + hh holds columns 32hh..32hh+31
+// of row r in cr[] and passes b[r].  A dense factorisation is a
 // chain of 64 dependent column steps, each with block barriers; here an iteration is one short
 // matrix-vector product and three 128-thread barriers, and the decode systems (>= 2d keys) need one
 // or two dozen iterations.  Each thread keeps its 32 matrix entries in registers for the whole
 // solve: re-reading the matrix from shared memory every iteration costs several times more than
 // the arithmetic while the SM's other block is streaming its cache through the same memory.  x lands in xs[]; returns false if the residual did not reach 1e-9 |b|
 // within the iteration cap (the caller then falls back to the factorisation).  C is not modified.
-__device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, double* xs, double* pbuf, double* redbuf, int& iters) {
+__device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double b_r, double* xs, double* pbuf, double* redbuf, int& iters) {
     const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
     const int r = tid >> 1, hh = tid & 1;
     auto sync128 = [&]() { asm volatile("bar.sync 2, 128;" ::: "memory"); };
@@ -113,13 +110,7 @@ __device__ __forceinline__ bool cg_solve_64(const double* C, const double* b, do
         sync128();
         return (redbuf[slot * 4] + redbuf[slot * 4 + 1]) + (redbuf[slot * 4 + 2] + redbuf[slot * 4 + 3]);
     };
-    double cr[32];
-    {
-        const double* crow = C + r * 65 + 32 * hh;
-#pragma unroll
-        for (int c = 0; c < 32; ++c) cr[c] = crow[c];
-    }
-    double x = 0.0, res = b[r], pv = res;
+    double x = 0.0, res = b_r, pv = res;
     if (hh == 0) pbuf[r] = pv;
     double rr = block_sum(res * res, 0);
     const double stop = rr * 1e-18;     // |r| <= 1e-9 |b|: far below what a bf16 or fp32 output resolves
@@ -176,6 +167,7 @@ struct DtParams {
     const int* lens;
     float* parts;
     int* status;
+    int defer;           // 1: write the moment record even for a single part; a solve kernel follows
 };
 
 template <typename TOut>
@@ -266,7 +258,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             tc_fence_after();
             const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
 #ifndef LLA_DEXP_NOMMA
-            mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), make_desc_b(bsm + DT_BTILE), t > 0);
+            mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), t > 0);
 #endif
             tc_commit_el(el, bar(DB_KVEMPTY + s));
             tc_commit_el(el, bar(DB_BFREE + b));
@@ -300,10 +292,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 raw[i] = *reinterpret_cast<const uint4*>(ktile + jl * 128 + (((4 * h + i) ^ (jl & 7)) << 4));
             return true;
         };
-        auto stage_score = [&](int t) -> bool {
+        float s2 = 0.f;
+        bool valid = false;
+        // first half of the score stage: arithmetic only (no barrier), so it can run while the
+        // stores of the tile before are still draining
+        auto stage_score_math = [&](int t) {
             const uint32_t s = t % DT_NST;
             uint8_t* ktile = smem + SMD_KV + s * 16384;
-            const bool valid = jbeg + t * DT_BK + jl < jend;
+            valid = jbeg + t * DT_BK + jl < jend;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint32_t wds[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
@@ -330,7 +326,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             for (int e = 0; e < 32; ++e) sd[e & 3] = fmaf(qv[e], kf[e], sd[e & 3]);
             float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
             sdot += __shfl_xor_sync(0xffffffffu, sdot, 1);
-            const float s2 = valid ? sdot * c1 : -INFINITY;
+            s2 = valid ? sdot * c1 : -INFINITY;
+        };
+        // second half: the block-wide rescale check and the weight
+        auto stage_score_sync = [&](int t) -> bool {
             // The reference maximum is the first tile's.  Later tiles only need to know whether any
             // score exceeds it by more than 2^40 (then the accumulator is rescaled): one barrier
             // that ORs a predicate over the 128 compute threads answers that; the tile maximum
@@ -364,7 +363,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tc_fence_after();
                 const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
 #pragma unroll 1
-                for (int cb = 0; cb < 96; cb += 32) {
+                for (int cb = 0; cb < 2 * DT_N; cb += 32) {
                     uint32_t v[32];
                     tmem_ld32(lane_addr + cb, v);
                     tc_wait_ld();
@@ -382,7 +381,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (h == 0) omega += w;
             return true;
         };
-        if (ntile > 0) ok = stage_load(0) && stage_score(0);
+        if (ntile > 0) {
+            ok = stage_load(0);
+            if (ok) {
+                stage_score_math(0);
+                ok = stage_score_sync(0);
+            }
+        }
         DT_T0;
         for (int t = 0; t < ntile && ok; ++t) {
             const uint32_t b = t & 1;
@@ -425,10 +430,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
                 *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
             }
+            // the next tile's score arithmetic fills the time the stores need to drain
+            if (more) stage_score_math(t + 1);
             fence_proxy_async();
             mbar_arrive(bar(DB_BFULL + b));
             DT_T(3);
-            if (more && !stage_score(t + 1)) { ok = false; break; }
+            if (more && !stage_score_sync(t + 1)) { ok = false; break; }
             DT_T(4);
         }
         // total weight of this part
@@ -455,6 +462,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (warp < 4) {
         if (ntile > 0 && d_ok) {
             const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+            // columns 0..79 hold D_hi, 80..159 D_lo; dv[e] = D_hi[e] + D_lo[e] for the 65 columns in use
 #pragma unroll
             for (int cb = 0; cb < 96; cb += 32) {
                 uint32_t v[32];
@@ -462,6 +470,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tc_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) dv[cb + e] = __uint_as_float(v[e]);
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) dv[e] += dv[80 + e];            // D_lo[0..15] sat in columns 80..95
+#pragma unroll
+            for (int cb = 96; cb < 160; cb += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + cb, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) dv[cb - 80 + e] += __uint_as_float(v[e]);   // D_lo[16..79]
             }
         } else {
 #pragma unroll
@@ -485,8 +503,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const float omega_tot = s_omega[0] + s_omega[1] + s_omega[2] + s_omega[3];
     const float mref_ln = s_mref * 0.6931471805599453f;          // back to natural-log units
 
-    if (prm.splits > 1) {
-        // partial record for the merge kernel: M, N, a, c, omega, m (same layout as the SIMT path)
+    if (prm.splits > 1 || prm.defer) {
+        // partial record for the solve kernel: M, N, a, c, omega, m (same layout as the SIMT path)
         float* dst = prm.parts + ((size_t)bh * prm.splits + part) * (2 * 64 * 64 + 2 * 64 + 4);
         if (warp < 4) {
             float* rowp = dst + (size_t)tid * 64;                 // tid < 64: M rows; 64..127: N rows
@@ -539,7 +557,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __shared__ int s_cg_ok;
     if (warp < 4) {
         int cg_its = 0;
-        const bool okc = cg_solve_64(Md, rhs, xs, xs + 64, xs + 128, cg_its);
+        double cr[32];
+        {
+            const double* crow = Md + (tid >> 1) * 65 + 32 * (tid & 1);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) cr[c] = crow[c];
+        }
+        const bool okc = cg_solve_64(cr, rhs[tid >> 1], xs, xs + 64, xs + 128, cg_its);
         if (tid == 0) {
             s_cg_ok = okc ? 1 : 0;
             if (prm.status) atomicAdd(prm.status + LLA_STATUS_ITER_SUM, cg_its);
@@ -563,13 +587,100 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (!solved && tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_BAD_PIVOT, 1);
 }
 
+// Second kernel of the two-kernel decode: merge the parts' moment records of one (sequence, head),
+// centre them, solve and emit the output row.  Everything a thread needs of the two matrices goes
+// straight from the records (L2) into registers, so a block holds almost no shared memory and several
+// of them share an SM; the solve itself is latency-bound (barriers and shuffles), which is why it is
+// kept out of the streaming kernel whenever the caller provides the record buffer.
+constexpr int DS_MAX_SPLITS = 64;
+template <typename TOut>
+__global__ void __launch_bounds__(DT_COMPUTE, 4)
+decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict__ parts, TOut* __restrict__ out,
+                    const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
+                    int* __restrict__ status) {
+    constexpr int D = DT_D, PF = 2 * D * D + 2 * D + 4;
+    __shared__ double s_a[D], s_c[D], s_x[D], s_p[D], s_red[24];
+    __shared__ double s_f[DS_MAX_SPLITS];
+    __shared__ double s_L[D * 65];          // only touched by the factorisation fallback
+    const int tid = threadIdx.x, r = tid >> 1, hh = tid & 1, bh = blockIdx.x;
+    if (max(1, min(lens[bh / H], Lmax)) < head_rows) return;
+    const float* src = parts + (size_t)bh * splits * PF;
+    float m = -INFINITY;
+    for (int p = 0; p < splits; ++p) m = fmaxf(m, src[(size_t)p * PF + 2 * D * D + 2 * D + 1]);
+    for (int p = tid; p < splits; p += DT_COMPUTE)
+        s_f[p] = exp((double)src[(size_t)p * PF + 2 * D * D + 2 * D + 1] - (double)m);   // 0 for empty parts
+    __syncthreads();
+    double omega = 0.0;
+    for (int p = 0; p < splits; ++p) omega += s_f[p] * (double)src[(size_t)p * PF + 2 * D * D + 2 * D];
+    const double inv = 1.0 / omega;
+    const double ridge = (double)lambda * exp(-(double)m) * inv;
+    {
+        double s1 = 0.0;                     // thread e < 64: a[e]; thread 64 + e: c[e]
+        for (int p = 0; p < splits; ++p) s1 += s_f[p] * (double)src[(size_t)p * PF + 2 * D * D + tid];
+        if (tid < D) s_a[tid] = s1 * inv; else s_c[tid - D] = s1 * inv;
+    }
+    __syncthreads();
+    // this thread's half row of the centred matrix
+    double cr[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) cr[c] = 0.0;
+    for (int p = 0; p < splits; ++p) {
+        const float4* mp = reinterpret_cast<const float4*>(src + (size_t)p * PF + r * D + 32 * hh);
+        const double f = s_f[p];
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 v = mp[c4];
+            cr[4 * c4] += f * (double)v.x; cr[4 * c4 + 1] += f * (double)v.y;
+            cr[4 * c4 + 2] += f * (double)v.z; cr[4 * c4 + 3] += f * (double)v.w;
+        }
+    }
+    const double ar = s_a[r];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) cr[c] = cr[c] * inv - ar * s_a[32 * hh + c];
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+        if (32 * hh + c == r) cr[c] += ridge;
+    const double b_r = (double)to_f32(q[(size_t)bh * D + r]) - ar;
+    int cg_its = 0;
+    const bool okc = cg_solve_64(cr, b_r, s_x, s_p, s_red, cg_its);
+    if (tid == 0 && status) atomicAdd(status + LLA_STATUS_ITER_SUM, cg_its);
+    bool solved = true;
+    if (!okc) {        // uniform over the block: the decision comes from block-wide sums
+#pragma unroll
+        for (int c = 0; c < 32; ++c) s_L[r * 65 + 32 * hh + c] = cr[c];
+        if (hh == 0) s_x[r] = b_r;
+        solved = block_ldlt_solve<D>(s_L, 65, s_x);
+    }
+    // o_e = vbar_e + sum_f (N[e][f] / omega - vbar_e kbar_f) y_f, two threads per output element
+    double nr[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) nr[c] = 0.0;
+    for (int p = 0; p < splits; ++p) {
+        const float4* np_ = reinterpret_cast<const float4*>(src + (size_t)p * PF + D * D + r * D + 32 * hh);
+        const double f = s_f[p];
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 v = np_[c4];
+            nr[4 * c4] += f * (double)v.x; nr[4 * c4 + 1] += f * (double)v.y;
+            nr[4 * c4 + 2] += f * (double)v.z; nr[4 * c4 + 3] += f * (double)v.w;
+        }
+    }
+    const double cb = s_c[r];
+    double o = 0.0;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) o += (nr[c] * inv - cb * s_a[32 * hh + c]) * s_x[32 * hh + c];
+    o += __shfl_xor_sync(0xffffffffu, o, 1);
+    if (hh == 0) store_out(out + (size_t)bh * D + r, (float)(o + cb));
+    if (!solved && tid == 0 && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
+}
+
 template <typename TOut>
 int launch_t(const DecodeArgs& a) {
     const int splits = a.splits < 1 ? 1 : a.splits;
-    if (splits > 1) {
-        const size_t need = decode_workspace_bytes(a.B, a.H, a.d, a.dv, splits);
-        if (!a.workspace || a.workspace_bytes < need) return LLA_ERR_WORKSPACE;
-    }
+    const size_t need = sizeof(float) * (size_t)a.B * a.H * splits * (2 * 64 * 64 + 2 * 64 + 4);
+    const bool have_ws = a.workspace && a.workspace_bytes >= need && ((uintptr_t)a.workspace & 15u) == 0;
+    if (splits > 1 && !have_ws) return LLA_ERR_WORKSPACE;
+    if (splits > DS_MAX_SPLITS) return LLA_ERR_INVALID_ARG;
     CUtensorMap mk, mv;
     const int BH = a.B * a.H;
     if (!make_map_bf16_64(&mk, a.kcache, BH, a.Lmax, DT_BK) || !make_map_bf16_64(&mv, a.vcache, BH, a.Lmax, DT_BK))
@@ -578,6 +689,7 @@ int launch_t(const DecodeArgs& a) {
     prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
     prm.parts = (float*)a.workspace; prm.status = a.status;
+    prm.defer = have_ws ? 1 : 0;      // with a record buffer the solve runs as its own kernel
     auto kern = decode_tc_kernel<TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMD_ALLOC));
     // two blocks per SM need the largest shared-memory carve-out
@@ -585,6 +697,12 @@ int launch_t(const DecodeArgs& a) {
     dim3 grid(splits, BH);
     kern<<<grid, DT_THREADS, SMD_ALLOC, a.stream>>>(mk, mv, (const __nv_bfloat16*)a.q, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());
+    if (have_ws) {
+        decode_solve_kernel<TOut><<<BH, DT_COMPUTE, 0, a.stream>>>((const __nv_bfloat16*)a.q, (const float*)a.workspace,
+                                                                   (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows,
+                                                                   a.lambda, splits, a.status);
+        LLA_CUDA_TRY(cudaGetLastError());
+    }
     return LLA_OK;
 }
 
@@ -594,7 +712,9 @@ bool decode_tensor_supported(const DecodeArgs& a) {
     return a.in_dtype == LLA_BF16 && a.d == DT_D && a.dv == DT_D && sm100::get_encode() != nullptr;
 }
 
-// Moment pass on tensor cores; with splits > 1 the caller still runs the merge kernel afterwards.
+// Tensor-core decode.  With a record buffer (always for splits > 1, optional for a single part) the
+// streaming kernel writes moment records and a solve kernel follows; without one, single-part
+// blocks solve in their own epilogue.
 int launch_decode_tensor_moments(const DecodeArgs& a) {
     if (!decode_tensor_supported(a)) return LLA_ERR_UNSUPPORTED;
     if (a.out_dtype == LLA_BF16) return launch_t<__nv_bfloat16>(a);

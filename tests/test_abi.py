@@ -76,7 +76,10 @@ def test_argument_validation_without_device(lib):
 
 def test_workspace_and_split_arithmetic(lib):
     assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == 0
-    assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=1) == 0
+    # unsplit: optional record buffer for the two-kernel tensor-core path (bf16, d = 64), else none
+    assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=1) == 4 * 2 * 4 * (2 * 64 * 64 + 132)
+    assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, in_dtype=binding.LLA_F32, splits=1) == 0
+    assert binding.lla_decode_workspace_bytes(2, 4, 4096, 128, 128, splits=1) == 0
     assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=3) == 4 * 2 * 4 * 3 * (2 * 64 * 64 + 132)
     assert binding.lla_decode_default_splits(64, 16, 8192) == 1          # 1024 blocks already fill the chip
     assert binding.lla_decode_default_splits(1, 16, 8192) == 16          # 512-key floor

@@ -136,6 +136,12 @@ def test_decode_matches_oracle_and_splits_agree(oracle, dtype, d):
         torch.cuda.synchronize()
         err = row_err(out.cpu().numpy(), ref)
         assert err.max() <= tol, (splits, err.max())
+    # unsplit and without the optional record buffer (the streaming kernel then solves in its epilogue)
+    out1 = torch.full((w.B, w.H, d), float("nan"), dtype=torch.float32, device="cuda")
+    L.lla_decode_ex(dq, dk, dv_, dl, out1, w.B, w.H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                    out_dtype=L.LLA_F32, splits=1, stream=stream_ptr())
+    torch.cuda.synchronize()
+    assert row_err(out1.cpu().numpy(), ref).max() <= tol
     # decode of the last token equals the last prefill row on the same data
     np.testing.assert_allclose(out.cpu().numpy()[0], vc[0, :, 0], rtol=1e-5, atol=1e-6)
 

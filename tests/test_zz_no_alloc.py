@@ -51,7 +51,7 @@ def test_no_alloc_decode_matches_workspace_decode_twice(oracle):
 
 
 def test_no_alloc_rejects_what_does_not_fit():
-    # 64 x 16 (sequence, head) pairs x 8 parts of 33 KB each exceed the 32 MiB array: refused on the host
+    # 64 x 16 (sequence, head) pairs x 8 parts of 33 KB each exceed the 64 MiB array: refused on the host
     ok = 0x1000
     assert L.lla_decode_workspace_bytes(64, 16, 8192, 64, 64, L.LLA_BF16, 8) > L.NOALLOC_SCRATCH_BYTES
     with pytest.raises(L.LlaError) as e:
