@@ -8,7 +8,7 @@
 // Per 64-key tile:
 //   TMA         K and V tiles -> 128B-swizzled shared memory (4-stage ring).  The two tiles sit back
 //               to back and together form the MN-major A operand [K^T ; V^T] of one M = 128 MMA.
-//   CUDA cores  two lanes per key: score s_j = scale q.k_j, weight w_j = exp(s_j - m_ref), then the
+//   CUDA cores  two lanes per key (16 lanes apart): score s_j = scale q.k_j, weight w_j = exp(s_j - m_ref), then the
 //               row w_j [k_j | 1] split into bf16 hi + lo is written to the B operand tiles
 //               (canonical MN-major layout without swizzle, 80 columns); omega += w_j.
 //   MMA (SS)    [D_hi | D_lo] += A [B_hi | B_lo]: the two B tiles lie back to back and are read as one
@@ -161,6 +161,16 @@ __device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128
 #define DT_T(ph)
 #endif
 
+// Optional event trace of one block for tuning (-DLLA_DT_TRACE=<blockIdx.y>): (tag, tile, clock) int
+// triples per role in status[64 + 12000 * role ...].
+#ifdef LLA_DT_TRACE
+#define DT_EV_DECL(role) int* ev_p_ = (prm.status && blockIdx.y == LLA_DT_TRACE) ? prm.status + 64 + 12000 * (role) : nullptr; int ev_n_ = 0
+#define DT_EV(tag, c) do { if (ev_p_ && ev_n_ < 4000) { ev_p_[3 * ev_n_] = (tag); ev_p_[3 * ev_n_ + 1] = (int)(c); ev_p_[3 * ev_n_ + 2] = (int)clock64(); ++ev_n_; } } while (0)
+#else
+#define DT_EV_DECL(role)
+#define DT_EV(tag, c)
+#endif
+
 struct DtParams {
     int B, H, Lmax, splits, head_rows;
     float scale, lambda;
@@ -239,9 +249,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (warp == 4) {
         // ================================ TMA producer ================================
         if (lane == 0) {
+            DT_EV_DECL(0);
             for (int t = 0; t < ntile; ++t) {
                 const uint32_t s = t % DT_NST;
                 if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
+                DT_EV(1, t);
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
                 tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, bh);
@@ -251,10 +263,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     } else if (warp == 5) {
         // ================================ MMA issuer (whole warp, predicated) ================================
         const uint32_t el = elect_one();
+        DT_EV_DECL(1);
         for (int t = 0; t < ntile; ++t) {
             const uint32_t s = t % DT_NST, b = t & 1;
             if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) break;
+            if (lane == 0) DT_EV(9, t);
             if (!mbar_wait(bar(DB_BFULL + b), (t >> 1) & 1, abort_flag)) break;
+            if (lane == 0) DT_EV(10, t);
             tc_fence_after();
             const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
 #ifndef LLA_DEXP_NOMMA
@@ -263,10 +278,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             tc_commit_el(el, bar(DB_KVEMPTY + s));
             tc_commit_el(el, bar(DB_BFREE + b));
             if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
+            if (lane == 0) DT_EV(11, t);
         }
     } else {
         // ================================ compute warps ================================
-        const int jl = tid >> 1, h = tid & 1;            // key inside the tile, feature half
+        // key inside the tile and feature half: lanes 0..15 of a warp take the low halves of 16 keys,
+        // lanes 16..31 the high halves, so the eight lanes that share a 128-byte shared-memory wavefront
+        // have the same half and neighbouring keys (no bank conflicts in the tile loads or B stores)
+        const int jl = warp * 16 + (lane & 15), h = lane >> 4;
         const float c1 = prm.scale * 1.4426950408889634f;
         float qv[32];
         {
@@ -325,7 +344,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
             for (int e = 0; e < 32; ++e) sd[e & 3] = fmaf(qv[e], kf[e], sd[e & 3]);
             float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
-            sdot += __shfl_xor_sync(0xffffffffu, sdot, 1);
+            sdot += __shfl_xor_sync(0xffffffffu, sdot, 16);
             s2 = valid ? sdot * c1 : -INFINITY;
         };
         // second half: the block-wide rescale check and the weight
@@ -389,54 +408,56 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
         }
         DT_T0;
+        DT_EV_DECL(2);
         for (int t = 0; t < ntile && ok; ++t) {
+            if (tid == 0) DT_EV(19, t);
             const uint32_t b = t & 1;
             const bool more = t + 1 < ntile;
-            // B rows of tile t: w * [k | 1] as bf16 hi + lo, computed into registers first
-#ifdef LLA_DEXP_NOSIMT
-            if (more && !stage_load(t + 1)) { ok = false; break; }
-            if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            mbar_arrive(bar(DB_BFULL + b));
-            if (h == 0) omega += kf[0] + __uint_as_float(raw[1].x);
-            continue;
-#endif
-            uint32_t hi[16], lo[16];
-            const uint64_t ww = pk2(w, w);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                float a, bq;
-                upk2(mul2(ww, pk2(kf[2 * e], kf[2 * e + 1])), a, bq);
-                hi[e] = split_bf16x2(a, bq, lo[e]);
-            }
-            uint32_t wlo;
-            const uint32_t whi = split_bf16x2(w, 0.f, wlo);
-            DT_T(0);
-            // loads of the next tile go out now; they land while the stores below are issued
-            if (more && !stage_load(t + 1)) { ok = false; break; }
-            DT_T(1);
-            // wait until the MMA of tile t-2 has released this B buffer
+            // wait until the MMA of tile t-2 has released this B buffer (long done in steady state)
             if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
             DT_T(2);
+            if (tid == 0) DT_EV(21, t);
+            // B rows of tile t: w * [k | 1] as bf16 hi + lo, eight features at a time straight into the
+            // operand tiles, so the stores drain while the rest of the iteration runs
             uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
             uint8_t* blo = bhi + DT_BTILE;
+            const uint64_t ww = pk2(w, w);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float a, bq;
+                    upk2(mul2(ww, pk2(kf[8 * i + 2 * e], kf[8 * i + 2 * e + 1])), a, bq);
+                    hi[e] = split_bf16x2(a, bq, lo[e]);
+                }
                 const uint32_t off = (4 * h + i) * 1024 + rowoff;          // column block 4h+i
-                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
-                *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
             {   // column blocks 8 (ones column first) and 9 (zero padding)
+                uint32_t wlo;
+                const uint32_t whi = split_bf16x2(w, 0.f, wlo);
                 const uint32_t off = (8 + h) * 1024 + rowoff;
                 *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
                 *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
             }
-            // the next tile's score arithmetic fills the time the stores need to drain
+            DT_T(0);
+            // the next tile: shared-memory loads, then the score arithmetic, while the stores drain
+            if (more && !stage_load(t + 1)) { ok = false; break; }
+            DT_T(1);
+            if (tid == 0) DT_EV(20, t);
+            if (tid == 0) DT_EV(24, t);
             if (more) stage_score_math(t + 1);
+            if (tid == 0) DT_EV(25, t);
             fence_proxy_async();
+            if (tid == 0) DT_EV(26, t);
             mbar_arrive(bar(DB_BFULL + b));
             DT_T(3);
+            if (tid == 0) DT_EV(22, t);
             if (more && !stage_score_sync(t + 1)) { ok = false; break; }
             DT_T(4);
+            if (tid == 0) DT_EV(23, t);
         }
         // total weight of this part
         if (ok) {
