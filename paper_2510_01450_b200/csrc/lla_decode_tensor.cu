@@ -91,34 +91,36 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
 
 // Solve C x = b for an explicit symmetric positive-definite 64 x 64 matrix with conjugate gradients in
 // double precision, run by the 128 threads of warps 0..3: thread 2r + hh holds columns 32hh..32hh+31
-// of row r in cr[] and passes b[r].  A dense factorisation is a
-// chain of 64 dependent column steps, each with block barriers; here an iteration is one short
-// matrix-vector product and three 128-thread barriers, and the decode systems (>= 2d keys) need one
-// or two dozen iterations.  Each thread keeps its 32 matrix entries in registers for the whole
-// solve: re-reading the matrix from shared memory every iteration costs several times more than
-// the arithmetic while the SM's other block is streaming its cache through the same memory.  x lands in xs[]; returns false if the residual did not reach 1e-9 |b|
-// within the iteration cap (the caller then falls back to the factorisation).  C is not modified.
-__device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double b_r, double* xs, double* pbuf, double* redbuf, int& iters) {
+// of row r in cr[] and passes b[r].  A dense factorisation is a chain of 64 dependent column steps;
+// here an iteration is one short matrix-vector product and the decode systems (>= 2d keys) need one
+// or two dozen of them.  The matrix stays in registers for the whole solve (re-reading it from shared
+// memory every iteration costs several times more than the arithmetic).  The recurrences are the
+// Chronopoulos-Gear form: both inner products of an iteration, (r, r) and (C r, r), are taken after the
+// matrix-vector product, so an iteration has one reduction and two 128-thread barriers.
+// x lands in xs[]; returns false if the residual did not reach 1e-9 |b| within the iteration cap or the
+// recurrence broke down (the caller then falls back to the factorisation).
+#ifdef LLA_DT_TIMING
+#define CG_TARG , int* tstat = nullptr
+#else
+#define CG_TARG
+#endif
+__device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double b_r, double* xs, double* pbuf, double* redbuf, int& iters CG_TARG) {
     const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
     const int r = tid >> 1, hh = tid & 1;
     auto sync128 = [&]() { asm volatile("bar.sync 2, 128;" ::: "memory"); };
-    auto block_sum = [&](double v, int slot) {       // v is counted once per row (hh == 0 lanes)
-        v = hh == 0 ? v : 0.0;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-        if (lane == 0) redbuf[slot * 4 + wp] = v;
-        sync128();
-        return (redbuf[slot * 4] + redbuf[slot * 4 + 1]) + (redbuf[slot * 4 + 2] + redbuf[slot * 4 + 3]);
-    };
-    double x = 0.0, res = b_r, pv = res;
-    if (hh == 0) pbuf[r] = pv;
-    double rr = block_sum(res * res, 0);
-    const double stop = rr * 1e-18;     // |r| <= 1e-9 |b|: far below what a bf16 or fp32 output resolves
-    bool done = !(rr > 0.0);
-    int slot = 1;
+    double x = 0.0, rv = b_r, pv = 0.0, sv = 0.0, alpha = 0.0, gamma_old = 0.0, stop = 0.0;
+    bool done = false;
     iters = 0;
-    for (int it = 0; it < LLA_CG_CAP && !done; ++it) {
-        ++iters;
+#ifdef LLA_DT_TIMING
+    long long cgt_[5] = {0, 0, 0, 0, 0}, cg0_ = clock64();
+#define CG_T(i) do { const long long n_ = clock64(); cgt_[i] += n_ - cg0_; cg0_ = n_; } while (0)
+#else
+#define CG_T(i)
+#endif
+    for (int it = 0; it <= LLA_CG_CAP; ++it) {
+        if (hh == 0) pbuf[r] = rv;
+        sync128();
+        CG_T(0);
         const double2* pp = reinterpret_cast<const double2*>(pbuf + 32 * hh);
         double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
 #pragma unroll
@@ -129,22 +131,43 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
             a2 = fma(cr[c + 2], p23.x, a2);
             a3 = fma(cr[c + 3], p23.y, a3);
         }
-        double ap = (a0 + a1) + (a2 + a3);
-        ap += __shfl_xor_sync(0xffffffffu, ap, 1);
-        const double pap = block_sum(pv * ap, slot);
-        slot = slot % 5 + 1;
-        if (!(pap > 0.0)) break;
-        const double alpha = rr * fast_rcp(pap);
-        x += alpha * pv;
-        res -= alpha * ap;
-        const double rr2 = block_sum(res * res, slot);
-        slot = slot % 5 + 1;
-        pv = res + (rr2 * fast_rcp(rr)) * pv;
-        rr = rr2;
-        done = rr <= stop;
-        if (hh == 0) pbuf[r] = pv;
+        double wv = (a0 + a1) + (a2 + a3);
+        wv += __shfl_xor_sync(0xffffffffu, wv, 1);           // both lanes of a row now hold (C r)_row
+        CG_T(1);
+        // (r, r) and (C r, r): each parity class of lanes sums the warp's 16 rows once
+        double g = rv * rv, dl = wv * rv;
+#pragma unroll
+        for (int off = 2; off <= 16; off <<= 1) {
+            g += __shfl_xor_sync(0xffffffffu, g, off);
+            dl += __shfl_xor_sync(0xffffffffu, dl, off);
+        }
+        CG_T(2);
+        double* rb = redbuf + (it & 1) * 8;
+        if (lane == 0) { rb[wp] = g; rb[4 + wp] = dl; }
         sync128();
+        const double gamma = (rb[0] + rb[1]) + (rb[2] + rb[3]);
+        const double delta = (rb[4] + rb[5]) + (rb[6] + rb[7]);
+        CG_T(3);
+        if (it == 0) stop = gamma * 1e-18;     // |r| <= 1e-9 |b|: far below what a bf16 or fp32 output resolves
+        if (!(gamma > stop)) { done = true; break; }
+        double beta = 0.0, denom = delta;
+        if (it > 0) {
+            beta = gamma * fast_rcp(gamma_old);
+            denom = delta - beta * gamma * fast_rcp(alpha);
+        }
+        if (!(denom > 0.0) || it == LLA_CG_CAP) break;
+        alpha = gamma * fast_rcp(denom);
+        pv = rv + beta * pv;
+        sv = wv + beta * sv;
+        x += alpha * pv;
+        rv -= alpha * sv;
+        gamma_old = gamma;
+        ++iters;
+        CG_T(4);
     }
+#ifdef LLA_DT_TIMING
+    if (tid == 0 && tstat) for (int i = 0; i < 5; ++i) atomicAdd(tstat + i, (int)(cgt_[i] >> 4));
+#endif
     if (hh == 0) xs[r] = x;
     sync128();
     return done;
@@ -610,7 +633,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
 // Second kernel of the two-kernel decode: merge the parts' moment records of one (sequence, head),
 // centre them, solve and emit the output row.  Everything a thread needs of the two matrices goes
-// straight from the records (L2) into registers, so a block holds almost no shared memory and several
+// straight from the records (L2) into registers, so a block holds little shared memory and several
 // of them share an SM; the solve itself is latency-bound (barriers and shuffles), which is why it is
 // kept out of the streaming kernel whenever the caller provides the record buffer.
 constexpr int DS_MAX_SPLITS = 64;
@@ -620,10 +643,17 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
                     const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
                     int* __restrict__ status) {
     constexpr int D = DT_D, PF = 2 * D * D + 2 * D + 4;
-    __shared__ double s_a[D], s_c[D], s_x[D], s_p[D], s_red[24];
+    __shared__ __align__(16) double s_a[D], s_c[D], s_x[D], s_p[D], s_red[24];
     __shared__ double s_f[DS_MAX_SPLITS];
     __shared__ double s_L[D * 65];          // only touched by the factorisation fallback
     const int tid = threadIdx.x, r = tid >> 1, hh = tid & 1, bh = blockIdx.x;
+#ifdef LLA_DT_TIMING
+    long long sv_t_ = clock64();
+#define SV_T(ph) do { if (threadIdx.x == 0 && status) { const long long now_ = clock64(); atomicAdd(status + 24 + (ph), (int)((now_ - sv_t_) >> 4)); sv_t_ = now_; } } while (0)
+#else
+#define SV_T(ph)
+#endif
+    {
     if (max(1, min(lens[bh / H], Lmax)) < head_rows) return;
     const float* src = parts + (size_t)bh * splits * PF;
     float m = -INFINITY;
@@ -641,6 +671,7 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
         if (tid < D) s_a[tid] = s1 * inv; else s_c[tid - D] = s1 * inv;
     }
     __syncthreads();
+    SV_T(0);
     // this thread's half row of the centred matrix
     double cr[32];
 #pragma unroll
@@ -663,7 +694,13 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
         if (32 * hh + c == r) cr[c] += ridge;
     const double b_r = (double)to_f32(q[(size_t)bh * D + r]) - ar;
     int cg_its = 0;
+    SV_T(1);
+#ifdef LLA_DT_TIMING
+    const bool okc = cg_solve_64(cr, b_r, s_x, s_p, s_red, cg_its, status ? status + 32 : nullptr);
+#else
     const bool okc = cg_solve_64(cr, b_r, s_x, s_p, s_red, cg_its);
+#endif
+    SV_T(2);
     if (tid == 0 && status) atomicAdd(status + LLA_STATUS_ITER_SUM, cg_its);
     bool solved = true;
     if (!okc) {        // uniform over the block: the decision comes from block-wide sums
@@ -692,7 +729,9 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     for (int c = 0; c < 32; ++c) o += (nr[c] * inv - cb * s_a[32 * hh + c]) * s_x[32 * hh + c];
     o += __shfl_xor_sync(0xffffffffu, o, 1);
     if (hh == 0) store_out(out + (size_t)bh * D + r, (float)(o + cb));
+    SV_T(3);
     if (!solved && tid == 0 && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
+    }
 }
 
 template <typename TOut>
