@@ -251,7 +251,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (tid == 0) {
         for (int s = 0; s < DT_NST; ++s) { mbar_init(bar(DB_KVFULL + s), 1); mbar_init(bar(DB_KVEMPTY + s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar(DB_BFULL + b), DT_COMPUTE); mbar_init(bar(DB_BFREE + b), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(DB_BFULL + b), DT_COMPUTE / 32); mbar_init(bar(DB_BFREE + b), 1); }
         mbar_init(bar(DB_DFULL), 1);
         misc[1] = 0;
         fence_barrier_init();
@@ -295,9 +295,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (lane == 0) DT_EV(10, t);
             tc_fence_after();
             const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
-#ifndef LLA_DEXP_NOMMA
             mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), t > 0);
-#endif
             tc_commit_el(el, bar(DB_KVEMPTY + s));
             tc_commit_el(el, bar(DB_BFREE + b));
             if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
@@ -475,7 +473,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (tid == 0) DT_EV(25, t);
             fence_proxy_async();
             if (tid == 0) DT_EV(26, t);
-            mbar_arrive(bar(DB_BFULL + b));
+            // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised shared-memory atomics
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(DB_BFULL + b));
             DT_T(3);
             if (tid == 0) DT_EV(22, t);
             if (more && !stage_score_sync(t + 1)) { ok = false; break; }
@@ -564,10 +564,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         return;
     }
 
-#ifdef LLA_DEXP_NOEPI
-    if (tid < 64) store_out(out + (size_t)bh * DT_D + tid, dv[3] + omega_tot);
-    return;
-#endif
     // single part: centre, solve and emit the output row here
     double* Md = reinterpret_cast<double*>(smem);              // 64 x 65
     double* av = Md + 64 * 65;                                  // a -> kbar
