@@ -32,7 +32,7 @@ ROTATE = 16           # input sets cycled through so no step finds its inputs in
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/
 # (forward_tc_kernel_cfg2.md and decode_tc_kernel_cfg5.md).
 NCU_TRAFFIC_BYTES = 12.68e6
-NCU_DECODE_TRAFFIC_BYTES = 1.189e9 + 35.6e6
+NCU_DECODE_TRAFFIC_BYTES = 1.188e9 + 27.8e6 + 34.3e6   # streaming kernel read + record write, solve kernel read
 
 
 def env_int(name, default):

@@ -242,11 +242,11 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         for (int b = 0; b < TC_NBUF; ++b) {
             mbar_init(bar(B_SAFULL + b), 1);
-            mbar_init(bar(B_UFULL + b), split ? TC_COMPUTE : TC_COMPUTE / 2);
+            mbar_init(bar(B_UFULL + b), (split ? TC_COMPUTE : TC_COMPUTE / 2) / 32);   // one arrival per warp
             mbar_init(bar(B_BUFFREE + b), 1);
         }
         mbar_init(bar(B_ACCFULL), 1);
-        mbar_init(bar(B_CTL), TC_COMPUTE);
+        mbar_init(bar(B_CTL), TC_COMPUTE / 32);
         misc[1] = SW_MAX;
         misc[2] = 0;
         fence_barrier_init();
@@ -547,7 +547,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 }
                 if (kind != SW_MAX) tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(B_UFULL + b));
+                // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised atomics
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_UFULL + b));
                 if (lane == 0 && quad == 0) TC_EV(34 + half, blk);
             }
             if (kind != SW_MAX) {
@@ -578,7 +580,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         auto start_sweep = [&](int kind) {
             if (tid == 0) misc[1] = kind;
             fence_proxy_async();       // operand tiles written with ordinary stores -> visible to the MMA
-            mbar_arrive(bar(B_CTL));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_CTL));
         };
 
         // residual r: registers for D = 64, the scratch slot for D = 128 (no registers to spare)
