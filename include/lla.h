@@ -180,6 +180,9 @@ int lla_decode_ex(const lla_decode_params *p);
  * memory works).  The call allocates device buffers from the stream-ordered pool, copies the
  * inputs up, runs the device path on `stream`, copies the result back and SYNCHRONISES the
  * stream before returning, so `out` is valid on return.  dtypes are lla_dtype values.
+ * lla_forward_host cuts larger problems into four chunks of (batch, head) units whose upload,
+ * kernels and download run on library-owned streams, so copies and kernels overlap (with pinned
+ * buffers); `stream` is joined with them before the call returns.
  * lla_decode_host reads lens[] on the host and uploads only the first lens[b] rows of every
  * (sequence, head) cache.
  */

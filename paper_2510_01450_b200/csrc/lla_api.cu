@@ -33,6 +33,33 @@ SideStream* side_stream() {
     return &s;
 }
 
+// Worker streams of the host-buffer forward: the (batch, head) units are cut into a few chunks and
+// each chunk's upload, kernels and download run on their own stream, so the copies of one chunk
+// overlap the kernels of another.
+constexpr int kHostChunks = 4;
+struct HostPipe {
+    cudaStream_t stream[kHostChunks] = {};
+    cudaEvent_t ready = nullptr, done[kHostChunks] = {};
+    bool ok = false;
+};
+HostPipe* host_pipe() {
+    static std::mutex mu;
+    static HostPipe per_dev[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    HostPipe& h = per_dev[dev];
+    if (!h.ok) {
+        if (cudaEventCreateWithFlags(&h.ready, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        for (int c = 0; c < kHostChunks; ++c) {
+            if (cudaStreamCreateWithFlags(&h.stream[c], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&h.done[c], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
+        h.ok = true;
+    }
+    return &h;
+}
+
 bool head_size_ok(int d, int dv) { return d == dv && (d == 16 || d == 64 || d == 128); }
 
 int check_forward(const lla_forward_params* p) {
@@ -305,15 +332,42 @@ int lla_forward_host(const void* q, const void* k, const void* v, void* out, int
     DeviceScratch mem(st);
     void* dq = mem.get(nq); void* dk = mem.get(nq); void* dvv = mem.get(nv); void* dout = mem.get(no);
     if (!dq || !dk || !dvv || !dout) return LLA_ERR_CUDA;
-    LLA_CUDA_TRY(cudaMemcpyAsync(dq, q, nq, cudaMemcpyHostToDevice, st));
-    LLA_CUDA_TRY(cudaMemcpyAsync(dk, k, nq, cudaMemcpyHostToDevice, st));
-    LLA_CUDA_TRY(cudaMemcpyAsync(dvv, v, nv, cudaMemcpyHostToDevice, st));
-    p.q = dq; p.k = dk; p.v = dvv; p.out = dout;
-    const int st_rc = lla_forward_ex(&p);
-    if (st_rc != LLA_OK) return st_rc;
-    LLA_CUDA_TRY(cudaMemcpyAsync(out, dout, no, cudaMemcpyDeviceToHost, st));
+    const int units = B * H;
+    HostPipe* pipe = (units >= 2 * kHostChunks && nq + nq + nv >= (size_t)(1u << 20)) ? host_pipe() : nullptr;
+    if (!pipe) {
+        LLA_CUDA_TRY(cudaMemcpyAsync(dq, q, nq, cudaMemcpyHostToDevice, st));
+        LLA_CUDA_TRY(cudaMemcpyAsync(dk, k, nq, cudaMemcpyHostToDevice, st));
+        LLA_CUDA_TRY(cudaMemcpyAsync(dvv, v, nv, cudaMemcpyHostToDevice, st));
+        p.q = dq; p.k = dk; p.v = dvv; p.out = dout;
+        const int st_rc = lla_forward_ex(&p);
+        if (st_rc != LLA_OK) return st_rc;
+        LLA_CUDA_TRY(cudaMemcpyAsync(out, dout, no, cudaMemcpyDeviceToHost, st));
+        LLA_CUDA_TRY(cudaStreamSynchronize(st));
+        return LLA_OK;
+    }
+    // chunked: (batch, head) units are independent and contiguous in memory
+    LLA_CUDA_TRY(cudaEventRecord(pipe->ready, st));            // the buffers exist from here on
+    const size_t uq = (size_t)n * d * esz_in, uv = (size_t)n * dv * esz_in, uo = (size_t)n * dv * esz_out;
+    int rc_chunks = LLA_OK;
+    for (int c = 0; c < kHostChunks; ++c) {
+        const int u0 = (int)((long long)units * c / kHostChunks), u1 = (int)((long long)units * (c + 1) / kHostChunks);
+        cudaStream_t w = pipe->stream[c];
+        LLA_CUDA_TRY(cudaStreamWaitEvent(w, pipe->ready, 0));
+        LLA_CUDA_TRY(cudaMemcpyAsync((char*)dq + u0 * uq, (const char*)q + u0 * uq, (u1 - u0) * uq, cudaMemcpyHostToDevice, w));
+        LLA_CUDA_TRY(cudaMemcpyAsync((char*)dk + u0 * uq, (const char*)k + u0 * uq, (u1 - u0) * uq, cudaMemcpyHostToDevice, w));
+        LLA_CUDA_TRY(cudaMemcpyAsync((char*)dvv + u0 * uv, (const char*)v + u0 * uv, (u1 - u0) * uv, cudaMemcpyHostToDevice, w));
+        lla_forward_params pc = p;
+        pc.q = (char*)dq + u0 * uq; pc.k = (char*)dk + u0 * uq; pc.v = (char*)dvv + u0 * uv; pc.out = (char*)dout + u0 * uo;
+        pc.B = 1; pc.H = u1 - u0;
+        pc.stream = w;
+        const int rc_c = lla_forward_ex(&pc);
+        if (rc_c != LLA_OK && rc_chunks == LLA_OK) rc_chunks = rc_c;
+        LLA_CUDA_TRY(cudaMemcpyAsync((char*)out + u0 * uo, (char*)dout + u0 * uo, (u1 - u0) * uo, cudaMemcpyDeviceToHost, w));
+        LLA_CUDA_TRY(cudaEventRecord(pipe->done[c], w));
+        LLA_CUDA_TRY(cudaStreamWaitEvent(st, pipe->done[c], 0));
+    }
     LLA_CUDA_TRY(cudaStreamSynchronize(st));
-    return LLA_OK;
+    return rc_chunks;
 }
 
 int lla_decode_host(const void* q, const void* kcache, const void* vcache, const int* lens, void* out, int B,

@@ -269,6 +269,15 @@ def test_host_buffer_entry_points(oracle):
         L.lla_forward_host(hq, hk, hv, hout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_F32, w.scale, w.lam, 1,
                            stream_ptr())
         assert row_err(hout.numpy(), ref).max() <= TOL_BF16
+    # enough (batch, head) units and bytes for the chunked form (upload, kernels and download of the
+    # chunks overlap on separate streams); pageable output buffer on purpose
+    w = inputs.CONFIGS[2].shrink(B=3, H=3, n=640, seed=18)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    hq, hk, hv = (torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in (q, k, v))
+    hout = torch.full((w.B, w.H, w.n, w.dv), float("nan"), dtype=torch.float32)
+    L.lla_forward_host(hq, hk, hv, hout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_F32, w.scale, w.lam, 1, stream_ptr())
+    assert row_err(hout.numpy(), ref).max() <= TOL_BF16
     wd = inputs.CONFIGS[5].shrink(B=3, H=2, n=700, len_min=5, len_max=700, seed=17)
     dq, kc, vc, lens = inputs.make_decode(wd)
     dref = oracle.decode(dq, kc, vc, lens, wd.scale, wd.lam)
