@@ -51,6 +51,8 @@
 #endif
 
 #define ORACLE_OK 0
+#define ORACLE_RIDGE_DEFINITION 0
+#define ORACLE_RIDGE_PRINTED 1
 #define ORACLE_NOT_SPD 1 /* Cholesky met a non-positive pivot (only possible at lambda = 0) */
 
 static inline double ld(const void *p, size_t idx, int in_f32)
@@ -107,8 +109,9 @@ static void cholesky_solve(const double *l, int d, double *b)
  * work must hold L + L*d + d*d + 2*d doubles.
  */
 static int oracle_row(const void *q, size_t q_off, const void *k, size_t k_off, const void *v,
-                      size_t v_off, int L, int d, int dv, double scale, double lambda, int in_f32,
-                      double *out, double *rho_out, double *aux_out, double *work)
+                      size_t v_off, int L, int d, int dv, double scale, double lambda,
+                      int ridge_mode, int in_f32, double *out, double *rho_out, double *aux_out,
+                      double *work)
 {
     double *w = work;                /* L   */
     double *z = w + L;               /* L*d */
@@ -130,7 +133,11 @@ static int oracle_row(const void *q, size_t q_off, const void *k, size_t k_off, 
         if (s > m)
             m = s;
     }
-    const double lambda_m = lambda * exp(-m);
+    /* Ridge in the max-subtracted frame.  Mode 0: the definition, raw weights exp(s) with
+     * ridge lambda, i.e. lambda * exp(-m) here.  Mode 1: Algorithm 1/2 as printed, which add
+     * lambda to the moments of the weights exp(s - m) unchanged (an effective ridge
+     * lambda * exp(m_i) in the raw frame). */
+    const double lambda_m = ridge_mode == ORACLE_RIDGE_PRINTED ? lambda : lambda * exp(-m);
 
     /* weights, centred keys, moments */
     double omega = 0.0;
@@ -215,10 +222,32 @@ static size_t work_doubles(int L, int d)
  *   status [n_rows] int (may be NULL): ORACLE_OK or ORACLE_NOT_SPD
  * Returns the number of rows whose Cholesky failed, or -1 on allocation failure.
  */
+/*
+ * As above with the ridge variants: lambda_rows (may be NULL) holds one ridge per query row,
+ * [B*H*n] in the flat row order, and replaces the scalar (per-token regularisation, the
+ * appendix on learnable lambda); ridge_mode is ORACLE_RIDGE_DEFINITION or ORACLE_RIDGE_PRINTED.
+ */
+int lla_oracle_forward_rows_ex(const void *q, const void *k, const void *v, int in_f32, int B,
+                               int H, int n, int d, int dv, double scale, double lambda,
+                               const double *lambda_rows, int ridge_mode, int causal,
+                               const long long *rows, long long n_rows, double *out, double *rho,
+                               double *aux, int *status);
+
 int lla_oracle_forward_rows(const void *q, const void *k, const void *v, int in_f32, int B, int H,
                             int n, int d, int dv, double scale, double lambda, int causal,
                             const long long *rows, long long n_rows, double *out, double *rho,
                             double *aux, int *status)
+{
+    return lla_oracle_forward_rows_ex(q, k, v, in_f32, B, H, n, d, dv, scale, lambda, NULL,
+                                      ORACLE_RIDGE_DEFINITION, causal, rows, n_rows, out, rho, aux,
+                                      status);
+}
+
+int lla_oracle_forward_rows_ex(const void *q, const void *k, const void *v, int in_f32, int B,
+                               int H, int n, int d, int dv, double scale, double lambda,
+                               const double *lambda_rows, int ridge_mode, int causal,
+                               const long long *rows, long long n_rows, double *out, double *rho,
+                               double *aux, int *status)
 {
     (void)B;
     (void)H;
@@ -240,7 +269,8 @@ int lla_oracle_forward_rows(const void *q, const void *k, const void *v, int in_
             const int i = (int)(flat % n);
             const int L = causal ? i + 1 : n;
             const int st = oracle_row(q, (size_t)flat * d, k, (size_t)bh * n * d, v,
-                                      (size_t)bh * n * dv, L, d, dv, scale, lambda, in_f32,
+                                      (size_t)bh * n * dv, L, d, dv, scale,
+                                      lambda_rows ? lambda_rows[flat] : lambda, ridge_mode, in_f32,
                                       out + (size_t)r * dv, rho ? rho + (size_t)r * d : NULL,
                                       aux ? aux + (size_t)r * 3 : NULL, work);
             if (status)
@@ -258,9 +288,24 @@ int lla_oracle_forward_rows(const void *q, const void *k, const void *v, int in_
  *   current token's key and value are already in the cache, matching j <= i)
  *   out [B,H,dv] float64
  */
+int lla_oracle_decode_ex(const void *q, const void *kcache, const void *vcache, int in_f32,
+                         const int *lens, int B, int H, int Lmax, int d, int dv, double scale,
+                         double lambda, const double *lambda_units, int ridge_mode, double *out,
+                         int *status);
+
 int lla_oracle_decode(const void *q, const void *kcache, const void *vcache, int in_f32,
                       const int *lens, int B, int H, int Lmax, int d, int dv, double scale,
                       double lambda, double *out, int *status)
+{
+    return lla_oracle_decode_ex(q, kcache, vcache, in_f32, lens, B, H, Lmax, d, dv, scale, lambda,
+                                NULL, ORACLE_RIDGE_DEFINITION, out, status);
+}
+
+/* Decode with the ridge variants: lambda_units (may be NULL) is one ridge per (sequence, head). */
+int lla_oracle_decode_ex(const void *q, const void *kcache, const void *vcache, int in_f32,
+                         const int *lens, int B, int H, int Lmax, int d, int dv, double scale,
+                         double lambda, const double *lambda_units, int ridge_mode, double *out,
+                         int *status)
 {
     long long failures = 0;
     int alloc_failed = 0;
@@ -277,7 +322,8 @@ int lla_oracle_decode(const void *q, const void *kcache, const void *vcache, int
                 continue;
             const int b = (int)(bh / H);
             const int st = oracle_row(q, (size_t)bh * d, kcache, (size_t)bh * Lmax * d, vcache,
-                                      (size_t)bh * Lmax * dv, lens[b], d, dv, scale, lambda,
+                                      (size_t)bh * Lmax * dv, lens[b], d, dv, scale,
+                                      lambda_units ? lambda_units[bh] : lambda, ridge_mode,
                                       in_f32, out + (size_t)bh * dv, NULL, NULL, work);
             if (status)
                 status[bh] = st;

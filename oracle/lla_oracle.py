@@ -46,6 +46,12 @@ def _load():
         lib.lla_oracle_decode.restype = i32
         lib.lla_oracle_decode.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, f64, f64,
                                           vp, vp]
+        lib.lla_oracle_forward_rows_ex.restype = i32
+        lib.lla_oracle_forward_rows_ex.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, f64, f64,
+                                                   vp, i32, i32, vp, i64, vp, vp, vp, vp]
+        lib.lla_oracle_decode_ex.restype = i32
+        lib.lla_oracle_decode_ex.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, f64, f64,
+                                             vp, i32, vp, vp]
         lib.lla_oracle_threads.restype = i32
         lib.lla_oracle_threads.argtypes = []
         _lib = lib
@@ -69,9 +75,24 @@ def _ptr(a):
     return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
 
 
-def forward_rows(q, k, v, scale, lam, causal=True, rows=None, want_aux=False):
+RIDGE_MODES = {"definition": 0, "printed": 1}
+
+
+def _ridge(lam, count):
+    """Scalar ridge and optional per-row array (float64, ``count`` entries)."""
+    if np.ndim(lam) == 0:
+        return float(lam), None
+    arr = np.ascontiguousarray(np.asarray(lam, dtype=np.float64).reshape(-1))
+    assert arr.size == count, (arr.size, count)
+    return 0.0, arr
+
+
+def forward_rows(q, k, v, scale, lam, causal=True, rows=None, want_aux=False, ridge_mode="definition"):
     """LLA outputs for selected query rows.
 
+    ``lam`` is a scalar or one ridge per query row ``[B,H,n]`` (per-token regularisation).
+    ``ridge_mode``: "definition" (raw weights, ridge lambda: Eq. "query_specific") or "printed"
+    (Algorithm 1/2 as printed: lambda added in the max-subtracted frame).
     q, k: [B,H,n,d]; v: [B,H,n,dv]; float32 (holds bf16 exactly) or float64.
     rows: 1-D int64 array of flat row indices ``(b*H + h)*n + i`` (default: every row).
     Returns ``out [n_rows, dv]`` float64, and with ``want_aux`` also
@@ -89,9 +110,11 @@ def forward_rows(q, k, v, scale, lam, causal=True, rows=None, want_aux=False):
     rho = np.empty((rows.size, d), dtype=np.float64) if want_aux else None
     aux = np.empty((rows.size, 3), dtype=np.float64) if want_aux else None
     status = np.zeros(rows.size, dtype=np.int32)
-    rc = _load().lla_oracle_forward_rows(_ptr(q), _ptr(k), _ptr(v), in_f32, B, H, n, d, dv,
-                                         float(scale), float(lam), int(bool(causal)), _ptr(rows),
-                                         rows.size, _ptr(out), _ptr(rho), _ptr(aux), _ptr(status))
+    lam0, lam_rows = _ridge(lam, B * H * n)
+    rc = _load().lla_oracle_forward_rows_ex(_ptr(q), _ptr(k), _ptr(v), in_f32, B, H, n, d, dv,
+                                            float(scale), lam0, _ptr(lam_rows), RIDGE_MODES[ridge_mode],
+                                            int(bool(causal)), _ptr(rows), rows.size, _ptr(out), _ptr(rho),
+                                            _ptr(aux), _ptr(status))
     if rc < 0:
         raise MemoryError("oracle work buffer allocation failed")
     if want_aux:
@@ -99,15 +122,17 @@ def forward_rows(q, k, v, scale, lam, causal=True, rows=None, want_aux=False):
     return out
 
 
-def forward(q, k, v, scale, lam, causal=True):
+def forward(q, k, v, scale, lam, causal=True, ridge_mode="definition"):
     """LLA output for every row, shaped [B,H,n,dv] float64."""
     B, H, n, _ = np.asarray(q).shape
-    out = forward_rows(q, k, v, scale, lam, causal)
+    out = forward_rows(q, k, v, scale, lam, causal, ridge_mode=ridge_mode)
     return out.reshape(B, H, n, -1)
 
 
-def decode(q, kcache, vcache, lens, scale, lam):
-    """Single-query decode: q [B,H,d], caches [B,H,Lmax,d|dv], lens [B] -> out [B,H,dv] float64."""
+def decode(q, kcache, vcache, lens, scale, lam, ridge_mode="definition"):
+    """Single-query decode: q [B,H,d], caches [B,H,Lmax,d|dv], lens [B] -> out [B,H,dv] float64.
+
+    ``lam`` is a scalar or one ridge per (sequence, head) ``[B,H]``."""
     (q, kcache, vcache), in_f32 = _as_input(q, kcache, vcache)
     B, H, d = q.shape
     Lmax = kcache.shape[2]
@@ -117,8 +142,10 @@ def decode(q, kcache, vcache, lens, scale, lam):
     assert lens.shape == (B,) and lens.min() >= 1 and lens.max() <= Lmax
     out = np.empty((B, H, dv), dtype=np.float64)
     status = np.zeros(B * H, dtype=np.int32)
-    rc = _load().lla_oracle_decode(_ptr(q), _ptr(kcache), _ptr(vcache), in_f32, _ptr(lens), B, H,
-                                   Lmax, d, dv, float(scale), float(lam), _ptr(out), _ptr(status))
+    lam0, lam_units = _ridge(lam, B * H)
+    rc = _load().lla_oracle_decode_ex(_ptr(q), _ptr(kcache), _ptr(vcache), in_f32, _ptr(lens), B, H,
+                                      Lmax, d, dv, float(scale), lam0, _ptr(lam_units),
+                                      RIDGE_MODES[ridge_mode], _ptr(out), _ptr(status))
     if rc < 0:
         raise MemoryError("oracle work buffer allocation failed")
     return out
