@@ -54,6 +54,13 @@ typedef enum lla_impl {
     LLA_IMPL_TENSOR = 2  /* tcgen05/TMEM kernel (bf16 inputs, d = dv = 64 or 128) */
 } lla_impl;
 
+/* How the ridge enters (lla_forward_params / lla_decode_params.ridge_mode).
+ * DEFINITION: Sigma_i = sum_j exp(s_ij) z z^T + lambda I with the raw weights of Eq. "query_specific";
+ *             computed with max-subtracted weights and the ridge lambda * exp(-m_i).
+ * PRINTED:    Algorithm 1/2 as printed: lambda is added to the moments of the max-subtracted weights
+ *             exp(s_ij - m_i) as it is, i.e. an effective ridge lambda * exp(m_i) in the raw frame. */
+typedef enum lla_ridge_mode { LLA_RIDGE_DEFINITION = 0, LLA_RIDGE_PRINTED = 1 } lla_ridge_mode;
+
 /* Row groups for lla_forward_params.phases. */
 enum { LLA_PHASE_ALL = 0, LLA_PHASE_DIRECT = 1, LLA_PHASE_ITERATIVE = 2 };
 
@@ -119,6 +126,9 @@ int lla_decode_f32(const void *q, const void *kcache, const void *vcache, const 
  *   iters     : optional [B, H, n] int32, CG iterations executed for the row (-1 for rows solved
  *               directly)
  *   device_status : optional int[LLA_STATUS_WORDS] on the device
+ *   lambda_rows : optional [B, H, n] fp32 on the device, one ridge per query row (the paper's
+ *               per-token regularisation); when not NULL it replaces `lambda`
+ *   ridge_mode : lla_ridge_mode (0 = the definition; 1 = Algorithm 1/2 as printed)
  *   workspace / workspace_bytes : device scratch of at least lla_forward_workspace_bytes(...)
  *               bytes, 256-byte aligned; may be NULL when that function returns 0
  */
@@ -141,6 +151,9 @@ typedef struct lla_forward_params {
     void *workspace;
     size_t workspace_bytes;
     void *stream;
+    const float *lambda_rows;   /* optional [B, H, n] fp32 on the device: one ridge per query row
+                                   (per-token regularisation); replaces `lambda` when not NULL */
+    int ridge_mode;             /* lla_ridge_mode */
 } lla_forward_params;
 
 int lla_forward_ex(const lla_forward_params *p);
@@ -151,6 +164,8 @@ int lla_forward_ex(const lla_forward_params *p);
  *   splits    : number of key-range parts each (sequence, head) is divided into so that long
  *               caches spread over more thread blocks (0 = chosen from B*H and Lmax; 1 = none).
  *               With splits > 1 partial moments go through `workspace`.
+ *   lambda_units : optional [B, H] fp32 on the device, one ridge per (sequence, head)
+ *   ridge_mode : lla_ridge_mode; LLA_RIDGE_PRINTED runs on the CUDA-core decode kernels
  *   workspace : device scratch of at least lla_decode_workspace_bytes(...) bytes, 256-byte
  *               aligned; required when the effective number of splits exceeds 1.  Unsplit, it
  *               is optional: given one, the tensor-core path (bf16, d = dv = 64) writes each
@@ -170,6 +185,8 @@ typedef struct lla_decode_params {
     void *workspace;
     size_t workspace_bytes;
     void *stream;
+    const float *lambda_units;  /* optional [B, H] fp32 on the device: one ridge per (sequence, head) */
+    int ridge_mode;             /* lla_ridge_mode */
 } lla_decode_params;
 
 int lla_decode_ex(const lla_decode_params *p);

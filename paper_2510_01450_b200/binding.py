@@ -19,6 +19,7 @@ LLA_IMPL_AUTO, LLA_IMPL_SIMT, LLA_IMPL_TENSOR = 0, 1, 2
 LLA_STATUS_WORDS = 4
 LLA_PHASE_ALL, LLA_PHASE_DIRECT, LLA_PHASE_ITERATIVE = 0, 1, 2
 STATUS_ROWS_AT_CAP, STATUS_BAD_PIVOT, STATUS_TIMEOUT, STATUS_ITER_SUM = 0, 1, 2, 3
+LLA_RIDGE_DEFINITION, LLA_RIDGE_PRINTED = 0, 1
 
 EXPORTS = (
     "lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex", "lla_decode_ex",
@@ -43,7 +44,7 @@ class ForwardParams(ctypes.Structure):
         ("head_rows", ctypes.c_int), ("impl", ctypes.c_int), ("phases", ctypes.c_int),
         ("rho", ctypes.c_void_p), ("stats", ctypes.c_void_p), ("iters", ctypes.c_void_p),
         ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
-        ("stream", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p), ("lambda_rows", ctypes.c_void_p), ("ridge_mode", ctypes.c_int),
     ]
 
 
@@ -56,7 +57,7 @@ class DecodeParams(ctypes.Structure):
         ("scale", ctypes.c_float), ("lambda_", ctypes.c_float),
         ("splits", ctypes.c_int), ("impl", ctypes.c_int),
         ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
-        ("stream", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p), ("lambda_units", ctypes.c_void_p), ("ridge_mode", ctypes.c_int),
     ]
 
 
@@ -152,7 +153,8 @@ def lla_decode_host(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, in_dtype, o
 
 def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=LLA_BF16, out_dtype=LLA_BF16,
                    max_iters=0, tol=0.0, head_rows=0, impl=LLA_IMPL_AUTO, phases=0, rho=None, stats=None, iters=None,
-                   device_status=None, workspace=None, workspace_bytes=0, stream=0):
+                   device_status=None, workspace=None, workspace_bytes=0, stream=0, lambda_rows=None,
+                   ridge_mode=LLA_RIDGE_DEFINITION):
     p = ForwardParams()
     p.q, p.k, p.v, p.out = _p(q), _p(k), _p(v), _p(out)
     p.B, p.H, p.n, p.d, p.dv = B, H, n, d, dv
@@ -161,18 +163,20 @@ def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=
     p.max_iters, p.tol, p.head_rows, p.impl, p.phases = max_iters, tol, head_rows, impl, phases
     p.rho, p.stats, p.iters, p.device_status = _p(rho), _p(stats), _p(iters), _p(device_status)
     p.workspace, p.workspace_bytes, p.stream = _p(workspace), workspace_bytes, _p(stream)
+    p.lambda_rows, p.ridge_mode = _p(lambda_rows), ridge_mode
     _check(load().lla_forward_ex(ctypes.byref(p)), "lla_forward_ex")
 
 
 def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, in_dtype=LLA_BF16,
                   out_dtype=LLA_BF16, splits=0, impl=LLA_IMPL_AUTO, device_status=None, workspace=None,
-                  workspace_bytes=0, stream=0):
+                  workspace_bytes=0, stream=0, lambda_units=None, ridge_mode=LLA_RIDGE_DEFINITION):
     p = DecodeParams()
     p.q, p.kcache, p.vcache, p.lens, p.out = _p(q), _p(kcache), _p(vcache), _p(lens), _p(out)
     p.B, p.H, p.Lmax, p.d, p.dv = B, H, Lmax, d, dv
     p.in_dtype, p.out_dtype = in_dtype, out_dtype
     p.scale, p.lambda_, p.splits, p.impl = scale, lam, splits, impl
     p.device_status, p.workspace, p.workspace_bytes, p.stream = _p(device_status), _p(workspace), workspace_bytes, _p(stream)
+    p.lambda_units, p.ridge_mode = _p(lambda_units), ridge_mode
     _check(load().lla_decode_ex(ctypes.byref(p)), "lla_decode_ex")
 
 

@@ -67,6 +67,7 @@ int check_forward(const lla_forward_params* p) {
     if (!p->q || !p->k || !p->v || !p->out) return LLA_ERR_INVALID_ARG;
     if (p->B < 1 || p->H < 1 || p->n < 1 || p->d < 1 || p->dv < 1) return LLA_ERR_INVALID_ARG;
     if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
+    if (p->ridge_mode != LLA_RIDGE_DEFINITION && p->ridge_mode != LLA_RIDGE_PRINTED) return LLA_ERR_INVALID_ARG;
     if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535 || (p->n + 127) / 128 > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
@@ -94,6 +95,8 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.rho = p->rho; a.stats = p->stats; a.iters = p->iters; a.status = p->device_status;
     a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
     a.stream = (cudaStream_t)p->stream;
+    a.lambda_rows = p->lambda_rows;
+    a.ridge_mode = p->ridge_mode;
     return a;
 }
 
@@ -103,6 +106,7 @@ int check_decode(const lla_decode_params* p) {
     if (p->B < 1 || p->H < 1 || p->Lmax < 1 || p->d < 1 || p->dv < 1 || p->splits < 0) return LLA_ERR_INVALID_ARG;
     if (p->impl != LLA_IMPL_AUTO && p->impl != LLA_IMPL_SIMT && p->impl != LLA_IMPL_TENSOR) return LLA_ERR_INVALID_ARG;
     if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
+    if (p->ridge_mode != LLA_RIDGE_DEFINITION && p->ridge_mode != LLA_RIDGE_PRINTED) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
     const bool dt_ok = (p->in_dtype == LLA_BF16 && (p->out_dtype == LLA_BF16 || p->out_dtype == LLA_F32)) ||
@@ -218,6 +222,8 @@ int lla_decode_ex(const lla_decode_params* p) {
     a.status = p->device_status;
     a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
     a.stream = (cudaStream_t)p->stream;
+    a.lambda_units = p->lambda_units;
+    a.ridge_mode = p->ridge_mode;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
     const int st = lla::launch_decode(a);
     if (st != LLA_OK) return st;

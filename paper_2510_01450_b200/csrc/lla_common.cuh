@@ -31,6 +31,8 @@ struct ForwardArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
+    const float* lambda_rows;   // optional per-row ridge [B, H, n]
+    int ridge_mode;             // lla_ridge_mode
 };
 
 struct DecodeArgs {
@@ -49,6 +51,8 @@ struct DecodeArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
+    const float* lambda_units;  // optional per-(sequence, head) ridge [B, H]
+    int ridge_mode;             // lla_ridge_mode
 };
 
 // Launchers implemented in the other translation units; each returns an lla_status.

@@ -31,11 +31,11 @@ struct DcCfg {
 //   a, c: first moments; returns through out[dv]
 template <int D, typename TOut>
 __device__ void finalize_row(double* Md, const float* Nd, double* a, double* c, double omega, double m,
-                             const double* qd, double lambda, TOut* out, int* status) {
+                             const double* qd, double lambda, int ridge_mode, TOut* out, int* status) {
     const int tid = threadIdx.x;
     constexpr int LDS = D + 1;
     const double inv = 1.0 / omega;
-    const double ridge = lambda * exp(-m) * inv;
+    const double ridge = (ridge_mode == LLA_RIDGE_PRINTED ? lambda : lambda * exp(-m)) * inv;
     __syncthreads();
     for (int e = tid; e < D * D; e += DC_THREADS) {
         const int r = e / D, cc = e - r * D;
@@ -62,7 +62,8 @@ template <int D, typename TIn, typename TOut>
 __global__ void __launch_bounds__(DC_THREADS)
 decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache, const TIn* __restrict__ vcache,
                       const int* __restrict__ lens, TOut* __restrict__ out, int H, int Lmax, float scale,
-                      float lambda, int splits, int head_rows, float* __restrict__ parts, int* __restrict__ status) {
+                      float lambda, int splits, int head_rows, float* __restrict__ parts, int* __restrict__ status,
+                      const float* __restrict__ lambda_units, int ridge_mode) {
     using C = DcCfg<D>;
     constexpr bool ACCURATE = sizeof(TIn) == 4;
     extern __shared__ double smem_d[];
@@ -210,14 +211,15 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     }
     if (tid < D) a[tid] = (double)first;
     else if (tid < 2 * D) c[tid - D] = (double)first;
-    finalize_row<D>(Md, Nd, a, c, (double)omega, (double)m, qd_s, (double)lambda, out + (size_t)bh * D, status);
+    finalize_row<D>(Md, Nd, a, c, (double)omega, (double)m, qd_s, (double)(lambda_units ? lambda_units[bh] : lambda),
+                    ridge_mode, out + (size_t)bh * D, status);
 }
 
 template <int D, typename TIn, typename TOut>
 __global__ void __launch_bounds__(DC_THREADS)
 decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts, TOut* __restrict__ out,
                       const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
-                      int* __restrict__ status) {
+                      int* __restrict__ status, const float* __restrict__ lambda_units, int ridge_mode) {
     using C = DcCfg<D>;
     extern __shared__ double smem_d[];
     double* Md = smem_d;
@@ -256,7 +258,8 @@ decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts
         const float* pp = src + (size_t)p * C::PART_FLOATS;
         omega += exp((double)pp[2 * D * D + 2 * D + 1] - (double)m) * (double)pp[2 * D * D + 2 * D];
     }
-    finalize_row<D>(Md, Nd, a, c, omega, (double)m, qd_s, (double)lambda, out + (size_t)bh * D, status);
+    finalize_row<D>(Md, Nd, a, c, omega, (double)m, qd_s, (double)(lambda_units ? lambda_units[bh] : lambda), ridge_mode,
+                    out + (size_t)bh * D, status);
 }
 
 template <int D>
@@ -274,7 +277,10 @@ int launch_t(const DecodeArgs& a) {
         const size_t need = decode_workspace_bytes(a.B, a.H, a.d, a.dv, splits);
         if (!a.workspace || a.workspace_bytes < need) return LLA_ERR_WORKSPACE;
     }
-    if (a.impl != LLA_IMPL_SIMT && decode_tensor_supported(a)) {
+    // The tensor-core path keeps its moments relative to the first tile's maximum, not the true one,
+    // which the printed ridge variant is defined against: that variant runs on the kernels below.
+    if (a.impl == LLA_IMPL_TENSOR && a.ridge_mode == LLA_RIDGE_PRINTED) return LLA_ERR_UNSUPPORTED;
+    if (a.impl != LLA_IMPL_SIMT && a.ridge_mode == LLA_RIDGE_DEFINITION && decode_tensor_supported(a)) {
         // tensor-core path: streaming kernel plus its own solve kernel (or fused epilogue)
         return launch_decode_tensor_moments(a);
     } else {
@@ -284,14 +290,15 @@ int launch_t(const DecodeArgs& a) {
         dim3 grid(splits, a.B * a.H);
         k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
                                                  a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
-                                                 a.head_rows, (float*)a.workspace, a.status);
+                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     if (splits > 1) {
         auto k2 = decode_combine_kernel<D, TIn, TOut>;
         LLA_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         k2<<<a.B * a.H, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const float*)a.workspace,
-                                                      (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows, a.lambda, splits, a.status);
+                                                      (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows, a.lambda, splits, a.status,
+                                                      a.lambda_units, a.ridge_mode);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     return LLA_OK;
@@ -373,6 +380,7 @@ extern "C" int lla_decode_noalloc(const void* q, const void* kcache, const void*
     a.B = B; a.H = H; a.Lmax = Lmax; a.d = d; a.dv = dv;
     a.in_dtype = in_dtype; a.out_dtype = out_dtype;
     a.scale = scale; a.lambda = lambda;
+    a.lambda_units = nullptr; a.ridge_mode = LLA_RIDGE_DEFINITION;
     a.splits = splits > 0 ? splits : lla_decode_default_splits(B, H, Lmax);
     a.head_rows = 2 * d;
     a.impl = LLA_IMPL_AUTO;

@@ -201,6 +201,8 @@ struct DtParams {
     float* parts;
     int* status;
     int defer;           // 1: write the moment record even for a single part; a solve kernel follows
+    const float* lambda_units;   // optional per-(sequence, head) ridge
+    int ridge_mode;
 };
 
 template <typename TOut>
@@ -571,7 +573,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     double* rhs = cv + 64;
     float* Nd = reinterpret_cast<float*>(rhs + 64);             // 64 x 65 (padded rows)
     const double inv = 1.0 / (double)omega_tot;
-    const double ridge = (double)prm.lambda * exp(-(double)mref_ln) * inv;
+    const double lam_u = prm.lambda_units ? (double)prm.lambda_units[bh] : (double)prm.lambda;
+    const double ridge = (prm.ridge_mode == LLA_RIDGE_PRINTED ? lam_u : lam_u * exp(-(double)mref_ln)) * inv;
     if (warp < 4) {
         if (tid < 64) av[tid] = (double)dv[64] * inv;
         else cv[tid - 64] = (double)dv[64] * inv;
@@ -637,7 +640,7 @@ template <typename TOut>
 __global__ void __launch_bounds__(DT_COMPUTE, 4)
 decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict__ parts, TOut* __restrict__ out,
                     const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
-                    int* __restrict__ status) {
+                    int* __restrict__ status, const float* __restrict__ lambda_units, int ridge_mode) {
     constexpr int D = DT_D, PF = 2 * D * D + 2 * D + 4;
     __shared__ __align__(16) double s_a[D], s_c[D], s_x[D], s_p[D], s_red[24];
     __shared__ double s_f[DS_MAX_SPLITS];
@@ -660,7 +663,8 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     double omega = 0.0;
     for (int p = 0; p < splits; ++p) omega += s_f[p] * (double)src[(size_t)p * PF + 2 * D * D + 2 * D];
     const double inv = 1.0 / omega;
-    const double ridge = (double)lambda * exp(-(double)m) * inv;
+    const double lam_u = lambda_units ? (double)lambda_units[bh] : (double)lambda;
+    const double ridge = (ridge_mode == LLA_RIDGE_PRINTED ? lam_u : lam_u * exp(-(double)m)) * inv;
     {
         double s1 = 0.0;                     // thread e < 64: a[e]; thread 64 + e: c[e]
         for (int p = 0; p < splits; ++p) s1 += s_f[p] * (double)src[(size_t)p * PF + 2 * D * D + tid];
@@ -744,6 +748,7 @@ int launch_t(const DecodeArgs& a) {
     DtParams prm;
     prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
+    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode;
     prm.parts = (float*)a.workspace; prm.status = a.status;
     prm.defer = have_ws ? 1 : 0;      // with a record buffer the solve runs as its own kernel
     auto kern = decode_tc_kernel<TOut>;
@@ -756,7 +761,7 @@ int launch_t(const DecodeArgs& a) {
     if (have_ws) {
         decode_solve_kernel<TOut><<<BH, DT_COMPUTE, 0, a.stream>>>((const __nv_bfloat16*)a.q, (const float*)a.workspace,
                                                                    (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows,
-                                                                   a.lambda, splits, a.status);
+                                                                   a.lambda, splits, a.status, a.lambda_units, a.ridge_mode);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     return LLA_OK;

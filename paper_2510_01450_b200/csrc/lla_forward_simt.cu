@@ -61,7 +61,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                     TOut* __restrict__ out, int n, int causal, float scale, float lambda,
                     int head_rows, int max_iters, float tol, int first_tile,
                     float* __restrict__ rho_out, float* __restrict__ stats, int* __restrict__ iters_out,
-                    int* __restrict__ status) {
+                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode) {
     constexpr int ROWS = FS_THREADS / TPR;
     constexpr int NG = D / (4 * TPR);    // float4 groups per thread (keys)
     constexpr int NGV = DV / (4 * TPR);  // float4 groups per thread (values)
@@ -129,7 +129,8 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
         }
     }
     const float inv_omega = row_ok ? 1.f / omega : 0.f;
-    const float ridge = row_ok ? lambda * exp_w<ACCURATE>(-m) * inv_omega : 0.f;
+    const float lam_i = (lambda_rows && row < n) ? lambda_rows[(size_t)bh * n + row] : lambda;
+    const float ridge = row_ok ? (ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * exp_w<ACCURATE>(-m)) * inv_omega : 0.f;
 
     // ---- conjugate gradients on C y = kbar - q (Algorithm 2) ----
     float4 x[NG], r[NG], p[NG];
@@ -309,7 +310,7 @@ int launch_t(const ForwardArgs& a) {
     kern<<<grid, FS_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, a.causal, a.scale,
         a.lambda, a.head_rows > 0 ? a.head_rows : 0, a.max_iters, a.tol, first_tile, a.rho, a.stats,
-        a.iters, a.status);
+        a.iters, a.status, a.lambda_rows, a.ridge_mode);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -180,6 +180,8 @@ struct TcParams {
     int* status;
     float* scratch;      // D = 128: per-SM slots for x, kbar, r (TcCfg::SCRATCH_FLOATS_PER_SM each)
     int scratch_slots;
+    const float* lambda_rows;   // optional per-row ridge [B, H, n]
+    int ridge_mode;
     int use_order;       // 1: blockIdx.y -> tile through order[]; 0: last tile first
     unsigned short order[TC_ORDER_MAX];
 };
@@ -613,7 +615,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (ok) {
                 omega = pair_sum(part);
                 inv_omega = 1.f / omega;
-                ridge = prm.lambda * ex2f(-mx2) * inv_omega;
+                const float lam_i = (prm.lambda_rows && row < n) ? prm.lambda_rows[(size_t)bh * n + row] : prm.lambda;
+                ridge = (prm.ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * ex2f(-mx2)) * inv_omega;
                 float rr_p = 0.f, ab_p = 0.f;
 #pragma unroll
                 for (int ch = 0; ch < NCOL / 8; ++ch) {
@@ -857,6 +860,7 @@ int launch_t(const ForwardArgs& a) {
     prm.n = a.n; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
+    prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     prm.dbg = nullptr;
     prm.scratch = nullptr;

@@ -105,7 +105,8 @@ __global__ void __launch_bounds__(HrCfg<D>::THREADS, HrCfg<D>::BLOCKS_PER_SM)
 head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
                  TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
-                 int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H) {
+                 int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H,
+                 const float* __restrict__ lambda_rows, int ridge_mode) {
     // Prefill (lens == nullptr): block (i, bh) solves row i of head bh; n is the sequence length.
     // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
     // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
@@ -153,7 +154,9 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         lsum += e;
     }
     const double omega = block_reduce<HR_THREADS>(lsum, false, red);
-    const double lambda_m = lambda * exp(-m);
+    // per-row ridge if given (prefill: [B,H,n]; decode: [B,H]); see lla_ridge_mode for the two frames
+    const double lam_i = lambda_rows ? (double)lambda_rows[row] : lambda;
+    const double lambda_m = ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * exp(-m);
     HR_T(1);
 
     // moments: Sigma (lower 4x4 tiles in registers) and mu
@@ -292,7 +295,8 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     dim3 grid(rows_per_head, a.B * a.H);
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
-        (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H);
+        (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H, a.lambda_rows,
+        a.ridge_mode);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -307,7 +311,8 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
     dim3 grid(1, a.B * a.H);
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
-        (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H);
+        (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H, a.lambda_units,
+        a.ridge_mode);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

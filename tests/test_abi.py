@@ -1,6 +1,7 @@
 """Host-only checks of the C ABI: the library loads, exports every symbol the header declares, and
 rejects bad arguments before touching a device."""
 import ctypes
+import os
 import re
 from pathlib import Path
 
@@ -38,10 +39,26 @@ def test_version_and_status_strings(lib):
     assert binding.status_string(99) == "unknown status"
 
 
-def test_struct_sizes_match_c_layout():
-    # 4 pointers, 5+2 ints, 2 floats, 2 ints, 1 float, 2 ints, 4 pointers, pointer, size_t, pointer
-    assert ctypes.sizeof(binding.ForwardParams) == 4 * 8 + 15 * 4 + 4 + 7 * 8
-    assert ctypes.sizeof(binding.DecodeParams) == 5 * 8 + 11 * 4 + 4 + 4 * 8
+def test_struct_sizes_match_c_layout(tmp_path):
+    # the ctypes mirrors against what a C compiler makes of include/lla.h
+    import subprocess
+    src = tmp_path / "sz.c"
+    src.write_text(
+        '#include <stdio.h>\n#include <stddef.h>\n#include "lla.h"\n'
+        'int main(void) { printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(lla_forward_params), sizeof(lla_decode_params),\n'
+        '  offsetof(lla_forward_params, lambda_rows), offsetof(lla_forward_params, ridge_mode),\n'
+        '  offsetof(lla_decode_params, lambda_units), offsetof(lla_decode_params, ridge_mode)); return 0; }\n')
+    exe = tmp_path / "sz"
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    subprocess.run(["gcc", "-I", inc, "-o", str(exe), str(src)], check=True)
+    got = [int(x) for x in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    F, D = binding.ForwardParams, binding.DecodeParams
+    assert got == [ctypes.sizeof(F), ctypes.sizeof(D), F.lambda_rows.offset, F.ridge_mode.offset,
+                   D.lambda_units.offset, D.ridge_mode.offset]
+    # 4 pointers, 5+2 ints, 2 floats, 2 ints, 1 float, 3 ints, 3+1 pointers, pointer, size_t, pointer; then the
+    # ridge fields (pointer, int, tail padding)
+    assert ctypes.sizeof(F) == 4 * 8 + 15 * 4 + 4 + 7 * 8 + 8 + 8
+    assert ctypes.sizeof(D) == 5 * 8 + 11 * 4 + 4 + 4 * 8 + 8 + 8
 
 
 def test_argument_validation_without_device(lib):

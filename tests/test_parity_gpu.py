@@ -287,3 +287,44 @@ def test_host_buffer_entry_points(oracle):
     L.lla_decode_host(hq, hk, hv, hl, hout, wd.B, wd.H, wd.n, wd.d, wd.dv, L.LLA_BF16, L.LLA_F32, wd.scale,
                       wd.lam, stream_ptr())
     assert row_err(hout.numpy(), dref).max() <= TOL_BF16
+
+
+@pytest.mark.parametrize("dtype,d,n", [("bf16", 64, 700), ("bf16", 128, 400), ("f32", 16, 200)])
+def test_ridge_variants_forward(oracle, dtype, d, n):
+    # per-token ridge and the ridge of the printed algorithm (both only change lambda'_i)
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=n, d=d, dv=d, dtype=dtype, seed=70 + d)
+    q, k, v = inputs.make_prefill(w)
+    q = (q * 3.0).astype(np.float32)                      # row maxima well away from 0: the two variants differ
+    if dtype == "bf16":
+        q = inputs.round_to_bf16(q)
+    lam_rows = np.random.default_rng(71).uniform(0.5, 2.0, size=(w.B, w.H, w.n)).astype(np.float32) * w.lam
+    dlam = torch.from_numpy(lam_rows).cuda()
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    ref_def = oracle.forward(q, k, v, w.scale, lam_rows.astype(np.float64))
+    got = forward(w, q, k, v, out_dtype="f32", lambda_rows=dlam)
+    assert row_err(got, ref_def).max() <= tol
+    ref_pr = oracle.forward(q, k, v, w.scale, w.lam, ridge_mode="printed")
+    got = forward(w, q, k, v, out_dtype="f32", ridge_mode=L.LLA_RIDGE_PRINTED)
+    assert row_err(got, ref_pr).max() <= tol
+    assert row_err(ref_pr.reshape(-1, d), oracle.forward(q, k, v, w.scale, w.lam).reshape(-1, d)).max() > 10 * tol
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 16)])
+def test_ridge_variants_decode(oracle, dtype, d):
+    w = inputs.CONFIGS[5].shrink(B=3, H=2, n=900, d=d, dv=d, dtype=dtype, len_min=40, len_max=900, seed=72 + d)
+    q, kc, vc, lens = inputs.make_decode(w)
+    q = (q * 3.0).astype(np.float32)
+    if dtype == "bf16":
+        q = inputs.round_to_bf16(q)
+    lam_units = np.random.default_rng(73).uniform(0.5, 2.0, size=(w.B, w.H)).astype(np.float32) * w.lam
+    dq, dk, dv_ = dev(q, dtype), dev(kc, dtype), dev(vc, dtype)
+    dl = torch.from_numpy(lens).cuda()
+    dlam = torch.from_numpy(lam_units).cuda()
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    for mode, name in ((L.LLA_RIDGE_DEFINITION, "definition"), (L.LLA_RIDGE_PRINTED, "printed")):
+        ref = oracle.decode(q, kc, vc, lens, w.scale, lam_units.astype(np.float64), ridge_mode=name)
+        out = torch.full((w.B, w.H, d), float("nan"), dtype=torch.float32, device="cuda")
+        L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, w.H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                        out_dtype=L.LLA_F32, splits=1, lambda_units=dlam, ridge_mode=mode, stream=stream_ptr())
+        torch.cuda.synchronize()
+        assert row_err(out.cpu().numpy(), ref).max() <= tol, name
