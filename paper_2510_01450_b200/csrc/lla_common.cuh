@@ -113,6 +113,7 @@ __device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __fl
 // Dense symmetric positive-definite solve in shared memory, double precision, by a whole block.
 //   S   : D x D, row stride lds doubles, lower triangle filled; destroyed (LDL^T in place)
 //   rhs : D doubles; replaced by the solution
+//   n   : active size, a multiple of 8 and at most D (D only sizes the register arrays)
 // Returns false if a pivot was not positive.  Every thread of the block must call it; blockDim.x
 // must be a multiple of 32.
 //
@@ -184,7 +185,7 @@ __device__ __forceinline__ void ldlt_diag_block(double* S, int lds, int c0) {
 }
 
 template <int D>
-__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs LDLT_TARG) {
+__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs, int n = D LDLT_TARG) {
     LDLT_T0;
     const int tid = threadIdx.x, nt = blockDim.x;
     const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
@@ -196,13 +197,13 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
     if (ty == 0) ldlt_diag_block<NB>(S, lds, 0);
     __syncthreads();
     LDLT_T(0);
-    for (int c0 = 0; c0 < D; c0 += NB) {
+    for (int c0 = 0; c0 < n; c0 += NB) {
         double dinv[NB];
 #pragma unroll
         for (int k = 0; k < NB; ++k) dinv[k] = S[(c0 + k) * lds + c0 + k + 1];
         // (ii)
-        for (int r = c0 + NB + tid; r <= D; r += nt) {
-            double* rowp = r < D ? S + r * lds : rhs;
+        for (int r = c0 + NB + tid; r <= n; r += nt) {
+            double* rowp = r < n ? S + r * lds : rhs;
             double x[NB];
 #pragma unroll
             for (int k = 0; k < NB; ++k) x[k] = rowp[c0 + k];
@@ -221,20 +222,20 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
         // panel entries of its columns c2 in registers for the whole update and walks down the rows;
         // a row's eight panel entries are the same address for every lane (broadcast loads), so
         // shared-memory traffic is one load and one store per updated element.
-        if (c0 + NB < D) {
+        if (c0 + NB < n) {
             double u[SLOTS][NB];
 #pragma unroll
             for (int sl = 0; sl < SLOTS; ++sl) {
                 const int c2 = c0 + NB + tx + 32 * sl;
 #pragma unroll
-                for (int k = 0; k < NB; ++k) u[sl][k] = c2 < D ? S[c2 * lds + c0 + k] * dinv[k] : 0.0;
+                for (int k = 0; k < NB; ++k) u[sl][k] = c2 < n ? S[c2 * lds + c0 + k] * dinv[k] : 0.0;
             }
             auto update_row = [&](int r) {
-                double* rowp = r < D ? S + r * lds : rhs;
+                double* rowp = r < n ? S + r * lds : rhs;
                 double a[NB];
 #pragma unroll
                 for (int k = 0; k < NB; ++k) a[k] = rowp[c0 + k];
-                const int cmax = r < D ? r : D - 1;
+                const int cmax = r < n ? r : n - 1;
 #pragma unroll
                 for (int sl = 0; sl < SLOTS; ++sl) {
                     const int c2 = c0 + NB + tx + 32 * sl;
@@ -265,16 +266,16 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
                 __syncwarp();
                 ldlt_diag_block<NB>(S, lds, c0 + NB);
                 if (ny == 1)
-                    for (int r = c0 + 2 * NB; r <= D; ++r) update_row(r);
+                    for (int r = c0 + 2 * NB; r <= n; ++r) update_row(r);
             } else {
-                for (int r = c0 + 2 * NB + ty - 1; r <= D; r += ny - 1) update_row(r);
+                for (int r = c0 + 2 * NB + ty - 1; r <= n; r += ny - 1) update_row(r);
             }
             __syncthreads();
             LDLT_T(2);
         }
     }
     bool ok = true;
-    for (int k = 0; k < D; ++k)
+    for (int k = 0; k < n; ++k)
         if (!(S[k * lds + k] > 0.0)) ok = false;
     LDLT_T(3);
     // rhs now holds y with L y = b.  Backward: x_t = (y_t - sum_{r>t} S[r][t] x_r) / D_t.
@@ -286,9 +287,9 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
         for (int u = 0; u < PER; ++u) {
             const int t = tx + 32 * u;
             part[u] = 0.0;
-            yv[u] = t < D ? rhs[t] : 0.0;
+            yv[u] = t < n ? rhs[t] : 0.0;
         }
-        for (int c0 = D - NB; c0 >= 0; c0 -= NB) {
+        for (int c0 = n - NB; c0 >= 0; c0 -= NB) {
             // y - (contributions of later panels) for the eight unknowns c0 + i of this panel
             double mine = 0.0;
 #pragma unroll

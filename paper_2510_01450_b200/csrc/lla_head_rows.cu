@@ -121,8 +121,10 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     double* zc = S;                         // HR_CHUNK * D  centred keys of the current chunk (over S)
 
     const int tid = threadIdx.x;
-    const int bh = blockIdx.y;
-    const int i = blockIdx.x;               // row index inside the head
+    // blockIdx.x (fastest in launch order) is the head, blockIdx.y counts rows from the last one down:
+    // rows with the most keys are the longest blocks and start first, so the tail of the launch is short
+    const int bh = blockIdx.x;
+    const int i = rows_per_head - 1 - blockIdx.y;   // row index inside the head
     if (i >= rows_per_head) return;
     int L = causal ? i + 1 : n;
     if (lens) {
@@ -159,111 +161,178 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     const double lambda_m = ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * exp(-m);
     HR_T(1);
 
-    // moments: Sigma (lower 4x4 tiles in registers) and mu
+    // Rows with at most d keys (and a positive ridge) go through the dual (Gram) form: with Z the
+    // L x d matrix of centred keys, w_j (1 - z_j . rho) = lambda' alpha_j where
+    // (Z Z^T + lambda' diag(1/w)) alpha = 1  --  an L x L system instead of d x d, free of the
+    // cancellation in 1 - z . rho, and rho = Z^T alpha.  The system is padded to a multiple of 8 with
+    // identity rows.
+    double csum = 0.0, rho_val = 0.0;
+    bool bad = false;
+    const bool dual = L <= D && lambda_m > 0.0;          // block-uniform
+    const int Lp = (L + 7) & ~7;                         // dual: system size padded to the panel width
+    // lower-triangular 4x4 register tiles of the matrix being built (Sigma, or the Gram matrix):
+    // tile index -> (row tile, column tile); interleaved: rows tr + T1 a, columns tc + T1 b
+    const int T1 = dual ? Lp / 4 : C::TILES_1D, ntiles = T1 * (T1 + 1) / 2;
     double acc[C::TILES_PER_THREAD][4][4];
     int tr[C::TILES_PER_THREAD], tc[C::TILES_PER_THREAD];
 #pragma unroll
     for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
         const int tile = tid + t * HR_THREADS;
-        // tile index -> (row tile, col tile) in the lower triangle
         int r = 0;
-        if (tile < C::TILES) {
+        if (tile < ntiles) {
             r = (int)((sqrt(8.0 * tile + 1.0) - 1.0) * 0.5);
             while ((r + 1) * (r + 2) / 2 <= tile) ++r;
             while (r * (r + 1) / 2 > tile) --r;
         }
-        tr[t] = tile < C::TILES ? r : -1;
-        tc[t] = tile < C::TILES ? tile - r * (r + 1) / 2 : 0;
+        tr[t] = tile < ntiles ? r : -1;
+        tc[t] = tile < ntiles ? tile - r * (r + 1) / 2 : 0;
 #pragma unroll
         for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) acc[t][a][b] = 0.0;
     }
-    double mu_acc = 0.0;  // thread tid < D owns mu[tid]
-    // The keys of a chunk are fetched (element pairs, coalesced) one chunk ahead, so the global-load
-    // latency hides behind the accumulation of the chunk before.
-    constexpr int PAIRS = (HR_CHUNK * D / 2 + HR_THREADS - 1) / HR_THREADS;
-    float pre[PAIRS][2];
-    auto fetch = [&](int j0) {
-        const int np = min(HR_CHUNK, L - j0) * (D / 2);
-#pragma unroll
-        for (int u = 0; u < PAIRS; ++u) {
-            const int pi = tid + HR_THREADS * u;
-            if (pi < np) load2(kb + (size_t)j0 * D + 2 * pi, pre[u][0], pre[u][1]);
-        }
-    };
-    fetch(0);
-    for (int j0 = 0; j0 < L; j0 += HR_CHUNK) {
-        const int jn = min(HR_CHUNK, L - j0);
-        __syncthreads();
-#pragma unroll
-        for (int u = 0; u < PAIRS; ++u) {
-            const int pi = tid + HR_THREADS * u;
-            if (pi < jn * (D / 2)) {
-                const int c = (2 * pi) % D;
-                *reinterpret_cast<double2*>(zc + 2 * pi) = make_double2((double)pre[u][0] - qd[c], (double)pre[u][1] - qd[c + 1]);
-            }
+    if (dual) {
+        const int LZ = Lp + 1;                            // odd row stride of the staged keys
+        double* zt = S;                                   // zt[c * LZ + j] = k_j[c] - q[c]  (over S: D * LZ <= S_DOUBLES)
+        for (int e = tid; e < Lp * D; e += HR_THREADS) {
+            const int j = e / D, c = e - j * D;
+            zt[c * LZ + j] = j < L ? (double)to_f32(kb[(size_t)j * D + c]) - qd[c] : 0.0;
         }
         __syncthreads();
-        if (j0 + HR_CHUNK < L) fetch(j0 + HR_CHUNK);
-        if (tid < D)
-            for (int jj = 0; jj < jn; ++jj) mu_acc += w[j0 + jj] * zc[jj * D + tid];
+        // Gram matrix
 #pragma unroll
         for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
             if (tr[t] < 0) continue;
-            // interleaved 4x4 tile: rows tr + T1*a, columns tc + T1*b, so that neighbouring threads
-            // read neighbouring doubles (no shared-memory bank conflicts)
-            const int r0 = tr[t], c0 = tc[t];
-            for (int jj = 0; jj < jn; ++jj) {
-                const double wj = w[j0 + jj];
-                double zr[4], zcv[4];
+            for (int c = 0; c < D; ++c) {
+                double zj[4], zl[4];
 #pragma unroll
-                for (int a = 0; a < 4; ++a) {
-                    zr[a] = wj * zc[jj * D + r0 + C::TILES_1D * a];
-                    zcv[a] = zc[jj * D + c0 + C::TILES_1D * a];
+                for (int x = 0; x < 4; ++x) {
+                    zj[x] = zt[c * LZ + tr[t] + T1 * x];
+                    zl[x] = zt[c * LZ + tc[t] + T1 * x];
                 }
 #pragma unroll
-                for (int a = 0; a < 4; ++a)
+                for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) acc[t][a][b] += zr[a] * zcv[b];
+                    for (int y = 0; y < 4; ++y) acc[t][x][y] += zj[x] * zl[y];
             }
         }
-    }
-    HR_T(2);
-    __syncthreads();   // the staged keys (lying over S) are no longer read
+        __syncthreads();       // the staged keys (lying over S) are no longer read
 #pragma unroll
-    for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
-        if (tr[t] < 0) continue;
+        for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
+            if (tr[t] < 0) continue;
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+            for (int x = 0; x < 4; ++x)
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int r = tr[t] + C::TILES_1D * a, c = tc[t] + C::TILES_1D * b;
-                if (c <= r) S[r * C::LDS + c] = acc[t][a][b] + (r == c ? lambda_m : 0.0);
-                else if (tr[t] != tc[t]) S[c * C::LDS + r] = acc[t][a][b];   // mirror of tile (tc, tr)
+                for (int y = 0; y < 4; ++y) {
+                    const int r = tr[t] + T1 * x, c = tc[t] + T1 * y;
+                    // diagonal: ridge / weight for live keys (weights clamped away from 0), 1 for padding
+                    const double dg = r < L ? lambda_m / fmax(w[r], 1e-290) : 1.0;
+                    if (c <= r) S[r * C::LDS + c] = acc[t][x][y] + (r == c ? dg : 0.0);
+                    else if (tr[t] != tc[t]) S[c * C::LDS + r] = acc[t][x][y];
+                }
+        }
+        for (int j = tid; j < Lp; j += HR_THREADS) rhs[j] = j < L ? 1.0 : 0.0;
+        __syncthreads();
+        bad = !block_ldlt_solve<D>(S, C::LDS, rhs, Lp);
+        // coefficients c_j = lambda' alpha_j
+        for (int j = tid; j < L; j += HR_THREADS) {
+            const double cj = lambda_m * rhs[j];
+            w[j] = cj;
+            csum += cj;
+        }
+        if (rho_out && tid < D) {                         // rho = Z^T alpha
+            double acc_r = 0.0;
+            for (int j = 0; j < L; ++j) acc_r += rhs[j] * ((double)to_f32(kb[(size_t)j * D + tid]) - qd[tid]);
+            rho_val = acc_r;
+        }
+    } else {
+        // moments: Sigma and mu
+        double mu_acc = 0.0;  // thread tid < D owns mu[tid]
+        // The keys of a chunk are fetched (element pairs, coalesced) one chunk ahead, so the global-load
+        // latency hides behind the accumulation of the chunk before.
+        constexpr int PAIRS = (HR_CHUNK * D / 2 + HR_THREADS - 1) / HR_THREADS;
+        float pre[PAIRS][2];
+        auto fetch = [&](int j0) {
+            const int np = min(HR_CHUNK, L - j0) * (D / 2);
+    #pragma unroll
+            for (int u = 0; u < PAIRS; ++u) {
+                const int pi = tid + HR_THREADS * u;
+                if (pi < np) load2(kb + (size_t)j0 * D + 2 * pi, pre[u][0], pre[u][1]);
             }
-    }
-    if (tid < D) rhs[tid] = mu_acc;
-    __syncthreads();
+        };
+        fetch(0);
+        for (int j0 = 0; j0 < L; j0 += HR_CHUNK) {
+            const int jn = min(HR_CHUNK, L - j0);
+            __syncthreads();
+    #pragma unroll
+            for (int u = 0; u < PAIRS; ++u) {
+                const int pi = tid + HR_THREADS * u;
+                if (pi < jn * (D / 2)) {
+                    const int c = (2 * pi) % D;
+                    *reinterpret_cast<double2*>(zc + 2 * pi) = make_double2((double)pre[u][0] - qd[c], (double)pre[u][1] - qd[c + 1]);
+                }
+            }
+            __syncthreads();
+            if (j0 + HR_CHUNK < L) fetch(j0 + HR_CHUNK);
+            if (tid < D)
+                for (int jj = 0; jj < jn; ++jj) mu_acc += w[j0 + jj] * zc[jj * D + tid];
+    #pragma unroll
+            for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
+                if (tr[t] < 0) continue;
+                // interleaved 4x4 tile: rows tr + T1*a, columns tc + T1*b, so that neighbouring threads
+                // read neighbouring doubles (no shared-memory bank conflicts)
+                const int r0 = tr[t], c0 = tc[t];
+                for (int jj = 0; jj < jn; ++jj) {
+                    const double wj = w[j0 + jj];
+                    double zr[4], zcv[4];
+    #pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        zr[a] = wj * zc[jj * D + r0 + C::TILES_1D * a];
+                        zcv[a] = zc[jj * D + c0 + C::TILES_1D * a];
+                    }
+    #pragma unroll
+                    for (int a = 0; a < 4; ++a)
+    #pragma unroll
+                        for (int b = 0; b < 4; ++b) acc[t][a][b] += zr[a] * zcv[b];
+                }
+            }
+        }
+        HR_T(2);
+        __syncthreads();   // the staged keys (lying over S) are no longer read
+    #pragma unroll
+        for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
+            if (tr[t] < 0) continue;
+    #pragma unroll
+            for (int a = 0; a < 4; ++a)
+    #pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int r = tr[t] + C::TILES_1D * a, c = tc[t] + C::TILES_1D * b;
+                    if (c <= r) S[r * C::LDS + c] = acc[t][a][b] + (r == c ? lambda_m : 0.0);
+                    else if (tr[t] != tc[t]) S[c * C::LDS + r] = acc[t][a][b];   // mirror of tile (tc, tr)
+                }
+        }
+        if (tid < D) rhs[tid] = mu_acc;
+        __syncthreads();
 
-    HR_T(3);
-    // rhs <- Sigma^{-1} mu (LDL^T in shared memory)
-#ifdef LLA_HR_TIMING
-    const bool bad = !block_ldlt_solve<D>(S, C::LDS, rhs, status ? status + 16 : nullptr);
-#else
-    const bool bad = !block_ldlt_solve<D>(S, C::LDS, rhs);
-#endif
-    HR_T(4);
+        HR_T(3);
+        // rhs <- Sigma^{-1} mu (LDL^T in shared memory)
+    #ifdef LLA_HR_TIMING
+        bad = !block_ldlt_solve<D>(S, C::LDS, rhs, D, status ? status + 16 : nullptr);
+    #else
+        bad = !block_ldlt_solve<D>(S, C::LDS, rhs);
+    #endif
+        HR_T(4);
 
-    // coefficients c_j = w_j (1 - z_j . rho) and their sum (= omega - mu . rho)
-    double qrho = 0.0;
-    for (int c = 0; c < D; ++c) qrho += qd[c] * rhs[c];
-    double csum = 0.0;
-    for (int j = tid; j < L; j += HR_THREADS) {
-        const double t = dot_row<D>(rhs, kb + (size_t)j * D) - qrho;
-        const double cj = w[j] * (1.0 - t);
-        w[j] = cj;
-        csum += cj;
+        // coefficients c_j = w_j (1 - z_j . rho) and their sum (= omega - mu . rho)
+        double qrho = 0.0;
+        for (int c = 0; c < D; ++c) qrho += qd[c] * rhs[c];
+        for (int j = tid; j < L; j += HR_THREADS) {
+            const double t = dot_row<D>(rhs, kb + (size_t)j * D) - qrho;
+            const double cj = w[j] * (1.0 - t);
+            w[j] = cj;
+            csum += cj;
+        }
+        if (tid < D) rho_val = rhs[tid];
     }
     const double denom = block_reduce<HR_THREADS>(csum, false, red);
     HR_T(5);
@@ -273,7 +342,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         store_out(out + row * DV + c, (float)(o / denom));
     }
     HR_T(6);
-    if (rho_out && tid < D) rho_out[row * D + tid] = (float)rhs[tid];
+    if (rho_out && tid < D) rho_out[row * D + tid] = (float)rho_val;
     if (tid == 0) {
         if (stats) {
             stats[row * 3 + 0] = (float)m;
@@ -292,7 +361,7 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     auto kern = head_rows_kernel<D, D, TIn, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
-    dim3 grid(rows_per_head, a.B * a.H);
+    dim3 grid(a.B * a.H, rows_per_head);
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
         (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H, a.lambda_rows,
@@ -308,7 +377,7 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
     auto kern = head_rows_kernel<D, D, TIn, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
-    dim3 grid(1, a.B * a.H);
+    dim3 grid(a.B * a.H, 1);
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
         (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H, a.lambda_units,
