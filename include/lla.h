@@ -241,10 +241,12 @@ int lla_decode_noalloc(const void *q, const void *kcache, const void *vcache, co
                        void *out, int B, int H, int Lmax, int d, int dv, int in_dtype,
                        int out_dtype, float scale, float lambda, int splits, void *stream);
 
-/* Scratch bytes lla_forward_ex needs for this problem (0 when none). Host-only arithmetic.
- * The d = 128 tensor-core kernel additionally keeps one library-owned device buffer per GPU
- * (2 x SM count x 192 KiB, allocated with cudaMalloc by the first such call and reused by all
- * later ones; blocks address it by SM id, so concurrent calls may share it). */
+/* Scratch bytes lla_forward_ex can use for this problem (0 when none).  Only the d = 128 tensor-core
+ * kernel has any (2 x SM count x 192 KiB: per-SM slots for the CG row vectors; the call queries the
+ * current device's SM count).  It is optional: given a workspace of that size the call allocates
+ * nothing (two calls that may run at the same time need separate workspaces); without one the
+ * library keeps its own buffer per GPU, allocated with cudaMalloc by the first such call and shared
+ * safely by all later ones (blocks address it by SM id and one block fills an SM). */
 size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl);
 
 /* Scratch bytes lla_decode_ex uses for this problem and split count: required when splits > 1,

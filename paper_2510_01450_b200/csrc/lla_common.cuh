@@ -61,6 +61,7 @@ int launch_head_rows(const ForwardArgs& a);
 int launch_forward_simt(const ForwardArgs& a);
 int launch_forward_tensor(const ForwardArgs& a);
 bool forward_tensor_supported(const ForwardArgs& a);
+size_t forward_tensor_scratch_bytes();         // d = 128 row-state scratch (0 if the device cannot be queried)
 int launch_decode(const DecodeArgs& a);
 int launch_head_rows_decode(const DecodeArgs& a);
 bool decode_tensor_supported(const DecodeArgs& a);

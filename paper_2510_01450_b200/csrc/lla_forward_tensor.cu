@@ -871,7 +871,11 @@ int launch_t(const ForwardArgs& a) {
         LLA_CUDA_TRY(cudaGetDevice(&dev));
         LLA_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         prm.scratch_slots = 2 * sms;     // SM ids are dense in practice; the margin is checked in the kernel
-        prm.scratch = scratch_for_device((size_t)prm.scratch_slots * Cfg::SCRATCH_FLOATS_PER_SM * sizeof(float));
+        const size_t need = (size_t)prm.scratch_slots * Cfg::SCRATCH_FLOATS_PER_SM * sizeof(float);
+        // the caller's workspace if it is large enough (then nothing is allocated, but two calls that may
+        // run at the same time must not share it), else the library's own per-device buffer
+        if (a.workspace && a.workspace_bytes >= need) prm.scratch = static_cast<float*>(a.workspace);
+        else prm.scratch = scratch_for_device(need);
         if (!prm.scratch) return LLA_ERR_CUDA;
     }
 #if defined(LLA_TC_TIMING) || defined(LLA_TC_TRACE)
@@ -886,6 +890,13 @@ int launch_t(const ForwardArgs& a) {
 }
 
 }  // namespace
+
+size_t forward_tensor_scratch_bytes() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return (size_t)2 * sms * TcCfg<128>::SCRATCH_FLOATS_PER_SM * sizeof(float);
+}
 
 bool forward_tensor_supported(const ForwardArgs& a) {
     return a.in_dtype == LLA_BF16 && (a.d == 64 || a.d == 128) && a.dv == a.d && get_encode() != nullptr;

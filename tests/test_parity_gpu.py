@@ -328,3 +328,16 @@ def test_ridge_variants_decode(oracle, dtype, d):
                         out_dtype=L.LLA_F32, splits=1, lambda_units=dlam, ridge_mode=mode, stream=stream_ptr())
         torch.cuda.synchronize()
         assert row_err(out.cpu().numpy(), ref).max() <= tol, name
+
+
+def test_forward_d128_with_caller_workspace(oracle):
+    # the d = 128 tensor-core kernel keeps its row vectors off chip: in the caller's workspace when one
+    # of the advertised size is passed (no allocation inside the call), else in the library's own buffer
+    w = inputs.CONFIGS[4].shrink(H=2, n=700)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    nbytes = L.lla_forward_workspace_bytes(w.B, w.H, w.n, w.d, w.dv)
+    assert nbytes >= 148 * 3 * 128 * 128 * 4
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    got = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, workspace=ws, workspace_bytes=nbytes)
+    assert row_err(got, ref).max() <= TOL_BF16
