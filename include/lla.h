@@ -126,6 +126,8 @@ int lla_decode_f32(const void *q, const void *kcache, const void *vcache, const 
  *   iters     : optional [B, H, n] int32, CG iterations executed for the row (-1 for rows solved
  *               directly)
  *   device_status : optional int[LLA_STATUS_WORDS] on the device
+ *   q_rows    : 0 (or n) for the plain forward; 0 < q_rows < n for a chunk of queries at the last
+ *               q_rows positions against all n keys (see the field's comment below)
  *   lambda_rows : optional [B, H, n] fp32 on the device, one ridge per query row (the paper's
  *               per-token regularisation); when not NULL it replaces `lambda`
  *   ridge_mode : lla_ridge_mode (0 = the definition; 1 = Algorithm 1/2 as printed)
@@ -154,6 +156,11 @@ typedef struct lla_forward_params {
     const float *lambda_rows;   /* optional [B, H, n] fp32 on the device: one ridge per query row
                                    (per-token regularisation); replaces `lambda` when not NULL */
     int ridge_mode;             /* lla_ridge_mode */
+    int q_rows;                 /* 0 or n: one query per key position.  0 < q_rows < n: prefill of the
+                                   LAST q_rows positions against all n keys (a chunk appended to an
+                                   existing cache): q, out, rho, stats, iters and lambda_rows then have
+                                   q_rows rows per head; query row r sits at position n - q_rows + r and,
+                                   when causal, sees keys 0 .. n - q_rows + r */
 } lla_forward_params;
 
 int lla_forward_ex(const lla_forward_params *p);

@@ -45,6 +45,7 @@ class ForwardParams(ctypes.Structure):
         ("rho", ctypes.c_void_p), ("stats", ctypes.c_void_p), ("iters", ctypes.c_void_p),
         ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p), ("lambda_rows", ctypes.c_void_p), ("ridge_mode", ctypes.c_int),
+        ("q_rows", ctypes.c_int),
     ]
 
 
@@ -154,7 +155,7 @@ def lla_decode_host(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, in_dtype, o
 def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=LLA_BF16, out_dtype=LLA_BF16,
                    max_iters=0, tol=0.0, head_rows=0, impl=LLA_IMPL_AUTO, phases=0, rho=None, stats=None, iters=None,
                    device_status=None, workspace=None, workspace_bytes=0, stream=0, lambda_rows=None,
-                   ridge_mode=LLA_RIDGE_DEFINITION):
+                   ridge_mode=LLA_RIDGE_DEFINITION, q_rows=0):
     p = ForwardParams()
     p.q, p.k, p.v, p.out = _p(q), _p(k), _p(v), _p(out)
     p.B, p.H, p.n, p.d, p.dv = B, H, n, d, dv
@@ -163,7 +164,7 @@ def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=
     p.max_iters, p.tol, p.head_rows, p.impl, p.phases = max_iters, tol, head_rows, impl, phases
     p.rho, p.stats, p.iters, p.device_status = _p(rho), _p(stats), _p(iters), _p(device_status)
     p.workspace, p.workspace_bytes, p.stream = _p(workspace), workspace_bytes, _p(stream)
-    p.lambda_rows, p.ridge_mode = _p(lambda_rows), ridge_mode
+    p.lambda_rows, p.ridge_mode, p.q_rows = _p(lambda_rows), ridge_mode, q_rows
     _check(load().lla_forward_ex(ctypes.byref(p)), "lla_forward_ex")
 
 

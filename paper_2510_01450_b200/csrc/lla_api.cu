@@ -68,6 +68,7 @@ int check_forward(const lla_forward_params* p) {
     if (p->B < 1 || p->H < 1 || p->n < 1 || p->d < 1 || p->dv < 1) return LLA_ERR_INVALID_ARG;
     if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
     if (p->ridge_mode != LLA_RIDGE_DEFINITION && p->ridge_mode != LLA_RIDGE_PRINTED) return LLA_ERR_INVALID_ARG;
+    if (p->q_rows < 0 || p->q_rows > p->n) return LLA_ERR_INVALID_ARG;
     if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535 || (p->n + 127) / 128 > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
@@ -97,6 +98,7 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.stream = (cudaStream_t)p->stream;
     a.lambda_rows = p->lambda_rows;
     a.ridge_mode = p->ridge_mode;
+    a.nq = p->q_rows > 0 ? p->q_rows : p->n;
     return a;
 }
 

@@ -31,8 +31,9 @@ struct ForwardArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
-    const float* lambda_rows;   // optional per-row ridge [B, H, n]
+    const float* lambda_rows;   // optional per-row ridge [B, H, nq]
     int ridge_mode;             // lla_ridge_mode
+    int nq;                     // query rows per head (the last nq of the n positions); nq == n: plain prefill
 };
 
 struct DecodeArgs {
@@ -56,7 +57,7 @@ struct DecodeArgs {
 };
 
 // Launchers implemented in the other translation units; each returns an lla_status.
-int head_rows_count(const ForwardArgs& a);   // leading rows per head solved directly
+int head_rows_count(const ForwardArgs& a);   // leading query rows per head solved directly
 int launch_head_rows(const ForwardArgs& a);
 int launch_forward_simt(const ForwardArgs& a);
 int launch_forward_tensor(const ForwardArgs& a);

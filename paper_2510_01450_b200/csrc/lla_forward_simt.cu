@@ -61,7 +61,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                     TOut* __restrict__ out, int n, int causal, float scale, float lambda,
                     int head_rows, int max_iters, float tol, int first_tile,
                     float* __restrict__ rho_out, float* __restrict__ stats, int* __restrict__ iters_out,
-                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode) {
+                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq) {
     constexpr int ROWS = FS_THREADS / TPR;
     constexpr int NG = D / (4 * TPR);    // float4 groups per thread (keys)
     constexpr int NGV = DV / (4 * TPR);  // float4 groups per thread (values)
@@ -76,16 +76,17 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     const int r0 = tile * ROWS;
     const int lr = threadIdx.x % TPR;
     const int row = r0 + threadIdx.x / TPR;
-    const int L = causal ? row + 1 : n;                 // visible keys of this row
-    const bool row_ok = row < n && L >= head_rows;      // other rows: out of range or solved directly
-    const int jend = causal ? min(n, r0 + ROWS) : n;    // keys this block must sweep
+    const int off = n - nq;                             // query row r sits at position off + r
+    const int L = causal ? off + row + 1 : n;           // visible keys of this row
+    const bool row_ok = row < nq && L >= head_rows;     // other rows: out of range or solved directly
+    const int jend = causal ? min(n, off + r0 + ROWS) : n;   // keys this block must sweep
     const TIn* kb = k + (size_t)bh * n * D;
     const TIn* vb = v + (size_t)bh * n * DV;
 
     float4 qv[NG], kbar[NG];
 #pragma unroll
     for (int g = 0; g < NG; ++g) {
-        qv[g] = row < n ? load4(q + ((size_t)bh * n + row) * D + 4 * (g * TPR + lr))
+        qv[g] = row < nq ? load4(q + ((size_t)bh * nq + row) * D + 4 * (g * TPR + lr))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
         kbar[g] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
@@ -129,7 +130,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
         }
     }
     const float inv_omega = row_ok ? 1.f / omega : 0.f;
-    const float lam_i = (lambda_rows && row < n) ? lambda_rows[(size_t)bh * n + row] : lambda;
+    const float lam_i = (lambda_rows && row < nq) ? lambda_rows[(size_t)bh * nq + row] : lambda;
     const float ridge = row_ok ? (ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * exp_w<ACCURATE>(-m)) * inv_omega : 0.f;
 
     // ---- conjugate gradients on C y = kbar - q (Algorithm 2) ----
@@ -262,7 +263,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     }
     if (row_ok) {
         const float inv_den = 1.f / den;
-        const size_t rowi = (size_t)bh * n + row;
+        const size_t rowi = (size_t)bh * nq + row;
         TOut* orow = out + rowi * DV;
 #pragma unroll
         for (int g = 0; g < NGV; ++g) {
@@ -298,10 +299,10 @@ template <int D, int TPR, typename TIn, typename TOut>
 int launch_t(const ForwardArgs& a) {
     constexpr int ROWS = FS_THREADS / TPR;
     const int hr = head_rows_count(a);
-    if (!a.causal && hr >= a.n) return LLA_OK;   // every row was solved directly
+    if (!a.causal && hr >= a.nq) return LLA_OK;  // every row was solved directly
     // causal: rows 0..hr-1 are done elsewhere; skip query tiles that hold only such rows
     const int first_tile = a.causal ? hr / ROWS : 0;
-    const int tiles = (a.n + ROWS - 1) / ROWS - first_tile;
+    const int tiles = (a.nq + ROWS - 1) / ROWS - first_tile;
     if (tiles <= 0) return LLA_OK;
     const size_t smem = sizeof(float) * (size_t)FS_BC * (D + D);
     auto kern = forward_simt_kernel<D, D, TPR, TIn, TOut>;
@@ -310,7 +311,7 @@ int launch_t(const ForwardArgs& a) {
     kern<<<grid, FS_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, a.causal, a.scale,
         a.lambda, a.head_rows > 0 ? a.head_rows : 0, a.max_iters, a.tol, first_tile, a.rho, a.stats,
-        a.iters, a.status, a.lambda_rows, a.ridge_mode);
+        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

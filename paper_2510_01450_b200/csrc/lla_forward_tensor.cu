@@ -172,7 +172,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(
 
 struct TcParams {
     unsigned long long* dbg;
-    int n, causal, head_rows, max_iters, first_tile;
+    int n, nq, causal, head_rows, max_iters, first_tile;   // n keys; nq query rows at positions n - nq .. n - 1
     float scale, lambda, tol;
     float* rho;
     float* stats;
@@ -230,9 +230,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int bh = blockIdx.x;
     const int tile = prm.first_tile + (prm.use_order ? (int)prm.order[blockIdx.y] : (int)(gridDim.y - 1 - blockIdx.y));
     const int r0 = tile * TC_BR;
-    const int n = prm.n;
+    const int n = prm.n, nq = prm.nq, off = n - nq;     // query row r sits at position off + r
     const int nblk_all = (n + TC_BC - 1) / TC_BC;
-    const int nblk = prm.causal ? min(nblk_all, (r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
+    const int nblk = prm.causal ? min(nblk_all, (off + r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
     const bool split = nblk <= TC_SPLIT_MAX;
 
     if (tid == 0) {
@@ -406,8 +406,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         TC_EV_DECL(2 + half);
         const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
         const int row = r0 + lrow;
-        const int L = prm.causal ? row + 1 : n;
-        const bool row_ok = row < n && L >= prm.head_rows;
+        const int L = prm.causal ? off + row + 1 : n;
+        const bool row_ok = row < nq && L >= prm.head_rows;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const int c0 = half * NCOL;                        // first row-vector column owned by this thread
         // byte offset of this thread's chunk ch (8 columns) of row lrow inside a swizzled operand
@@ -615,7 +615,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (ok) {
                 omega = pair_sum(part);
                 inv_omega = 1.f / omega;
-                const float lam_i = (prm.lambda_rows && row < n) ? prm.lambda_rows[(size_t)bh * n + row] : prm.lambda;
+                const float lam_i = (prm.lambda_rows && row < nq) ? prm.lambda_rows[(size_t)bh * nq + row] : prm.lambda;
                 ridge = (prm.ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * ex2f(-mx2)) * inv_omega;
                 float rr_p = 0.f, ab_p = 0.f;
 #pragma unroll
@@ -745,7 +745,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 den = pair_sum(part);
                 if (row_ok) {
                     const float inv_den = 1.f / den;
-                    const size_t rowi = (size_t)bh * n + row;
+                    const size_t rowi = (size_t)bh * nq + row;
                     TOut* orow = out + rowi * D + c0;
 #pragma unroll
                     for (int e = 0; e < NCOL; ++e) store_out(orow + e, o[e] * inv_den);
@@ -828,12 +828,12 @@ float* scratch_for_device(size_t bytes) {
 // times more than the rest), so at short sequence lengths the first tiles are the longest blocks
 // even though their sweeps are the shortest.  The numbers are a fit to measured runs; they only
 // steer the order, never the result.
-void tile_order(TcParams& prm, int tiles, int first_tile, int n, int d, int causal) {
+void tile_order(TcParams& prm, int tiles, int first_tile, int n, int off, int d, int causal) {
     prm.use_order = 0;
     if (!causal || tiles > TC_ORDER_MAX) return;
     float cost[TC_ORDER_MAX];
     for (int t = 0; t < tiles; ++t) {
-        const int r_end = std::min(n, (first_tile + t + 1) * TC_BR);
+        const int r_end = std::min(n, off + (first_tile + t + 1) * TC_BR);      // keys the tile's last row sees
         const float its = 6.f + 50.f * (float)d / (float)r_end;
         const float nblk = (float)((r_end + TC_BC - 1) / TC_BC);
         cost[t] = (its + 3.f) * (6.f + nblk);
@@ -847,17 +847,17 @@ template <int D, typename TOut>
 int launch_t(const ForwardArgs& a) {
     using Cfg = TcCfg<D>;
     const int hr = head_rows_count(a);
-    if (!a.causal && hr >= a.n) return LLA_OK;
+    if (!a.causal && hr >= a.nq) return LLA_OK;
     const int first_tile = a.causal ? hr / TC_BR : 0;
-    const int tiles = (a.n + TC_BR - 1) / TC_BR - first_tile;
+    const int tiles = (a.nq + TC_BR - 1) / TC_BR - first_tile;
     if (tiles <= 0) return LLA_OK;
     CUtensorMap mq, mk, mv;
     const int BH = a.B * a.H;
-    if (!make_map_bf16(&mq, a.q, BH, a.n, D, TC_BR) || !make_map_bf16(&mk, a.k, BH, a.n, D, TC_BC) ||
+    if (!make_map_bf16(&mq, a.q, BH, a.nq, D, TC_BR) || !make_map_bf16(&mk, a.k, BH, a.n, D, TC_BC) ||
         !make_map_bf16(&mv, a.v, BH, a.n, D, TC_BC))
         return LLA_ERR_CUDA;
     TcParams prm;
-    prm.n = a.n; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
+    prm.n = a.n; prm.nq = a.nq; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
@@ -865,7 +865,7 @@ int launch_t(const ForwardArgs& a) {
     prm.dbg = nullptr;
     prm.scratch = nullptr;
     prm.scratch_slots = 0;
-    tile_order(prm, tiles, first_tile, a.n, D, a.causal);
+    tile_order(prm, tiles, first_tile, a.n, a.n - a.nq, D, a.causal);
     if constexpr (!Cfg::STATE_IN_SMEM) {
         int dev = 0, sms = 0;
         LLA_CUDA_TRY(cudaGetDevice(&dev));

@@ -106,7 +106,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
                  TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
                  int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H,
-                 const float* __restrict__ lambda_rows, int ridge_mode) {
+                 const float* __restrict__ lambda_rows, int ridge_mode, int nq) {
     // Prefill (lens == nullptr): block (i, bh) solves row i of head bh; n is the sequence length.
     // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
     // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
@@ -126,12 +126,12 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     const int bh = blockIdx.x;
     const int i = rows_per_head - 1 - blockIdx.y;   // row index inside the head
     if (i >= rows_per_head) return;
-    int L = causal ? i + 1 : n;
+    int L = causal ? (n - nq) + i + 1 : n;    // query row i sits at position n - nq + i
     if (lens) {
         L = max(1, min(lens[bh / H], n));
         if (L > lcap) return;               // long caches go through the moment kernel
     }
-    const size_t row = lens ? (size_t)bh : (size_t)bh * n + i;
+    const size_t row = lens ? (size_t)bh : (size_t)bh * nq + i;
     const TIn* qrow = q + row * D;
     const TIn* kb = k + (size_t)bh * n * D;
     const TIn* vb = v + (size_t)bh * n * DV;
@@ -365,7 +365,7 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
         (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H, a.lambda_rows,
-        a.ridge_mode);
+        a.ridge_mode, a.nq);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -381,7 +381,7 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
         (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H, a.lambda_units,
-        a.ridge_mode);
+        a.ridge_mode, 1);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -413,14 +413,17 @@ int launch_d(const ForwardArgs& a, int rows_per_head, int lcap) {
 // Number of leading rows per head handled directly (causal), or n / 0 (non-causal).
 int head_rows_count(const ForwardArgs& a) {
     if (a.head_rows <= 0) return 0;
-    if (a.causal) return a.n < a.head_rows - 1 ? a.n : a.head_rows - 1;
-    return a.n < a.head_rows ? a.n : 0;
+    if (a.causal) {     // query row i sees n - nq + i + 1 keys
+        const int rows = a.head_rows - 1 - (a.n - a.nq);
+        return rows < 0 ? 0 : (rows > a.nq ? a.nq : rows);
+    }
+    return a.n < a.head_rows ? a.nq : 0;
 }
 
 int launch_head_rows(const ForwardArgs& a) {
     const int rows = head_rows_count(a);
     if (rows <= 0) return LLA_OK;
-    const int lcap = a.causal ? rows : a.n;
+    const int lcap = a.causal ? (a.n - a.nq) + rows : a.n;
     if (a.d != a.dv) return LLA_ERR_UNSUPPORTED;
     switch (a.d) {
         case 16: return launch_d<16>(a, rows, lcap);

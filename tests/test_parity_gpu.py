@@ -341,3 +341,32 @@ def test_forward_d128_with_caller_workspace(oracle):
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     got = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, workspace=ws, workspace_bytes=nbytes)
     assert row_err(got, ref).max() <= TOL_BF16
+
+
+@pytest.mark.parametrize("dtype,d,n,nq", [("bf16", 64, 900, 300), ("bf16", 64, 330, 280), ("bf16", 128, 700, 129),
+                                           ("f32", 16, 400, 130), ("bf16", 64, 1024, 1)])
+def test_chunked_prefill_against_existing_keys(oracle, dtype, d, n, nq):
+    # q_rows < n: the last nq positions are the queries (a chunk appended to a cache of n - nq keys).
+    # Every such row must equal the same row of the full causal forward.
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=n, d=d, dv=d, dtype=dtype, seed=80 + nq)
+    q, k, v = inputs.make_prefill(w)
+    off = n - nq
+    rows = np.concatenate([np.arange(h * n + off, (h + 1) * n) for h in range(w.B * w.H)]).astype(np.int64)
+    ref = oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows).reshape(w.B, w.H, nq, d)
+    dq = dev(np.ascontiguousarray(q[:, :, off:]), dtype)
+    dk, dv_ = dev(k, dtype), dev(v, dtype)
+    out = torch.full((w.B, w.H, nq, d), float("nan"), dtype=torch.float32, device="cuda")
+    iters = torch.zeros((w.B, w.H, nq), dtype=torch.int32, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    L.lla_forward_ex(dq, dk, dv_, out, w.B, w.H, n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                     out_dtype=L.LLA_F32, q_rows=nq, iters=iters, device_status=status, stream=stream_ptr())
+    torch.cuda.synchronize()
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    assert row_err(out.cpu().numpy(), ref).max() <= tol
+    st = status.cpu().numpy()
+    assert st[L.STATUS_ROWS_AT_CAP] == 0 and st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
+    # rows that see fewer keys than the direct-solve threshold are marked -1, the others iterated
+    thr = 2 * d if dtype == "f32" else d + d // 2
+    seen = off + np.arange(nq) + 1
+    it = iters.cpu().numpy()[0, 0]
+    assert ((it == -1) == (seen < thr)).all()
