@@ -1,0 +1,92 @@
+"""Float64 CPU oracle for the gradient of the causal LLA forward pass.
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by the smoke check and by the
+bench's CPU-baseline leg.  The CUDA library never imports this module and this
+module never imports the CUDA package.
+
+What it computes.  The forward pass maps (Q, K, V) to the local-linear
+intercepts o_i (paper Section 2.3, Eq. "query_specific" and Eq. "lla").  For an
+upstream gradient g_i = dL/do_i (the paper's g_i of the backward appendix) the
+backward pass returns dL/dQ, dL/dK, dL/dV.  The gradient has a plain
+definition -- the derivative of the forward map -- so the oracle is that
+definition written out: the forward is evaluated from its defining formulas
+(explicit z_ij = k_j - q_i, explicit moments omega_i, mu_i, Sigma_i, a dense
+solve) in float64 with plain PyTorch CPU ops, and reverse-mode differentiation
+of exactly those ops gives the gradient.  None of the hand-derived expressions
+of the backward appendix (u_i, Delta_mu, relmm terms) is used here, so the
+oracle is independent of them; ``tests/test_backward_oracle_pins.py`` pins it
+against finite differences of the separate C forward oracle, closed forms and
+the appendix's own formulas.
+
+Weights are exp(score - m_i) with the ridge lambda * exp(-m_i): the forward
+value does not depend on the shift m_i (the joint scaling of weights and ridge
+leaves Eq. "lla" unchanged), so m_i is treated as a constant and carries no
+gradient.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+
+def _forward_rows(Q, K, V, rows, scale, lam, causal):
+    """o_i for the given row indices of one head, from the definition (float64 tensors)."""
+    n = K.shape[0]
+    d = K.shape[1]
+    L = int(rows.max()) + 1 if causal else n
+    Kl, Vl = K[:L], V[:L]
+    Qr = Q[rows]
+    s = scale * (Qr @ Kl.T)                                        # scores, Section 3.1
+    if causal:
+        mask = torch.arange(L)[None, :] <= rows[:, None]           # row i sees keys j <= i
+    else:
+        mask = torch.ones(len(rows), L, dtype=torch.bool)
+    m = torch.where(mask, s, torch.full_like(s, -torch.inf)).max(dim=1).values.detach()
+    w = torch.where(mask, torch.exp(s - m[:, None]), torch.zeros_like(s))
+    lam_i = lam * torch.exp(-m)
+    Z = Kl[None, :, :] - Qr[:, None, :]                            # z_ij = k_j - q_i
+    mu = torch.einsum("rj,rjc->rc", w, Z)                          # mu_i
+    Sigma = torch.einsum("rj,rjc,rje->rce", w, Z, Z) + lam_i[:, None, None] * torch.eye(d, dtype=Q.dtype)
+    rho = torch.linalg.solve(Sigma, mu)                            # Sigma_i rho_i = mu_i
+    c = w * (1.0 - torch.einsum("rjc,rc->rj", Z, rho))             # w_ij (1 - z_ij^T rho_i)
+    return (c @ Vl) / c.sum(dim=1, keepdim=True)                   # Eq. "lla"
+
+
+def backward(q, k, v, g, scale, lam, causal=True, chunk=32):
+    """Gradients of sum_i <g_i, o_i> with respect to q, k, v.
+
+    q, k: [B, H, n, d]; v, g: [B, H, n, dv]; numpy arrays (any float dtype; widened to float64).
+    Returns (dq, dk, dv) as float64 numpy arrays of the inputs' shapes.
+    """
+    q, k, v, g = (np.asarray(a, dtype=np.float64) for a in (q, k, v, g))
+    B, H, n, _ = q.shape
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    for b in range(B):
+        for h in range(H):
+            Q = torch.tensor(q[b, h], requires_grad=True)
+            K = torch.tensor(k[b, h], requires_grad=True)
+            V = torch.tensor(v[b, h], requires_grad=True)
+            G = torch.tensor(g[b, h])
+            for r0 in range(0, n, chunk):
+                rows = torch.arange(r0, min(n, r0 + chunk))
+                o = _forward_rows(Q, K, V, rows, float(scale), float(lam), bool(causal))
+                (o * G[rows]).sum().backward()
+            dq[b, h], dk[b, h], dv[b, h] = Q.grad.numpy(), K.grad.numpy(), V.grad.numpy()
+    return dq, dk, dv
+
+
+def forward(q, k, v, scale, lam, causal=True, chunk=32):
+    """The forward values the gradient above differentiates (used by the pins to tie this module's
+    forward to the C oracle's)."""
+    q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
+    B, H, n, _ = q.shape
+    out = np.zeros(v.shape[:2] + (n, v.shape[3]))
+    with torch.no_grad():
+        for b in range(B):
+            for h in range(H):
+                Q, K, V = (torch.tensor(a[b, h]) for a in (q, k, v))
+                for r0 in range(0, n, chunk):
+                    rows = torch.arange(r0, min(n, r0 + chunk))
+                    out[b, h, r0:r0 + len(rows)] = _forward_rows(Q, K, V, rows, float(scale), float(lam),
+                                                                 bool(causal)).numpy()
+    return out

@@ -1,0 +1,129 @@
+"""Pins for the gradient oracle (oracle/lla_backward_oracle.py): everything here is fixed by the paper or
+by mathematics, none of it by the CUDA path.
+
+  (a) central finite differences of the separate C forward oracle (different code, different solver)
+  (b) the forward the gradient differentiates equals the C oracle's forward
+  (c) sum_j s_ij = 1  =>  sum_j dV_j = sum_i g_i;   v -> v + c leaves dQ, dK unchanged
+  (d) lambda -> infinity: the gradient tends to the textbook softmax-attention gradient, error ~ 1/lambda
+  (e) a single token: o_0 = v_0 for every lambda > 0, so dQ = dK = 0 and dV = g
+  (f) the hand-derived formulas of the paper's backward appendix, evaluated literally in numpy
+"""
+import numpy as np
+import pytest
+
+from oracle import lla_backward_oracle as bwd
+from oracle import lla_oracle as fwd_c
+
+
+def _inputs(seed, n, d, dv, B=1, H=1):
+    rng = np.random.default_rng(seed)
+    q = rng.standard_normal((B, H, n, d)) / np.sqrt(d)
+    k = rng.standard_normal((B, H, n, d)) / np.sqrt(d)
+    v = rng.standard_normal((B, H, n, dv))
+    g = rng.standard_normal((B, H, n, dv))
+    return q, k, v, g
+
+
+def test_forward_of_gradient_oracle_equals_c_oracle():
+    q, k, v, _ = _inputs(1, 40, 8, 5)
+    a = bwd.forward(q, k, v, 0.35, 1e-2)
+    b = fwd_c.forward(q, k, v, 0.35, 1e-2)
+    assert np.abs(a - b).max() <= 1e-9 * np.abs(b).max()
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_finite_differences_of_c_forward_oracle(causal):
+    n, d, dv, scale, lam = 7, 3, 2, 0.6, 5e-2
+    q, k, v, g = _inputs(2, n, d, dv)
+    dq, dk, dv_ = bwd.backward(q, k, v, g, scale, lam, causal=causal)
+
+    def loss(q_, k_, v_):
+        return float((fwd_c.forward(q_, k_, v_, scale, lam, causal=causal) * g).sum())
+
+    eps = 1e-5
+    for name, x, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv_)):
+        num = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps
+            xm[idx] -= eps
+            args_p = {"q": q, "k": k, "v": v, name: xp}
+            args_m = {"q": q, "k": k, "v": v, name: xm}
+            num[idx] = (loss(args_p["q"], args_p["k"], args_p["v"]) - loss(args_m["q"], args_m["k"], args_m["v"])) / (2 * eps)
+        assert np.abs(num - grad).max() <= 2e-7 * max(1.0, np.abs(grad).max()), name
+
+
+def test_value_gradient_sums_and_shift_invariance():
+    q, k, v, g = _inputs(3, 48, 6, 4, B=1, H=2)
+    dq, dk, dv = bwd.backward(q, k, v, g, 0.4, 1e-2)
+    assert np.abs(dv.sum(axis=2) - g.sum(axis=2)).max() <= 1e-9
+    dq2, dk2, _ = bwd.backward(q, k, v + 3.0, g, 0.4, 1e-2)
+    assert np.abs(dq2 - dq).max() <= 1e-8 * np.abs(dq).max()
+    assert np.abs(dk2 - dk).max() <= 1e-8 * np.abs(dk).max()
+
+
+def _softmax_attention_grad(q, k, v, g, scale):
+    n = q.shape[0]
+    s = scale * q @ k.T
+    s = np.where(np.tril(np.ones((n, n), bool)), s, -np.inf)
+    p = np.exp(s - s.max(axis=1, keepdims=True))
+    p /= p.sum(axis=1, keepdims=True)
+    o = p @ v
+    ds = p * (g @ v.T - (g * o).sum(axis=1, keepdims=True))
+    return scale * ds @ k, scale * ds.T @ q, p.T @ g
+
+
+def test_large_ridge_limit_is_softmax_attention_gradient():
+    q, k, v, g = _inputs(4, 24, 4, 3)
+    ref = _softmax_attention_grad(q[0, 0], k[0, 0], v[0, 0], g[0, 0], 0.5)
+    errs = []
+    for lam in (1e4, 1e6):
+        got = bwd.backward(q, k, v, g, 0.5, lam)
+        errs.append(max(np.abs(a[0, 0] - b).max() for a, b in zip(got, ref)))
+    assert errs[0] < 1e-2 and errs[1] < 1e-4 and errs[1] < 0.02 * errs[0]
+
+
+def test_single_token():
+    q, k, v, g = _inputs(5, 1, 4, 3)
+    dq, dk, dv = bwd.backward(q, k, v, g, 0.5, 1e-3)
+    assert np.abs(dq).max() <= 1e-12 and np.abs(dk).max() <= 1e-12
+    assert np.abs(dv - g).max() <= 1e-12
+
+
+def _appendix_formulas(q, k, v, g, scale, lam):
+    """Backward appendix, literally: gamma, beta, c, u, Delta_mu, dL/dSigma, dL/dw, dL/dz, then the
+    chain rule to k_j and q_i.  Raw weights exp(scale q.k), ridge lam (no max shift)."""
+    n, d = q.shape
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    for i in range(n):
+        K, V = k[: i + 1], v[: i + 1]
+        Z = K - q[i]
+        w = np.exp(scale * K @ q[i])
+        omega, mu = w.sum(), w @ Z
+        Sigma = (Z * w[:, None]).T @ Z + lam * np.eye(d)
+        rho = np.linalg.solve(Sigma, mu)
+        delta = omega - mu @ rho
+        nij = 1.0 - Z @ rho
+        s = w * nij / delta
+        gamma = V @ g[i]
+        beta = (gamma * s).sum() / delta
+        c = gamma * w / delta
+        u = np.linalg.solve(Sigma, c @ Z)
+        dmu = -u + 2.0 * beta * rho
+        dSigma = -0.5 * np.outer(rho, dmu) + 0.5 * np.outer(u, rho)
+        dw = gamma * nij / delta - beta + Z @ dmu + np.einsum("jc,ce,je->j", Z, dSigma, Z)
+        dz = -np.outer(c, rho) + np.outer(w, dmu) + 2.0 * w[:, None] * (Z @ dSigma.T)
+        dv[: i + 1] += np.outer(s, g[i])
+        dk[: i + 1] += (dw * w * scale)[:, None] * q[i] + dz
+        dq[i] += (dw * w * scale) @ K - dz.sum(axis=0)
+    return dq, dk, dv
+
+
+def test_backward_appendix_formulas():
+    q, k, v, g = _inputs(6, 20, 5, 4)
+    got = bwd.backward(q, k, v, g, 0.45, 2e-2)
+    ref = _appendix_formulas(q[0, 0], k[0, 0], v[0, 0], g[0, 0], 0.45, 2e-2)
+    for a, b in zip(got, ref):
+        assert np.abs(a[0, 0] - b).max() <= 1e-9 * max(1.0, np.abs(b).max())
