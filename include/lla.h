@@ -263,6 +263,50 @@ size_t lla_decode_workspace_bytes(int B, int H, int Lmax, int d, int dv, int in_
 /* Number of key-range parts lla_decode / lla_decode_ex(splits = 0) would use. */
 int lla_decode_default_splits(int B, int H, int Lmax);
 
+/*
+ * Backward pass (the paper's backward appendix): gradients of a scalar loss L with respect to Q, K and
+ * V, given g_i = dL/do_i and the tensors the forward saved (Section 3.2 keeps R and delta next to the
+ * output for this purpose).  Causal, ridge as in the definition (LLA_RIDGE_DEFINITION), one scalar lambda,
+ * q_rows = n.  Supported: bf16 q, k, v with d = dv in {64, 128}; anything else is LLA_ERR_UNSUPPORTED.
+ *
+ * Per query row the appendix's quantities are gamma_ij = g_i . v_j, one further linear solve with the
+ * row's Sigma_i (its u_i; the forward's conjugate-gradient kernel is run on it, rows that see fewer than
+ * head_rows keys are solved directly in fp64 like in the forward), and then
+ *     Delta_V = S^T G,  Delta_K = Delta_W^K + Delta_Z^K,  Delta_Q = Delta_W^Q + Delta_Z^Q.
+ *
+ *   q, k, v   : [B, H, n, d] bf16 on the device, as given to the forward
+ *   out       : [B, H, n, d] the forward's output, out_dtype (LLA_BF16 or LLA_F32).  Only g_i . o_i is
+ *               taken from it; a bf16 `out` limits the accuracy of dq and dk to its rounding
+ *   dout      : [B, H, n, d] g, dout_dtype (LLA_BF16 or LLA_F32)
+ *   rho, stats: [B, H, n, d] and [B, H, n, 3] fp32, written by lla_forward_ex for the same inputs,
+ *               scale, lambda and head_rows
+ *   dq, dk, dv: [B, H, n, d] fp32 on the device, overwritten
+ *   max_iters, tol, head_rows : as in lla_forward_params (0 = defaults)
+ *   device_status : optional int[LLA_STATUS_WORDS], zeroed by the call
+ *   workspace / workspace_bytes : device scratch of at least lla_backward_workspace_bytes(B, H, n, d)
+ *               bytes, 256-byte aligned (required; LLA_ERR_WORKSPACE otherwise)
+ * All pointers 16-byte aligned; no output may alias an input.  Work is enqueued on `stream`; the call
+ * does not synchronise and keeps no pointer.
+ */
+typedef struct lla_backward_params {
+    const void *q, *k, *v, *out, *dout;
+    const float *rho, *stats;
+    float *dq, *dk, *dv;
+    int B, H, n, d;
+    int out_dtype, dout_dtype;
+    float scale, lambda;
+    int max_iters;
+    float tol;
+    int head_rows;
+    int *device_status;
+    void *workspace;
+    size_t workspace_bytes;
+    void *stream;
+} lla_backward_params;
+
+int lla_backward_ex(const lla_backward_params *p);
+size_t lla_backward_workspace_bytes(int B, int H, int n, int d);
+
 /* Static, NUL-terminated description of a status code. */
 const char *lla_status_string(int status);
 

@@ -24,8 +24,22 @@ LLA_RIDGE_DEFINITION, LLA_RIDGE_PRINTED = 0, 1
 EXPORTS = (
     "lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex", "lla_decode_ex",
     "lla_forward_host", "lla_decode_host", "lla_decode_noalloc", "lla_forward_workspace_bytes", "lla_decode_workspace_bytes",
-    "lla_decode_default_splits", "lla_status_string", "lla_version",
+    "lla_decode_default_splits", "lla_status_string", "lla_version", "lla_backward_ex", "lla_backward_workspace_bytes",
 )
+
+
+class BackwardParams(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
+        ("dout", ctypes.c_void_p), ("rho", ctypes.c_void_p), ("stats", ctypes.c_void_p),
+        ("dq", ctypes.c_void_p), ("dk", ctypes.c_void_p), ("dv", ctypes.c_void_p),
+        ("B", ctypes.c_int), ("H", ctypes.c_int), ("n", ctypes.c_int), ("d", ctypes.c_int),
+        ("out_dtype", ctypes.c_int), ("dout_dtype", ctypes.c_int),
+        ("scale", ctypes.c_float), ("lambda_", ctypes.c_float),
+        ("max_iters", ctypes.c_int), ("tol", ctypes.c_float), ("head_rows", ctypes.c_int),
+        ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("stream", ctypes.c_void_p),
+    ]
 
 
 class LlaError(RuntimeError):
@@ -84,6 +98,10 @@ def load():
     lib.lla_decode_noalloc.restype = i
     lib.lla_forward_ex.argtypes = [ctypes.POINTER(ForwardParams)]
     lib.lla_decode_ex.argtypes = [ctypes.POINTER(DecodeParams)]
+    lib.lla_backward_ex.argtypes = [ctypes.POINTER(BackwardParams)]
+    lib.lla_backward_ex.restype = i
+    lib.lla_backward_workspace_bytes.argtypes = [i, i, i, i]
+    lib.lla_backward_workspace_bytes.restype = sz
     for name in ("lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex",
                  "lla_decode_ex", "lla_forward_host", "lla_decode_host", "lla_decode_noalloc", "lla_version",
                  "lla_decode_default_splits"):
@@ -179,6 +197,24 @@ def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, i
     p.device_status, p.workspace, p.workspace_bytes, p.stream = _p(device_status), _p(workspace), workspace_bytes, _p(stream)
     p.lambda_units, p.ridge_mode = _p(lambda_units), ridge_mode
     _check(load().lla_decode_ex(ctypes.byref(p)), "lla_decode_ex")
+
+
+def lla_backward_ex(q, k, v, out, dout, rho, stats, dq, dk, dv, B, H, n, d, scale, lam, out_dtype=LLA_F32,
+                    dout_dtype=LLA_F32, max_iters=0, tol=0.0, head_rows=0, device_status=None, workspace=None,
+                    workspace_bytes=0, stream=0):
+    p = BackwardParams()
+    p.q, p.k, p.v, p.out, p.dout = _p(q), _p(k), _p(v), _p(out), _p(dout)
+    p.rho, p.stats, p.dq, p.dk, p.dv = _p(rho), _p(stats), _p(dq), _p(dk), _p(dv)
+    p.B, p.H, p.n, p.d = B, H, n, d
+    p.out_dtype, p.dout_dtype = out_dtype, dout_dtype
+    p.scale, p.lambda_ = scale, lam
+    p.max_iters, p.tol, p.head_rows = max_iters, tol, head_rows
+    p.device_status, p.workspace, p.workspace_bytes, p.stream = _p(device_status), _p(workspace), workspace_bytes, _p(stream)
+    _check(load().lla_backward_ex(ctypes.byref(p)), "lla_backward_ex")
+
+
+def lla_backward_workspace_bytes(B, H, n, d) -> int:
+    return int(load().lla_backward_workspace_bytes(B, H, n, d))
 
 
 NOALLOC_SCRATCH_BYTES = 64 << 20

@@ -9,6 +9,7 @@ namespace {
 
 using lla::DecodeArgs;
 using lla::ForwardArgs;
+using lla::BackwardArgs;
 
 // Side stream on which the directly-solved rows run next to the iterative kernel (fork/join with
 // events, so the caller's stream semantics are unchanged).  One per device, created on first use.
@@ -266,6 +267,46 @@ int lla_decode_f32(const void* q, const void* kcache, const void* vcache, const 
     p.scale = scale; p.lambda = lambda;
     p.stream = stream;
     return lla_decode_ex(&p);
+}
+
+int lla_backward_ex(const lla_backward_params* p) {
+    if (!p) return LLA_ERR_INVALID_ARG;
+    if (!p->q || !p->k || !p->v || !p->out || !p->dout || !p->rho || !p->stats || !p->dq || !p->dk || !p->dv)
+        return LLA_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->n < 1 || p->d < 1) return LLA_ERR_INVALID_ARG;
+    if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
+    const uintptr_t align = (uintptr_t)p->q | (uintptr_t)p->k | (uintptr_t)p->v | (uintptr_t)p->out | (uintptr_t)p->dout |
+                            (uintptr_t)p->rho | (uintptr_t)p->dq | (uintptr_t)p->dk | (uintptr_t)p->dv;
+    if (align & 15u) return LLA_ERR_INVALID_ARG;
+    if (p->d != 64 && p->d != 128) return LLA_ERR_UNSUPPORTED;
+    if ((long long)p->B * p->H > 65535) return LLA_ERR_UNSUPPORTED;
+    auto dt_ok = [](int t) { return t == LLA_BF16 || t == LLA_F32; };
+    if (!dt_ok(p->out_dtype) || !dt_ok(p->dout_dtype)) return LLA_ERR_UNSUPPORTED;
+    if (!p->workspace || ((uintptr_t)p->workspace & 255u) ||
+        p->workspace_bytes < lla::backward_workspace_bytes(p->B, p->H, p->n, p->d))
+        return LLA_ERR_WORKSPACE;
+    BackwardArgs a = {};
+    a.q = p->q; a.k = p->k; a.v = p->v; a.out = p->out; a.dout = p->dout;
+    a.rho = p->rho; a.stats = p->stats; a.dq = p->dq; a.dk = p->dk; a.dv = p->dv;
+    a.B = p->B; a.H = p->H; a.n = p->n; a.d = p->d;
+    a.out_dtype = p->out_dtype; a.dout_dtype = p->dout_dtype;
+    a.scale = p->scale; a.lambda = p->lambda;
+    a.max_iters = p->max_iters > 0 ? p->max_iters : 64;
+    a.tol = p->tol > 0.f ? p->tol : 1e-4f;
+    a.head_rows = p->head_rows == 0 ? p->d + p->d / 2 : (p->head_rows < 0 ? 0 : p->head_rows);
+    a.status = p->device_status;
+    a.workspace = p->workspace; a.workspace_bytes = p->workspace_bytes;
+    a.stream = (cudaStream_t)p->stream;
+    ForwardArgs probe = {};
+    probe.in_dtype = LLA_BF16; probe.d = p->d; probe.dv = p->d;
+    if (!lla::forward_tensor_supported(probe)) return LLA_ERR_UNSUPPORTED;
+    if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
+    return lla::launch_backward(a);
+}
+
+size_t lla_backward_workspace_bytes(int B, int H, int n, int d) {
+    if (B < 1 || H < 1 || n < 1 || d < 1) return 0;
+    return lla::backward_workspace_bytes(B, H, n, d);
 }
 
 size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl) {

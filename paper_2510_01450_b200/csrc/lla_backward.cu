@@ -1,0 +1,586 @@
+// Backward pass of causal local linear attention (the paper's backward appendix), bf16 inputs, d = dv in
+// {64, 128}, fp32 gradients.
+//
+// The gradient is taken in the weighted-mean-centred form the forward kernels use.  Per query row i with
+// visible keys j <= i, p_j = w_ij / omega_i, kbar = sum_j p_j k_j, xi_j = k_j - kbar,
+// C = sum_j p_j xi_j xi_j^T + (lambda e^{-m_i} / omega_i) I, mbar = kbar - q_i, the forward computes
+//     y = C^{-1} mbar,  e_j = xi_j . y,  a_j = p_j (1 - e_j)  (the paper's s_ij),  o_i = sum_j a_j v_j.
+// With g = dL/do_i and gamma_j = g . v_j (the appendix's gamma_ij), gbar = sum_j p_j gamma_j and
+//     h = sum_j p_j gamma_j xi_j,   t = C^{-1} h   (the one extra solve; the appendix's u_i in this frame),
+//     f_j = xi_j . t,   kappa = g . o_i + t . mbar,
+// the chain rule through p (a softmax of the scores), k_j and q_i gives
+//     dL/ds_ij = p_j [gamma_j (1 - e_j) + (gbar + f_j) e_j - f_j - kappa]
+//     dV_j += a_j g
+//     dK_j += scale dL/ds_ij q_i + p_j [(f_j - gamma_j + gbar) y + (e_j - 1) t]
+//     dQ_i  = scale sum_j dL/ds_ij k_j + t.
+// In exact arithmetic this is the appendix's Delta_Q, Delta_K, Delta_V (same function, same derivative);
+// y follows from the saved rho and delta as y = rho omega / delta.
+//
+// Kernels, in launch order:
+//   bwd_moments_kernel    per 64- or 32-row query tile: kbar_i, gbar_i, h_i          (CUDA cores, fp32)
+//   forward_tc_kernel     in solve mode: C_i t_i = h_i by conjugate gradients        (tensor cores)
+//   bwd_rowprep_kernel    y_i, the per-row scalars, dQ_i = t_i
+//   bwd_pairs_kernel      per 64-key tile over all later query tiles: dK, dV (registers), dQ (atomics)
+//   bwd_head_rows_kernel  rows with fewer than head_rows keys: everything in fp64 with a direct solve
+#include "lla_common.cuh"
+
+namespace lla {
+namespace {
+
+constexpr int BW_THREADS = 256;
+constexpr int BW_BJ = 64;      // keys per tile
+constexpr int BW_LDP = 68;     // row stride of the [query][key] pair matrices (floats)
+constexpr int BW_ROWSC = 8;    // floats per row of the scalar record: m, 1/omega, gbar, kappa, kbar.y, kbar.t
+
+template <int D>
+struct BwCfg {
+    static constexpr int BI = D <= 64 ? 64 : 32;   // query rows per tile
+    static constexpr int LD = D + 4;               // row stride of the operand tiles (floats)
+    static constexpr int RI = BI / 16;             // query rows per thread
+    static constexpr int CU = D / 64;              // float4 column groups per thread
+    static constexpr int LDT = BI + 4;             // row stride of the [key][query] matrices
+    static constexpr size_t MOMENTS_SMEM = sizeof(float) * ((size_t)(2 * BI + 2 * BW_BJ) * LD + 2 * BW_BJ * LDT + BI);
+    static constexpr size_t PAIRS_SMEM = sizeof(float) * ((size_t)(4 * BI + 2 * BW_BJ) * LD + 3 * BI * BW_LDP + BW_BJ * LDT);
+};
+
+// rows [row0, row0 + rows) of a row-major [.., D] array -> fp32 shared tile [rows][D + 4]; rows outside
+// [lo, nvalid) are zero (never read: their memory may be uninitialised)
+template <int D>
+__device__ __forceinline__ void load_tile(float* dst, const void* src, int dtype, size_t row0, int rows, int nvalid, int lo = 0) {
+    constexpr int LD = D + 4;
+    for (int idx = threadIdx.x; idx < rows * (D / 4); idx += BW_THREADS) {
+        const int r = idx / (D / 4), c = (idx % (D / 4)) * 4;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < nvalid && r >= lo) {
+            if (dtype == LLA_F32) x = load4(static_cast<const float*>(src) + (row0 + r) * D + c);
+            else x = load4(static_cast<const __nv_bfloat16*>(src) + (row0 + r) * D + c);
+        }
+        *reinterpret_cast<float4*>(dst + r * LD + c) = x;
+    }
+}
+
+__device__ __forceinline__ float ld_any(const void* p, int dtype, size_t i) {
+    return dtype == LLA_F32 ? static_cast<const float*>(p)[i] : __bfloat162float(static_cast<const __nv_bfloat16*>(p)[i]);
+}
+
+// acc[r][4u + x] += sum_l M[l][a0 + r] * X[l][4 tc + 64 u + x]   for l < len
+template <int NR, int CU>
+__device__ __forceinline__ void mac_tile(float (&acc)[NR][4 * CU], const float* M, int ldm, int a0, const float* X, int ldx,
+                                         int tc, int len, float sign = 1.f) {
+#pragma unroll 4
+    for (int l = 0; l < len; ++l) {
+        float mv[NR];
+#pragma unroll
+        for (int r = 0; r < NR; ++r) mv[r] = sign * M[l * ldm + a0 + r];
+#pragma unroll
+        for (int u = 0; u < CU; ++u) {
+            const float4 x = *reinterpret_cast<const float4*>(X + l * ldx + 4 * tc + 64 * u);
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+                acc[r][4 * u + 0] = fmaf(mv[r], x.x, acc[r][4 * u + 0]);
+                acc[r][4 * u + 1] = fmaf(mv[r], x.y, acc[r][4 * u + 1]);
+                acc[r][4 * u + 2] = fmaf(mv[r], x.z, acc[r][4 * u + 2]);
+                acc[r][4 * u + 3] = fmaf(mv[r], x.w, acc[r][4 * u + 3]);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// kbar_i = sum_j p_ij k_j,  gbar_i = sum_j p_ij gamma_ij,  h_i = sum_j p_ij gamma_ij k_j - gbar_i kbar_i
+// ------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(BW_THREADS)
+bwd_moments_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                   const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
+                   const float* __restrict__ stats, float* __restrict__ kbar, float* __restrict__ hvec,
+                   float* __restrict__ rowsc, int n, int first, float scale) {
+    using C = BwCfg<D>;
+    constexpr int BI = C::BI, LD = C::LD, RI = C::RI, CU = C::CU, LDT = C::LDT;
+    extern __shared__ __align__(16) float bw_smem[];
+    float* Qs = bw_smem;
+    float* Gs = Qs + BI * LD;
+    float* Ks = Gs + BI * LD;
+    float* Vs = Ks + BW_BJ * LD;
+    float* Pt = Vs + BW_BJ * LD;          // [key][query]
+    float* PGt = Pt + BW_BJ * LDT;
+    float* gbs = PGt + BW_BJ * LDT;       // [BI]
+    const int tid = threadIdx.x, ti = tid >> 4, tj = tid & 15;
+    const int tile = gridDim.x - 1 - blockIdx.x;      // longest tiles first
+    const int bh = blockIdx.y;
+    const int i0 = tile * BI;
+    if (i0 + BI <= first) return;                      // every row of the tile is solved directly
+    const size_t base = (size_t)bh * n;
+    const int nrow = min(BI, n - i0);
+    load_tile<D>(Qs, q, LLA_BF16, base + i0, BI, nrow);
+    load_tile<D>(Gs, dout, dout_dtype, base + i0, BI, nrow);
+    float mrow[RI], iom[RI], gb[RI];
+#pragma unroll
+    for (int r = 0; r < RI; ++r) {
+        const int gi = i0 + ti + 16 * r;
+        const bool okr = gi < n && gi >= first;
+        mrow[r] = okr ? stats[(base + gi) * 3 + 0] : 0.f;
+        iom[r] = okr ? 1.f / stats[(base + gi) * 3 + 1] : 0.f;
+        gb[r] = 0.f;
+    }
+    float akb[RI][4 * CU] = {}, ah[RI][4 * CU] = {};
+    const int jt_end = (min(n, i0 + BI) + BW_BJ - 1) / BW_BJ;
+    for (int jt = 0; jt < jt_end; ++jt) {
+        const int j0 = jt * BW_BJ;
+        __syncthreads();
+        load_tile<D>(Ks, k, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
+        load_tile<D>(Vs, v, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
+        __syncthreads();
+        float s[RI][4] = {}, gm[RI][4] = {};
+#pragma unroll 2
+        for (int c = 0; c < D; c += 4) {
+            float4 qv[RI], gv[RI];
+#pragma unroll
+            for (int r = 0; r < RI; ++r) {
+                qv[r] = *reinterpret_cast<const float4*>(Qs + (ti + 16 * r) * LD + c);
+                gv[r] = *reinterpret_cast<const float4*>(Gs + (ti + 16 * r) * LD + c);
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const float4 kv = *reinterpret_cast<const float4*>(Ks + (tj + 16 * x) * LD + c);
+                const float4 vv = *reinterpret_cast<const float4*>(Vs + (tj + 16 * x) * LD + c);
+#pragma unroll
+                for (int r = 0; r < RI; ++r) {
+                    s[r][x] = fmaf(qv[r].x, kv.x, fmaf(qv[r].y, kv.y, fmaf(qv[r].z, kv.z, fmaf(qv[r].w, kv.w, s[r][x]))));
+                    gm[r][x] = fmaf(gv[r].x, vv.x, fmaf(gv[r].y, vv.y, fmaf(gv[r].z, vv.z, fmaf(gv[r].w, vv.w, gm[r][x]))));
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < RI; ++r) {
+            const int il = ti + 16 * r, gi = i0 + il;
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int jl = tj + 16 * x, gj = j0 + jl;
+                const float p = (gj <= gi && iom[r] > 0.f) ? __expf(fmaf(scale, s[r][x], -mrow[r])) * iom[r] : 0.f;
+                const float pg = p * gm[r][x];
+                Pt[jl * LDT + il] = p;
+                PGt[jl * LDT + il] = pg;
+                gb[r] += pg;
+            }
+        }
+        __syncthreads();
+        mac_tile<RI, CU>(akb, Pt, LDT, RI * ti, Ks, LD, tj, BW_BJ);
+        mac_tile<RI, CU>(ah, PGt, LDT, RI * ti, Ks, LD, tj, BW_BJ);
+    }
+#pragma unroll
+    for (int r = 0; r < RI; ++r) {
+#pragma unroll
+        for (int o = 8; o >= 1; o >>= 1) gb[r] += __shfl_xor_sync(0xffffffffu, gb[r], o);
+        if (tj == 0) gbs[ti + 16 * r] = gb[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < RI; ++r) {
+        const int il = RI * ti + r, gi = i0 + il;
+        if (gi >= n || gi < first) continue;
+        const float gbar = gbs[il];
+        if (tj == 0) rowsc[(base + gi) * BW_ROWSC + 2] = gbar;
+#pragma unroll
+        for (int u = 0; u < CU; ++u) {
+            const int c = 4 * tj + 64 * u;
+            float4 kb4 = make_float4(akb[r][4 * u], akb[r][4 * u + 1], akb[r][4 * u + 2], akb[r][4 * u + 3]);
+            float4 h4 = make_float4(ah[r][4 * u] - gbar * kb4.x, ah[r][4 * u + 1] - gbar * kb4.y,
+                                    ah[r][4 * u + 2] - gbar * kb4.z, ah[r][4 * u + 3] - gbar * kb4.w);
+            *reinterpret_cast<float4*>(kbar + (base + gi) * D + c) = kb4;
+            *reinterpret_cast<float4*>(hvec + (base + gi) * D + c) = h4;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Per iterative row: y = rho omega / delta, the scalars the pair kernel needs, and dQ_i = t_i (the pair
+// kernel adds the rest with atomics).  One warp per row.
+// ------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(BW_THREADS)
+bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__ out, int out_dtype,
+                   const void* __restrict__ dout, int dout_dtype, const float* __restrict__ rho,
+                   const float* __restrict__ stats, const float* __restrict__ kbar, const float* __restrict__ tvec,
+                   float* __restrict__ yvec, float* __restrict__ rowsc, float* __restrict__ dq, int n, int first,
+                   long long rows) {
+    const long long row = (long long)blockIdx.x * (BW_THREADS / 32) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const int i = (int)(row % n);
+    if (i < first) return;
+    const float m = stats[row * 3 + 0], omega = stats[row * 3 + 1], delta = stats[row * 3 + 2];
+    const float fac = omega / delta;
+    float ky = 0.f, kt = 0.f, qt = 0.f, go = 0.f;
+#pragma unroll
+    for (int c = lane; c < D; c += 32) {
+        const size_t e = (size_t)row * D + c;
+        const float yv = rho[e] * fac, tv = tvec[e], kb = kbar[e];
+        yvec[e] = yv;
+        dq[e] = tv;
+        ky = fmaf(kb, yv, ky);
+        kt = fmaf(kb, tv, kt);
+        qt = fmaf(__bfloat162float(q[e]), tv, qt);
+        go = fmaf(ld_any(dout, dout_dtype, e), ld_any(out, out_dtype, e), go);
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        ky += __shfl_xor_sync(0xffffffffu, ky, o);
+        kt += __shfl_xor_sync(0xffffffffu, kt, o);
+        qt += __shfl_xor_sync(0xffffffffu, qt, o);
+        go += __shfl_xor_sync(0xffffffffu, go, o);
+    }
+    if (lane == 0) {
+        float* rs = rowsc + row * BW_ROWSC;
+        rs[0] = m;
+        rs[1] = 1.f / omega;
+        rs[3] = go + kt - qt;      // kappa = g.o + t.(kbar - q)
+        rs[4] = ky;
+        rs[5] = kt;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// One block per 64-key tile: dK and dV of its keys accumulate in registers over every query tile that
+// sees them; each query tile's dQ contribution goes out with atomic adds.
+// ------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(BW_THREADS)
+bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                 const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
+                 const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ rowsc,
+                 float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale) {
+    using C = BwCfg<D>;
+    constexpr int BI = C::BI, LD = C::LD, RI = C::RI, CU = C::CU, LDT = C::LDT, LDP = BW_LDP;
+    extern __shared__ __align__(16) float bw_smem[];
+    float* Ks = bw_smem;
+    float* Vs = Ks + BW_BJ * LD;
+    float* Qs = Vs + BW_BJ * LD;
+    float* Ys = Qs + BI * LD;
+    float* Ts = Ys + BI * LD;
+    float* Gs = Ts + BI * LD;
+    float* Am = Gs + BI * LD;             // [query][key]: a_ij
+    float* DSm = Am + BI * LDP;           //               scale dL/ds_ij
+    float* P1m = DSm + BI * LDP;          //               p_ij (f_ij - gamma_ij + gbar_i)
+    float* DSt = P1m + BI * LDP;          // [key][query]: scale dL/ds_ij
+    const int tid = threadIdx.x, ti = tid >> 4, tj = tid & 15;
+    const int bh = blockIdx.y;
+    const int j0 = blockIdx.x * BW_BJ;    // key tile 0 sees the most query tiles and starts first
+    const size_t base = (size_t)bh * n;
+    load_tile<D>(Ks, k, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
+    load_tile<D>(Vs, v, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
+    float adk[4][4 * CU] = {}, adv[4][4 * CU] = {};
+    const int it0 = max(j0, first) / BI, it1 = (n + BI - 1) / BI;
+    for (int it = it0; it < it1; ++it) {
+        const int i0 = it * BI;
+        const int nrow = min(BI, n - i0);
+        __syncthreads();
+        load_tile<D>(Qs, q, LLA_BF16, base + i0, BI, nrow);
+        load_tile<D>(Ys, yvec, LLA_F32, base + i0, BI, nrow, first - i0);
+        load_tile<D>(Ts, tvec, LLA_F32, base + i0, BI, nrow, first - i0);
+        load_tile<D>(Gs, dout, dout_dtype, base + i0, BI, nrow);
+        __syncthreads();
+        float s[RI][4] = {}, e[RI][4] = {}, f[RI][4] = {}, gm[RI][4] = {};
+#pragma unroll 1
+        for (int c = 0; c < D; c += 4) {
+            float4 kv[4], vv[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                kv[x] = *reinterpret_cast<const float4*>(Ks + (tj + 16 * x) * LD + c);
+                vv[x] = *reinterpret_cast<const float4*>(Vs + (tj + 16 * x) * LD + c);
+            }
+#pragma unroll
+            for (int r = 0; r < RI; ++r) {
+                const float4 qv = *reinterpret_cast<const float4*>(Qs + (ti + 16 * r) * LD + c);
+                const float4 yv = *reinterpret_cast<const float4*>(Ys + (ti + 16 * r) * LD + c);
+                const float4 tv = *reinterpret_cast<const float4*>(Ts + (ti + 16 * r) * LD + c);
+                const float4 gv = *reinterpret_cast<const float4*>(Gs + (ti + 16 * r) * LD + c);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    s[r][x] = fmaf(qv.x, kv[x].x, fmaf(qv.y, kv[x].y, fmaf(qv.z, kv[x].z, fmaf(qv.w, kv[x].w, s[r][x]))));
+                    e[r][x] = fmaf(yv.x, kv[x].x, fmaf(yv.y, kv[x].y, fmaf(yv.z, kv[x].z, fmaf(yv.w, kv[x].w, e[r][x]))));
+                    f[r][x] = fmaf(tv.x, kv[x].x, fmaf(tv.y, kv[x].y, fmaf(tv.z, kv[x].z, fmaf(tv.w, kv[x].w, f[r][x]))));
+                    gm[r][x] = fmaf(gv.x, vv[x].x, fmaf(gv.y, vv[x].y, fmaf(gv.z, vv[x].z, fmaf(gv.w, vv[x].w, gm[r][x]))));
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < RI; ++r) {
+            const int il = ti + 16 * r, gi = i0 + il;
+            const bool okr = gi < n && gi >= first;
+            const float* rs = rowsc + (base + gi) * BW_ROWSC;
+            const float m = okr ? rs[0] : 0.f, iom = okr ? rs[1] : 0.f, gbar = okr ? rs[2] : 0.f;
+            const float kappa = okr ? rs[3] : 0.f, ky = okr ? rs[4] : 0.f, kt = okr ? rs[5] : 0.f;
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int jl = tj + 16 * x, gj = j0 + jl;
+                const float p = (okr && gj <= gi) ? __expf(fmaf(scale, s[r][x], -m)) * iom : 0.f;
+                const float ev = e[r][x] - ky, fv = f[r][x] - kt, gam = gm[r][x];
+                const float a = p * (1.f - ev);
+                const float ds = scale * p * (gam * (1.f - ev) + (gbar + fv) * ev - fv - kappa);
+                Am[il * LDP + jl] = a;
+                DSm[il * LDP + jl] = ds;
+                P1m[il * LDP + jl] = p * (fv - gam + gbar);
+                DSt[jl * LDT + il] = ds;
+            }
+        }
+        __syncthreads();
+        // dV += A^T G;  dK += DS^T Q + P1^T Y - A^T T      (rows = this thread's four keys)
+        mac_tile<4, CU>(adv, Am, LDP, 4 * ti, Gs, LD, tj, nrow);
+        mac_tile<4, CU>(adk, DSm, LDP, 4 * ti, Qs, LD, tj, nrow);
+        mac_tile<4, CU>(adk, P1m, LDP, 4 * ti, Ys, LD, tj, nrow);
+        mac_tile<4, CU>(adk, Am, LDP, 4 * ti, Ts, LD, tj, nrow, -1.f);
+        // dQ += DS K                                        (rows = RI query rows)
+        float adq[RI][4 * CU] = {};
+        mac_tile<RI, CU>(adq, DSt, LDT, RI * ti, Ks, LD, tj, BW_BJ);
+#pragma unroll
+        for (int r = 0; r < RI; ++r) {
+            const int gi = i0 + RI * ti + r;
+            if (gi >= n || gi < first) continue;
+#pragma unroll
+            for (int u = 0; u < CU; ++u)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) atomicAdd(dq + (base + gi) * D + 4 * tj + 64 * u + x, adq[r][4 * u + x]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int gj = j0 + 4 * ti + r;
+        if (gj >= n) continue;
+#pragma unroll
+        for (int u = 0; u < CU; ++u) {
+            const int c = 4 * tj + 64 * u;
+            *reinterpret_cast<float4*>(dk + (base + gj) * D + c) =
+                make_float4(adk[r][4 * u], adk[r][4 * u + 1], adk[r][4 * u + 2], adk[r][4 * u + 3]);
+            *reinterpret_cast<float4*>(dv + (base + gj) * D + c) =
+                make_float4(adv[r][4 * u], adv[r][4 * u + 1], adv[r][4 * u + 2], adv[r][4 * u + 3]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rows that see fewer than head_rows keys: C is ill-conditioned (rank-deficient up to the ridge), so the
+// whole row -- both solves and every pair term -- runs in fp64 with an explicit C and a direct LDL^T
+// solve, the same split the forward makes.  One block per row; dK and dV go out with atomic adds.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+template <int D>
+__global__ void __launch_bounds__(BW_THREADS)
+bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                     const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
+                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int lcap,
+                     double scale, double lambda, int* __restrict__ status) {
+    constexpr int LDS = D + 1;
+    extern __shared__ __align__(16) double hb_smem[];
+    double* S = hb_smem;                  // D x (D + 1)
+    double* rhs = S + D * LDS;            // [2][D]: mbar -> y, h -> t
+    double* kb = rhs + 2 * D;
+    double* mb = kb + D;
+    double* qd = mb + D;
+    double* gd = qd + D;
+    double* hp = gd + D;                  // sum_j p_j gamma_j k_j
+    double* pj = hp + D;                  // [lcap] each
+    double* gam = pj + lcap;
+    double* ee = gam + lcap;
+    double* ff = ee + lcap;
+    __nv_bfloat16* Kr = reinterpret_cast<__nv_bfloat16*>(ff + lcap);   // [lcap][D]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.x;
+    const int i = gridDim.y - 1 - blockIdx.y;       // rows with the most keys first
+    const int L = i + 1;
+    const size_t base = (size_t)bh * n;
+    for (int c = tid; c < D; c += BW_THREADS) {
+        qd[c] = (double)__bfloat162float(q[(base + i) * D + c]);
+        gd[c] = (double)ld_any(dout, dout_dtype, (base + i) * D + c);
+    }
+    for (int idx = tid; idx < L * (D / 8); idx += BW_THREADS)
+        reinterpret_cast<uint4*>(Kr)[idx] = reinterpret_cast<const uint4*>(k + base * D)[idx];
+    __syncthreads();
+    // scores and gamma_j = g . v_j: a warp per key
+    for (int j = warp; j < L; j += BW_THREADS / 32) {
+        double s = 0.0, gv = 0.0;
+        for (int c = lane; c < D; c += 32) {
+            s += qd[c] * (double)__bfloat162float(Kr[j * D + c]);
+            gv += gd[c] * (double)__bfloat162float(v[(base + j) * D + c]);
+        }
+        s = warp_sum(s);
+        gv = warp_sum(gv);
+        if (lane == 0) { pj[j] = scale * s; gam[j] = gv; }
+    }
+    __syncthreads();
+    double m = -1e300;
+    for (int j = 0; j < L; ++j) m = fmax(m, pj[j]);
+    __syncthreads();
+    for (int j = tid; j < L; j += BW_THREADS) pj[j] = exp(pj[j] - m);
+    __syncthreads();
+    double omega = 0.0;
+    for (int j = 0; j < L; ++j) omega += pj[j];
+    const double eps = lambda * exp(-m) / omega;
+    __syncthreads();
+    for (int j = tid; j < L; j += BW_THREADS) pj[j] /= omega;
+    __syncthreads();
+    double gbar = 0.0;
+    for (int j = 0; j < L; ++j) gbar += pj[j] * gam[j];
+    for (int c = tid; c < 2 * D; c += BW_THREADS) {
+        const int cc = c % D;
+        double acc = 0.0;
+        if (c < D) for (int j = 0; j < L; ++j) acc += pj[j] * (double)__bfloat162float(Kr[j * D + cc]);
+        else for (int j = 0; j < L; ++j) acc += pj[j] * gam[j] * (double)__bfloat162float(Kr[j * D + cc]);
+        (c < D ? kb : hp)[cc] = acc;
+    }
+    __syncthreads();
+    for (int c = tid; c < D; c += BW_THREADS) {
+        mb[c] = kb[c] - qd[c];
+        rhs[c] = mb[c];
+        rhs[D + c] = hp[c] - gbar * kb[c];
+    }
+    // C (lower triangle) in 4 x 4 blocks
+    for (int blk = tid; blk < (D / 4) * (D / 4); blk += BW_THREADS) {
+        const int a0 = (blk / (D / 4)) * 4, b0 = (blk % (D / 4)) * 4;
+        if (b0 > a0) continue;
+        double acc[4][4] = {};
+        for (int j = 0; j < L; ++j) {
+            double ka[4], kc[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                ka[x] = (double)__bfloat162float(Kr[j * D + a0 + x]);
+                kc[x] = (double)__bfloat162float(Kr[j * D + b0 + x]);
+            }
+            const double p = pj[j];
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] += p * ka[x] * kc[y];
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+                const int a = a0 + x, b = b0 + y;
+                if (b <= a) S[a * LDS + b] = acc[x][y] - kb[a] * kb[b] + (a == b ? eps : 0.0);
+            }
+    }
+    const bool okf = block_ldlt_solve<D>(S, LDS, rhs, D LDLT_NOARG, 2, D);
+    if (!okf && tid == 0 && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
+    const double* y = rhs;
+    const double* t = rhs + D;
+    // e_j = xi_j . y, f_j = xi_j . t
+    for (int j = warp; j < L; j += BW_THREADS / 32) {
+        double e = 0.0, f = 0.0;
+        for (int c = lane; c < D; c += 32) {
+            const double xi = (double)__bfloat162float(Kr[j * D + c]) - kb[c];
+            e += xi * y[c];
+            f += xi * t[c];
+        }
+        e = warp_sum(e);
+        f = warp_sum(f);
+        if (lane == 0) { ee[j] = e; ff[j] = f; }
+    }
+    __syncthreads();
+    double kappa = 0.0;
+    for (int j = 0; j < L; ++j) kappa += pj[j] * (1.0 - ee[j]) * gam[j];      // g . o_i
+    for (int c = 0; c < D; ++c) kappa += t[c] * mb[c];
+    __syncthreads();
+    // per key: a_j -> pj, scale dL/ds_ij -> gam, p (f - gamma + gbar) -> ff, p (e - 1) -> ee
+    for (int j = tid; j < L; j += BW_THREADS) {
+        const double p = pj[j], e = ee[j], f = ff[j], gmj = gam[j];
+        pj[j] = p * (1.0 - e);
+        gam[j] = scale * p * (gmj * (1.0 - e) + (gbar + f) * e - f - kappa);
+        ff[j] = p * (f - gmj + gbar);
+        ee[j] = p * (e - 1.0);
+    }
+    __syncthreads();
+    for (int c = tid; c < D; c += BW_THREADS) {
+        double acc = t[c];
+        for (int j = 0; j < L; ++j) acc += gam[j] * (double)__bfloat162float(Kr[j * D + c]);
+        dq[(base + i) * D + c] = (float)acc;
+    }
+    for (int idx = tid; idx < L * D; idx += BW_THREADS) {
+        const int j = idx / D, c = idx % D;
+        atomicAdd(dk + (base + j) * D + c, (float)(gam[j] * qd[c] + ff[j] * y[c] + ee[j] * t[c]));
+        atomicAdd(dv + (base + j) * D + c, (float)(pj[j] * gd[c]));
+    }
+}
+
+template <int D>
+size_t head_smem_bytes(int lcap) {
+    return sizeof(double) * ((size_t)D * (D + 1) + 7 * D + 4 * lcap) + sizeof(__nv_bfloat16) * (size_t)lcap * D;
+}
+
+// workspace: kbar, h, t, y as [rows][D] fp32, then the scalar records
+size_t ws_floats(long long rows, int d) { return (size_t)rows * (4 * (size_t)d + BW_ROWSC); }
+
+template <int D>
+int launch_t(const BackwardArgs& a) {
+    using C = BwCfg<D>;
+    const long long rows = (long long)a.B * a.H * a.n;
+    const int BH = a.B * a.H;
+    const int first = max(0, min(a.n, a.head_rows - 1));      // rows [0, first) are solved directly
+    if (a.workspace_bytes < ws_floats(rows, D) * sizeof(float) || !a.workspace) return LLA_ERR_WORKSPACE;
+    float* kbar = static_cast<float*>(a.workspace);
+    float* hvec = kbar + rows * D;
+    float* tvec = hvec + rows * D;
+    float* yvec = tvec + rows * D;
+    float* rowsc = yvec + rows * D;
+    const auto* q = static_cast<const __nv_bfloat16*>(a.q);
+    const auto* k = static_cast<const __nv_bfloat16*>(a.k);
+    const auto* v = static_cast<const __nv_bfloat16*>(a.v);
+    const size_t head_smem = head_smem_bytes<D>(first);
+    if (head_smem > 227u * 1024u) return LLA_ERR_UNSUPPORTED;
+    LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::MOMENTS_SMEM));
+    LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::PAIRS_SMEM));
+    LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_head_rows_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem));
+    if (first < a.n) {
+        const dim3 gm((a.n + C::BI - 1) / C::BI, BH);
+        bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
+                                                                          rowsc, a.n, first, a.scale);
+        LLA_CUDA_TRY(cudaGetLastError());
+        // C_i t_i = h_i for the iterative rows: the forward's tensor-core CG with h as right-hand side
+        ForwardArgs f = {};
+        f.q = a.q; f.k = a.k; f.v = a.v; f.out = nullptr;
+        f.B = a.B; f.H = a.H; f.n = a.n; f.d = D; f.dv = D;
+        f.in_dtype = LLA_BF16; f.out_dtype = LLA_F32;
+        f.scale = a.scale; f.lambda = a.lambda; f.causal = 1;
+        f.max_iters = a.max_iters; f.tol = a.tol; f.head_rows = a.head_rows;
+        f.status = a.status; f.stream = a.stream;
+        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n;
+        f.rhs = hvec; f.sol = tvec;
+        const int rc = launch_forward_tensor(f);
+        if (rc != LLA_OK) return rc;
+        bwd_rowprep_kernel<D><<<(unsigned)((rows + 7) / 8), BW_THREADS, 0, a.stream>>>(
+            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, a.n, first, rows);
+        LLA_CUDA_TRY(cudaGetLastError());
+    }
+    {
+        const dim3 gp((a.n + BW_BJ - 1) / BW_BJ, BH);
+        bwd_pairs_kernel<D><<<gp, BW_THREADS, C::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
+                                                                      a.dk, a.dv, a.n, first, a.scale);
+        LLA_CUDA_TRY(cudaGetLastError());
+    }
+    if (first > 0) {
+        const dim3 gh(BH, first);
+        bwd_head_rows_kernel<D><<<gh, BW_THREADS, head_smem, a.stream>>>(
+            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status);
+        LLA_CUDA_TRY(cudaGetLastError());
+    }
+    return LLA_OK;
+}
+
+}  // namespace
+
+size_t backward_workspace_bytes(int B, int H, int n, int d) {
+    return ws_floats((long long)B * H * n, d) * sizeof(float);
+}
+
+int launch_backward(const BackwardArgs& a) {
+    if (a.d == 64) return launch_t<64>(a);
+    if (a.d == 128) return launch_t<128>(a);
+    return LLA_ERR_UNSUPPORTED;
+}
+
+}  // namespace lla

@@ -34,6 +34,8 @@ struct ForwardArgs {
     const float* lambda_rows;   // optional per-row ridge [B, H, nq]
     int ridge_mode;             // lla_ridge_mode
     int nq;                     // query rows per head (the last nq of the n positions); nq == n: plain prefill
+    const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
+    float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
 };
 
 struct DecodeArgs {
@@ -55,6 +57,33 @@ struct DecodeArgs {
     const float* lambda_units;  // optional per-(sequence, head) ridge [B, H]
     int ridge_mode;             // lla_ridge_mode
 };
+
+// Backward pass (backward appendix): gradients of a scalar loss with respect to q, k, v given
+// g = dL/d(out) and the tensors the forward saved.
+struct BackwardArgs {
+    const void* q;
+    const void* k;
+    const void* v;
+    const void* out;      // forward output [B, H, n, d] (out_dtype)
+    const void* dout;     // upstream gradient g [B, H, n, d] (dout_dtype)
+    const float* rho;     // saved by the forward [B, H, n, d]
+    const float* stats;   // saved by the forward [B, H, n, 3]
+    float* dq;            // [B, H, n, d] fp32
+    float* dk;
+    float* dv;
+    int B, H, n, d;
+    int out_dtype, dout_dtype;
+    float scale, lambda;
+    int max_iters;
+    float tol;
+    int head_rows;
+    int* status;
+    void* workspace;
+    size_t workspace_bytes;
+    cudaStream_t stream;
+};
+size_t backward_workspace_bytes(int B, int H, int n, int d);
+int launch_backward(const BackwardArgs& a);
 
 // Launchers implemented in the other translation units; each returns an lla_status.
 int head_rows_count(const ForwardArgs& a);   // leading query rows per head solved directly
@@ -149,10 +178,12 @@ __device__ __forceinline__ double fast_rcp1(double x) {
 // Optional phase timing for tuning (-DLLA_HR_TIMING): clock totals of thread 0 go to tst[phase].
 #ifdef LLA_HR_TIMING
 #define LDLT_TARG , int* tst = nullptr
+#define LDLT_NOARG , nullptr
 #define LDLT_T0 long long lt_ = clock64()
 #define LDLT_T(ph) do { if (threadIdx.x == 0 && tst) { const long long now_ = clock64(); atomicAdd(tst + (ph), (int)((now_ - lt_) >> 4)); lt_ = now_; } } while (0)
 #else
 #define LDLT_TARG
+#define LDLT_NOARG
 #define LDLT_T0
 #define LDLT_T(ph)
 #endif
@@ -187,7 +218,10 @@ __device__ __forceinline__ void ldlt_diag_block(double* S, int lds, int c0) {
 }
 
 template <int D>
-__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs, int n = D LDLT_TARG) {
+__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs, int n = D LDLT_TARG,
+                                                 int nrhs = 1, int rhs_stride = 0) {
+    // nrhs right-hand sides at rhs + q * rhs_stride, each replaced by its solution
+    const int nend = n + nrhs;
     LDLT_T0;
     const int tid = threadIdx.x, nt = blockDim.x;
     const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
@@ -204,8 +238,8 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
 #pragma unroll
         for (int k = 0; k < NB; ++k) dinv[k] = S[(c0 + k) * lds + c0 + k + 1];
         // (ii)
-        for (int r = c0 + NB + tid; r <= n; r += nt) {
-            double* rowp = r < n ? S + r * lds : rhs;
+        for (int r = c0 + NB + tid; r < nend; r += nt) {
+            double* rowp = r < n ? S + r * lds : rhs + (r - n) * rhs_stride;
             double x[NB];
 #pragma unroll
             for (int k = 0; k < NB; ++k) x[k] = rowp[c0 + k];
@@ -233,7 +267,7 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
                 for (int k = 0; k < NB; ++k) u[sl][k] = c2 < n ? S[c2 * lds + c0 + k] * dinv[k] : 0.0;
             }
             auto update_row = [&](int r) {
-                double* rowp = r < n ? S + r * lds : rhs;
+                double* rowp = r < n ? S + r * lds : rhs + (r - n) * rhs_stride;
                 double a[NB];
 #pragma unroll
                 for (int k = 0; k < NB; ++k) a[k] = rowp[c0 + k];
@@ -268,9 +302,9 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
                 __syncwarp();
                 ldlt_diag_block<NB>(S, lds, c0 + NB);
                 if (ny == 1)
-                    for (int r = c0 + 2 * NB; r <= n; ++r) update_row(r);
+                    for (int r = c0 + 2 * NB; r < nend; ++r) update_row(r);
             } else {
-                for (int r = c0 + 2 * NB + ty - 1; r <= n; r += ny - 1) update_row(r);
+                for (int r = c0 + 2 * NB + ty - 1; r < nend; r += ny - 1) update_row(r);
             }
             __syncthreads();
             LDLT_T(2);
@@ -281,6 +315,7 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
         if (!(S[k * lds + k] > 0.0)) ok = false;
     LDLT_T(3);
     // rhs now holds y with L y = b.  Backward: x_t = (y_t - sum_{r>t} S[r][t] x_r) / D_t.
+    for (int q = 0; q < nrhs; ++q, rhs += rhs_stride)
     if (tid < 32) {
         constexpr int PER = (D + 31) / 32;
         const int i = tx & 7;

@@ -176,6 +176,8 @@ struct TcParams {
     float scale, lambda, tol;
     float* rho;
     float* stats;
+    const float* rhs;    // solve mode: right-hand sides h_i [B, H, nq, D]; the CG then solves C_i x = h_i ...
+    float* sol;          // ... and x_i is written here instead of running the output sweep
     int* iters;
     int* status;
     float* scratch;      // D = 128: per-SM slots for x, kbar, r (TcCfg::SCRATCH_FLOATS_PER_SM each)
@@ -629,7 +631,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         const float kb = acc[col] * inv_omega;
                         kbs[(c0 + col) * TC_BR + lrow] = kb;
                         xs[(c0 + col) * TC_BR + lrow] = 0.f;
-                        const float bv = row_ok ? kb - qv : 0.f;
+                        const float bv = !row_ok ? 0.f : prm.rhs ? prm.rhs[((size_t)bh * nq + row) * D + c0 + col] : kb - qv;
                         r_set(col, bv);
                         p[col] = bv;
                         rr_p += bv * bv;
@@ -717,7 +719,17 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const bool at_cap = active && rr > stop;
         // ---- output sweep ----
         float gfac = 1.f;
-        if (ok) {
+        if (ok && prm.sol) {
+            if (row_ok) {
+                const size_t rowi = (size_t)bh * nq + row;
+#pragma unroll
+                for (int e = 0; e < NCOL; ++e) prm.sol[rowi * D + c0 + e] = xs[(c0 + e) * TC_BR + lrow];
+                if (half == 0 && prm.status) {
+                    if (at_cap) atomicAdd(prm.status + LLA_STATUS_ROWS_AT_CAP, 1);
+                    atomicAdd(prm.status + LLA_STATUS_ITER_SUM, its);
+                }
+            }
+        } else if (ok) {
             float y[NCOL];
             float yb_p = 0.f, g_p = 0.f;
 #pragma unroll
@@ -861,6 +873,7 @@ int launch_t(const ForwardArgs& a) {
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
+    prm.rhs = a.rhs; prm.sol = a.sol;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     prm.dbg = nullptr;
     prm.scratch = nullptr;

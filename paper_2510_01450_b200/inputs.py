@@ -107,6 +107,14 @@ def make_prefill(w: Workload):
     return _finish(q, w.dtype), _finish(k, w.dtype), _finish(v, w.dtype)
 
 
+def make_upstream_grad(w: Workload, dtype: str = "f32") -> np.ndarray:
+    """Upstream gradient g = dL/d(out) for the backward pass, [B,H,n,dv]: standard normal entries (the
+    gradient a unit-variance loss head hands back), drawn from a stream of its own so that q, k, v
+    of the same workload are unchanged."""
+    rng = np.random.default_rng([w.seed, 0x6772])
+    return _finish(rng.standard_normal((w.B, w.H, w.n, w.dv), dtype=np.float32), dtype)
+
+
 def make_decode(w: Workload):
     """Return (q [B,H,d], kcache [B,H,Lmax,d], vcache [B,H,Lmax,dv], lens [B] int32)."""
     assert w.kind == "decode"

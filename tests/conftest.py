@@ -17,3 +17,9 @@ def oracle():
     from oracle import lla_oracle
     lla_oracle.build()
     return lla_oracle
+
+
+@pytest.fixture(scope="session")
+def backward_oracle():
+    from oracle import lla_backward_oracle
+    return lla_backward_oracle

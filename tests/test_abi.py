@@ -61,6 +61,22 @@ def test_struct_sizes_match_c_layout(tmp_path):
     assert ctypes.sizeof(D) == 5 * 8 + 11 * 4 + 4 + 4 * 8 + 8 + 8
 
 
+def test_backward_struct_matches_c_layout(tmp_path):
+    import subprocess
+    fields = [name for name, _ in binding.BackwardParams._fields_]
+    cnames = ["lambda" if f == "lambda_" else f for f in fields]
+    src = tmp_path / "bw.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "lla.h"\nint main(void) {\n'
+                   '  printf("%zu", sizeof(lla_backward_params));\n'
+                   + "".join(f'  printf(" %zu", offsetof(lla_backward_params, {c}));\n' for c in cnames)
+                   + "  return 0; }\n")
+    exe = tmp_path / "bw"
+    subprocess.run(["gcc", "-I", str(ROOT / "include"), "-o", str(exe), str(src)], check=True)
+    got = [int(x) for x in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    B = binding.BackwardParams
+    assert got == [ctypes.sizeof(B)] + [getattr(B, f).offset for f in fields]
+
+
 def test_argument_validation_without_device(lib):
     ok_ptr = 0x1000
     args = dict(B=1, H=1, n=8, d=64, dv=64, scale=0.125, lam=1e-3)
