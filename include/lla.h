@@ -302,6 +302,7 @@ typedef struct lla_backward_params {
     void *workspace;
     size_t workspace_bytes;
     void *stream;
+    int impl;     /* LLA_IMPL_AUTO: pair kernel on the tensor cores where it exists (d = 64); LLA_IMPL_SIMT: CUDA cores */
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -106,8 +106,8 @@ bwd_moments_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
     float* PGt = Pt + BW_BJ * LDT;
     float* gbs = PGt + BW_BJ * LDT;       // [BI]
     const int tid = threadIdx.x, ti = tid >> 4, tj = tid & 15;
-    const int tile = gridDim.x - 1 - blockIdx.x;      // longest tiles first
-    const int bh = blockIdx.y;
+    const int tile = gridDim.y - 1 - blockIdx.y;      // longest tiles first, heads fastest
+    const int bh = blockIdx.x;
     const int i0 = tile * BI;
     if (i0 + BI <= first) return;                      // every row of the tile is solved directly
     const size_t base = (size_t)bh * n;
@@ -264,8 +264,8 @@ bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
     float* P1m = DSm + BI * LDP;          //               p_ij (f_ij - gamma_ij + gbar_i)
     float* DSt = P1m + BI * LDP;          // [key][query]: scale dL/ds_ij
     const int tid = threadIdx.x, ti = tid >> 4, tj = tid & 15;
-    const int bh = blockIdx.y;
-    const int j0 = blockIdx.x * BW_BJ;    // key tile 0 sees the most query tiles and starts first
+    const int bh = blockIdx.x;
+    const int j0 = blockIdx.y * BW_BJ;    // key tile 0 sees the most query tiles and starts first (heads fastest)
     const size_t base = (size_t)bh * n;
     load_tile<D>(Ks, k, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
     load_tile<D>(Vs, v, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
@@ -350,12 +350,249 @@ bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
 #pragma unroll
         for (int u = 0; u < CU; ++u) {
             const int c = 4 * tj + 64 * u;
-            *reinterpret_cast<float4*>(dk + (base + gj) * D + c) =
-                make_float4(adk[r][4 * u], adk[r][4 * u + 1], adk[r][4 * u + 2], adk[r][4 * u + 3]);
-            *reinterpret_cast<float4*>(dv + (base + gj) * D + c) =
-                make_float4(adv[r][4 * u], adv[r][4 * u + 1], adv[r][4 * u + 2], adv[r][4 * u + 3]);
+            // (added, not stored: the directly-solved rows add their share from another stream)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                atomicAdd(dk + (base + gj) * D + c + x, adk[r][4 * u + x]);
+                atomicAdd(dv + (base + gj) * D + c + x, adv[r][4 * u + x]);
+            }
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The pair kernel on the tensor cores (d = 64): the same block-per-key-tile loop with every product a
+// warp-level bf16 MMA (m16n8k16, fp32 accumulate).  fp32 operands (y, t, g and the pair coefficients)
+// enter as bf16 hi + lo pairs and each product keeps the three leading terms, so the result has fp32-like
+// accuracy.  A warp owns 16 of the block's 64 keys and forms the pair tiles transposed ([key][query]):
+// their accumulator fragments are then, after packing, the A operands of the dK / dV products with no
+// trip through shared memory.  Only scale dL/ds goes to shared memory, for the dQ product.
+// ------------------------------------------------------------------------------------------------
+constexpr int MM_LDB = 72;          // bf16 row stride of the operand tiles (64 + 8: conflict-free ldmatrix)
+constexpr int MM_THREADS = 128;
+constexpr int MM_TILE = 64 * MM_LDB;                         // bf16 elements per tile
+constexpr size_t MM_SMEM = sizeof(__nv_bfloat16) * (size_t)11 * MM_TILE + sizeof(float) * 6 * 64;
+
+__device__ __forceinline__ void ldsm4(uint32_t (&r)[4], const __nv_bfloat16* p) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm4t(uint32_t (&r)[4], const __nv_bfloat16* p) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// (x0, x1) -> packed bf16 pairs hi and lo with x = hi + lo up to 2^-17 relative
+__device__ __forceinline__ void split_pack(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+    const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0)), l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+    hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+    lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+// 64 rows x 64 columns -> bf16 tile(s) [64][MM_LDB]; fp32 sources are split into hi and lo tiles
+__device__ __forceinline__ void mm_load_bf16(__nv_bfloat16* dst, const __nv_bfloat16* src, size_t row0, int nvalid) {
+    for (int idx = threadIdx.x; idx < 64 * 8; idx += MM_THREADS) {
+        const int r = idx >> 3, c = (idx & 7) * 8;
+        uint4 x = make_uint4(0, 0, 0, 0);
+        if (r < nvalid) x = *reinterpret_cast<const uint4*>(src + (row0 + r) * 64 + c);
+        *reinterpret_cast<uint4*>(dst + r * MM_LDB + c) = x;
+    }
+}
+__device__ __forceinline__ void mm_load_split(__nv_bfloat16* hi, __nv_bfloat16* lo, const void* src, int dtype, size_t row0,
+                                              int nvalid, int lo_row) {
+    for (int idx = threadIdx.x; idx < 64 * 16; idx += MM_THREADS) {
+        const int r = idx >> 4, c = (idx & 15) * 4;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < nvalid && r >= lo_row) {
+            if (dtype == LLA_F32) x = load4(static_cast<const float*>(src) + (row0 + r) * 64 + c);
+            else x = load4(static_cast<const __nv_bfloat16*>(src) + (row0 + r) * 64 + c);
+        }
+        uint2 h, l;
+        split_pack(x.x, x.y, h.x, l.x);
+        split_pack(x.z, x.w, h.y, l.y);
+        *reinterpret_cast<uint2*>(hi + r * MM_LDB + c) = h;
+        *reinterpret_cast<uint2*>(lo + r * MM_LDB + c) = l;
+    }
+}
+
+__global__ void __launch_bounds__(MM_THREADS, 2)
+bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                     const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
+                     const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ rowsc,
+                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale) {
+    constexpr int D = 64, LDB = MM_LDB;
+    extern __shared__ __align__(16) unsigned char mm_smem[];
+    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(mm_smem);
+    __nv_bfloat16* Vs = Ks + MM_TILE;
+    __nv_bfloat16* Qs = Vs + MM_TILE;
+    __nv_bfloat16* Gh = Qs + MM_TILE;
+    __nv_bfloat16* Gl = Gh + MM_TILE;
+    __nv_bfloat16* Yh = Gl + MM_TILE;
+    __nv_bfloat16* Yl = Yh + MM_TILE;
+    __nv_bfloat16* Th = Yl + MM_TILE;
+    __nv_bfloat16* Tl = Th + MM_TILE;
+    __nv_bfloat16* DSh = Tl + MM_TILE;      // [key][query]
+    __nv_bfloat16* DSl = DSh + MM_TILE;
+    float* rs = reinterpret_cast<float*>(DSl + MM_TILE);   // [6][64]: m, 1/omega, gbar, kappa, kbar.y, kbar.t
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int bh = blockIdx.x;
+    const int j0 = blockIdx.y * 64;
+    const size_t base = (size_t)bh * n;
+    mm_load_bf16(Ks, k, base + j0, min(64, n - j0));
+    mm_load_bf16(Vs, v, base + j0, min(64, n - j0));
+    // ldmatrix lane offsets: (rows +8 by bit 3, columns +8 by bit 4) and (columns +8 by bit 3, rows +8 by bit 4)
+    const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
+    const int offA = (l7 + 8 * b3) * LDB + 8 * b4;     // A operand, or B^T-stored operand read with .trans
+    const int offB = (l7 + 8 * b4) * LDB + 8 * b3;     // B operand stored [n][k], or A^T-stored operand read with .trans
+    const int kr0 = 16 * warp;
+    float adk[8][4] = {}, adv[8][4] = {};
+    const int it0 = max(j0, first) / 64, it1 = (n + 63) / 64;
+    for (int it = it0; it < it1; ++it) {
+        const int i0 = it * 64;
+        const int nrow = min(64, n - i0);
+        __syncthreads();
+        mm_load_bf16(Qs, q, base + i0, nrow);
+        mm_load_split(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
+        mm_load_split(Yh, Yl, yvec, LLA_F32, base + i0, nrow, first - i0);
+        mm_load_split(Th, Tl, tvec, LLA_F32, base + i0, nrow, first - i0);
+        for (int idx = tid; idx < 6 * 64; idx += MM_THREADS) {
+            const int w = idx >> 6, r = idx & 63, gi = i0 + r;
+            rs[idx] = (gi < n && gi >= first) ? rowsc[(base + gi) * BW_ROWSC + w] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            const int ih = 32 * half;
+            float sT[4][4] = {}, eT[4][4] = {}, fT[4][4] = {}, gT[4][4] = {};
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t ak[4], av[4];
+                ldsm4(ak, Ks + kr0 * LDB + 16 * ks + offA);
+                ldsm4(av, Vs + kr0 * LDB + 16 * ks + offA);
+#pragma unroll
+                for (int nbp = 0; nbp < 2; ++nbp) {
+                    const int o = (ih + 16 * nbp) * LDB + 16 * ks + offB;
+                    uint32_t b[4];
+                    ldsm4(b, Qs + o);
+                    mma_bf16(sT[2 * nbp], ak, b[0], b[1]);
+                    mma_bf16(sT[2 * nbp + 1], ak, b[2], b[3]);
+                    ldsm4(b, Yh + o);
+                    mma_bf16(eT[2 * nbp], ak, b[0], b[1]);
+                    mma_bf16(eT[2 * nbp + 1], ak, b[2], b[3]);
+                    ldsm4(b, Yl + o);
+                    mma_bf16(eT[2 * nbp], ak, b[0], b[1]);
+                    mma_bf16(eT[2 * nbp + 1], ak, b[2], b[3]);
+                    ldsm4(b, Th + o);
+                    mma_bf16(fT[2 * nbp], ak, b[0], b[1]);
+                    mma_bf16(fT[2 * nbp + 1], ak, b[2], b[3]);
+                    ldsm4(b, Tl + o);
+                    mma_bf16(fT[2 * nbp], ak, b[0], b[1]);
+                    mma_bf16(fT[2 * nbp + 1], ak, b[2], b[3]);
+                    ldsm4(b, Gh + o);
+                    mma_bf16(gT[2 * nbp], av, b[0], b[1]);
+                    mma_bf16(gT[2 * nbp + 1], av, b[2], b[3]);
+                    ldsm4(b, Gl + o);
+                    mma_bf16(gT[2 * nbp], av, b[0], b[1]);
+                    mma_bf16(gT[2 * nbp + 1], av, b[2], b[3]);
+                }
+            }
+            // pair coefficients in place: sT <- a, eT <- scale dL/ds, fT <- p (f - gamma + gbar)
+#pragma unroll
+            for (int nb = 0; nb < 4; ++nb) {
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    const int il = ih + 8 * nb + 2 * t4 + (x & 1), gi = i0 + il;
+                    const int gj = j0 + kr0 + g + 8 * (x >> 1);
+                    const float iom = rs[64 + il];
+                    const float p = (iom > 0.f && gj <= gi) ? __expf(fmaf(scale, sT[nb][x], -rs[il])) * iom : 0.f;
+                    const float gbar = rs[128 + il], kappa = rs[192 + il];
+                    const float ev = eT[nb][x] - rs[256 + il], fv = fT[nb][x] - rs[320 + il], gam = gT[nb][x];
+                    sT[nb][x] = p * (1.f - ev);
+                    eT[nb][x] = scale * p * (gam * (1.f - ev) + (gbar + fv) * ev - fv - kappa);
+                    fT[nb][x] = p * (fv - gam + gbar);
+                }
+            }
+#pragma unroll
+            for (int ks2 = 0; ks2 < 2; ++ks2) {
+                // A fragments (rows = this warp's keys, k = 16 queries) of a, -a, ds, p1 as hi and lo
+                uint32_t ah[4], al[4], nh[4], nl[4], dh[4], dl[4], ph[4], pl[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int nb = 2 * ks2 + (r >> 1), x = 2 * (r & 1);
+                    split_pack(sT[nb][x], sT[nb][x + 1], ah[r], al[r]);
+                    nh[r] = ah[r] ^ 0x80008000u;
+                    nl[r] = al[r] ^ 0x80008000u;
+                    split_pack(eT[nb][x], eT[nb][x + 1], dh[r], dl[r]);
+                    split_pack(fT[nb][x], fT[nb][x + 1], ph[r], pl[r]);
+                    const int row = kr0 + g + 8 * (r & 1), col = ih + 8 * nb + 2 * t4;
+                    *reinterpret_cast<uint32_t*>(DSh + row * LDB + col) = dh[r];
+                    *reinterpret_cast<uint32_t*>(DSl + row * LDB + col) = dl[r];
+                }
+#pragma unroll
+                for (int ncp = 0; ncp < 4; ++ncp) {
+                    const int o = (ih + 16 * ks2) * LDB + 16 * ncp + offA;
+                    uint32_t b[4], c[4];
+                    ldsm4t(b, Gh + o);
+                    ldsm4t(c, Gl + o);
+                    mma_bf16(adv[2 * ncp], ah, b[0], b[1]);  mma_bf16(adv[2 * ncp + 1], ah, b[2], b[3]);
+                    mma_bf16(adv[2 * ncp], al, b[0], b[1]);  mma_bf16(adv[2 * ncp + 1], al, b[2], b[3]);
+                    mma_bf16(adv[2 * ncp], ah, c[0], c[1]);  mma_bf16(adv[2 * ncp + 1], ah, c[2], c[3]);
+                    ldsm4t(b, Qs + o);
+                    mma_bf16(adk[2 * ncp], dh, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], dh, b[2], b[3]);
+                    mma_bf16(adk[2 * ncp], dl, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], dl, b[2], b[3]);
+                    ldsm4t(b, Yh + o);
+                    ldsm4t(c, Yl + o);
+                    mma_bf16(adk[2 * ncp], ph, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], ph, b[2], b[3]);
+                    mma_bf16(adk[2 * ncp], pl, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], pl, b[2], b[3]);
+                    mma_bf16(adk[2 * ncp], ph, c[0], c[1]);  mma_bf16(adk[2 * ncp + 1], ph, c[2], c[3]);
+                    ldsm4t(b, Th + o);
+                    ldsm4t(c, Tl + o);
+                    mma_bf16(adk[2 * ncp], nh, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], nh, b[2], b[3]);
+                    mma_bf16(adk[2 * ncp], nl, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], nl, b[2], b[3]);
+                    mma_bf16(adk[2 * ncp], nh, c[0], c[1]);  mma_bf16(adk[2 * ncp + 1], nh, c[2], c[3]);
+                }
+            }
+        }
+        __syncthreads();
+        // dQ rows 16 warp .. +15 of the tile: sum over the block's 64 keys of (scale dL/ds) k_j
+        float adq[8][4] = {};
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            uint32_t ah[4], al[4];
+            ldsm4t(ah, DSh + 16 * ks * LDB + 16 * warp + offB);
+            ldsm4t(al, DSl + 16 * ks * LDB + 16 * warp + offB);
+#pragma unroll
+            for (int ncp = 0; ncp < 4; ++ncp) {
+                uint32_t b[4];
+                ldsm4t(b, Ks + 16 * ks * LDB + 16 * ncp + offA);
+                mma_bf16(adq[2 * ncp], ah, b[0], b[1]);  mma_bf16(adq[2 * ncp + 1], ah, b[2], b[3]);
+                mma_bf16(adq[2 * ncp], al, b[0], b[1]);  mma_bf16(adq[2 * ncp + 1], al, b[2], b[3]);
+            }
+        }
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int gi = i0 + 16 * warp + g + 8 * (x >> 1);
+                if (gi < n && gi >= first) atomicAdd(dq + (base + gi) * D + 8 * nb + 2 * t4 + (x & 1), adq[nb][x]);
+            }
+    }
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int gj = j0 + kr0 + g + 8 * (x >> 1);
+            if (gj >= n) continue;
+            const size_t e = (base + gj) * D + 8 * nb + 2 * t4 + (x & 1);
+            atomicAdd(dk + e, adk[nb][x]);
+            atomicAdd(dv + e, adv[nb][x]);
+        }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -535,8 +772,24 @@ int launch_t(const BackwardArgs& a) {
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::MOMENTS_SMEM));
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::PAIRS_SMEM));
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_head_rows_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem));
+    LLA_CUDA_TRY(cudaMemsetAsync(a.dk, 0, sizeof(float) * rows * D, a.stream));
+    LLA_CUDA_TRY(cudaMemsetAsync(a.dv, 0, sizeof(float) * rows * D, a.stream));
+    // the directly-solved rows depend on nothing the other kernels make: they run beside them on the side stream
+    const bool forked = first > 0 && a.side_stream != nullptr;
+    cudaStream_t hs = forked ? a.side_stream : a.stream;
+    if (forked) {
+        LLA_CUDA_TRY(cudaEventRecord(a.fork, a.stream));
+        LLA_CUDA_TRY(cudaStreamWaitEvent(hs, a.fork, 0));
+    }
+    if (first > 0) {
+        const dim3 gh(BH, first);
+        bwd_head_rows_kernel<D><<<gh, BW_THREADS, head_smem, hs>>>(
+            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status);
+        LLA_CUDA_TRY(cudaGetLastError());
+        if (forked) LLA_CUDA_TRY(cudaEventRecord(a.join, hs));
+    }
     if (first < a.n) {
-        const dim3 gm((a.n + C::BI - 1) / C::BI, BH);
+        const dim3 gm(BH, (a.n + C::BI - 1) / C::BI);
         bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
                                                                           rowsc, a.n, first, a.scale);
         LLA_CUDA_TRY(cudaGetLastError());
@@ -557,17 +810,18 @@ int launch_t(const BackwardArgs& a) {
         LLA_CUDA_TRY(cudaGetLastError());
     }
     {
-        const dim3 gp((a.n + BW_BJ - 1) / BW_BJ, BH);
-        bwd_pairs_kernel<D><<<gp, BW_THREADS, C::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
-                                                                      a.dk, a.dv, a.n, first, a.scale);
+        const dim3 gp(BH, (a.n + BW_BJ - 1) / BW_BJ);
+        if (D == 64 && !a.cuda_core_pairs) {
+            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MM_SMEM));
+            bwd_pairs_mma_kernel<<<gp, MM_THREADS, MM_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
+                                                                     a.dk, a.dv, a.n, first, a.scale);
+        } else {
+            bwd_pairs_kernel<D><<<gp, BW_THREADS, C::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc,
+                                                                          a.dq, a.dk, a.dv, a.n, first, a.scale);
+        }
         LLA_CUDA_TRY(cudaGetLastError());
     }
-    if (first > 0) {
-        const dim3 gh(BH, first);
-        bwd_head_rows_kernel<D><<<gh, BW_THREADS, head_smem, a.stream>>>(
-            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status);
-        LLA_CUDA_TRY(cudaGetLastError());
-    }
+    if (forked) LLA_CUDA_TRY(cudaStreamWaitEvent(a.stream, a.join, 0));
     return LLA_OK;
 }
 

@@ -81,6 +81,9 @@ struct BackwardArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
+    int cuda_core_pairs;        // 1: pair kernel on the CUDA cores even where the tensor-core one exists
+    cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
+    cudaEvent_t fork, join;
 };
 size_t backward_workspace_bytes(int B, int H, int n, int d);
 int launch_backward(const BackwardArgs& a);

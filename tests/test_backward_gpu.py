@@ -30,7 +30,7 @@ def grad_err(got, ref):
     return diff / np.maximum(rn, max(0.1 * float(np.median(rn)), 1e-4))
 
 
-def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", **kw):
+def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IMPL_AUTO, **kw):
     dq_, dk_, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
     dg = dev(g, dout_dtype)
     shape = (w.B, w.H, w.n, w.d)
@@ -45,21 +45,22 @@ def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", **kw):
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
     L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, *grads, w.B, w.H, w.n, w.d, w.scale, w.lam,
                       out_dtype=LLA_DT[out_dtype], dout_dtype=LLA_DT[dout_dtype], device_status=status,
-                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), **kw)
+                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), impl=impl, **kw)
     torch.cuda.synchronize()
     st = status.cpu().numpy()
     assert st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
     return [t.cpu().numpy().astype(np.float64) for t in grads]
 
 
-@pytest.mark.parametrize("d,n,B,H", [(64, 1, 1, 1), (64, 70, 1, 2), (64, 96, 1, 1), (64, 333, 2, 2), (64, 640, 1, 2),
-                                     (128, 150, 1, 1), (128, 420, 1, 2)])
-def test_backward_matches_gradient_oracle(backward_oracle, d, n, B, H):
+@pytest.mark.parametrize("d,n,B,H,impl", [(64, 1, 1, 1, 0), (64, 70, 1, 2, 0), (64, 96, 1, 1, 0), (64, 333, 2, 2, 0),
+                                          (64, 640, 1, 2, 0), (64, 333, 2, 2, 1), (64, 200, 1, 1, 1),
+                                          (128, 150, 1, 1, 0), (128, 420, 1, 2, 0)])
+def test_backward_matches_gradient_oracle(backward_oracle, d, n, B, H, impl):
     w = inputs.CONFIGS[2].shrink(B=B, H=H, n=n, d=d, dv=d, seed=200 + n)
     q, k, v = inputs.make_prefill(w)
     g = inputs.make_upstream_grad(w)
     ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
-    got = run_backward(w, q, k, v, g)
+    got = run_backward(w, q, k, v, g, impl=impl)
     for name, a, b in zip(("dq", "dk", "dv"), got, ref):
         assert np.isfinite(a).all(), name
         err = grad_err(a, b)
