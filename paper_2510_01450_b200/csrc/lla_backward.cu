@@ -595,6 +595,120 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         }
 }
 
+// The moments kernel on the tensor cores (d = 64): a warp owns 16 of the tile's 64 query rows; S = Q K^T
+// and Gamma = G V^T accumulate in registers, p and p gamma are packed straight into A fragments (hi + lo)
+// and multiply the key tile again for kbar and sum_j p gamma k.
+constexpr size_t MM_MOMENTS_SMEM = sizeof(__nv_bfloat16) * (size_t)5 * MM_TILE;
+
+__global__ void __launch_bounds__(MM_THREADS, 2)
+bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                       const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
+                       const float* __restrict__ stats, float* __restrict__ kbar, float* __restrict__ hvec,
+                       float* __restrict__ rowsc, int n, int first, float scale) {
+    constexpr int D = 64, LDB = MM_LDB;
+    extern __shared__ __align__(16) unsigned char mm_smem[];
+    __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(mm_smem);
+    __nv_bfloat16* Gh = Qs + MM_TILE;
+    __nv_bfloat16* Gl = Gh + MM_TILE;
+    __nv_bfloat16* Ks = Gl + MM_TILE;
+    __nv_bfloat16* Vs = Ks + MM_TILE;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int tile = gridDim.y - 1 - blockIdx.y;
+    const int bh = blockIdx.x;
+    const int i0 = tile * 64;
+    if (i0 + 64 <= first) return;
+    const size_t base = (size_t)bh * n;
+    const int nrow = min(64, n - i0);
+    mm_load_bf16(Qs, q, base + i0, nrow);
+    mm_load_split(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
+    const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
+    const int offA = (l7 + 8 * b3) * LDB + 8 * b4;
+    const int offB = (l7 + 8 * b4) * LDB + 8 * b3;
+    const int r0 = 16 * warp;
+    float mrow[2], iom[2], gb[2] = {0.f, 0.f};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int gi = i0 + r0 + g + 8 * h;
+        const bool okr = gi < n && gi >= first;
+        mrow[h] = okr ? stats[(base + gi) * 3 + 0] : 0.f;
+        iom[h] = okr ? 1.f / stats[(base + gi) * 3 + 1] : 0.f;
+    }
+    float akb[8][4] = {}, ah[8][4] = {};
+    const int jt_end = (min(n, i0 + 64) + 63) / 64;
+    for (int jt = 0; jt < jt_end; ++jt) {
+        const int j0 = jt * 64;
+        __syncthreads();
+        mm_load_bf16(Ks, k, base + j0, min(64, n - j0));
+        mm_load_bf16(Vs, v, base + j0, min(64, n - j0));
+        __syncthreads();
+        float s[8][4] = {}, gm[8][4] = {};
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            uint32_t aq[4], agh[4], agl[4];
+            ldsm4(aq, Qs + r0 * LDB + 16 * ks + offA);
+            ldsm4(agh, Gh + r0 * LDB + 16 * ks + offA);
+            ldsm4(agl, Gl + r0 * LDB + 16 * ks + offA);
+#pragma unroll
+            for (int nbp = 0; nbp < 4; ++nbp) {
+                uint32_t b[4];
+                ldsm4(b, Ks + 16 * nbp * LDB + 16 * ks + offB);
+                mma_bf16(s[2 * nbp], aq, b[0], b[1]);
+                mma_bf16(s[2 * nbp + 1], aq, b[2], b[3]);
+                ldsm4(b, Vs + 16 * nbp * LDB + 16 * ks + offB);
+                mma_bf16(gm[2 * nbp], agh, b[0], b[1]);
+                mma_bf16(gm[2 * nbp + 1], agh, b[2], b[3]);
+                mma_bf16(gm[2 * nbp], agl, b[0], b[1]);
+                mma_bf16(gm[2 * nbp + 1], agl, b[2], b[3]);
+            }
+        }
+        // s <- p, gm <- p gamma
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int h = x >> 1, gi = i0 + r0 + g + 8 * h, gj = j0 + 8 * nb + 2 * t4 + (x & 1);
+                const float p = (gj <= gi && iom[h] > 0.f) ? __expf(fmaf(scale, s[nb][x], -mrow[h])) * iom[h] : 0.f;
+                s[nb][x] = p;
+                gm[nb][x] *= p;
+                gb[h] += gm[nb][x];
+            }
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            uint32_t ph[4], pl[4], gh[4], gl[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int nb = 2 * ks + (r >> 1), x = 2 * (r & 1);
+                split_pack(s[nb][x], s[nb][x + 1], ph[r], pl[r]);
+                split_pack(gm[nb][x], gm[nb][x + 1], gh[r], gl[r]);
+            }
+#pragma unroll
+            for (int ncp = 0; ncp < 4; ++ncp) {
+                uint32_t b[4];
+                ldsm4t(b, Ks + 16 * ks * LDB + 16 * ncp + offA);
+                mma_bf16(akb[2 * ncp], ph, b[0], b[1]);  mma_bf16(akb[2 * ncp + 1], ph, b[2], b[3]);
+                mma_bf16(akb[2 * ncp], pl, b[0], b[1]);  mma_bf16(akb[2 * ncp + 1], pl, b[2], b[3]);
+                mma_bf16(ah[2 * ncp], gh, b[0], b[1]);   mma_bf16(ah[2 * ncp + 1], gh, b[2], b[3]);
+                mma_bf16(ah[2 * ncp], gl, b[0], b[1]);   mma_bf16(ah[2 * ncp + 1], gl, b[2], b[3]);
+            }
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        gb[h] += __shfl_xor_sync(0xffffffffu, gb[h], 1);
+        gb[h] += __shfl_xor_sync(0xffffffffu, gb[h], 2);
+        const int gi = i0 + r0 + g + 8 * h;
+        if (gi >= n || gi < first) continue;
+        if (t4 == 0) rowsc[(base + gi) * BW_ROWSC + 2] = gb[h];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+            const float kb0 = akb[nb][2 * h], kb1 = akb[nb][2 * h + 1];
+            const size_t e = (base + gi) * D + 8 * nb + 2 * t4;
+            *reinterpret_cast<float2*>(kbar + e) = make_float2(kb0, kb1);
+            *reinterpret_cast<float2*>(hvec + e) = make_float2(ah[nb][2 * h] - gb[h] * kb0, ah[nb][2 * h + 1] - gb[h] * kb1);
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Rows that see fewer than head_rows keys: C is ill-conditioned (rank-deficient up to the ridge), so the
 // whole row -- both solves and every pair term -- runs in fp64 with an explicit C and a direct LDL^T
@@ -790,8 +904,14 @@ int launch_t(const BackwardArgs& a) {
     }
     if (first < a.n) {
         const dim3 gm(BH, (a.n + C::BI - 1) / C::BI);
-        bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
-                                                                          rowsc, a.n, first, a.scale);
+        if (D == 64 && !a.cuda_core_pairs) {
+            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MM_MOMENTS_SMEM));
+            bwd_moments_mma_kernel<<<gm, MM_THREADS, MM_MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
+                                                                               rowsc, a.n, first, a.scale);
+        } else {
+            bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
+                                                                              rowsc, a.n, first, a.scale);
+        }
         LLA_CUDA_TRY(cudaGetLastError());
         // C_i t_i = h_i for the iterative rows: the forward's tensor-core CG with h as right-hand side
         ForwardArgs f = {};
