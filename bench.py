@@ -277,6 +277,9 @@ def run_ours(args):
         decode = None
         if rank == 0 and not args.no_decode:
             decode = bench_decode(L, torch, peaks, sp, stream)
+        backward = None
+        if rank == 0 and not args.no_backward:
+            backward = bench_backward(L, torch, peaks, w, sets, sp, stream)
 
     tokens_step = w.B * w.n
     ms_step = ms_total / args.steps
@@ -307,6 +310,8 @@ def run_ours(args):
     }
     if decode is not None:
         line["decode"] = decode
+    if backward is not None:
+        line["backward"] = backward
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, q0, k0, v0)
@@ -355,6 +360,56 @@ def bench_decode(L, torch, peaks, sp, stream, steps=20, warmup=5):
             "l2": "live cache bytes (1.2 GB) exceed L2 (126 MB)"}
 
 
+def bench_backward(L, torch, peaks, w, sets, sp, stream, steps=20, warmup=3, nsets=4):
+    """Backward pass (gradients with respect to q, k, v) on the bench workload: the forward runs once per
+    input set outside the timed region to save rho, stats and the fp32 output; the timed steps are
+    lla_backward_ex alone, rotating over nsets sets of inputs and saved tensors (together larger than L2)."""
+    shape = (w.B, w.H, w.n, w.d)
+    g = torch.from_numpy(inputs.make_upstream_grad(w)).cuda()
+    saved = []
+    for r in range(nsets):
+        q, k, v = sets[r]
+        out = torch.empty(shape, dtype=torch.float32, device="cuda")
+        rho = torch.empty(shape, dtype=torch.float32, device="cuda")
+        stats = torch.empty((w.B, w.H, w.n, 3), dtype=torch.float32, device="cuda")
+        L.lla_forward_ex(q, k, v, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1, out_dtype=L.LLA_F32,
+                         rho=rho, stats=stats, stream=sp)
+        saved.append((q, k, v, out, torch.roll(g, r, 1).contiguous(), rho, stats))
+    grads = [torch.empty(shape, dtype=torch.float32, device="cuda") for _ in range(3)]
+    nbytes = L.lla_backward_workspace_bytes(w.B, w.H, w.n, w.d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    iters = torch.full((w.B, w.H, w.n), -1, dtype=torch.int32, device="cuda")
+
+    def step(i, **kw):
+        L.lla_backward_ex(*saved[i % nsets], *grads, w.B, w.H, w.n, w.d, w.scale, w.lam, workspace=ws,
+                          workspace_bytes=nbytes, stream=sp, **kw)
+
+    step(0, iters=iters)
+    torch.cuda.synchronize()
+    it = iters.cpu().numpy().reshape(-1, w.n).astype(np.float64)
+    pairs = np.arange(1, w.n + 1, dtype=np.float64)
+    # per (query, key) pair: four score-like products and five output products (18 d) in the pair kernel, four
+    # products (8 d) in the moments kernel, 6 d per executed CG iteration of the extra solve
+    flops = float((26.0 * w.d * pairs[None, :] + 6.0 * w.d * pairs[None, :] * np.maximum(it, 0.0)).sum())
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(warmup + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    set_bytes = sum(t.numel() * t.element_size() for t in saved[0])
+    return {"ms_per_step": ms, "tokens_per_s": w.B * w.n / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
+            "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "cg_mean_iters": float(it[it >= 0].mean()) if (it >= 0).any() else 0.0,
+            "algorithmic_flops_per_step": flops, "gpu_launches_per_step": 5,
+            "l2": f"inputs and saved tensors rotate over {nsets} sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)",
+            "inputs": "bf16 q, k, v; fp32 upstream gradient, forward output, rho, stats; fp32 gradients"}
+
+
 def cpu_baseline(w, q, k, v):
     """The oracle, untuned, on this machine's host cores, on a bounded uniform row sample."""
     from oracle import lla_oracle
@@ -380,6 +435,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-decode", action="store_true", help="skip the decode measurement")
+    ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -302,6 +302,8 @@ typedef struct lla_backward_params {
     void *workspace;
     size_t workspace_bytes;
     void *stream;
+    int *iters;   /* optional [B, H, n] on the device: CG iterations of the extra solve per row (rows that are
+                     solved directly are left untouched) */
     int impl;     /* LLA_IMPL_AUTO: pair kernel on the tensor cores where it exists (d = 64); LLA_IMPL_SIMT: CUDA cores */
 } lla_backward_params;
 

@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     LLA_PHASE_ITERATIVE, LLA_STATUS_WORDS, STATUS_BAD_PIVOT, STATUS_ITER_SUM, STATUS_ROWS_AT_CAP, STATUS_TIMEOUT, LlaError,
     lla_decode, lla_decode_default_splits, lla_decode_ex, lla_decode_f32, lla_decode_host, lla_decode_noalloc,
     lla_decode_workspace_bytes, lla_forward, lla_forward_ex, lla_forward_f32, lla_forward_host,
-    lla_forward_workspace_bytes, lla_version, status_string,
+    lla_forward_workspace_bytes, lla_version, status_string, lla_backward_ex, lla_backward_workspace_bytes,
 )

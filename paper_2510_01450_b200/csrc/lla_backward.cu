@@ -920,7 +920,7 @@ int launch_t(const BackwardArgs& a) {
         f.in_dtype = LLA_BF16; f.out_dtype = LLA_F32;
         f.scale = a.scale; f.lambda = a.lambda; f.causal = 1;
         f.max_iters = a.max_iters; f.tol = a.tol; f.head_rows = a.head_rows;
-        f.status = a.status; f.stream = a.stream;
+        f.status = a.status; f.iters = a.iters; f.stream = a.stream;
         f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n;
         f.rhs = hvec; f.sol = tvec;
         const int rc = launch_forward_tensor(f);

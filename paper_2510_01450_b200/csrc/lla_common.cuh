@@ -78,6 +78,7 @@ struct BackwardArgs {
     float tol;
     int head_rows;
     int* status;
+    int* iters;           // optional [B, H, n]: CG iterations of the extra solve (rows solved directly: untouched)
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;

@@ -724,6 +724,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const size_t rowi = (size_t)bh * nq + row;
 #pragma unroll
                 for (int e = 0; e < NCOL; ++e) prm.sol[rowi * D + c0 + e] = xs[(c0 + e) * TC_BR + lrow];
+                if (half == 0 && prm.iters) prm.iters[rowi] = its;
                 if (half == 0 && prm.status) {
                     if (at_cap) atomicAdd(prm.status + LLA_STATUS_ROWS_AT_CAP, 1);
                     atomicAdd(prm.status + LLA_STATUS_ITER_SUM, its);

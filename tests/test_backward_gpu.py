@@ -38,7 +38,7 @@ def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IM
     rho = torch.empty(shape, dtype=torch.float32, device="cuda")
     stats = torch.empty((w.B, w.H, w.n, 3), dtype=torch.float32, device="cuda")
     L.lla_forward_ex(dq_, dk_, dv_, out, w.B, w.H, w.n, w.d, w.d, w.scale, w.lam, in_dtype=L.LLA_BF16,
-                     out_dtype=LLA_DT[out_dtype], rho=rho, stats=stats, stream=stream_ptr(), **kw)
+                     out_dtype=LLA_DT[out_dtype], rho=rho, stats=stats, stream=stream_ptr())
     grads = [torch.full(shape, float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
     nbytes = L.lla_backward_workspace_bytes(w.B, w.H, w.n, w.d)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
@@ -82,6 +82,21 @@ def test_backward_regression_recipe_and_bf16_tensors(backward_oracle):
         rows = np.linalg.norm(b.reshape(-1, w.d), axis=1)
         diff = np.linalg.norm((a - b).reshape(-1, w.d), axis=1)
         assert diff.max() <= 2.0 ** -8 * rows.max()
+
+
+def test_backward_bench_shape_one_head(backward_oracle):
+    # one head of the bench workload (n = 1024: 16 query tiles by 16 key tiles, the first 95 rows direct)
+    w = inputs.CONFIGS[2].shrink(B=1, H=1, seed=260)
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
+    iters = torch.full((1, 1, w.n), -1, dtype=torch.int32, device="cuda")
+    got = run_backward(w, q, k, v, g, iters=iters)
+    for name, a, b in zip(("dq", "dk", "dv"), got, ref):
+        err = grad_err(a, b)
+        assert err.max() <= TOL, (name, float(err.max()), int(err.argmax()))
+    it = iters.cpu().numpy().ravel()
+    assert (it[:95] == -1).all() and (it[95:] > 0).all() and it.max() <= 64
 
 
 def test_backward_argument_checks():
