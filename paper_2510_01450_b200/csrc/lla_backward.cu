@@ -368,10 +368,18 @@ bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
 // their accumulator fragments are then, after packing, the A operands of the dK / dV products with no
 // trip through shared memory.  Only scale dL/ds goes to shared memory, for the dQ product.
 // ------------------------------------------------------------------------------------------------
-constexpr int MM_LDB = 72;          // bf16 row stride of the operand tiles (64 + 8: conflict-free ldmatrix)
-constexpr int MM_THREADS = 128;
-constexpr int MM_TILE = 64 * MM_LDB;                         // bf16 elements per tile
-constexpr size_t MM_SMEM = sizeof(__nv_bfloat16) * (size_t)11 * MM_TILE + sizeof(float) * 6 * 64;
+// d = 128: the 128 output columns are split over two warps per key (query) group -- a warp's registers
+// hold accumulators for 64 columns only -- and both form the same pair tiles.
+template <int D>
+struct MmCfg {
+    static constexpr int LDB = D + 8;             // bf16 row stride of the operand tiles (conflict-free ldmatrix)
+    static constexpr int TILE = 64 * LDB;         // bf16 elements per 64-row tile
+    static constexpr int NCG = D / 64;            // column groups
+    static constexpr int THREADS = 128 * NCG;
+    static constexpr int KS = D / 16;             // k-steps of a contraction over the head dimension
+    static constexpr size_t PAIRS_SMEM = sizeof(__nv_bfloat16) * (size_t)11 * TILE + sizeof(float) * 6 * 64;
+    static constexpr size_t MOMENTS_SMEM = sizeof(__nv_bfloat16) * (size_t)5 * TILE;
+};
 
 __device__ __forceinline__ void ldsm4(uint32_t (&r)[4], const __nv_bfloat16* p) {
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
@@ -395,23 +403,26 @@ __device__ __forceinline__ void split_pack(float x0, float x1, uint32_t& hi, uin
     hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
     lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
 }
-// 64 rows x 64 columns -> bf16 tile(s) [64][MM_LDB]; fp32 sources are split into hi and lo tiles
+// 64 rows x D columns -> bf16 tile(s) [64][D + 8]; fp32 sources are split into hi and lo tiles
+template <int D>
 __device__ __forceinline__ void mm_load_bf16(__nv_bfloat16* dst, const __nv_bfloat16* src, size_t row0, int nvalid) {
-    for (int idx = threadIdx.x; idx < 64 * 8; idx += MM_THREADS) {
-        const int r = idx >> 3, c = (idx & 7) * 8;
+    for (int idx = threadIdx.x; idx < 64 * (D / 8); idx += MmCfg<D>::THREADS) {
+        const int r = idx / (D / 8), c = (idx % (D / 8)) * 8;
         uint4 x = make_uint4(0, 0, 0, 0);
-        if (r < nvalid) x = *reinterpret_cast<const uint4*>(src + (row0 + r) * 64 + c);
-        *reinterpret_cast<uint4*>(dst + r * MM_LDB + c) = x;
+        if (r < nvalid) x = *reinterpret_cast<const uint4*>(src + (row0 + r) * D + c);
+        *reinterpret_cast<uint4*>(dst + r * MmCfg<D>::LDB + c) = x;
     }
 }
+template <int D>
 __device__ __forceinline__ void mm_load_split(__nv_bfloat16* hi, __nv_bfloat16* lo, const void* src, int dtype, size_t row0,
                                               int nvalid, int lo_row) {
-    for (int idx = threadIdx.x; idx < 64 * 16; idx += MM_THREADS) {
-        const int r = idx >> 4, c = (idx & 15) * 4;
+    constexpr int MM_LDB = MmCfg<D>::LDB;
+    for (int idx = threadIdx.x; idx < 64 * (D / 4); idx += MmCfg<D>::THREADS) {
+        const int r = idx / (D / 4), c = (idx % (D / 4)) * 4;
         float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
         if (r < nvalid && r >= lo_row) {
-            if (dtype == LLA_F32) x = load4(static_cast<const float*>(src) + (row0 + r) * 64 + c);
-            else x = load4(static_cast<const __nv_bfloat16*>(src) + (row0 + r) * 64 + c);
+            if (dtype == LLA_F32) x = load4(static_cast<const float*>(src) + (row0 + r) * D + c);
+            else x = load4(static_cast<const __nv_bfloat16*>(src) + (row0 + r) * D + c);
         }
         uint2 h, l;
         split_pack(x.x, x.y, h.x, l.x);
@@ -421,12 +432,13 @@ __device__ __forceinline__ void mm_load_split(__nv_bfloat16* hi, __nv_bfloat16* 
     }
 }
 
-__global__ void __launch_bounds__(MM_THREADS, 2)
+template <int D>
+__global__ void __launch_bounds__(MmCfg<D>::THREADS, D == 64 ? 2 : 1)
 bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                      const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ rowsc,
                      float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale) {
-    constexpr int D = 64, LDB = MM_LDB;
+    constexpr int LDB = MmCfg<D>::LDB, MM_TILE = MmCfg<D>::TILE, MM_THREADS = MmCfg<D>::THREADS, KS = MmCfg<D>::KS;
     extern __shared__ __align__(16) unsigned char mm_smem[];
     __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(mm_smem);
     __nv_bfloat16* Vs = Ks + MM_TILE;
@@ -440,12 +452,14 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     __nv_bfloat16* DSh = Tl + MM_TILE;      // [key][query]
     __nv_bfloat16* DSl = DSh + MM_TILE;
     float* rs = reinterpret_cast<float*>(DSl + MM_TILE);   // [6][64]: m, 1/omega, gbar, kappa, kbar.y, kbar.t
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int warp = (tid >> 5) & 3;      // key group (16 keys); query group in the dQ product
+    const int cg = tid >> 7;              // column group (64 output columns)
     const int bh = blockIdx.x;
     const int j0 = blockIdx.y * 64;
     const size_t base = (size_t)bh * n;
-    mm_load_bf16(Ks, k, base + j0, min(64, n - j0));
-    mm_load_bf16(Vs, v, base + j0, min(64, n - j0));
+    mm_load_bf16<D>(Ks, k, base + j0, min(64, n - j0));
+    mm_load_bf16<D>(Vs, v, base + j0, min(64, n - j0));
     // ldmatrix lane offsets: (rows +8 by bit 3, columns +8 by bit 4) and (columns +8 by bit 3, rows +8 by bit 4)
     const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
     const int offA = (l7 + 8 * b3) * LDB + 8 * b4;     // A operand, or B^T-stored operand read with .trans
@@ -457,10 +471,10 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         const int i0 = it * 64;
         const int nrow = min(64, n - i0);
         __syncthreads();
-        mm_load_bf16(Qs, q, base + i0, nrow);
-        mm_load_split(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
-        mm_load_split(Yh, Yl, yvec, LLA_F32, base + i0, nrow, first - i0);
-        mm_load_split(Th, Tl, tvec, LLA_F32, base + i0, nrow, first - i0);
+        mm_load_bf16<D>(Qs, q, base + i0, nrow);
+        mm_load_split<D>(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
+        mm_load_split<D>(Yh, Yl, yvec, LLA_F32, base + i0, nrow, first - i0);
+        mm_load_split<D>(Th, Tl, tvec, LLA_F32, base + i0, nrow, first - i0);
         for (int idx = tid; idx < 6 * 64; idx += MM_THREADS) {
             const int w = idx >> 6, r = idx & 63, gi = i0 + r;
             rs[idx] = (gi < n && gi >= first) ? rowsc[(base + gi) * BW_ROWSC + w] : 0.f;
@@ -471,7 +485,7 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
             const int ih = 32 * half;
             float sT[4][4] = {}, eT[4][4] = {}, fT[4][4] = {}, gT[4][4] = {};
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
+            for (int ks = 0; ks < KS; ++ks) {
                 uint32_t ak[4], av[4];
                 ldsm4(ak, Ks + kr0 * LDB + 16 * ks + offA);
                 ldsm4(av, Vs + kr0 * LDB + 16 * ks + offA);
@@ -531,12 +545,14 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
                     split_pack(eT[nb][x], eT[nb][x + 1], dh[r], dl[r]);
                     split_pack(fT[nb][x], fT[nb][x + 1], ph[r], pl[r]);
                     const int row = kr0 + g + 8 * (r & 1), col = ih + 8 * nb + 2 * t4;
-                    *reinterpret_cast<uint32_t*>(DSh + row * LDB + col) = dh[r];
-                    *reinterpret_cast<uint32_t*>(DSl + row * LDB + col) = dl[r];
+                    if (cg == 0) {
+                        *reinterpret_cast<uint32_t*>(DSh + row * LDB + col) = dh[r];
+                        *reinterpret_cast<uint32_t*>(DSl + row * LDB + col) = dl[r];
+                    }
                 }
 #pragma unroll
                 for (int ncp = 0; ncp < 4; ++ncp) {
-                    const int o = (ih + 16 * ks2) * LDB + 16 * ncp + offA;
+                    const int o = (ih + 16 * ks2) * LDB + 64 * cg + 16 * ncp + offA;
                     uint32_t b[4], c[4];
                     ldsm4t(b, Gh + o);
                     ldsm4t(c, Gl + o);
@@ -570,7 +586,7 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 #pragma unroll
             for (int ncp = 0; ncp < 4; ++ncp) {
                 uint32_t b[4];
-                ldsm4t(b, Ks + 16 * ks * LDB + 16 * ncp + offA);
+                ldsm4t(b, Ks + 16 * ks * LDB + 64 * cg + 16 * ncp + offA);
                 mma_bf16(adq[2 * ncp], ah, b[0], b[1]);  mma_bf16(adq[2 * ncp + 1], ah, b[2], b[3]);
                 mma_bf16(adq[2 * ncp], al, b[0], b[1]);  mma_bf16(adq[2 * ncp + 1], al, b[2], b[3]);
             }
@@ -580,7 +596,7 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int gi = i0 + 16 * warp + g + 8 * (x >> 1);
-                if (gi < n && gi >= first) atomicAdd(dq + (base + gi) * D + 8 * nb + 2 * t4 + (x & 1), adq[nb][x]);
+                if (gi < n && gi >= first) atomicAdd(dq + (base + gi) * D + 64 * cg + 8 * nb + 2 * t4 + (x & 1), adq[nb][x]);
             }
     }
 #pragma unroll
@@ -589,7 +605,7 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         for (int x = 0; x < 4; ++x) {
             const int gj = j0 + kr0 + g + 8 * (x >> 1);
             if (gj >= n) continue;
-            const size_t e = (base + gj) * D + 8 * nb + 2 * t4 + (x & 1);
+            const size_t e = (base + gj) * D + 64 * cg + 8 * nb + 2 * t4 + (x & 1);
             atomicAdd(dk + e, adk[nb][x]);
             atomicAdd(dv + e, adv[nb][x]);
         }
@@ -598,29 +614,30 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 // The moments kernel on the tensor cores (d = 64): a warp owns 16 of the tile's 64 query rows; S = Q K^T
 // and Gamma = G V^T accumulate in registers, p and p gamma are packed straight into A fragments (hi + lo)
 // and multiply the key tile again for kbar and sum_j p gamma k.
-constexpr size_t MM_MOMENTS_SMEM = sizeof(__nv_bfloat16) * (size_t)5 * MM_TILE;
-
-__global__ void __launch_bounds__(MM_THREADS, 2)
+template <int D>
+__global__ void __launch_bounds__(MmCfg<D>::THREADS, D == 64 ? 2 : 1)
 bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                        const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                        const float* __restrict__ stats, float* __restrict__ kbar, float* __restrict__ hvec,
                        float* __restrict__ rowsc, int n, int first, float scale) {
-    constexpr int D = 64, LDB = MM_LDB;
+    constexpr int LDB = MmCfg<D>::LDB, MM_TILE = MmCfg<D>::TILE, KS = MmCfg<D>::KS;
     extern __shared__ __align__(16) unsigned char mm_smem[];
     __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(mm_smem);
     __nv_bfloat16* Gh = Qs + MM_TILE;
     __nv_bfloat16* Gl = Gh + MM_TILE;
     __nv_bfloat16* Ks = Gl + MM_TILE;
     __nv_bfloat16* Vs = Ks + MM_TILE;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int warp = (tid >> 5) & 3;      // query group (16 rows)
+    const int cg = tid >> 7;              // column group (64 output columns)
     const int tile = gridDim.y - 1 - blockIdx.y;
     const int bh = blockIdx.x;
     const int i0 = tile * 64;
     if (i0 + 64 <= first) return;
     const size_t base = (size_t)bh * n;
     const int nrow = min(64, n - i0);
-    mm_load_bf16(Qs, q, base + i0, nrow);
-    mm_load_split(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
+    mm_load_bf16<D>(Qs, q, base + i0, nrow);
+    mm_load_split<D>(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
     const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
     const int offA = (l7 + 8 * b3) * LDB + 8 * b4;
     const int offB = (l7 + 8 * b4) * LDB + 8 * b3;
@@ -638,12 +655,12 @@ bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
     for (int jt = 0; jt < jt_end; ++jt) {
         const int j0 = jt * 64;
         __syncthreads();
-        mm_load_bf16(Ks, k, base + j0, min(64, n - j0));
-        mm_load_bf16(Vs, v, base + j0, min(64, n - j0));
+        mm_load_bf16<D>(Ks, k, base + j0, min(64, n - j0));
+        mm_load_bf16<D>(Vs, v, base + j0, min(64, n - j0));
         __syncthreads();
         float s[8][4] = {}, gm[8][4] = {};
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
+        for (int ks = 0; ks < KS; ++ks) {
             uint32_t aq[4], agh[4], agl[4];
             ldsm4(aq, Qs + r0 * LDB + 16 * ks + offA);
             ldsm4(agh, Gh + r0 * LDB + 16 * ks + offA);
@@ -684,7 +701,7 @@ bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 #pragma unroll
             for (int ncp = 0; ncp < 4; ++ncp) {
                 uint32_t b[4];
-                ldsm4t(b, Ks + 16 * ks * LDB + 16 * ncp + offA);
+                ldsm4t(b, Ks + 16 * ks * LDB + 64 * cg + 16 * ncp + offA);
                 mma_bf16(akb[2 * ncp], ph, b[0], b[1]);  mma_bf16(akb[2 * ncp + 1], ph, b[2], b[3]);
                 mma_bf16(akb[2 * ncp], pl, b[0], b[1]);  mma_bf16(akb[2 * ncp + 1], pl, b[2], b[3]);
                 mma_bf16(ah[2 * ncp], gh, b[0], b[1]);   mma_bf16(ah[2 * ncp + 1], gh, b[2], b[3]);
@@ -698,11 +715,11 @@ bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
         gb[h] += __shfl_xor_sync(0xffffffffu, gb[h], 2);
         const int gi = i0 + r0 + g + 8 * h;
         if (gi >= n || gi < first) continue;
-        if (t4 == 0) rowsc[(base + gi) * BW_ROWSC + 2] = gb[h];
+        if (t4 == 0 && cg == 0) rowsc[(base + gi) * BW_ROWSC + 2] = gb[h];
 #pragma unroll
         for (int nb = 0; nb < 8; ++nb) {
             const float kb0 = akb[nb][2 * h], kb1 = akb[nb][2 * h + 1];
-            const size_t e = (base + gi) * D + 8 * nb + 2 * t4;
+            const size_t e = (base + gi) * D + 64 * cg + 8 * nb + 2 * t4;
             *reinterpret_cast<float2*>(kbar + e) = make_float2(kb0, kb1);
             *reinterpret_cast<float2*>(hvec + e) = make_float2(ah[nb][2 * h] - gb[h] * kb0, ah[nb][2 * h + 1] - gb[h] * kb1);
         }
@@ -904,9 +921,11 @@ int launch_t(const BackwardArgs& a) {
     }
     if (first < a.n) {
         const dim3 gm(BH, (a.n + C::BI - 1) / C::BI);
-        if (D == 64 && !a.cuda_core_pairs) {
-            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MM_MOMENTS_SMEM));
-            bwd_moments_mma_kernel<<<gm, MM_THREADS, MM_MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
+        if (!a.cuda_core_pairs) {
+            using M = MmCfg<D>;
+            const dim3 gm(BH, (a.n + 63) / 64);
+            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::MOMENTS_SMEM));
+            bwd_moments_mma_kernel<D><<<gm, M::THREADS, M::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
                                                                                rowsc, a.n, first, a.scale);
         } else {
             bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
@@ -931,9 +950,10 @@ int launch_t(const BackwardArgs& a) {
     }
     {
         const dim3 gp(BH, (a.n + BW_BJ - 1) / BW_BJ);
-        if (D == 64 && !a.cuda_core_pairs) {
-            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MM_SMEM));
-            bwd_pairs_mma_kernel<<<gp, MM_THREADS, MM_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
+        if (!a.cuda_core_pairs) {
+            using M = MmCfg<D>;
+            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::PAIRS_SMEM));
+            bwd_pairs_mma_kernel<D><<<gp, M::THREADS, M::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
                                                                      a.dk, a.dv, a.n, first, a.scale);
         } else {
             bwd_pairs_kernel<D><<<gp, BW_THREADS, C::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc,

@@ -54,7 +54,7 @@ def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IM
 
 @pytest.mark.parametrize("d,n,B,H,impl", [(64, 1, 1, 1, 0), (64, 70, 1, 2, 0), (64, 96, 1, 1, 0), (64, 333, 2, 2, 0),
                                           (64, 640, 1, 2, 0), (64, 333, 2, 2, 1), (64, 200, 1, 1, 1),
-                                          (128, 150, 1, 1, 0), (128, 420, 1, 2, 0)])
+                                          (128, 150, 1, 1, 0), (128, 420, 1, 2, 0), (128, 420, 1, 2, 1)])
 def test_backward_matches_gradient_oracle(backward_oracle, d, n, B, H, impl):
     w = inputs.CONFIGS[2].shrink(B=B, H=H, n=n, d=d, dv=d, seed=200 + n)
     q, k, v = inputs.make_prefill(w)
