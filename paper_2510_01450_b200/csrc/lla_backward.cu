@@ -737,12 +737,13 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
+constexpr int HB_THREADS = 128;   // four or five blocks per SM hide each other's factorisation latency
 template <int D>
-__global__ void __launch_bounds__(BW_THREADS)
+__global__ void __launch_bounds__(HB_THREADS)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
-                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int lcap,
-                     double scale, double lambda, int* __restrict__ status) {
+                     float* __restrict__ dq, float* __restrict__ yvec, float* __restrict__ tvec,
+                     float* __restrict__ hcoef, int n, int lcap, double scale, double lambda, int* __restrict__ status) {
     constexpr int LDS = D + 1;
     extern __shared__ __align__(16) double hb_smem[];
     double* S = hb_smem;                  // D x (D + 1)
@@ -762,15 +763,15 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int i = gridDim.y - 1 - blockIdx.y;       // rows with the most keys first
     const int L = i + 1;
     const size_t base = (size_t)bh * n;
-    for (int c = tid; c < D; c += BW_THREADS) {
+    for (int c = tid; c < D; c += HB_THREADS) {
         qd[c] = (double)__bfloat162float(q[(base + i) * D + c]);
         gd[c] = (double)ld_any(dout, dout_dtype, (base + i) * D + c);
     }
-    for (int idx = tid; idx < L * (D / 8); idx += BW_THREADS)
+    for (int idx = tid; idx < L * (D / 8); idx += HB_THREADS)
         reinterpret_cast<uint4*>(Kr)[idx] = reinterpret_cast<const uint4*>(k + base * D)[idx];
     __syncthreads();
     // scores and gamma_j = g . v_j: a warp per key
-    for (int j = warp; j < L; j += BW_THREADS / 32) {
+    for (int j = warp; j < L; j += HB_THREADS / 32) {
         double s = 0.0, gv = 0.0;
         for (int c = lane; c < D; c += 32) {
             s += qd[c] * (double)__bfloat162float(Kr[j * D + c]);
@@ -784,17 +785,17 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     double m = -1e300;
     for (int j = 0; j < L; ++j) m = fmax(m, pj[j]);
     __syncthreads();
-    for (int j = tid; j < L; j += BW_THREADS) pj[j] = exp(pj[j] - m);
+    for (int j = tid; j < L; j += HB_THREADS) pj[j] = exp(pj[j] - m);
     __syncthreads();
     double omega = 0.0;
     for (int j = 0; j < L; ++j) omega += pj[j];
     const double eps = lambda * exp(-m) / omega;
     __syncthreads();
-    for (int j = tid; j < L; j += BW_THREADS) pj[j] /= omega;
+    for (int j = tid; j < L; j += HB_THREADS) pj[j] /= omega;
     __syncthreads();
     double gbar = 0.0;
     for (int j = 0; j < L; ++j) gbar += pj[j] * gam[j];
-    for (int c = tid; c < 2 * D; c += BW_THREADS) {
+    for (int c = tid; c < 2 * D; c += HB_THREADS) {
         const int cc = c % D;
         double acc = 0.0;
         if (c < D) for (int j = 0; j < L; ++j) acc += pj[j] * (double)__bfloat162float(Kr[j * D + cc]);
@@ -802,13 +803,13 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         (c < D ? kb : hp)[cc] = acc;
     }
     __syncthreads();
-    for (int c = tid; c < D; c += BW_THREADS) {
+    for (int c = tid; c < D; c += HB_THREADS) {
         mb[c] = kb[c] - qd[c];
         rhs[c] = mb[c];
         rhs[D + c] = hp[c] - gbar * kb[c];
     }
     // C (lower triangle) in 4 x 4 blocks
-    for (int blk = tid; blk < (D / 4) * (D / 4); blk += BW_THREADS) {
+    for (int blk = tid; blk < (D / 4) * (D / 4); blk += HB_THREADS) {
         const int a0 = (blk / (D / 4)) * 4, b0 = (blk % (D / 4)) * 4;
         if (b0 > a0) continue;
         double acc[4][4] = {};
@@ -838,7 +839,7 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const double* y = rhs;
     const double* t = rhs + D;
     // e_j = xi_j . y, f_j = xi_j . t
-    for (int j = warp; j < L; j += BW_THREADS / 32) {
+    for (int j = warp; j < L; j += HB_THREADS / 32) {
         double e = 0.0, f = 0.0;
         for (int c = lane; c < D; c += 32) {
             const double xi = (double)__bfloat162float(Kr[j * D + c]) - kb[c];
@@ -855,7 +856,7 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     for (int c = 0; c < D; ++c) kappa += t[c] * mb[c];
     __syncthreads();
     // per key: a_j -> pj, scale dL/ds_ij -> gam, p (f - gamma + gbar) -> ff, p (e - 1) -> ee
-    for (int j = tid; j < L; j += BW_THREADS) {
+    for (int j = tid; j < L; j += HB_THREADS) {
         const double p = pj[j], e = ee[j], f = ff[j], gmj = gam[j];
         pj[j] = p * (1.0 - e);
         gam[j] = scale * p * (gmj * (1.0 - e) + (gbar + f) * e - f - kappa);
@@ -863,15 +864,53 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         ee[j] = p * (e - 1.0);
     }
     __syncthreads();
-    for (int c = tid; c < D; c += BW_THREADS) {
+    for (int c = tid; c < D; c += HB_THREADS) {
         double acc = t[c];
         for (int j = 0; j < L; ++j) acc += gam[j] * (double)__bfloat162float(Kr[j * D + c]);
         dq[(base + i) * D + c] = (float)acc;
     }
-    for (int idx = tid; idx < L * D; idx += BW_THREADS) {
-        const int j = idx / D, c = idx % D;
-        atomicAdd(dk + (base + j) * D + c, (float)(gam[j] * qd[c] + ff[j] * y[c] + ee[j] * t[c]));
-        atomicAdd(dv + (base + j) * D + c, (float)(pj[j] * gd[c]));
+    // dK_j and dV_j sum over the rows i >= j: the per-key coefficients and y, t go to the workspace and
+    // bwd_head_accum_kernel adds the rows up (one atomic per output instead of one per row and output)
+    float* hc = hcoef + ((size_t)bh * lcap + i) * 4 * lcap;
+    for (int j = tid; j < L; j += HB_THREADS) {
+        hc[j] = (float)pj[j];
+        hc[lcap + j] = (float)gam[j];
+        hc[2 * lcap + j] = (float)ff[j];
+        hc[3 * lcap + j] = (float)ee[j];
+    }
+    for (int c = tid; c < D; c += HB_THREADS) {
+        yvec[(base + i) * D + c] = (float)y[c];
+        tvec[(base + i) * D + c] = (float)t[c];
+    }
+}
+
+// dK_j += sum_{i >= j} (ds_ij q_i + c1_ij y_i + c2_ij t_i),  dV_j += sum_{i >= j} a_ij g_i  over the directly
+// solved rows i < first.  A warp per key, lanes over the columns.
+template <int D>
+__global__ void __launch_bounds__(BW_THREADS)
+bwd_head_accum_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__ dout, int dout_dtype,
+                      const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ hcoef,
+                      float* __restrict__ dk, float* __restrict__ dv, int n, int first) {
+    constexpr int CPL = D / 32;      // columns per lane
+    const int bh = blockIdx.x, lane = threadIdx.x & 31;
+    const int j = blockIdx.y * (BW_THREADS / 32) + (threadIdx.x >> 5);
+    if (j >= first) return;
+    const size_t base = (size_t)bh * n;
+    float adk[CPL] = {}, adv[CPL] = {};
+    for (int i = j; i < first; ++i) {
+        const float* hc = hcoef + ((size_t)bh * first + i) * 4 * first + j;
+        const float a = hc[0], ds = hc[first], c1 = hc[2 * first], c2 = hc[3 * first];
+#pragma unroll
+        for (int x = 0; x < CPL; ++x) {
+            const size_t e = (base + i) * D + CPL * lane + x;
+            adk[x] = fmaf(ds, __bfloat162float(q[e]), fmaf(c1, yvec[e], fmaf(c2, tvec[e], adk[x])));
+            adv[x] = fmaf(a, ld_any(dout, dout_dtype, e), adv[x]);
+        }
+    }
+#pragma unroll
+    for (int x = 0; x < CPL; ++x) {
+        atomicAdd(dk + (base + j) * D + CPL * lane + x, adk[x]);
+        atomicAdd(dv + (base + j) * D + CPL * lane + x, adv[x]);
     }
 }
 
@@ -880,8 +919,11 @@ size_t head_smem_bytes(int lcap) {
     return sizeof(double) * ((size_t)D * (D + 1) + 7 * D + 4 * lcap) + sizeof(__nv_bfloat16) * (size_t)lcap * D;
 }
 
-// workspace: kbar, h, t, y as [rows][D] fp32, then the scalar records
-size_t ws_floats(long long rows, int d) { return (size_t)rows * (4 * (size_t)d + BW_ROWSC); }
+// workspace: kbar, h, t, y as [rows][D] fp32, the scalar records, then the directly-solved rows' per-key
+// coefficients ([heads][first][4][first], first <= 2 d)
+size_t ws_floats(long long rows, int d, long long heads) {
+    return (size_t)rows * (4 * (size_t)d + BW_ROWSC) + (size_t)heads * 4 * (2 * (size_t)d) * (2 * (size_t)d);
+}
 
 template <int D>
 int launch_t(const BackwardArgs& a) {
@@ -889,12 +931,14 @@ int launch_t(const BackwardArgs& a) {
     const long long rows = (long long)a.B * a.H * a.n;
     const int BH = a.B * a.H;
     const int first = max(0, min(a.n, a.head_rows - 1));      // rows [0, first) are solved directly
-    if (a.workspace_bytes < ws_floats(rows, D) * sizeof(float) || !a.workspace) return LLA_ERR_WORKSPACE;
+    if (a.workspace_bytes < ws_floats(rows, D, BH) * sizeof(float) || !a.workspace) return LLA_ERR_WORKSPACE;
+    if (first > 2 * D) return LLA_ERR_UNSUPPORTED;
     float* kbar = static_cast<float*>(a.workspace);
     float* hvec = kbar + rows * D;
     float* tvec = hvec + rows * D;
     float* yvec = tvec + rows * D;
     float* rowsc = yvec + rows * D;
+    float* hcoef = rowsc + rows * BW_ROWSC;
     const auto* q = static_cast<const __nv_bfloat16*>(a.q);
     const auto* k = static_cast<const __nv_bfloat16*>(a.k);
     const auto* v = static_cast<const __nv_bfloat16*>(a.v);
@@ -914,8 +958,11 @@ int launch_t(const BackwardArgs& a) {
     }
     if (first > 0) {
         const dim3 gh(BH, first);
-        bwd_head_rows_kernel<D><<<gh, BW_THREADS, head_smem, hs>>>(
-            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status);
+        bwd_head_rows_kernel<D><<<gh, HB_THREADS, head_smem, hs>>>(
+            q, k, v, a.dout, a.dout_dtype, a.dq, yvec, tvec, hcoef, a.n, first, (double)a.scale, (double)a.lambda, a.status);
+        LLA_CUDA_TRY(cudaGetLastError());
+        const dim3 ga(BH, (first + BW_THREADS / 32 - 1) / (BW_THREADS / 32));
+        bwd_head_accum_kernel<D><<<ga, BW_THREADS, 0, hs>>>(q, a.dout, a.dout_dtype, yvec, tvec, hcoef, a.dk, a.dv, a.n, first);
         LLA_CUDA_TRY(cudaGetLastError());
         if (forked) LLA_CUDA_TRY(cudaEventRecord(a.join, hs));
     }
@@ -968,7 +1015,7 @@ int launch_t(const BackwardArgs& a) {
 }  // namespace
 
 size_t backward_workspace_bytes(int B, int H, int n, int d) {
-    return ws_floats((long long)B * H * n, d) * sizeof(float);
+    return ws_floats((long long)B * H * n, d, (long long)B * H) * sizeof(float);
 }
 
 int launch_backward(const BackwardArgs& a) {
