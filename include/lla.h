@@ -161,6 +161,9 @@ typedef struct lla_forward_params {
                                    existing cache): q, out, rho, stats, iters and lambda_rows then have
                                    q_rows rows per head; query row r sits at position n - q_rows + r and,
                                    when causal, sees keys 0 .. n - q_rows + r */
+    int kv_heads;   /* 0 or H: every query head has its own k, v.  Otherwise H must be a multiple of kv_heads and
+                       k, v are [B, kv_heads, n, d]: query head h reads key/value head h / (H / kv_heads)
+                       (grouped-query sharing) */
 } lla_forward_params;
 
 int lla_forward_ex(const lla_forward_params *p);
@@ -194,6 +197,7 @@ typedef struct lla_decode_params {
     void *stream;
     const float *lambda_units;  /* optional [B, H] fp32 on the device: one ridge per (sequence, head) */
     int ridge_mode;             /* lla_ridge_mode */
+    int kv_heads;   /* as in lla_forward_params: the caches are [B, kv_heads, Lmax, d] */
 } lla_decode_params;
 
 int lla_decode_ex(const lla_decode_params *p);

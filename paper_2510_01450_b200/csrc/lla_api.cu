@@ -70,6 +70,7 @@ int check_forward(const lla_forward_params* p) {
     if (!(p->lambda >= 0.f) || !isfinite(p->lambda) || !isfinite(p->scale)) return LLA_ERR_INVALID_ARG;
     if (p->ridge_mode != LLA_RIDGE_DEFINITION && p->ridge_mode != LLA_RIDGE_PRINTED) return LLA_ERR_INVALID_ARG;
     if (p->q_rows < 0 || p->q_rows > p->n) return LLA_ERR_INVALID_ARG;
+    if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
     if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535 || (p->n + 127) / 128 > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
@@ -100,6 +101,7 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.lambda_rows = p->lambda_rows;
     a.ridge_mode = p->ridge_mode;
     a.nq = p->q_rows > 0 ? p->q_rows : p->n;
+    a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     return a;
 }
 
@@ -226,6 +228,8 @@ int lla_decode_ex(const lla_decode_params* p) {
     a.stream = (cudaStream_t)p->stream;
     a.lambda_units = p->lambda_units;
     a.ridge_mode = p->ridge_mode;
+    if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
+    a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
     const int st = lla::launch_decode(a);
     if (st != LLA_OK) return st;

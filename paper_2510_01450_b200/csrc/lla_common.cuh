@@ -12,6 +12,11 @@ namespace lla {
 // ---------------------------------------------------------------------------------------------
 // Launch arguments handed from the C-ABI layer to the kernel launchers (plain pointers + sizes).
 // ---------------------------------------------------------------------------------------------
+// (batch, query head) unit -> (batch, key/value head) unit when `group` query heads share one K/V head
+__host__ __device__ __forceinline__ int kv_unit(int bh, int H, int group) {
+    return group <= 1 ? bh : (bh / H) * (H / group) + (bh % H) / group;
+}
+
 struct ForwardArgs {
     const void* q;
     const void* k;
@@ -34,6 +39,7 @@ struct ForwardArgs {
     const float* lambda_rows;   // optional per-row ridge [B, H, nq]
     int ridge_mode;             // lla_ridge_mode
     int nq;                     // query rows per head (the last nq of the n positions); nq == n: plain prefill
+    int kv_group = 1;           // query heads per key/value head: k, v are [B, H / kv_group, n, d]
     const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
 };
@@ -56,6 +62,7 @@ struct DecodeArgs {
     cudaStream_t stream;
     const float* lambda_units;  // optional per-(sequence, head) ridge [B, H]
     int ridge_mode;             // lla_ridge_mode
+    int kv_group = 1;           // query heads per key/value head: caches are [B, H / kv_group, Lmax, d]
 };
 
 // Backward pass (backward appendix): gradients of a scalar loss with respect to q, k, v given

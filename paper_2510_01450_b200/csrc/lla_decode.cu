@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(DC_THREADS)
 decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache, const TIn* __restrict__ vcache,
                       const int* __restrict__ lens, TOut* __restrict__ out, int H, int Lmax, float scale,
                       float lambda, int splits, int head_rows, float* __restrict__ parts, int* __restrict__ status,
-                      const float* __restrict__ lambda_units, int ridge_mode) {
+                      const float* __restrict__ lambda_units, int ridge_mode, int kv_group) {
     using C = DcCfg<D>;
     constexpr bool ACCURATE = sizeof(TIn) == 4;
     extern __shared__ double smem_d[];
@@ -81,8 +81,9 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     if (L < head_rows) return;   // short caches are solved directly by the fp64 kernel
     const int chunk = ((L + splits - 1) / splits + DC_BK - 1) / DC_BK * DC_BK;
     const int jbeg = part * chunk, jend = min(L, jbeg + chunk);
-    const TIn* kb = kcache + (size_t)bh * Lmax * D;
-    const TIn* vb = vcache + (size_t)bh * Lmax * D;
+    const int kvh = kv_unit(bh, H, kv_group);
+    const TIn* kb = kcache + (size_t)kvh * Lmax * D;
+    const TIn* vb = vcache + (size_t)kvh * Lmax * D;
 
     for (int e = tid; e < D; e += DC_THREADS) qs[e] = to_f32(q[(size_t)bh * D + e]);
 
@@ -290,7 +291,7 @@ int launch_t(const DecodeArgs& a) {
         dim3 grid(splits, a.B * a.H);
         k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
                                                  a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
-                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode);
+                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode, a.kv_group);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     if (splits > 1) {

@@ -203,6 +203,7 @@ struct DtParams {
     int defer;           // 1: write the moment record even for a single part; a solve kernel follows
     const float* lambda_units;   // optional per-(sequence, head) ridge
     int ridge_mode;
+    int kv_group;        // query heads per key/value head
 };
 
 template <typename TOut>
@@ -275,14 +276,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // ================================ TMA producer ================================
         if (lane == 0) {
             DT_EV_DECL(0);
+            const int kvh = kv_unit(bh, prm.H, prm.kv_group);
             for (int t = 0; t < ntile; ++t) {
                 const uint32_t s = t % DT_NST;
                 if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
                 DT_EV(1, t);
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
-                tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, bh);
-                tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, bh);
+                tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, kvh);
+                tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, kvh);
             }
         }
     } else if (warp == 5) {
@@ -743,12 +745,13 @@ int launch_t(const DecodeArgs& a) {
     if (splits > DS_MAX_SPLITS) return LLA_ERR_INVALID_ARG;
     CUtensorMap mk, mv;
     const int BH = a.B * a.H;
-    if (!make_map_bf16_64(&mk, a.kcache, BH, a.Lmax, DT_BK) || !make_map_bf16_64(&mv, a.vcache, BH, a.Lmax, DT_BK))
+    const int kvg = a.kv_group > 0 ? a.kv_group : 1;
+    if (!make_map_bf16_64(&mk, a.kcache, BH / kvg, a.Lmax, DT_BK) || !make_map_bf16_64(&mv, a.vcache, BH / kvg, a.Lmax, DT_BK))
         return LLA_ERR_CUDA;
     DtParams prm;
     prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
-    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode;
+    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode; prm.kv_group = kvg;
     prm.parts = (float*)a.workspace; prm.status = a.status;
     prm.defer = have_ws ? 1 : 0;      // with a record buffer the solve runs as its own kernel
     auto kern = decode_tc_kernel<TOut>;

@@ -61,7 +61,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                     TOut* __restrict__ out, int n, int causal, float scale, float lambda,
                     int head_rows, int max_iters, float tol, int first_tile,
                     float* __restrict__ rho_out, float* __restrict__ stats, int* __restrict__ iters_out,
-                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq) {
+                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq, int H, int kv_group) {
     constexpr int ROWS = FS_THREADS / TPR;
     constexpr int NG = D / (4 * TPR);    // float4 groups per thread (keys)
     constexpr int NGV = DV / (4 * TPR);  // float4 groups per thread (values)
@@ -80,8 +80,9 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     const int L = causal ? off + row + 1 : n;           // visible keys of this row
     const bool row_ok = row < nq && L >= head_rows;     // other rows: out of range or solved directly
     const int jend = causal ? min(n, off + r0 + ROWS) : n;   // keys this block must sweep
-    const TIn* kb = k + (size_t)bh * n * D;
-    const TIn* vb = v + (size_t)bh * n * DV;
+    const int kvh = kv_unit(bh, H, kv_group);
+    const TIn* kb = k + (size_t)kvh * n * D;
+    const TIn* vb = v + (size_t)kvh * n * DV;
 
     float4 qv[NG], kbar[NG];
 #pragma unroll
@@ -311,7 +312,7 @@ int launch_t(const ForwardArgs& a) {
     kern<<<grid, FS_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, a.causal, a.scale,
         a.lambda, a.head_rows > 0 ? a.head_rows : 0, a.max_iters, a.tol, first_tile, a.rho, a.stats,
-        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq);
+        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq, a.H, a.kv_group);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -176,6 +176,7 @@ struct TcParams {
     float scale, lambda, tol;
     float* rho;
     float* stats;
+    int H, kv_group;     // query heads per (batch), query heads per key/value head
     const float* rhs;    // solve mode: right-hand sides h_i [B, H, nq, D]; the CG then solves C_i x = h_i ...
     float* sol;          // ... and x_i is written here instead of running the output sweep
     int* iters;
@@ -275,6 +276,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mbar_expect_tx(bar(B_QFULL), Cfg::OPER_BYTES);
             for (int sub = 0; sub < KSUB; ++sub)
                 tma_load_3d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, bh);
+            const int kvh = kv_unit(bh, prm.H, prm.kv_group);
             uint32_t kit = 0;      // K blocks issued so far
             int pre = 0;           // blocks of the coming sweep already issued
             bool ok = true;
@@ -283,14 +285,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag)) { ok = false; return; }
                 mbar_expect_tx(bar(B_KVFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, &tmK, bar(B_KVFULL + s), 64 * sub, c * TC_BC, bh);
+                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, &tmK, bar(B_KVFULL + s), 64 * sub, c * TC_BC, kvh);
                 ++kit;
             };
             auto issue_v = [&](int c, uint32_t g) {
                 const uint32_t s = g % TC_NST;
                 mbar_expect_tx(bar(B_VFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, c * TC_BC, bh);
+                    tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, c * TC_BC, kvh);
             };
             for (uint32_t sweep = 0; ok; ++sweep) {
                 if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
@@ -866,8 +868,8 @@ int launch_t(const ForwardArgs& a) {
     if (tiles <= 0) return LLA_OK;
     CUtensorMap mq, mk, mv;
     const int BH = a.B * a.H;
-    if (!make_map_bf16(&mq, a.q, BH, a.nq, D, TC_BR) || !make_map_bf16(&mk, a.k, BH, a.n, D, TC_BC) ||
-        !make_map_bf16(&mv, a.v, BH, a.n, D, TC_BC))
+    if (!make_map_bf16(&mq, a.q, BH, a.nq, D, TC_BR) || !make_map_bf16(&mk, a.k, BH / a.kv_group, a.n, D, TC_BC) ||
+        !make_map_bf16(&mv, a.v, BH / a.kv_group, a.n, D, TC_BC))
         return LLA_ERR_CUDA;
     TcParams prm;
     prm.n = a.n; prm.nq = a.nq; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
@@ -875,6 +877,7 @@ int launch_t(const ForwardArgs& a) {
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
     prm.rhs = a.rhs; prm.sol = a.sol;
+    prm.H = a.H; prm.kv_group = a.kv_group > 0 ? a.kv_group : 1;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     prm.dbg = nullptr;
     prm.scratch = nullptr;

@@ -45,19 +45,20 @@ def test_struct_sizes_match_c_layout(tmp_path):
     src = tmp_path / "sz.c"
     src.write_text(
         '#include <stdio.h>\n#include <stddef.h>\n#include "lla.h"\n'
-        'int main(void) { printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(lla_forward_params), sizeof(lla_decode_params),\n'
+        'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(lla_forward_params), sizeof(lla_decode_params),\n'
         '  offsetof(lla_forward_params, lambda_rows), offsetof(lla_forward_params, ridge_mode),\n'
-        '  offsetof(lla_decode_params, lambda_units), offsetof(lla_decode_params, ridge_mode)); return 0; }\n')
+        '  offsetof(lla_decode_params, lambda_units), offsetof(lla_decode_params, ridge_mode),\n'
+        '  offsetof(lla_forward_params, kv_heads), offsetof(lla_decode_params, kv_heads)); return 0; }\n')
     exe = tmp_path / "sz"
     inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
     subprocess.run(["gcc", "-I", inc, "-o", str(exe), str(src)], check=True)
     got = [int(x) for x in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
     F, D = binding.ForwardParams, binding.DecodeParams
     assert got == [ctypes.sizeof(F), ctypes.sizeof(D), F.lambda_rows.offset, F.ridge_mode.offset,
-                   D.lambda_units.offset, D.ridge_mode.offset]
+                   D.lambda_units.offset, D.ridge_mode.offset, F.kv_heads.offset, D.kv_heads.offset]
     # 4 pointers, 5+2 ints, 2 floats, 2 ints, 1 float, 3 ints, 3+1 pointers, pointer, size_t, pointer; then the
     # ridge fields (pointer, int, tail padding)
-    assert ctypes.sizeof(F) == 4 * 8 + 15 * 4 + 4 + 7 * 8 + 8 + 8
+    assert ctypes.sizeof(F) == 4 * 8 + 15 * 4 + 4 + 7 * 8 + 8 + 8 + 8
     assert ctypes.sizeof(D) == 5 * 8 + 11 * 4 + 4 + 4 * 8 + 8 + 8
 
 

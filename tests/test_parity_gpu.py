@@ -370,3 +370,41 @@ def test_chunked_prefill_against_existing_keys(oracle, dtype, d, n, nq):
     seen = off + np.arange(nq) + 1
     it = iters.cpu().numpy()[0, 0]
     assert ((it == -1) == (seen < thr)).all()
+
+
+@pytest.mark.parametrize("dtype,d,n,H,Hkv", [("bf16", 64, 500, 4, 2), ("bf16", 128, 300, 4, 1), ("f32", 16, 150, 6, 2)])
+def test_grouped_kv_heads_forward(oracle, dtype, d, n, H, Hkv):
+    # H query heads read H / Hkv-fold shared key/value heads: the oracle sees k, v repeated per query head
+    w = inputs.CONFIGS[2].shrink(B=2, H=H, n=n, d=d, dv=d, dtype=dtype, seed=90 + d)
+    q, _, _ = inputs.make_prefill(w)
+    wk = w.shrink(H=Hkv, seed=91 + d)
+    _, k, v = inputs.make_prefill(wk)
+    ref = oracle.forward(q, np.repeat(k, H // Hkv, axis=1), np.repeat(v, H // Hkv, axis=1), w.scale, w.lam)
+    dq, dk, dv_ = dev(q, dtype), dev(k, dtype), dev(v, dtype)
+    out = torch.full((w.B, H, n, d), float("nan"), dtype=torch.float32, device="cuda")
+    L.lla_forward_ex(dq, dk, dv_, out, w.B, H, n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype], out_dtype=L.LLA_F32,
+                     kv_heads=Hkv, stream=stream_ptr())
+    torch.cuda.synchronize()
+    assert row_err(out.cpu().numpy(), ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16)
+    with pytest.raises(L.LlaError):
+        L.lla_forward_ex(dq, dk, dv_, out, w.B, H, n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                         out_dtype=L.LLA_F32, kv_heads=H - 1 if H > 2 else 3, stream=stream_ptr())
+
+
+@pytest.mark.parametrize("dtype,d,splits", [("bf16", 64, 1), ("bf16", 64, 3), ("f32", 16, 1)])
+def test_grouped_kv_heads_decode(oracle, dtype, d, splits):
+    H, Hkv = 4, 2
+    w = inputs.CONFIGS[5].shrink(B=3, H=H, n=1100, d=d, dv=d, dtype=dtype, len_min=20, len_max=1100, seed=92 + d)
+    q, _, _, lens = inputs.make_decode(w)
+    _, kc, vc, _ = inputs.make_decode(w.shrink(H=Hkv))
+    ref = oracle.decode(q, np.repeat(kc, H // Hkv, axis=1), np.repeat(vc, H // Hkv, axis=1), lens, w.scale, w.lam)
+    dq, dk, dv_ = dev(q, dtype), dev(kc, dtype), dev(vc, dtype)
+    dl = torch.from_numpy(lens).cuda()
+    out = torch.full((w.B, H, d), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = L.lla_decode_workspace_bytes(w.B, H, w.n, d, d, in_dtype=LLA_DT[dtype], splits=splits)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                    out_dtype=L.LLA_F32, splits=splits, workspace=ws, workspace_bytes=nbytes, kv_heads=Hkv,
+                    stream=stream_ptr())
+    torch.cuda.synchronize()
+    assert row_err(out.cpu().numpy(), ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16)
