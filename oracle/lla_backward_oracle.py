@@ -43,7 +43,7 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal):
         mask = torch.ones(len(rows), L, dtype=torch.bool)
     m = torch.where(mask, s, torch.full_like(s, -torch.inf)).max(dim=1).values.detach()
     w = torch.where(mask, torch.exp(s - m[:, None]), torch.zeros_like(s))
-    lam_i = lam * torch.exp(-m)
+    lam_i = (lam[rows] if torch.is_tensor(lam) else lam) * torch.exp(-m)    # one ridge per row when lam is a tensor
     Z = Kl[None, :, :] - Qr[:, None, :]                            # z_ij = k_j - q_i
     mu = torch.einsum("rj,rjc->rc", w, Z)                          # mu_i
     Sigma = torch.einsum("rj,rjc,rje->rce", w, Z, Z) + lam_i[:, None, None] * torch.eye(d, dtype=Q.dtype)
@@ -52,27 +52,33 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal):
     return (c @ Vl) / c.sum(dim=1, keepdim=True)                   # Eq. "lla"
 
 
-def backward(q, k, v, g, scale, lam, causal=True, chunk=32):
+def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False):
     """Gradients of sum_i <g_i, o_i> with respect to q, k, v.
 
     q, k: [B, H, n, d]; v, g: [B, H, n, dv]; numpy arrays (any float dtype; widened to float64).
-    Returns (dq, dk, dv) as float64 numpy arrays of the inputs' shapes.
+    Returns (dq, dk, dv) as float64 numpy arrays of the inputs' shapes; with want_dlambda also
+    dlambda [B, H, n], the derivative with respect to a ridge of its own per query row (the paper's
+    learnable per-token regularisation, Appendix on the regularisation), each evaluated at lam.
     """
     q, k, v, g = (np.asarray(a, dtype=np.float64) for a in (q, k, v, g))
     B, H, n, _ = q.shape
     dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    dlam = np.zeros((B, H, n))
     for b in range(B):
         for h in range(H):
             Q = torch.tensor(q[b, h], requires_grad=True)
             K = torch.tensor(k[b, h], requires_grad=True)
             V = torch.tensor(v[b, h], requires_grad=True)
             G = torch.tensor(g[b, h])
+            lam_rows = torch.full((n,), float(lam), dtype=torch.float64, requires_grad=True)
             for r0 in range(0, n, chunk):
                 rows = torch.arange(r0, min(n, r0 + chunk))
-                o = _forward_rows(Q, K, V, rows, float(scale), float(lam), bool(causal))
+                o = _forward_rows(Q, K, V, rows, float(scale), lam_rows if want_dlambda else float(lam), bool(causal))
                 (o * G[rows]).sum().backward()
             dq[b, h], dk[b, h], dv[b, h] = Q.grad.numpy(), K.grad.numpy(), V.grad.numpy()
-    return dq, dk, dv
+            if want_dlambda:
+                dlam[b, h] = lam_rows.grad.numpy()
+    return (dq, dk, dv, dlam) if want_dlambda else (dq, dk, dv)
 
 
 def forward(q, k, v, scale, lam, causal=True, chunk=32):

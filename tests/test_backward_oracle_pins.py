@@ -127,3 +127,20 @@ def test_backward_appendix_formulas():
     ref = _appendix_formulas(q[0, 0], k[0, 0], v[0, 0], g[0, 0], 0.45, 2e-2)
     for a, b in zip(got, ref):
         assert np.abs(a[0, 0] - b).max() <= 1e-9 * max(1.0, np.abs(b).max())
+
+
+def test_ridge_gradient_by_finite_differences_of_c_oracle():
+    # d loss / d lambda_i for a ridge of its own per query row: the C forward oracle takes per-row ridges
+    n, d, dv, scale, lam = 9, 3, 2, 0.6, 5e-2
+    q, k, v, g = _inputs(7, n, d, dv)
+    *_, dlam = bwd.backward(q, k, v, g, scale, lam, want_dlambda=True)
+    eps = 1e-6
+    for i in range(n):
+        lp = np.full((1, 1, n), lam)
+        lm = lp.copy()
+        lp[0, 0, i] += eps
+        lm[0, 0, i] -= eps
+        num = float(((fwd_c.forward(q, k, v, scale, lp) - fwd_c.forward(q, k, v, scale, lm)) * g).sum()) / (2 * eps)
+        assert abs(num - dlam[0, 0, i]) <= 1e-6 * max(1.0, abs(num)), i
+    # the first row's output is v_0 for every positive ridge: no dependence on lambda
+    assert abs(dlam[0, 0, 0]) <= 1e-12
