@@ -308,6 +308,9 @@ typedef struct lla_backward_params {
     void *stream;
     int *iters;   /* optional [B, H, n] on the device: CG iterations of the extra solve per row (rows that are
                      solved directly are left untouched) */
+    float *dlambda; /* optional [B, H, n] fp32 on the device: dL/d(lambda_i), the derivative with respect to a
+                       ridge of its own per query row (the paper's learnable regularisation), evaluated at
+                       lambda; their sum over i is the derivative with respect to the scalar */
     int impl;     /* LLA_IMPL_AUTO: pair kernel on the tensor cores where it exists (d = 64); LLA_IMPL_SIMT: CUDA cores */
 } lla_backward_params;
 

@@ -304,6 +304,7 @@ int lla_backward_ex(const lla_backward_params* p) {
     if (p->impl != LLA_IMPL_AUTO && p->impl != LLA_IMPL_SIMT) return LLA_ERR_INVALID_ARG;
     a.cuda_core_pairs = p->impl == LLA_IMPL_SIMT;
     a.iters = p->iters;
+    a.dlambda = p->dlambda;
     if (SideStream* side = side_stream()) { a.side_stream = side->stream; a.fork = side->fork; a.join = side->join; }
     ForwardArgs probe = {};
     probe.in_dtype = LLA_BF16; probe.d = p->d; probe.dv = p->d;

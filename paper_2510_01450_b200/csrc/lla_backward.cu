@@ -203,7 +203,7 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
                    const void* __restrict__ dout, int dout_dtype, const float* __restrict__ rho,
                    const float* __restrict__ stats, const float* __restrict__ kbar, const float* __restrict__ tvec,
                    float* __restrict__ yvec, float* __restrict__ rowsc, float* __restrict__ dq, int n, int first,
-                   long long rows) {
+                   long long rows, float* __restrict__ dlambda) {
     const long long row = (long long)blockIdx.x * (BW_THREADS / 32) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= rows) return;
@@ -211,7 +211,7 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
     if (i < first) return;
     const float m = stats[row * 3 + 0], omega = stats[row * 3 + 1], delta = stats[row * 3 + 2];
     const float fac = omega / delta;
-    float ky = 0.f, kt = 0.f, qt = 0.f, go = 0.f;
+    float ky = 0.f, kt = 0.f, qt = 0.f, go = 0.f, ty = 0.f;
 #pragma unroll
     for (int c = lane; c < D; c += 32) {
         const size_t e = (size_t)row * D + c;
@@ -220,6 +220,7 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
         dq[e] = tv;
         ky = fmaf(kb, yv, ky);
         kt = fmaf(kb, tv, kt);
+        ty = fmaf(tv, yv, ty);
         qt = fmaf(__bfloat162float(q[e]), tv, qt);
         go = fmaf(ld_any(dout, dout_dtype, e), ld_any(out, out_dtype, e), go);
     }
@@ -229,6 +230,7 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
         kt += __shfl_xor_sync(0xffffffffu, kt, o);
         qt += __shfl_xor_sync(0xffffffffu, qt, o);
         go += __shfl_xor_sync(0xffffffffu, go, o);
+        ty += __shfl_xor_sync(0xffffffffu, ty, o);
     }
     if (lane == 0) {
         float* rs = rowsc + row * BW_ROWSC;
@@ -237,6 +239,8 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
         rs[3] = go + kt - qt;      // kappa = g.o + t.(kbar - q)
         rs[4] = ky;
         rs[5] = kt;
+        // dL/d(lambda_i): lambda enters C as (e^{-m} / omega) lambda I and dL = t^T dC y
+        if (dlambda) dlambda[row] = __expf(-m) / omega * ty;
     }
 }
 
@@ -743,7 +747,8 @@ __global__ void __launch_bounds__(HB_THREADS)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                      float* __restrict__ dq, float* __restrict__ yvec, float* __restrict__ tvec,
-                     float* __restrict__ hcoef, int n, int lcap, double scale, double lambda, int* __restrict__ status) {
+                     float* __restrict__ hcoef, int n, int lcap, double scale, double lambda, int* __restrict__ status,
+                     float* __restrict__ dlambda) {
     constexpr int LDS = D + 1;
     extern __shared__ __align__(16) double hb_smem[];
     double* S = hb_smem;                  // D x (D + 1)
@@ -854,6 +859,11 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     double kappa = 0.0;
     for (int j = 0; j < L; ++j) kappa += pj[j] * (1.0 - ee[j]) * gam[j];      // g . o_i
     for (int c = 0; c < D; ++c) kappa += t[c] * mb[c];
+    if (dlambda && tid == 0) {
+        double ty = 0.0;
+        for (int c = 0; c < D; ++c) ty += t[c] * y[c];
+        dlambda[base + i] = (float)(exp(-m) / omega * ty);
+    }
     __syncthreads();
     // per key: a_j -> pj, scale dL/ds_ij -> gam, p (f - gamma + gbar) -> ff, p (e - 1) -> ee
     for (int j = tid; j < L; j += HB_THREADS) {
@@ -959,7 +969,7 @@ int launch_t(const BackwardArgs& a) {
     if (first > 0) {
         const dim3 gh(BH, first);
         bwd_head_rows_kernel<D><<<gh, HB_THREADS, head_smem, hs>>>(
-            q, k, v, a.dout, a.dout_dtype, a.dq, yvec, tvec, hcoef, a.n, first, (double)a.scale, (double)a.lambda, a.status);
+            q, k, v, a.dout, a.dout_dtype, a.dq, yvec, tvec, hcoef, a.n, first, (double)a.scale, (double)a.lambda, a.status, a.dlambda);
         LLA_CUDA_TRY(cudaGetLastError());
         const dim3 ga(BH, (first + BW_THREADS / 32 - 1) / (BW_THREADS / 32));
         bwd_head_accum_kernel<D><<<ga, BW_THREADS, 0, hs>>>(q, a.dout, a.dout_dtype, yvec, tvec, hcoef, a.dk, a.dv, a.n, first);
@@ -992,7 +1002,7 @@ int launch_t(const BackwardArgs& a) {
         const int rc = launch_forward_tensor(f);
         if (rc != LLA_OK) return rc;
         bwd_rowprep_kernel<D><<<(unsigned)((rows + 7) / 8), BW_THREADS, 0, a.stream>>>(
-            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, a.n, first, rows);
+            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, a.n, first, rows, a.dlambda);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     {

@@ -85,6 +85,7 @@ struct BackwardArgs {
     float tol;
     int head_rows;
     int* status;
+    float* dlambda;       // optional [B, H, n]: dL/d(lambda_i) for a ridge of its own per query row
     int* iters;           // optional [B, H, n]: CG iterations of the extra solve (rows solved directly: untouched)
     void* workspace;
     size_t workspace_bytes;

@@ -89,12 +89,16 @@ def test_backward_bench_shape_one_head(backward_oracle):
     w = inputs.CONFIGS[2].shrink(B=1, H=1, seed=260)
     q, k, v = inputs.make_prefill(w)
     g = inputs.make_upstream_grad(w)
-    ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
+    *ref, ref_dlam = backward_oracle.backward(q, k, v, g, w.scale, w.lam, want_dlambda=True)
     iters = torch.full((1, 1, w.n), -1, dtype=torch.int32, device="cuda")
-    got = run_backward(w, q, k, v, g, iters=iters)
+    dlam = torch.full((1, 1, w.n), float("nan"), dtype=torch.float32, device="cuda")
+    got = run_backward(w, q, k, v, g, iters=iters, dlambda=dlam)
     for name, a, b in zip(("dq", "dk", "dv"), got, ref):
         err = grad_err(a, b)
         assert err.max() <= TOL, (name, float(err.max()), int(err.argmax()))
+    dl = dlam.cpu().numpy().astype(np.float64).ravel()
+    assert np.abs(dl - ref_dlam.ravel()).max() <= TOL * np.abs(ref_dlam).max()
+    assert np.abs(dl - ref_dlam.ravel())[200:].max() <= TOL * np.abs(ref_dlam.ravel()[200:]).max()
     it = iters.cpu().numpy().ravel()
     assert (it[:95] == -1).all() and (it[95:] > 0).all() and it.max() <= 64
 
