@@ -198,6 +198,12 @@ typedef struct lla_decode_params {
     const float *lambda_units;  /* optional [B, H] fp32 on the device: one ridge per (sequence, head) */
     int ridge_mode;             /* lla_ridge_mode */
     int kv_heads;   /* as in lla_forward_params: the caches are [B, kv_heads, Lmax, d] */
+    /* Paged cache (block_table != NULL): kcache, vcache are [num_pages, kv heads, page_size, d] and the keys
+       j of sequence b are rows j % page_size of page block_table[b * max_pages + j / page_size]
+       (int32 on the device, entries in [0, num_pages)).  page_size must be a multiple of 128 and
+       max_pages * page_size >= Lmax; Lmax then only bounds lens.  bf16 and fp32 caches alike. */
+    const int *block_table;
+    int page_size, max_pages, num_pages;
 } lla_decode_params;
 
 int lla_decode_ex(const lla_decode_params *p);

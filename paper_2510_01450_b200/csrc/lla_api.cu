@@ -230,6 +230,12 @@ int lla_decode_ex(const lla_decode_params* p) {
     a.ridge_mode = p->ridge_mode;
     if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
+    if (p->block_table) {
+        if (p->page_size < 128 || p->page_size % 128 != 0 || p->max_pages < 1 || p->num_pages < 1 ||
+            (long long)p->max_pages * p->page_size < p->Lmax)
+            return LLA_ERR_INVALID_ARG;
+        a.paged = lla::PagedKv{p->block_table, p->page_size, p->max_pages, p->num_pages};
+    }
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
     const int st = lla::launch_decode(a);
     if (st != LLA_OK) return st;

@@ -17,6 +17,21 @@ __host__ __device__ __forceinline__ int kv_unit(int bh, int H, int group) {
     return group <= 1 ? bh : (bh / H) * (H / group) + (bh % H) / group;
 }
 
+// Paged key/value cache of the decode entry points: pages of page_size keys laid out
+// [num_pages][kv heads][page_size][d]; sequence b's keys j live in page table[b * max_pages + j / page_size].
+// table == nullptr: the contiguous [B][kv heads][Lmax][d] cache.
+struct PagedKv {
+    const int* table;
+    int page_size, max_pages, num_pages;
+};
+// row (in units of d elements) of key j of (sequence b, key/value head kvl of hkv) -- j's page must hold it
+__device__ __forceinline__ size_t kv_row(const PagedKv& pg, int b, int kvl, int hkv, int Lmax, int j) {
+    if (!pg.table) return ((size_t)b * hkv + kvl) * Lmax + j;
+    int page = pg.table[(size_t)b * pg.max_pages + j / pg.page_size];
+    page = min(max(page, 0), pg.num_pages - 1);      // a bad table entry reads the wrong page, never outside the cache
+    return ((size_t)page * hkv + kvl) * pg.page_size + j % pg.page_size;
+}
+
 struct ForwardArgs {
     const void* q;
     const void* k;
@@ -63,6 +78,7 @@ struct DecodeArgs {
     const float* lambda_units;  // optional per-(sequence, head) ridge [B, H]
     int ridge_mode;             // lla_ridge_mode
     int kv_group = 1;           // query heads per key/value head: caches are [B, H / kv_group, Lmax, d]
+    PagedKv paged = {nullptr, 0, 0, 0};
 };
 
 // Backward pass (backward appendix): gradients of a scalar loss with respect to q, k, v given

@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(DC_THREADS)
 decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache, const TIn* __restrict__ vcache,
                       const int* __restrict__ lens, TOut* __restrict__ out, int H, int Lmax, float scale,
                       float lambda, int splits, int head_rows, float* __restrict__ parts, int* __restrict__ status,
-                      const float* __restrict__ lambda_units, int ridge_mode, int kv_group) {
+                      const float* __restrict__ lambda_units, int ridge_mode, int kv_group, const PagedKv paged) {
     using C = DcCfg<D>;
     constexpr bool ACCURATE = sizeof(TIn) == 4;
     extern __shared__ double smem_d[];
@@ -81,9 +81,7 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     if (L < head_rows) return;   // short caches are solved directly by the fp64 kernel
     const int chunk = ((L + splits - 1) / splits + DC_BK - 1) / DC_BK * DC_BK;
     const int jbeg = part * chunk, jend = min(L, jbeg + chunk);
-    const int kvh = kv_unit(bh, H, kv_group);
-    const TIn* kb = kcache + (size_t)kvh * Lmax * D;
-    const TIn* vb = vcache + (size_t)kvh * Lmax * D;
+    const int hkv = H / max(kv_group, 1), kvl = (bh % H) / max(kv_group, 1);
 
     for (int e = tid; e < D; e += DC_THREADS) qs[e] = to_f32(q[(size_t)bh * D + e]);
 
@@ -99,13 +97,17 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
 
     for (int j0 = jbeg; j0 < jend; j0 += DC_BK) {
         const int jn = min(DC_BK, jend - j0);
+        // a tile never straddles a page (page_size is a multiple of the tile, j0 of the tile)
+        const size_t row0 = kv_row(paged, b, kvl, hkv, Lmax, j0);
+        const TIn* kb = kcache + row0 * D;
+        const TIn* vb = vcache + row0 * D;
         __syncthreads();
         for (int e = tid; e < DC_BK * D / 4; e += DC_THREADS) {
             const int jj = e / (D / 4), f = e - jj * (D / 4);
             float4 kv = make_float4(0.f, 0.f, 0.f, 0.f), vv = kv;
             if (jj < jn) {
-                kv = load4(kb + (size_t)(j0 + jj) * D + 4 * f);
-                vv = load4(vb + (size_t)(j0 + jj) * D + 4 * f);
+                kv = load4(kb + (size_t)jj * D + 4 * f);
+                vv = load4(vb + (size_t)jj * D + 4 * f);
             }
             reinterpret_cast<float4*>(Ks)[e] = kv;
             reinterpret_cast<float4*>(Vs)[e] = vv;
@@ -291,7 +293,7 @@ int launch_t(const DecodeArgs& a) {
         dim3 grid(splits, a.B * a.H);
         k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
                                                  a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
-                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode, a.kv_group);
+                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode, a.kv_group, a.paged);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     if (splits > 1) {

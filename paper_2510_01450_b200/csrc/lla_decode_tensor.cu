@@ -204,6 +204,7 @@ struct DtParams {
     const float* lambda_units;   // optional per-(sequence, head) ridge
     int ridge_mode;
     int kv_group;        // query heads per key/value head
+    PagedKv paged;       // table != nullptr: the tensor maps cover [num_pages * kv heads][page_size][64]
 };
 
 template <typename TOut>
@@ -276,15 +277,19 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // ================================ TMA producer ================================
         if (lane == 0) {
             DT_EV_DECL(0);
-            const int kvh = kv_unit(bh, prm.H, prm.kv_group);
+            const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group, bq = bh / prm.H;
             for (int t = 0; t < ntile; ++t) {
                 const uint32_t s = t % DT_NST;
                 if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
                 DT_EV(1, t);
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
-                tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, kvh);
-                tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jbeg + t * DT_BK, kvh);
+                // (rows per unit in the map: Lmax, or page_size for a paged cache; a tile never straddles a page)
+                const size_t row = kv_row(prm.paged, bq, kvl, hkv, prm.Lmax, jbeg + t * DT_BK);
+                const int rpu = prm.paged.table ? prm.paged.page_size : prm.Lmax;
+                const int unit = (int)(row / rpu), jrow = (int)(row % rpu);
+                tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jrow, unit);
+                tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jrow, unit);
             }
         }
     } else if (warp == 5) {
@@ -746,12 +751,14 @@ int launch_t(const DecodeArgs& a) {
     CUtensorMap mk, mv;
     const int BH = a.B * a.H;
     const int kvg = a.kv_group > 0 ? a.kv_group : 1;
-    if (!make_map_bf16_64(&mk, a.kcache, BH / kvg, a.Lmax, DT_BK) || !make_map_bf16_64(&mv, a.vcache, BH / kvg, a.Lmax, DT_BK))
+    const int map_units = a.paged.table ? a.paged.num_pages * (a.H / kvg) : BH / kvg;
+    const int map_rows = a.paged.table ? a.paged.page_size : a.Lmax;
+    if (!make_map_bf16_64(&mk, a.kcache, map_units, map_rows, DT_BK) || !make_map_bf16_64(&mv, a.vcache, map_units, map_rows, DT_BK))
         return LLA_ERR_CUDA;
     DtParams prm;
     prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
-    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode; prm.kv_group = kvg;
+    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode; prm.kv_group = kvg; prm.paged = a.paged;
     prm.parts = (float*)a.workspace; prm.status = a.status;
     prm.defer = have_ws ? 1 : 0;      // with a record buffer the solve runs as its own kernel
     auto kern = decode_tc_kernel<TOut>;

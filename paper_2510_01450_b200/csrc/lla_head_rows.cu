@@ -106,7 +106,8 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
                  TOut* __restrict__ out, int n, int rows_per_head, int causal, double scale,
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
                  int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H,
-                 const float* __restrict__ lambda_rows, int ridge_mode, int nq, int kv_group) {
+                 const float* __restrict__ lambda_rows, int ridge_mode, int nq, int kv_group,
+                 const PagedKv paged) {
     // Prefill (lens == nullptr): block (i, bh) solves row i of head bh; n is the sequence length.
     // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
     // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
@@ -133,9 +134,10 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     }
     const size_t row = lens ? (size_t)bh : (size_t)bh * nq + i;
     const TIn* qrow = q + row * D;
-    const int kvh = kv_unit(bh, H, kv_group);
-    const TIn* kb = k + (size_t)kvh * n * D;
-    const TIn* vb = v + (size_t)kvh * n * DV;
+    // (decode over a paged cache: the at most lcap <= page_size keys of a directly-solved unit sit in its first page)
+    const size_t kvrow = kv_row(paged, bh / H, (bh % H) / max(kv_group, 1), H / max(kv_group, 1), n, 0);
+    const TIn* kb = k + kvrow * D;
+    const TIn* vb = v + kvrow * DV;
 
     HR_T0;
     for (int c = tid; c < D; c += HR_THREADS) qd[c] = (double)to_f32(qrow[c]);
@@ -366,7 +368,7 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
         (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H, a.lambda_rows,
-        a.ridge_mode, a.nq, a.kv_group);
+        a.ridge_mode, a.nq, a.kv_group, PagedKv{nullptr, 0, 0, 0});
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -382,7 +384,7 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
         (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H, a.lambda_units,
-        a.ridge_mode, 1, a.kv_group);
+        a.ridge_mode, 1, a.kv_group, a.paged);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -39,43 +39,27 @@ def test_version_and_status_strings(lib):
     assert binding.status_string(99) == "unknown status"
 
 
-def test_struct_sizes_match_c_layout(tmp_path):
-    # the ctypes mirrors against what a C compiler makes of include/lla.h
+def test_struct_layouts_match_c(tmp_path):
+    # every field offset and the size of the three parameter structs: the ctypes mirrors against what a C
+    # compiler makes of include/lla.h
     import subprocess
-    src = tmp_path / "sz.c"
-    src.write_text(
-        '#include <stdio.h>\n#include <stddef.h>\n#include "lla.h"\n'
-        'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(lla_forward_params), sizeof(lla_decode_params),\n'
-        '  offsetof(lla_forward_params, lambda_rows), offsetof(lla_forward_params, ridge_mode),\n'
-        '  offsetof(lla_decode_params, lambda_units), offsetof(lla_decode_params, ridge_mode),\n'
-        '  offsetof(lla_forward_params, kv_heads), offsetof(lla_decode_params, kv_heads)); return 0; }\n')
-    exe = tmp_path / "sz"
-    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
-    subprocess.run(["gcc", "-I", inc, "-o", str(exe), str(src)], check=True)
-    got = [int(x) for x in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
-    F, D = binding.ForwardParams, binding.DecodeParams
-    assert got == [ctypes.sizeof(F), ctypes.sizeof(D), F.lambda_rows.offset, F.ridge_mode.offset,
-                   D.lambda_units.offset, D.ridge_mode.offset, F.kv_heads.offset, D.kv_heads.offset]
-    # 4 pointers, 5+2 ints, 2 floats, 2 ints, 1 float, 3 ints, 3+1 pointers, pointer, size_t, pointer; then the
-    # ridge fields (pointer, int, tail padding)
-    assert ctypes.sizeof(F) == 4 * 8 + 15 * 4 + 4 + 7 * 8 + 8 + 8 + 8
-    assert ctypes.sizeof(D) == 5 * 8 + 11 * 4 + 4 + 4 * 8 + 8 + 8
-
-
-def test_backward_struct_matches_c_layout(tmp_path):
-    import subprocess
-    fields = [name for name, _ in binding.BackwardParams._fields_]
-    cnames = ["lambda" if f == "lambda_" else f for f in fields]
-    src = tmp_path / "bw.c"
-    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "lla.h"\nint main(void) {\n'
-                   '  printf("%zu", sizeof(lla_backward_params));\n'
-                   + "".join(f'  printf(" %zu", offsetof(lla_backward_params, {c}));\n' for c in cnames)
+    structs = (("lla_forward_params", binding.ForwardParams), ("lla_decode_params", binding.DecodeParams),
+               ("lla_backward_params", binding.BackwardParams))
+    lines = []
+    for cname, cls in structs:
+        lines.append(f'  printf("%zu", sizeof({cname}));\n')
+        for f, _ in cls._fields_:
+            lines.append(f'  printf(" %zu", offsetof({cname}, {"lambda" if f == "lambda_" else f}));\n')
+        lines.append('  printf("\\n");\n')
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "lla.h"\nint main(void) {\n' + "".join(lines)
                    + "  return 0; }\n")
-    exe = tmp_path / "bw"
+    exe = tmp_path / "layout"
     subprocess.run(["gcc", "-I", str(ROOT / "include"), "-o", str(exe), str(src)], check=True)
-    got = [int(x) for x in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
-    B = binding.BackwardParams
-    assert got == [ctypes.sizeof(B)] + [getattr(B, f).offset for f in fields]
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.strip().splitlines()
+    for (cname, cls), line in zip(structs, out):
+        got = [int(x) for x in line.split()]
+        assert got == [ctypes.sizeof(cls)] + [getattr(cls, f).offset for f, _ in cls._fields_], cname
 
 
 def test_argument_validation_without_device(lib):

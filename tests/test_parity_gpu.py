@@ -408,3 +408,50 @@ def test_grouped_kv_heads_decode(oracle, dtype, d, splits):
                     stream=stream_ptr())
     torch.cuda.synchronize()
     assert row_err(out.cpu().numpy(), ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16)
+
+
+def _to_pages(cache, lens, page_size, rng):
+    """[B, Hkv, Lmax, d] contiguous cache -> ([num_pages, Hkv, page_size, d] pages in a random order, block table)."""
+    B, Hkv, Lmax, d = cache.shape
+    max_pages = (Lmax + page_size - 1) // page_size
+    need = [(int(l) + page_size - 1) // page_size for l in lens]
+    num_pages = sum(need) + 3                       # a few pages nobody owns
+    order = rng.permutation(num_pages)
+    pages = np.zeros((num_pages, Hkv, page_size, d), dtype=cache.dtype)
+    table = np.full((B, max_pages), -1, dtype=np.int32)          # unused entries are never read
+    nxt = 0
+    for b in range(B):
+        for pi in range(need[b]):
+            pg = int(order[nxt]); nxt += 1
+            lo, hi = pi * page_size, min(Lmax, (pi + 1) * page_size)
+            pages[pg, :, : hi - lo] = cache[b, :, lo:hi]
+            table[b, pi] = pg
+    return pages, table, max_pages, num_pages
+
+
+@pytest.mark.parametrize("dtype,d,splits,page_size,Hkv", [("bf16", 64, 1, 128, 4), ("bf16", 64, 3, 256, 2),
+                                                          ("f32", 16, 1, 128, 4), ("f32", 16, 2, 128, 2)])
+def test_paged_cache_decode(oracle, dtype, d, splits, page_size, Hkv):
+    H = 4
+    w = inputs.CONFIGS[5].shrink(B=4, H=H, n=1200, d=d, dv=d, dtype=dtype, len_min=10, len_max=1200, seed=95 + d)
+    q, _, _, lens = inputs.make_decode(w)
+    _, kc, vc, _ = inputs.make_decode(w.shrink(H=Hkv))
+    ref = oracle.decode(q, np.repeat(kc, H // Hkv, axis=1), np.repeat(vc, H // Hkv, axis=1), lens, w.scale, w.lam)
+    rng = np.random.default_rng(96)
+    kp, table, max_pages, num_pages = _to_pages(kc, lens, page_size, rng)
+    vp, table_v, _, _ = _to_pages(vc, lens, page_size, np.random.default_rng(96))
+    assert (table == table_v).all()
+    dq, dk, dv_ = dev(q, dtype), dev(kp, dtype), dev(vp, dtype)
+    dl, dt = torch.from_numpy(lens).cuda(), torch.from_numpy(table).cuda()
+    out = torch.full((w.B, H, d), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = L.lla_decode_workspace_bytes(w.B, H, w.n, d, d, in_dtype=LLA_DT[dtype], splits=splits)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                    out_dtype=L.LLA_F32, splits=splits, workspace=ws, workspace_bytes=nbytes, kv_heads=Hkv,
+                    block_table=dt, page_size=page_size, max_pages=max_pages, num_pages=num_pages, stream=stream_ptr())
+    torch.cuda.synchronize()
+    assert row_err(out.cpu().numpy(), ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16)
+    with pytest.raises(L.LlaError):
+        L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                        out_dtype=L.LLA_F32, block_table=dt, page_size=96, max_pages=max_pages, num_pages=num_pages,
+                        stream=stream_ptr())
