@@ -277,17 +277,23 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // ================================ TMA producer ================================
         if (lane == 0) {
             DT_EV_DECL(0);
-            const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group, bq = bh / prm.H;
+            // K/V unit and row of a tile in the tensor map: (batch, key/value head) and the key index, or for a
+            // paged cache (page, key/value head) and the row inside the page (a tile never straddles a page)
+            const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group;
+            const int kvh = (bh / prm.H) * hkv + kvl;
+            const int* table = prm.paged.table ? prm.paged.table + (size_t)(bh / prm.H) * prm.paged.max_pages : nullptr;
             for (int t = 0; t < ntile; ++t) {
                 const uint32_t s = t % DT_NST;
                 if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
                 DT_EV(1, t);
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
-                // (rows per unit in the map: Lmax, or page_size for a paged cache; a tile never straddles a page)
-                const size_t row = kv_row(prm.paged, bq, kvl, hkv, prm.Lmax, jbeg + t * DT_BK);
-                const int rpu = prm.paged.table ? prm.paged.page_size : prm.Lmax;
-                const int unit = (int)(row / rpu), jrow = (int)(row % rpu);
+                int unit = kvh, jrow = jbeg + t * DT_BK;
+                if (table) {
+                    const int page = min(max(table[jrow / prm.paged.page_size], 0), prm.paged.num_pages - 1);
+                    unit = page * hkv + kvl;
+                    jrow %= prm.paged.page_size;
+                }
                 tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jrow, unit);
                 tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jrow, unit);
             }

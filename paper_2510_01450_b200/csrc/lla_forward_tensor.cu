@@ -254,6 +254,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_init(bar(B_CTL), TC_COMPUTE / 32);
         misc[1] = SW_MAX;
         misc[2] = 0;
+        misc[3] = kv_unit(bh, prm.H, prm.kv_group);   // worked out here: in the producer's own path it delays the first loads
         fence_barrier_init();
     }
     if (warp == 8) {   // TMEM allocation by one full warp; the base address lands in shared memory
@@ -276,7 +277,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mbar_expect_tx(bar(B_QFULL), Cfg::OPER_BYTES);
             for (int sub = 0; sub < KSUB; ++sub)
                 tma_load_3d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, bh);
-            const int kvh = kv_unit(bh, prm.H, prm.kv_group);
+            const int kvh = misc[3];
             uint32_t kit = 0;      // K blocks issued so far
             int pre = 0;           // blocks of the coming sweep already issued
             bool ok = true;
