@@ -741,14 +741,13 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
-constexpr int HB_THREADS = 128;   // four or five blocks per SM hide each other's factorisation latency
+constexpr int HB_THREADS = 256;
 template <int D>
-__global__ void __launch_bounds__(HB_THREADS)
+__global__ void __launch_bounds__(HB_THREADS, D == 64 ? 3 : 1)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
-                     float* __restrict__ dq, float* __restrict__ yvec, float* __restrict__ tvec,
-                     float* __restrict__ hcoef, int n, int lcap, double scale, double lambda, int* __restrict__ status,
-                     float* __restrict__ dlambda) {
+                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int lcap,
+                     double scale, double lambda, int* __restrict__ status, float* __restrict__ dlambda) {
     constexpr int LDS = D + 1;
     extern __shared__ __align__(16) double hb_smem[];
     double* S = hb_smem;                  // D x (D + 1)
@@ -794,7 +793,8 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     __syncthreads();
     double omega = 0.0;
     for (int j = 0; j < L; ++j) omega += pj[j];
-    const double eps = lambda * exp(-m) / omega;
+    const double em_om = exp(-m) / omega;     // d(ridge of C) / d(lambda)
+    const double eps = lambda * em_om;
     __syncthreads();
     for (int j = tid; j < L; j += HB_THREADS) pj[j] /= omega;
     __syncthreads();
@@ -858,12 +858,12 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     __syncthreads();
     double kappa = 0.0;
     for (int j = 0; j < L; ++j) kappa += pj[j] * (1.0 - ee[j]) * gam[j];      // g . o_i
-    for (int c = 0; c < D; ++c) kappa += t[c] * mb[c];
-    if (dlambda && tid == 0) {
-        double ty = 0.0;
-        for (int c = 0; c < D; ++c) ty += t[c] * y[c];
-        dlambda[base + i] = (float)(exp(-m) / omega * ty);
+    double ty = 0.0;
+    for (int c = 0; c < D; ++c) {
+        kappa += t[c] * mb[c];
+        ty += t[c] * y[c];
     }
+    if (dlambda && tid == 0) dlambda[base + i] = (float)(em_om * ty);     // dL = t^T dC y
     __syncthreads();
     // per key: a_j -> pj, scale dL/ds_ij -> gam, p (f - gamma + gbar) -> ff, p (e - 1) -> ee
     for (int j = tid; j < L; j += HB_THREADS) {
@@ -879,48 +879,12 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         for (int j = 0; j < L; ++j) acc += gam[j] * (double)__bfloat162float(Kr[j * D + c]);
         dq[(base + i) * D + c] = (float)acc;
     }
-    // dK_j and dV_j sum over the rows i >= j: the per-key coefficients and y, t go to the workspace and
-    // bwd_head_accum_kernel adds the rows up (one atomic per output instead of one per row and output)
-    float* hc = hcoef + ((size_t)bh * lcap + i) * 4 * lcap;
-    for (int j = tid; j < L; j += HB_THREADS) {
-        hc[j] = (float)pj[j];
-        hc[lcap + j] = (float)gam[j];
-        hc[2 * lcap + j] = (float)ff[j];
-        hc[3 * lcap + j] = (float)ee[j];
-    }
-    for (int c = tid; c < D; c += HB_THREADS) {
-        yvec[(base + i) * D + c] = (float)y[c];
-        tvec[(base + i) * D + c] = (float)t[c];
-    }
-}
-
-// dK_j += sum_{i >= j} (ds_ij q_i + c1_ij y_i + c2_ij t_i),  dV_j += sum_{i >= j} a_ij g_i  over the directly
-// solved rows i < first.  A warp per key, lanes over the columns.
-template <int D>
-__global__ void __launch_bounds__(BW_THREADS)
-bwd_head_accum_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__ dout, int dout_dtype,
-                      const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ hcoef,
-                      float* __restrict__ dk, float* __restrict__ dv, int n, int first) {
-    constexpr int CPL = D / 32;      // columns per lane
-    const int bh = blockIdx.x, lane = threadIdx.x & 31;
-    const int j = blockIdx.y * (BW_THREADS / 32) + (threadIdx.x >> 5);
-    if (j >= first) return;
-    const size_t base = (size_t)bh * n;
-    float adk[CPL] = {}, adv[CPL] = {};
-    for (int i = j; i < first; ++i) {
-        const float* hc = hcoef + ((size_t)bh * first + i) * 4 * first + j;
-        const float a = hc[0], ds = hc[first], c1 = hc[2 * first], c2 = hc[3 * first];
-#pragma unroll
-        for (int x = 0; x < CPL; ++x) {
-            const size_t e = (base + i) * D + CPL * lane + x;
-            adk[x] = fmaf(ds, __bfloat162float(q[e]), fmaf(c1, yvec[e], fmaf(c2, tvec[e], adk[x])));
-            adv[x] = fmaf(a, ld_any(dout, dout_dtype, e), adv[x]);
-        }
-    }
-#pragma unroll
-    for (int x = 0; x < CPL; ++x) {
-        atomicAdd(dk + (base + j) * D + CPL * lane + x, adk[x]);
-        atomicAdd(dv + (base + j) * D + CPL * lane + x, adv[x]);
+    // (one atomic per row and output: a version that wrote the per-key coefficients out and summed the rows in
+    //  a second kernel was slower, the sum's serial loop costing more than the atomics it saved)
+    for (int idx = tid; idx < L * D; idx += HB_THREADS) {
+        const int j = idx / D, c = idx % D;
+        atomicAdd(dk + (base + j) * D + c, (float)(gam[j] * qd[c] + ff[j] * y[c] + ee[j] * t[c]));
+        atomicAdd(dv + (base + j) * D + c, (float)(pj[j] * gd[c]));
     }
 }
 
@@ -929,10 +893,10 @@ size_t head_smem_bytes(int lcap) {
     return sizeof(double) * ((size_t)D * (D + 1) + 7 * D + 4 * lcap) + sizeof(__nv_bfloat16) * (size_t)lcap * D;
 }
 
-// workspace: kbar, h, t, y as [rows][D] fp32, the scalar records, then the directly-solved rows' per-key
-// coefficients ([heads][first][4][first], first <= 2 d)
+// workspace: kbar, h, t, y as [rows][D] fp32, then the scalar records
 size_t ws_floats(long long rows, int d, long long heads) {
-    return (size_t)rows * (4 * (size_t)d + BW_ROWSC) + (size_t)heads * 4 * (2 * (size_t)d) * (2 * (size_t)d);
+    (void)heads;
+    return (size_t)rows * (4 * (size_t)d + BW_ROWSC);
 }
 
 template <int D>
@@ -948,7 +912,6 @@ int launch_t(const BackwardArgs& a) {
     float* tvec = hvec + rows * D;
     float* yvec = tvec + rows * D;
     float* rowsc = yvec + rows * D;
-    float* hcoef = rowsc + rows * BW_ROWSC;
     const auto* q = static_cast<const __nv_bfloat16*>(a.q);
     const auto* k = static_cast<const __nv_bfloat16*>(a.k);
     const auto* v = static_cast<const __nv_bfloat16*>(a.v);
@@ -969,10 +932,7 @@ int launch_t(const BackwardArgs& a) {
     if (first > 0) {
         const dim3 gh(BH, first);
         bwd_head_rows_kernel<D><<<gh, HB_THREADS, head_smem, hs>>>(
-            q, k, v, a.dout, a.dout_dtype, a.dq, yvec, tvec, hcoef, a.n, first, (double)a.scale, (double)a.lambda, a.status, a.dlambda);
-        LLA_CUDA_TRY(cudaGetLastError());
-        const dim3 ga(BH, (first + BW_THREADS / 32 - 1) / (BW_THREADS / 32));
-        bwd_head_accum_kernel<D><<<ga, BW_THREADS, 0, hs>>>(q, a.dout, a.dout_dtype, yvec, tvec, hcoef, a.dk, a.dv, a.n, first);
+            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status, a.dlambda);
         LLA_CUDA_TRY(cudaGetLastError());
         if (forked) LLA_CUDA_TRY(cudaEventRecord(a.join, hs));
     }
