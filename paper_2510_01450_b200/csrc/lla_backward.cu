@@ -741,9 +741,9 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
-constexpr int HB_THREADS = 256;
+constexpr int HB_THREADS = 128;   // four blocks per SM hide each other's factorisation latency
 template <int D>
-__global__ void __launch_bounds__(HB_THREADS, D == 64 ? 3 : 1)
+__global__ void __launch_bounds__(HB_THREADS, D == 64 ? 4 : 1)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                      float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int lcap,

@@ -103,6 +103,21 @@ def test_backward_bench_shape_one_head(backward_oracle):
     assert (it[:95] == -1).all() and (it[95:] > 0).all() and it.max() <= 64
 
 
+def test_backward_full_bench_workload_sampled_heads(backward_oracle):
+    # the whole bench workload (4 x 8 heads, n = 1024) in the launch configuration bench.py times; the oracle
+    # checks two of the 32 heads (heads are independent, so it is given those heads' inputs alone)
+    w = inputs.CONFIGS[2]
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    got = run_backward(w, q, k, v, g)
+    for b, h in ((0, 0), (w.B - 1, w.H - 1)):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        ref = backward_oracle.backward(q[sl], k[sl], v[sl], g[sl], w.scale, w.lam)
+        for name, a, r in zip(("dq", "dk", "dv"), got, ref):
+            err = grad_err(a[sl], r)
+            assert err.max() <= TOL, (name, b, h, float(err.max()))
+
+
 def test_backward_argument_checks():
     ok = 0x1000
     with pytest.raises(L.LlaError) as e:
