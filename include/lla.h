@@ -317,7 +317,9 @@ typedef struct lla_backward_params {
     float *dlambda; /* optional [B, H, n] fp32 on the device: dL/d(lambda_i), the derivative with respect to a
                        ridge of its own per query row (the paper's learnable regularisation), evaluated at
                        lambda; their sum over i is the derivative with respect to the scalar */
-    int impl;     /* LLA_IMPL_AUTO: pair kernel on the tensor cores where it exists (d = 64); LLA_IMPL_SIMT: CUDA cores */
+    int impl;     /* LLA_IMPL_AUTO: moments and pair kernels on the tensor cores; LLA_IMPL_SIMT: on the CUDA cores */
+    int kv_heads; /* as in lla_forward_params: k, v, dk, dv are [B, kv_heads, n, d]; a key/value head's gradient
+                     sums over the query heads that read it */
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -311,6 +311,8 @@ int lla_backward_ex(const lla_backward_params* p) {
     a.cuda_core_pairs = p->impl == LLA_IMPL_SIMT;
     a.iters = p->iters;
     a.dlambda = p->dlambda;
+    if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
+    a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     if (SideStream* side = side_stream()) { a.side_stream = side->stream; a.fork = side->fork; a.join = side->join; }
     ForwardArgs probe = {};
     probe.in_dtype = LLA_BF16; probe.d = p->d; probe.dv = p->d;

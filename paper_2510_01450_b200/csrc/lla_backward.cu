@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(BW_THREADS)
 bwd_moments_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                    const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                    const float* __restrict__ stats, float* __restrict__ kbar, float* __restrict__ hvec,
-                   float* __restrict__ rowsc, int n, int first, float scale) {
+                   float* __restrict__ rowsc, int n, int first, float scale, int H, int kv_group) {
     using C = BwCfg<D>;
     constexpr int BI = C::BI, LD = C::LD, RI = C::RI, CU = C::CU, LDT = C::LDT;
     extern __shared__ __align__(16) float bw_smem[];
@@ -111,6 +111,7 @@ bwd_moments_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
     const int i0 = tile * BI;
     if (i0 + BI <= first) return;                      // every row of the tile is solved directly
     const size_t base = (size_t)bh * n;
+    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
     const int nrow = min(BI, n - i0);
     load_tile<D>(Qs, q, LLA_BF16, base + i0, BI, nrow);
     load_tile<D>(Gs, dout, dout_dtype, base + i0, BI, nrow);
@@ -128,8 +129,8 @@ bwd_moments_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
     for (int jt = 0; jt < jt_end; ++jt) {
         const int j0 = jt * BW_BJ;
         __syncthreads();
-        load_tile<D>(Ks, k, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
-        load_tile<D>(Vs, v, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
+        load_tile<D>(Ks, k, LLA_BF16, kvbase + j0, BW_BJ, min(BW_BJ, n - j0));
+        load_tile<D>(Vs, v, LLA_BF16, kvbase + j0, BW_BJ, min(BW_BJ, n - j0));
         __syncthreads();
         float s[RI][4] = {}, gm[RI][4] = {};
 #pragma unroll 2
@@ -253,7 +254,7 @@ __global__ void __launch_bounds__(BW_THREADS)
 bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                  const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                  const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ rowsc,
-                 float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale) {
+                 float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale, int H, int kv_group) {
     using C = BwCfg<D>;
     constexpr int BI = C::BI, LD = C::LD, RI = C::RI, CU = C::CU, LDT = C::LDT, LDP = BW_LDP;
     extern __shared__ __align__(16) float bw_smem[];
@@ -271,8 +272,9 @@ bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
     const int bh = blockIdx.x;
     const int j0 = blockIdx.y * BW_BJ;    // key tile 0 sees the most query tiles and starts first (heads fastest)
     const size_t base = (size_t)bh * n;
-    load_tile<D>(Ks, k, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
-    load_tile<D>(Vs, v, LLA_BF16, base + j0, BW_BJ, min(BW_BJ, n - j0));
+    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
+    load_tile<D>(Ks, k, LLA_BF16, kvbase + j0, BW_BJ, min(BW_BJ, n - j0));
+    load_tile<D>(Vs, v, LLA_BF16, kvbase + j0, BW_BJ, min(BW_BJ, n - j0));
     float adk[4][4 * CU] = {}, adv[4][4 * CU] = {};
     const int it0 = max(j0, first) / BI, it1 = (n + BI - 1) / BI;
     for (int it = it0; it < it1; ++it) {
@@ -357,8 +359,8 @@ bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
             // (added, not stored: the directly-solved rows add their share from another stream)
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
-                atomicAdd(dk + (base + gj) * D + c + x, adk[r][4 * u + x]);
-                atomicAdd(dv + (base + gj) * D + c + x, adv[r][4 * u + x]);
+                atomicAdd(dk + (kvbase + gj) * D + c + x, adk[r][4 * u + x]);
+                atomicAdd(dv + (kvbase + gj) * D + c + x, adv[r][4 * u + x]);
             }
         }
     }
@@ -441,7 +443,7 @@ __global__ void __launch_bounds__(MmCfg<D>::THREADS, D == 64 ? 2 : 1)
 bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                      const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ rowsc,
-                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale) {
+                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale, int H, int kv_group) {
     constexpr int LDB = MmCfg<D>::LDB, MM_TILE = MmCfg<D>::TILE, MM_THREADS = MmCfg<D>::THREADS, KS = MmCfg<D>::KS;
     extern __shared__ __align__(16) unsigned char mm_smem[];
     __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(mm_smem);
@@ -462,8 +464,9 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int bh = blockIdx.x;
     const int j0 = blockIdx.y * 64;
     const size_t base = (size_t)bh * n;
-    mm_load_bf16<D>(Ks, k, base + j0, min(64, n - j0));
-    mm_load_bf16<D>(Vs, v, base + j0, min(64, n - j0));
+    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
+    mm_load_bf16<D>(Ks, k, kvbase + j0, min(64, n - j0));
+    mm_load_bf16<D>(Vs, v, kvbase + j0, min(64, n - j0));
     // ldmatrix lane offsets: (rows +8 by bit 3, columns +8 by bit 4) and (columns +8 by bit 3, rows +8 by bit 4)
     const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
     const int offA = (l7 + 8 * b3) * LDB + 8 * b4;     // A operand, or B^T-stored operand read with .trans
@@ -609,7 +612,7 @@ bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         for (int x = 0; x < 4; ++x) {
             const int gj = j0 + kr0 + g + 8 * (x >> 1);
             if (gj >= n) continue;
-            const size_t e = (base + gj) * D + 64 * cg + 8 * nb + 2 * t4 + (x & 1);
+            const size_t e = (kvbase + gj) * D + 64 * cg + 8 * nb + 2 * t4 + (x & 1);
             atomicAdd(dk + e, adk[nb][x]);
             atomicAdd(dv + e, adv[nb][x]);
         }
@@ -623,7 +626,7 @@ __global__ void __launch_bounds__(MmCfg<D>::THREADS, D == 64 ? 2 : 1)
 bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                        const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                        const float* __restrict__ stats, float* __restrict__ kbar, float* __restrict__ hvec,
-                       float* __restrict__ rowsc, int n, int first, float scale) {
+                       float* __restrict__ rowsc, int n, int first, float scale, int H, int kv_group) {
     constexpr int LDB = MmCfg<D>::LDB, MM_TILE = MmCfg<D>::TILE, KS = MmCfg<D>::KS;
     extern __shared__ __align__(16) unsigned char mm_smem[];
     __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(mm_smem);
@@ -639,6 +642,7 @@ bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
     const int i0 = tile * 64;
     if (i0 + 64 <= first) return;
     const size_t base = (size_t)bh * n;
+    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
     const int nrow = min(64, n - i0);
     mm_load_bf16<D>(Qs, q, base + i0, nrow);
     mm_load_split<D>(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
@@ -659,8 +663,8 @@ bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
     for (int jt = 0; jt < jt_end; ++jt) {
         const int j0 = jt * 64;
         __syncthreads();
-        mm_load_bf16<D>(Ks, k, base + j0, min(64, n - j0));
-        mm_load_bf16<D>(Vs, v, base + j0, min(64, n - j0));
+        mm_load_bf16<D>(Ks, k, kvbase + j0, min(64, n - j0));
+        mm_load_bf16<D>(Vs, v, kvbase + j0, min(64, n - j0));
         __syncthreads();
         float s[8][4] = {}, gm[8][4] = {};
 #pragma unroll
@@ -747,7 +751,7 @@ __global__ void __launch_bounds__(HB_THREADS, D == 64 ? 4 : 1)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                      float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int lcap,
-                     double scale, double lambda, int* __restrict__ status, float* __restrict__ dlambda) {
+                     double scale, double lambda, int* __restrict__ status, float* __restrict__ dlambda, int H, int kv_group) {
     constexpr int LDS = D + 1;
     extern __shared__ __align__(16) double hb_smem[];
     double* S = hb_smem;                  // D x (D + 1)
@@ -767,19 +771,20 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int i = gridDim.y - 1 - blockIdx.y;       // rows with the most keys first
     const int L = i + 1;
     const size_t base = (size_t)bh * n;
+    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
     for (int c = tid; c < D; c += HB_THREADS) {
         qd[c] = (double)__bfloat162float(q[(base + i) * D + c]);
         gd[c] = (double)ld_any(dout, dout_dtype, (base + i) * D + c);
     }
     for (int idx = tid; idx < L * (D / 8); idx += HB_THREADS)
-        reinterpret_cast<uint4*>(Kr)[idx] = reinterpret_cast<const uint4*>(k + base * D)[idx];
+        reinterpret_cast<uint4*>(Kr)[idx] = reinterpret_cast<const uint4*>(k + kvbase * D)[idx];
     __syncthreads();
     // scores and gamma_j = g . v_j: a warp per key
     for (int j = warp; j < L; j += HB_THREADS / 32) {
         double s = 0.0, gv = 0.0;
         for (int c = lane; c < D; c += 32) {
             s += qd[c] * (double)__bfloat162float(Kr[j * D + c]);
-            gv += gd[c] * (double)__bfloat162float(v[(base + j) * D + c]);
+            gv += gd[c] * (double)__bfloat162float(v[(kvbase + j) * D + c]);
         }
         s = warp_sum(s);
         gv = warp_sum(gv);
@@ -883,8 +888,8 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     //  a second kernel was slower, the sum's serial loop costing more than the atomics it saved)
     for (int idx = tid; idx < L * D; idx += HB_THREADS) {
         const int j = idx / D, c = idx % D;
-        atomicAdd(dk + (base + j) * D + c, (float)(gam[j] * qd[c] + ff[j] * y[c] + ee[j] * t[c]));
-        atomicAdd(dv + (base + j) * D + c, (float)(pj[j] * gd[c]));
+        atomicAdd(dk + (kvbase + j) * D + c, (float)(gam[j] * qd[c] + ff[j] * y[c] + ee[j] * t[c]));
+        atomicAdd(dv + (kvbase + j) * D + c, (float)(pj[j] * gd[c]));
     }
 }
 
@@ -905,6 +910,8 @@ int launch_t(const BackwardArgs& a) {
     const long long rows = (long long)a.B * a.H * a.n;
     const int BH = a.B * a.H;
     const int first = max(0, min(a.n, a.head_rows - 1));      // rows [0, first) are solved directly
+    const int kvg = a.kv_group > 0 ? a.kv_group : 1;
+    const long long kvrows = rows / kvg;                       // rows of k, v, dk, dv
     if (a.workspace_bytes < ws_floats(rows, D, BH) * sizeof(float) || !a.workspace) return LLA_ERR_WORKSPACE;
     if (first > 2 * D) return LLA_ERR_UNSUPPORTED;
     float* kbar = static_cast<float*>(a.workspace);
@@ -920,8 +927,8 @@ int launch_t(const BackwardArgs& a) {
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::MOMENTS_SMEM));
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::PAIRS_SMEM));
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_head_rows_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem));
-    LLA_CUDA_TRY(cudaMemsetAsync(a.dk, 0, sizeof(float) * rows * D, a.stream));
-    LLA_CUDA_TRY(cudaMemsetAsync(a.dv, 0, sizeof(float) * rows * D, a.stream));
+    LLA_CUDA_TRY(cudaMemsetAsync(a.dk, 0, sizeof(float) * kvrows * D, a.stream));
+    LLA_CUDA_TRY(cudaMemsetAsync(a.dv, 0, sizeof(float) * kvrows * D, a.stream));
     // the directly-solved rows depend on nothing the other kernels make: they run beside them on the side stream
     const bool forked = first > 0 && a.side_stream != nullptr;
     cudaStream_t hs = forked ? a.side_stream : a.stream;
@@ -932,7 +939,7 @@ int launch_t(const BackwardArgs& a) {
     if (first > 0) {
         const dim3 gh(BH, first);
         bwd_head_rows_kernel<D><<<gh, HB_THREADS, head_smem, hs>>>(
-            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status, a.dlambda);
+            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status, a.dlambda, a.H, kvg);
         LLA_CUDA_TRY(cudaGetLastError());
         if (forked) LLA_CUDA_TRY(cudaEventRecord(a.join, hs));
     }
@@ -943,10 +950,10 @@ int launch_t(const BackwardArgs& a) {
             const dim3 gm(BH, (a.n + 63) / 64);
             LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::MOMENTS_SMEM));
             bwd_moments_mma_kernel<D><<<gm, M::THREADS, M::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
-                                                                               rowsc, a.n, first, a.scale);
+                                                                               rowsc, a.n, first, a.scale, a.H, kvg);
         } else {
             bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
-                                                                              rowsc, a.n, first, a.scale);
+                                                                              rowsc, a.n, first, a.scale, a.H, kvg);
         }
         LLA_CUDA_TRY(cudaGetLastError());
         // C_i t_i = h_i for the iterative rows: the forward's tensor-core CG with h as right-hand side
@@ -957,7 +964,7 @@ int launch_t(const BackwardArgs& a) {
         f.scale = a.scale; f.lambda = a.lambda; f.causal = 1;
         f.max_iters = a.max_iters; f.tol = a.tol; f.head_rows = a.head_rows;
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
-        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n;
+        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg;
         f.rhs = hvec; f.sol = tvec;
         const int rc = launch_forward_tensor(f);
         if (rc != LLA_OK) return rc;
@@ -971,10 +978,10 @@ int launch_t(const BackwardArgs& a) {
             using M = MmCfg<D>;
             LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::PAIRS_SMEM));
             bwd_pairs_mma_kernel<D><<<gp, M::THREADS, M::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
-                                                                     a.dk, a.dv, a.n, first, a.scale);
+                                                                     a.dk, a.dv, a.n, first, a.scale, a.H, kvg);
         } else {
             bwd_pairs_kernel<D><<<gp, BW_THREADS, C::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc,
-                                                                          a.dq, a.dk, a.dv, a.n, first, a.scale);
+                                                                          a.dq, a.dk, a.dv, a.n, first, a.scale, a.H, kvg);
         }
         LLA_CUDA_TRY(cudaGetLastError());
     }

@@ -106,6 +106,7 @@ struct BackwardArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
+    int kv_group;               // query heads per key/value head (k, v, dk, dv are [B, H / kv_group, n, d])
     int cuda_core_pairs;        // 1: pair kernel on the CUDA cores even where the tensor-core one exists
     cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
     cudaEvent_t fork, join;

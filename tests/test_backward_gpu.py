@@ -118,6 +118,39 @@ def test_backward_full_bench_workload_sampled_heads(backward_oracle):
             assert err.max() <= TOL, (name, b, h, float(err.max()))
 
 
+@pytest.mark.parametrize("d,impl", [(64, 0), (128, 0), (64, 1)])
+def test_backward_grouped_kv_heads(backward_oracle, d, impl):
+    # H query heads over Hkv shared key/value heads: the oracle sees k, v repeated per query head and the
+    # shared head's gradient is the sum over its group
+    B, H, Hkv, n = 1, 4, 2, 300
+    w = inputs.CONFIGS[2].shrink(B=B, H=H, n=n, d=d, dv=d, seed=270 + d)
+    q, _, _ = inputs.make_prefill(w)
+    _, k, v = inputs.make_prefill(w.shrink(H=Hkv, seed=271 + d))
+    g = inputs.make_upstream_grad(w)
+    grp = H // Hkv
+    rq, rk, rv = backward_oracle.backward(q, np.repeat(k, grp, axis=1), np.repeat(v, grp, axis=1), g, w.scale, w.lam)
+    rk = rk.reshape(B, Hkv, grp, n, d).sum(axis=2)
+    rv = rv.reshape(B, Hkv, grp, n, d).sum(axis=2)
+    dq_, dk_, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
+    dg = dev(g, "f32")
+    out = torch.empty((B, H, n, d), dtype=torch.float32, device="cuda")
+    rho = torch.empty((B, H, n, d), dtype=torch.float32, device="cuda")
+    stats = torch.empty((B, H, n, 3), dtype=torch.float32, device="cuda")
+    L.lla_forward_ex(dq_, dk_, dv_, out, B, H, n, d, d, w.scale, w.lam, out_dtype=L.LLA_F32, rho=rho, stats=stats,
+                     kv_heads=Hkv, stream=stream_ptr())
+    gq = torch.full((B, H, n, d), float("nan"), dtype=torch.float32, device="cuda")
+    gk = torch.full((B, Hkv, n, d), float("nan"), dtype=torch.float32, device="cuda")
+    gv = torch.full((B, Hkv, n, d), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = L.lla_backward_workspace_bytes(B, H, n, d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, gq, gk, gv, B, H, n, d, w.scale, w.lam, workspace=ws,
+                      workspace_bytes=nbytes, impl=impl, kv_heads=Hkv, stream=stream_ptr())
+    torch.cuda.synchronize()
+    for name, a, r in (("dq", gq, rq), ("dk", gk, rk), ("dv", gv, rv)):
+        err = grad_err(a.cpu().numpy().astype(np.float64), r)
+        assert err.max() <= TOL, (name, float(err.max()))
+
+
 def test_backward_argument_checks():
     ok = 0x1000
     with pytest.raises(L.LlaError) as e:
