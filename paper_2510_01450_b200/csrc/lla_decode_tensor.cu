@@ -104,9 +104,19 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
 #else
 #define CG_TARG
 #endif
+// Thread layout of the 64 x 64 solve over 128 threads: a thread keeps a 4 x 8 block of the matrix --
+// rows cg_row0(tid) .. +3, columns cg_col0(tid) .. +7, as cr[8 i + j] -- so that a matrix-vector product
+// reads eight entries of the vector per thread (the shared-memory-to-register path bounds this kernel;
+// half rows of 32 entries read four times as much).  The eight lanes that share four rows then reduce
+// their partial sums by recursive halving (four 64-bit shuffles), after which lane pairs hold the
+// product's entry for row cg_row(tid).
+__device__ __forceinline__ int cg_row0(int tid) { return 16 * (tid >> 5) + 4 * ((tid & 31) >> 3); }
+__device__ __forceinline__ int cg_col0(int tid) { return 8 * (tid & 7); }
+__device__ __forceinline__ int cg_row(int tid) { return cg_row0(tid) + 2 * ((tid >> 2) & 1) + ((tid >> 1) & 1); }
 __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double b_r, double* xs, double* pbuf, double* redbuf, int& iters CG_TARG) {
     const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
-    const int r = tid >> 1, hh = tid & 1;
+    const int r = cg_row(tid);
+    const bool owner = (tid & 1) == 0, b4 = (tid & 4) != 0, b2 = (tid & 2) != 0;
     auto sync128 = [&]() { asm volatile("bar.sync 2, 128;" ::: "memory"); };
     double x = 0.0, rv = b_r, pv = 0.0, sv = 0.0, alpha = 0.0, gamma_old = 0.0, stop = 0.0;
     bool done = false;
@@ -118,21 +128,25 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
 #define CG_T(i)
 #endif
     for (int it = 0; it <= LLA_CG_CAP; ++it) {
-        if (hh == 0) pbuf[r] = rv;
+        if (owner) pbuf[r] = rv;
         sync128();
         CG_T(0);
-        const double2* pp = reinterpret_cast<const double2*>(pbuf + 32 * hh);
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+        const double2* pp = reinterpret_cast<const double2*>(pbuf + cg_col0(tid));
+        const double2 p01 = pp[0], p23 = pp[1], p45 = pp[2], p67 = pp[3];
+        double a[4];
 #pragma unroll
-        for (int c = 0; c < 32; c += 4) {
-            const double2 p01 = pp[c >> 1], p23 = pp[(c >> 1) + 1];
-            a0 = fma(cr[c], p01.x, a0);
-            a1 = fma(cr[c + 1], p01.y, a1);
-            a2 = fma(cr[c + 2], p23.x, a2);
-            a3 = fma(cr[c + 3], p23.y, a3);
+        for (int i = 0; i < 4; ++i) {
+            const double e0 = fma(cr[8 * i + 1], p01.y, cr[8 * i] * p01.x);
+            const double e1 = fma(cr[8 * i + 3], p23.y, cr[8 * i + 2] * p23.x);
+            const double e2 = fma(cr[8 * i + 5], p45.y, cr[8 * i + 4] * p45.x);
+            const double e3 = fma(cr[8 * i + 7], p67.y, cr[8 * i + 6] * p67.x);
+            a[i] = (e0 + e1) + (e2 + e3);
         }
-        double wv = (a0 + a1) + (a2 + a3);
-        wv += __shfl_xor_sync(0xffffffffu, wv, 1);           // both lanes of a row now hold (C r)_row
+        // recursive halving over the eight lanes of a row group: 4 -> 2 -> 1 partial sums, then the pair
+        const double k0 = (b4 ? a[2] : a[0]) + __shfl_xor_sync(0xffffffffu, b4 ? a[0] : a[2], 4);
+        const double k1 = (b4 ? a[3] : a[1]) + __shfl_xor_sync(0xffffffffu, b4 ? a[1] : a[3], 4);
+        double wv = (b2 ? k1 : k0) + __shfl_xor_sync(0xffffffffu, b2 ? k0 : k1, 2);
+        wv += __shfl_xor_sync(0xffffffffu, wv, 1);           // both lanes of a pair now hold (C r)_row
         CG_T(1);
         // (r, r) and (C r, r): each parity class of lanes sums the warp's 16 rows once
         double g = rv * rv, dl = wv * rv;
@@ -168,7 +182,7 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
 #ifdef LLA_DT_TIMING
     if (tid == 0 && tstat) for (int i = 0; i < 5; ++i) atomicAdd(tstat + i, (int)(cgt_[i] >> 4));
 #endif
-    if (hh == 0) xs[r] = x;
+    if (owner) xs[r] = x;
     sync128();
     return done;
 }
@@ -614,12 +628,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (warp < 4) {
         int cg_its = 0;
         double cr[32];
-        {
-            const double* crow = Md + (tid >> 1) * 65 + 32 * (tid & 1);
 #pragma unroll
-            for (int c = 0; c < 32; ++c) cr[c] = crow[c];
-        }
-        const bool okc = cg_solve_64(cr, rhs[tid >> 1], xs, xs + 64, xs + 128, cg_its);
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) cr[8 * i + j] = Md[(cg_row0(tid) + i) * 65 + cg_col0(tid) + j];
+        const bool okc = cg_solve_64(cr, rhs[cg_row(tid)], xs, xs + 64, xs + 128, cg_its);
         if (tid == 0) {
             s_cg_ok = okc ? 1 : 0;
             if (prm.status) atomicAdd(prm.status + LLA_STATUS_ITER_SUM, cg_its);
@@ -685,27 +698,33 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     }
     __syncthreads();
     SV_T(0);
-    // this thread's half row of the centred matrix
+    // this thread's 4 x 8 block of the centred matrix (see cg_solve_64)
+    const int row0 = cg_row0(tid), col0 = cg_col0(tid), myrow = cg_row(tid);
     double cr[32];
 #pragma unroll
     for (int c = 0; c < 32; ++c) cr[c] = 0.0;
     for (int p = 0; p < splits; ++p) {
-        const float4* mp = reinterpret_cast<const float4*>(src + (size_t)p * PF + r * D + 32 * hh);
         const double f = s_f[p];
 #pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4) {
-            const float4 v = mp[c4];
-            cr[4 * c4] += f * (double)v.x; cr[4 * c4 + 1] += f * (double)v.y;
-            cr[4 * c4 + 2] += f * (double)v.z; cr[4 * c4 + 3] += f * (double)v.w;
+        for (int i = 0; i < 4; ++i) {
+            const float4* mp = reinterpret_cast<const float4*>(src + (size_t)p * PF + (row0 + i) * D + col0);
+            const float4 v0 = mp[0], v1 = mp[1];
+            cr[8 * i] += f * (double)v0.x; cr[8 * i + 1] += f * (double)v0.y;
+            cr[8 * i + 2] += f * (double)v0.z; cr[8 * i + 3] += f * (double)v0.w;
+            cr[8 * i + 4] += f * (double)v1.x; cr[8 * i + 5] += f * (double)v1.y;
+            cr[8 * i + 6] += f * (double)v1.z; cr[8 * i + 7] += f * (double)v1.w;
         }
     }
-    const double ar = s_a[r];
 #pragma unroll
-    for (int c = 0; c < 32; ++c) cr[c] = cr[c] * inv - ar * s_a[32 * hh + c];
+    for (int i = 0; i < 4; ++i) {
+        const double ai = s_a[row0 + i];
 #pragma unroll
-    for (int c = 0; c < 32; ++c)
-        if (32 * hh + c == r) cr[c] += ridge;
-    const double b_r = (double)to_f32(q[(size_t)bh * D + r]) - ar;
+        for (int j = 0; j < 8; ++j) {
+            cr[8 * i + j] = cr[8 * i + j] * inv - ai * s_a[col0 + j];
+            if (row0 + i == col0 + j) cr[8 * i + j] += ridge;
+        }
+    }
+    const double b_r = (double)to_f32(q[(size_t)bh * D + myrow]) - s_a[myrow];
     int cg_its = 0;
     SV_T(1);
 #ifdef LLA_DT_TIMING
@@ -718,8 +737,10 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     bool solved = true;
     if (!okc) {        // uniform over the block: the decision comes from block-wide sums
 #pragma unroll
-        for (int c = 0; c < 32; ++c) s_L[r * 65 + 32 * hh + c] = cr[c];
-        if (hh == 0) s_x[r] = b_r;
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s_L[(row0 + i) * 65 + col0 + j] = cr[8 * i + j];
+        if ((tid & 1) == 0) s_x[myrow] = b_r;
         solved = block_ldlt_solve<D>(s_L, 65, s_x);
     }
     // o_e = vbar_e + sum_f (N[e][f] / omega - vbar_e kbar_f) y_f, two threads per output element
