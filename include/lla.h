@@ -204,6 +204,8 @@ typedef struct lla_decode_params {
        max_pages * page_size >= Lmax; Lmax then only bounds lens.  bf16 and fp32 caches alike. */
     const int *block_table;
     int page_size, max_pages, num_pages;
+    int window;     /* sliding window: 0 = the query sees all lens[b] cached keys; W > 0 = only the last
+                       min(W, lens[b]) of them (positions lens[b] - W .. lens[b] - 1).  Not with a paged cache */
 } lla_decode_params;
 
 int lla_decode_ex(const lla_decode_params *p);

@@ -236,6 +236,8 @@ int lla_decode_ex(const lla_decode_params* p) {
             return LLA_ERR_INVALID_ARG;
         a.paged = lla::PagedKv{p->block_table, p->page_size, p->max_pages, p->num_pages};
     }
+    if (p->window < 0 || (p->window > 0 && p->block_table)) return LLA_ERR_INVALID_ARG;
+    a.window = p->window;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
     const int st = lla::launch_decode(a);
     if (st != LLA_OK) return st;

@@ -32,6 +32,17 @@ __device__ __forceinline__ size_t kv_row(const PagedKv& pg, int b, int kvl, int 
     return ((size_t)page * hkv + kvl) * pg.page_size + j % pg.page_size;
 }
 
+// Keys a decode unit sees: all len cached keys, or with a sliding window the last `window` of them
+// (positions len - window .. len - 1).
+__host__ __device__ __forceinline__ int visible_keys(int len, int Lmax, int window) {
+    const int L = len < 1 ? 1 : (len > Lmax ? Lmax : len);
+    return window > 0 && window < L ? window : L;
+}
+__host__ __device__ __forceinline__ int first_visible_key(int len, int Lmax, int window) {
+    const int L = len < 1 ? 1 : (len > Lmax ? Lmax : len);
+    return L - visible_keys(len, Lmax, window);
+}
+
 struct ForwardArgs {
     const void* q;
     const void* k;
@@ -79,6 +90,7 @@ struct DecodeArgs {
     int ridge_mode;             // lla_ridge_mode
     int kv_group = 1;           // query heads per key/value head: caches are [B, H / kv_group, Lmax, d]
     PagedKv paged = {nullptr, 0, 0, 0};
+    int window = 0;             // sliding window: only the last `window` cached keys are visible (0: all)
 };
 
 // Backward pass (backward appendix): gradients of a scalar loss with respect to q, k, v given

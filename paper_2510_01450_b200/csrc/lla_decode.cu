@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(DC_THREADS)
 decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache, const TIn* __restrict__ vcache,
                       const int* __restrict__ lens, TOut* __restrict__ out, int H, int Lmax, float scale,
                       float lambda, int splits, int head_rows, float* __restrict__ parts, int* __restrict__ status,
-                      const float* __restrict__ lambda_units, int ridge_mode, int kv_group, const PagedKv paged) {
+                      const float* __restrict__ lambda_units, int ridge_mode, int kv_group, const PagedKv paged, int window) {
     using C = DcCfg<D>;
     constexpr bool ACCURATE = sizeof(TIn) == 4;
     extern __shared__ double smem_d[];
@@ -76,8 +76,8 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     const int tid = threadIdx.x;
     const int bh = blockIdx.y, part = blockIdx.x;
     const int b = bh / H;
-    int L = lens[b];
-    L = max(1, min(L, Lmax));
+    const int start = first_visible_key(lens[b], Lmax, window);     // sliding window: keys start .. start + L - 1
+    const int L = visible_keys(lens[b], Lmax, window);
     if (L < head_rows) return;   // short caches are solved directly by the fp64 kernel
     const int chunk = ((L + splits - 1) / splits + DC_BK - 1) / DC_BK * DC_BK;
     const int jbeg = part * chunk, jend = min(L, jbeg + chunk);
@@ -98,7 +98,7 @@ decode_moments_kernel(const TIn* __restrict__ q, const TIn* __restrict__ kcache,
     for (int j0 = jbeg; j0 < jend; j0 += DC_BK) {
         const int jn = min(DC_BK, jend - j0);
         // a tile never straddles a page (page_size is a multiple of the tile, j0 of the tile)
-        const size_t row0 = kv_row(paged, b, kvl, hkv, Lmax, j0);
+        const size_t row0 = kv_row(paged, b, kvl, hkv, Lmax, start + j0);
         const TIn* kb = kcache + row0 * D;
         const TIn* vb = vcache + row0 * D;
         __syncthreads();
@@ -222,7 +222,7 @@ template <int D, typename TIn, typename TOut>
 __global__ void __launch_bounds__(DC_THREADS)
 decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts, TOut* __restrict__ out,
                       const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
-                      int* __restrict__ status, const float* __restrict__ lambda_units, int ridge_mode) {
+                      int* __restrict__ status, const float* __restrict__ lambda_units, int ridge_mode, int window) {
     using C = DcCfg<D>;
     extern __shared__ double smem_d[];
     double* Md = smem_d;
@@ -231,7 +231,7 @@ decode_combine_kernel(const TIn* __restrict__ q, const float* __restrict__ parts
     float* Nd = reinterpret_cast<float*>(c + 2 * D);
     __shared__ double qd_s[D];
     const int tid = threadIdx.x, bh = blockIdx.x;
-    if (max(1, min(lens[bh / H], Lmax)) < head_rows) return;
+    if (visible_keys(lens[bh / H], Lmax, window) < head_rows) return;
     const float* src = parts + (size_t)bh * splits * C::PART_FLOATS;
     for (int e = tid; e < D; e += DC_THREADS) qd_s[e] = (double)to_f32(q[(size_t)bh * D + e]);
     float m = -INFINITY;
@@ -293,7 +293,7 @@ int launch_t(const DecodeArgs& a) {
         dim3 grid(splits, a.B * a.H);
         k1<<<grid, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache,
                                                  a.lens, (TOut*)a.out, a.H, a.Lmax, a.scale, a.lambda, splits,
-                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode, a.kv_group, a.paged);
+                                                 a.head_rows, (float*)a.workspace, a.status, a.lambda_units, a.ridge_mode, a.kv_group, a.paged, a.window);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     if (splits > 1) {
@@ -301,7 +301,7 @@ int launch_t(const DecodeArgs& a) {
         LLA_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         k2<<<a.B * a.H, DC_THREADS, smem, a.stream>>>((const TIn*)a.q, (const float*)a.workspace,
                                                       (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows, a.lambda, splits, a.status,
-                                                      a.lambda_units, a.ridge_mode);
+                                                      a.lambda_units, a.ridge_mode, a.window);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     return LLA_OK;

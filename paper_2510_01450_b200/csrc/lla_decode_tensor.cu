@@ -220,6 +220,7 @@ struct DtParams {
     const float* lambda_units;   // optional per-(sequence, head) ridge
     int ridge_mode;
     int kv_group;        // query heads per key/value head
+    int window;          // sliding window (0: none)
     PagedKv paged;       // table != nullptr: the tensor maps cover [num_pages * kv heads][page_size][64]
 };
 
@@ -250,7 +251,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (prm.B <= DT_MAX_RANKED) {
         __shared__ int s_len[DT_MAX_RANKED];
         __shared__ int s_pick;
-        for (int b = tid; b < prm.B; b += DT_THREADS) s_len[b] = max(1, min(prm.lens[b], prm.Lmax));
+        for (int b = tid; b < prm.B; b += DT_THREADS) s_len[b] = visible_keys(prm.lens[b], prm.Lmax, prm.window);
         __syncthreads();
         const int want = blockIdx.y / prm.H;
         for (int b = tid; b < prm.B; b += DT_THREADS) {
@@ -262,8 +263,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         __syncthreads();
         bh = s_pick * prm.H + blockIdx.y % prm.H;
     }
-    int L = prm.lens[bh / prm.H];
-    L = max(1, min(L, prm.Lmax));
+    const int kstart = first_visible_key(prm.lens[bh / prm.H], prm.Lmax, prm.window);   // sliding window
+    const int L = visible_keys(prm.lens[bh / prm.H], prm.Lmax, prm.window);
     if (L < prm.head_rows) return;                      // short caches: solved by the direct fp64 kernel
     const int chunk = ((L + prm.splits - 1) / prm.splits + DT_BK - 1) / DT_BK * DT_BK;
     const int jbeg = part * chunk, jend = min(L, jbeg + chunk);
@@ -304,7 +305,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 DT_EV(1, t);
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
-                int unit = kvh, jrow = jbeg + t * DT_BK;
+                int unit = kvh, jrow = kstart + jbeg + t * DT_BK;
                 if (table) {
                     const int page = min(max(table[jrow / prm.paged.page_size], 0), prm.paged.num_pages - 1);
                     unit = page * hkv + kvl;
@@ -668,7 +669,7 @@ template <typename TOut>
 __global__ void __launch_bounds__(DT_COMPUTE, 4)
 decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict__ parts, TOut* __restrict__ out,
                     const int* __restrict__ lens, int H, int Lmax, int head_rows, float lambda, int splits,
-                    int* __restrict__ status, const float* __restrict__ lambda_units, int ridge_mode) {
+                    int* __restrict__ status, const float* __restrict__ lambda_units, int ridge_mode, int window) {
     constexpr int D = DT_D, PF = 2 * D * D + 2 * D + 4;
     __shared__ __align__(16) double s_a[D], s_c[D], s_x[D], s_p[D], s_red[24];
     __shared__ double s_f[DS_MAX_SPLITS];
@@ -681,7 +682,7 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
 #define SV_T(ph)
 #endif
     {
-    if (max(1, min(lens[bh / H], Lmax)) < head_rows) return;
+    if (visible_keys(lens[bh / H], Lmax, window) < head_rows) return;
     const float* src = parts + (size_t)bh * splits * PF;
     float m = -INFINITY;
     for (int p = 0; p < splits; ++p) m = fmaxf(m, src[(size_t)p * PF + 2 * D * D + 2 * D + 1]);
@@ -787,7 +788,7 @@ int launch_t(const DecodeArgs& a) {
     DtParams prm;
     prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
-    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode; prm.kv_group = kvg; prm.paged = a.paged;
+    prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode; prm.kv_group = kvg; prm.paged = a.paged; prm.window = a.window;
     prm.parts = (float*)a.workspace; prm.status = a.status;
     prm.defer = have_ws ? 1 : 0;      // with a record buffer the solve runs as its own kernel
     auto kern = decode_tc_kernel<TOut>;
@@ -800,7 +801,7 @@ int launch_t(const DecodeArgs& a) {
     if (have_ws) {
         decode_solve_kernel<TOut><<<BH, DT_COMPUTE, 0, a.stream>>>((const __nv_bfloat16*)a.q, (const float*)a.workspace,
                                                                    (TOut*)a.out, a.lens, a.H, a.Lmax, a.head_rows,
-                                                                   a.lambda, splits, a.status, a.lambda_units, a.ridge_mode);
+                                                                   a.lambda, splits, a.status, a.lambda_units, a.ridge_mode, a.window);
         LLA_CUDA_TRY(cudaGetLastError());
     }
     return LLA_OK;

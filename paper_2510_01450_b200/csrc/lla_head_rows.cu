@@ -107,7 +107,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
                  int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H,
                  const float* __restrict__ lambda_rows, int ridge_mode, int nq, int kv_group,
-                 const PagedKv paged) {
+                 const PagedKv paged, int window) {
     // Prefill (lens == nullptr): block (i, bh) solves row i of head bh; n is the sequence length.
     // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
     // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
@@ -129,13 +129,14 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     if (i >= rows_per_head) return;
     int L = causal ? (n - nq) + i + 1 : n;    // query row i sits at position n - nq + i
     if (lens) {
-        L = max(1, min(lens[bh / H], n));
+        L = visible_keys(lens[bh / H], n, window);
         if (L > lcap) return;               // long caches go through the moment kernel
     }
     const size_t row = lens ? (size_t)bh : (size_t)bh * nq + i;
     const TIn* qrow = q + row * D;
     // (decode over a paged cache: the at most lcap <= page_size keys of a directly-solved unit sit in its first page)
-    const size_t kvrow = kv_row(paged, bh / H, (bh % H) / max(kv_group, 1), H / max(kv_group, 1), n, 0);
+    const int kstart = lens ? first_visible_key(lens[bh / H], n, window) : 0;      // sliding-window decode
+    const size_t kvrow = kv_row(paged, bh / H, (bh % H) / max(kv_group, 1), H / max(kv_group, 1), n, kstart);
     const TIn* kb = k + kvrow * D;
     const TIn* vb = v + kvrow * DV;
 
@@ -368,7 +369,7 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
         (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H, a.lambda_rows,
-        a.ridge_mode, a.nq, a.kv_group, PagedKv{nullptr, 0, 0, 0});
+        a.ridge_mode, a.nq, a.kv_group, PagedKv{nullptr, 0, 0, 0}, 0);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -384,7 +385,7 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
         (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H, a.lambda_units,
-        a.ridge_mode, 1, a.kv_group, a.paged);
+        a.ridge_mode, 1, a.kv_group, a.paged, a.window);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -455,3 +455,29 @@ def test_paged_cache_decode(oracle, dtype, d, splits, page_size, Hkv):
         L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
                         out_dtype=L.LLA_F32, block_table=dt, page_size=96, max_pages=max_pages, num_pages=num_pages,
                         stream=stream_ptr())
+
+
+@pytest.mark.parametrize("dtype,d,splits,window", [("bf16", 64, 1, 300), ("bf16", 64, 2, 1000), ("bf16", 64, 1, 50),
+                                                   ("f32", 16, 1, 200), ("f32", 16, 2, 20)])
+def test_sliding_window_decode(oracle, dtype, d, splits, window):
+    # the query sees the last `window` cached keys: the oracle is given exactly those keys as a cache of its own
+    w = inputs.CONFIGS[5].shrink(B=5, H=2, n=1500, d=d, dv=d, dtype=dtype, len_min=10, len_max=1500, seed=97 + d)
+    q, kc, vc, lens = inputs.make_decode(w)
+    lens[0] = window                      # exactly one window
+    lens[1] = window + 1
+    kw, vw = np.zeros_like(kc), np.zeros_like(vc)
+    cnt = np.minimum(lens, window).astype(np.int32)
+    for b in range(w.B):
+        kw[b, :, : cnt[b]] = kc[b, :, lens[b] - cnt[b]: lens[b]]
+        vw[b, :, : cnt[b]] = vc[b, :, lens[b] - cnt[b]: lens[b]]
+    ref = oracle.decode(q, kw, vw, cnt, w.scale, w.lam)
+    dq, dk, dv_ = dev(q, dtype), dev(kc, dtype), dev(vc, dtype)
+    dl = torch.from_numpy(lens).cuda()
+    out = torch.full((w.B, w.H, d), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = L.lla_decode_workspace_bytes(w.B, w.H, w.n, d, d, in_dtype=LLA_DT[dtype], splits=splits)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, w.H, w.n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                    out_dtype=L.LLA_F32, splits=splits, workspace=ws, workspace_bytes=nbytes, window=window,
+                    stream=stream_ptr())
+    torch.cuda.synchronize()
+    assert row_err(out.cpu().numpy(), ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16)
