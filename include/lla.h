@@ -164,6 +164,9 @@ typedef struct lla_forward_params {
     int kv_heads;   /* 0 or H: every query head has its own k, v.  Otherwise H must be a multiple of kv_heads and
                        k, v are [B, kv_heads, n, d]: query head h reads key/value head h / (H / kv_heads)
                        (grouped-query sharing) */
+    int window;     /* causal sliding window: 0 = a row sees every earlier position; W > 0 = only its last W
+                       positions (itself included).  Needs causal != 0 and W >= the direct-row threshold
+                       (head_rows; 1.5 d for bf16, 2 d for fp32 by default), else LLA_ERR_UNSUPPORTED */
 } lla_forward_params;
 
 int lla_forward_ex(const lla_forward_params *p);

@@ -102,6 +102,7 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.ridge_mode = p->ridge_mode;
     a.nq = p->q_rows > 0 ? p->q_rows : p->n;
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
+    a.window = p->window;
     return a;
 }
 
@@ -143,6 +144,8 @@ int lla_forward_ex(const lla_forward_params* p) {
     const int rc = check_forward(p);
     if (rc != LLA_OK) return rc;
     ForwardArgs a = to_args(p);
+    if (a.window < 0) return LLA_ERR_INVALID_ARG;
+    if (a.window > 0 && (!a.causal || a.window < a.head_rows)) return LLA_ERR_UNSUPPORTED;
     const bool tensor_ok = lla::forward_tensor_supported(a);
     if (p->impl == LLA_IMPL_TENSOR && !tensor_ok) return LLA_ERR_UNSUPPORTED;
     const bool use_tensor = tensor_ok && p->impl != LLA_IMPL_SIMT;

@@ -66,6 +66,7 @@ struct ForwardArgs {
     int ridge_mode;             // lla_ridge_mode
     int nq;                     // query rows per head (the last nq of the n positions); nq == n: plain prefill
     int kv_group = 1;           // query heads per key/value head: k, v are [B, H / kv_group, n, d]
+    int window = 0;             // causal sliding window: a row sees its last `window` positions (0: all)
     const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
 };

@@ -61,7 +61,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                     TOut* __restrict__ out, int n, int causal, float scale, float lambda,
                     int head_rows, int max_iters, float tol, int first_tile,
                     float* __restrict__ rho_out, float* __restrict__ stats, int* __restrict__ iters_out,
-                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq, int H, int kv_group) {
+                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq, int H, int kv_group, int window) {
     constexpr int ROWS = FS_THREADS / TPR;
     constexpr int NG = D / (4 * TPR);    // float4 groups per thread (keys)
     constexpr int NGV = DV / (4 * TPR);  // float4 groups per thread (values)
@@ -80,6 +80,9 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     const int L = causal ? off + row + 1 : n;           // visible keys of this row
     const bool row_ok = row < nq && L >= head_rows;     // other rows: out of range or solved directly
     const int jend = causal ? min(n, off + r0 + ROWS) : n;   // keys this block must sweep
+    // sliding window (causal only): a row sees keys jlo .. L - 1, the block starts at its first row's window
+    const int jlo = (causal && window > 0) ? max(0, L - window) : 0;
+    const int jbeg = (causal && window > 0) ? max(0, off + r0 + 1 - window) / FS_BC * FS_BC : 0;
     const int kvh = kv_unit(bh, H, kv_group);
     const TIn* kb = k + (size_t)kvh * n * D;
     const TIn* vb = v + (size_t)kvh * n * DV;
@@ -94,7 +97,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
 
     // ---- sweep 1: running maximum, omega, weighted key sum (Algorithm 1, first loop) ----
     float m = -INFINITY, omega = 0.f;
-    for (int j0 = 0; j0 < jend; j0 += FS_BC) {
+    for (int j0 = jbeg; j0 < jend; j0 += FS_BC) {
         __syncthreads();
         load_tile<D>(Ks, kb, j0, n);
         __syncthreads();
@@ -110,7 +113,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                 s += qv[g].x * kv[g].x + qv[g].y * kv[g].y + qv[g].z * kv[g].z + qv[g].w * kv[g].w;
             }
             s = row_sum<TPR>(s) * scale;
-            if (jj < lim) {
+            if (jj < lim && jj >= jlo - j0) {
                 if (s > m) {
                     const float c = exp_w<ACCURATE>(m - s);
                     omega *= c;
@@ -161,7 +164,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
         float4 acc[NG];
 #pragma unroll
         for (int g = 0; g < NG; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int j0 = 0; j0 < jend; j0 += FS_BC) {
+        for (int j0 = jbeg; j0 < jend; j0 += FS_BC) {
             __syncthreads();
             load_tile<D>(Ks, kb, j0, n);
             __syncthreads();
@@ -179,7 +182,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                 }
                 s = row_sum<TPR>(s) * scale;
                 a = row_sum<TPR>(a);
-                const float u = jj < lim ? exp_w<ACCURATE>(s - m) * (a - abar) : 0.f;
+                const float u = (jj < lim && jj >= jlo - j0) ? exp_w<ACCURATE>(s - m) * (a - abar) : 0.f;
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
                     acc[g].x += u * kv[g].x; acc[g].y += u * kv[g].y;
@@ -234,7 +237,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
 #pragma unroll
     for (int g = 0; g < NGV; ++g) o[g] = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
-    for (int j0 = 0; j0 < jend; j0 += FS_BC) {
+    for (int j0 = jbeg; j0 < jend; j0 += FS_BC) {
         __syncthreads();
         load_tile<D>(Ks, kb, j0, n);
         load_tile<DV>(Vs, vb, j0, n);
@@ -253,7 +256,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
             }
             s = row_sum<TPR>(s) * scale;
             a = row_sum<TPR>(a);
-            const float c = jj < lim ? exp_w<ACCURATE>(s - m) * (1.f - (a - ybar)) : 0.f;
+            const float c = (jj < lim && jj >= jlo - j0) ? exp_w<ACCURATE>(s - m) * (1.f - (a - ybar)) : 0.f;
             den += c;
 #pragma unroll
             for (int g = 0; g < NGV; ++g) {
@@ -312,7 +315,7 @@ int launch_t(const ForwardArgs& a) {
     kern<<<grid, FS_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, a.causal, a.scale,
         a.lambda, a.head_rows > 0 ? a.head_rows : 0, a.max_iters, a.tol, first_tile, a.rho, a.stats,
-        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq, a.H, a.kv_group);
+        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq, a.H, a.kv_group, a.window);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -177,6 +177,7 @@ struct TcParams {
     float* rho;
     float* stats;
     int H, kv_group;     // query heads per (batch), query heads per key/value head
+    int window;          // causal sliding window (0: none): a row sees its last `window` positions
     const float* rhs;    // solve mode: right-hand sides h_i [B, H, nq, D]; the CG then solves C_i x = h_i ...
     float* sol;          // ... and x_i is written here instead of running the output sweep
     int* iters;
@@ -235,7 +236,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int r0 = tile * TC_BR;
     const int n = prm.n, nq = prm.nq, off = n - nq;     // query row r sits at position off + r
     const int nblk_all = (n + TC_BC - 1) / TC_BC;
-    const int nblk = prm.causal ? min(nblk_all, (off + r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
+    const int cend = prm.causal ? min(nblk_all, (off + r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
+    // sliding window: the tile's sweeps start at the block that holds its first row's first visible key
+    const int cbeg = (prm.causal && prm.window > 0) ? max(0, off + r0 + 1 - prm.window) / TC_BC : 0;
+    const int nblk = cend - cbeg;                        // key blocks per sweep: cbeg .. cend - 1
     const bool split = nblk <= TC_SPLIT_MAX;
 
     if (tid == 0) {
@@ -286,14 +290,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag)) { ok = false; return; }
                 mbar_expect_tx(bar(B_KVFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, &tmK, bar(B_KVFULL + s), 64 * sub, c * TC_BC, kvh);
+                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, &tmK, bar(B_KVFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
                 ++kit;
             };
             auto issue_v = [&](int c, uint32_t g) {
                 const uint32_t s = g % TC_NST;
                 mbar_expect_tx(bar(B_VFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, c * TC_BC, kvh);
+                    tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
             };
             for (uint32_t sweep = 0; ok; ++sweep) {
                 if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
@@ -412,6 +416,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
         const int row = r0 + lrow;
         const int L = prm.causal ? off + row + 1 : n;
+        const int jlo = (prm.causal && prm.window > 0) ? max(0, L - prm.window) : 0;     // first visible key
         const bool row_ok = row < nq && L >= prm.head_rows;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const int c0 = half * NCOL;                        // first row-vector column owned by this thread
@@ -513,11 +518,20 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     tc_wait_ld();
                     if (tid == 0) TC_ACC(1, t_l);
                     TC_T0(t_m);
-                    const int jlim = min(L, n) - (c * TC_BC + 32 * h);   // keys e < jlim are visible
+                    // keys jfirst <= e < jlim of this half block are visible.  Only the diagonal blocks and a
+                    // window's first blocks hide any: there the hidden scores are overwritten with a large negative
+                    // number, whose weight is exactly zero, so the loops below carry no mask
+                    const int jlim = min(L, n) - ((cbeg + c) * TC_BC + 32 * h);
+                    const int jfirst = jlo - ((cbeg + c) * TC_BC + 32 * h);
+                    if (jlim < 32 || jfirst > 0) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (e >= jlim || e < jfirst) sv[e] = __float_as_uint(-1e30f);
+                    }
                     if (kind == SW_MAX) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (e < jlim) part = fmaxf(part, __uint_as_float(sv[e]) * c1);
+                            part = fmaxf(part, __uint_as_float(sv[e]) * c1);
                     } else {
                         uint32_t pk[32];
 #pragma unroll
@@ -536,11 +550,6 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                                 u2 = mul2(u2, fma2(pk2(__uint_as_float(av[2 * e2]), __uint_as_float(av[2 * e2 + 1])), neg1, oab));
                             float u0, u1;
                             upk2(u2, u0, u1);
-                            if (jlim < 32) {                       // only the diagonal blocks mask
-                                u0 = 2 * e2 < jlim ? u0 : 0.f;
-                                u1 = 2 * e2 + 1 < jlim ? u1 : 0.f;
-                                u2 = pk2(u0, u1);
-                            }
                             if (kind != SW_CG) part2 = add2(part2, u2);
                             // 16 keys per k-step: 8 columns of hi, then 8 columns of lo
                             const int ks = e2 >> 3, e = e2 & 7;
@@ -844,14 +853,16 @@ float* scratch_for_device(size_t bytes) {
 // times more than the rest), so at short sequence lengths the first tiles are the longest blocks
 // even though their sweeps are the shortest.  The numbers are a fit to measured runs; they only
 // steer the order, never the result.
-void tile_order(TcParams& prm, int tiles, int first_tile, int n, int off, int d, int causal) {
+void tile_order(TcParams& prm, int tiles, int first_tile, int n, int off, int d, int causal, int window) {
     prm.use_order = 0;
     if (!causal || tiles > TC_ORDER_MAX) return;
     float cost[TC_ORDER_MAX];
     for (int t = 0; t < tiles; ++t) {
         const int r_end = std::min(n, off + (first_tile + t + 1) * TC_BR);      // keys the tile's last row sees
-        const float its = 6.f + 50.f * (float)d / (float)r_end;
-        const float nblk = (float)((r_end + TC_BC - 1) / TC_BC);
+        const int seen = window > 0 ? std::min(r_end, window) : r_end;
+        const float its = 6.f + 50.f * (float)d / (float)seen;
+        const int c_first = window > 0 ? std::max(0, off + (first_tile + t) * TC_BR + 1 - window) / TC_BC : 0;
+        const float nblk = (float)((r_end + TC_BC - 1) / TC_BC - c_first);
         cost[t] = (its + 3.f) * (6.f + nblk);
         prm.order[t] = (unsigned short)t;
     }
@@ -883,7 +894,8 @@ int launch_t(const ForwardArgs& a) {
     prm.dbg = nullptr;
     prm.scratch = nullptr;
     prm.scratch_slots = 0;
-    tile_order(prm, tiles, first_tile, a.n, a.n - a.nq, D, a.causal);
+    prm.window = a.causal ? a.window : 0;
+    tile_order(prm, tiles, first_tile, a.n, a.n - a.nq, D, a.causal, prm.window);
     if constexpr (!Cfg::STATE_IN_SMEM) {
         int dev = 0, sms = 0;
         LLA_CUDA_TRY(cudaGetDevice(&dev));

@@ -481,3 +481,32 @@ def test_sliding_window_decode(oracle, dtype, d, splits, window):
                     stream=stream_ptr())
     torch.cuda.synchronize()
     assert row_err(out.cpu().numpy(), ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16)
+
+
+@pytest.mark.parametrize("dtype,d,n,window,impl", [("bf16", 64, 900, 200, 0), ("bf16", 64, 900, 96, 0), ("bf16", 64, 700, 333, 1),
+                                                   ("bf16", 128, 600, 256, 0), ("f32", 16, 300, 40, 0)])
+def test_sliding_window_forward(oracle, dtype, d, n, window, impl):
+    # row i sees positions max(0, i + 1 - window) .. i; the oracle solves sampled rows as single queries over
+    # exactly those keys (its decode entry point: one "sequence" per sampled row)
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=n, d=d, dv=d, dtype=dtype, seed=98 + d)
+    q, k, v = inputs.make_prefill(w)
+    got = forward(w, q, k, v, out_dtype="f32", window=window, impl=impl)
+    rng = np.random.default_rng(99)
+    rows = np.unique(np.concatenate([np.arange(0, min(n, window + 70)), rng.integers(0, n, 120), [n - 1]]))
+    S = len(rows)
+    qs = np.zeros((S, w.H, d), dtype=np.float32)
+    kc = np.zeros((S, w.H, window, d), dtype=np.float32)
+    vc = np.zeros((S, w.H, window, d), dtype=np.float32)
+    cnt = np.zeros(S, dtype=np.int32)
+    for s, i in enumerate(rows):
+        lo = max(0, i + 1 - window)
+        cnt[s] = i + 1 - lo
+        qs[s] = q[0, :, i]
+        kc[s, :, : cnt[s]] = k[0, :, lo: i + 1]
+        vc[s, :, : cnt[s]] = v[0, :, lo: i + 1]
+    ref = oracle.decode(qs, kc, vc, cnt, w.scale, w.lam)                 # [S, H, d]
+    err = row_err(got[0][:, rows].transpose(1, 0, 2), ref)
+    assert err.max() <= (TOL_F32 if dtype == "f32" else TOL_BF16), (float(err.max()), int(err.argmax()))
+    # without the window the late rows differ: the window is really applied
+    full = forward(w, q, k, v, out_dtype="f32", impl=impl)
+    assert row_err(full[0][:, -1], ref[-1]).max() > 10 * (TOL_F32 if dtype == "f32" else TOL_BF16)
