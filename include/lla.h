@@ -294,7 +294,8 @@ int lla_decode_default_splits(int B, int H, int Lmax);
  *               taken from it; a bf16 `out` limits the accuracy of dq and dk to its rounding
  *   dout      : [B, H, n, d] g, dout_dtype (LLA_BF16 or LLA_F32)
  *   rho, stats: [B, H, n, d] and [B, H, n, 3] fp32, written by lla_forward_ex for the same inputs,
- *               scale, lambda and head_rows
+ *               scale, lambda and head_rows (a plain causal forward: no window, q_rows = n, the ridge of
+ *               the definition; the call cannot tell and would return the gradient of that forward)
  *   dq, dk, dv: [B, H, n, d] fp32 on the device, overwritten
  *   max_iters, tol, head_rows : as in lla_forward_params (0 = defaults)
  *   device_status : optional int[LLA_STATUS_WORDS], zeroed by the call

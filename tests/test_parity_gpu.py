@@ -510,3 +510,31 @@ def test_sliding_window_forward(oracle, dtype, d, n, window, impl):
     # without the window the late rows differ: the window is really applied
     full = forward(w, q, k, v, out_dtype="f32", impl=impl)
     assert row_err(full[0][:, -1], ref[-1]).max() > 10 * (TOL_F32 if dtype == "f32" else TOL_BF16)
+
+
+def test_window_with_chunked_queries_and_grouped_heads(oracle):
+    # the three position-dependent options together: the last q_rows queries of n keys, a window, shared K/V heads
+    d, n, nq, window, H, Hkv = 64, 800, 300, 160, 4, 2
+    w = inputs.CONFIGS[2].shrink(B=1, H=H, n=n, d=d, dv=d, seed=110)
+    q, _, _ = inputs.make_prefill(w)
+    _, k, v = inputs.make_prefill(w.shrink(H=Hkv, seed=111))
+    qc = np.ascontiguousarray(q[:, :, n - nq:])
+    dq, dk, dv_ = dev(qc, "bf16"), dev(k, "bf16"), dev(v, "bf16")
+    out = torch.full((1, H, nq, d), float("nan"), dtype=torch.float32, device="cuda")
+    L.lla_forward_ex(dq, dk, dv_, out, 1, H, n, d, d, w.scale, w.lam, out_dtype=L.LLA_F32, q_rows=nq, kv_heads=Hkv,
+                     window=window, stream=stream_ptr())
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    rows = np.unique(np.concatenate([np.arange(0, 40), np.random.default_rng(112).integers(0, nq, 60), [nq - 1]]))
+    S = len(rows)
+    qs = np.zeros((S, H, d), dtype=np.float32)
+    kc = np.zeros((S, H, window, d), dtype=np.float32)
+    vc = np.zeros((S, H, window, d), dtype=np.float32)
+    kk, vv = np.repeat(k, H // Hkv, axis=1), np.repeat(v, H // Hkv, axis=1)
+    for s, r in enumerate(rows):
+        pos = n - nq + r
+        qs[s] = qc[0, :, r]
+        kc[s] = kk[0, :, pos + 1 - window: pos + 1]
+        vc[s] = vv[0, :, pos + 1 - window: pos + 1]
+    ref = oracle.decode(qs, kc, vc, np.full(S, window, dtype=np.int32), w.scale, w.lam)
+    assert row_err(got[0][:, rows].transpose(1, 0, 2), ref).max() <= TOL_BF16
