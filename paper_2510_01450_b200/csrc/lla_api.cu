@@ -242,6 +242,21 @@ int lla_decode_ex(const lla_decode_params* p) {
     if (p->window < 0 || (p->window > 0 && p->block_table)) return LLA_ERR_INVALID_ARG;
     a.window = p->window;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
+    // The units with short caches go to the direct kernel, which writes rows of `out` nobody else writes and
+    // returns at once for every other unit: it runs on the side stream beside the streaming kernel instead of
+    // behind the solve (its launch alone is 2-3 us of a 300 us step).
+    SideStream* side = side_stream();
+    if (side) {
+        LLA_CUDA_TRY(cudaEventRecord(side->fork, a.stream));
+        LLA_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+        DecodeArgs h = a;
+        h.stream = side->stream;
+        const int rc_head = lla::launch_head_rows_decode(h);
+        LLA_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+        const int st = lla::launch_decode(a);
+        LLA_CUDA_TRY(cudaStreamWaitEvent(a.stream, side->join, 0));
+        return st != LLA_OK ? st : rc_head;
+    }
     const int st = lla::launch_decode(a);
     if (st != LLA_OK) return st;
     return lla::launch_head_rows_decode(a);
