@@ -16,12 +16,16 @@
 // In exact arithmetic this is the appendix's Delta_Q, Delta_K, Delta_V (same function, same derivative);
 // y follows from the saved rho and delta as y = rho omega / delta.
 //
-// Kernels, in launch order:
-//   bwd_moments_kernel    per 64- or 32-row query tile: kbar_i, gbar_i, h_i          (CUDA cores, fp32)
-//   forward_tc_kernel     in solve mode: C_i t_i = h_i by conjugate gradients        (tensor cores)
-//   bwd_rowprep_kernel    y_i, the per-row scalars, dQ_i = t_i
-//   bwd_pairs_kernel      per 64-key tile over all later query tiles: dK, dV (registers), dQ (atomics)
+// Kernels (the direct rows run on a side stream beside the other four, which run in this order):
+//   bwd_moments_*         per 64-row query tile: kbar_i, gbar_i, h_i
+//   forward_tc_kernel     in solve mode: C_i t_i = h_i by conjugate gradients           (tcgen05 tensor cores)
+//   bwd_rowprep_kernel    y_i, the per-row scalars, dQ_i = t_i, dL/dlambda_i
+//   bwd_pairs_*           per 64-key tile over all later query tiles: dK, dV (registers), dQ (atomics)
 //   bwd_head_rows_kernel  rows with fewer than head_rows keys: everything in fp64 with a direct solve
+// The moments and pair kernels exist twice: *_mma_kernel on the tensor cores (warp-level bf16 MMAs with hi/lo
+// operand splits; the default) and the fp32 CUDA-core versions (impl = LLA_IMPL_SIMT), kept as an independent
+// cross-check.  With grouped heads (kv_group > 1) k, v, dk, dv are indexed by the key/value head; dk and dv are
+// zeroed first and every kernel adds into them atomically.
 #include "lla_common.cuh"
 
 namespace lla {
