@@ -17,6 +17,9 @@ struct SideStream {
     cudaStream_t stream = nullptr;
     cudaEvent_t fork = nullptr, join = nullptr;
     bool ok = false;
+    // held while a call enqueues its fork / side work / join: a wait captures the event's latest record, so two
+    // host threads interleaving their records on the shared events would wait on each other's points
+    std::mutex use;
 };
 SideStream* side_stream() {
     static std::mutex mu;
@@ -158,6 +161,7 @@ int lla_forward_ex(const lla_forward_params* p) {
     const bool both = p->phases == LLA_PHASE_ALL && lla::head_rows_count(a) > 0;
     SideStream* side = both ? side_stream() : nullptr;
     if (side) {
+        std::lock_guard<std::mutex> lock(side->use);
         LLA_CUDA_TRY(cudaEventRecord(side->fork, a.stream));
         LLA_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
         const int rc_main = use_tensor ? lla::launch_forward_tensor(a) : lla::launch_forward_simt(a);
@@ -247,6 +251,7 @@ int lla_decode_ex(const lla_decode_params* p) {
     // behind the solve (its launch alone is 2-3 us of a 300 us step).
     SideStream* side = side_stream();
     if (side) {
+        std::lock_guard<std::mutex> lock(side->use);
         LLA_CUDA_TRY(cudaEventRecord(side->fork, a.stream));
         LLA_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
         DecodeArgs h = a;
@@ -333,7 +338,12 @@ int lla_backward_ex(const lla_backward_params* p) {
     a.dlambda = p->dlambda;
     if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
-    if (SideStream* side = side_stream()) { a.side_stream = side->stream; a.fork = side->fork; a.join = side->join; }
+    SideStream* side = side_stream();
+    std::unique_lock<std::mutex> side_lock;
+    if (side) {
+        side_lock = std::unique_lock<std::mutex>(side->use);
+        a.side_stream = side->stream; a.fork = side->fork; a.join = side->join;
+    }
     ForwardArgs probe = {};
     probe.in_dtype = LLA_BF16; probe.d = p->d; probe.dv = p->d;
     if (!lla::forward_tensor_supported(probe)) return LLA_ERR_UNSUPPORTED;
