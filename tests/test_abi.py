@@ -92,6 +92,62 @@ def test_argument_validation_without_device(lib):
         binding.lla_forward(None, ok_ptr, ok_ptr, ok_ptr, 1, 1, 8, 64, 64, 0.125, 1e-3)
 
 
+def test_validation_of_the_position_options(lib):
+    # grouped heads, windows, paged caches and the backward's arguments are checked before any device call
+    ok = 0x1000
+
+    def fwd(**kw):
+        p = binding.ForwardParams()
+        p.q = p.k = p.v = p.out = ok
+        p.B, p.H, p.n, p.d, p.dv, p.scale, p.lambda_, p.causal = 1, 4, 512, 64, 64, 0.125, 1e-3, 1
+        p.in_dtype = p.out_dtype = binding.LLA_BF16
+        for name, val in kw.items():
+            setattr(p, name, val)
+        return lib.lla_forward_ex(ctypes.byref(p))
+
+    assert fwd(kv_heads=3) == 1                    # H is not a multiple
+    assert fwd(kv_heads=-1) == 1
+    assert fwd(window=-5) == 1
+    assert fwd(window=200, causal=0) == 2          # a window needs the causal order
+    assert fwd(window=50) == 2                     # below the direct-row threshold (96)
+    assert fwd(q_rows=600) == 1                    # more queries than keys
+
+    def dec(**kw):
+        p = binding.DecodeParams()
+        p.q = p.kcache = p.vcache = p.lens = p.out = ok
+        p.B, p.H, p.Lmax, p.d, p.dv, p.scale, p.lambda_ = 2, 4, 1024, 64, 64, 0.125, 1e-3
+        p.in_dtype = p.out_dtype = binding.LLA_BF16
+        p.splits = 1
+        for name, val in kw.items():
+            setattr(p, name, val)
+        return lib.lla_decode_ex(ctypes.byref(p))
+
+    assert dec(kv_heads=3) == 1
+    assert dec(block_table=ok, page_size=96, max_pages=16, num_pages=64) == 1      # not a multiple of 128
+    assert dec(block_table=ok, page_size=128, max_pages=4, num_pages=64) == 1      # 4 pages cannot hold Lmax keys
+    assert dec(block_table=ok, page_size=128, max_pages=8, num_pages=64, window=256) == 1
+    assert dec(window=-1) == 1
+
+    def bwd(**kw):
+        p = binding.BackwardParams()
+        for f in ("q", "k", "v", "out", "dout", "rho", "stats", "dq", "dk", "dv"):
+            setattr(p, f, ok)
+        p.B, p.H, p.n, p.d, p.scale, p.lambda_ = 1, 4, 256, 64, 0.125, 1e-3
+        p.out_dtype = p.dout_dtype = binding.LLA_F32
+        p.workspace, p.workspace_bytes = 0x10000, 1 << 40
+        for name, val in kw.items():
+            setattr(p, name, val)
+        return lib.lla_backward_ex(ctypes.byref(p))
+
+    assert bwd(dq=None) == 1
+    assert bwd(d=16) == 2
+    assert bwd(workspace_bytes=1024) == 3
+    assert bwd(workspace=0x10010) == 3             # not 256-byte aligned
+    assert bwd(kv_heads=3) == 1
+    assert bwd(impl=7) == 1
+    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == 4 * 4 * 256 * (4 * 64 + 8)
+
+
 def test_workspace_and_split_arithmetic(lib):
     assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == 0
     # unsplit: optional record buffer for the two-kernel tensor-core path (bf16, d = 64), else none
