@@ -828,12 +828,13 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         if (b0 > a0) continue;
         double acc[4][4] = {};
         for (int j = 0; j < L; ++j) {
-            double ka[4], kc[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                ka[x] = (double)__bfloat162float(Kr[j * D + a0 + x]);
-                kc[x] = (double)__bfloat162float(Kr[j * D + b0 + x]);
-            }
+            // four consecutive bf16 keys per 8-byte load (a0, b0 are multiples of four)
+            const uint2 ra = *reinterpret_cast<const uint2*>(Kr + j * D + a0);
+            const uint2 rb = *reinterpret_cast<const uint2*>(Kr + j * D + b0);
+            const double ka[4] = {(double)__uint_as_float(ra.x << 16), (double)__uint_as_float(ra.x & 0xFFFF0000u),
+                                  (double)__uint_as_float(ra.y << 16), (double)__uint_as_float(ra.y & 0xFFFF0000u)};
+            const double kc[4] = {(double)__uint_as_float(rb.x << 16), (double)__uint_as_float(rb.x & 0xFFFF0000u),
+                                  (double)__uint_as_float(rb.y << 16), (double)__uint_as_float(rb.y & 0xFFFF0000u)};
             const double p = pj[j];
 #pragma unroll
             for (int x = 0; x < 4; ++x)
