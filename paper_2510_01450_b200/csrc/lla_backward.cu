@@ -743,13 +743,28 @@ bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 // whole row -- both solves and every pair term -- runs in fp64 with an explicit C and a direct LDL^T
 // solve, the same split the forward makes.  One block per row; dK and dV go out with atomic adds.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ double warp_sum(double x) {
+
+constexpr int HB_THREADS = 160;   // 136 4x4 tiles of the matrix build fit one round; four blocks per SM
+// eight lanes per key: sum over the lanes of a group of eight
+__device__ __forceinline__ double group8_sum(double x) {
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    for (int o = 4; o >= 1; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
 }
-
-constexpr int HB_THREADS = 128;   // four blocks per SM hide each other's factorisation latency
+// D / 8 consecutive bf16 of a row -> doubles
+template <int NE>
+__device__ __forceinline__ void load_bf16_run(const __nv_bfloat16* p, double (&dst)[NE]) {
+#pragma unroll
+    for (int e = 0; e < NE; e += 8) {
+        const uint4 r = *reinterpret_cast<const uint4*>(p + e);
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            dst[e + 2 * x] = (double)__uint_as_float(w[x] << 16);
+            dst[e + 2 * x + 1] = (double)__uint_as_float(w[x] & 0xFFFF0000u);
+        }
+    }
+}
 template <int D>
 __global__ void __launch_bounds__(HB_THREADS, D == 64 ? 4 : 1)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -783,16 +798,25 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     for (int idx = tid; idx < L * (D / 8); idx += HB_THREADS)
         reinterpret_cast<uint4*>(Kr)[idx] = reinterpret_cast<const uint4*>(k + kvbase * D)[idx];
     __syncthreads();
-    // scores and gamma_j = g . v_j: a warp per key
-    for (int j = warp; j < L; j += HB_THREADS / 32) {
+    // scores and gamma_j = g . v_j: eight lanes per key (D / 8 consecutive elements each), four keys per warp
+    constexpr int NE = D / 8;
+    const int l8 = lane & 7, kslot = warp * 4 + (lane >> 3);
+    for (int j0 = 0; j0 < L; j0 += 4 * (HB_THREADS / 32)) {
+        const int j = j0 + kslot;
         double s = 0.0, gv = 0.0;
-        for (int c = lane; c < D; c += 32) {
-            s += qd[c] * (double)__bfloat162float(Kr[j * D + c]);
-            gv += gd[c] * (double)__bfloat162float(v[(kvbase + j) * D + c]);
+        if (j < L) {
+            double kk[NE], vv[NE];
+            load_bf16_run<NE>(Kr + j * D + NE * l8, kk);
+            load_bf16_run<NE>(v + (kvbase + j) * D + NE * l8, vv);
+#pragma unroll
+            for (int e = 0; e < NE; ++e) {
+                s += qd[NE * l8 + e] * kk[e];
+                gv += gd[NE * l8 + e] * vv[e];
+            }
         }
-        s = warp_sum(s);
-        gv = warp_sum(gv);
-        if (lane == 0) { pj[j] = scale * s; gam[j] = gv; }
+        s = group8_sum(s);
+        gv = group8_sum(gv);
+        if (j < L && l8 == 0) { pj[j] = scale * s; gam[j] = gv; }
     }
     __syncthreads();
     double m = -1e300;
@@ -854,16 +878,22 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const double* y = rhs;
     const double* t = rhs + D;
     // e_j = xi_j . y, f_j = xi_j . t
-    for (int j = warp; j < L; j += HB_THREADS / 32) {
+    for (int j0 = 0; j0 < L; j0 += 4 * (HB_THREADS / 32)) {
+        const int j = j0 + kslot;
         double e = 0.0, f = 0.0;
-        for (int c = lane; c < D; c += 32) {
-            const double xi = (double)__bfloat162float(Kr[j * D + c]) - kb[c];
-            e += xi * y[c];
-            f += xi * t[c];
+        if (j < L) {
+            double kk[NE];
+            load_bf16_run<NE>(Kr + j * D + NE * l8, kk);
+#pragma unroll
+            for (int x = 0; x < NE; ++x) {
+                const double xi = kk[x] - kb[NE * l8 + x];
+                e += xi * y[NE * l8 + x];
+                f += xi * t[NE * l8 + x];
+            }
         }
-        e = warp_sum(e);
-        f = warp_sum(f);
-        if (lane == 0) { ee[j] = e; ff[j] = f; }
+        e = group8_sum(e);
+        f = group8_sum(f);
+        if (j < L && l8 == 0) { ee[j] = e; ff[j] = f; }
     }
     __syncthreads();
     double kappa = 0.0;
