@@ -357,8 +357,9 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
         if (!(S[k * lds + k] > 0.0)) ok = false;
     LDLT_T(3);
     // rhs now holds y with L y = b.  Backward: x_t = (y_t - sum_{r>t} S[r][t] x_r) / D_t.
-    for (int q = 0; q < nrhs; ++q, rhs += rhs_stride)
-    if (tid < 32) {
+    // (one warp per right-hand side: warp ty takes the sides ty, ty + ny, ...)
+    for (int q = ty; q < nrhs; q += ny) {
+        double* rhs_q = rhs + q * rhs_stride;
         constexpr int PER = (D + 31) / 32;
         const int i = tx & 7;
         double part[PER], yv[PER];
@@ -366,7 +367,7 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
         for (int u = 0; u < PER; ++u) {
             const int t = tx + 32 * u;
             part[u] = 0.0;
-            yv[u] = t < n ? rhs[t] : 0.0;
+            yv[u] = t < n ? rhs_q[t] : 0.0;
         }
         for (int c0 = n - NB; c0 >= 0; c0 -= NB) {
             // y - (contributions of later panels) for the eight unknowns c0 + i of this panel
@@ -390,7 +391,7 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
 #pragma unroll
                 for (int t = 0; t < NB; ++t)
                     if (t == tx) xm = xb[t];
-                rhs[c0 + tx] = xm;
+                rhs_q[c0 + tx] = xm;
             }
 #pragma unroll
             for (int u = 0; u < PER; ++u) {
