@@ -1,7 +1,7 @@
 /*
  * lla.h - C ABI of the B200 (sm_100a) Local Linear Attention library.
  *
- * One hot path: the causal LLA forward pass and its single-query decode variant.
+ * One hot path: the causal LLA forward pass, its single-query decode variant, and the backward pass.
  * For every query i the pass forms kernel weights w_ij = exp(scale * q_i.k_j) over the
  * visible keys (j <= i when causal), the query-centred moments
  *     omega_i = sum_j w_ij,  mu_i = sum_j w_ij (k_j - q_i),
@@ -16,7 +16,10 @@
  *   - The caller owns every buffer.  The library reads inputs, writes outputs (outputs must
  *     not alias inputs), and keeps no pointer once the enqueued work has completed.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work
- *     is enqueued on it; no entry point synchronises the device.
+ *     is ordered after what `stream` holds at the call and before anything enqueued on it later; part
+ *     of it (the directly-solved rows) may run on a library-owned side stream that is forked from and
+ *     joined back to `stream` with events.  No entry point synchronises the device (the *_host forms
+ *     synchronise `stream`).  Calls may come from several host threads.
  *   - Return value: an lla_status as int.  Argument errors are detected on the host before any
  *     launch.  Nothing throws or aborts.  Conditions that only the device can see (rows that hit
  *     the iteration cap, a failed pivot in a directly-solved row) are counted in the optional
