@@ -1,13 +1,15 @@
 #!/usr/bin/env python
-"""Benchmark of the LLA hot path on B200: causal forward (prefill) throughput with its roofline,
-the decode step against HBM bandwidth, the end-to-end host-buffer number and the CPU oracle
-baseline.  Prints ONE JSON line on rank 0.
+"""Benchmark of the LLA hot path on B200.  Prints ONE JSON line on rank 0.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 2|3|4]
 
-A step is one pass of the whole forward path (direct early rows + iterative rows) over one batch
-of the bf16 prefill workload B=4, H=8, n=1024, d=dv=64.  With N > 1 every rank runs that batch on
-its own GPU (independent (batch, head) problems, no collective on the data path: weak scaling).
+Headline: the causal forward (prefill) on the largest single-GPU prefill workload, bf16 B=1, H=16,
+n=16384, d=dv=128.  A step is one pass of the whole forward path (direct early rows + iterative rows)
+over one batch.  The line also carries the two smaller prefill workloads (n=1024 and n=4096, d=64)
+as legs measured the same way, the decode step against HBM bandwidth, the backward pass, the
+end-to-end host-buffer number and the CPU oracle baseline with parity figures per leg.  With N > 1
+every rank runs the whole batch on its own GPU (independent (batch, head) problems, no collective
+on the data path: weak scaling).
 """
 from __future__ import annotations
 
@@ -27,12 +29,18 @@ from paper_2510_01450_b200 import inputs  # noqa: E402
 
 METRIC = "lla_prefill_tokens_per_s"
 UNIT = "tokens/s"
-WORKLOAD = 2          # the bf16 prefill workload the headline metric is quoted on
-ROTATE = 16           # input sets cycled through so no step finds its inputs in L2
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/
-# (forward_tc_kernel_cfg2.md and decode_tc_kernel_cfg5.md).
-NCU_TRAFFIC_BYTES = 12.68e6
-NCU_DECODE_TRAFFIC_BYTES = 1.188e9 + 27.8e6 + 34.3e6   # streaming kernel read + record write, solve kernel read
+HEADLINE = 4          # the largest single-GPU prefill workload
+LEGS = (2, 3)         # the other bf16 prefill workloads, reported as sub-objects
+L2_BYTES = 126e6
+# DRAM bytes (read + write) per launch of the dominant kernel from the ncu captures summarised under
+# profiles/: (bytes, summary file).  Workload 4 was captured with 2 of its 16 heads and scaled by 8
+# (traffic is per head: Q, K, V once).
+NCU_TRAFFIC = {
+    2: (12.68e6, "profiles/forward_tc_kernel_cfg2.md"),
+    3: (None, None),
+    4: (None, None),
+}
+NCU_DECODE_TRAFFIC = (1.188e9 + 27.8e6 + 34.3e6, "profiles/decode_tc_kernel_cfg5.md")
 
 
 def env_int(name, default):
@@ -54,9 +62,9 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Polls SM clock and throttle reasons through NVML while the timed regions run."""
+    """Polls SM clock and throttle reasons through NVML while a timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.01):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
@@ -107,14 +115,37 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def algorithmic_flops(w, iters: np.ndarray) -> float:
+def merge_clocks(parts):
+    """One clocks object for the whole run from the per-region samplers."""
+    samples = [s for p in parts for s in p.samples]
+    reasons = sorted(set().union(*[p.reasons for p in parts])) if parts else []
+    mx = next((p.max_mhz for p in parts if p.max_mhz), None)
+    return {"sm_mhz": float(np.median(samples)) if samples else None, "sm_max_mhz": mx, "reasons": reasons,
+            "samples": len(samples)}
+
+
+def algorithmic_flops(w, iters: np.ndarray, iterative_only: bool = False) -> float:
     """N_p (8d + 2dv) + 6d sum_i (i+1) T_i per head, with the CG iterations actually executed
-    (rows solved directly contribute no iteration term)."""
+    (rows solved directly contribute no iteration term; with iterative_only they are left out)."""
     n, d, dv = w.n, w.d, w.dv
-    pairs = n * (n + 1) / 2.0
-    it = np.maximum(iters.reshape(-1, n).astype(np.float64), 0.0)
+    it = iters.reshape(-1, n).astype(np.float64)
     vis = np.arange(1, n + 1, dtype=np.float64)
-    return float(it.shape[0] * pairs * (8 * d + 2 * dv) + 6.0 * d * (it * vis).sum())
+    base = (it >= 0) if iterative_only else np.ones_like(it, dtype=bool)
+    return float((8 * d + 2 * dv) * (base * vis).sum() + 6.0 * d * (np.maximum(it, 0.0) * vis).sum())
+
+
+def workload_config(w):
+    """The keys both arms print: the workload and how L2 is kept out of the measurement."""
+    set_bytes = 4 * w.B * w.H * w.n * w.d * 2
+    rot = rotate_sets(w)
+    return {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "dv": w.dv, "lambda": w.lam, "causal": True,
+            "l2": f"inputs rotate over {rot} sets of {set_bytes / 1e6:.0f} MB ({rot * set_bytes / 1e6:.0f} MB > 126 MB L2)"}
+
+
+def rotate_sets(w) -> int:
+    """Input sets cycled through so that no step finds its inputs in L2 (at least 2, together > 2 x L2)."""
+    set_bytes = 4 * w.B * w.H * w.n * w.d * 2
+    return int(max(2, min(16, np.ceil(2.2 * L2_BYTES / set_bytes))))
 
 
 def oracle_sample_rows(w, n_rows: int, seed: int) -> np.ndarray:
@@ -128,17 +159,17 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import lla_oracle
-    w = inputs.CONFIGS[WORKLOAD]
+    w = inputs.CONFIGS[args.workload]
     q, k, v = inputs.make_prefill(w)
     total_rows = w.B * w.H * w.n
     # calibrate: rows are drawn uniformly over (batch, head, position), so the sample's mean cost
     # per row equals the workload's
-    probe = oracle_sample_rows(w, 512, 1)
+    probe = oracle_sample_rows(w, 128, 1)
     t0 = time.perf_counter()
     lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=probe)
     per_row = (time.perf_counter() - t0) / probe.size
     budget_s = 120.0
-    rows_per_step = int(max(64, min(total_rows, budget_s / max(per_row, 1e-9) / (args.steps + args.warmup))))
+    rows_per_step = int(max(32, min(total_rows, budget_s / max(per_row, 1e-9) / (args.steps + args.warmup))))
     for i in range(args.warmup):
         lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=oracle_sample_rows(w, rows_per_step, 100 + i))
     t0 = time.perf_counter()
@@ -152,13 +183,114 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "dv": w.dv, "lambda": w.lam,
-                   "causal": True},
+        "config": workload_config(w),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
+
+
+class Prefill:
+    """One prefill workload resident on the device: rotating input sets, outputs, timing helpers."""
+
+    def __init__(self, L, torch, w, local):
+        self.L, self.torch, self.w, self.local = L, torch, w, local
+        self.stream = torch.cuda.current_stream()
+        self.sp = self.stream.cuda_stream
+        self.host = inputs.make_prefill(w)
+        hq, hk, hv = (torch.from_numpy(x).to(torch.bfloat16) for x in self.host)
+        self.host_bf16 = (hq, hk, hv)
+        self.rot = rotate_sets(w)
+        self.sets = []
+        for r in range(self.rot):
+            # every set is the same seeded batch with its (batch, head) order rotated: same work, new addresses
+            sh = r % (w.B * w.H)
+            self.sets.append(tuple(torch.roll(t.reshape(w.B * w.H, w.n, -1), sh, 0).reshape(t.shape).contiguous().cuda()
+                                   for t in (hq, hk, hv)))
+        self.outs = [torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16, device="cuda") for _ in range(self.rot)]
+        self.set_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]) + self.outs[0].numel() * 2
+        nws = L.lla_forward_workspace_bytes(w.B, w.H, w.n, w.d, w.dv)
+        self.ws = torch.empty(max(nws, 256), dtype=torch.uint8, device="cuda") if nws else None
+        self.ws_bytes = nws
+
+    def step(self, i, phases=0):
+        w, L = self.w, self.L
+        q, k, v = self.sets[i % self.rot]
+        L.lla_forward_ex(q, k, v, self.outs[i % self.rot], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1,
+                         phases=phases, workspace=self.ws, workspace_bytes=self.ws_bytes, stream=self.sp)
+
+    def probe(self):
+        """Iterations actually executed (for the algorithmic flop count) and an fp32 copy of set 0's
+        output for the parity figures; outside every timed region."""
+        w, L, torch = self.w, self.L, self.torch
+        iters = torch.zeros((w.B, w.H, w.n), dtype=torch.int32, device="cuda")
+        status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+        out32 = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.float32, device="cuda")
+        L.lla_forward_ex(*self.sets[0], out32, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1, iters=iters,
+                         out_dtype=L.LLA_F32, device_status=status, workspace=self.ws, workspace_bytes=self.ws_bytes,
+                         stream=self.sp)
+        torch.cuda.synchronize()
+        self.iters = iters.cpu().numpy()
+        self.status = status.cpu().numpy()
+        self.out32 = out32.cpu().numpy().reshape(-1, w.dv)
+        del out32
+
+    def timed(self, steps, warmup, phases=0, barrier=None):
+        """(ms for `steps` launches, clock summary): CUDA events on the launching stream."""
+        torch = self.torch
+        for i in range(warmup):
+            self.step(i, phases)
+        (barrier or torch.cuda.synchronize)()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(self.local) as clk:
+            e0.record(self.stream)
+            for i in range(steps):
+                self.step(warmup + i, phases)
+            e1.record(self.stream)
+            (barrier or torch.cuda.synchronize)()
+        return e0.elapsed_time(e1), clk
+
+    def roofline(self, peaks, ms_kernel, ms_direct, clk):
+        w = self.w
+        fl = algorithmic_flops(w, self.iters, iterative_only=True)
+        tf = fl / (ms_kernel * 1e-3) / 1e12
+        traffic, src = NCU_TRAFFIC.get(int(w.name[3]), (None, None))
+        c = clk.summary()
+        return {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": tf / peaks["bf16_tflops"], "traffic": traffic, "traffic_source": src,
+                "kernel": f"iterative-rows forward kernel (forward_tc_kernel<{w.d}>)", "ms_per_launch": ms_kernel,
+                "algorithmic_flops_per_launch": fl, "algorithmic_bytes_per_launch": int(self.set_bytes),
+                "peak_source": f"{peaks['source']} burst bf16 (MEASURED_PEAKS.json)",
+                "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
+                "direct_rows_ms_per_launch": ms_direct, "sm_mhz": c["sm_mhz"],
+                "ms_x_mhz": ms_kernel * c["sm_mhz"] if c["sm_mhz"] else None}
+
+    def solver(self):
+        L = self.L
+        cg = self.iters[self.iters >= 0]
+        return {"cg_tol": 1e-4, "cg_max_iters": 64, "cg_mean_iters": float(cg.mean()) if cg.size else 0.0,
+                "cg_max_iters_seen": int(cg.max()) if cg.size else 0,
+                "rows_at_iter_cap": int(self.status[L.STATUS_ROWS_AT_CAP]),
+                "direct_rows_per_head": int((self.iters.reshape(-1, self.w.n)[0] < 0).sum())}
+
+
+def measure_leg(L, torch, peaks, w, local, steps, warmup):
+    """A prefill workload as a sub-object: whole step, dominant kernel alone, direct rows alone."""
+    p = Prefill(L, torch, w, local)
+    p.probe()
+    ms_all, clk_all = p.timed(steps, warmup)
+    ms_k, clk_k = p.timed(steps, 3, L.LLA_PHASE_ITERATIVE)
+    ms_d, _ = p.timed(steps, 3, L.LLA_PHASE_DIRECT)
+    ms_step = ms_all / steps
+    c = clk_all.summary()
+    leg = {"config": workload_config(w), "steps": steps, "ms_per_step": ms_step,
+           "tokens_per_s": w.B * w.n / (ms_step * 1e-3),
+           "tflops": algorithmic_flops(w, p.iters) / (ms_step * 1e-3) / 1e12,
+           "frac_of_bf16_peak_whole_step": algorithmic_flops(w, p.iters) / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+           "sm_mhz": c["sm_mhz"], "ms_x_mhz": ms_step * c["sm_mhz"] if c["sm_mhz"] else None,
+           "roofline": p.roofline(peaks, ms_k / steps, ms_d / steps, clk_k), "solver": p.solver()}
+    return leg, p, [clk_all, clk_k]
 
 
 def run_ours(args):
@@ -189,147 +321,109 @@ def run_ours(args):
         return float(t.item())
 
     peaks = load_peaks()
-    w = inputs.CONFIGS[WORKLOAD].shrink(seed=inputs.CONFIGS[WORKLOAD].seed + 1000 * rank)
-    stream = torch.cuda.current_stream()
-    sp = stream.cuda_stream
+    base = inputs.CONFIGS[args.workload]
+    w = base.shrink(seed=base.seed + 1000 * rank)
+    samplers = []
 
-    # ---- inputs: ROTATE seeded sets resident in HBM (together larger than L2) ----
-    q0, k0, v0 = inputs.make_prefill(w)
-    hq, hk, hv = (torch.from_numpy(x).to(torch.bfloat16) for x in (q0, k0, v0))
-    sets = []
-    for r in range(ROTATE):
-        # every set is the same seeded batch with its (batch, head) order rotated: same work, new addresses
-        sh = r % (w.B * w.H)
-        roll = lambda t: torch.roll(t.reshape(w.B * w.H, w.n, -1), sh, 0).reshape(t.shape).contiguous()
-        sets.append(tuple(roll(t).cuda() for t in (hq, hk, hv)))
-    outs = [torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16, device="cuda") for _ in range(ROTATE)]
-    set_bytes = sum(t.numel() * t.element_size() for t in sets[0]) + outs[0].numel() * 2
+    # ---- headline: device-resident throughput of the whole forward step ----
+    head = Prefill(L, torch, w, local)
+    head.probe()
+    ms_total, clk = head.timed(args.steps, args.warmup, barrier=barrier)
+    ms_total = max_over_ranks(ms_total)
+    samplers.append(clk)
+    c_head = clk.summary()
+    # ---- dominant kernel alone (iterative rows) and the direct rows alone, per-launch average ----
+    ms_kernel, clk_k = head.timed(args.steps, 3, L.LLA_PHASE_ITERATIVE)
+    ms_direct, _ = head.timed(args.steps, 3, L.LLA_PHASE_DIRECT)
+    samplers.append(clk_k)
+    ms_kernel /= args.steps
+    ms_direct /= args.steps
 
-    def step(i, phases=L.LLA_PHASE_ALL):
-        q, k, v = sets[i % ROTATE]
-        L.lla_forward_ex(q, k, v, outs[i % ROTATE], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1,
-                         phases=phases, stream=sp)
+    # ---- end to end through the host-buffer entry point (pinned memory) ----
+    hq, hk, hv = head.host_bf16
+    pq, pk, pv = (t.pin_memory() for t in (hq, hk, hv))
+    pout = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16).pin_memory()
 
-    # iterations actually executed (for the algorithmic flop count), outside the timed region
-    iters = torch.zeros((w.B, w.H, w.n), dtype=torch.int32, device="cuda")
-    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
-    L.lla_forward_ex(*sets[0], outs[0], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1, iters=iters,
-                     device_status=status, stream=sp)
-    torch.cuda.synchronize()
-    it_np = iters.cpu().numpy()
-    flops_step = algorithmic_flops(w, it_np)
-    cg_rows = it_np[it_np >= 0]
-    mean_iters = float(cg_rows.mean()) if cg_rows.size else 0.0
+    def e2e_step():
+        L.lla_forward_host(pq, pk, pv, pout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_BF16, w.scale,
+                           w.lam, 1, head.sp)
 
-    clocks = ClockSampler(local)
-    with clocks:
-        # ---- device-resident throughput ----
-        for i in range(args.warmup):
-            step(i)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(args.steps):
-            step(args.warmup + i)
-        e1.record(stream)
-        barrier()
-        ms_total = max_over_ranks(e0.elapsed_time(e1))
-
-        # ---- dominant kernel alone (iterative rows), per-launch average, same rotation ----
-        for i in range(3):
-            step(i, L.LLA_PHASE_ITERATIVE)
-        torch.cuda.synchronize()
-        k0e, k1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        k0e.record(stream)
-        for i in range(args.steps):
-            step(3 + i, L.LLA_PHASE_ITERATIVE)
-        k1e.record(stream)
-        torch.cuda.synchronize()
-        ms_kernel = k0e.elapsed_time(k1e) / args.steps
-        d0e, d1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        d0e.record(stream)
-        for i in range(args.steps):
-            step(i, L.LLA_PHASE_DIRECT)
-        d1e.record(stream)
-        torch.cuda.synchronize()
-        ms_direct = d0e.elapsed_time(d1e) / args.steps
-
-        # ---- end to end through the host-buffer entry point (pinned memory) ----
-        pq, pk, pv = (t.pin_memory() for t in (hq, hk, hv))
-        pout = torch.empty((w.B, w.H, w.n, w.dv), dtype=torch.bfloat16).pin_memory()
-
-        def e2e_step():
-            L.lla_forward_host(pq, pk, pv, pout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_BF16, w.scale,
-                               w.lam, 1, sp)
-
-        for _ in range(max(3, args.warmup // 4)):
-            e2e_step()
-        e2e_steps = max(5, args.steps // 4)
-        barrier()
+    for _ in range(3):
+        e2e_step()
+    e2e_steps = max(5, args.steps // 4)
+    barrier()
+    with ClockSampler(local) as clk_e:
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             e2e_step()
         torch.cuda.synchronize()
         e2e_s = max_over_ranks(time.perf_counter() - t0)
-        barrier()
+    samplers.append(clk_e)
+    barrier()
+    del pq, pk, pv
 
-        # ---- decode step (64 sequences x 16 heads over a bf16 KV cache), rank 0 only ----
-        decode = None
-        if rank == 0 and not args.no_decode:
-            decode = bench_decode(L, torch, peaks, sp, stream)
-        backward = None
-        if rank == 0 and not args.no_backward:
-            backward = bench_backward(L, torch, peaks, w, sets, sp, stream)
+    # ---- the other prefill workloads, decode and backward: rank 0 only ----
+    legs, decode, backward, parity = {}, None, None, {}
+    leg_objs = {}
+    if rank == 0 and not args.no_legs:
+        for c in LEGS:
+            if c == args.workload:
+                continue
+            wl = inputs.CONFIGS[c]
+            est_ms = {2: 0.4, 3: 1.6}.get(c, 5.0)
+            leg_steps = int(max(20, min(400, 300.0 / est_ms)))      # about 0.3 s per timed region
+            leg, obj, cl = measure_leg(L, torch, peaks, wl, local, leg_steps, max(3, args.warmup))
+            legs[f"prefill_cfg{c}"] = leg
+            leg_objs[c] = obj
+            samplers += cl
+    if rank == 0 and not args.no_decode:
+        decode, cl = bench_decode(L, torch, peaks, head.sp, head.stream, local)
+        samplers.append(cl)
+    if rank == 0 and not args.no_backward:
+        bw_obj = leg_objs.get(2) or Prefill(L, torch, inputs.CONFIGS[2], local)
+        backward, cl = bench_backward(L, torch, peaks, bw_obj, local)
+        samplers.append(cl)
 
     tokens_step = w.B * w.n
     ms_step = ms_total / args.steps
     value = world * tokens_step / (ms_step * 1e-3)
-    tflops_kernel = flops_step_iterative(w, it_np) / (ms_kernel * 1e-3) / 1e12
-    peak = peaks["bf16_tflops"]
+    flops_step = algorithmic_flops(w, head.iters)
+    roof = head.roofline(peaks, ms_kernel, ms_direct, clk_k)
+    h2d = int(sum(t.numel() * 2 for t in (hq, hk, hv)))
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "dv": w.dv, "lambda": w.lam,
-                   "causal": True, "cg_tol": 1e-4, "cg_mean_iters": mean_iters,
-                   "rows_at_iter_cap": int(status.cpu()[L.STATUS_ROWS_AT_CAP]),
-                   "l2": f"inputs rotate over {ROTATE} sets ({ROTATE * set_bytes / 1e6:.0f} MB > 126 MB L2)"},
+        "config": workload_config(w), "solver": head.solver(),
         "tflops": flops_step / (ms_step * 1e-3) / 1e12,
-        "roofline": {"bound": "tensor", "achieved": tflops_kernel, "peak": peak, "unit": "TFLOP/s",
-                     "frac": tflops_kernel / peak, "traffic": NCU_TRAFFIC_BYTES,
-                     "kernel": "iterative-rows forward kernel (forward_tc_kernel)", "ms_per_launch": ms_kernel,
-                     "algorithmic_flops_per_launch": flops_step_iterative(w, it_np),
-                     "algorithmic_bytes_per_launch": int(set_bytes),
-                     "peak_source": f"{peaks['source']} burst bf16 (MEASURED_PEAKS.json)",
-                     "direct_rows_ms_per_launch": ms_direct},
-        "e2e": {"value": world * tokens_step * e2e_steps / e2e_s, "unit": UNIT,
-                "h2d_bytes_per_step": int(sum(t.numel() * 2 for t in (hq, hk, hv))),
-                "d2h_bytes_per_step": int(pout.numel() * 2), "steps": e2e_steps},
+        "frac_of_bf16_peak_whole_step": flops_step / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "sm_mhz": c_head["sm_mhz"], "ms_x_mhz": ms_step * c_head["sm_mhz"] if c_head["sm_mhz"] else None,
+        "roofline": roof,
+        "e2e": {"value": world * tokens_step * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": int(pout.numel() * 2), "steps": e2e_steps,
+                "ms_per_step": 1e3 * e2e_s / e2e_steps,
+                "note": "lla_forward_host on pinned buffers; the host link carries "
+                        f"{(h2d + pout.numel() * 2) / 1e6:.0f} MB per step"},
         "gpu_launches": 2 * args.steps,
-        "clocks": clocks.summary(),
     }
+    line.update(legs)
     if decode is not None:
         line["decode"] = decode
     if backward is not None:
         line["backward"] = backward
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(w, q0, k0, v0)
+            line["cpu_baseline"], parity[f"cfg{args.workload}"] = cpu_baseline(head, 15.0)
+            for c, obj in leg_objs.items():
+                _, parity[f"cfg{c}"] = cpu_baseline(obj, 4.0)
+            line["parity"] = parity
+        line["clocks"] = merge_clocks(samplers)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
-def flops_step_iterative(w, iters):
-    """Algorithmic flops of the rows the iterative kernel computes (rows with iters >= 0)."""
-    n, d, dv = w.n, w.d, w.dv
-    it = iters.reshape(-1, n).astype(np.float64)
-    vis = np.arange(1, n + 1, dtype=np.float64)
-    mask = it >= 0
-    return float(((8 * d + 2 * dv) * (mask * vis).sum()) + 6.0 * d * (np.maximum(it, 0) * vis).sum())
-
-
-def bench_decode(L, torch, peaks, sp, stream, steps=20, warmup=5):
+def bench_decode(L, torch, peaks, sp, stream, local, steps=30, warmup=5):
     wd = inputs.CONFIGS[5]
     gen = torch.Generator(device="cuda").manual_seed(wd.seed)
     inv = 1.0 / np.sqrt(wd.d)
@@ -343,32 +437,37 @@ def bench_decode(L, torch, peaks, sp, stream, steps=20, warmup=5):
         L.lla_decode(q, kc, vc, lens, out, wd.B, wd.H, wd.n, wd.d, wd.dv, wd.scale, wd.lam, sp)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(steps):
-        L.lla_decode(q, kc, vc, lens, out, wd.B, wd.H, wd.n, wd.d, wd.dv, wd.scale, wd.lam, sp)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        e0.record(stream)
+        for _ in range(steps):
+            L.lla_decode(q, kc, vc, lens, out, wd.B, wd.H, wd.n, wd.d, wd.dv, wd.scale, wd.lam, sp)
+        e1.record(stream)
+        torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     live_bytes = float(lens_np.astype(np.int64).sum()) * wd.H * (wd.d + wd.dv) * 2
     gbs = live_bytes / (ms * 1e-3) / 1e9
+    c = clk.summary()
     del kc, vc
     return {"workload": wd.name, "us_per_step": ms * 1e3, "us_per_token": ms * 1e3 / wd.B, "steps": steps,
+            "sm_mhz": c["sm_mhz"], "ms_x_mhz": ms * c["sm_mhz"] if c["sm_mhz"] else None,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_DECODE_TRAFFIC_BYTES, "algorithmic_bytes": live_bytes,
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_DECODE_TRAFFIC[0],
+                         "traffic_source": NCU_DECODE_TRAFFIC[1], "algorithmic_bytes": live_bytes,
                          "frac_of_nominal_8TBs": gbs / 8000.0,
                          "peak_source": f"{peaks['source']} copy bandwidth (MEASURED_PEAKS.json)"},
-            "l2": "live cache bytes (1.2 GB) exceed L2 (126 MB)"}
+            "l2": "live cache bytes (1.2 GB) exceed L2 (126 MB)"}, clk
 
 
-def bench_backward(L, torch, peaks, w, sets, sp, stream, steps=20, warmup=3, nsets=4):
-    """Backward pass (gradients with respect to q, k, v) on the bench workload: the forward runs once per
-    input set outside the timed region to save rho, stats and the fp32 output; the timed steps are
-    lla_backward_ex alone, rotating over nsets sets of inputs and saved tensors (together larger than L2)."""
+def bench_backward(L, torch, peaks, pre, local, steps=20, warmup=3, nsets=4):
+    """Backward pass (gradients with respect to q, k, v) on the n=1024, d=64 prefill workload: the forward
+    runs once per input set outside the timed region to save rho, stats and the fp32 output; the timed steps
+    are lla_backward_ex alone, rotating over nsets sets of inputs and saved tensors (together larger than L2)."""
+    w, sp, stream = pre.w, pre.sp, pre.stream
     shape = (w.B, w.H, w.n, w.d)
     g = torch.from_numpy(inputs.make_upstream_grad(w)).cuda()
     saved = []
     for r in range(nsets):
-        q, k, v = sets[r]
+        q, k, v = pre.sets[r]
         out = torch.empty(shape, dtype=torch.float32, device="cuda")
         rho = torch.empty(shape, dtype=torch.float32, device="cuda")
         stats = torch.empty((w.B, w.H, w.n, 3), dtype=torch.float32, device="cuda")
@@ -395,48 +494,68 @@ def bench_backward(L, torch, peaks, w, sets, sp, stream, steps=20, warmup=3, nse
         step(i)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(steps):
-        step(warmup + i)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        e0.record(stream)
+        for i in range(steps):
+            step(warmup + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     set_bytes = sum(t.numel() * t.element_size() for t in saved[0])
-    return {"ms_per_step": ms, "tokens_per_s": w.B * w.n / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
+    c = clk.summary()
+    return {"workload": w.name, "ms_per_step": ms, "tokens_per_s": w.B * w.n / (ms * 1e-3),
+            "tflops": flops / (ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "cg_mean_iters": float(it[it >= 0].mean()) if (it >= 0).any() else 0.0,
             "algorithmic_flops_per_step": flops, "gpu_launches_per_step": 5,
+            "sm_mhz": c["sm_mhz"], "ms_x_mhz": ms * c["sm_mhz"] if c["sm_mhz"] else None,
             "l2": f"inputs and saved tensors rotate over {nsets} sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)",
-            "inputs": "bf16 q, k, v; fp32 upstream gradient, forward output, rho, stats; fp32 gradients"}
+            "inputs": "bf16 q, k, v; fp32 upstream gradient, forward output, rho, stats; fp32 gradients"}, clk
 
 
-def cpu_baseline(w, q, k, v):
-    """The oracle, untuned, on this machine's host cores, on a bounded uniform row sample."""
+def cpu_baseline(pre, budget_s):
+    """The oracle, untuned, on this machine's host cores, on a bounded uniform row sample of the workload, and
+    the parity figures of the device output (fp32 buffer) on those same rows."""
     from oracle import lla_oracle
-    probe = oracle_sample_rows(w, 256, 7)
+    w = pre.w
+    q, k, v = pre.host
+    probe = oracle_sample_rows(w, 64, 7)
     t0 = time.perf_counter()
     lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=probe)
     per_row = (time.perf_counter() - t0) / probe.size
     total = w.B * w.H * w.n
-    n_rows = int(max(256, min(total, 15.0 / max(per_row, 1e-9))))
+    n_rows = int(max(64, min(total, budget_s / max(per_row, 1e-9))))
     rows = oracle_sample_rows(w, n_rows, 8)
     t0 = time.perf_counter()
-    lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows)
+    ref = lla_oracle.forward_rows(q, k, v, w.scale, w.lam, rows=rows)
     dt = time.perf_counter() - t0
-    return {"value": rows.size / w.H / dt, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
+    got = pre.out32[rows].astype(np.float64)
+    diff = got - ref
+    e_row = np.linalg.norm(diff, axis=1) / np.linalg.norm(ref, axis=1)
+    e_elem = np.abs(diff).max(axis=1) / np.abs(ref).max(axis=1)
+    parity = {"rows": int(rows.size), "output": "fp32 buffer, bf16 inputs",
+              "E_row_max": float(e_row.max()), "E_row_median": float(np.median(e_row)),
+              "E_elem_max": float(e_elem.max()), "E_glob": float(np.abs(diff).max() / np.abs(ref).max()),
+              "metrics": "E_row = |o_i - ref_i|_2 / |ref_i|_2; E_elem = |o_i - ref_i|_inf / |ref_i|_inf; "
+                         "E_glob = max|o - ref| / max|ref|; gate 2e-3 on E_row"}
+    base = {"value": rows.size / w.H / dt, "unit": UNIT, "cores": lla_oracle.threads(), "kind": "oracle",
             "sample": f"{rows.size} of {total} rows of {w.name}, drawn uniformly over (batch, head, position); "
                       f"{dt:.1f} s; tokens = rows / H"}
+    return base, parity
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", type=int, choices=[2, 3, 4], default=HEADLINE,
+                    help="prefill workload of the headline (default: the largest, n=16384, d=128)")
+    ap.add_argument("--no-legs", action="store_true", help="skip the other prefill workloads")
     ap.add_argument("--no-decode", action="store_true", help="skip the decode measurement")
     ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass measurement")
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity figures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

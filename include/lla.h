@@ -170,7 +170,20 @@ typedef struct lla_forward_params {
     int window;     /* causal sliding window: 0 = a row sees every earlier position; W > 0 = only its last W
                        positions (itself included).  Needs causal != 0 and W >= the direct-row threshold
                        (head_rows; 1.5 d for bf16, 2 d for fp32 by default), else LLA_ERR_UNSUPPORTED */
+    int cg_precise_iters; /* tensor-core kernel only.  The operands formed on the fly in a CG iteration (the search
+                       direction P and the weighted products W .* (P K^T) of Algorithm 2) enter the tensor cores
+                       as bf16 hi + lo pairs (16 mantissa bits, two products each) during the first
+                       cg_precise_iters iterations of a row tile and as single fp16 values (11 bits, one product)
+                       afterwards: an iteration's products are scaled by the size of its search direction,
+                       which has fallen by then, so the coarser operands of the later iterations add less
+                       error than the tolerance leaves.  The fp16 sweeps read an fp16 copy of k made by a
+                       pre-pass into `workspace` (without room for it there, or with an entry of q or k beyond
+                       6e4 in magnitude, every iteration uses pairs).  0 = default (1 iteration; 4 for the row
+                       tiles within the first 8 d positions, which converge more slowly); n > 0 = n
+                       iterations for every tile; LLA_CG_PRECISE_ALL = every iteration with pairs;
+                       LLA_CG_PRECISE_NONE = fp16 from the first iteration on */
 } lla_forward_params;
+enum { LLA_CG_PRECISE_ALL = -1, LLA_CG_PRECISE_NONE = -2 };
 
 int lla_forward_ex(const lla_forward_params *p);
 

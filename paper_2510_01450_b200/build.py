@@ -1,21 +1,26 @@
 """Build ``liblla.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
 Usage: ``python -m paper_2510_01450_b200.build [--force] [--verbose]``
+
+Every ``csrc/*.cu`` is compiled to an object file of its own (in parallel, only when it or a header
+is newer than the object) and the objects are linked into one shared library next to the package.
 """
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 from pathlib import Path
 
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
+OBJ = PKG / "build"
 LIB = PKG / "liblla.so"
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--shared", "-Xcompiler", "-fPIC",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -23,27 +28,40 @@ def sources():
     return sorted(CSRC.glob("*.cu"))
 
 
-def _stale() -> bool:
-    if not LIB.exists():
-        return True
-    newest = max(p.stat().st_mtime for p in list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh"))
-                 + [PKG.parent / "include" / "lla.h"])
-    return LIB.stat().st_mtime < newest
+def _headers_mtime() -> float:
+    return max(p.stat().st_mtime for p in list(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "lla.h"])
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
-    """Compile every ``csrc/*.cu`` into one shared object next to the package."""
-    if not force and not _stale():
-        return LIB
+    """Compile every ``csrc/*.cu`` and link them into one shared object next to the package."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc, *NVCC_FLAGS, "-lcuda", "-o", str(tmp), *map(str, sources())]
-    if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-        print(" ".join(cmd), flush=True)
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
+    hdr = _headers_mtime()
+    if not force and LIB.exists() and LIB.stat().st_mtime >= max([hdr] + [s.stat().st_mtime for s in sources()]):
+        return LIB      # up to date (the objects need not exist: only the library travels to a GPU box)
+    OBJ.mkdir(exist_ok=True)
+    jobs = []
+    for src in sources():
+        obj = OBJ / (src.stem + ".o")
+        if force or not obj.exists() or obj.stat().st_mtime < max(src.stat().st_mtime, hdr):
+            cmd = [nvcc, *NVCC_FLAGS, "-c", "-o", str(obj), str(src)]
+            if verbose:
+                cmd[1:1] = ["-Xptxas", "-v"]
+            jobs.append(cmd)
+    if jobs:
+        def run(cmd):
+            if verbose:
+                print(" ".join(cmd), flush=True)
+            return subprocess.run(cmd, capture_output=not verbose, text=True)
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4)) as pool:
+            for cmd, res in zip(jobs, pool.map(run, jobs)):
+                if res.returncode != 0:
+                    raise RuntimeError(f"nvcc failed: {' '.join(cmd)}\n{res.stdout or ''}\n{res.stderr or ''}")
+    objs = [OBJ / (s.stem + ".o") for s in sources()]
+    if jobs or not LIB.exists() or LIB.stat().st_mtime < max(o.stat().st_mtime for o in objs):
+        tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
+        subprocess.run([nvcc, "--shared", "-gencode", "arch=compute_100a,code=sm_100a", "-lcuda", "-o", str(tmp),
+                        *map(str, objs)], check=True)
+        os.replace(tmp, LIB)
     return LIB
 
 

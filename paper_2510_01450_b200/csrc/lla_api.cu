@@ -106,6 +106,10 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.nq = p->q_rows > 0 ? p->q_rows : p->n;
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     a.window = p->window;
+    if (p->cg_precise_iters != 0) {
+        a.precise_iters = p->cg_precise_iters == LLA_CG_PRECISE_NONE ? 0 : p->cg_precise_iters < 0 ? (1 << 30) : p->cg_precise_iters;
+        a.precise_iters_early = a.precise_iters;
+    }
     return a;
 }
 
@@ -158,6 +162,12 @@ int lla_forward_ex(const lla_forward_params* p) {
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
     // The two row groups write disjoint rows of `out`; when both run, the direct rows go to a side
     // stream so they fill the SMs the iterative kernel's last wave leaves idle.
+    // (the pre-pass of the tensor-core kernel goes first so that the fork below comes after it: the direct rows
+    // then start beside the iterative kernel, not ahead of it, and fill the SMs its last wave leaves idle)
+    if (use_tensor && p->phases != LLA_PHASE_DIRECT) {
+        const int rc_pre = lla::forward_tensor_prepass(a);
+        if (rc_pre != LLA_OK) return rc_pre;
+    }
     const bool both = p->phases == LLA_PHASE_ALL && lla::head_rows_count(a) > 0;
     SideStream* side = both ? side_stream() : nullptr;
     if (side) {
@@ -188,7 +198,22 @@ int lla_forward(const void* q, const void* k, const void* v, void* out, int B, i
     p.in_dtype = LLA_BF16; p.out_dtype = LLA_BF16;
     p.scale = scale; p.lambda = lambda; p.causal = causal;
     p.stream = stream;
-    return lla_forward_ex(&p);
+    // scratch from the stream-ordered pool (kept warm between calls); without it the call still works
+    // (see lla_forward_workspace_bytes)
+    const size_t ws = lla_forward_workspace_bytes(B, H, n, d, dv, LLA_BF16, LLA_IMPL_AUTO);
+    void* scratch = nullptr;
+    if (ws > 0 && check_forward(&p) == LLA_OK) {
+        keep_pool_memory();
+        if (cudaMallocAsync(&scratch, ws, (cudaStream_t)stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            scratch = nullptr;
+        }
+    }
+    p.workspace = scratch;
+    p.workspace_bytes = scratch ? ws : 0;
+    const int rc = lla_forward_ex(&p);
+    if (scratch) (void)cudaFreeAsync(scratch, (cudaStream_t)stream);
+    return rc;
 }
 
 int lla_forward_f32(const void* q, const void* k, const void* v, void* out, int B, int H, int n, int d,
@@ -357,9 +382,11 @@ size_t lla_backward_workspace_bytes(int B, int H, int n, int d) {
 }
 
 size_t lla_forward_workspace_bytes(int B, int H, int n, int d, int dv, int in_dtype, int impl) {
-    (void)B; (void)H; (void)n;
-    // Only the d = 128 tensor-core kernel keeps state off chip: one slot per SM id (see forward_tensor).
-    if (in_dtype == LLA_BF16 && d == 128 && dv == 128 && impl != LLA_IMPL_SIMT) return lla::forward_tensor_scratch_bytes();
+    if (B < 1 || H < 1 || n < 1) return 0;
+    // Only the tensor-core kernel uses any: the fp16 copy of k for its later CG sweeps and, for d = 128, one
+    // slot per SM id for the row vectors it keeps off chip (see lla_forward_tensor.cu).
+    if (in_dtype == LLA_BF16 && (d == 64 || d == 128) && dv == d && impl != LLA_IMPL_SIMT)
+        return lla::forward_tensor_workspace_bytes(B, H, n, d);
     return 0;
 }
 
@@ -432,6 +459,11 @@ int lla_forward_host(const void* q, const void* k, const void* v, void* out, int
     const int units = B * H;
     HostPipe* pipe = (units >= 2 * kHostChunks && nq + nq + nv >= (size_t)(1u << 20)) ? host_pipe() : nullptr;
     if (!pipe) {
+        const size_t wsb = lla_forward_workspace_bytes(B, H, n, d, dv, in_dtype, LLA_IMPL_AUTO);
+        if (wsb > 0) {
+            p.workspace = mem.get(wsb);
+            p.workspace_bytes = p.workspace ? wsb : 0;
+        }
         LLA_CUDA_TRY(cudaMemcpyAsync(dq, q, nq, cudaMemcpyHostToDevice, st));
         LLA_CUDA_TRY(cudaMemcpyAsync(dk, k, nq, cudaMemcpyHostToDevice, st));
         LLA_CUDA_TRY(cudaMemcpyAsync(dvv, v, nv, cudaMemcpyHostToDevice, st));
@@ -442,7 +474,10 @@ int lla_forward_host(const void* q, const void* k, const void* v, void* out, int
         LLA_CUDA_TRY(cudaStreamSynchronize(st));
         return LLA_OK;
     }
-    // chunked: (batch, head) units are independent and contiguous in memory
+    // chunked: (batch, head) units are independent and contiguous in memory; every chunk has its own scratch
+    const int chunk_units = (units + kHostChunks - 1) / kHostChunks;
+    const size_t wsb = lla_forward_workspace_bytes(1, chunk_units, n, d, dv, in_dtype, LLA_IMPL_AUTO);
+    char* wsp = wsb > 0 ? static_cast<char*>(mem.get(wsb * kHostChunks)) : nullptr;
     LLA_CUDA_TRY(cudaEventRecord(pipe->ready, st));            // the buffers exist from here on
     const size_t uq = (size_t)n * d * esz_in, uv = (size_t)n * dv * esz_in, uo = (size_t)n * dv * esz_out;
     int rc_chunks = LLA_OK;
@@ -457,6 +492,7 @@ int lla_forward_host(const void* q, const void* k, const void* v, void* out, int
         pc.q = (char*)dq + u0 * uq; pc.k = (char*)dk + u0 * uq; pc.v = (char*)dvv + u0 * uv; pc.out = (char*)dout + u0 * uo;
         pc.B = 1; pc.H = u1 - u0;
         pc.stream = w;
+        if (wsp) { pc.workspace = wsp + (size_t)c * wsb; pc.workspace_bytes = wsb; }
         const int rc_c = lla_forward_ex(&pc);
         if (rc_c != LLA_OK && rc_chunks == LLA_OK) rc_chunks = rc_c;
         LLA_CUDA_TRY(cudaMemcpyAsync((char*)out + u0 * uo, (char*)dout + u0 * uo, (u1 - u0) * uo, cudaMemcpyDeviceToHost, w));

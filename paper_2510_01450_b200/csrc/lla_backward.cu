@@ -1001,6 +1001,15 @@ int launch_t(const BackwardArgs& a) {
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
         f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg;
         f.rhs = hvec; f.sol = tvec;
+        // what the workspace holds beyond this pass's own vectors serves the solve (the fp16 copy of k; for
+        // d = 128 the row-state slots), so that the backward pass allocates nothing
+        const size_t own = (ws_floats(rows, D, BH) * sizeof(float) + 255) & ~(size_t)255;
+        if (a.workspace_bytes > own) {
+            f.workspace = static_cast<char*>(a.workspace) + own;
+            f.workspace_bytes = a.workspace_bytes - own;
+        }
+        const int rc_pre = forward_tensor_prepass(f);
+        if (rc_pre != LLA_OK) return rc_pre;
         const int rc = launch_forward_tensor(f);
         if (rc != LLA_OK) return rc;
         bwd_rowprep_kernel<D><<<(unsigned)((rows + 7) / 8), BW_THREADS, 0, a.stream>>>(
@@ -1027,7 +1036,8 @@ int launch_t(const BackwardArgs& a) {
 }  // namespace
 
 size_t backward_workspace_bytes(int B, int H, int n, int d) {
-    return ws_floats((long long)B * H * n, d, (long long)B * H) * sizeof(float);
+    const size_t own = (ws_floats((long long)B * H * n, d, (long long)B * H) * sizeof(float) + 255) & ~(size_t)255;
+    return own + forward_tensor_workspace_bytes(B, H, n, d);
 }
 
 int launch_backward(const BackwardArgs& a) {

@@ -69,6 +69,11 @@ struct ForwardArgs {
     int window = 0;             // causal sliding window: a row sees its last `window` positions (0: all)
     const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
+    const void* k16 = nullptr;  // fp16 copy of k and its validity word, set by forward_tensor_prepass
+    const int* f16_ok = nullptr;
+    int precise_iters = 1;      // tensor-core kernel: CG iterations run with bf16 hi + lo operand pairs before the
+    int precise_iters_early = 4;   // switch to single fp16 operands (see lla_forward_params.cg_precise_iters); the
+                                // second value is for row tiles that end within the first 8 d positions
 };
 
 struct DecodeArgs {
@@ -133,7 +138,9 @@ int launch_head_rows(const ForwardArgs& a);
 int launch_forward_simt(const ForwardArgs& a);
 int launch_forward_tensor(const ForwardArgs& a);
 bool forward_tensor_supported(const ForwardArgs& a);
+int forward_tensor_prepass(ForwardArgs& a);    // fp16 copy of k into the workspace (no-op without room)
 size_t forward_tensor_scratch_bytes();         // d = 128 row-state scratch (0 if the device cannot be queried)
+size_t forward_tensor_workspace_bytes(int B, int H, int n, int d);   // that scratch + the fp16 copy of k (upper bound: kv heads = H)
 int launch_decode(const DecodeArgs& a);
 int launch_head_rows_decode(const DecodeArgs& a);
 bool decode_tensor_supported(const DecodeArgs& a);

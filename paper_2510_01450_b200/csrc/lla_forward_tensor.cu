@@ -29,6 +29,8 @@
 // The mathematics is the centred form described in lla_forward_simt.cu (same CG, same freeze rule).
 // All waits on mbarriers are bounded; a wait that expires sets LLA_STATUS_TIMEOUT and the block
 // leaves through the common exit (TMEM is released there).
+#include <cuda_fp16.h>
+
 #include <algorithm>
 #include <mutex>
 
@@ -50,7 +52,8 @@ constexpr int TC_NST_MAX = 4;
 constexpr int TC_ORDER_MAX = 256;    // launch-order table size (query tiles)
 constexpr int TC_SPLIT_MAX = 4;      // sweeps of at most this many key blocks run in split mode (see the compute role)
 
-enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4 };
+// SW_CG16: a CG sweep whose on-the-fly operands (P, U) are single fp16 values instead of bf16 hi + lo pairs
+enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4, SW_CG16 = 5 };
 
 // Shared-memory carve-up (bytes, from a 1024-byte aligned base), per head size D (64 or 128).
 // Operand tiles are stored as D/64 sub-tiles of 64 columns (128-byte rows, 128B swizzle) one after
@@ -81,6 +84,7 @@ struct TcCfg {
     static constexpr int SM_TOTAL = SM_MISC + 64;
     static constexpr int SM_ALLOC = SM_TOTAL + 1024;                              // slack for 1024-byte alignment
     static constexpr uint32_t IDESC_TS = sm100::make_idesc(TC_BR, D, 0, 1);   // ACC: A from TMEM, B MN-major, N = D
+    static constexpr uint32_t IDESC_TS16 = sm100::make_idesc(TC_BR, D, 0, 1, /*f16=*/1);   // same, both operands fp16
     static constexpr size_t SCRATCH_FLOATS_PER_SM = STATE_IN_SMEM ? 0 : 3 * (size_t)D * TC_BR;   // x, kbar, r
 };
 static_assert(TcCfg<64>::SM_ALLOC <= 227 * 1024 && TcCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
@@ -131,6 +135,22 @@ __device__ __forceinline__ void mma_ts_hilo_k64(uint32_t el, uint32_t d, uint32_
         "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3l], b3, %4, p;\n\t}"
         ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
 }
+// D[tmem] (+)= U[tmem] * B[smem] over 64 keys with U a single 16-bit operand: the compute threads leave the
+// 16-key steps 0, 1 at columns a, a + 8 and the steps 2, 3 at a + 32, a + 40 (each 32-key pass writes into
+// the columns it read its scores from).
+__device__ __forceinline__ void mma_ts_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a1, %2, 8; add.u32 a2, %2, 32; add.u32 a3, %2, 40;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
 // Shared-memory matrix descriptors (128-byte swizzle, tile base 1024-byte aligned).
 //   K-major:  rows of 128 bytes, 8-row groups 1024 bytes apart; a 16-element K step is +32 bytes.
 //   MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements; 8-row groups
@@ -147,32 +167,17 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_b
 }
 
 constexpr uint32_t IDESC_SS = make_idesc(TC_BR, TC_BC, 0, 0);   // S/A: A, B K-major; ACC uses make_idesc(128, D, 0, 1)
+constexpr uint32_t IDESC_SS16 = make_idesc(TC_BR, TC_BC, 0, 0, /*f16=*/1);   // the same products with both operands fp16
 
 // byte offset of the 16-byte chunk `chunk` (8 bf16) of row `row` in a swizzled 128 x 64 bf16 tile
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
-// Optional phase timing for tuning (compile with -DLLA_TC_TIMING; totals are added to prm.dbg).
-#ifdef LLA_TC_TIMING
-#define TC_T0(var) const long long var = clock64()
-#define TC_ACC(slot, var) do { if (prm.dbg) atomicAdd(prm.dbg + (slot), (unsigned long long)(clock64() - (var))); } while (0)
-#else
-#define TC_T0(var)
-#define TC_ACC(slot, var)
-#endif
-
-// Optional event trace of one block for tuning (-DLLA_TC_TRACE; (tag, block, clock) triples in prm.dbg).
-#ifdef LLA_TC_TRACE
-// each traced thread appends to its own region (role r: entries [r*4000, (r+1)*4000)), no atomics
-#define TC_EV_DECL(role) unsigned long long* ev_p_ = (prm.dbg && blockIdx.x == 0 && blockIdx.y == gridDim.y - 1 - LLA_TC_TRACE) ? prm.dbg + 1 + 3ull * 4000 * (role) : nullptr; int ev_n_ = 0
-#define TC_EV(tag, c) do { if (ev_p_ && ev_n_ < 4000) { ev_p_[3 * ev_n_] = (tag); ev_p_[3 * ev_n_ + 1] = (unsigned long long)(c); ev_p_[3 * ev_n_ + 2] = (unsigned long long)clock64(); ++ev_n_; } } while (0)
-#else
-#define TC_EV_DECL(role)
-#define TC_EV(tag, c)
-#endif
-
 struct TcParams {
-    unsigned long long* dbg;
     int n, nq, causal, head_rows, max_iters, first_tile;   // n keys; nq query rows at positions n - nq .. n - 1
+    int precise_iters;   // CG iterations whose operands are bf16 hi + lo pairs; later ones use single fp16 operands
+    int precise_iters_early;   // the same for the row tiles that end within the first 8 D positions
+    const int* f16_ok;   // device word written by the conversion pre-pass: nonzero = q and k fit the fp16 range and
+                         // the fp16 copy of k (tmK16) is valid; NULL or zero = every sweep in bf16
     float scale, lambda, tol;
     float* rho;
     float* stats;
@@ -193,7 +198,8 @@ struct TcParams {
 template <int D, typename TOut>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, TOut* __restrict__ out, const TcParams prm) {
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmK16,
+                  TOut* __restrict__ out, const TcParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     using Cfg = TcCfg<D>;
@@ -201,7 +207,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     constexpr int SM_Q = Cfg::SM_Q, SM_PHI = Cfg::SM_PHI, SM_PLO = Cfg::SM_PLO, SM_KV = Cfg::SM_KV;
     constexpr int SM_RED = Cfg::SM_RED, SM_FLAGS = Cfg::SM_FLAGS, SM_BAR = Cfg::SM_BAR, SM_MISC = Cfg::SM_MISC;
     constexpr int STAGE = Cfg::STAGE_BYTES, KBLK = Cfg::KBLK_BYTES;
-    constexpr uint32_t IDESC_TS = Cfg::IDESC_TS;
+    constexpr uint32_t IDESC_TS = Cfg::IDESC_TS, IDESC_TS16 = Cfg::IDESC_TS16;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bars = sbase + SM_BAR;
     auto bar = [&](int i) { return bars + 8u * i; };
@@ -241,6 +247,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int cbeg = (prm.causal && prm.window > 0) ? max(0, off + r0 + 1 - prm.window) / TC_BC : 0;
     const int nblk = cend - cbeg;                        // key blocks per sweep: cbeg .. cend - 1
     const bool split = nblk <= TC_SPLIT_MAX;
+    // Operand format of a sweep, fixed by its index alone so that every role knows it without being told:
+    // sweeps 0 (maxima), 1 (statistics) and the first precise_iters CG sweeps run on the bf16 inputs; every
+    // later sweep (the remaining CG sweeps and, if CG got that far, the output sweep) runs its Q K^T and P K^T
+    // products on fp16 copies of Q and K (one kind::f16 MMA takes both operands in the same 16-bit format).
+    // The values of the copies equal the bf16 inputs (the pre-pass checks the range).
+    // (tiles whose rows see fewer than 8 D keys converge more slowly and keep the pairs for more iterations)
+    const int precise = off + r0 + TC_BR <= 8 * D ? prm.precise_iters_early : prm.precise_iters;
+    const int f16_from = (prm.f16_ok && *prm.f16_ok && precise < (1 << 29)) ? precise + 2 : (1 << 30);
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
@@ -285,12 +299,13 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             uint32_t kit = 0;      // K blocks issued so far
             int pre = 0;           // blocks of the coming sweep already issued
             bool ok = true;
-            auto issue_k = [&](int c) {
+            auto issue_k = [&](int c, bool f16) {
                 const uint32_t s = kit % TC_NST;
                 if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag)) { ok = false; return; }
                 mbar_expect_tx(bar(B_KVFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, &tmK, bar(B_KVFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
+                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, f16 ? &tmK16 : &tmK, bar(B_KVFULL + s), 64 * sub,
+                                (cbeg + c) * TC_BC, kvh);
                 ++kit;
             };
             auto issue_v = [&](int c, uint32_t g) {
@@ -314,12 +329,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (kind == SW_OUT)
                     for (int c = 0; c < pre; ++c) issue_v(c, g0 + c);
                 for (int c = pre; c < nblk && ok; ++c) {
-                    issue_k(c);
+                    issue_k(c, (int)sweep >= f16_from);
                     if (ok && kind == SW_OUT) issue_v(c, g0 + c);
                 }
                 pre = 0;
                 if (kind != SW_OUT)
-                    for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c); ++pre; }
+                    for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c, (int)sweep + 1 >= f16_from); ++pre; }
             }
         }
     } else if (warp == 9) {
@@ -328,7 +343,6 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // tcgen05.mma issue is throttled to the execution rate, so the time an issuing warp spends
         // in barrier waits is tensor-pipe idle time: two warps (this one and warp 10) feed the pipe
         // and each one's waits hide behind the other's instructions.
-        TC_EV_DECL(0);
         const uint32_t el = elect_one();
         // broadcast through a shuffle so the compiler treats these as warp-uniform values and keeps
         // the MMA operands in uniform registers (otherwise every operand is moved there one by one)
@@ -340,20 +354,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint64_t pldesc = make_desc(sb_u + SM_PLO);
         uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it % NBUF)
         for (uint32_t sweep = 0; ok; ++sweep) {
-            TC_T0(t_c);
             if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
-            if (lane == 0) TC_ACC(11, t_c);
             const int kind = misc[1];
             if (kind == SW_DONE) break;
             tc_fence_after();
+            const uint32_t idesc = (int)sweep >= f16_from ? IDESC_SS16 : IDESC_SS;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
-                TC_T0(t_k);
                 if (!mbar_wait(bar(B_KVFULL + s), (it / TC_NST) & 1, abort_flag)) { ok = false; break; }
-                if (lane == 0) TC_ACC(8, t_k);
-                TC_T0(t_b);
                 if (!mbar_wait(bar(B_BUFFREE + b), (bu & 1) ^ 1, abort_flag)) { ok = false; break; }
-                if (lane == 0) TC_ACC(9, t_b);
                 tc_fence_after();
                 const uint64_t kdesc = make_desc(sb_u + SM_KV + s * STAGE);
                 const uint32_t s_tm = tm_u + b * 128, a_tm = s_tm + 64;
@@ -361,22 +370,22 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 // (sub-tiles are QSUB_BYTES / KSUB_BYTES apart: 1024 / 512 descriptor units)
 #pragma unroll
                 for (int sub = 0; sub < KSUB; ++sub)
-                    mma_ss_k64(el, s_tm, qdesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), IDESC_SS, sub > 0);
-                if (kind == SW_CG || kind == SW_OUT) {
+                    mma_ss_k64(el, s_tm, qdesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), idesc, sub > 0);
+                if (kind == SW_CG || kind == SW_OUT || kind == SW_CG16) {
 #pragma unroll
                     for (int sub = 0; sub < KSUB; ++sub)
-                        mma_ss_k64(el, a_tm, phdesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), IDESC_SS, sub > 0);
+                        mma_ss_k64(el, a_tm, phdesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), idesc, sub > 0);
+                    if (kind != SW_CG16) {     // second half of the operand pair
 #pragma unroll
-                    for (int sub = 0; sub < KSUB; ++sub)
-                        mma_ss_k64(el, a_tm, pldesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), IDESC_SS, 1);
+                        for (int sub = 0; sub < KSUB; ++sub)
+                            mma_ss_k64(el, a_tm, pldesc + sub * (Cfg::QSUB_BYTES >> 4), kdesc + sub * (Cfg::KSUB_BYTES >> 4), idesc, 1);
+                    }
                 }
                 tc_commit_el(el, bar(B_SAFULL + b));
-                if (lane == 0) TC_EV(11, it);
             }
         }
     } else if (warp == 10) {
         // ================================ MMA issuer 2: ACC += U B ================================
-        TC_EV_DECL(1);
         const uint32_t el = elect_one();
         const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
         const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
@@ -388,20 +397,17 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (kind == SW_DONE) break;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
-                TC_T0(t_u);
                 if (!mbar_wait(bar(B_UFULL + b), bu & 1, abort_flag)) { ok = false; break; }
-                if (lane == 0) TC_ACC(10, t_u);
                 if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), (c / TC_NST) & 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                if (lane == 0) TC_EV(20, it);
                 if (kind != SW_MAX) {
                     const uint32_t bsm = sb_u + SM_KV + s * STAGE + (kind == SW_OUT ? KBLK : 0);
                     // B = the K (or V) block read MN-major, N = D: 64-wide column groups are one sub-tile apart
-                    mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS, c > 0);
+                    if (kind == SW_CG16) mma_ts_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS16, c > 0);
+                    else mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS, c > 0);
                     tc_commit_el(el, bar(B_KVEMPTY + s));
                     tc_commit_el(el, bar(B_BUFFREE + b));
                     if (c == nblk - 1) tc_commit_el(el, bar(B_ACCFULL));
-                    if (lane == 0) TC_EV(21, it);
                 } else if (el) {
                     mbar_arrive(bar(B_KVEMPTY + s));
                     mbar_arrive(bar(B_BUFFREE + b));
@@ -410,9 +416,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
     } else {
         // ================================ compute warps ================================
-        TC_T0(t_all);
         const int quad = warp & 3, half = warp >> 2;
-        TC_EV_DECL(2 + half);
         const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
         const int row = r0 + lrow;
         const int L = prm.causal ? off + row + 1 : n;
@@ -480,9 +484,67 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         };
 
+        // the same vector as an fp16 hi + lo pair (the output sweep's y once the sweeps run on fp16 operands)
+        auto write_operand16_pair = [&](const float* vec) {
+#pragma unroll
+            for (int ch = 0; ch < NCOL / 8; ++ch) {
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float a = vec[ch * 8 + 2 * e], b = vec[ch * 8 + 2 * e + 1];
+                    const __half2 h2 = __floats2half2_rn(a, b);
+                    const float2 f = __half22float2(h2);
+                    const __half2 l2 = __floats2half2_rn(a - f.x, b - f.y);
+                    hi[e] = *reinterpret_cast<const uint32_t*>(&h2);
+                    lo[e] = *reinterpret_cast<const uint32_t*>(&l2);
+                }
+                const uint32_t off = oper_off(ch);
+                *reinterpret_cast<uint4*>(smem + SM_PHI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(smem + SM_PLO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+        };
+        // Q tile: bf16 as loaded, or fp16 once the sweeps have switched format (converted in place by
+        // convert_q, each thread its own chunks, between two sweeps when no MMA reads the tile)
+        bool q_is_f16 = false;
+        auto q_elem = [&](const uint32_t* qw, int e) -> float {
+            if (q_is_f16) {
+                const __half2 h2 = *reinterpret_cast<const __half2*>(&qw[e >> 1]);
+                return (e & 1) ? __high2float(h2) : __low2float(h2);
+            }
+            return (e & 1) ? __uint_as_float(qw[e >> 1] & 0xFFFF0000u) : __uint_as_float(qw[e >> 1] << 16);
+        };
+        auto convert_q = [&]() {
+#pragma unroll
+            for (int ch = 0; ch < NCOL / 8; ++ch) {
+                uint4* qp = reinterpret_cast<uint4*>(smem + SM_Q + oper_off(ch));
+                const uint4 qraw = *qp;
+                const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
+                uint32_t h[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    h[e] = pack_f16(__uint_as_float(qw[e] << 16), __uint_as_float(qw[e] & 0xFFFF0000u));
+                *qp = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+            q_is_f16 = true;
+        };
+        // the same vector as one fp16 value per entry, scaled by the power of two sc (see write_p)
+        auto write_operand16 = [&](const float* vec, float sc) {
+#pragma unroll
+            for (int ch = 0; ch < NCOL / 8; ++ch) {
+                uint32_t h[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) h[e] = pack_f16(vec[ch * 8 + 2 * e] * sc, vec[ch * 8 + 2 * e + 1] * sc);
+                *reinterpret_cast<uint4*>(smem + SM_PHI + oper_off(ch)) = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+        };
+
         const float c1 = prm.scale * 1.4426950408889634f;    // scores in log2 units
         float mx2 = -INFINITY, omega = 0.f, inv_omega = 0.f, ridge = 0.f, den = 0.f;
         float abar = 0.f;                                     // kbar.p (CG) or kbar.y (output)
+        // fp16 sweeps: the search direction is stored as p * psc with psc a power of two that brings |p| to
+        // [1, 2.83), so that its entries and u = w (a - abar) sit in the middle of the fp16 range whatever the
+        // scale of the right-hand side; pn2 tracks |p|^2 through the recurrence |p'|^2 = |r'|^2 + beta^2 |p|^2
+        float pn2 = 0.f, psc = 1.f, ipsc = 1.f;
         uint32_t blk = 0;                                     // global block counter (buffer = blk & 1)
         bool ok = true;
 
@@ -497,27 +559,21 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             float part = 0.f;                                 // omega / den partial, or max
             if (kind == SW_MAX) part = -INFINITY;
             const uint64_t c1c1 = pk2(c1, c1), nmx = pk2(-mx2, -mx2);
-            const uint64_t nab = pk2(-abar, -abar), oab = pk2(1.f + abar, 1.f + abar), neg1 = pk2(-1.f, -1.f);
+            const float ab_s = kind == SW_CG16 ? abar * psc : abar;
+            const uint64_t nab = pk2(-ab_s, -ab_s), oab = pk2(1.f + abar, 1.f + abar), neg1 = pk2(-1.f, -1.f);
             uint64_t part2 = pk2(0.f, 0.f);
             for (int c = 0; c < nblk; ++c, ++blk) {
                 if (!split && (int)(blk & 1) != half) continue;
                 const uint32_t b = blk % TC_NBUF;
-                TC_T0(t_w);
-                if (lane == 0 && quad == 0) TC_EV(30 + half, blk);
                 if (!mbar_wait(bar(B_SAFULL + b), (blk / TC_NBUF) & 1, abort_flag)) { ok = false; return part; }
-                if (lane == 0 && quad == 0) TC_EV(32 + half, blk);
-                if (tid == 0) TC_ACC(0, t_w);
                 tc_fence_after();
 #pragma unroll 1
                 for (int h = split ? half : 0; h < (split ? half + 1 : 2); ++h) {
-                    TC_T0(t_l);
                     const uint32_t s_addr = tmem + lane_addr + b * 128 + 32 * h;
                     uint32_t sv[32], av[32];
                     tmem_ld32(s_addr, sv);
-                    if (kind == SW_CG || kind == SW_OUT) tmem_ld32(s_addr + 64, av);
+                    if (kind == SW_CG || kind == SW_OUT || kind == SW_CG16) tmem_ld32(s_addr + 64, av);
                     tc_wait_ld();
-                    if (tid == 0) TC_ACC(1, t_l);
-                    TC_T0(t_m);
                     // keys jfirst <= e < jlim of this half block are visible.  Only the diagonal blocks and a
                     // window's first blocks hide any: there the hidden scores are overwritten with a large negative
                     // number, whose weight is exactly zero, so the loops below carry no mask
@@ -532,14 +588,25 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
                             part = fmaxf(part, __uint_as_float(sv[e]) * c1);
+                    } else if (kind == SW_CG16) {
+                        // u = w (a - abar) as one fp16 value per key: 16 keys per k-step in 8 columns
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e2 = 0; e2 < 16; ++e2) {
+                            const uint64_t t2 = fma2(pk2(__uint_as_float(sv[2 * e2]), __uint_as_float(sv[2 * e2 + 1])), c1c1, nmx);
+                            float t0, t1;
+                            upk2(t2, t0, t1);
+                            const uint64_t u2 = mul2(pk2(ex2f(t0), ex2f(t1)),
+                                                     add2(pk2(__uint_as_float(av[2 * e2]), __uint_as_float(av[2 * e2 + 1])), nab));
+                            float u0, u1;
+                            upk2(u2, u0, u1);
+                            pk[e2] = pack_f16(u0, u1);
+                        }
+                        tmem_st16(s_addr, pk);
                     } else {
                         uint32_t pk[32];
 #pragma unroll
                         for (int e2 = 0; e2 < 16; ++e2) {
-#ifdef LLA_EXP_NO_MATH
-                            pk[e2] = sv[2 * e2]; pk[16 + e2] = sv[2 * e2 + 1];
-                            continue;
-#endif
                             const uint64_t t2 = fma2(pk2(__uint_as_float(sv[2 * e2]), __uint_as_float(sv[2 * e2 + 1])), c1c1, nmx);
                             float t0, t1;
                             upk2(t2, t0, t1);
@@ -555,10 +622,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             const int ks = e2 >> 3, e = e2 & 7;
                             pk[ks * 16 + e] = split_bf16x2(u0, u1, pk[ks * 16 + 8 + e]);
                         }
-                        if (tid == 0) TC_ACC(2, t_m);
-                        TC_T0(t_s);
                         tmem_st32(s_addr, pk);
-                        if (tid == 0) TC_ACC(3, t_s);
                     }
                 }
                 if (kind != SW_MAX) tc_wait_st();
@@ -566,7 +630,6 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised atomics
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_UFULL + b));
-                if (lane == 0 && quad == 0) TC_EV(34 + half, blk);
             }
             if (kind != SW_MAX) {
                 float p0, p1;
@@ -578,9 +641,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // read this thread's NCOL ACC columns after the sweep's last MMA
         uint32_t acc_uses = 0;
         auto read_acc = [&](float* dst) {
-            TC_T0(t_a);
             if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag)) { ok = false; return; }
-            if (tid == 0) TC_ACC(4, t_a);
             ++acc_uses;
             tc_fence_after();
 #pragma unroll
@@ -593,7 +654,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             tc_fence_before();
         };
+        int sweeps_started = 0;
         auto start_sweep = [&](int kind) {
+            if (sweeps_started >= f16_from && !q_is_f16) convert_q();
+            ++sweeps_started;
             if (tid == 0) misc[1] = kind;
             fence_proxy_async();       // operand tiles written with ordinary stores -> visible to the MMA
             __syncwarp();
@@ -613,6 +677,20 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float rr = 0.f, stop = 0.f;
         int its = 0;
         bool active = false;
+        // P operand for CG iteration t_next: bf16 hi + lo for the first precise_iters iterations, one fp16 after
+        // (the products of an iteration enter x and r scaled by |p|, which has fallen by then: the coarser
+        // operands of the later iterations cost no accuracy that the early ones have not already spent)
+        auto write_p = [&](int t_next) {
+            if (t_next + 2 >= f16_from) {
+                const int e2 = (int)((__float_as_uint(pn2) >> 23) & 0xffu) - 127;      // floor(log2 |p|^2)
+                const int k = max(-100, min(100, -(e2 >> 1)));
+                psc = __uint_as_float((uint32_t)(127 + k) << 23);
+                ipsc = __uint_as_float((uint32_t)(127 - k) << 23);
+                write_operand16(p, psc);
+            } else {
+                write_operand(p);
+            }
+        };
 
         // ---- sweep 0: row maxima ----
         start_sweep(SW_MAX);
@@ -638,7 +716,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const float qv = (e & 1) ? __uint_as_float(qw[e >> 1] & 0xFFFF0000u) : __uint_as_float(qw[e >> 1] << 16);
+                        const float qv = q_elem(qw, e);
                         const int col = ch * 8 + e;
                         const float kb = acc[col] * inv_omega;
                         kbs[(c0 + col) * TC_BR + lrow] = kb;
@@ -654,39 +732,33 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 abar = pair_sum(ab_p);
                 stop = prm.tol * prm.tol * rr;
                 active = row_ok && rr > 0.f;
-                write_operand(p);
+                pn2 = rr;
+                write_p(0);
             }
         }
         // ---- conjugate gradients (Algorithm 2) ----
         for (int t = 0; ok && t < prm.max_iters; ++t) {
             active = active && rr > stop;
-#ifdef LLA_EXP_FIXED
-            (void)group_any(active);     // tuning builds: always run max_iters sweeps
-#else
             if (!group_any(active)) break;
-#endif
-            if (lane == 0 && quad == 0) TC_EV(45, t);
-            start_sweep(SW_CG);
-            if (lane == 0 && quad == 0) TC_EV(46, t);
-            sweep(SW_CG);
-            if (lane == 0 && quad == 0) TC_EV(47, t);
+            const bool cheap = t + 2 >= f16_from;
+            start_sweep(cheap ? SW_CG16 : SW_CG);
+            sweep(cheap ? SW_CG16 : SW_CG);
             float ap[NCOL];
             if (ok) read_acc(ap);
             if (!ok) break;
-            if (lane == 0 && quad == 0) TC_EV(40, t);
             // (the loops below keep four independent partial sums and move the row-vector state in
             //  batches of eight so that the loads overlap: two warps per scheduler hide no latency)
             float pp[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
+            const float acc_scale = cheap ? inv_omega * ipsc : inv_omega;
+#pragma unroll
             for (int e = 0; e < NCOL; ++e) {
-                ap[e] = fmaf(ap[e], inv_omega, ridge * p[e]);
+                ap[e] = fmaf(ap[e], acc_scale, ridge * p[e]);
                 pp[e & 3] = fmaf(p[e], ap[e], pp[e & 3]);
             }
             const float pap = pair_sum((pp[0] + pp[1]) + (pp[2] + pp[3]));
-            if (lane == 0 && quad == 0) TC_EV(41, t);
             if (active && !(pap > 0.f)) active = false;
             const float alpha = active ? rr / pap : 0.f;
-            if (lane == 0 && quad == 0) TC_EV(48, t);
             float r2[4] = {0.f, 0.f, 0.f, 0.f}, kr[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int e0 = 0; e0 < NCOL; e0 += 8) {
@@ -713,20 +785,17 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             // ||r_new||^2 and kbar . r_new in one exchange; kbar . p_new follows from the recurrence
             float rr2 = (r2[0] + r2[1]) + (r2[2] + r2[3]), kbr = (kr[0] + kr[1]) + (kr[2] + kr[3]);
-            if (lane == 0 && quad == 0) TC_EV(49, t);
             pair_sum2(rr2, kbr);
-            if (lane == 0 && quad == 0) TC_EV(42, t);
             if (active) {
                 const float beta = rr2 / rr;
 #pragma unroll
                 for (int e = 0; e < NCOL; ++e) p[e] = fmaf(beta, p[e], ap[e]);
                 abar = fmaf(beta, abar, kbr);
+                pn2 = fmaf(beta * beta, pn2, rr2);
                 rr = rr2;
                 ++its;
             }
-            if (lane == 0 && quad == 0) TC_EV(43, t);
-            write_operand(p);
-            if (lane == 0 && quad == 0) TC_EV(44, t);
+            write_p(t + 1);
         }
         const bool at_cap = active && rr > stop;
         // ---- output sweep ----
@@ -751,7 +820,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const uint32_t qw[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float qv = (e & 1) ? __uint_as_float(qw[e >> 1] & 0xFFFF0000u) : __uint_as_float(qw[e >> 1] << 16);
+                    const float qv = q_elem(qw, e);
                     const int col = ch * 8 + e;
                     const float kb = kbs[(c0 + col) * TC_BR + lrow];
                     y[col] = xs[(c0 + col) * TC_BR + lrow];
@@ -761,7 +830,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             abar = pair_sum(yb_p);
             gfac = 1.f + pair_sum(g_p);
-            write_operand(y);
+            if (sweeps_started >= f16_from) write_operand16_pair(y);
+            else write_operand(y);
             start_sweep(SW_OUT);
             const float part = sweep(SW_OUT);
             float o[NCOL];
@@ -795,17 +865,6 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
         if (ok) start_sweep(SW_DONE);
-        if (tid == 0) TC_ACC(5, t_all);
-#ifdef LLA_TC_TIMING
-        if (tid == 0 && prm.dbg) {   // per-block duration and end time (tuning builds)
-            const size_t idx = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
-            unsigned long long gt;
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-            prm.dbg[32 + 2 * idx] = (unsigned long long)(clock64() - t_all);
-            prm.dbg[33 + 2 * idx] = gt;
-        }
-#endif
-        if (tid == 0) { TC_T0(t_one); TC_ACC(6, t_one - 1); (void)nblk; }
     }
 
     // ================================ common exit ================================
@@ -822,9 +881,42 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (tid == 0 && *abort_flag && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
 }
 
+// Pre-pass of the fp16 sweeps: writes an fp16 copy of k and clears *ok if an entry of k or q lies outside
+// the range in which that copy is faithful (magnitude above 60000; bf16 values below the fp16 subnormal
+// spacing simply round, an absolute change under 3e-8).  Eight elements per thread and step.
+__global__ void __launch_bounds__(256)
+f16_copy_kernel(const uint4* __restrict__ k, uint4* __restrict__ k16, size_t k_vec, const uint4* __restrict__ q,
+                size_t q_vec, int* __restrict__ ok) {
+    bool bad = false;
+    const size_t stride = (size_t)gridDim.x * blockDim.x, t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (size_t i = t0; i < k_vec; i += stride) {
+        const uint4 raw = k[i];
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        uint32_t h[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float a = __uint_as_float(w[e] << 16), b = __uint_as_float(w[e] & 0xFFFF0000u);
+            bad |= !(fabsf(a) <= 60000.f) || !(fabsf(b) <= 60000.f);
+            h[e] = pack_f16(a, b);
+        }
+        k16[i] = make_uint4(h[0], h[1], h[2], h[3]);
+    }
+    for (size_t i = t0; i < q_vec; i += stride) {
+        const uint4 raw = q[i];
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            bad |= !(fabsf(__uint_as_float(w[e] << 16)) <= 60000.f) || !(fabsf(__uint_as_float(w[e] & 0xFFFF0000u)) <= 60000.f);
+    }
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) *ok = 0;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
+size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+// bytes of the fp16 copy of k plus its status word
+size_t f16_copy_bytes(size_t k_elems) { return round256(k_elems * 2) + 256; }
 // Per-device scratch for the D = 128 kernel: one slot per SM id, shared by every launch on the device.
 // A block of this kernel fills an SM (shared memory), so two blocks never use one slot at a time,
 // whichever launches or streams they come from.
@@ -878,22 +970,28 @@ int launch_t(const ForwardArgs& a) {
     const int first_tile = a.causal ? hr / TC_BR : 0;
     const int tiles = (a.nq + TC_BR - 1) / TC_BR - first_tile;
     if (tiles <= 0) return LLA_OK;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mk16;
     const int BH = a.B * a.H;
     if (!make_map_bf16(&mq, a.q, BH, a.nq, D, TC_BR) || !make_map_bf16(&mk, a.k, BH / a.kv_group, a.n, D, TC_BC) ||
         !make_map_bf16(&mv, a.v, BH / a.kv_group, a.n, D, TC_BC))
         return LLA_ERR_CUDA;
+    mk16 = mk;
     TcParams prm;
     prm.n = a.n; prm.nq = a.nq; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
+    prm.precise_iters = a.precise_iters;
+    prm.precise_iters_early = a.precise_iters_early;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
     prm.rhs = a.rhs; prm.sol = a.sol;
     prm.H = a.H; prm.kv_group = a.kv_group > 0 ? a.kv_group : 1;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
-    prm.dbg = nullptr;
     prm.scratch = nullptr;
     prm.scratch_slots = 0;
+    prm.f16_ok = nullptr;
+    // the caller's workspace is cut into the D = 128 row-state slots (if it holds them) and the fp16 copy of k
+    char* ws = static_cast<char*>(a.workspace);
+    size_t ws_left = a.workspace ? a.workspace_bytes : 0;
     prm.window = a.causal ? a.window : 0;
     tile_order(prm, tiles, first_tile, a.n, a.n - a.nq, D, a.causal, prm.window);
     if constexpr (!Cfg::STATE_IN_SMEM) {
@@ -904,17 +1002,25 @@ int launch_t(const ForwardArgs& a) {
         const size_t need = (size_t)prm.scratch_slots * Cfg::SCRATCH_FLOATS_PER_SM * sizeof(float);
         // the caller's workspace if it is large enough (then nothing is allocated, but two calls that may
         // run at the same time must not share it), else the library's own per-device buffer
-        if (a.workspace && a.workspace_bytes >= need) prm.scratch = static_cast<float*>(a.workspace);
-        else prm.scratch = scratch_for_device(need);
+        if (ws && ws_left >= need) {
+            prm.scratch = reinterpret_cast<float*>(ws);
+            ws += round256(need);
+            ws_left -= std::min(ws_left, round256(need));
+        } else {
+            prm.scratch = scratch_for_device(need);
+        }
         if (!prm.scratch) return LLA_ERR_CUDA;
     }
-#if defined(LLA_TC_TIMING) || defined(LLA_TC_TRACE)
-    prm.dbg = (unsigned long long*)a.workspace;   // tuning builds only: caller passes a zeroed buffer
-#endif
+    // fp16 sweeps: only with the copy of k that forward_tensor_prepass made; without it every sweep runs on
+    // the bf16 inputs
+    if (a.k16 && a.f16_ok) {
+        if (!make_map_bf16(&mk16, a.k16, BH / a.kv_group, a.n, D, TC_BC, CU_TENSOR_MAP_DATA_TYPE_FLOAT16)) return LLA_ERR_CUDA;
+        prm.f16_ok = a.f16_ok;
+    }
     auto kern = forward_tc_kernel<D, TOut>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
     dim3 grid(BH, tiles);
-    kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, (TOut*)a.out, prm);
+    kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, mk16, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -925,7 +1031,35 @@ size_t forward_tensor_scratch_bytes() {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return (size_t)2 * sms * TcCfg<128>::SCRATCH_FLOATS_PER_SM * sizeof(float);
+    return round256((size_t)2 * sms * TcCfg<128>::SCRATCH_FLOATS_PER_SM * sizeof(float));
+}
+
+size_t forward_tensor_workspace_bytes(int B, int H, int n, int d) {
+    return (d == 128 ? forward_tensor_scratch_bytes() : 0) + f16_copy_bytes((size_t)B * H * n * d);
+}
+
+// Enqueues the fp16 copy of k (and the range check of q and k) when the tail of the caller's workspace has
+// room for it, and records where it is in `a`; the head of the workspace is left to the D = 128 row state.
+int forward_tensor_prepass(ForwardArgs& a) {
+    a.k16 = nullptr;
+    a.f16_ok = nullptr;
+    if (!forward_tensor_supported(a) || !a.workspace) return LLA_OK;
+    if (std::min(a.precise_iters, a.precise_iters_early) >= (1 << 29)) return LLA_OK;
+    const size_t head = a.d == 128 ? forward_tensor_scratch_bytes() : 0;
+    const size_t k_elems = (size_t)(a.B * a.H / a.kv_group) * a.n * a.d;
+    if (a.workspace_bytes < head + f16_copy_bytes(k_elems)) return LLA_OK;
+    char* ws = static_cast<char*>(a.workspace) + head;
+    uint4* k16 = reinterpret_cast<uint4*>(ws);
+    int* okw = reinterpret_cast<int*>(ws + round256(k_elems * 2));
+    LLA_CUDA_TRY(cudaMemsetAsync(okw, 1, sizeof(int), a.stream));
+    const size_t k_vec = k_elems / 8, q_vec = (size_t)a.B * a.H * a.nq * a.d / 8;
+    const unsigned blocks = (unsigned)std::min<size_t>((k_vec + 255) / 256, 148 * 8);
+    f16_copy_kernel<<<blocks, 256, 0, a.stream>>>(static_cast<const uint4*>(a.k), k16, k_vec, static_cast<const uint4*>(a.q), q_vec,
+                                                   okw);
+    LLA_CUDA_TRY(cudaGetLastError());
+    a.k16 = k16;
+    a.f16_ok = okw;
+    return LLA_OK;
 }
 
 bool forward_tensor_supported(const ForwardArgs& a) {

@@ -141,6 +141,21 @@ __device__ __forceinline__ uint32_t split_bf16x2(float a, float b, uint32_t& lo)
     lo = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
     return hi;
 }
+// 16 consecutive TMEM columns of this thread's lane <- registers
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+// {lo16: fp16(a), hi16: fp16(b)}, round to nearest, values beyond the fp16 range saturate to the largest finite one
+__device__ __forceinline__ uint32_t pack_f16(float a, float b) {
+    uint32_t r;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+    return r;
+}
 // {hi16: bf16(a), lo16: bf16(b)}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     uint32_t r;
@@ -148,8 +163,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return r;
 }
 
-constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+// kind::f16 instruction descriptor: fp32 accumulator, both operands bf16 (f16 = 0) or both fp16 (f16 = 1).
+// The two format fields are set alike: an MMA with an fp16 A operand and a bf16 B operand raised "illegal
+// instruction" on B200.
+constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn, int f16 = 0) {
+    return (1u << 4) | (f16 ? 0u : (1u << 7) | (1u << 10)) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
@@ -190,14 +208,15 @@ inline bool make_map_bf16_64(CUtensorMap* map, const void* base, int outer, int 
 
 // bf16 [outer][rows][cols] (cols a multiple of 64), box = 64 columns x box_rows rows, 128B swizzle:
 // one copy per 64-column sub-tile, x coordinate 64 * sub.
-inline bool make_map_bf16(CUtensorMap* map, const void* base, int outer, int rows, int cols, int box_rows) {
+inline bool make_map_bf16(CUtensorMap* map, const void* base, int outer, int rows, int cols, int box_rows,
+                          CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)outer};
     const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)rows * cols * 2};
     const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+    return enc(map, dtype, 3, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

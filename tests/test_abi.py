@@ -145,11 +145,14 @@ def test_validation_of_the_position_options(lib):
     assert bwd(workspace=0x10010) == 3             # not 256-byte aligned
     assert bwd(kv_heads=3) == 1
     assert bwd(impl=7) == 1
-    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == 4 * 4 * 256 * (4 * 64 + 8)
+    # the pass's own vectors, then the scratch of the forward's CG kernel that it runs (fp16 copy of k + a status word)
+    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == 4 * 4 * 256 * (4 * 64 + 8) + 4 * 256 * 64 * 2 + 256
 
 
 def test_workspace_and_split_arithmetic(lib):
-    assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == 0
+    # tensor-core forward: fp16 copy of k + a status word (d = 128 adds per-SM slots, which need the device's SM count)
+    assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == 4 * 8 * 1024 * 64 * 2 + 256
+    assert binding.lla_forward_workspace_bytes(1, 1, 256, 16, 16, in_dtype=binding.LLA_F32) == 0
     # unsplit: optional record buffer for the two-kernel tensor-core path (bf16, d = 64), else none
     assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=1) == 4 * 2 * 4 * (2 * 64 * 64 + 132)
     assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, in_dtype=binding.LLA_F32, splits=1) == 0

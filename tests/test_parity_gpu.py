@@ -14,7 +14,7 @@ import torch
 
 from paper_2510_01450_b200 import binding as L
 from paper_2510_01450_b200 import inputs
-from tests.gpu_util import LLA_DT, dev, forward, row_err, stream_ptr
+from tests.gpu_util import LLA_DT, dev, elem_err, forward, row_err, stream_ptr
 
 pytestmark = pytest.mark.gpu
 
@@ -50,6 +50,7 @@ def test_config2_bf16_full(oracle, impl):
     got = forward(w, q, k, v, out_dtype="f32", impl=impl, device_status=status)
     err = row_err(got, ref)
     assert err.max() <= TOL_BF16, err.max()
+    assert elem_err(got, ref).max() <= TOL_BF16
     st = status.cpu().numpy()
     assert st[L.STATUS_ROWS_AT_CAP] == 0 and st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
     # the plain entry point (bf16 output)
@@ -328,6 +329,43 @@ def test_ridge_variants_decode(oracle, dtype, d):
                         out_dtype=L.LLA_F32, splits=1, lambda_units=dlam, ridge_mode=mode, stream=stream_ptr())
         torch.cuda.synchronize()
         assert row_err(out.cpu().numpy(), ref).max() <= tol, name
+
+
+@pytest.mark.parametrize("d,n", [(64, 1100), (128, 900)])
+def test_operand_precision_modes_and_missing_workspace(oracle, d, n):
+    # the CG sweeps' on-the-fly operands: bf16 pairs throughout, fp16 from the first iteration, the default mix,
+    # and the default without a workspace (no fp16 copy of k: pairs throughout, bit-identical to the first)
+    w = inputs.CONFIGS[2 if d == 64 else 4].shrink(B=1, H=2, n=n)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    outs = {}
+    for name, kw in (("pairs", dict(cg_precise_iters=L.LLA_CG_PRECISE_ALL)), ("fp16", dict(cg_precise_iters=L.LLA_CG_PRECISE_NONE)),
+                     ("three", dict(cg_precise_iters=3)), ("default", {}), ("no_ws", dict(workspace=None, workspace_bytes=0))):
+        outs[name] = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, device_status=status, **kw)
+        assert row_err(outs[name], ref).max() <= TOL_BF16, name
+        assert elem_err(outs[name], ref).max() <= TOL_BF16, name
+        assert status.cpu().tolist()[L.STATUS_TIMEOUT] == 0
+    assert np.array_equal(outs["pairs"], outs["no_ws"])      # same arithmetic, same bits
+    assert not np.array_equal(outs["pairs"], outs["fp16"])
+    # fewer precise iterations cost accuracy, never more than a few 1e-4
+    assert row_err(outs["pairs"], ref).max() <= 2.5e-4
+    assert row_err(outs["fp16"], ref).max() <= 1.2e-3
+
+
+def test_values_beyond_the_fp16_range_fall_back_to_pairs(oracle):
+    # a key entry of 7e4 cannot be held in fp16: the pre-pass notices and every sweep of the call runs on the bf16
+    # inputs.  The entry sits in the last key, which only the last row sees (that row's system is hopelessly
+    # ill-conditioned and is left out of the comparison).
+    w = inputs.CONFIGS[2].shrink(B=1, H=1, n=600)
+    q, k, v = inputs.make_prefill(w)
+    k = k.copy()
+    k[0, 0, w.n - 1, 3] = inputs.round_to_bf16(np.float32([7.0e4]))[0]
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    got = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR)
+    pairs = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, cg_precise_iters=L.LLA_CG_PRECISE_ALL)
+    assert np.array_equal(got[..., :-1, :], pairs[..., :-1, :])
+    assert row_err(got[..., :-1, :], ref[..., :-1, :]).max() <= TOL_BF16
 
 
 def test_forward_d128_with_caller_workspace(oracle):
