@@ -37,8 +37,8 @@ L2_BYTES = 126e6
 # (traffic is per head: Q, K, V once).
 NCU_TRAFFIC = {
     2: (12.68e6, "profiles/forward_tc_kernel_cfg2.md"),
-    3: (None, None),
-    4: (None, None),
+    3: (4 * 17.06e6, "profiles/forward_tc_kernel_cfg3.md (8 of 32 units captured, x 4)"),
+    4: (8 * (33.98e6 + 5.35e6), "profiles/forward_tc_kernel_cfg4.md (2 of 16 heads captured, x 8)"),
 }
 NCU_DECODE_TRAFFIC = (1.188e9 + 27.8e6 + 34.3e6, "profiles/decode_tc_kernel_cfg5.md")
 
@@ -255,7 +255,7 @@ class Prefill:
         w = self.w
         fl = algorithmic_flops(w, self.iters, iterative_only=True)
         tf = fl / (ms_kernel * 1e-3) / 1e12
-        traffic, src = NCU_TRAFFIC.get(int(w.name[3]), (None, None))
+        traffic, src = NCU_TRAFFIC.get(int(w.name[3]), (None, None)) if w.name in [c.name for c in inputs.CONFIGS.values()] else (None, None)
         c = clk.summary()
         return {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": tf / peaks["bf16_tflops"], "traffic": traffic, "traffic_source": src,
@@ -323,6 +323,8 @@ def run_ours(args):
     peaks = load_peaks()
     base = inputs.CONFIGS[args.workload]
     w = base.shrink(seed=base.seed + 1000 * rank)
+    if args.heads > 0:
+        w = w.shrink(H=args.heads, name=f"{base.name}_H{args.heads}")
     samplers = []
 
     # ---- headline: device-resident throughput of the whole forward step ----
@@ -552,6 +554,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", type=int, choices=[2, 3, 4], default=HEADLINE,
                     help="prefill workload of the headline (default: the largest, n=16384, d=128)")
+    ap.add_argument("--heads", type=int, default=0,
+                    help="profiling aid: run the headline workload with this many heads (a small case of the same "
+                         "kernel for an ncu capture; the line's config shows it)")
     ap.add_argument("--no-legs", action="store_true", help="skip the other prefill workloads")
     ap.add_argument("--no-decode", action="store_true", help="skip the decode measurement")
     ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass measurement")

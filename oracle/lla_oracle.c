@@ -14,7 +14,7 @@
  *   w_j    = exp(scale * <q_i, k_j>)     kernel weight (Section 3.2, W=exp(QK^T/h),
  *                                        scale = 1/h)
  *   z_j    = k_j - q_i
- *   omega  = sum_j w_j                   (spec name: s0)
+ *   omega  = sum_j w_j                   (also written s0)
  *   mu     = sum_j w_j z_j               (s1)
  *   Sigma  = sum_j w_j z_j z_j^T + lambda I   (S2)
  *   rho    = Sigma^{-1} mu               (dense Cholesky, no iteration)

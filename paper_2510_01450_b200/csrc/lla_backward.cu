@@ -873,7 +873,7 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
                 if (b <= a) S[a * LDS + b] = acc[x][y] - kb[a] * kb[b] + (a == b ? eps : 0.0);
             }
     }
-    const bool okf = block_ldlt_solve<D>(S, LDS, rhs, D LDLT_NOARG, 2, D);
+    const bool okf = block_ldlt_solve<D>(S, LDS, rhs, D, 2, D);
     if (!okf && tid == 0 && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
     const double* y = rhs;
     const double* t = rhs + D;

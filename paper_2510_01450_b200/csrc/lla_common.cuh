@@ -224,18 +224,6 @@ __device__ __forceinline__ double fast_rcp1(double x) {
     return r;
 }
 
-// Optional phase timing for tuning (-DLLA_HR_TIMING): clock totals of thread 0 go to tst[phase].
-#ifdef LLA_HR_TIMING
-#define LDLT_TARG , int* tst = nullptr
-#define LDLT_NOARG , nullptr
-#define LDLT_T0 long long lt_ = clock64()
-#define LDLT_T(ph) do { if (threadIdx.x == 0 && tst) { const long long now_ = clock64(); atomicAdd(tst + (ph), (int)((now_ - lt_) >> 4)); lt_ = now_; } } while (0)
-#else
-#define LDLT_TARG
-#define LDLT_NOARG
-#define LDLT_T0
-#define LDLT_T(ph)
-#endif
 
 // (i): factorise the NB x NB diagonal block at c0 (called by one full warp).  The reciprocal of
 // pivot c is left in S[c][c + 1], an element of the unused upper triangle (lds >= D + 1).
@@ -267,11 +255,10 @@ __device__ __forceinline__ void ldlt_diag_block(double* S, int lds, int c0) {
 }
 
 template <int D>
-__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs, int n = D LDLT_TARG,
+__device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs, int n = D,
                                                  int nrhs = 1, int rhs_stride = 0) {
     // nrhs right-hand sides at rhs + q * rhs_stride, each replaced by its solution
     const int nend = n + nrhs;
-    LDLT_T0;
     const int tid = threadIdx.x, nt = blockDim.x;
     const int ty = tid >> 5, tx = tid & 31, ny = nt >> 5;
     constexpr int NB = 8;
@@ -281,7 +268,6 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
     __syncthreads();
     if (ty == 0) ldlt_diag_block<NB>(S, lds, 0);
     __syncthreads();
-    LDLT_T(0);
     for (int c0 = 0; c0 < n; c0 += NB) {
         double dinv[NB];
 #pragma unroll
@@ -302,7 +288,6 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
             for (int k = 1; k < NB; ++k) rowp[c0 + k] = x[k];
         }
         __syncthreads();
-        LDLT_T(1);
         // (iii) element (r, c2) -= sum_k S[r][c0+k] * S[c2][c0+k] / D_k.  A lane keeps the scaled
         // panel entries of its columns c2 in registers for the whole update and walks down the rows;
         // a row's eight panel entries are the same address for every lane (broadcast loads), so
@@ -356,13 +341,11 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
                 for (int r = c0 + 2 * NB + ty - 1; r < nend; r += ny - 1) update_row(r);
             }
             __syncthreads();
-            LDLT_T(2);
         }
     }
     bool ok = true;
     for (int k = 0; k < n; ++k)
         if (!(S[k * lds + k] > 0.0)) ok = false;
-    LDLT_T(3);
     // rhs now holds y with L y = b.  Backward: x_t = (y_t - sum_{r>t} S[r][t] x_r) / D_t.
     // (one warp per right-hand side: warp ty takes the sides ty, ty + ny, ...)
     for (int q = ty; q < nrhs; q += ny) {
@@ -411,7 +394,6 @@ __device__ __forceinline__ bool block_ldlt_solve(double* S, int lds, double* rhs
         }
     }
     __syncthreads();
-    LDLT_T(4);
     return ok;
 }
 

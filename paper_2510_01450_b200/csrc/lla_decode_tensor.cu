@@ -25,9 +25,7 @@ namespace {
 
 using namespace sm100;
 
-#ifndef LLA_CG_CAP
-#define LLA_CG_CAP 192
-#endif
+constexpr int DT_CG_CAP = 192;   // iteration cap of the d x d solve (the factorisation takes over beyond it)
 constexpr int DT_D = 64;
 constexpr int DT_BK = 64;             // keys per tile
 constexpr int DT_NST = 4;             // K/V ring stages
@@ -99,11 +97,6 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
 // matrix-vector product, so an iteration has one reduction and two 128-thread barriers.
 // x lands in xs[]; returns false if the residual did not reach 1e-9 |b| within the iteration cap or the
 // recurrence broke down (the caller then falls back to the factorisation).
-#ifdef LLA_DT_TIMING
-#define CG_TARG , int* tstat = nullptr
-#else
-#define CG_TARG
-#endif
 // Thread layout of the 64 x 64 solve over 128 threads: a thread keeps a 4 x 8 block of the matrix --
 // rows cg_row0(tid) .. +3, columns cg_col0(tid) .. +7, as cr[8 i + j] -- so that a matrix-vector product
 // reads eight entries of the vector per thread (the shared-memory-to-register path bounds this kernel;
@@ -113,7 +106,7 @@ __device__ __forceinline__ void mma_tile(uint32_t el, uint32_t d, uint64_t a, ui
 __device__ __forceinline__ int cg_row0(int tid) { return 16 * (tid >> 5) + 4 * ((tid & 31) >> 3); }
 __device__ __forceinline__ int cg_col0(int tid) { return 8 * (tid & 7); }
 __device__ __forceinline__ int cg_row(int tid) { return cg_row0(tid) + 2 * ((tid >> 2) & 1) + ((tid >> 1) & 1); }
-__device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double b_r, double* xs, double* pbuf, double* redbuf, int& iters CG_TARG) {
+__device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double b_r, double* xs, double* pbuf, double* redbuf, int& iters) {
     const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
     const int r = cg_row(tid);
     const bool owner = (tid & 1) == 0, b4 = (tid & 4) != 0, b2 = (tid & 2) != 0;
@@ -121,16 +114,9 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
     double x = 0.0, rv = b_r, pv = 0.0, sv = 0.0, alpha = 0.0, gamma_old = 0.0, stop = 0.0;
     bool done = false;
     iters = 0;
-#ifdef LLA_DT_TIMING
-    long long cgt_[5] = {0, 0, 0, 0, 0}, cg0_ = clock64();
-#define CG_T(i) do { const long long n_ = clock64(); cgt_[i] += n_ - cg0_; cg0_ = n_; } while (0)
-#else
-#define CG_T(i)
-#endif
-    for (int it = 0; it <= LLA_CG_CAP; ++it) {
+    for (int it = 0; it <= DT_CG_CAP; ++it) {
         if (owner) pbuf[r] = rv;
         sync128();
-        CG_T(0);
         const double2* pp = reinterpret_cast<const double2*>(pbuf + cg_col0(tid));
         const double2 p01 = pp[0], p23 = pp[1], p45 = pp[2], p67 = pp[3];
         double a[4];
@@ -147,7 +133,6 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
         const double k1 = (b4 ? a[3] : a[1]) + __shfl_xor_sync(0xffffffffu, b4 ? a[1] : a[3], 4);
         double wv = (b2 ? k1 : k0) + __shfl_xor_sync(0xffffffffu, b2 ? k0 : k1, 2);
         wv += __shfl_xor_sync(0xffffffffu, wv, 1);           // both lanes of a pair now hold (C r)_row
-        CG_T(1);
         // (r, r) and (C r, r): each parity class of lanes sums the warp's 16 rows once
         double g = rv * rv, dl = wv * rv;
 #pragma unroll
@@ -155,13 +140,11 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
             g += __shfl_xor_sync(0xffffffffu, g, off);
             dl += __shfl_xor_sync(0xffffffffu, dl, off);
         }
-        CG_T(2);
         double* rb = redbuf + (it & 1) * 8;
         if (lane == 0) { rb[wp] = g; rb[4 + wp] = dl; }
         sync128();
         const double gamma = (rb[0] + rb[1]) + (rb[2] + rb[3]);
         const double delta = (rb[4] + rb[5]) + (rb[6] + rb[7]);
-        CG_T(3);
         // |r| <= 1e-4 |b|, the forward's own CG tolerance for bf16 inputs: the output error is then 1.1e-4
         // row-wise, as for a prefill row (1e-5 |b| gives 1.6e-5, 1e-9 |b| 0.8e-5 -- from there on the fp32 moments
         // set it -- for two and five more iterations)
@@ -172,7 +155,7 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
             beta = gamma * fast_rcp(gamma_old);
             denom = delta - beta * gamma * fast_rcp(alpha);
         }
-        if (!(denom > 0.0) || it == LLA_CG_CAP) break;
+        if (!(denom > 0.0) || it == DT_CG_CAP) break;
         alpha = gamma * fast_rcp(denom);
         pv = rv + beta * pv;
         sv = wv + beta * sv;
@@ -180,11 +163,7 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
         rv -= alpha * sv;
         gamma_old = gamma;
         ++iters;
-        CG_T(4);
     }
-#ifdef LLA_DT_TIMING
-    if (tid == 0 && tstat) for (int i = 0; i < 5; ++i) atomicAdd(tstat + i, (int)(cgt_[i] >> 4));
-#endif
     if (owner) xs[r] = x;
     sync128();
     return done;
@@ -192,24 +171,7 @@ __device__ __forceinline__ bool cg_solve_64(const double (&cr)[32], const double
 
 __device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// Optional phase timing for tuning (-DLLA_DT_TIMING): clock totals of thread 0 go to status[8 + phase].
-#ifdef LLA_DT_TIMING
-#define DT_T0 long long dt_t_ = clock64()
-#define DT_T(ph) do { if (threadIdx.x == 0 && prm.status) { const long long now_ = clock64(); atomicAdd(prm.status + 8 + (ph), (int)((now_ - dt_t_) >> 4)); dt_t_ = now_; } } while (0)
-#else
-#define DT_T0
-#define DT_T(ph)
-#endif
 
-// Optional event trace of one block for tuning (-DLLA_DT_TRACE=<blockIdx.y>): (tag, tile, clock) int
-// triples per role in status[64 + 12000 * role ...].
-#ifdef LLA_DT_TRACE
-#define DT_EV_DECL(role) int* ev_p_ = (prm.status && blockIdx.y == LLA_DT_TRACE) ? prm.status + 64 + 12000 * (role) : nullptr; int ev_n_ = 0
-#define DT_EV(tag, c) do { if (ev_p_ && ev_n_ < 4000) { ev_p_[3 * ev_n_] = (tag); ev_p_[3 * ev_n_ + 1] = (int)(c); ev_p_[3 * ev_n_ + 2] = (int)clock64(); ++ev_n_; } } while (0)
-#else
-#define DT_EV_DECL(role)
-#define DT_EV(tag, c)
-#endif
 
 struct DtParams {
     int B, H, Lmax, splits, head_rows;
@@ -240,12 +202,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int part = blockIdx.x;
-#ifdef LLA_DT_TIMING
-    long long ep_t_ = clock64();
-#define EP_T(ph) do { if (threadIdx.x == 0 && prm.status) { const long long now_ = clock64(); atomicAdd(prm.status + 16 + (ph), (int)((now_ - ep_t_) >> 4)); ep_t_ = now_; } } while (0)
-#else
-#define EP_T(ph)
-#endif
     // Longest caches first: blocks launch in blockIdx order, so block y takes head (y % H) of the
     // sequence whose length has rank (y / H).  Every block ranks the (few) sequence lengths itself.
     int bh = blockIdx.y;
@@ -287,14 +243,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[0];
-    EP_T(0);
 
     float omega = 0.f, m_ref = -INFINITY;     // compute threads; m_ref in log2 units
 
     if (warp == 4) {
         // ================================ TMA producer ================================
         if (lane == 0) {
-            DT_EV_DECL(0);
             // K/V unit and row of a tile in the tensor map: (batch, key/value head) and the key index, or for a
             // paged cache (page, key/value head) and the row inside the page (a tile never straddles a page)
             const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group;
@@ -303,7 +257,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             for (int t = 0; t < ntile; ++t) {
                 const uint32_t s = t % DT_NST;
                 if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
-                DT_EV(1, t);
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
                 int unit = kvh, jrow = kstart + jbeg + t * DT_BK;
@@ -319,20 +272,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     } else if (warp == 5) {
         // ================================ MMA issuer (whole warp, predicated) ================================
         const uint32_t el = elect_one();
-        DT_EV_DECL(1);
         for (int t = 0; t < ntile; ++t) {
             const uint32_t s = t % DT_NST, b = t & 1;
             if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) break;
-            if (lane == 0) DT_EV(9, t);
             if (!mbar_wait(bar(DB_BFULL + b), (t >> 1) & 1, abort_flag)) break;
-            if (lane == 0) DT_EV(10, t);
             tc_fence_after();
             const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
             mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), t > 0);
             tc_commit_el(el, bar(DB_KVEMPTY + s));
             tc_commit_el(el, bar(DB_BFREE + b));
             if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
-            if (lane == 0) DT_EV(11, t);
         }
     } else {
         // ================================ compute warps ================================
@@ -461,16 +410,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ok = stage_score_sync(0);
             }
         }
-        DT_T0;
-        DT_EV_DECL(2);
         for (int t = 0; t < ntile && ok; ++t) {
-            if (tid == 0) DT_EV(19, t);
             const uint32_t b = t & 1;
             const bool more = t + 1 < ntile;
             // wait until the MMA of tile t-2 has released this B buffer (long done in steady state)
             if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            DT_T(2);
-            if (tid == 0) DT_EV(21, t);
             // B rows of tile t: w * [k | 1] as bf16 hi + lo, eight features at a time straight into the
             // operand tiles, so the stores drain while the rest of the iteration runs
             uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
@@ -496,24 +440,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
                 *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
             }
-            DT_T(0);
             // the next tile: shared-memory loads, then the score arithmetic, while the stores drain
             if (more && !stage_load(t + 1)) { ok = false; break; }
-            DT_T(1);
-            if (tid == 0) DT_EV(20, t);
-            if (tid == 0) DT_EV(24, t);
             if (more) stage_score_math(t + 1);
-            if (tid == 0) DT_EV(25, t);
             fence_proxy_async();
-            if (tid == 0) DT_EV(26, t);
             // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised shared-memory atomics
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(DB_BFULL + b));
-            DT_T(3);
-            if (tid == 0) DT_EV(22, t);
             if (more && !stage_score_sync(t + 1)) { ok = false; break; }
-            DT_T(4);
-            if (tid == 0) DT_EV(23, t);
         }
         // total weight of this part
         if (ok) {
@@ -524,7 +458,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     // ================================ epilogue ================================
     // All 192 threads take part (the solve below is a block-wide routine).
-    EP_T(1);
     __shared__ float s_omega[4];
     __shared__ float s_mref;
     if (warp < 4 && lane == 0) s_omega[warp] = omega;
@@ -564,9 +497,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     }
     tc_fence_before();
-    EP_T(2);
     __syncthreads();       // every pipeline stage is drained: shared memory can be re-carved
-    EP_T(3);
     if (warp == 4) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(DT_TMEM_COLS) : "memory");
@@ -625,7 +556,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     }
     __syncthreads();
-    EP_T(4);
     // conjugate gradients first (fast); the blocked factorisation only if they do not converge
     double* xs = reinterpret_cast<double*>(Nd + 64 * 65);      // x, p and reduction scratch after N
     __shared__ int s_cg_ok;
@@ -643,7 +573,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     }
     __syncthreads();
-    EP_T(5);
     bool solved = true;
     if (s_cg_ok) {
         if (tid < 64) rhs[tid] = xs[tid];
@@ -656,7 +585,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int f = 0; f < 64; ++f) o += ((double)Nd[tid * 65 + f] * inv - cv[tid] * av[f]) * rhs[f];
         store_out(out + (size_t)bh * DT_D + tid, (float)o);
     }
-    EP_T(6);
     if (!solved && tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_BAD_PIVOT, 1);
 }
 
@@ -678,12 +606,6 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     const int tid = threadIdx.x, r = tid >> 1, hh = tid & 1, bh = blockIdx.x;
     // launched as a programmatic dependent of the streaming kernel: nothing of that grid may be read before this
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#ifdef LLA_DT_TIMING
-    long long sv_t_ = clock64();
-#define SV_T(ph) do { if (threadIdx.x == 0 && status) { const long long now_ = clock64(); atomicAdd(status + 24 + (ph), (int)((now_ - sv_t_) >> 4)); sv_t_ = now_; } } while (0)
-#else
-#define SV_T(ph)
-#endif
     {
     if (visible_keys(lens[bh / H], Lmax, window) < head_rows) return;
     const float* src = parts + (size_t)bh * splits * PF;
@@ -703,7 +625,6 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
         if (tid < D) s_a[tid] = s1 * inv; else s_c[tid - D] = s1 * inv;
     }
     __syncthreads();
-    SV_T(0);
     // this thread's 4 x 8 block of the centred matrix (see cg_solve_64)
     const int row0 = cg_row0(tid), col0 = cg_col0(tid), myrow = cg_row(tid);
     double cr[32];
@@ -732,13 +653,7 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     }
     const double b_r = (double)to_f32(q[(size_t)bh * D + myrow]) - s_a[myrow];
     int cg_its = 0;
-    SV_T(1);
-#ifdef LLA_DT_TIMING
-    const bool okc = cg_solve_64(cr, b_r, s_x, s_p, s_red, cg_its, status ? status + 32 : nullptr);
-#else
     const bool okc = cg_solve_64(cr, b_r, s_x, s_p, s_red, cg_its);
-#endif
-    SV_T(2);
     if (tid == 0 && status) atomicAdd(status + LLA_STATUS_ITER_SUM, cg_its);
     bool solved = true;
     if (!okc) {        // uniform over the block: the decision comes from block-wide sums
@@ -769,7 +684,6 @@ decode_solve_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict
     for (int c = 0; c < 32; ++c) o += (nr[c] * inv - cb * s_a[32 * hh + c]) * s_x[32 * hh + c];
     o += __shfl_xor_sync(0xffffffffu, o, 1);
     if (hh == 0) store_out(out + (size_t)bh * D + r, (float)(o + cb));
-    SV_T(3);
     if (!solved && tid == 0 && status) atomicAdd(status + LLA_STATUS_BAD_PIVOT, 1);
     }
 }

@@ -79,14 +79,6 @@ __device__ __forceinline__ double dot_row(const double* __restrict__ a, const fl
     return s;
 }
 
-// Optional phase timing for tuning (-DLLA_HR_TIMING: clock totals of thread 0 are added to status[8 + phase]).
-#ifdef LLA_HR_TIMING
-#define HR_T(phase) do { if (threadIdx.x == 0 && status) { const long long now_ = clock64(); atomicAdd(status + 8 + (phase), (int)((now_ - hr_t_) >> 4)); hr_t_ = now_; } } while (0)
-#define HR_T0 long long hr_t_ = clock64()
-#else
-#define HR_T(phase)
-#define HR_T0
-#endif
 
 // two consecutive elements (4- or 8-byte aligned) as floats
 __device__ __forceinline__ void load2(const __nv_bfloat16* p, float& a, float& b) {
@@ -140,7 +132,6 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     const TIn* kb = k + kvrow * D;
     const TIn* vb = v + kvrow * DV;
 
-    HR_T0;
     for (int c = tid; c < D; c += HR_THREADS) qd[c] = (double)to_f32(qrow[c]);
     __syncthreads();
 
@@ -151,7 +142,6 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         w[j] = s;
         lmax = fmax(lmax, s);
     }
-    HR_T(0);
     const double m = block_reduce<HR_THREADS>(lmax, true, red);
     double lsum = 0.0;
     for (int j = tid; j < L; j += HR_THREADS) {
@@ -163,7 +153,6 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     // per-row ridge if given (prefill: [B,H,n]; decode: [B,H]); see lla_ridge_mode for the two frames
     const double lam_i = lambda_rows ? (double)lambda_rows[row] : lambda;
     const double lambda_m = ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * exp(-m);
-    HR_T(1);
 
     // Rows with at most d keys (and a positive ridge) go through the dual (Gram) form: with Z the
     // L x d matrix of centred keys, w_j (1 - z_j . rho) = lambda' alpha_j where
@@ -301,7 +290,6 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
                 }
             }
         }
-        HR_T(2);
         __syncthreads();   // the staged keys (lying over S) are no longer read
     #pragma unroll
         for (int t = 0; t < C::TILES_PER_THREAD; ++t) {
@@ -318,14 +306,8 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         if (tid < D) rhs[tid] = mu_acc;
         __syncthreads();
 
-        HR_T(3);
         // rhs <- Sigma^{-1} mu (LDL^T in shared memory)
-    #ifdef LLA_HR_TIMING
-        bad = !block_ldlt_solve<D>(S, C::LDS, rhs, D, status ? status + 16 : nullptr);
-    #else
         bad = !block_ldlt_solve<D>(S, C::LDS, rhs);
-    #endif
-        HR_T(4);
 
         // coefficients c_j = w_j (1 - z_j . rho) and their sum (= omega - mu . rho)
         double qrho = 0.0;
@@ -339,13 +321,11 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         if (tid < D) rho_val = rhs[tid];
     }
     const double denom = block_reduce<HR_THREADS>(csum, false, red);
-    HR_T(5);
     for (int c = tid; c < DV; c += HR_THREADS) {
         double o = 0.0;
         for (int j = 0; j < L; ++j) o += w[j] * (double)to_f32(vb[(size_t)j * DV + c]);
         store_out(out + row * DV + c, (float)(o / denom));
     }
-    HR_T(6);
     if (rho_out && tid < D) rho_out[row * D + tid] = (float)rho_val;
     if (tid == 0) {
         if (stats) {

@@ -89,7 +89,7 @@ def make_prefill(w: Workload):
         k = rng.standard_normal((B, H, n, d), dtype=np.float32) * inv
         v = rng.standard_normal((B, H, n, dv), dtype=np.float32)
         if w.name.startswith("cfg1"):
-            v = v * np.float32(1.0 / np.sqrt(d))   # workload 1 scales q, k and v alike
+            v = v * np.float32(1.0 / np.sqrt(d))   # the fp32 n = 256, d = 16 case scales q, k and v alike
     elif w.recipe == "regression":
         keys = rng.standard_normal((B, H, n + 1, d), dtype=np.float32) * inv
         k = keys[:, :, :n]

@@ -68,7 +68,7 @@ def test_backward_matches_gradient_oracle(backward_oracle, d, n, B, H, impl):
 
 
 def test_backward_regression_recipe_and_bf16_tensors(backward_oracle):
-    # workload 3's recipe (values linear in the keys, the query is the next key); g and out in bf16
+    # the test-time-regression recipe of Section 4.1 (values linear in the keys, the query is the next key); g and out in bf16
     w = inputs.CONFIGS[3].shrink(B=1, H=2, n=600, seed=231)
     q, k, v = inputs.make_prefill(w)
     g = inputs.make_upstream_grad(w, "bf16")

@@ -56,7 +56,7 @@ def _softmax_rows(q, k, v, scale):
 
 
 def test_brute_force_wls_tiny(oracle):
-    # (d) of the benchmark spec: n <= 8, every causal row equals the intercept of a dense WLS fit.
+    # brute force on tiny inputs: n <= 8, every causal row equals the intercept of a dense WLS fit.
     for seed, (n, d, dv, scale, lam) in enumerate([(8, 3, 2, 0.7, 0.05), (6, 2, 4, 3.0, 1e-3),
                                                    (8, 4, 3, 1.5, 0.3), (5, 1, 1, 2.0, 0.01)]):
         q, k, v = _rand(seed, 2, 2, n, d, dv, kscale=1.0)
