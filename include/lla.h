@@ -240,6 +240,10 @@ int lla_decode_ex(const lla_decode_params *p);
  * buffers); `stream` is joined with them before the call returns.
  * lla_decode_host reads lens[] on the host and uploads only the first lens[b] rows of every
  * (sequence, head) cache.
+ * Side effect on the process: the entry points that take scratch from the pool (these two, lla_forward and
+ * lla_decode) set the release threshold of the current device's DEFAULT stream-ordered memory pool to
+ * "keep everything", once per device, so that repeated calls do not return their scratch to the driver.
+ * A host program that trims that pool itself should use the _ex forms with its own workspace instead.
  */
 int lla_forward_host(const void *q, const void *k, const void *v, void *out, int B, int H, int n,
                      int d, int dv, int in_dtype, int out_dtype, float scale, float lambda,
@@ -267,9 +271,11 @@ int lla_decode_host(const void *q, const void *kcache, const void *vcache, const
  * Arguments are those of lla_decode plus the dtypes and `splits` (0 = the default of
  * lla_decode_default_splits; 1 = no split, which uses the array only if the records fit).  All tensor pointers are
  * device pointers owned by the caller.
- * Errors: LLA_ERR_WORKSPACE if B*H*splits partial records do not fit in the fixed array
+ * Errors: LLA_ERR_WORKSPACE if an explicit `splits` > 1 needs more than the fixed array holds
  * (lla_decode_workspace_bytes(...) > LLA_NOALLOC_SCRATCH_BYTES): use fewer splits or lla_decode_ex
- * with a caller workspace.  Other codes as for lla_decode_ex.
+ * with a caller workspace.  With splits = 0 a default split count that does not fit runs unsplit instead.
+ * Other codes as for lla_decode_ex.  The array's device address is looked up once per device and kept for
+ * the life of the process: after cudaDeviceReset on that device the entry point must not be used again.
  * Sharing: all calls on a device use the same array.  Each call overwrites every record it later
  * reads, so nothing needs clearing between calls, but two calls whose kernels may run at the same
  * time (different streams, or different host threads) race on it: serialise them.

@@ -45,6 +45,9 @@ struct HostPipe {
     cudaStream_t stream[kHostChunks] = {};
     cudaEvent_t ready = nullptr, done[kHostChunks] = {};
     bool ok = false;
+    // held for a whole call: the events and worker streams are shared by every caller on the device, and a wait
+    // takes an event's latest record, so two host threads must not interleave their record/wait sequences
+    std::mutex use;
 };
 HostPipe* host_pipe() {
     static std::mutex mu;
@@ -131,16 +134,19 @@ int check_decode(const lla_decode_params* p) {
 }
 
 void keep_pool_memory() {
-    // let the stream-ordered pool keep freed blocks so repeated host-buffer calls do not re-allocate
-    static bool done = false;
-    if (done) return;
+    // Let the current device's default stream-ordered pool keep freed blocks, so that repeated calls of the
+    // entry points that take their scratch from it do not go back to the driver every time.  Once per device.
+    // (A process-wide setting of that pool: include/lla.h says so.)
+    static std::once_flag once[64];
     int dev = 0;
-    cudaMemPool_t pool;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
-        unsigned long long keep = ~0ull;
-        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
-    }
-    done = true;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+    std::call_once(once[dev], [dev]() {
+        cudaMemPool_t pool;
+        if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+            unsigned long long keep = ~0ull;
+            cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        }
+    });
 }
 
 }  // namespace
@@ -478,26 +484,38 @@ int lla_forward_host(const void* q, const void* k, const void* v, void* out, int
     const int chunk_units = (units + kHostChunks - 1) / kHostChunks;
     const size_t wsb = lla_forward_workspace_bytes(1, chunk_units, n, d, dv, in_dtype, LLA_IMPL_AUTO);
     char* wsp = wsb > 0 ? static_cast<char*>(mem.get(wsb * kHostChunks)) : nullptr;
-    LLA_CUDA_TRY(cudaEventRecord(pipe->ready, st));            // the buffers exist from here on
+    std::lock_guard<std::mutex> pipe_lock(pipe->use);
     const size_t uq = (size_t)n * d * esz_in, uv = (size_t)n * dv * esz_in, uo = (size_t)n * dv * esz_out;
     int rc_chunks = LLA_OK;
-    for (int c = 0; c < kHostChunks; ++c) {
-        const int u0 = (int)((long long)units * c / kHostChunks), u1 = (int)((long long)units * (c + 1) / kHostChunks);
-        cudaStream_t w = pipe->stream[c];
-        LLA_CUDA_TRY(cudaStreamWaitEvent(w, pipe->ready, 0));
-        LLA_CUDA_TRY(cudaMemcpyAsync((char*)dq + u0 * uq, (const char*)q + u0 * uq, (u1 - u0) * uq, cudaMemcpyHostToDevice, w));
-        LLA_CUDA_TRY(cudaMemcpyAsync((char*)dk + u0 * uq, (const char*)k + u0 * uq, (u1 - u0) * uq, cudaMemcpyHostToDevice, w));
-        LLA_CUDA_TRY(cudaMemcpyAsync((char*)dvv + u0 * uv, (const char*)v + u0 * uv, (u1 - u0) * uv, cudaMemcpyHostToDevice, w));
-        lla_forward_params pc = p;
-        pc.q = (char*)dq + u0 * uq; pc.k = (char*)dk + u0 * uq; pc.v = (char*)dvv + u0 * uv; pc.out = (char*)dout + u0 * uo;
-        pc.B = 1; pc.H = u1 - u0;
-        pc.stream = w;
-        if (wsp) { pc.workspace = wsp + (size_t)c * wsb; pc.workspace_bytes = wsb; }
-        const int rc_c = lla_forward_ex(&pc);
-        if (rc_c != LLA_OK && rc_chunks == LLA_OK) rc_chunks = rc_c;
-        LLA_CUDA_TRY(cudaMemcpyAsync((char*)out + u0 * uo, (char*)dout + u0 * uo, (u1 - u0) * uo, cudaMemcpyDeviceToHost, w));
-        LLA_CUDA_TRY(cudaEventRecord(pipe->done[c], w));
-        LLA_CUDA_TRY(cudaStreamWaitEvent(st, pipe->done[c], 0));
+    auto enqueue = [&]() -> int {
+        LLA_CUDA_TRY(cudaEventRecord(pipe->ready, st));            // the buffers exist from here on
+        for (int c = 0; c < kHostChunks; ++c) {
+            const int u0 = (int)((long long)units * c / kHostChunks), u1 = (int)((long long)units * (c + 1) / kHostChunks);
+            cudaStream_t w = pipe->stream[c];
+            LLA_CUDA_TRY(cudaStreamWaitEvent(w, pipe->ready, 0));
+            LLA_CUDA_TRY(cudaMemcpyAsync((char*)dq + u0 * uq, (const char*)q + u0 * uq, (u1 - u0) * uq, cudaMemcpyHostToDevice, w));
+            LLA_CUDA_TRY(cudaMemcpyAsync((char*)dk + u0 * uq, (const char*)k + u0 * uq, (u1 - u0) * uq, cudaMemcpyHostToDevice, w));
+            LLA_CUDA_TRY(cudaMemcpyAsync((char*)dvv + u0 * uv, (const char*)v + u0 * uv, (u1 - u0) * uv, cudaMemcpyHostToDevice, w));
+            lla_forward_params pc = p;
+            pc.q = (char*)dq + u0 * uq; pc.k = (char*)dk + u0 * uq; pc.v = (char*)dvv + u0 * uv; pc.out = (char*)dout + u0 * uo;
+            pc.B = 1; pc.H = u1 - u0;
+            pc.stream = w;
+            if (wsp) { pc.workspace = wsp + (size_t)c * wsb; pc.workspace_bytes = wsb; }
+            const int rc_c = lla_forward_ex(&pc);
+            if (rc_c != LLA_OK && rc_chunks == LLA_OK) rc_chunks = rc_c;
+            LLA_CUDA_TRY(cudaMemcpyAsync((char*)out + u0 * uo, (char*)dout + u0 * uo, (u1 - u0) * uo, cudaMemcpyDeviceToHost, w));
+            LLA_CUDA_TRY(cudaEventRecord(pipe->done[c], w));
+            LLA_CUDA_TRY(cudaStreamWaitEvent(st, pipe->done[c], 0));
+        }
+        return LLA_OK;
+    };
+    const int rc_q = enqueue();
+    if (rc_q != LLA_OK) {
+        // something could not be enqueued: the workers may still be using the buffers that go back to the pool
+        // when this function returns, so wait for them here
+        for (int c = 0; c < kHostChunks; ++c) (void)cudaStreamSynchronize(pipe->stream[c]);
+        (void)cudaStreamSynchronize(st);
+        return rc_q;
     }
     LLA_CUDA_TRY(cudaStreamSynchronize(st));
     return rc_chunks;

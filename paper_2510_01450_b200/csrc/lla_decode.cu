@@ -392,7 +392,11 @@ extern "C" int lla_decode_noalloc(const void* q, const void* kcache, const void*
     a.stream = (cudaStream_t)stream;
     // records are required for a split decode and optional otherwise (they let the tensor-core path
     // run its solve as a separate kernel)
-    const size_t need = lla::decode_record_bytes(B, H, d, dv, a.splits);
+    size_t need = lla::decode_record_bytes(B, H, d, dv, a.splits);
+    if (splits == 0 && a.splits > 1 && need > (size_t)LLA_NOALLOC_SCRATCH_BYTES) {
+        a.splits = 1;      // the default split count does not fit the fixed array: run unsplit, as lla_decode_ex does
+        need = lla::decode_record_bytes(B, H, d, dv, 1);
+    }
     if (a.splits > 1 && need > (size_t)LLA_NOALLOC_SCRATCH_BYTES) return LLA_ERR_WORKSPACE;   // beyond the fixed array
     if (need <= (size_t)LLA_NOALLOC_SCRATCH_BYTES) {
         void* scratch = nullptr;

@@ -290,6 +290,41 @@ def test_host_buffer_entry_points(oracle):
     assert row_err(hout.numpy(), dref).max() <= TOL_BF16
 
 
+def test_host_buffer_forward_from_two_threads(oracle):
+    # two host threads, each with its own stream and its own problem, in the chunked host-buffer form at the same
+    # time: the library's worker streams and events are shared per device, so the calls must not mix them up
+    import threading
+    jobs = []
+    for seed, n in ((31, 640), (32, 512)):
+        w = inputs.CONFIGS[2].shrink(B=3, H=3, n=n, seed=seed)
+        q, k, v = inputs.make_prefill(w)
+        host = tuple(torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in (q, k, v))
+        hout = torch.full((w.B, w.H, w.n, w.dv), float("nan"), dtype=torch.float32).pin_memory()
+        jobs.append((w, host, hout, oracle.forward(q, k, v, w.scale, w.lam), torch.cuda.Stream()))
+    errors = []
+
+    def work(job):
+        w, (hq, hk, hv), hout, _, stream = job
+        try:
+            for _ in range(6):
+                hout.fill_(float("nan"))
+                L.lla_forward_host(hq, hk, hv, hout, w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, L.LLA_F32, w.scale, w.lam, 1,
+                                   stream.cuda_stream)
+                if not np.isfinite(hout.numpy()).all():
+                    errors.append("non-finite output")
+        except Exception as e:      # noqa: BLE001
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for w, _, hout, ref, _ in jobs:
+        assert row_err(hout.numpy(), ref).max() <= TOL_BF16
+
+
 @pytest.mark.parametrize("dtype,d,n", [("bf16", 64, 700), ("bf16", 128, 400), ("f32", 16, 200)])
 def test_ridge_variants_forward(oracle, dtype, d, n):
     # per-token ridge and the ridge of the printed algorithm (both only change lambda'_i)

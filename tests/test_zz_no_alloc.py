@@ -40,14 +40,36 @@ def test_no_alloc_decode_matches_workspace_decode_twice(oracle):
         dl = torch.from_numpy(lens).cuda()
         want = _reference(dq, dk, dv_, dl, w, splits)
         out = torch.full((w.B, w.H, w.dv), float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         L.lla_decode_noalloc(dq, dk, dv_, dl, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam,
                              out_dtype=L.LLA_F32, splits=splits, stream=stream_ptr())
         torch.cuda.synchronize()
+        if seed != 70:      # (the first call of a process may load the module's kernels)
+            assert torch.cuda.mem_get_info()[0] == free_before      # the call took no device memory
         got = out.cpu().numpy()
         assert np.isfinite(got).all()
         assert row_err(got, want).max() <= 2e-3       # same tolerance as the parity tests (same kernels: equal)
         ref = oracle.decode(q, kc, vc, lens, w.scale, w.lam)
         assert row_err(got, ref).max() <= 2e-3
+
+
+def test_no_alloc_default_splits_that_do_not_fit_run_unsplit(oracle):
+    # d = 128, 280 (sequence, head) pairs: the default of 2 parts needs 74 MB of records; with splits = 0 the call
+    # falls back to one part instead of refusing
+    w = inputs.CONFIGS[5].shrink(B=70, H=4, n=1024, d=128, dv=128, len_min=300, len_max=1024, seed=72)
+    assert L.lla_decode_default_splits(w.B, w.H, w.n) > 1
+    assert L.lla_decode_workspace_bytes(w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16,
+                                        L.lla_decode_default_splits(w.B, w.H, w.n)) > L.NOALLOC_SCRATCH_BYTES
+    q, kc, vc, lens = inputs.make_decode(w)
+    dq, dk, dv_ = dev(q, "bf16"), dev(kc, "bf16"), dev(vc, "bf16")
+    dl = torch.from_numpy(lens).cuda()
+    out = torch.full((w.B, w.H, w.dv), float("nan"), dtype=torch.float32, device="cuda")
+    L.lla_decode_noalloc(dq, dk, dv_, dl, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, out_dtype=L.LLA_F32,
+                         splits=0, stream=stream_ptr())
+    torch.cuda.synchronize()
+    ref = oracle.decode(q, kc, vc, lens, w.scale, w.lam)
+    assert row_err(out.cpu().numpy(), ref).max() <= 2e-3
 
 
 def test_no_alloc_rejects_what_does_not_fit():
