@@ -182,8 +182,17 @@ typedef struct lla_forward_params {
                        tiles within the first 8 d positions, which converge more slowly); n > 0 = n
                        iterations for every tile; LLA_CG_PRECISE_ALL = every iteration with pairs;
                        LLA_CG_PRECISE_NONE = fp16 from the first iteration on */
+    long long debug_wait_clocks; /* tensor-core kernel only: cap, in SM clocks, of every bounded wait on a barrier
+                       inside the kernel (0 = default, about 2^31).  A wait that runs out makes its thread block
+                       stop: the block waits for the copies and MMAs it has issued itself, releases its tensor
+                       memory and returns without writing its rows; the call still returns LLA_OK and
+                       device_status[LLA_STATUS_TIMEOUT] counts the blocks that gave up */
+    int debug_flags;          /* LLA_DEBUG_NO_LOADS: the kernel's copy-issuing warp issues nothing, so that every
+                       wait of every block expires with no copy or MMA in flight.  For testing the path above
+                       without faulting or hanging anything; the output is left unwritten */
 } lla_forward_params;
 enum { LLA_CG_PRECISE_ALL = -1, LLA_CG_PRECISE_NONE = -2 };
+enum { LLA_DEBUG_NO_LOADS = 1 };
 
 int lla_forward_ex(const lla_forward_params *p);
 

@@ -21,6 +21,7 @@ LLA_PHASE_ALL, LLA_PHASE_DIRECT, LLA_PHASE_ITERATIVE = 0, 1, 2
 STATUS_ROWS_AT_CAP, STATUS_BAD_PIVOT, STATUS_TIMEOUT, STATUS_ITER_SUM = 0, 1, 2, 3
 LLA_RIDGE_DEFINITION, LLA_RIDGE_PRINTED = 0, 1
 LLA_CG_PRECISE_ALL, LLA_CG_PRECISE_NONE = -1, -2
+LLA_DEBUG_NO_LOADS = 1
 
 EXPORTS = (
     "lla_forward", "lla_forward_f32", "lla_decode", "lla_decode_f32", "lla_forward_ex", "lla_decode_ex",
@@ -61,7 +62,7 @@ class ForwardParams(ctypes.Structure):
         ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p), ("lambda_rows", ctypes.c_void_p), ("ridge_mode", ctypes.c_int),
         ("q_rows", ctypes.c_int), ("kv_heads", ctypes.c_int), ("window", ctypes.c_int),
-        ("cg_precise_iters", ctypes.c_int),
+        ("cg_precise_iters", ctypes.c_int), ("debug_wait_clocks", ctypes.c_longlong), ("debug_flags", ctypes.c_int),
     ]
 
 
@@ -177,8 +178,10 @@ def lla_decode_host(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, in_dtype, o
 def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=LLA_BF16, out_dtype=LLA_BF16,
                    max_iters=0, tol=0.0, head_rows=0, impl=LLA_IMPL_AUTO, phases=0, rho=None, stats=None, iters=None,
                    device_status=None, workspace=None, workspace_bytes=0, stream=0, lambda_rows=None,
-                   ridge_mode=LLA_RIDGE_DEFINITION, q_rows=0, kv_heads=0, window=0, cg_precise_iters=0):
+                   ridge_mode=LLA_RIDGE_DEFINITION, q_rows=0, kv_heads=0, window=0, cg_precise_iters=0,
+                   debug_wait_clocks=0, debug_flags=0):
     p = ForwardParams()
+    p.debug_wait_clocks, p.debug_flags = debug_wait_clocks, debug_flags
     p.kv_heads, p.window, p.cg_precise_iters = kv_heads, window, cg_precise_iters
     p.q, p.k, p.v, p.out = _p(q), _p(k), _p(v), _p(out)
     p.B, p.H, p.n, p.d, p.dv = B, H, n, d, dv

@@ -69,6 +69,8 @@ struct ForwardArgs {
     int window = 0;             // causal sliding window: a row sees its last `window` positions (0: all)
     const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
+    long long wait_clocks = 0;  // tensor-core kernel: cap of its bounded waits in SM clocks (0: default) and a test
+    int no_loads = 0;           // aid: issue no copy at all (lla_forward_params.debug_*)
     const void* k16 = nullptr;  // fp16 copy of k and its validity word, set by forward_tensor_prepass
     const int* f16_ok = nullptr;
     int precise_iters = 1;      // tensor-core kernel: CG iterations run with bf16 hi + lo operand pairs before the

@@ -93,7 +93,8 @@ static_assert(TcCfg<64>::SM_ALLOC <= 227 * 1024 && TcCfg<128>::SM_ALLOC <= 227 *
 enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST_MAX, B_VFULL = B_KVEMPTY + TC_NST_MAX,
        B_SAFULL = B_VFULL + TC_NST_MAX,
        B_UFULL = B_SAFULL + TC_NBUF, B_BUFFREE = B_UFULL + TC_NBUF, B_ACCFULL = B_BUFFREE + TC_NBUF, B_CTL = B_ACCFULL + 1,
-       B_COUNT = B_CTL + 1 };
+       B_EXIT = B_CTL + 1,   // two: the MMA warps' last commits on an aborted run
+       B_COUNT = B_EXIT + 2 };
 static_assert(B_COUNT * 8 <= 256, "barrier area too small");
 
 // MMA issue.  The whole MMA warp runs these convergently and the instructions are predicated on the
@@ -176,6 +177,8 @@ struct TcParams {
     int n, nq, causal, head_rows, max_iters, first_tile;   // n keys; nq query rows at positions n - nq .. n - 1
     int precise_iters;   // CG iterations whose operands are bf16 hi + lo pairs; later ones use single fp16 operands
     int precise_iters_early;   // the same for the row tiles that end within the first 8 D positions
+    long long wait_clocks;   // cap of every bounded wait, in SM clocks
+    int no_loads;        // test aid: the TMA warp issues no copy at all, so that every wait expires with nothing in flight
     const int* f16_ok;   // device word written by the conversion pre-pass: nonzero = q and k fit the fp16 range and
                          // the fp16 copy of k (tmK16) is valid; NULL or zero = every sweep in bf16
     float scale, lambda, tol;
@@ -232,7 +235,6 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         rs = kbs + (size_t)D * TC_BR;
     }
     float* red = reinterpret_cast<float*>(smem + SM_RED);
-    volatile int* flags = reinterpret_cast<volatile int*>(smem + SM_FLAGS);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // blockIdx.x runs fastest in launch order: all heads of one query tile start together, the tiles
@@ -254,6 +256,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // The values of the copies equal the bf16 inputs (the pre-pass checks the range).
     // (tiles whose rows see fewer than 8 D keys converge more slowly and keep the pairs for more iterations)
     const int precise = off + r0 + TC_BR <= 8 * D ? prm.precise_iters_early : prm.precise_iters;
+    const long long wcap = prm.wait_clocks;
     const int f16_from = (prm.f16_ok && *prm.f16_ok && precise < (1 << 29)) ? precise + 2 : (1 << 30);
 
     if (tid == 0) {
@@ -270,6 +273,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         mbar_init(bar(B_ACCFULL), 1);
         mbar_init(bar(B_CTL), TC_COMPUTE / 32);
+        mbar_init(bar(B_EXIT), 1);
+        mbar_init(bar(B_EXIT + 1), 1);
         misc[1] = SW_MAX;
         misc[2] = 0;
         misc[3] = kv_unit(bh, prm.H, prm.kv_group);   // worked out here: in the producer's own path it delays the first loads
@@ -291,7 +296,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // blocks of the next sweep are prefetched without waiting to learn what kind of sweep it is
         // (every kind needs K).  V blocks are added, on their own barriers, once the output sweep
         // is announced.
-        if (lane == 0) {
+        if (lane == 0 && !prm.no_loads) {
             mbar_expect_tx(bar(B_QFULL), Cfg::OPER_BYTES);
             for (int sub = 0; sub < KSUB; ++sub)
                 tma_load_3d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, bh);
@@ -301,27 +306,31 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             bool ok = true;
             auto issue_k = [&](int c, bool f16) {
                 const uint32_t s = kit % TC_NST;
-                if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag, wcap)) { ok = false; return; }
                 mbar_expect_tx(bar(B_KVFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
                     tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, f16 ? &tmK16 : &tmK, bar(B_KVFULL + s), 64 * sub,
                                 (cbeg + c) * TC_BC, kvh);
                 ++kit;
             };
+            uint32_t v_g0 = 0;
+            int v_issued = 0;      // V blocks issued (output sweep only), the first at ring position v_g0
             auto issue_v = [&](int c, uint32_t g) {
+                if (v_issued == 0) v_g0 = g - c;
+                v_issued = c + 1;
                 const uint32_t s = g % TC_NST;
                 mbar_expect_tx(bar(B_VFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
                     tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
             };
             for (uint32_t sweep = 0; ok; ++sweep) {
-                if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+                if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag, wcap)) break;
                 const int kind = misc[1];
                 if (kind == SW_DONE) {
                     // prefetched blocks nobody will consume: wait until they have landed
                     for (int i = 0; i < pre; ++i) {
                         const uint32_t g = kit - pre + i;
-                        if (!mbar_wait(bar(B_KVFULL + g % TC_NST), (g / TC_NST) & 1, abort_flag)) break;
+                        if (!mbar_wait(bar(B_KVFULL + g % TC_NST), (g / TC_NST) & 1, abort_flag, wcap)) break;
                     }
                     break;
                 }
@@ -336,6 +345,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (kind != SW_OUT)
                     for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c, (int)sweep + 1 >= f16_from); ++pre; }
             }
+            if (*abort_flag) {
+                // an aborted block: the copies issued above write into this block's shared memory, so they must
+                // have landed before the block exits (on a completed run their consumers have waited for them)
+                (void)mbar_wait_landed(bar(B_QFULL), 0, wcap);
+                for (uint32_t g = kit > (uint32_t)TC_NST ? kit - TC_NST : 0; g < kit; ++g)
+                    (void)mbar_wait_landed(bar(B_KVFULL + g % TC_NST), (g / TC_NST) & 1, wcap);
+                for (int c = max(0, v_issued - TC_NST); c < v_issued; ++c)
+                    (void)mbar_wait_landed(bar(B_VFULL + (v_g0 + c) % TC_NST), (c / TC_NST) & 1, wcap);
+            }
         }
     } else if (warp == 9) {
         // ================================ MMA issuer 1: S = Q K^T, A = P K^T ================================
@@ -348,21 +366,21 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // the MMA operands in uniform registers (otherwise every operand is moved there one by one)
         const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
         const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
-        bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
+        bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, wcap);
         const uint64_t qdesc = make_desc(sb_u + SM_Q);
         const uint64_t phdesc = make_desc(sb_u + SM_PHI);
         const uint64_t pldesc = make_desc(sb_u + SM_PLO);
         uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it % NBUF)
         for (uint32_t sweep = 0; ok; ++sweep) {
-            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag, wcap)) break;
             const int kind = misc[1];
             if (kind == SW_DONE) break;
             tc_fence_after();
             const uint32_t idesc = (int)sweep >= f16_from ? IDESC_SS16 : IDESC_SS;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
-                if (!mbar_wait(bar(B_KVFULL + s), (it / TC_NST) & 1, abort_flag)) { ok = false; break; }
-                if (!mbar_wait(bar(B_BUFFREE + b), (bu & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bar(B_KVFULL + s), (it / TC_NST) & 1, abort_flag, wcap)) { ok = false; break; }
+                if (!mbar_wait(bar(B_BUFFREE + b), (bu & 1) ^ 1, abort_flag, wcap)) { ok = false; break; }
                 tc_fence_after();
                 const uint64_t kdesc = make_desc(sb_u + SM_KV + s * STAGE);
                 const uint32_t s_tm = tm_u + b * 128, a_tm = s_tm + 64;
@@ -384,6 +402,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tc_commit_el(el, bar(B_SAFULL + b));
             }
         }
+        if (*abort_flag) {      // an aborted block: the MMAs this warp issued must be done before TMEM and shared memory go
+            tc_commit_el(el, bar(B_EXIT + 0));
+            (void)mbar_wait_landed(bar(B_EXIT + 0), 0, wcap);
+        }
     } else if (warp == 10) {
         // ================================ MMA issuer 2: ACC += U B ================================
         const uint32_t el = elect_one();
@@ -392,13 +414,13 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         bool ok = true;
         uint32_t it = 0;
         for (uint32_t sweep = 0; ok; ++sweep) {
-            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag)) break;
+            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag, wcap)) break;
             const int kind = misc[1];
             if (kind == SW_DONE) break;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
-                if (!mbar_wait(bar(B_UFULL + b), bu & 1, abort_flag)) { ok = false; break; }
-                if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), (c / TC_NST) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bar(B_UFULL + b), bu & 1, abort_flag, wcap)) { ok = false; break; }
+                if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), (c / TC_NST) & 1, abort_flag, wcap)) { ok = false; break; }
                 tc_fence_after();
                 if (kind != SW_MAX) {
                     const uint32_t bsm = sb_u + SM_KV + s * STAGE + (kind == SW_OUT ? KBLK : 0);
@@ -413,6 +435,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     mbar_arrive(bar(B_BUFFREE + b));
                 }
             }
+        }
+        if (*abort_flag) {      // an aborted block: the MMAs this warp issued must be done before TMEM and shared memory go
+            tc_commit_el(el, bar(B_EXIT + 1));
+            (void)mbar_wait_landed(bar(B_EXIT + 1), 0, wcap);
         }
     } else {
         // ================================ compute warps ================================
@@ -457,18 +483,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             pair_sync();
             return fmaxf(buf[lrow], buf[128 + lrow]);
         };
-        int flag_sel = 0;
-        auto group_any = [&](bool v) {
-            volatile int* f = flags + flag_sel * 8;
-            flag_sel ^= 1;
-            const int any = __any_sync(0xffffffffu, v);
-            if (lane == 0) f[warp] = any;
-            named_sync_compute();
-            int r = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) r |= f[i];
-            return r != 0;
-        };
+        // OR over the 256 compute threads
+        auto group_any = [&](bool v) { return bar_or(1, TC_COMPUTE, v); };
+        // After the waits of a sweep every compute thread learns whether any of them gave up, so that all of them
+        // take the same path from there on: a thread whose waits all succeeded must not go on to a pair
+        // exchange with a partner that has left.
+        auto all_ok = [&](bool mine) { return !bar_or(1, TC_COMPUTE, !mine); };
         // store this thread's NCOL fp32 values of the row as bf16 hi/lo into the swizzled operand tiles
         auto write_operand = [&](const float* vec) {
 #pragma unroll
@@ -565,7 +585,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int c = 0; c < nblk; ++c, ++blk) {
                 if (!split && (int)(blk & 1) != half) continue;
                 const uint32_t b = blk % TC_NBUF;
-                if (!mbar_wait(bar(B_SAFULL + b), (blk / TC_NBUF) & 1, abort_flag)) { ok = false; return part; }
+                if (!mbar_wait(bar(B_SAFULL + b), (blk / TC_NBUF) & 1, abort_flag, wcap)) { ok = false; return part; }
                 tc_fence_after();
 #pragma unroll 1
                 for (int h = split ? half : 0; h < (split ? half + 1 : 2); ++h) {
@@ -641,7 +661,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // read this thread's NCOL ACC columns after the sweep's last MMA
         uint32_t acc_uses = 0;
         auto read_acc = [&](float* dst) {
-            if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag)) { ok = false; return; }
+            if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag, wcap)) { ok = false; return; }
             ++acc_uses;
             tc_fence_after();
 #pragma unroll
@@ -696,6 +716,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         start_sweep(SW_MAX);
         {
             const float part = sweep(SW_MAX);
+            ok = all_ok(ok);
             if (ok) mx2 = pair_max(part);
         }
         // ---- sweep 1: omega and kbar ----
@@ -704,6 +725,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const float part = sweep(SW_STATS);
             float acc[NCOL];
             if (ok) read_acc(acc);
+            ok = all_ok(ok);
             if (ok) {
                 omega = pair_sum(part);
                 inv_omega = 1.f / omega;
@@ -745,6 +767,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             sweep(cheap ? SW_CG16 : SW_CG);
             float ap[NCOL];
             if (ok) read_acc(ap);
+            ok = all_ok(ok);
             if (!ok) break;
             // (the loops below keep four independent partial sums and move the row-vector state in
             //  batches of eight so that the loads overlap: two warps per scheduler hide no latency)
@@ -836,6 +859,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const float part = sweep(SW_OUT);
             float o[NCOL];
             if (ok) read_acc(o);
+            ok = all_ok(ok);
             if (ok) {
                 den = pair_sum(part);
                 if (row_ok) {
@@ -868,10 +892,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
 
     // ================================ common exit ================================
-    if (*abort_flag) {
-        // let copies that are still in flight land before the block's shared memory goes away
-        for (int i = 0; i < 64; ++i) __nanosleep(1000);
-    }
+    // (on an aborted run the TMA warp and the MMA warps have waited above for what they had issued)
     tc_fence_before();
     __syncthreads();
     if (warp == 8) {
@@ -981,6 +1002,8 @@ int launch_t(const ForwardArgs& a) {
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
     prm.precise_iters = a.precise_iters;
     prm.precise_iters_early = a.precise_iters_early;
+    prm.wait_clocks = a.wait_clocks > 0 ? a.wait_clocks : kWaitClocks;
+    prm.no_loads = a.no_loads;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
     prm.rhs = a.rhs; prm.sol = a.sol;

@@ -42,32 +42,36 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_test(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (true) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_test(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > (1ll << 31)) {
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-// Bounded wait: gives up after ~2^31 clock ticks or as soon as another thread flagged an abort.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+constexpr long long kWaitClocks = 1ll << 31;   // default cap of a bounded wait (about a second)
+// Bounded wait: gives up after `cap` clock ticks or as soon as another thread flagged an abort.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long cap = kWaitClocks) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > (1ll << 31)) {
+        if (clock64() - t0 > cap) {
             *abort_flag = 1;
             return false;
         }
     }
+}
+// Bounded wait of the exit path: for work this thread issued itself (copies, MMAs) to finish before the
+// block's shared memory and TMEM go away.  Ignores the abort flag, which is already set there.
+__device__ __forceinline__ bool mbar_wait_landed(uint32_t bar, uint32_t parity, long long cap = kWaitClocks) {
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity))
+        if (clock64() - t0 > cap) return false;
+    return true;
+}
+// OR of a predicate over the threads of named barrier `id` (every thread gets the result)
+__device__ __forceinline__ bool bar_or(int id, int threads, bool v) {
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+                 "barrier.cta.red.or.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r) : "r"((uint32_t)v), "r"(id), "r"(threads) : "memory");
+    return r != 0;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }

@@ -290,6 +290,27 @@ def test_host_buffer_entry_points(oracle):
     assert row_err(hout.numpy(), dref).max() <= TOL_BF16
 
 
+def test_bounded_waits_run_out_and_the_context_stays_usable(oracle):
+    # Failure detection without a fault: with the kernel's copy-issuing warp told to issue nothing, no barrier of a
+    # block is ever completed, so every role's bounded wait runs out (cap 2^20 clocks, about half a millisecond)
+    # with no copy or MMA in flight; the blocks release their tensor memory and leave, the call reports the
+    # time-outs in the status words, and the next call on the same context is correct.
+    w = inputs.CONFIGS[2].shrink(B=1, H=1, n=256, seed=41)
+    q, k, v = inputs.make_prefill(w)
+    ref = oracle.forward(q, k, v, w.scale, w.lam)
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    got = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, device_status=status,
+                  debug_wait_clocks=1 << 20, debug_flags=L.LLA_DEBUG_NO_LOADS)
+    tiles = 2                                            # rows 95..127 of the first tile, the second tile
+    assert status.cpu().tolist()[L.STATUS_TIMEOUT] == tiles
+    assert np.isnan(got[0, 0, 95:]).all()                # the iterative rows were left unwritten
+    assert row_err(got[0, 0, :95], ref[0, 0, :95]).max() <= TOL_BF16     # the direct rows (fewer than 96 keys) are another kernel
+    for _ in range(2):
+        got = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, device_status=status)
+        assert status.cpu().tolist()[L.STATUS_TIMEOUT] == 0
+        assert row_err(got, ref).max() <= TOL_BF16
+
+
 def test_host_buffer_forward_from_two_threads(oracle):
     # two host threads, each with its own stream and its own problem, in the chunked host-buffer form at the same
     # time: the library's worker streams and events are shared per device, so the calls must not mix them up
