@@ -91,20 +91,51 @@ def make_prefill(w: Workload):
         if w.name.startswith("cfg1"):
             v = v * np.float32(1.0 / np.sqrt(d))   # the fp32 n = 256, d = 16 case scales q, k and v alike
     elif w.recipe == "regression":
-        keys = rng.standard_normal((B, H, n + 1, d), dtype=np.float32) * inv
+        keys, A, noise = _regression_draws(w, rng)
         k = keys[:, :, :n]
         q = keys[:, :, 1:]                        # the query at position i is the next key
-        nseg = (n + w.segment - 1) // w.segment
-        A = rng.standard_normal((B, H, nseg, dv, d), dtype=np.float32) * inv
-        noise = rng.standard_normal((B, H, n, dv), dtype=np.float32)
         v = np.empty((B, H, n, dv), dtype=np.float32)
-        for s in range(nseg):
+        for s in range(A.shape[2]):
             lo, hi = s * w.segment, min(n, (s + 1) * w.segment)
             v[:, :, lo:hi] = np.einsum("bhvd,bhjd->bhjv", A[:, :, s], k[:, :, lo:hi]) \
-                + np.float32(0.1) * noise[:, :, lo:hi]
+                + np.float32(REGRESSION_NOISE) * noise[:, :, lo:hi]
     else:
         raise ValueError(w.recipe)
     return _finish(q, w.dtype), _finish(k, w.dtype), _finish(v, w.dtype)
+
+
+REGRESSION_NOISE = 0.1     # standard deviation of the value noise of the regression recipe
+
+
+def _regression_draws(w: Workload, rng):
+    """The regression recipe's random draws, in the order make_prefill consumes them: n + 1 keys, one linear map
+    per segment, the value noise."""
+    B, H, n, d, dv = w.B, w.H, w.n, w.d, w.dv
+    inv = np.float32(1.0 / np.sqrt(d))
+    keys = rng.standard_normal((B, H, n + 1, d), dtype=np.float32) * inv
+    nseg = (n + w.segment - 1) // w.segment
+    A = rng.standard_normal((B, H, nseg, dv, d), dtype=np.float32) * inv
+    noise = rng.standard_normal((B, H, n, dv), dtype=np.float32)
+    return keys, A, noise
+
+
+def regression_targets(w: Workload) -> np.ndarray:
+    """For the regression recipe: the noise-free value of the query at every position, A_s q_i with s the segment
+    of the NEXT position (query i is key i + 1), [B,H,n,dv] float32.  A regressor that has identified the
+    current segment's linear map predicts exactly this; at a segment's last position the query already belongs to
+    the next segment, whose map nothing seen so far determines."""
+    assert w.recipe == "regression"
+    keys, A, _ = _regression_draws(w, np.random.default_rng(w.seed))
+    n = w.n
+    out = np.empty((w.B, w.H, n, w.dv), dtype=np.float32)
+    nseg = A.shape[2]
+    for s in range(nseg + 1):
+        lo, hi = max(0, s * w.segment - 1), min(n, (s + 1) * w.segment - 1)     # positions whose next position lies in s
+        if lo >= hi:
+            continue
+        a_s = A[:, :, min(s, nseg - 1)]
+        out[:, :, lo:hi] = np.einsum("bhvd,bhjd->bhjv", a_s, keys[:, :, lo + 1:hi + 1])
+    return out
 
 
 def make_upstream_grad(w: Workload, dtype: str = "f32") -> np.ndarray:

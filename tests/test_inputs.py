@@ -54,3 +54,15 @@ def test_decode_workload_and_sharding():
     assert cover == list(range(10))
     rows = inputs.sample_rows(inputs.CONFIGS[2], per_head=8, heads=3, dense_below=16)
     assert rows.min() >= 0 and rows.max() < 32 * 1024 and len(np.unique(rows)) == len(rows)
+
+
+def test_regression_targets_are_the_noise_free_next_values():
+    # target_i = A_s q_i with s the segment of position i + 1 and q_i = k_{i+1}: equal to v_{i+1} minus its noise,
+    # also across a segment boundary (bf16 rounding of v is the only other difference)
+    w = inputs.CONFIGS[3].shrink(B=1, H=2, n=300, segment=64, dtype="f32")
+    q, k, v = inputs.make_prefill(w)
+    t = inputs.regression_targets(w)
+    resid = (t[:, :, :-1] - v[:, :, 1:]) / inputs.REGRESSION_NOISE
+    assert abs(resid.std() - 1.0) < 0.05 and abs(resid.mean()) < 0.05
+    per_pos = np.abs(resid).max(axis=(0, 1, 3))
+    assert per_pos.max() < 6.0            # no position (boundaries included) is off by more than noise
