@@ -213,12 +213,14 @@ class Prefill:
         nws = L.lla_forward_workspace_bytes(w.B, w.H, w.n, w.d, w.dv)
         self.ws = torch.empty(max(nws, 256), dtype=torch.uint8, device="cuda") if nws else None
         self.ws_bytes = nws
+        self.precondition = 0
 
     def step(self, i, phases=0):
         w, L = self.w, self.L
         q, k, v = self.sets[i % self.rot]
         L.lla_forward_ex(q, k, v, self.outs[i % self.rot], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1,
-                         phases=phases, workspace=self.ws, workspace_bytes=self.ws_bytes, stream=self.sp)
+                         phases=phases, workspace=self.ws, workspace_bytes=self.ws_bytes, stream=self.sp,
+                         cg_precondition=self.precondition)
 
     def probe(self):
         """Iterations actually executed (for the algorithmic flop count) and an fp32 copy of set 0's
@@ -266,6 +268,27 @@ class Prefill:
                 "direct_rows_ms_per_launch": ms_direct, "sm_mhz": c["sm_mhz"],
                 "ms_x_mhz": ms_kernel * c["sm_mhz"] if c["sm_mhz"] else None}
 
+    def preconditioned(self, peaks, steps, warmup):
+        """The same step with cg_precondition = 1 (inverse key covariance per block of 128 keys as CG preconditioner,
+        built by a pre-pass inside the timed call): fewer iterations, so fewer algorithmic flops and less time."""
+        w, L, torch = self.w, self.L, self.torch
+        self.precondition = 1
+        iters = torch.zeros((w.B, w.H, w.n), dtype=torch.int32, device="cuda")
+        L.lla_forward_ex(*self.sets[0], self.outs[0], w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, causal=1, iters=iters,
+                         workspace=self.ws, workspace_bytes=self.ws_bytes, stream=self.sp, cg_precondition=1)
+        torch.cuda.synchronize()
+        it = iters.cpu().numpy()
+        ms, clk = self.timed(steps, warmup)
+        self.precondition = 0
+        ms /= steps
+        fl = algorithmic_flops(w, it)
+        cg = it[it >= 0]
+        c = clk.summary()
+        return {"ms_per_step": ms, "tokens_per_s": w.B * w.n / (ms * 1e-3), "cg_mean_iters": float(cg.mean()) if cg.size else 0.0,
+                "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_bf16_peak_whole_step": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                "sm_mhz": c["sm_mhz"], "note": "optional mode (lla_forward_params.cg_precondition = 1); pre-pass kernels "
+                "inside the timed step; flops count the iterations executed, which this mode roughly halves"}, clk
+
     def solver(self):
         L = self.L
         cg = self.iters[self.iters >= 0]
@@ -284,13 +307,14 @@ def measure_leg(L, torch, peaks, w, local, steps, warmup):
     ms_d, _ = p.timed(steps, 3, L.LLA_PHASE_DIRECT)
     ms_step = ms_all / steps
     c = clk_all.summary()
-    leg = {"config": workload_config(w), "steps": steps, "ms_per_step": ms_step,
+    pre, clk_p = p.preconditioned(peaks, max(10, steps // 2), 3)
+    leg = {"config": workload_config(w), "steps": steps, "ms_per_step": ms_step, "preconditioned": pre,
            "tokens_per_s": w.B * w.n / (ms_step * 1e-3),
            "tflops": algorithmic_flops(w, p.iters) / (ms_step * 1e-3) / 1e12,
            "frac_of_bf16_peak_whole_step": algorithmic_flops(w, p.iters) / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
            "sm_mhz": c["sm_mhz"], "ms_x_mhz": ms_step * c["sm_mhz"] if c["sm_mhz"] else None,
            "roofline": p.roofline(peaks, ms_k / steps, ms_d / steps, clk_k), "solver": p.solver()}
-    return leg, p, [clk_all, clk_k]
+    return leg, p, [clk_all, clk_k, clk_p]
 
 
 def run_ours(args):
@@ -340,6 +364,9 @@ def run_ours(args):
     samplers.append(clk_k)
     ms_kernel /= args.steps
     ms_direct /= args.steps
+
+    pre_leg, clk_p = head.preconditioned(peaks, max(5, args.steps // 2), 3)
+    samplers.append(clk_p)
 
     # ---- end to end through the host-buffer entry point (pinned memory) ----
     hq, hk, hv = head.host_bf16
@@ -400,7 +427,7 @@ def run_ours(args):
         "tflops": flops_step / (ms_step * 1e-3) / 1e12,
         "frac_of_bf16_peak_whole_step": flops_step / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
         "sm_mhz": c_head["sm_mhz"], "ms_x_mhz": ms_step * c_head["sm_mhz"] if c_head["sm_mhz"] else None,
-        "roofline": roof,
+        "roofline": roof, "preconditioned": pre_leg,
         "e2e": {"value": world * tokens_step * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": int(pout.numel() * 2), "steps": e2e_steps,
                 "ms_per_step": 1e3 * e2e_s / e2e_steps,

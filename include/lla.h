@@ -182,6 +182,14 @@ typedef struct lla_forward_params {
                        tiles within the first 8 d positions, which converge more slowly); n > 0 = n
                        iterations for every tile; LLA_CG_PRECISE_ALL = every iteration with pairs;
                        LLA_CG_PRECISE_NONE = fp16 from the first iteration on */
+    int cg_precondition;  /* tensor-core kernel only.  0 = plain conjugate gradients as in Algorithm 2 (default).
+                       1 = preconditioned with the inverse covariance of the visible keys: one d x d matrix per
+                       block of 128 keys, built by a pre-pass into `workspace` (plain CG without room for it
+                       there).  The system of a row is that covariance under the row's attention weights, so the
+                       closer the weights are to uniform the fewer iterations remain -- about half on the
+                       synthetic workloads; with sharply peaked weights it may not pay for its pre-pass.  The
+                       solution is the same within the tolerance; a row on which the rounded matrix turns out
+                       not to be positive definite carries on with plain CG */
     long long debug_wait_clocks; /* tensor-core kernel only: cap, in SM clocks, of every bounded wait on a barrier
                        inside the kernel (0 = default, about 2^31).  A wait that runs out makes its thread block
                        stop: the block waits for the copies and MMAs it has issued itself, releases its tensor

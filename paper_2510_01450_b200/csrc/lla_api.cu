@@ -78,6 +78,7 @@ int check_forward(const lla_forward_params* p) {
     if (p->q_rows < 0 || p->q_rows > p->n) return LLA_ERR_INVALID_ARG;
     if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
     if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
+    if (p->cg_precondition < 0 || p->cg_precondition > 1) return LLA_ERR_INVALID_ARG;
     if (p->debug_wait_clocks < 0 || (p->debug_flags & ~LLA_DEBUG_NO_LOADS)) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535 || (p->n + 127) / 128 > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
@@ -111,6 +112,7 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     a.window = p->window;
     a.wait_clocks = p->debug_wait_clocks;
+    a.precondition = p->cg_precondition > 0 ? 1 : 0;
     a.no_loads = (p->debug_flags & LLA_DEBUG_NO_LOADS) ? 1 : 0;
     if (p->cg_precise_iters != 0) {
         a.precise_iters = p->cg_precise_iters == LLA_CG_PRECISE_NONE ? 0 : p->cg_precise_iters < 0 ? (1 << 30) : p->cg_precise_iters;

@@ -71,6 +71,8 @@ struct ForwardArgs {
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
     long long wait_clocks = 0;  // tensor-core kernel: cap of its bounded waits in SM clocks (0: default) and a test
     int no_loads = 0;           // aid: issue no copy at all (lla_forward_params.debug_*)
+    const void* minv = nullptr; // CG preconditioner matrices (fp16), set by forward_tensor_prepass when enabled
+    int precondition = 0;       // 1: preconditioned CG when the workspace has room for the matrices
     const void* k16 = nullptr;  // fp16 copy of k and its validity word, set by forward_tensor_prepass
     const int* f16_ok = nullptr;
     int precise_iters = 1;      // tensor-core kernel: CG iterations run with bf16 hi + lo operand pairs before the
@@ -143,6 +145,11 @@ bool forward_tensor_supported(const ForwardArgs& a);
 int forward_tensor_prepass(ForwardArgs& a);    // fp16 copy of k into the workspace (no-op without room)
 size_t forward_tensor_scratch_bytes();         // d = 128 row-state scratch (0 if the device cannot be queried)
 size_t forward_tensor_workspace_bytes(int B, int H, int n, int d);   // that scratch + the fp16 copy of k (upper bound: kv heads = H)
+// CG preconditioner of the tensor-core forward (lla_precond.cu): one d x d fp16 matrix per block of 128 keys
+int precond_blocks(int n);
+size_t precond_gram_bytes(int units, int n, int d);     // fp32 running Gram sums (scratch of the pre-pass)
+size_t precond_minv_bytes(int units, int n, int d);     // the fp16 matrices [units][blocks][d][d]
+int launch_precond(const void* k, int units, int n, int d, float lambda, int window, void* gram, void* minv, cudaStream_t st);
 int launch_decode(const DecodeArgs& a);
 int launch_head_rows_decode(const DecodeArgs& a);
 bool decode_tensor_supported(const DecodeArgs& a);

@@ -48,6 +48,8 @@ constexpr int TC_THREADS = 352;      // + TMA warp + two MMA warps
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_NBUF = 3;           // S/A/U buffers in TMEM (128 columns each)
 constexpr int TC_ACC_COL = TC_NBUF * 128;   // ACC columns [384, 384 + D)
+constexpr int TC_R_COL = 0;                 // preconditioner product, between sweeps: R (fp16) in buffer 0's columns,
+constexpr int TC_Z_COL = 128;               // Z = R M (fp32, D columns) from buffer 1's columns on
 constexpr int TC_NST_MAX = 4;
 constexpr int TC_ORDER_MAX = 256;    // launch-order table size (query tiles)
 constexpr int TC_SPLIT_MAX = 4;      // sweeps of at most this many key blocks run in split mode (see the compute role)
@@ -77,8 +79,8 @@ struct TcCfg {
     static constexpr int SM_KV = SM_PLO + OPER_BYTES;
     static constexpr int SM_X = SM_KV + NST * STAGE_BYTES;                        // fp32 [D][128] (D = 64 only)
     static constexpr int SM_KBAR = SM_X + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);
-    static constexpr int SM_RED = SM_KBAR + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);  // pair reductions 2 x 2 x 2 x 128 floats
-    static constexpr int SM_FLAGS = SM_RED + 4096;                                // 2 x 8 ints
+    static constexpr int SM_RED = SM_KBAR + (STATE_IN_SMEM ? D * TC_BR * 4 : 0);  // pair reductions: 2 buffers x 4 values x 2 x 128 floats
+    static constexpr int SM_FLAGS = SM_RED + 8192;                                // 2 x 8 ints
     static constexpr int SM_BAR = SM_FLAGS + 64;                                  // mbarriers
     static constexpr int SM_MISC = SM_BAR + 256;                                  // tmem base, ctl kind, abort
     static constexpr int SM_TOTAL = SM_MISC + 64;
@@ -94,7 +96,8 @@ enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST_MAX, B_VFULL = B
        B_SAFULL = B_VFULL + TC_NST_MAX,
        B_UFULL = B_SAFULL + TC_NBUF, B_BUFFREE = B_UFULL + TC_NBUF, B_ACCFULL = B_BUFFREE + TC_NBUF, B_CTL = B_ACCFULL + 1,
        B_EXIT = B_CTL + 1,   // two: the MMA warps' last commits on an aborted run
-       B_COUNT = B_EXIT + 2 };
+       B_MFULL = B_EXIT + 2, // the preconditioner matrix has landed
+       B_COUNT = B_MFULL + 1 };
 static_assert(B_COUNT * 8 <= 256, "barrier area too small");
 
 // MMA issue.  The whole MMA warp runs these convergently and the instructions are predicated on the
@@ -152,6 +155,20 @@ __device__ __forceinline__ void mma_ts_k64(uint32_t el, uint32_t d, uint32_t a, 
         "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
         ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
 }
+// The same with the four 16-element steps of the TMEM operand in consecutive groups of 8 columns.
+__device__ __forceinline__ void mma_ts_k64c(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a1, %2, 8; add.u32 a2, %2, 16; add.u32 a3, %2, 24;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
 // Shared-memory matrix descriptors (128-byte swizzle, tile base 1024-byte aligned).
 //   K-major:  rows of 128 bytes, 8-row groups 1024 bytes apart; a 16-element K step is +32 bytes.
 //   MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements; 8-row groups
@@ -198,11 +215,12 @@ struct TcParams {
     unsigned short order[TC_ORDER_MAX];
 };
 
-template <int D, typename TOut>
+// PC: preconditioned CG compiled in (an instance of its own, so that the plain path carries none of its code)
+template <int D, typename TOut, bool PC>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmK16,
-                  TOut* __restrict__ out, const TcParams prm) {
+                  const __grid_constant__ CUtensorMap tmM, TOut* __restrict__ out, const TcParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     using Cfg = TcCfg<D>;
@@ -214,7 +232,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bars = sbase + SM_BAR;
     auto bar = [&](int i) { return bars + 8u * i; };
-    volatile int* misc = reinterpret_cast<volatile int*>(smem + SM_MISC);   // [0] tmem base, [1] kind, [2] abort
+    volatile int* misc = reinterpret_cast<volatile int*>(smem + SM_MISC);   // [0] tmem base, [2] abort, [3] kv unit, [4..5] kind
     volatile int* abort_flag = misc + 2;
     // row-vector state: shared memory (D = 64) or this SM's slot of the global scratch (D = 128)
     float* xs;
@@ -249,7 +267,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int cbeg = (prm.causal && prm.window > 0) ? max(0, off + r0 + 1 - prm.window) / TC_BC : 0;
     const int nblk = cend - cbeg;                        // key blocks per sweep: cbeg .. cend - 1
     const bool split = nblk <= TC_SPLIT_MAX;
-    // Operand format of a sweep, fixed by its index alone so that every role knows it without being told:
+    // Operand format of a sweep over the keys, fixed by its index among those sweeps alone so that every role
+    // knows it without being told (the preconditioner products in between do not count):
     // sweeps 0 (maxima), 1 (statistics) and the first precise_iters CG sweeps run on the bf16 inputs; every
     // later sweep (the remaining CG sweeps and, if CG got that far, the output sweep) runs its Q K^T and P K^T
     // products on fp16 copies of Q and K (one kind::f16 MMA takes both operands in the same 16-bit format).
@@ -275,7 +294,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_init(bar(B_CTL), TC_COMPUTE / 32);
         mbar_init(bar(B_EXIT), 1);
         mbar_init(bar(B_EXIT + 1), 1);
-        misc[1] = SW_MAX;
+        mbar_init(bar(B_MFULL), 1);
+        misc[4] = SW_MAX;
+        misc[5] = SW_MAX;
         misc[2] = 0;
         misc[3] = kv_unit(bh, prm.H, prm.kv_group);   // worked out here: in the producer's own path it delays the first loads
         fence_barrier_init();
@@ -301,6 +322,16 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int sub = 0; sub < KSUB; ++sub)
                 tma_load_3d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, bh);
             const int kvh = misc[3];
+            if (PC) {
+                // the preconditioner of this tile's key range: D x D fp16, laid out like D / 64 key blocks, into the
+                // V halves of the first ring stages (idle until the output sweep, when it is no longer needed)
+                const int gm = (prm.causal ? min(n - 1, off + r0 + TC_BR - 1) : n - 1) / 128;
+                mbar_expect_tx(bar(B_MFULL), D * D * 2);
+                for (int rb = 0; rb < D / 64; ++rb)
+                    for (int sub = 0; sub < KSUB; ++sub)
+                        tma_load_3d(sbase + SM_KV + rb * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmM, bar(B_MFULL), 64 * sub,
+                                    gm * D + 64 * rb, kvh);
+            }
             uint32_t kit = 0;      // K blocks issued so far
             int pre = 0;           // blocks of the coming sweep already issued
             bool ok = true;
@@ -323,9 +354,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int sub = 0; sub < KSUB; ++sub)
                     tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
             };
-            for (uint32_t sweep = 0; ok; ++sweep) {
-                if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag, wcap)) break;
-                const int kind = misc[1];
+            int sweep = 0;         // index among the sweeps over the keys
+            for (uint32_t ctl = 0; ok; ++ctl) {
+                if (!mbar_wait(bar(B_CTL), ctl & 1, abort_flag, wcap)) break;
+                const int kind = misc[4 + (ctl & 1)];
                 if (kind == SW_DONE) {
                     // prefetched blocks nobody will consume: wait until they have landed
                     for (int i = 0; i < pre; ++i) {
@@ -344,8 +376,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 pre = 0;
                 if (kind != SW_OUT)
                     for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c, (int)sweep + 1 >= f16_from); ++pre; }
+                ++sweep;
             }
             if (*abort_flag) {
+                if (PC) (void)mbar_wait_landed(bar(B_MFULL), 0, wcap);
                 // an aborted block: the copies issued above write into this block's shared memory, so they must
                 // have landed before the block exits (on a completed run their consumers have waited for them)
                 (void)mbar_wait_landed(bar(B_QFULL), 0, wcap);
@@ -371,12 +405,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint64_t phdesc = make_desc(sb_u + SM_PHI);
         const uint64_t pldesc = make_desc(sb_u + SM_PLO);
         uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it % NBUF)
-        for (uint32_t sweep = 0; ok; ++sweep) {
-            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag, wcap)) break;
-            const int kind = misc[1];
+        int sweep = 0;     // index among the sweeps over the keys
+        for (uint32_t ctl = 0; ok; ++ctl) {
+            if (!mbar_wait(bar(B_CTL), ctl & 1, abort_flag, wcap)) break;
+            const int kind = misc[4 + (ctl & 1)];
             if (kind == SW_DONE) break;
             tc_fence_after();
-            const uint32_t idesc = (int)sweep >= f16_from ? IDESC_SS16 : IDESC_SS;
+            const uint32_t idesc = sweep >= f16_from ? IDESC_SS16 : IDESC_SS;
+            ++sweep;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
                 if (!mbar_wait(bar(B_KVFULL + s), (it / TC_NST) & 1, abort_flag, wcap)) { ok = false; break; }
@@ -413,9 +449,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
         bool ok = true;
         uint32_t it = 0;
-        for (uint32_t sweep = 0; ok; ++sweep) {
-            if (!mbar_wait(bar(B_CTL), sweep & 1, abort_flag, wcap)) break;
-            const int kind = misc[1];
+        for (uint32_t ctl = 0; ok; ++ctl) {
+            if (!mbar_wait(bar(B_CTL), ctl & 1, abort_flag, wcap)) break;
+            const int kind = misc[4 + (ctl & 1)];
             if (kind == SW_DONE) break;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
@@ -460,7 +496,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + quad) : "memory"); };
         int red_sel = 0;
         auto pair_sum = [&](float v) {
-            float* buf = red + red_sel * 512;
+            float* buf = red + red_sel * 1024;
             red_sel ^= 1;
             buf[half * 128 + lrow] = v;
             pair_sync();
@@ -468,7 +504,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         };
         // two sums for one barrier
         auto pair_sum2 = [&](float& a, float& b) {
-            float* buf = red + red_sel * 512;
+            float* buf = red + red_sel * 1024;
             red_sel ^= 1;
             buf[half * 128 + lrow] = a;
             buf[256 + half * 128 + lrow] = b;
@@ -476,8 +512,22 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             a = buf[lrow] + buf[128 + lrow];
             b = buf[256 + lrow] + buf[384 + lrow];
         };
+        // four sums for one barrier
+        auto pair_sum4 = [&](float& a, float& b, float& c, float& d4) {
+            float* buf = red + red_sel * 1024;
+            red_sel ^= 1;
+            buf[half * 128 + lrow] = a;
+            buf[256 + half * 128 + lrow] = b;
+            buf[512 + half * 128 + lrow] = c;
+            buf[768 + half * 128 + lrow] = d4;
+            pair_sync();
+            a = buf[lrow] + buf[128 + lrow];
+            b = buf[256 + lrow] + buf[384 + lrow];
+            c = buf[512 + lrow] + buf[640 + lrow];
+            d4 = buf[768 + lrow] + buf[896 + lrow];
+        };
         auto pair_max = [&](float v) {
-            float* buf = red + red_sel * 512;
+            float* buf = red + red_sel * 1024;
             red_sel ^= 1;
             buf[half * 128 + lrow] = v;
             pair_sync();
@@ -660,10 +710,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         };
         // read this thread's NCOL ACC columns after the sweep's last MMA
         uint32_t acc_uses = 0;
-        auto read_acc = [&](float* dst) {
+        // (in two steps, so that the threads can agree on success between the wait and the loads: no array of
+        //  accumulator values is live across that barrier)
+        auto acc_wait = [&]() {
             if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag, wcap)) { ok = false; return; }
             ++acc_uses;
             tc_fence_after();
+        };
+        auto acc_load = [&](float* dst) {
 #pragma unroll
             for (int cb = 0; cb < NCOL; cb += 32) {
                 uint32_t v[32];
@@ -675,10 +729,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tc_fence_before();
         };
         int sweeps_started = 0;
+        uint32_t ctl_phase = 0;
         auto start_sweep = [&](int kind) {
             if (sweeps_started >= f16_from && !q_is_f16) convert_q();
             ++sweeps_started;
-            if (tid == 0) misc[1] = kind;
+            if (tid == 0) misc[4 + (ctl_phase & 1)] = kind;
+            ++ctl_phase;
             fence_proxy_async();       // operand tiles written with ordinary stores -> visible to the MMA
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(B_CTL));
@@ -712,6 +768,54 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         };
 
+        // z = M r with the tile's preconditioner: vec holds this thread's NCOL entries of r on entry (|r|^2 is about
+        // nrm2 over the whole row) and of z on return.  r goes to TMEM as fp16, scaled by a power of two into the
+        // middle of the fp16 range (M is stored with a largest entry of one); once every compute thread has stored
+        // its part, warp 0 issues the product Z = R M itself (no hand-over to the MMA warps, which are idle between
+        // sweeps, as are the TMEM columns of the S/A/U buffers that R and Z use).
+        const uint32_t el0 = PC ? elect_one() : 0u;
+        const uint32_t sb_c = PC ? __shfl_sync(0xffffffffu, sbase, 0) : 0u, tm_c = PC ? __shfl_sync(0xffffffffu, tmem, 0) : 0u;
+        bool m_ready = false;
+        auto precondition = [&](float* vec, float nrm2) {
+            const int e2 = (int)((__float_as_uint(nrm2) >> 23) & 0xffu) - 127;
+            const int k = max(-100, min(100, -(e2 >> 1)));
+            const float sc = __uint_as_float((uint32_t)(127 + k) << 23), isc = __uint_as_float((uint32_t)(127 - k) << 23);
+            uint32_t pk[NCOL / 2];
+#pragma unroll
+            for (int e = 0; e < NCOL / 2; ++e) pk[e] = pack_f16(vec[2 * e] * sc, vec[2 * e + 1] * sc);
+            const uint32_t r_addr = tmem + lane_addr + TC_R_COL + half * (NCOL / 2);
+            if constexpr (NCOL == 32) tmem_st16(r_addr, pk);
+            else tmem_st32(r_addr, pk);
+            tc_wait_st();
+            tc_fence_before();
+            named_sync_compute();
+            if (warp == 0) {
+                if (!m_ready) m_ready = mbar_wait(bar(B_MFULL), 0, abort_flag, wcap);     // the matrix has landed (first use)
+                tc_fence_after();
+                if (m_ready) {
+#pragma unroll
+                    for (int rb = 0; rb < D / 64; ++rb)
+                        mma_ts_k64c(el0, tm_c + TC_Z_COL, tm_c + TC_R_COL + 32 * rb,
+                                    make_desc(sb_c + SM_KV + rb * STAGE + KBLK, Cfg::KSUB_BYTES), IDESC_TS16, rb > 0);
+                    tc_commit_el(el0, bar(B_ACCFULL));
+                }
+            }
+            if (!mbar_wait(bar(B_ACCFULL), acc_uses & 1, abort_flag, wcap)) { ok = false; return; }
+            ++acc_uses;
+            tc_fence_after();
+#pragma unroll
+            for (int cb = 0; cb < NCOL; cb += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_addr + TC_Z_COL + c0 + cb, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) vec[cb + e] = __uint_as_float(v[e]) * isc;
+            }
+            tc_fence_before();
+        };
+        float rz = 0.f;      // r . z of the preconditioned recurrence
+        bool prec_row = true;   // false once the preconditioner has failed this row (z = r from then on)
+
         // ---- sweep 0: row maxima ----
         start_sweep(SW_MAX);
         {
@@ -723,10 +827,11 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (ok) {
             start_sweep(SW_STATS);
             const float part = sweep(SW_STATS);
-            float acc[NCOL];
-            if (ok) read_acc(acc);
+            if (ok) acc_wait();
             ok = all_ok(ok);
             if (ok) {
+                float acc[NCOL];
+                acc_load(acc);
                 omega = pair_sum(part);
                 inv_omega = 1.f / omega;
                 const float lam_i = (prm.lambda_rows && row < nq) ? prm.lambda_rows[(size_t)bh * nq + row] : prm.lambda;
@@ -755,9 +860,34 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 stop = prm.tol * prm.tol * rr;
                 active = row_ok && rr > 0.f;
                 pn2 = rr;
-                write_p(0);
+                rz = rr;
             }
         }
+        if (ok && PC) {
+            // preconditioned start: p = z = M r, with r . z, kbar . z and |z|^2 for the recurrences
+            precondition(p, rr);
+            ok = all_ok(ok);
+            if (ok) {
+                float rz_p = 0.f, kz_p = 0.f, zz_p = 0.f, unused = 0.f;
+#pragma unroll
+                for (int e = 0; e < NCOL; ++e) {
+                    rz_p = fmaf(r_get(e), p[e], rz_p);
+                    kz_p = fmaf(kbs[(c0 + e) * TC_BR + lrow], p[e], kz_p);
+                    zz_p = fmaf(p[e], p[e], zz_p);
+                }
+                pair_sum4(rz_p, kz_p, zz_p, unused);
+                if (rz_p > 0.f) {
+                    rz = rz_p; abar = kz_p; pn2 = zz_p;
+                } else {
+                    // the rounded matrix is not positive on this residual: the row runs unpreconditioned
+                    // (abar, pn2 and rz already hold the values for p = r)
+                    prec_row = false;
+#pragma unroll
+                    for (int e = 0; e < NCOL; ++e) p[e] = r_get(e);
+                }
+            }
+        }
+        if (ok) write_p(0);
         // ---- conjugate gradients (Algorithm 2) ----
         for (int t = 0; ok && t < prm.max_iters; ++t) {
             active = active && rr > stop;
@@ -765,14 +895,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const bool cheap = t + 2 >= f16_from;
             start_sweep(cheap ? SW_CG16 : SW_CG);
             sweep(cheap ? SW_CG16 : SW_CG);
-            float ap[NCOL];
-            if (ok) read_acc(ap);
+            if (ok) acc_wait();
             ok = all_ok(ok);
             if (!ok) break;
+            float ap[NCOL];
+            acc_load(ap);
             // (the loops below keep four independent partial sums and move the row-vector state in
             //  batches of eight so that the loads overlap: two warps per scheduler hide no latency)
             float pp[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
             const float acc_scale = cheap ? inv_omega * ipsc : inv_omega;
 #pragma unroll
             for (int e = 0; e < NCOL; ++e) {
@@ -781,7 +911,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             const float pap = pair_sum((pp[0] + pp[1]) + (pp[2] + pp[3]));
             if (active && !(pap > 0.f)) active = false;
-            const float alpha = active ? rr / pap : 0.f;
+            const float alpha = active ? rz / pap : 0.f;       // rz = |r|^2 without a preconditioner
             float r2[4] = {0.f, 0.f, 0.f, 0.f}, kr[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int e0 = 0; e0 < NCOL; e0 += 8) {
@@ -806,17 +936,65 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     r_set(e0 + i, rv[i]);
                 }
             }
-            // ||r_new||^2 and kbar . r_new in one exchange; kbar . p_new follows from the recurrence
             float rr2 = (r2[0] + r2[1]) + (r2[2] + r2[3]), kbr = (kr[0] + kr[1]) + (kr[2] + kr[3]);
-            pair_sum2(rr2, kbr);
-            if (active) {
-                const float beta = rr2 / rr;
+            if constexpr (!PC) {
+                // ||r_new||^2 and kbar . r_new in one exchange; kbar . p_new follows from the recurrence
+                pair_sum2(rr2, kbr);
+                if (active) {
+                    const float beta = rr2 / rr;
 #pragma unroll
-                for (int e = 0; e < NCOL; ++e) p[e] = fmaf(beta, p[e], ap[e]);
-                abar = fmaf(beta, abar, kbr);
-                pn2 = fmaf(beta * beta, pn2, rr2);
-                rr = rr2;
-                ++its;
+                    for (int e = 0; e < NCOL; ++e) p[e] = fmaf(beta, p[e], ap[e]);
+                    abar = fmaf(beta, abar, kbr);
+                    pn2 = fmaf(beta * beta, pn2, rr2);
+                    rr = rr2;
+                    rz = rr2;
+                    ++its;
+                }
+            } else {
+                // preconditioned: z = M r_new (ap <- z), then beta = (r_new . z_new) / (r . z), p = z + beta p;
+                // kbar . p and a bound on |p| follow from kbar . z and |z|
+                rr2 = pair_sum(rr2);
+                precondition(ap, rr2);
+                ok = all_ok(ok);
+                if (!ok) break;
+                float rz_p = 0.f, kz_p = 0.f, zz_p = 0.f;
+#pragma unroll
+                for (int e0 = 0; e0 < NCOL; e0 += 8) {
+                    float kv[8], rv[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        kv[i] = kbs[(c0 + e0 + i) * TC_BR + lrow];
+                        rv[i] = r_get(e0 + i);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (!prec_row) ap[e0 + i] = rv[i];           // a row whose preconditioner failed: z = r
+                        rz_p = fmaf(rv[i], ap[e0 + i], rz_p);
+                        kz_p = fmaf(kv[i], ap[e0 + i], kz_p);
+                        zz_p = fmaf(ap[e0 + i], ap[e0 + i], zz_p);
+                    }
+                }
+                pair_sum4(rz_p, kz_p, zz_p, kbr);
+                if (active) {
+                    float beta = rz_p / rz;
+                    if (!(rz_p > 0.f)) {
+                        // r . M r is not positive (the rounded matrix is not definite on this residual): restart the
+                        // row from its current x as plain CG, p = r
+                        prec_row = false;
+                        beta = 0.f;
+                        rz_p = rr2; kz_p = kbr; zz_p = rr2;
+#pragma unroll
+                        for (int e = 0; e < NCOL; ++e) ap[e] = r_get(e);
+                    }
+#pragma unroll
+                    for (int e = 0; e < NCOL; ++e) p[e] = fmaf(beta, p[e], ap[e]);
+                    abar = fmaf(beta, abar, kz_p);
+                    const float pn = sqrtf(zz_p) + fabsf(beta) * sqrtf(pn2);      // |p_new| <= |z| + |beta| |p|
+                    pn2 = pn * pn;
+                    rr = rr2;
+                    rz = rz_p;
+                    ++its;
+                }
             }
             write_p(t + 1);
         }
@@ -857,10 +1035,11 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             else write_operand(y);
             start_sweep(SW_OUT);
             const float part = sweep(SW_OUT);
-            float o[NCOL];
-            if (ok) read_acc(o);
+            if (ok) acc_wait();
             ok = all_ok(ok);
             if (ok) {
+                float o[NCOL];
+                acc_load(o);
                 den = pair_sum(part);
                 if (row_ok) {
                     const float inv_den = 1.f / den;
@@ -966,17 +1145,18 @@ float* scratch_for_device(size_t bytes) {
 // times more than the rest), so at short sequence lengths the first tiles are the longest blocks
 // even though their sweeps are the shortest.  The numbers are a fit to measured runs; they only
 // steer the order, never the result.
-void tile_order(TcParams& prm, int tiles, int first_tile, int n, int off, int d, int causal, int window) {
+void tile_order(TcParams& prm, int tiles, int first_tile, int n, int off, int d, int causal, int window, bool precond) {
     prm.use_order = 0;
     if (!causal || tiles > TC_ORDER_MAX) return;
     float cost[TC_ORDER_MAX];
     for (int t = 0; t < tiles; ++t) {
         const int r_end = std::min(n, off + (first_tile + t + 1) * TC_BR);      // keys the tile's last row sees
         const int seen = window > 0 ? std::min(r_end, window) : r_end;
-        const float its = 6.f + 50.f * (float)d / (float)seen;
+        const float x = (float)d / (float)seen;
+        const float its = precond ? std::min(16.f, 4.f + 190.f * x * x) : 6.f + 50.f * x;
         const int c_first = window > 0 ? std::max(0, off + (first_tile + t) * TC_BR + 1 - window) / TC_BC : 0;
         const float nblk = (float)((r_end + TC_BC - 1) / TC_BC - c_first);
-        cost[t] = (its + 3.f) * (6.f + nblk);
+        cost[t] = (its + 3.f) * (6.f + nblk) + (precond ? 3.f * its : 0.f);
         prm.order[t] = (unsigned short)t;
     }
     std::stable_sort(prm.order, prm.order + tiles, [&](unsigned short x, unsigned short y) { return cost[x] > cost[y]; });
@@ -991,12 +1171,13 @@ int launch_t(const ForwardArgs& a) {
     const int first_tile = a.causal ? hr / TC_BR : 0;
     const int tiles = (a.nq + TC_BR - 1) / TC_BR - first_tile;
     if (tiles <= 0) return LLA_OK;
-    CUtensorMap mq, mk, mv, mk16;
+    CUtensorMap mq, mk, mv, mk16, mm;
     const int BH = a.B * a.H;
     if (!make_map_bf16(&mq, a.q, BH, a.nq, D, TC_BR) || !make_map_bf16(&mk, a.k, BH / a.kv_group, a.n, D, TC_BC) ||
         !make_map_bf16(&mv, a.v, BH / a.kv_group, a.n, D, TC_BC))
         return LLA_ERR_CUDA;
     mk16 = mk;
+    mm = mk;
     TcParams prm;
     prm.n = a.n; prm.nq = a.nq; prm.causal = a.causal; prm.head_rows = a.head_rows > 0 ? a.head_rows : 0;
     prm.max_iters = a.max_iters; prm.first_tile = first_tile;
@@ -1016,7 +1197,7 @@ int launch_t(const ForwardArgs& a) {
     char* ws = static_cast<char*>(a.workspace);
     size_t ws_left = a.workspace ? a.workspace_bytes : 0;
     prm.window = a.causal ? a.window : 0;
-    tile_order(prm, tiles, first_tile, a.n, a.n - a.nq, D, a.causal, prm.window);
+    tile_order(prm, tiles, first_tile, a.n, a.n - a.nq, D, a.causal, prm.window, a.minv != nullptr);
     if constexpr (!Cfg::STATE_IN_SMEM) {
         int dev = 0, sms = 0;
         LLA_CUDA_TRY(cudaGetDevice(&dev));
@@ -1040,10 +1221,17 @@ int launch_t(const ForwardArgs& a) {
         if (!make_map_bf16(&mk16, a.k16, BH / a.kv_group, a.n, D, TC_BC, CU_TENSOR_MAP_DATA_TYPE_FLOAT16)) return LLA_ERR_CUDA;
         prm.f16_ok = a.f16_ok;
     }
-    auto kern = forward_tc_kernel<D, TOut>;
+    bool precond = false;
+    // preconditioned CG: only with the matrices that forward_tensor_prepass made ([units][blocks][D][D] fp16)
+    if (a.minv) {
+        if (!make_map_bf16(&mm, a.minv, BH / a.kv_group, precond_blocks(a.n) * D, D, 64, CU_TENSOR_MAP_DATA_TYPE_FLOAT16))
+            return LLA_ERR_CUDA;
+        precond = true;
+    }
+    auto kern = precond ? forward_tc_kernel<D, TOut, true> : forward_tc_kernel<D, TOut, false>;
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
     dim3 grid(BH, tiles);
-    kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, mk16, (TOut*)a.out, prm);
+    kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, mk16, mm, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -1058,7 +1246,8 @@ size_t forward_tensor_scratch_bytes() {
 }
 
 size_t forward_tensor_workspace_bytes(int B, int H, int n, int d) {
-    return (d == 128 ? forward_tensor_scratch_bytes() : 0) + f16_copy_bytes((size_t)B * H * n * d);
+    return (d == 128 ? forward_tensor_scratch_bytes() : 0) + f16_copy_bytes((size_t)B * H * n * d) +
+           precond_gram_bytes(B * H, n, d) + precond_minv_bytes(B * H, n, d);
 }
 
 // Enqueues the fp16 copy of k (and the range check of q and k) when the tail of the caller's workspace has
@@ -1066,6 +1255,7 @@ size_t forward_tensor_workspace_bytes(int B, int H, int n, int d) {
 int forward_tensor_prepass(ForwardArgs& a) {
     a.k16 = nullptr;
     a.f16_ok = nullptr;
+    a.minv = nullptr;
     if (!forward_tensor_supported(a) || !a.workspace) return LLA_OK;
     if (std::min(a.precise_iters, a.precise_iters_early) >= (1 << 29)) return LLA_OK;
     const size_t head = a.d == 128 ? forward_tensor_scratch_bytes() : 0;
@@ -1082,6 +1272,17 @@ int forward_tensor_prepass(ForwardArgs& a) {
     LLA_CUDA_TRY(cudaGetLastError());
     a.k16 = k16;
     a.f16_ok = okw;
+    // the preconditioner behind it, if enabled and there is room (Gram scratch, then the matrices)
+    const int units = a.B * a.H / a.kv_group;
+    const size_t used = head + f16_copy_bytes(k_elems);
+    const size_t gram_b = precond_gram_bytes(units, a.n, a.d), minv_b = precond_minv_bytes(units, a.n, a.d);
+    if (a.precondition && a.workspace_bytes >= used + gram_b + minv_b) {
+        char* gram = static_cast<char*>(a.workspace) + used;
+        char* minv = gram + gram_b;
+        const int rc = launch_precond(a.k, units, a.n, a.d, a.lambda, a.causal ? a.window : 0, gram, minv, a.stream);
+        if (rc != LLA_OK) return rc;
+        a.minv = minv;
+    }
     return LLA_OK;
 }
 
