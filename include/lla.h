@@ -124,8 +124,11 @@ int lla_decode_f32(const void *q, const void *kcache, const void *vcache, const 
  *               the other rows of `out` are left untouched)
  *   rho       : optional [B, H, n, d] fp32, the solutions Sigma_i^{-1} mu_i (Algorithm 1 keeps
  *               them for the backward pass)
- *   stats     : optional [B, H, n, 3] fp32: row maximum m_i of the scaled scores, omega_i and
- *               delta_i = omega_i - mu_i^T rho_i, the last two for weights exp(score - m_i)
+ *   stats     : optional [B, H, n, 3] fp32: a shift m_i of the scaled scores, omega_i and
+ *               delta_i = omega_i - mu_i^T rho_i, the last two for weights exp(score - m_i).  m_i is the row
+ *               maximum in the directly-solved rows and in the CUDA-core kernel; the tensor-core kernel uses
+ *               shift zero whenever every maximum of the row tile lies within 2^+-8 (Eq. "lla" does not depend on
+ *               the shift; m_i + log omega_i and m_i + log delta_i are the shift-free quantities)
  *   iters     : optional [B, H, n] int32, CG iterations executed for the row (-1 for rows solved
  *               directly)
  *   device_status : optional int[LLA_STATUS_WORDS] on the device

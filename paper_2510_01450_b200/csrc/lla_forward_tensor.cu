@@ -55,7 +55,7 @@ constexpr int TC_ORDER_MAX = 256;    // launch-order table size (query tiles)
 constexpr int TC_SPLIT_MAX = 4;      // sweeps of at most this many key blocks run in split mode (see the compute role)
 
 // SW_CG16: a CG sweep whose on-the-fly operands (P, U) are single fp16 values instead of bf16 hi + lo pairs
-enum SweepKind : int { SW_MAX = 0, SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4, SW_CG16 = 5 };
+enum SweepKind : int { SW_STATS = 1, SW_CG = 2, SW_OUT = 3, SW_DONE = 4, SW_CG16 = 5 };
 
 // Shared-memory carve-up (bytes, from a 1024-byte aligned base), per head size D (64 or 128).
 // Operand tiles are stored as D/64 sub-tiles of 64 columns (128-byte rows, 128B swizzle) one after
@@ -267,16 +267,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int cbeg = (prm.causal && prm.window > 0) ? max(0, off + r0 + 1 - prm.window) / TC_BC : 0;
     const int nblk = cend - cbeg;                        // key blocks per sweep: cbeg .. cend - 1
     const bool split = nblk <= TC_SPLIT_MAX;
-    // Operand format of a sweep over the keys, fixed by its index among those sweeps alone so that every role
-    // knows it without being told (the preconditioner products in between do not count):
-    // sweeps 0 (maxima), 1 (statistics) and the first precise_iters CG sweeps run on the bf16 inputs; every
-    // later sweep (the remaining CG sweeps and, if CG got that far, the output sweep) runs its Q K^T and P K^T
-    // products on fp16 copies of Q and K (one kind::f16 MMA takes both operands in the same 16-bit format).
-    // The values of the copies equal the bf16 inputs (the pre-pass checks the range).
-    // (tiles whose rows see fewer than 8 D keys converge more slowly and keep the pairs for more iterations)
+    // Operand format of a sweep over the keys.  The statistics sweep(s) and the first `precise` CG sweeps run on
+    // the bf16 inputs; every later sweep (the remaining CG sweeps and, if CG got that far, the output sweep) runs
+    // its Q K^T and P K^T products on fp16 copies of Q and K (one kind::f16 MMA takes both operands in the same
+    // 16-bit format).  The values of the copies equal the bf16 inputs (the pre-pass checks the range).  Every role
+    // counts the CG sweeps it has seen, so all of them know a sweep's format, and the next one's, without being
+    // told.  (Tiles whose rows see fewer than 8 D keys converge more slowly and keep the pairs for longer.)
     const int precise = off + r0 + TC_BR <= 8 * D ? prm.precise_iters_early : prm.precise_iters;
+    const bool f16_on = prm.f16_ok && *prm.f16_ok && precise < (1 << 29);
     const long long wcap = prm.wait_clocks;
-    const int f16_from = (prm.f16_ok && *prm.f16_ok && precise < (1 << 29)) ? precise + 2 : (1 << 30);
 
     if (tid == 0) {
         mbar_init(bar(B_QFULL), 1);
@@ -295,8 +294,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_init(bar(B_EXIT), 1);
         mbar_init(bar(B_EXIT + 1), 1);
         mbar_init(bar(B_MFULL), 1);
-        misc[4] = SW_MAX;
-        misc[5] = SW_MAX;
+        misc[4] = SW_STATS;
+        misc[5] = SW_STATS;
         misc[2] = 0;
         misc[3] = kv_unit(bh, prm.H, prm.kv_group);   // worked out here: in the producer's own path it delays the first loads
         fence_barrier_init();
@@ -354,7 +353,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int sub = 0; sub < KSUB; ++sub)
                     tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
             };
-            int sweep = 0;         // index among the sweeps over the keys
+            int cg_seen = 0;       // CG sweeps issued so far
             for (uint32_t ctl = 0; ok; ++ctl) {
                 if (!mbar_wait(bar(B_CTL), ctl & 1, abort_flag, wcap)) break;
                 const int kind = misc[4 + (ctl & 1)];
@@ -369,14 +368,19 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const uint32_t g0 = kit - pre;
                 if (kind == SW_OUT)
                     for (int c = 0; c < pre; ++c) issue_v(c, g0 + c);
+                const bool f16_cur = kind == SW_CG16 || (kind == SW_OUT && f16_on && cg_seen >= precise);
                 for (int c = pre; c < nblk && ok; ++c) {
-                    issue_k(c, (int)sweep >= f16_from);
+                    issue_k(c, f16_cur);
                     if (ok && kind == SW_OUT) issue_v(c, g0 + c);
                 }
                 pre = 0;
-                if (kind != SW_OUT)
-                    for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c, (int)sweep + 1 >= f16_from); ++pre; }
-                ++sweep;
+                if (kind == SW_CG || kind == SW_CG16) ++cg_seen;
+                // first blocks of the next sweep, in the format it will have.  After a statistics sweep the next one
+                // is another statistics sweep, the first CG sweep or the output sweep: all on the bf16 inputs unless
+                // precise == 0, where nothing is fetched ahead
+                const bool f16_next = f16_on && cg_seen >= precise;
+                if (kind != SW_OUT && !(kind == SW_STATS && f16_next))
+                    for (int c = 0; c < min(TC_NST, nblk) && ok; ++c) { issue_k(c, f16_next); ++pre; }
             }
             if (*abort_flag) {
                 if (PC) (void)mbar_wait_landed(bar(B_MFULL), 0, wcap);
@@ -405,14 +409,14 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint64_t phdesc = make_desc(sb_u + SM_PHI);
         const uint64_t pldesc = make_desc(sb_u + SM_PLO);
         uint32_t it = 0;   // global block counter (stage = it % NST, buffer = it % NBUF)
-        int sweep = 0;     // index among the sweeps over the keys
+        int cg_seen = 0;   // CG sweeps issued so far
         for (uint32_t ctl = 0; ok; ++ctl) {
             if (!mbar_wait(bar(B_CTL), ctl & 1, abort_flag, wcap)) break;
             const int kind = misc[4 + (ctl & 1)];
             if (kind == SW_DONE) break;
             tc_fence_after();
-            const uint32_t idesc = sweep >= f16_from ? IDESC_SS16 : IDESC_SS;
-            ++sweep;
+            const uint32_t idesc = (kind == SW_CG16 || (kind == SW_OUT && f16_on && cg_seen >= precise)) ? IDESC_SS16 : IDESC_SS;
+            if (kind == SW_CG || kind == SW_CG16) ++cg_seen;
             for (int c = 0; c < nblk && ok; ++c, ++it) {
                 const uint32_t s = it % TC_NST, b = it % TC_NBUF, bu = it / TC_NBUF;
                 if (!mbar_wait(bar(B_KVFULL + s), (it / TC_NST) & 1, abort_flag, wcap)) { ok = false; break; }
@@ -458,18 +462,13 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!mbar_wait(bar(B_UFULL + b), bu & 1, abort_flag, wcap)) { ok = false; break; }
                 if (kind == SW_OUT && !mbar_wait(bar(B_VFULL + s), (c / TC_NST) & 1, abort_flag, wcap)) { ok = false; break; }
                 tc_fence_after();
-                if (kind != SW_MAX) {
-                    const uint32_t bsm = sb_u + SM_KV + s * STAGE + (kind == SW_OUT ? KBLK : 0);
-                    // B = the K (or V) block read MN-major, N = D: 64-wide column groups are one sub-tile apart
-                    if (kind == SW_CG16) mma_ts_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS16, c > 0);
-                    else mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS, c > 0);
-                    tc_commit_el(el, bar(B_KVEMPTY + s));
-                    tc_commit_el(el, bar(B_BUFFREE + b));
-                    if (c == nblk - 1) tc_commit_el(el, bar(B_ACCFULL));
-                } else if (el) {
-                    mbar_arrive(bar(B_KVEMPTY + s));
-                    mbar_arrive(bar(B_BUFFREE + b));
-                }
+                const uint32_t bsm = sb_u + SM_KV + s * STAGE + (kind == SW_OUT ? KBLK : 0);
+                // B = the K (or V) block read MN-major, N = D: 64-wide column groups are one sub-tile apart
+                if (kind == SW_CG16) mma_ts_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS16, c > 0);
+                else mma_ts_hilo_k64(el, tm_u + TC_ACC_COL, tm_u + b * 128, make_desc(bsm, Cfg::KSUB_BYTES), IDESC_TS, c > 0);
+                tc_commit_el(el, bar(B_KVEMPTY + s));
+                tc_commit_el(el, bar(B_BUFFREE + b));
+                if (c == nblk - 1) tc_commit_el(el, bar(B_ACCFULL));
             }
         }
         if (*abort_flag) {      // an aborted block: the MMAs this warp issued must be done before TMEM and shared memory go
@@ -615,6 +614,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // [1, 2.83), so that its entries and u = w (a - abar) sit in the middle of the fp16 range whatever the
         // scale of the right-hand side; pn2 tracks |p|^2 through the recurrence |p'|^2 = |r'|^2 + beta^2 |p|^2
         float pn2 = 0.f, psc = 1.f, ipsc = 1.f;
+        float smax = -INFINITY;                               // statistics sweep: largest score of the row, relative to the shift
         uint32_t blk = 0;                                     // global block counter (buffer = blk & 1)
         bool ok = true;
 
@@ -626,8 +626,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // instead: there both groups work on every block, each thread on its half of the keys, which
         // halves the time from a block's scores to its contribution.
         auto sweep = [&](int kind) {
-            float part = 0.f;                                 // omega / den partial, or max
-            if (kind == SW_MAX) part = -INFINITY;
+            float part = 0.f;                                 // omega / den partial
             const uint64_t c1c1 = pk2(c1, c1), nmx = pk2(-mx2, -mx2);
             const float ab_s = kind == SW_CG16 ? abar * psc : abar;
             const uint64_t nab = pk2(-ab_s, -ab_s), oab = pk2(1.f + abar, 1.f + abar), neg1 = pk2(-1.f, -1.f);
@@ -654,11 +653,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         for (int e = 0; e < 32; ++e)
                             if (e >= jlim || e < jfirst) sv[e] = __float_as_uint(-1e30f);
                     }
-                    if (kind == SW_MAX) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            part = fmaxf(part, __uint_as_float(sv[e]) * c1);
-                    } else if (kind == SW_CG16) {
+                    if (kind == SW_CG16) {
                         // u = w (a - abar) as one fp16 value per key: 16 keys per k-step in 8 columns
                         uint32_t pk[16];
 #pragma unroll
@@ -680,6 +675,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             const uint64_t t2 = fma2(pk2(__uint_as_float(sv[2 * e2]), __uint_as_float(sv[2 * e2 + 1])), c1c1, nmx);
                             float t0, t1;
                             upk2(t2, t0, t1);
+                            if (kind == SW_STATS) smax = fmaxf(smax, fmaxf(t0, t1));     // largest score, relative to the shift
                             uint64_t u2 = pk2(ex2f(t0), ex2f(t1));
                             if (kind == SW_CG)
                                 u2 = mul2(u2, add2(pk2(__uint_as_float(av[2 * e2]), __uint_as_float(av[2 * e2 + 1])), nab));
@@ -695,17 +691,15 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         tmem_st32(s_addr, pk);
                     }
                 }
-                if (kind != SW_MAX) tc_wait_st();
+                tc_wait_st();
                 tc_fence_before();
                 // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised atomics
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_UFULL + b));
             }
-            if (kind != SW_MAX) {
-                float p0, p1;
-                upk2(part2, p0, p1);
-                part = p0 + p1;
-            }
+            float p0, p1;
+            upk2(part2, p0, p1);
+            part = p0 + p1;
             return part;
         };
         // read this thread's NCOL ACC columns after the sweep's last MMA
@@ -728,11 +722,9 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             tc_fence_before();
         };
-        int sweeps_started = 0;
         uint32_t ctl_phase = 0;
-        auto start_sweep = [&](int kind) {
-            if (sweeps_started >= f16_from && !q_is_f16) convert_q();
-            ++sweeps_started;
+        auto start_sweep = [&](int kind, bool f16 = false) {
+            if (f16 && !q_is_f16) convert_q();
             if (tid == 0) misc[4 + (ctl_phase & 1)] = kind;
             ++ctl_phase;
             fence_proxy_async();       // operand tiles written with ordinary stores -> visible to the MMA
@@ -757,7 +749,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // (the products of an iteration enter x and r scaled by |p|, which has fallen by then: the coarser
         // operands of the later iterations cost no accuracy that the early ones have not already spent)
         auto write_p = [&](int t_next) {
-            if (t_next + 2 >= f16_from) {
+            if (f16_on && t_next >= precise) {
                 const int e2 = (int)((__float_as_uint(pn2) >> 23) & 0xffu) - 127;      // floor(log2 |p|^2)
                 const int k = max(-100, min(100, -(e2 >> 1)));
                 psc = __uint_as_float((uint32_t)(127 + k) << 23);
@@ -816,26 +808,36 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float rz = 0.f;      // r . z of the preconditioned recurrence
         bool prec_row = true;   // false once the preconditioner has failed this row (z = r from then on)
 
-        // ---- sweep 0: row maxima ----
-        start_sweep(SW_MAX);
+        // ---- statistics sweep: omega and kbar ----
+        // No sweep of its own finds the row maxima: Eq. "lla" is unchanged under a joint scaling of the weights and
+        // the ridge, so any shift of the scores serves as long as the weights stay in range.  The sweep runs with
+        // shift zero and notes the largest score on the way; only if some row's maximum lies outside 2^+-8 (the
+        // fp16 operands of the later sweeps want the leading weights near one) is it run again with every row's
+        // own maximum as shift, which is then known.
+        float tmax = 0.f;          // the row's largest scaled score (log2 units)
         {
-            const float part = sweep(SW_MAX);
-            ok = all_ok(ok);
-            if (ok) mx2 = pair_max(part);
-        }
-        // ---- sweep 1: omega and kbar ----
-        if (ok) {
-            start_sweep(SW_STATS);
-            const float part = sweep(SW_STATS);
-            if (ok) acc_wait();
-            ok = all_ok(ok);
+            float part = 0.f;
+            mx2 = 0.f;
+            for (int attempt = 0; attempt < 2 && ok; ++attempt) {
+                smax = -INFINITY;
+                start_sweep(SW_STATS);
+                part = sweep(SW_STATS);
+                if (ok) acc_wait();
+                ok = all_ok(ok);
+                if (!ok) break;
+                tmax = pair_max(smax) + mx2;
+                if (attempt == 1 || !group_any(row_ok && !(fabsf(tmax) <= 8.f))) break;
+                mx2 = fabsf(tmax) < 1e30f ? tmax : 0.f;     // (a row without a finite score keeps shift zero)
+            }
             if (ok) {
                 float acc[NCOL];
                 acc_load(acc);
                 omega = pair_sum(part);
                 inv_omega = 1.f / omega;
                 const float lam_i = (prm.lambda_rows && row < nq) ? prm.lambda_rows[(size_t)bh * nq + row] : prm.lambda;
-                ridge = (prm.ridge_mode == LLA_RIDGE_PRINTED ? lam_i : lam_i * ex2f(-mx2)) * inv_omega;
+                // ridge in the frame of the shift: lambda e^{-shift} by the definition; the printed algorithm adds
+                // lambda in the frame of the row maximum, i.e. lambda e^{max - shift} here
+                ridge = lam_i * ex2f((prm.ridge_mode == LLA_RIDGE_PRINTED ? tmax : 0.f) - mx2) * inv_omega;
                 float rr_p = 0.f, ab_p = 0.f;
 #pragma unroll
                 for (int ch = 0; ch < NCOL / 8; ++ch) {
@@ -889,11 +891,12 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         if (ok) write_p(0);
         // ---- conjugate gradients (Algorithm 2) ----
-        for (int t = 0; ok && t < prm.max_iters; ++t) {
+        int t = 0;      // CG sweeps run
+        for (; ok && t < prm.max_iters; ++t) {
             active = active && rr > stop;
             if (!group_any(active)) break;
-            const bool cheap = t + 2 >= f16_from;
-            start_sweep(cheap ? SW_CG16 : SW_CG);
+            const bool cheap = f16_on && t >= precise;
+            start_sweep(cheap ? SW_CG16 : SW_CG, cheap);
             sweep(cheap ? SW_CG16 : SW_CG);
             if (ok) acc_wait();
             ok = all_ok(ok);
@@ -1031,9 +1034,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             abar = pair_sum(yb_p);
             gfac = 1.f + pair_sum(g_p);
-            if (sweeps_started >= f16_from) write_operand16_pair(y);
+            const bool out16 = f16_on && t >= precise;      // the format every role derives from the CG sweeps it has seen
+            if (out16) write_operand16_pair(y);
             else write_operand(y);
-            start_sweep(SW_OUT);
+            start_sweep(SW_OUT, out16);
             const float part = sweep(SW_OUT);
             if (ok) acc_wait();
             ok = all_ok(ok);
@@ -1054,7 +1058,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                     if (half == 0) {
                         if (prm.stats) {
-                            prm.stats[rowi * 3 + 0] = mx2 * 0.6931471805599453f;
+                            prm.stats[rowi * 3 + 0] = mx2 * 0.6931471805599453f;      // the shift the weights were formed with
                             prm.stats[rowi * 3 + 1] = omega;
                             prm.stats[rowi * 3 + 2] = omega / gfac;
                         }
@@ -1156,7 +1160,7 @@ void tile_order(TcParams& prm, int tiles, int first_tile, int n, int off, int d,
         const float its = precond ? std::min(16.f, 4.f + 190.f * x * x) : 6.f + 50.f * x;
         const int c_first = window > 0 ? std::max(0, off + (first_tile + t) * TC_BR + 1 - window) / TC_BC : 0;
         const float nblk = (float)((r_end + TC_BC - 1) / TC_BC - c_first);
-        cost[t] = (its + 3.f) * (6.f + nblk) + (precond ? 3.f * its : 0.f);
+        cost[t] = (its + 2.f) * (6.f + nblk) + (precond ? 3.f * its : 0.f);
         prm.order[t] = (unsigned short)t;
     }
     std::stable_sort(prm.order, prm.order + tiles, [&](unsigned short x, unsigned short y) { return cost[x] > cost[y]; });
