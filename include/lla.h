@@ -185,6 +185,13 @@ typedef struct lla_forward_params {
                        tiles within the first 8 d positions, which converge more slowly); n > 0 = n
                        iterations for every tile; LLA_CG_PRECISE_ALL = every iteration with pairs;
                        LLA_CG_PRECISE_NONE = fp16 from the first iteration on */
+    long long q_strides[3], k_strides[3], v_strides[3], out_strides[3];
+                          /* element strides (batch, head, row) of q [B, H, rows, d], k and v [B, kv heads, n, d] and
+                       out; the innermost index always has stride 1.  All zero = contiguous in that order.  Any other
+                       layout whose strides are positive multiples of 8 elements is read in place, e.g. tensors kept
+                       as [B, n, H, d]: strides (n H d, d, H d).  The caller guarantees that the strides address
+                       memory it owns and that rows of `out` do not overlap.  The optional per-row outputs (rho,
+                       stats, iters) and lambda_rows stay contiguous [B, H, rows, ...].  Forward only */
     int cg_precondition;  /* tensor-core kernel only.  0 = plain conjugate gradients as in Algorithm 2 (default).
                        1 = preconditioned with the inverse covariance of the visible keys: one d x d matrix per
                        block of 128 keys, built by a pre-pass into `workspace` (plain CG without room for it

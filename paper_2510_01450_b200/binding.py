@@ -62,7 +62,10 @@ class ForwardParams(ctypes.Structure):
         ("device_status", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p), ("lambda_rows", ctypes.c_void_p), ("ridge_mode", ctypes.c_int),
         ("q_rows", ctypes.c_int), ("kv_heads", ctypes.c_int), ("window", ctypes.c_int),
-        ("cg_precise_iters", ctypes.c_int), ("cg_precondition", ctypes.c_int), ("debug_wait_clocks", ctypes.c_longlong),
+        ("cg_precise_iters", ctypes.c_int),
+        ("q_strides", ctypes.c_longlong * 3), ("k_strides", ctypes.c_longlong * 3), ("v_strides", ctypes.c_longlong * 3),
+        ("out_strides", ctypes.c_longlong * 3),
+        ("cg_precondition", ctypes.c_int), ("debug_wait_clocks", ctypes.c_longlong),
         ("debug_flags", ctypes.c_int),
     ]
 
@@ -180,8 +183,12 @@ def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=
                    max_iters=0, tol=0.0, head_rows=0, impl=LLA_IMPL_AUTO, phases=0, rho=None, stats=None, iters=None,
                    device_status=None, workspace=None, workspace_bytes=0, stream=0, lambda_rows=None,
                    ridge_mode=LLA_RIDGE_DEFINITION, q_rows=0, kv_heads=0, window=0, cg_precise_iters=0,
-                   debug_wait_clocks=0, debug_flags=0, cg_precondition=0):
+                   debug_wait_clocks=0, debug_flags=0, cg_precondition=0, q_strides=None, k_strides=None, v_strides=None,
+                   out_strides=None):
     p = ForwardParams()
+    for name, val in (("q_strides", q_strides), ("k_strides", k_strides), ("v_strides", v_strides), ("out_strides", out_strides)):
+        if val is not None:
+            setattr(p, name, (ctypes.c_longlong * 3)(*[int(x) for x in val]))
     p.cg_precondition = cg_precondition
     p.debug_wait_clocks, p.debug_flags = debug_wait_clocks, debug_flags
     p.kv_heads, p.window, p.cg_precise_iters = kv_heads, window, cg_precise_iters

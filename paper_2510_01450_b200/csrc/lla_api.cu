@@ -79,6 +79,12 @@ int check_forward(const lla_forward_params* p) {
     if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
     if (p->max_iters < 0 || p->tol < 0.f || !isfinite(p->tol)) return LLA_ERR_INVALID_ARG;
     if (p->cg_precondition < 0 || p->cg_precondition > 1) return LLA_ERR_INVALID_ARG;
+    for (const long long* st : {p->q_strides, p->k_strides, p->v_strides, p->out_strides}) {
+        const bool set = st[0] || st[1] || st[2];
+        // given strides: positive, and multiples of 8 elements so that every row starts on a 16-byte boundary
+        // (vector loads, TMA); the innermost index always has stride 1
+        if (set && (st[0] <= 0 || st[1] <= 0 || st[2] <= 0 || (st[0] | st[1] | st[2]) % 8 != 0)) return LLA_ERR_INVALID_ARG;
+    }
     if (p->debug_wait_clocks < 0 || (p->debug_flags & ~LLA_DEBUG_NO_LOADS)) return LLA_ERR_INVALID_ARG;
     if ((long long)p->B * p->H > 65535 || (p->n + 127) / 128 > 65535) return LLA_ERR_UNSUPPORTED;
     if (!head_size_ok(p->d, p->dv)) return LLA_ERR_UNSUPPORTED;
@@ -112,6 +118,12 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     a.window = p->window;
     a.wait_clocks = p->debug_wait_clocks;
+    // layouts: all-zero strides mean contiguous [B, heads, rows, width]
+    a.set_contiguous();
+    auto take = [](lla::Strides& dst, const long long* src) {
+        if (src[0] || src[1] || src[2]) dst = lla::Strides{src[0], src[1], src[2]};
+    };
+    take(a.sq, p->q_strides); take(a.sk, p->k_strides); take(a.sv, p->v_strides); take(a.so, p->out_strides);
     a.precondition = p->cg_precondition > 0 ? 1 : 0;
     a.no_loads = (p->debug_flags & LLA_DEBUG_NO_LOADS) ? 1 : 0;
     if (p->cg_precise_iters != 0) {

@@ -1001,6 +1001,7 @@ int launch_t(const BackwardArgs& a) {
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
         f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg;
         f.rhs = hvec; f.sol = tvec;
+        f.set_contiguous();
         // what the workspace holds beyond this pass's own vectors serves the solve (the fp16 copy of k; for
         // d = 128 the row-state slots), so that the backward pass allocates nothing
         const size_t own = (ws_floats(rows, D, BH) * sizeof(float) + 255) & ~(size_t)255;

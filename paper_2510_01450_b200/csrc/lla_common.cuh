@@ -43,6 +43,17 @@ __host__ __device__ __forceinline__ int first_visible_key(int len, int Lmax, int
     return L - visible_keys(len, Lmax, window);
 }
 
+// Element strides (batch, head, row) of a [B, heads, rows, width] tensor whose innermost index has stride 1.
+struct Strides {
+    long long b, h, r;
+    __host__ __device__ __forceinline__ size_t at(int batch, int head, long long row) const {
+        return (size_t)((long long)batch * b + (long long)head * h + row * r);
+    }
+};
+__host__ __device__ __forceinline__ Strides contiguous_strides(int heads, long long rows, int width) {
+    return Strides{(long long)heads * rows * width, rows * width, (long long)width};
+}
+
 struct ForwardArgs {
     const void* q;
     const void* k;
@@ -69,6 +80,14 @@ struct ForwardArgs {
     int window = 0;             // causal sliding window: a row sees its last `window` positions (0: all)
     const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
+    // layouts of q [B, H, nq, d], k [B, H / kv_group, n, d], v [.., dv] and out [B, H, nq, dv]; zero = not set: the
+    // launchers that build a ForwardArgs themselves call set_contiguous()
+    Strides sq = {0, 0, 0}, sk = {0, 0, 0}, sv = {0, 0, 0}, so = {0, 0, 0};
+    void set_contiguous() {
+        const int hk = H / (kv_group > 0 ? kv_group : 1);
+        sq = contiguous_strides(H, nq, d); sk = contiguous_strides(hk, n, d);
+        sv = contiguous_strides(hk, n, dv); so = contiguous_strides(H, nq, dv);
+    }
     long long wait_clocks = 0;  // tensor-core kernel: cap of its bounded waits in SM clocks (0: default) and a test
     int no_loads = 0;           // aid: issue no copy at all (lla_forward_params.debug_*)
     const void* minv = nullptr; // CG preconditioner matrices (fp16), set by forward_tensor_prepass when enabled
@@ -149,7 +168,8 @@ size_t forward_tensor_workspace_bytes(int B, int H, int n, int d);   // that scr
 int precond_blocks(int n);
 size_t precond_gram_bytes(int units, int n, int d);     // fp32 running Gram sums (scratch of the pre-pass)
 size_t precond_minv_bytes(int units, int n, int d);     // the fp16 matrices [units][blocks][d][d]
-int launch_precond(const void* k, int units, int n, int d, float lambda, int window, void* gram, void* minv, cudaStream_t st);
+int launch_precond(const void* k, int B, int Hk, Strides sk, int n, int d, float lambda, int window, void* gram, void* minv,
+                   cudaStream_t st);
 int launch_decode(const DecodeArgs& a);
 int launch_head_rows_decode(const DecodeArgs& a);
 bool decode_tensor_supported(const DecodeArgs& a);

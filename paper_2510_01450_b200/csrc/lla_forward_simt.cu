@@ -44,13 +44,13 @@ __device__ __forceinline__ float exp_w(float x) {
 
 template <int D, typename TIn>
 __device__ __forceinline__ void load_tile(float* __restrict__ dst, const TIn* __restrict__ src,
-                                          int j0, int n) {
-    // dst[FS_BC][D] <- src rows j0 .. j0+FS_BC-1 (zero beyond n)
+                                          int j0, int n, long long row_stride) {
+    // dst[FS_BC][D] <- src rows j0 .. j0+FS_BC-1 (zero beyond n); rows are row_stride elements apart
     constexpr int VEC = FS_BC * D / 4;
     for (int e = threadIdx.x; e < VEC; e += FS_THREADS) {
         const int jj = e / (D / 4), f = e - jj * (D / 4);
         float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j0 + jj < n) val = load4(src + (size_t)(j0 + jj) * D + 4 * f);
+        if (j0 + jj < n) val = load4(src + (size_t)(j0 + jj) * row_stride + 4 * f);
         reinterpret_cast<float4*>(dst)[e] = val;
     }
 }
@@ -61,7 +61,8 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
                     TOut* __restrict__ out, int n, int causal, float scale, float lambda,
                     int head_rows, int max_iters, float tol, int first_tile,
                     float* __restrict__ rho_out, float* __restrict__ stats, int* __restrict__ iters_out,
-                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq, int H, int kv_group, int window) {
+                    int* __restrict__ status, const float* __restrict__ lambda_rows, int ridge_mode, int nq, int H, int kv_group, int window,
+                    const Strides sq, const Strides sk, const Strides sv, const Strides so) {
     constexpr int ROWS = FS_THREADS / TPR;
     constexpr int NG = D / (4 * TPR);    // float4 groups per thread (keys)
     constexpr int NGV = DV / (4 * TPR);  // float4 groups per thread (values)
@@ -83,14 +84,14 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     // sliding window (causal only): a row sees keys jlo .. L - 1, the block starts at its first row's window
     const int jlo = (causal && window > 0) ? max(0, L - window) : 0;
     const int jbeg = (causal && window > 0) ? max(0, off + r0 + 1 - window) / FS_BC * FS_BC : 0;
-    const int kvh = kv_unit(bh, H, kv_group);
-    const TIn* kb = k + (size_t)kvh * n * D;
-    const TIn* vb = v + (size_t)kvh * n * DV;
+    const int hk = (bh % H) / max(kv_group, 1);             // key/value head of this query head
+    const TIn* kb = k + sk.at(bh / H, hk, 0);
+    const TIn* vb = v + sv.at(bh / H, hk, 0);
 
     float4 qv[NG], kbar[NG];
 #pragma unroll
     for (int g = 0; g < NG; ++g) {
-        qv[g] = row < nq ? load4(q + ((size_t)bh * nq + row) * D + 4 * (g * TPR + lr))
+        qv[g] = row < nq ? load4(q + sq.at(bh / H, bh % H, row) + 4 * (g * TPR + lr))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
         kbar[g] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
@@ -99,7 +100,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     float m = -INFINITY, omega = 0.f;
     for (int j0 = jbeg; j0 < jend; j0 += FS_BC) {
         __syncthreads();
-        load_tile<D>(Ks, kb, j0, n);
+        load_tile<D>(Ks, kb, j0, n, sk.r);
         __syncthreads();
         const int lim = row_ok ? min(FS_BC, L - j0) : 0;
         const int wlim = __reduce_max_sync(0xffffffffu, lim);
@@ -166,7 +167,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
         for (int g = 0; g < NG; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int j0 = jbeg; j0 < jend; j0 += FS_BC) {
             __syncthreads();
-            load_tile<D>(Ks, kb, j0, n);
+            load_tile<D>(Ks, kb, j0, n, sk.r);
             __syncthreads();
             const int lim = active ? min(FS_BC, L - j0) : 0;
             const int wlim = __reduce_max_sync(0xffffffffu, lim);
@@ -239,8 +240,8 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     float den = 0.f;
     for (int j0 = jbeg; j0 < jend; j0 += FS_BC) {
         __syncthreads();
-        load_tile<D>(Ks, kb, j0, n);
-        load_tile<DV>(Vs, vb, j0, n);
+        load_tile<D>(Ks, kb, j0, n, sk.r);
+        load_tile<DV>(Vs, vb, j0, n, sv.r);
         __syncthreads();
         const int lim = row_ok ? min(FS_BC, L - j0) : 0;
         const int wlim = __reduce_max_sync(0xffffffffu, lim);
@@ -268,7 +269,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     if (row_ok) {
         const float inv_den = 1.f / den;
         const size_t rowi = (size_t)bh * nq + row;
-        TOut* orow = out + rowi * DV;
+        TOut* orow = out + so.at(bh / H, bh % H, row);
 #pragma unroll
         for (int g = 0; g < NGV; ++g) {
             const int c0 = 4 * (g * TPR + lr);
@@ -315,7 +316,7 @@ int launch_t(const ForwardArgs& a) {
     kern<<<grid, FS_THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, a.causal, a.scale,
         a.lambda, a.head_rows > 0 ? a.head_rows : 0, a.max_iters, a.tol, first_tile, a.rho, a.stats,
-        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq, a.H, a.kv_group, a.window);
+        a.iters, a.status, a.lambda_rows, a.ridge_mode, a.nq, a.H, a.kv_group, a.window, a.sq, a.sk, a.sv, a.so);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -202,6 +202,7 @@ struct TcParams {
     float* rho;
     float* stats;
     int H, kv_group;     // query heads per (batch), query heads per key/value head
+    Strides so;          // layout of out [B, H, nq, D]
     int window;          // causal sliding window (0: none): a row sees its last `window` positions
     const float* rhs;    // solve mode: right-hand sides h_i [B, H, nq, D]; the CG then solves C_i x = h_i ...
     float* sol;          // ... and x_i is written here instead of running the output sweep
@@ -297,7 +298,6 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         misc[4] = SW_STATS;
         misc[5] = SW_STATS;
         misc[2] = 0;
-        misc[3] = kv_unit(bh, prm.H, prm.kv_group);   // worked out here: in the producer's own path it delays the first loads
         fence_barrier_init();
     }
     if (warp == 8) {   // TMEM allocation by one full warp; the base address lands in shared memory
@@ -318,9 +318,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // is announced.
         if (lane == 0 && !prm.no_loads) {
             mbar_expect_tx(bar(B_QFULL), Cfg::OPER_BYTES);
+            // tensor-map coordinates: (column, row, head, batch); keys and values by their own head
+            const int bb = bh / prm.H, hq = bh % prm.H, hk = hq / prm.kv_group;
             for (int sub = 0; sub < KSUB; ++sub)
-                tma_load_3d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, bh);
-            const int kvh = misc[3];
+                tma_load_4d(sbase + SM_Q + sub * Cfg::QSUB_BYTES, &tmQ, bar(B_QFULL), 64 * sub, r0, hq, bb);
             if (PC) {
                 // the preconditioner of this tile's key range: D x D fp16, laid out like D / 64 key blocks, into the
                 // V halves of the first ring stages (idle until the output sweep, when it is no longer needed)
@@ -328,8 +329,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 mbar_expect_tx(bar(B_MFULL), D * D * 2);
                 for (int rb = 0; rb < D / 64; ++rb)
                     for (int sub = 0; sub < KSUB; ++sub)
-                        tma_load_3d(sbase + SM_KV + rb * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmM, bar(B_MFULL), 64 * sub,
-                                    gm * D + 64 * rb, kvh);
+                        tma_load_4d(sbase + SM_KV + rb * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmM, bar(B_MFULL), 64 * sub,
+                                    gm * D + 64 * rb, hk, bb);
             }
             uint32_t kit = 0;      // K blocks issued so far
             int pre = 0;           // blocks of the coming sweep already issued
@@ -339,8 +340,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!mbar_wait(bar(B_KVEMPTY + s), ((kit / TC_NST) & 1) ^ 1, abort_flag, wcap)) { ok = false; return; }
                 mbar_expect_tx(bar(B_KVFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, f16 ? &tmK16 : &tmK, bar(B_KVFULL + s), 64 * sub,
-                                (cbeg + c) * TC_BC, kvh);
+                    tma_load_4d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, f16 ? &tmK16 : &tmK, bar(B_KVFULL + s), 64 * sub,
+                                (cbeg + c) * TC_BC, hk, bb);
                 ++kit;
             };
             uint32_t v_g0 = 0;
@@ -351,7 +352,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const uint32_t s = g % TC_NST;
                 mbar_expect_tx(bar(B_VFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_3d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, kvh);
+                    tma_load_4d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, hk, bb);
             };
             int cg_seen = 0;       // CG sweeps issued so far
             for (uint32_t ctl = 0; ok; ++ctl) {
@@ -1048,7 +1049,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (row_ok) {
                     const float inv_den = 1.f / den;
                     const size_t rowi = (size_t)bh * nq + row;
-                    TOut* orow = out + rowi * D + c0;
+                    TOut* orow = out + prm.so.at(bh / prm.H, bh % prm.H, row) + c0;
 #pragma unroll
                     for (int e = 0; e < NCOL; ++e) store_out(orow + e, o[e] * inv_den);
                     if (prm.rho) {
@@ -1089,12 +1090,17 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 // the range in which that copy is faithful (magnitude above 60000; bf16 values below the fp16 subnormal
 // spacing simply round, an absolute change under 3e-8).  Eight elements per thread and step.
 __global__ void __launch_bounds__(256)
-f16_copy_kernel(const uint4* __restrict__ k, uint4* __restrict__ k16, size_t k_vec, const uint4* __restrict__ q,
-                size_t q_vec, int* __restrict__ ok) {
+f16_copy_kernel(const __nv_bfloat16* __restrict__ k, uint4* __restrict__ k16, int Hk, int n, int d, Strides sk,
+                const __nv_bfloat16* __restrict__ q, int H, int nq, Strides sq, int B, int* __restrict__ ok) {
     bool bad = false;
     const size_t stride = (size_t)gridDim.x * blockDim.x, t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int vpr = d / 8;                                   // 16-byte groups per row
+    const size_t k_vec = (size_t)B * Hk * n * vpr, q_vec = (size_t)B * H * nq * vpr;
     for (size_t i = t0; i < k_vec; i += stride) {
-        const uint4 raw = k[i];
+        const int c = (int)(i % vpr);
+        const size_t rowi = i / vpr;
+        const int row = (int)(rowi % n), unit = (int)(rowi / n);
+        const uint4 raw = *reinterpret_cast<const uint4*>(k + sk.at(unit / Hk, unit % Hk, row) + 8 * c);
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
         uint32_t h[4];
 #pragma unroll
@@ -1103,10 +1109,13 @@ f16_copy_kernel(const uint4* __restrict__ k, uint4* __restrict__ k16, size_t k_v
             bad |= !(fabsf(a) <= 60000.f) || !(fabsf(b) <= 60000.f);
             h[e] = pack_f16(a, b);
         }
-        k16[i] = make_uint4(h[0], h[1], h[2], h[3]);
+        k16[i] = make_uint4(h[0], h[1], h[2], h[3]);         // the copy is contiguous [B][Hk][n][d]
     }
     for (size_t i = t0; i < q_vec; i += stride) {
-        const uint4 raw = q[i];
+        const int c = (int)(i % vpr);
+        const size_t rowi = i / vpr;
+        const int row = (int)(rowi % nq), unit = (int)(rowi / nq);
+        const uint4 raw = *reinterpret_cast<const uint4*>(q + sq.at(unit / H, unit % H, row) + 8 * c);
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e)
@@ -1177,8 +1186,11 @@ int launch_t(const ForwardArgs& a) {
     if (tiles <= 0) return LLA_OK;
     CUtensorMap mq, mk, mv, mk16, mm;
     const int BH = a.B * a.H;
-    if (!make_map_bf16(&mq, a.q, BH, a.nq, D, TC_BR) || !make_map_bf16(&mk, a.k, BH / a.kv_group, a.n, D, TC_BC) ||
-        !make_map_bf16(&mv, a.v, BH / a.kv_group, a.n, D, TC_BC))
+    const int Hk = a.H / a.kv_group;
+    const auto BF = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, F16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    if (!make_map_16bit_4d(&mq, a.q, a.B, a.H, a.nq, D, a.sq.b, a.sq.h, a.sq.r, TC_BR, BF) ||
+        !make_map_16bit_4d(&mk, a.k, a.B, Hk, a.n, D, a.sk.b, a.sk.h, a.sk.r, TC_BC, BF) ||
+        !make_map_16bit_4d(&mv, a.v, a.B, Hk, a.n, D, a.sv.b, a.sv.h, a.sv.r, TC_BC, BF))
         return LLA_ERR_CUDA;
     mk16 = mk;
     mm = mk;
@@ -1193,6 +1205,7 @@ int launch_t(const ForwardArgs& a) {
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
     prm.rhs = a.rhs; prm.sol = a.sol;
     prm.H = a.H; prm.kv_group = a.kv_group > 0 ? a.kv_group : 1;
+    prm.so = a.so;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
     prm.scratch = nullptr;
     prm.scratch_slots = 0;
@@ -1222,14 +1235,15 @@ int launch_t(const ForwardArgs& a) {
     // fp16 sweeps: only with the copy of k that forward_tensor_prepass made; without it every sweep runs on
     // the bf16 inputs
     if (a.k16 && a.f16_ok) {
-        if (!make_map_bf16(&mk16, a.k16, BH / a.kv_group, a.n, D, TC_BC, CU_TENSOR_MAP_DATA_TYPE_FLOAT16)) return LLA_ERR_CUDA;
+        const Strides c16 = contiguous_strides(Hk, a.n, D);
+        if (!make_map_16bit_4d(&mk16, a.k16, a.B, Hk, a.n, D, c16.b, c16.h, c16.r, TC_BC, F16)) return LLA_ERR_CUDA;
         prm.f16_ok = a.f16_ok;
     }
     bool precond = false;
     // preconditioned CG: only with the matrices that forward_tensor_prepass made ([units][blocks][D][D] fp16)
     if (a.minv) {
-        if (!make_map_bf16(&mm, a.minv, BH / a.kv_group, precond_blocks(a.n) * D, D, 64, CU_TENSOR_MAP_DATA_TYPE_FLOAT16))
-            return LLA_ERR_CUDA;
+        const Strides cm = contiguous_strides(Hk, (long long)precond_blocks(a.n) * D, D);
+        if (!make_map_16bit_4d(&mm, a.minv, a.B, Hk, (long long)precond_blocks(a.n) * D, D, cm.b, cm.h, cm.r, 64, F16)) return LLA_ERR_CUDA;
         precond = true;
     }
     auto kern = precond ? forward_tc_kernel<D, TOut, true> : forward_tc_kernel<D, TOut, false>;
@@ -1269,10 +1283,10 @@ int forward_tensor_prepass(ForwardArgs& a) {
     uint4* k16 = reinterpret_cast<uint4*>(ws);
     int* okw = reinterpret_cast<int*>(ws + round256(k_elems * 2));
     LLA_CUDA_TRY(cudaMemsetAsync(okw, 1, sizeof(int), a.stream));
-    const size_t k_vec = k_elems / 8, q_vec = (size_t)a.B * a.H * a.nq * a.d / 8;
+    const size_t k_vec = k_elems / 8;
     const unsigned blocks = (unsigned)std::min<size_t>((k_vec + 255) / 256, 148 * 8);
-    f16_copy_kernel<<<blocks, 256, 0, a.stream>>>(static_cast<const uint4*>(a.k), k16, k_vec, static_cast<const uint4*>(a.q), q_vec,
-                                                   okw);
+    f16_copy_kernel<<<blocks, 256, 0, a.stream>>>(static_cast<const __nv_bfloat16*>(a.k), k16, a.H / a.kv_group, a.n, a.d, a.sk,
+                                                   static_cast<const __nv_bfloat16*>(a.q), a.H, a.nq, a.sq, a.B, okw);
     LLA_CUDA_TRY(cudaGetLastError());
     a.k16 = k16;
     a.f16_ok = okw;
@@ -1283,7 +1297,7 @@ int forward_tensor_prepass(ForwardArgs& a) {
     if (a.precondition && a.workspace_bytes >= used + gram_b + minv_b) {
         char* gram = static_cast<char*>(a.workspace) + used;
         char* minv = gram + gram_b;
-        const int rc = launch_precond(a.k, units, a.n, a.d, a.lambda, a.causal ? a.window : 0, gram, minv, a.stream);
+        const int rc = launch_precond(a.k, a.B, a.H / a.kv_group, a.sk, a.n, a.d, a.lambda, a.causal ? a.window : 0, gram, minv, a.stream);
         if (rc != LLA_OK) return rc;
         a.minv = minv;
     }

@@ -99,7 +99,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
                  double lambda, int lcap, float* __restrict__ rho_out, float* __restrict__ stats,
                  int* __restrict__ iters, int* __restrict__ status, const int* __restrict__ lens, int H,
                  const float* __restrict__ lambda_rows, int ridge_mode, int nq, int kv_group,
-                 const PagedKv paged, int window) {
+                 const PagedKv paged, int window, const Strides sq, const Strides sk, const Strides sv, const Strides so) {
     // Prefill (lens == nullptr): block (i, bh) solves row i of head bh; n is the sequence length.
     // Decode (lens != nullptr): block (0, bh) solves the single query of (sequence, head) bh over
     // lens[bh / H] cached keys, but only when that is at most lcap; n is the cache stride Lmax.
@@ -124,13 +124,17 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         L = visible_keys(lens[bh / H], n, window);
         if (L > lcap) return;               // long caches go through the moment kernel
     }
-    const size_t row = lens ? (size_t)bh : (size_t)bh * nq + i;
-    const TIn* qrow = q + row * D;
+    const size_t row = lens ? (size_t)bh : (size_t)bh * nq + i;      // row of the contiguous per-row outputs (rho, stats, ...)
+    // prefill: q, k, v and out are addressed through their strides; decode keeps its contiguous / paged layout
+    const TIn* qrow = lens ? q + row * D : q + sq.at(bh / H, bh % H, i);
     // (decode over a paged cache: the at most lcap <= page_size keys of a directly-solved unit sit in its first page)
     const int kstart = lens ? first_visible_key(lens[bh / H], n, window) : 0;      // sliding-window decode
     const size_t kvrow = kv_row(paged, bh / H, (bh % H) / max(kv_group, 1), H / max(kv_group, 1), n, kstart);
-    const TIn* kb = k + kvrow * D;
-    const TIn* vb = v + kvrow * DV;
+    const int hk = (bh % H) / max(kv_group, 1);
+    const TIn* kb = lens ? k + kvrow * D : k + sk.at(bh / H, hk, 0);
+    const TIn* vb = lens ? v + kvrow * DV : v + sv.at(bh / H, hk, 0);
+    const size_t krs = lens ? (size_t)D : (size_t)sk.r, vrs = lens ? (size_t)DV : (size_t)sv.r;      // row strides of k and v
+    TOut* orow = lens ? out + row * DV : out + so.at(bh / H, bh % H, i);
 
     for (int c = tid; c < D; c += HR_THREADS) qd[c] = (double)to_f32(qrow[c]);
     __syncthreads();
@@ -138,7 +142,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     // scores, their maximum, weights exp(s - m), ridge lambda * exp(-m)
     double lmax = -INFINITY;
     for (int j = tid; j < L; j += HR_THREADS) {
-        const double s = dot_row<D>(qd, kb + (size_t)j * D) * scale;
+        const double s = dot_row<D>(qd, kb + (size_t)j * krs) * scale;
         w[j] = s;
         lmax = fmax(lmax, s);
     }
@@ -189,7 +193,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         double* zt = S;                                   // zt[c * LZ + j] = k_j[c] - q[c]  (over S: D * LZ <= S_DOUBLES)
         for (int e = tid; e < Lp * D; e += HR_THREADS) {
             const int j = e / D, c = e - j * D;
-            zt[c * LZ + j] = j < L ? (double)to_f32(kb[(size_t)j * D + c]) - qd[c] : 0.0;
+            zt[c * LZ + j] = j < L ? (double)to_f32(kb[(size_t)j * krs + c]) - qd[c] : 0.0;
         }
         __syncthreads();
         // Gram matrix
@@ -235,7 +239,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         }
         if (rho_out && tid < D) {                         // rho = Z^T alpha
             double acc_r = 0.0;
-            for (int j = 0; j < L; ++j) acc_r += rhs[j] * ((double)to_f32(kb[(size_t)j * D + tid]) - qd[tid]);
+            for (int j = 0; j < L; ++j) acc_r += rhs[j] * ((double)to_f32(kb[(size_t)j * krs + tid]) - qd[tid]);
             rho_val = acc_r;
         }
     } else {
@@ -250,7 +254,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     #pragma unroll
             for (int u = 0; u < PAIRS; ++u) {
                 const int pi = tid + HR_THREADS * u;
-                if (pi < np) load2(kb + (size_t)j0 * D + 2 * pi, pre[u][0], pre[u][1]);
+                if (pi < np) load2(kb + (size_t)(j0 + (2 * pi) / D) * krs + (2 * pi) % D, pre[u][0], pre[u][1]);
             }
         };
         fetch(0);
@@ -313,7 +317,7 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         double qrho = 0.0;
         for (int c = 0; c < D; ++c) qrho += qd[c] * rhs[c];
         for (int j = tid; j < L; j += HR_THREADS) {
-            const double t = dot_row<D>(rhs, kb + (size_t)j * D) - qrho;
+            const double t = dot_row<D>(rhs, kb + (size_t)j * krs) - qrho;
             const double cj = w[j] * (1.0 - t);
             w[j] = cj;
             csum += cj;
@@ -323,8 +327,8 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
     const double denom = block_reduce<HR_THREADS>(csum, false, red);
     for (int c = tid; c < DV; c += HR_THREADS) {
         double o = 0.0;
-        for (int j = 0; j < L; ++j) o += w[j] * (double)to_f32(vb[(size_t)j * DV + c]);
-        store_out(out + row * DV + c, (float)(o / denom));
+        for (int j = 0; j < L; ++j) o += w[j] * (double)to_f32(vb[(size_t)j * vrs + c]);
+        store_out(orow + c, (float)(o / denom));
     }
     if (rho_out && tid < D) rho_out[row * D + tid] = (float)rho_val;
     if (tid == 0) {
@@ -349,7 +353,7 @@ int launch_t(const ForwardArgs& a, int rows_per_head, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.k, (const TIn*)a.v, (TOut*)a.out, a.n, rows_per_head, a.causal,
         (double)a.scale, (double)a.lambda, lcap, a.rho, a.stats, a.iters, a.status, nullptr, a.H, a.lambda_rows,
-        a.ridge_mode, a.nq, a.kv_group, PagedKv{nullptr, 0, 0, 0}, 0);
+        a.ridge_mode, a.nq, a.kv_group, PagedKv{nullptr, 0, 0, 0}, 0, a.sq, a.sk, a.sv, a.so);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
@@ -365,7 +369,7 @@ int launch_decode_t(const DecodeArgs& a, int lcap) {
     kern<<<grid, C::THREADS, smem, a.stream>>>(
         (const TIn*)a.q, (const TIn*)a.kcache, (const TIn*)a.vcache, (TOut*)a.out, a.Lmax, 1, 0,
         (double)a.scale, (double)a.lambda, lcap, nullptr, nullptr, nullptr, a.status, a.lens, a.H, a.lambda_units,
-        a.ridge_mode, 1, a.kv_group, a.paged, a.window);
+        a.ridge_mode, 1, a.kv_group, a.paged, a.window, Strides{0, 0, 0}, Strides{0, 0, 0}, Strides{0, 0, 0}, Strides{0, 0, 0});
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }

@@ -27,17 +27,17 @@ constexpr int PC_BLOCK = 128;      // keys per Gram block
 
 template <int D>
 __global__ void __launch_bounds__(PC_THREADS)
-gram_blocks_kernel(const __nv_bfloat16* __restrict__ k, float* __restrict__ gram, int n, int nb) {
+gram_blocks_kernel(const __nv_bfloat16* __restrict__ k, float* __restrict__ gram, int n, int nb, int Hk, Strides sk) {
     constexpr int LD = D + 1, TR = D / 16;
     extern __shared__ float pc_smem[];
     float* ks = pc_smem;                                   // [PC_BLOCK][LD]
     const int b = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
     const int j0 = b * PC_BLOCK, rows = min(PC_BLOCK, n - j0);
-    const __nv_bfloat16* src = k + ((size_t)u * n + j0) * D;
+    const __nv_bfloat16* src = k + sk.at(u / Hk, u % Hk, j0);
     for (int idx = tid; idx < PC_BLOCK * (D / 8); idx += PC_THREADS) {
         const int r = idx / (D / 8), c = (idx % (D / 8)) * 8;
         float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        if (r < rows) load8(src + (size_t)r * D + c, x);
+        if (r < rows) load8(src + (size_t)r * sk.r + c, x);
 #pragma unroll
         for (int e = 0; e < 8; ++e) ks[r * LD + c + e] = x[e];
     }
@@ -207,12 +207,13 @@ precond_invert_kernel(const float* __restrict__ gram, __half* __restrict__ minv,
 }
 
 template <int D>
-int launch_t(const __nv_bfloat16* k, int units, int n, float lambda, int window, float* gram, __half* minv, cudaStream_t st) {
+int launch_t(const __nv_bfloat16* k, int B, int Hk, Strides sk, int n, float lambda, int window, float* gram, __half* minv, cudaStream_t st) {
+    const int units = B * Hk;
     const int nb = precond_blocks(n), rec = D * D + D;
     const size_t smem_g = sizeof(float) * PC_BLOCK * (D + 1), smem_i = sizeof(float) * (D * (D + 1) + D);
     LLA_CUDA_TRY(cudaFuncSetAttribute(gram_blocks_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_g));
     LLA_CUDA_TRY(cudaFuncSetAttribute(precond_invert_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_i));
-    gram_blocks_kernel<D><<<dim3(nb, units), PC_THREADS, smem_g, st>>>(k, gram, n, nb);
+    gram_blocks_kernel<D><<<dim3(nb, units), PC_THREADS, smem_g, st>>>(k, gram, n, nb, Hk, sk);
     LLA_CUDA_TRY(cudaGetLastError());
     if (nb > 1) {
         gram_scan_kernel<<<dim3((rec + PC_THREADS - 1) / PC_THREADS, units), PC_THREADS, 0, st>>>(gram, nb, rec);
@@ -234,10 +235,11 @@ size_t precond_minv_bytes(int units, int n, int d) {
     return ((size_t)units * precond_blocks(n) * (size_t)d * d * sizeof(__half) + 255) & ~(size_t)255;
 }
 
-int launch_precond(const void* k, int units, int n, int d, float lambda, int window, void* gram, void* minv, cudaStream_t st) {
-    if (d == 64) return launch_t<64>(static_cast<const __nv_bfloat16*>(k), units, n, lambda, window, static_cast<float*>(gram),
+int launch_precond(const void* k, int B, int Hk, Strides sk, int n, int d, float lambda, int window, void* gram, void* minv,
+                   cudaStream_t st) {
+    if (d == 64) return launch_t<64>(static_cast<const __nv_bfloat16*>(k), B, Hk, sk, n, lambda, window, static_cast<float*>(gram),
                                      static_cast<__half*>(minv), st);
-    if (d == 128) return launch_t<128>(static_cast<const __nv_bfloat16*>(k), units, n, lambda, window, static_cast<float*>(gram),
+    if (d == 128) return launch_t<128>(static_cast<const __nv_bfloat16*>(k), B, Hk, sk, n, lambda, window, static_cast<float*>(gram),
                                        static_cast<__half*>(minv), st);
     return LLA_ERR_UNSUPPORTED;
 }

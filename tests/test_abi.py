@@ -111,6 +111,11 @@ def test_validation_of_the_position_options(lib):
     assert fwd(window=200, causal=0) == 2          # a window needs the causal order
     assert fwd(window=50) == 2                     # below the direct-row threshold (96)
     assert fwd(q_rows=600) == 1                    # more queries than keys
+    L3 = ctypes.c_longlong * 3
+    assert fwd(q_strides=L3(512 * 64, 64, 4 * 64 + 4)) == 1     # a row stride that is not a multiple of 8 elements
+    assert fwd(out_strides=L3(512 * 64, -64, 64)) == 1
+    assert fwd(cg_precondition=2) == 1
+    assert fwd(debug_flags=8) == 1
 
     def dec(**kw):
         p = binding.DecodeParams()
@@ -145,13 +150,17 @@ def test_validation_of_the_position_options(lib):
     assert bwd(workspace=0x10010) == 3             # not 256-byte aligned
     assert bwd(kv_heads=3) == 1
     assert bwd(impl=7) == 1
-    # the pass's own vectors, then the scratch of the forward's CG kernel that it runs (fp16 copy of k + a status word)
-    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == 4 * 4 * 256 * (4 * 64 + 8) + 4 * 256 * 64 * 2 + 256
+    # the pass's own vectors, then the scratch of the forward's CG kernel that it runs: fp16 copy of k + a status word,
+    # Gram sums and preconditioner matrices per block of 128 keys (2 blocks, 4 heads)
+    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == (4 * 4 * 256 * (4 * 64 + 8) + 4 * 256 * 64 * 2 + 256
+                                                                  + 4 * 2 * (64 * 64 + 64) * 4 + 4 * 2 * 64 * 64 * 2)
 
 
 def test_workspace_and_split_arithmetic(lib):
     # tensor-core forward: fp16 copy of k + a status word (d = 128 adds per-SM slots, which need the device's SM count)
-    assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == 4 * 8 * 1024 * 64 * 2 + 256
+    assert binding.lla_forward_workspace_bytes(4, 8, 1024, 64, 64) == (4 * 8 * 1024 * 64 * 2 + 256          # fp16 copy of k, status word
+                                                                       + 32 * 8 * (64 * 64 + 64) * 4     # Gram sums, 8 blocks of 128 keys
+                                                                       + 32 * 8 * 64 * 64 * 2)           # preconditioner matrices
     assert binding.lla_forward_workspace_bytes(1, 1, 256, 16, 16, in_dtype=binding.LLA_F32) == 0
     # unsplit: optional record buffer for the two-kernel tensor-core path (bf16, d = 64), else none
     assert binding.lla_decode_workspace_bytes(2, 4, 4096, 64, 64, splits=1) == 4 * 2 * 4 * (2 * 64 * 64 + 132)

@@ -492,6 +492,39 @@ def test_preconditioned_cg_gives_the_same_rows_in_fewer_iterations(oracle, case)
         assert its[1] <= 0.75 * its[0], its
 
 
+@pytest.mark.parametrize("dtype,d,n,impl", [("bf16", 64, 700, L.LLA_IMPL_AUTO), ("bf16", 128, 450, L.LLA_IMPL_AUTO),
+                                             ("bf16", 64, 300, L.LLA_IMPL_SIMT), ("f32", 16, 200, L.LLA_IMPL_AUTO)])
+def test_strided_layouts_are_read_in_place(oracle, dtype, d, n, impl):
+    # tensors kept as [B, n, H, d] (position-major, as many frameworks store them), grouped key/value heads, a padded
+    # row pitch for v and an output that is a column slice of a wider buffer: all addressed through the strides
+    B, H, Hk = 2, 4, 2
+    w = inputs.CONFIGS[2].shrink(B=B, H=H, n=n, d=d, dv=d, dtype=dtype, seed=111 + d)
+    q, k, v = inputs.make_prefill(w)
+    k, v = k[:, :Hk], v[:, :Hk]
+    ref = oracle.forward(q, np.repeat(k, H // Hk, axis=1), np.repeat(v, H // Hk, axis=1), w.scale, w.lam)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    q_bnhd = torch.from_numpy(q).to(tdt).cuda().permute(0, 2, 1, 3).contiguous()            # [B, n, H, d]
+    k_bnhd = torch.from_numpy(k).to(tdt).cuda().permute(0, 2, 1, 3).contiguous()            # [B, n, Hk, d]
+    pitch = d + 8
+    v_pad = torch.zeros((B, Hk, n, pitch), dtype=tdt, device="cuda")                       # rows of d + 8 elements
+    v_pad[..., :d] = torch.from_numpy(v).to(tdt).cuda()
+    out_wide = torch.full((B, n, H, 2 * d), float("nan"), dtype=torch.float32, device="cuda")   # out in columns d .. 2d
+    out_view = out_wide[..., d:]
+    nbytes = L.lla_forward_workspace_bytes(B, H, n, d, d, LLA_DT[dtype], impl)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    for pc in ((0, 1) if dtype == "bf16" and impl == L.LLA_IMPL_AUTO else (0,)):
+        out_wide.fill_(float("nan"))
+        L.lla_forward_ex(q_bnhd, k_bnhd, v_pad, out_view, B, H, n, d, d, w.scale, w.lam, in_dtype=LLA_DT[dtype],
+                         out_dtype=L.LLA_F32, impl=impl, kv_heads=Hk, cg_precondition=pc, workspace=ws if nbytes else None,
+                         workspace_bytes=nbytes, stream=stream_ptr(),
+                         q_strides=(n * H * d, d, H * d), k_strides=(n * Hk * d, d, Hk * d),
+                         v_strides=(Hk * n * pitch, n * pitch, pitch), out_strides=(n * H * 2 * d, 2 * d, H * 2 * d))
+        torch.cuda.synchronize()
+        got = out_wide[..., d:].permute(0, 2, 1, 3).cpu().numpy()
+        assert torch.isnan(out_wide[..., :d]).all()                                          # nothing written beside the slice
+        assert row_err(got, ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16), pc
+
+
 def test_values_beyond_the_fp16_range_fall_back_to_pairs(oracle):
     # a key entry of 7e4 cannot be held in fp16: the pre-pass notices and every sweep of the call runs on the bf16
     # inputs.  The entry sits in the last key, which only the last row sees (that row's system is hopelessly
