@@ -192,6 +192,14 @@ typedef struct lla_forward_params {
                        as [B, n, H, d]: strides (n H d, d, H d).  The caller guarantees that the strides address
                        memory it owns and that rows of `out` do not overlap.  The optional per-row outputs (rho,
                        stats, iters) and lambda_rows stay contiguous [B, H, rows, ...].  Forward only */
+    const unsigned char *block_mask; /* block sparsity (tensor-core kernel, causal, no window): device array
+                       [ceil(q_rows / 128)][ceil(n / 64)] of bytes, row t for the query rows 128 t .. 128 t + 127,
+                       entry c for the keys 64 c .. 64 c + 63; nonzero = the rows of that tile attend to the keys
+                       of that block (those at or before their own position).  Always attended whatever the mask
+                       says: the blocks of the first head_rows keys (so that every row's system stays well posed
+                       and the directly-solved rows are untouched) and the blocks on the tile's diagonal.  NULL =
+                       dense.  n <= 65536.  Shapes the tensor-core kernel does not cover: LLA_ERR_UNSUPPORTED */
+    long long block_mask_stride;     /* bytes from one (batch, head) unit's mask to the next; 0 = one mask for all */
     int cg_precondition;  /* tensor-core kernel only.  0 = plain conjugate gradients as in Algorithm 2 (default).
                        1 = preconditioned with the inverse covariance of the visible keys: one d x d matrix per
                        block of 128 keys, built by a pre-pass into `workspace` (plain CG without room for it

@@ -64,7 +64,7 @@ class ForwardParams(ctypes.Structure):
         ("q_rows", ctypes.c_int), ("kv_heads", ctypes.c_int), ("window", ctypes.c_int),
         ("cg_precise_iters", ctypes.c_int),
         ("q_strides", ctypes.c_longlong * 3), ("k_strides", ctypes.c_longlong * 3), ("v_strides", ctypes.c_longlong * 3),
-        ("out_strides", ctypes.c_longlong * 3),
+        ("out_strides", ctypes.c_longlong * 3), ("block_mask", ctypes.c_void_p), ("block_mask_stride", ctypes.c_longlong),
         ("cg_precondition", ctypes.c_int), ("debug_wait_clocks", ctypes.c_longlong),
         ("debug_flags", ctypes.c_int),
     ]
@@ -184,8 +184,9 @@ def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=
                    device_status=None, workspace=None, workspace_bytes=0, stream=0, lambda_rows=None,
                    ridge_mode=LLA_RIDGE_DEFINITION, q_rows=0, kv_heads=0, window=0, cg_precise_iters=0,
                    debug_wait_clocks=0, debug_flags=0, cg_precondition=0, q_strides=None, k_strides=None, v_strides=None,
-                   out_strides=None):
+                   out_strides=None, block_mask=None, block_mask_stride=0):
     p = ForwardParams()
+    p.block_mask, p.block_mask_stride = _p(block_mask), block_mask_stride
     for name, val in (("q_strides", q_strides), ("k_strides", k_strides), ("v_strides", v_strides), ("out_strides", out_strides)):
         if val is not None:
             setattr(p, name, (ctypes.c_longlong * 3)(*[int(x) for x in val]))

@@ -118,6 +118,7 @@ ForwardArgs to_args(const lla_forward_params* p) {
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
     a.window = p->window;
     a.wait_clocks = p->debug_wait_clocks;
+    a.block_mask = p->block_mask; a.block_mask_stride = p->block_mask_stride;
     // layouts: all-zero strides mean contiguous [B, heads, rows, width]
     a.set_contiguous();
     auto take = [](lla::Strides& dst, const long long* src) {
@@ -179,6 +180,7 @@ int lla_forward_ex(const lla_forward_params* p) {
     const bool tensor_ok = lla::forward_tensor_supported(a);
     if (p->impl == LLA_IMPL_TENSOR && !tensor_ok) return LLA_ERR_UNSUPPORTED;
     const bool use_tensor = tensor_ok && p->impl != LLA_IMPL_SIMT;
+    if (p->block_mask && (!use_tensor || !a.causal || a.window > 0 || a.n > 65536 || p->block_mask_stride < 0)) return LLA_ERR_UNSUPPORTED;
     // the forward workspace is optional (see lla_forward_workspace_bytes); a misaligned one is an error
     if (a.workspace && a.workspace_bytes > 0 && ((uintptr_t)a.workspace & 255u)) return LLA_ERR_WORKSPACE;
     (void)use_tensor;

@@ -88,6 +88,8 @@ struct ForwardArgs {
         sq = contiguous_strides(H, nq, d); sk = contiguous_strides(hk, n, d);
         sv = contiguous_strides(hk, n, dv); so = contiguous_strides(H, nq, dv);
     }
+    const unsigned char* block_mask = nullptr;   // tensor-core kernel: block sparsity (lla_forward_params.block_mask)
+    long long block_mask_stride = 0;
     long long wait_clocks = 0;  // tensor-core kernel: cap of its bounded waits in SM clocks (0: default) and a test
     int no_loads = 0;           // aid: issue no copy at all (lla_forward_params.debug_*)
     const void* minv = nullptr; // CG preconditioner matrices (fp16), set by forward_tensor_prepass when enabled

@@ -52,6 +52,7 @@ constexpr int TC_R_COL = 0;                 // preconditioner product, between s
 constexpr int TC_Z_COL = 128;               // Z = R M (fp32, D columns) from buffer 1's columns on
 constexpr int TC_NST_MAX = 4;
 constexpr int TC_ORDER_MAX = 256;    // launch-order table size (query tiles)
+constexpr int TC_BLIST_MAX = 1024;   // key blocks a block-sparse tile can list (n <= 65536)
 constexpr int TC_SPLIT_MAX = 4;      // sweeps of at most this many key blocks run in split mode (see the compute role)
 
 // SW_CG16: a CG sweep whose on-the-fly operands (P, U) are single fp16 values instead of bf16 hi + lo pairs
@@ -83,7 +84,8 @@ struct TcCfg {
     static constexpr int SM_FLAGS = SM_RED + 8192;                                // 2 x 8 ints
     static constexpr int SM_BAR = SM_FLAGS + 64;                                  // mbarriers
     static constexpr int SM_MISC = SM_BAR + 256;                                  // tmem base, ctl kind, abort
-    static constexpr int SM_TOTAL = SM_MISC + 64;
+    static constexpr int SM_BLIST = SM_MISC + 64;                                 // block-sparse: the tile's key blocks (uint16)
+    static constexpr int SM_TOTAL = SM_BLIST + 2 * TC_BLIST_MAX;
     static constexpr int SM_ALLOC = SM_TOTAL + 1024;                              // slack for 1024-byte alignment
     static constexpr uint32_t IDESC_TS = sm100::make_idesc(TC_BR, D, 0, 1);   // ACC: A from TMEM, B MN-major, N = D
     static constexpr uint32_t IDESC_TS16 = sm100::make_idesc(TC_BR, D, 0, 1, /*f16=*/1);   // same, both operands fp16
@@ -211,6 +213,8 @@ struct TcParams {
     float* scratch;      // D = 128: per-SM slots for x, kbar, r (TcCfg::SCRATCH_FLOATS_PER_SM each)
     int scratch_slots;
     const float* lambda_rows;   // optional per-row ridge [B, H, n]
+    const unsigned char* block_mask;   // optional [query tiles][key blocks] (+ bh * block_mask_stride): nonzero = attended
+    long long block_mask_stride;
     int ridge_mode;
     int use_order;       // 1: blockIdx.y -> tile through order[]; 0: last tile first
     unsigned short order[TC_ORDER_MAX];
@@ -266,7 +270,27 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int cend = prm.causal ? min(nblk_all, (off + r0 + TC_BR + TC_BC - 1) / TC_BC) : nblk_all;
     // sliding window: the tile's sweeps start at the block that holds its first row's first visible key
     const int cbeg = (prm.causal && prm.window > 0) ? max(0, off + r0 + 1 - prm.window) / TC_BC : 0;
-    const int nblk = cend - cbeg;                        // key blocks per sweep: cbeg .. cend - 1
+    // Block sparsity: the sweeps visit only the key blocks that the caller's mask lists for this query tile, plus
+    // the ones that are always attended -- the blocks of the first head_rows keys (so that every row keeps enough
+    // keys for its system to be well posed and the directly-solved rows are untouched) and the tile's diagonal blocks.
+    unsigned short* blist = reinterpret_cast<unsigned short*>(smem + Cfg::SM_BLIST);
+    if (prm.block_mask) {
+        if (warp == 0) {
+            const unsigned char* mrow = prm.block_mask + (size_t)bh * prm.block_mask_stride + (size_t)tile * nblk_all;
+            int cnt = 0;
+            for (int c0 = cbeg; c0 < cend; c0 += 32) {
+                const int c = c0 + lane;
+                const bool on = c < cend && (mrow[c] != 0 || c * TC_BC < prm.head_rows || c * TC_BC + TC_BC - 1 >= off + r0);
+                const unsigned m = __ballot_sync(0xffffffffu, on);
+                if (on) blist[cnt + __popc(m & ((1u << lane) - 1))] = (unsigned short)c;
+                cnt += __popc(m);
+            }
+            if (lane == 0) misc[6] = cnt;
+        }
+        __syncthreads();
+    }
+    const int nblk = prm.block_mask ? misc[6] : cend - cbeg;      // key blocks per sweep
+    auto kblock = [&](int c) { return prm.block_mask ? (int)blist[c] : cbeg + c; };     // c-th key block of a sweep
     const bool split = nblk <= TC_SPLIT_MAX;
     // Operand format of a sweep over the keys.  The statistics sweep(s) and the first `precise` CG sweeps run on
     // the bf16 inputs; every later sweep (the remaining CG sweeps and, if CG got that far, the output sweep) runs
@@ -341,7 +365,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 mbar_expect_tx(bar(B_KVFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
                     tma_load_4d(sbase + SM_KV + s * STAGE + sub * Cfg::KSUB_BYTES, f16 ? &tmK16 : &tmK, bar(B_KVFULL + s), 64 * sub,
-                                (cbeg + c) * TC_BC, hk, bb);
+                                kblock(c) * TC_BC, hk, bb);
                 ++kit;
             };
             uint32_t v_g0 = 0;
@@ -352,7 +376,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const uint32_t s = g % TC_NST;
                 mbar_expect_tx(bar(B_VFULL + s), KBLK);
                 for (int sub = 0; sub < KSUB; ++sub)
-                    tma_load_4d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, (cbeg + c) * TC_BC, hk, bb);
+                    tma_load_4d(sbase + SM_KV + s * STAGE + KBLK + sub * Cfg::KSUB_BYTES, &tmV, bar(B_VFULL + s), 64 * sub, kblock(c) * TC_BC, hk, bb);
             };
             int cg_seen = 0;       // CG sweeps issued so far
             for (uint32_t ctl = 0; ok; ++ctl) {
@@ -647,8 +671,8 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     // keys jfirst <= e < jlim of this half block are visible.  Only the diagonal blocks and a
                     // window's first blocks hide any: there the hidden scores are overwritten with a large negative
                     // number, whose weight is exactly zero, so the loops below carry no mask
-                    const int jlim = min(L, n) - ((cbeg + c) * TC_BC + 32 * h);
-                    const int jfirst = jlo - ((cbeg + c) * TC_BC + 32 * h);
+                    const int jlim = min(L, n) - (kblock(c) * TC_BC + 32 * h);
+                    const int jfirst = jlo - (kblock(c) * TC_BC + 32 * h);
                     if (jlim < 32 || jfirst > 0) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
@@ -1203,6 +1227,7 @@ int launch_t(const ForwardArgs& a) {
     prm.no_loads = a.no_loads;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
+    prm.block_mask = a.block_mask; prm.block_mask_stride = a.block_mask_stride;
     prm.rhs = a.rhs; prm.sol = a.sol;
     prm.H = a.H; prm.kv_group = a.kv_group > 0 ? a.kv_group : 1;
     prm.so = a.so;

@@ -525,6 +525,55 @@ def test_strided_layouts_are_read_in_place(oracle, dtype, d, n, impl):
         assert row_err(got, ref).max() <= (TOL_F32 if dtype == "f32" else TOL_BF16), pc
 
 
+@pytest.mark.parametrize("d,n,per_head", [(64, 1500, False), (128, 1100, True)])
+def test_block_sparse_forward(oracle, d, n, per_head):
+    # a random block mask (about 40 % of the [query tile] x [key block] pairs kept); the blocks of the first head_rows
+    # keys and each tile's diagonal blocks are attended whatever the mask says.  The oracle solves sampled rows as
+    # single queries over exactly their visible keys (its decode entry point).
+    B, H = 1, 3
+    w = inputs.CONFIGS[2 if d == 64 else 4].shrink(B=B, H=H, n=n, seed=130 + d)
+    q, k, v = inputs.make_prefill(w)
+    tiles, blocks = (n + 127) // 128, (n + 63) // 64
+    rng = np.random.default_rng(7)
+    units = B * H if per_head else 1
+    mask = (rng.random((units, tiles, blocks)) < 0.4).astype(np.uint8)
+    head_rows = d + d // 2
+    dmask = torch.from_numpy(mask).cuda()
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    got = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR, block_mask=dmask,
+                  block_mask_stride=tiles * blocks if per_head else 0, device_status=status)
+    st = status.cpu().tolist()
+    assert st[L.STATUS_TIMEOUT] == 0 and st[L.STATUS_ROWS_AT_CAP] == 0
+
+    def visible(u, i):
+        t = i // 128
+        keep = np.zeros(i + 1, dtype=bool)
+        for c in range(i // 64 + 1):
+            on = mask[u if per_head else 0, t, c] != 0 or c * 64 < head_rows or c * 64 + 63 >= t * 128
+            if on:
+                keep[c * 64:min(i + 1, c * 64 + 64)] = True
+        return np.nonzero(keep)[0]
+
+    pos = np.unique(np.concatenate([np.arange(0, 260, 7), rng.integers(0, n, 60), [n - 1]]))
+    samples = [(h, i) for h in range(H) for i in pos]
+    S = len(samples)
+    qs = np.zeros((S, 1, d), dtype=np.float32)
+    kc = np.zeros((S, 1, n, d), dtype=np.float32)
+    vc = np.zeros((S, 1, n, d), dtype=np.float32)
+    cnt = np.zeros(S, dtype=np.int32)
+    for s_, (h, i) in enumerate(samples):
+        idx = visible(h, i)
+        cnt[s_] = len(idx)
+        qs[s_, 0] = q[0, h, i]
+        kc[s_, 0, :len(idx)] = k[0, h, idx]
+        vc[s_, 0, :len(idx)] = v[0, h, idx]
+    ref = oracle.decode(qs, kc, vc, cnt, w.scale, w.lam)[:, 0]
+    mine = np.stack([got[0, h, i] for h, i in samples])
+    assert row_err(mine, ref).max() <= TOL_BF16
+    dense = forward(w, q, k, v, out_dtype="f32", impl=L.LLA_IMPL_TENSOR)
+    assert row_err(np.stack([dense[0, h, n - 1] for h in range(H)]), np.stack([got[0, h, n - 1] for h in range(H)])).max() > 10 * TOL_BF16
+
+
 def test_values_beyond_the_fp16_range_fall_back_to_pairs(oracle):
     # a key entry of 7e4 cannot be held in fp16: the pre-pass notices and every sweep of the call runs on the bf16
     # inputs.  The entry sits in the last key, which only the last row sees (that row's system is hopelessly
