@@ -14,8 +14,9 @@
 //   MMA (SS)    [D_hi | D_lo] += A [B_hi | B_lo]: the two B tiles lie back to back and are read as one
 //               N = 160 operand, so A is fetched once per 16-key step; D = D_hi + D_lo is formed
 //               when the accumulator is read out.
-// m_ref is the maximum of the first tile; if a later tile's maximum exceeds it by more than 2^40 the
-// accumulator is rescaled in TMEM (never triggered by bounded scores, covered by a test).  After
+// m_ref is the maximum of the first tile.  The threads only note whether a later score exceeds it by more
+// than 2^90 (no barrier per tile); if one did, the whole pass is repeated with the true maximum, which is
+// known by then (never triggered by bounded scores, covered by a test).  After
 // the last tile the moments are copied to shared memory and either solved on the spot (d x d LDL^T
 // in double precision, as in lla_decode.cu) or written as a partial record for the split-key merge.
 #include "lla_sm100.cuh"
@@ -46,7 +47,7 @@ constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 65 + 8 * (128 + 24);
 constexpr int SMD_ALLOC = (SMD_TOTAL > SMD_FIN ? SMD_TOTAL : SMD_FIN) + 1024;
 
 enum { DB_KVFULL = 0, DB_KVEMPTY = DB_KVFULL + DT_NST, DB_BFULL = DB_KVEMPTY + DT_NST, DB_BFREE = DB_BFULL + 2,
-       DB_DFULL = DB_BFREE + 2, DB_COUNT = DB_DFULL + 1 };
+       DB_DFULL = DB_BFREE + 2, DB_PASS = DB_DFULL + 1, DB_COUNT = DB_PASS + 1 };
 static_assert(DB_COUNT * 8 <= 128, "barrier area too small");
 
 // A = [K^T ; V^T]: MN-major, 128B swizzle; the V tile (second group of 64 rows of M) lies 8192 bytes
@@ -231,7 +232,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int s = 0; s < DT_NST; ++s) { mbar_init(bar(DB_KVFULL + s), 1); mbar_init(bar(DB_KVEMPTY + s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(bar(DB_BFULL + b), DT_COMPUTE / 32); mbar_init(bar(DB_BFREE + b), 1); }
         mbar_init(bar(DB_DFULL), 1);
+        mbar_init(bar(DB_PASS), DT_COMPUTE / 32);
         misc[1] = 0;
+        misc[2] = 0;      // set by the compute warps when the pass has to be repeated
         fence_barrier_init();
     }
     if (warp == 4) {
@@ -245,6 +248,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const uint32_t tmem = (uint32_t)misc[0];
 
     float omega = 0.f, m_ref = -INFINITY;     // compute threads; m_ref in log2 units
+    uint32_t d_parity = 0;                     // compute threads: phase of the accumulator barrier to wait for
 
     if (warp == 4) {
         // ================================ TMA producer ================================
@@ -254,9 +258,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group;
             const int kvh = (bh / prm.H) * hkv + kvl;
             const int* table = prm.paged.table ? prm.paged.table + (size_t)(bh / prm.H) * prm.paged.max_pages : nullptr;
-            for (int t = 0; t < ntile; ++t) {
-                const uint32_t s = t % DT_NST;
-                if (!mbar_wait(bar(DB_KVEMPTY + s), ((t / DT_NST) & 1) ^ 1, abort_flag)) break;
+            for (int g = 0, pass = 0; pass < 2; ++pass) {
+              bool okp = true;
+              for (int t = 0; t < ntile; ++t, ++g) {      // g: running tile count over both passes (ring position)
+                const uint32_t s = g % DT_NST;
+                if (!mbar_wait(bar(DB_KVEMPTY + s), ((g / DT_NST) & 1) ^ 1, abort_flag)) { okp = false; break; }
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
                 int unit = kvh, jrow = kstart + jbeg + t * DT_BK;
@@ -267,21 +273,28 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 tma_load_3d(dst, &tmK, bar(DB_KVFULL + s), 0, jrow, unit);
                 tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jrow, unit);
+              }
+              // a second pass only if the compute warps ask for it
+              if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag) || misc[2] == 0) break;
             }
         }
     } else if (warp == 5) {
         // ================================ MMA issuer (whole warp, predicated) ================================
         const uint32_t el = elect_one();
-        for (int t = 0; t < ntile; ++t) {
-            const uint32_t s = t % DT_NST, b = t & 1;
-            if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) break;
-            if (!mbar_wait(bar(DB_BFULL + b), (t >> 1) & 1, abort_flag)) break;
-            tc_fence_after();
-            const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
-            mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), t > 0);
-            tc_commit_el(el, bar(DB_KVEMPTY + s));
-            tc_commit_el(el, bar(DB_BFREE + b));
-            if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
+        for (int g = 0, pass = 0; pass < 2; ++pass) {
+            bool okp = true;
+            for (int t = 0; t < ntile; ++t, ++g) {
+                const uint32_t s = g % DT_NST, b = g & 1;
+                if (!mbar_wait(bar(DB_KVFULL + s), (g / DT_NST) & 1, abort_flag)) { okp = false; break; }
+                if (!mbar_wait(bar(DB_BFULL + b), (g >> 1) & 1, abort_flag)) { okp = false; break; }
+                tc_fence_after();
+                const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
+                mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), t > 0);     // t == 0 overwrites
+                tc_commit_el(el, bar(DB_KVEMPTY + s));
+                tc_commit_el(el, bar(DB_BFREE + b));
+                if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
+            }
+            if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag) || misc[2] == 0) break;
         }
     } else {
         // ================================ compute warps ================================
@@ -305,9 +318,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         uint4 raw[4];
         float kf[32];
         float w = 0.f;
-        auto stage_load = [&](int t) -> bool {
-            const uint32_t s = t % DT_NST;
-            if (!mbar_wait(bar(DB_KVFULL + s), (t / DT_NST) & 1, abort_flag)) return false;
+        // (t: tile of the pass, it fixes the keys; g: running tile count over both passes, it fixes ring stage,
+        //  buffer and barrier phase)
+        auto stage_load = [&](int g) -> bool {
+            const uint32_t s = g % DT_NST;
+            if (!mbar_wait(bar(DB_KVFULL + s), (g / DT_NST) & 1, abort_flag)) return false;
             uint8_t* ktile = smem + SMD_KV + s * 16384;
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -318,8 +333,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         bool valid = false;
         // first half of the score stage: arithmetic only (no barrier), so it can run while the
         // stores of the tile before are still draining
-        auto stage_score_math = [&](int t) {
-            const uint32_t s = t % DT_NST;
+        auto stage_score_math = [&](int t, int g) {
+            const uint32_t s = g % DT_NST;
             uint8_t* ktile = smem + SMD_KV + s * 16384;
             valid = jbeg + t * DT_BK + jl < jend;
 #pragma unroll
@@ -350,104 +365,95 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             sdot += __shfl_xor_sync(0xffffffffu, sdot, 16);
             s2 = valid ? sdot * c1 : -INFINITY;
         };
-        // second half: the block-wide rescale check and the weight
-        auto stage_score_sync = [&](int t) -> bool {
-            // The reference maximum is the first tile's.  Later tiles only need to know whether any
-            // score exceeds it by more than 2^40 (then the accumulator is rescaled): one barrier
-            // that ORs a predicate over the 128 compute threads answers that; the tile maximum
-            // itself is reduced only for the first tile and in the rare rescale.
-            bool need_max = t == 0;
-            if (t > 0) {
-                uint32_t any;
-                asm volatile(
-                    "{\n\t.reg .pred p, q;\n\tsetp.gt.f32 q, %1, %2;\n\t"
-                    "barrier.cta.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                    : "=r"(any) : "f"(s2), "f"(m_ref + 40.f) : "memory");
-                need_max = any != 0;
-            }
-            float tile_max = m_ref;
-            if (need_max) {
+        // second half: the weight.  The reference maximum is the first tile's (one block-wide reduction per pass at
+        // most); later tiles only note, per thread and without any barrier, the largest score seen and whether one
+        // exceeded the reference by more than 2^90 -- then the weights of this pass are useless (they are clamped,
+        // so nothing overflows) and the pass is repeated with the true maximum as reference.
+        float run_max = -INFINITY;
+        bool over = false;
+        auto stage_score_sync = [&](int t, bool first_pass) {
+            if (t == 0 && first_pass) {
                 float wm = s2;
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
-                volatile float* tm = tmax + (t & 1) * 4;
-                if (lane == 0) tm[warp] = wm;
+                if (lane == 0) tmax[warp] = wm;
                 named_sync_128();
-                tile_max = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
+                m_ref = fmaxf(fmaxf(tmax[0], tmax[1]), fmaxf(tmax[2], tmax[3]));
             }
-            if (t == 0) {
-                m_ref = tile_max;
-            } else if (tile_max > m_ref + 40.f) {
-                // rare: rescale the accumulator (all MMAs of earlier tiles must have finished; this
-                // thread's B rows of tile t-1 were handed over before this call)
-                const float f = ex2f(m_ref - tile_max);
-                if (!mbar_wait(bar(DB_BFREE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag)) return false;
-                tc_fence_after();
-                const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-#pragma unroll 1
-                for (int cb = 0; cb < 2 * DT_N; cb += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_addr + cb, v);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
-                    tmem_st32(lane_addr + cb, v);
-                    tc_wait_st();
-                }
-                tc_fence_before();
-                omega *= f;
-                m_ref = tile_max;
-                named_sync_128();
-            }
-            w = valid ? ex2f(s2 - m_ref) : 0.f;
+            run_max = fmaxf(run_max, s2);
+            over |= s2 > m_ref + 90.f;
+            w = valid ? ex2f(fminf(s2 - m_ref, 100.f)) : 0.f;
             if (h == 0) omega += w;
-            return true;
         };
-        if (ntile > 0) {
-            ok = stage_load(0);
-            if (ok) {
-                stage_score_math(0);
-                ok = stage_score_sync(0);
-            }
-        }
-        for (int t = 0; t < ntile && ok; ++t) {
-            const uint32_t b = t & 1;
-            const bool more = t + 1 < ntile;
-            // wait until the MMA of tile t-2 has released this B buffer (long done in steady state)
-            if (!mbar_wait(bar(DB_BFREE + b), ((t >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            // B rows of tile t: w * [k | 1] as bf16 hi + lo, eight features at a time straight into the
-            // operand tiles, so the stores drain while the rest of the iteration runs
-            uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
-            uint8_t* blo = bhi + DT_BTILE;
-            const uint64_t ww = pk2(w, w);
+        for (int pass = 0, g0 = 0; pass < 2 && ok && ntile > 0; ++pass, g0 += ntile) {
+            omega = 0.f;
+            ok = stage_load(g0);
+            if (!ok) break;
+            stage_score_math(0, g0);
+            stage_score_sync(0, pass == 0);
+            for (int t = 0; t < ntile && ok; ++t) {
+                const int g = g0 + t;
+                const uint32_t b = g & 1;
+                const bool more = t + 1 < ntile;
+                // wait until the MMA of the tile two before has released this B buffer (long done in steady state)
+                if (!mbar_wait(bar(DB_BFREE + b), ((g >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                // B rows of tile t: w * [k | 1] as bf16 hi + lo, eight features at a time straight into the
+                // operand tiles, so the stores drain while the rest of the iteration runs
+                uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
+                uint8_t* blo = bhi + DT_BTILE;
+                const uint64_t ww = pk2(w, w);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t hi[4], lo[4];
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t hi[4], lo[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float a, bq;
-                    upk2(mul2(ww, pk2(kf[8 * i + 2 * e], kf[8 * i + 2 * e + 1])), a, bq);
-                    hi[e] = split_bf16x2(a, bq, lo[e]);
+                    for (int e = 0; e < 4; ++e) {
+                        float a, bq;
+                        upk2(mul2(ww, pk2(kf[8 * i + 2 * e], kf[8 * i + 2 * e + 1])), a, bq);
+                        hi[e] = split_bf16x2(a, bq, lo[e]);
+                    }
+                    const uint32_t off = (4 * h + i) * 1024 + rowoff;          // column block 4h+i
+                    *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
-                const uint32_t off = (4 * h + i) * 1024 + rowoff;          // column block 4h+i
-                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4*>(blo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                {   // column blocks 8 (ones column first) and 9 (zero padding)
+                    uint32_t wlo;
+                    const uint32_t whi = split_bf16x2(w, 0.f, wlo);
+                    const uint32_t off = (8 + h) * 1024 + rowoff;
+                    *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
+                }
+                // the next tile: shared-memory loads, then the score arithmetic, while the stores drain
+                if (more && !stage_load(g + 1)) { ok = false; break; }
+                if (more) stage_score_math(t + 1, g + 1);
+                fence_proxy_async();
+                // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised shared-memory atomics
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(DB_BFULL + b));
+                if (more) stage_score_sync(t + 1, false);
             }
-            {   // column blocks 8 (ones column first) and 9 (zero padding)
-                uint32_t wlo;
-                const uint32_t whi = split_bf16x2(w, 0.f, wlo);
-                const uint32_t off = (8 + h) * 1024 + rowoff;
-                *reinterpret_cast<uint4*>(bhi + off) = make_uint4(h == 0 ? whi : 0u, 0, 0, 0);
-                *reinterpret_cast<uint4*>(blo + off) = make_uint4(h == 0 ? wlo : 0u, 0, 0, 0);
+            if (!ok || pass == 1) break;
+            // end of the first pass: did any score leave the range of the reference?  (one barrier per pass)
+            uint32_t any;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+                "barrier.cta.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(any) : "r"((uint32_t)over) : "memory");
+            if (any) {
+                float wm = run_max;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
+                if (lane == 0) tmax[4 + warp] = wm;
             }
-            // the next tile: shared-memory loads, then the score arithmetic, while the stores drain
-            if (more && !stage_load(t + 1)) { ok = false; break; }
-            if (more) stage_score_math(t + 1);
-            fence_proxy_async();
-            // one arrival per warp: 32 lanes arriving on one mbarrier are 32 serialised shared-memory atomics
+            if (tid == 0) misc[2] = (int)any;
+            named_sync_128();
+            if (any) {
+                m_ref = fmaxf(fmaxf(tmax[4], tmax[5]), fmaxf(tmax[6], tmax[7]));
+                over = false;
+                d_parity = 1;            // the accumulator of the second pass completes the barrier's second phase
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(DB_BFULL + b));
-            if (more && !stage_score_sync(t + 1)) { ok = false; break; }
+            if (lane == 0) mbar_arrive(bar(DB_PASS));      // the TMA and MMA warps read misc[2] after this
+            if (!any) break;
         }
         // total weight of this part
         if (ok) {
@@ -464,7 +470,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (tid == 0) s_mref = m_ref;
     bool d_ok = true;
     if (warp < 4 && ntile > 0) {
-        d_ok = mbar_wait(bar(DB_DFULL), 0, abort_flag);
+        d_ok = mbar_wait(bar(DB_DFULL), d_parity, abort_flag);
         tc_fence_after();
     }
     // moments -> registers (lane f: row f of M plus a[f]; lane 64+f: row f of N plus c[f])

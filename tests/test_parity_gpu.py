@@ -152,8 +152,8 @@ def test_decode_matches_oracle_and_splits_agree(oracle, dtype, d):
 @pytest.mark.parametrize("impl", [L.LLA_IMPL_SIMT, L.LLA_IMPL_AUTO])
 def test_decode_unused_slots_and_late_maximum(oracle, impl):
     """Slots past lens[b] may hold anything (here NaN) and must not leak into the result; and a cache
-    whose first 64 keys score ~70 units below the rest forces the tensor path to rescale its running
-    accumulator when the later, larger scores arrive."""
+    whose first 64 keys score ~70 units (2^101) below the rest forces the tensor path to give up its first
+    pass, whose weights are relative to the first tile's maximum, and stream the cache again with the true maximum."""
     w = inputs.CONFIGS[5].shrink(B=2, H=2, n=1200, len_min=300, len_max=1200, seed=61)
     q, kc, vc, lens = inputs.make_decode(w)
     lens[:] = [1111, 333]
