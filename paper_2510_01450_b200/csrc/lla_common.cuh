@@ -168,6 +168,9 @@ size_t forward_tensor_scratch_bytes();         // d = 128 row-state scratch (0 i
 size_t forward_tensor_workspace_bytes(int B, int H, int n, int d);   // that scratch + the fp16 copy of k (upper bound: kv heads = H)
 // CG preconditioner of the tensor-core forward (lla_precond.cu): one d x d fp16 matrix per block of 128 keys
 int precond_blocks(int n);
+// Beyond the first 16 blocks (2048 keys) the covariance changes little from one block of 128 keys to the next: only
+// every fourth block gets a matrix of its own there, and a tile takes the last one at or before its key block.
+__host__ __device__ __forceinline__ int precond_block_used(int g) { return g < 16 ? g : ((g + 1) / 4) * 4 - 1; }
 size_t precond_gram_bytes(int units, int n, int d);     // fp32 running Gram sums (scratch of the pre-pass)
 size_t precond_minv_bytes(int units, int n, int d);     // the fp16 matrices [units][blocks][d][d]
 int launch_precond(const void* k, int B, int Hk, Strides sk, int n, int d, float lambda, int window, void* gram, void* minv,

@@ -349,7 +349,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (PC) {
                 // the preconditioner of this tile's key range: D x D fp16, laid out like D / 64 key blocks, into the
                 // V halves of the first ring stages (idle until the output sweep, when it is no longer needed)
-                const int gm = (prm.causal ? min(n - 1, off + r0 + TC_BR - 1) : n - 1) / 128;
+                const int gm = precond_block_used((prm.causal ? min(n - 1, off + r0 + TC_BR - 1) : n - 1) / 128);
                 mbar_expect_tx(bar(B_MFULL), D * D * 2);
                 for (int rb = 0; rb < D / 64; ++rb)
                     for (int sub = 0; sub < KSUB; ++sub)

@@ -90,6 +90,7 @@ precond_invert_kernel(const float* __restrict__ gram, __half* __restrict__ minv,
     __shared__ float s_red[PC_THREADS / 32];
     __shared__ int s_bad;
     const int g = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    if (precond_block_used(g) != g) return;        // no tile asks for this block's matrix
     const int rec = D * D + D;
     const int hi = min(n, PC_BLOCK * (g + 1));
     const int glo = window > 0 ? max(0, hi - window) / PC_BLOCK : 0;     // first block that counts
