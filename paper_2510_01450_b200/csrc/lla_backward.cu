@@ -16,16 +16,17 @@
 // In exact arithmetic this is the appendix's Delta_Q, Delta_K, Delta_V (same function, same derivative);
 // y follows from the saved rho and delta as y = rho omega / delta.
 //
-// Kernels (the direct rows run on a side stream beside the other four, which run in this order):
-//   bwd_moments_*         per 64-row query tile: kbar_i, gbar_i, h_i
+// Kernels (the direct rows run on a side stream beside the others, which run in this order):
+//   bwd_split_kernel      an fp32 upstream gradient as bf16 pairs hi + lo
+//   moments               per query tile: kbar_i, gbar_i, h_i
 //   forward_tc_kernel     in solve mode: C_i t_i = h_i by conjugate gradients           (tcgen05 tensor cores)
-//   bwd_rowprep_kernel    y_i, the per-row scalars, dQ_i = t_i, dL/dlambda_i
-//   bwd_pairs_*           per 64-key tile over all later query tiles: dK, dV (registers), dQ (atomics)
+//   bwd_rowprep_kernel    y_i, the per-row scalars, dL/dlambda_i; y and -t as bf16 pairs
+//   pairs                 dQ per query tile, dK and dV per key tile
 //   bwd_head_rows_kernel  rows with fewer than head_rows keys: everything in fp64 with a direct solve
-// The moments and pair kernels exist twice: *_mma_kernel on the tensor cores (warp-level bf16 MMAs with hi/lo
-// operand splits; the default) and the fp32 CUDA-core versions (impl = LLA_IMPL_SIMT), kept as an independent
-// cross-check.  With grouped heads (kv_group > 1) k, v, dk, dv are indexed by the key/value head; dk and dv are
-// zeroed first and every kernel adds into them atomically.
+// The moments and pair kernels are the tcgen05 kernels of lla_backward_tensor.cu (dQ by plain stores of the tile
+// that owns the rows; dK and dV by atomic adds, which the direct rows and grouped heads also add into).  The fp32
+// CUDA-core versions in this file (impl = LLA_IMPL_SIMT) are kept as an independent cross-check; their pair kernel
+// adds dQ atomically.  With grouped heads (kv_group > 1) k, v, dk, dv are indexed by the key/value head.
 #include "lla_common.cuh"
 
 namespace lla {
@@ -199,35 +200,66 @@ bwd_moments_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 }
 
 // ------------------------------------------------------------------------------------------------
-// Per iterative row: y = rho omega / delta, the scalars the pair kernel needs, and dQ_i = t_i (the pair
-// kernel adds the rest with atomics).  One warp per row.
+// Per iterative row: y = rho omega / delta and the scalars the pair kernels need.  One warp per row.
+// CUDA-core pair kernel (pairs16 == nullptr): dQ_i = t_i, to which that kernel adds the rest with atomics.
+// Tensor-core pair kernels: y and -t also as bf16 pairs hi + lo (pairs16 = yh, yl, tnh, tnl, each [rows][D]); the
+// rows solved directly get zero operands and a zero record, which switches them off in those kernels.
 // ------------------------------------------------------------------------------------------------
+// (x0, x1) -> packed bf16 pairs hi and lo with x = hi + lo up to 2^-17 relative
+__device__ __forceinline__ void split_pack(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+    const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0)), l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+    hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+    lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+struct Pairs16 {
+    uint32_t *yh, *yl, *tnh, *tnl;      // two bf16 per word
+};
 template <int D>
 __global__ void __launch_bounds__(BW_THREADS)
 bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__ out, int out_dtype,
                    const void* __restrict__ dout, int dout_dtype, const float* __restrict__ rho,
                    const float* __restrict__ stats, const float* __restrict__ kbar, const float* __restrict__ tvec,
                    float* __restrict__ yvec, float* __restrict__ rowsc, float* __restrict__ dq, int n, int first,
-                   long long rows, float* __restrict__ dlambda) {
+                   long long rows, float* __restrict__ dlambda, Pairs16 p16) {
     const long long row = (long long)blockIdx.x * (BW_THREADS / 32) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= rows) return;
     const int i = (int)(row % n);
-    if (i < first) return;
+    if (i < first) {
+        if (p16.yh) {
+            for (int c = 2 * lane; c < D; c += 64) {
+                const size_t w = ((size_t)row * D + c) >> 1;
+                p16.yh[w] = 0; p16.yl[w] = 0; p16.tnh[w] = 0; p16.tnl[w] = 0;
+            }
+            if (lane < BW_ROWSC) rowsc[row * BW_ROWSC + lane] = 0.f;
+        }
+        return;
+    }
     const float m = stats[row * 3 + 0], omega = stats[row * 3 + 1], delta = stats[row * 3 + 2];
     const float fac = omega / delta;
     float ky = 0.f, kt = 0.f, qt = 0.f, go = 0.f, ty = 0.f;
 #pragma unroll
-    for (int c = lane; c < D; c += 32) {
+    for (int c = 2 * lane; c < D; c += 64) {
         const size_t e = (size_t)row * D + c;
-        const float yv = rho[e] * fac, tv = tvec[e], kb = kbar[e];
-        yvec[e] = yv;
-        dq[e] = tv;
-        ky = fmaf(kb, yv, ky);
-        kt = fmaf(kb, tv, kt);
-        ty = fmaf(tv, yv, ty);
-        qt = fmaf(__bfloat162float(q[e]), tv, qt);
-        go = fmaf(ld_any(dout, dout_dtype, e), ld_any(out, out_dtype, e), go);
+        const float2 r2 = *reinterpret_cast<const float2*>(rho + e), t2 = *reinterpret_cast<const float2*>(tvec + e);
+        const float2 kb = *reinterpret_cast<const float2*>(kbar + e);
+        const float y0 = r2.x * fac, y1 = r2.y * fac;
+        *reinterpret_cast<float2*>(yvec + e) = make_float2(y0, y1);
+        if (p16.yh) {
+            uint32_t h, l;
+            split_pack(y0, y1, h, l);
+            p16.yh[e >> 1] = h; p16.yl[e >> 1] = l;
+            split_pack(-t2.x, -t2.y, h, l);
+            p16.tnh[e >> 1] = h; p16.tnl[e >> 1] = l;
+        } else {
+            *reinterpret_cast<float2*>(dq + e) = t2;
+        }
+        ky = fmaf(kb.x, y0, fmaf(kb.y, y1, ky));
+        kt = fmaf(kb.x, t2.x, fmaf(kb.y, t2.y, kt));
+        ty = fmaf(t2.x, y0, fmaf(t2.y, y1, ty));
+        qt = fmaf(__bfloat162float(q[e]), t2.x, fmaf(__bfloat162float(q[e + 1]), t2.y, qt));
+        go = fmaf(ld_any(dout, dout_dtype, e), ld_any(out, out_dtype, e), fmaf(ld_any(dout, dout_dtype, e + 1), ld_any(out, out_dtype, e + 1), go));
     }
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) {
@@ -244,9 +276,24 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
         rs[3] = go + kt - qt;      // kappa = g.o + t.(kbar - q)
         rs[4] = ky;
         rs[5] = kt;
+        rs[6] = -m * 1.4426950408889634f;
+        rs[7] = 0.f;
         // dL/d(lambda_i): lambda enters C as (e^{-m} / omega) lambda I and dL = t^T dC y
         if (dlambda) dlambda[row] = __expf(-m) / omega * ty;
     }
+}
+
+// fp32 upstream gradient -> bf16 pairs hi + lo (the tensor-core kernels' operand format), four elements per thread
+__global__ void __launch_bounds__(256)
+bwd_split_kernel(const float* __restrict__ src, uint2* __restrict__ hi, uint2* __restrict__ lo, size_t quads) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= quads) return;
+    const float4 x = reinterpret_cast<const float4*>(src)[i];
+    uint2 h, l;
+    split_pack(x.x, x.y, h.x, l.x);
+    split_pack(x.z, x.w, h.y, l.y);
+    hi[i] = h;
+    lo[i] = l;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -366,374 +413,6 @@ bwd_pairs_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
                 atomicAdd(dk + (kvbase + gj) * D + c + x, adk[r][4 * u + x]);
                 atomicAdd(dv + (kvbase + gj) * D + c + x, adv[r][4 * u + x]);
             }
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// The pair kernel on the tensor cores (d = 64): the same block-per-key-tile loop with every product a
-// warp-level bf16 MMA (m16n8k16, fp32 accumulate).  fp32 operands (y, t, g and the pair coefficients)
-// enter as bf16 hi + lo pairs and each product keeps the three leading terms, so the result has fp32-like
-// accuracy.  A warp owns 16 of the block's 64 keys and forms the pair tiles transposed ([key][query]):
-// their accumulator fragments are then, after packing, the A operands of the dK / dV products with no
-// trip through shared memory.  Only scale dL/ds goes to shared memory, for the dQ product.
-// ------------------------------------------------------------------------------------------------
-// d = 128: the 128 output columns are split over two warps per key (query) group -- a warp's registers
-// hold accumulators for 64 columns only -- and both form the same pair tiles.
-template <int D>
-struct MmCfg {
-    static constexpr int LDB = D + 8;             // bf16 row stride of the operand tiles (conflict-free ldmatrix)
-    static constexpr int TILE = 64 * LDB;         // bf16 elements per 64-row tile
-    static constexpr int NCG = D / 64;            // column groups
-    static constexpr int THREADS = 128 * NCG;
-    static constexpr int KS = D / 16;             // k-steps of a contraction over the head dimension
-    static constexpr size_t PAIRS_SMEM = sizeof(__nv_bfloat16) * (size_t)11 * TILE + sizeof(float) * 6 * 64;
-    static constexpr size_t MOMENTS_SMEM = sizeof(__nv_bfloat16) * (size_t)5 * TILE;
-};
-
-__device__ __forceinline__ void ldsm4(uint32_t (&r)[4], const __nv_bfloat16* p) {
-    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
-}
-__device__ __forceinline__ void ldsm4t(uint32_t (&r)[4], const __nv_bfloat16* p) {
-    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// (x0, x1) -> packed bf16 pairs hi and lo with x = hi + lo up to 2^-17 relative
-__device__ __forceinline__ void split_pack(float x0, float x1, uint32_t& hi, uint32_t& lo) {
-    const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
-    const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0)), l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
-    hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-    lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-}
-// 64 rows x D columns -> bf16 tile(s) [64][D + 8]; fp32 sources are split into hi and lo tiles
-template <int D>
-__device__ __forceinline__ void mm_load_bf16(__nv_bfloat16* dst, const __nv_bfloat16* src, size_t row0, int nvalid) {
-    for (int idx = threadIdx.x; idx < 64 * (D / 8); idx += MmCfg<D>::THREADS) {
-        const int r = idx / (D / 8), c = (idx % (D / 8)) * 8;
-        uint4 x = make_uint4(0, 0, 0, 0);
-        if (r < nvalid) x = *reinterpret_cast<const uint4*>(src + (row0 + r) * D + c);
-        *reinterpret_cast<uint4*>(dst + r * MmCfg<D>::LDB + c) = x;
-    }
-}
-template <int D>
-__device__ __forceinline__ void mm_load_split(__nv_bfloat16* hi, __nv_bfloat16* lo, const void* src, int dtype, size_t row0,
-                                              int nvalid, int lo_row) {
-    constexpr int MM_LDB = MmCfg<D>::LDB;
-    for (int idx = threadIdx.x; idx < 64 * (D / 4); idx += MmCfg<D>::THREADS) {
-        const int r = idx / (D / 4), c = (idx % (D / 4)) * 4;
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r < nvalid && r >= lo_row) {
-            if (dtype == LLA_F32) x = load4(static_cast<const float*>(src) + (row0 + r) * D + c);
-            else x = load4(static_cast<const __nv_bfloat16*>(src) + (row0 + r) * D + c);
-        }
-        uint2 h, l;
-        split_pack(x.x, x.y, h.x, l.x);
-        split_pack(x.z, x.w, h.y, l.y);
-        *reinterpret_cast<uint2*>(hi + r * MM_LDB + c) = h;
-        *reinterpret_cast<uint2*>(lo + r * MM_LDB + c) = l;
-    }
-}
-
-template <int D>
-__global__ void __launch_bounds__(MmCfg<D>::THREADS, D == 64 ? 2 : 1)
-bwd_pairs_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-                     const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
-                     const float* __restrict__ yvec, const float* __restrict__ tvec, const float* __restrict__ rowsc,
-                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int first, float scale, int H, int kv_group) {
-    constexpr int LDB = MmCfg<D>::LDB, MM_TILE = MmCfg<D>::TILE, MM_THREADS = MmCfg<D>::THREADS, KS = MmCfg<D>::KS;
-    extern __shared__ __align__(16) unsigned char mm_smem[];
-    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(mm_smem);
-    __nv_bfloat16* Vs = Ks + MM_TILE;
-    __nv_bfloat16* Qs = Vs + MM_TILE;
-    __nv_bfloat16* Gh = Qs + MM_TILE;
-    __nv_bfloat16* Gl = Gh + MM_TILE;
-    __nv_bfloat16* Yh = Gl + MM_TILE;
-    __nv_bfloat16* Yl = Yh + MM_TILE;
-    __nv_bfloat16* Th = Yl + MM_TILE;
-    __nv_bfloat16* Tl = Th + MM_TILE;
-    __nv_bfloat16* DSh = Tl + MM_TILE;      // [key][query]
-    __nv_bfloat16* DSl = DSh + MM_TILE;
-    float* rs = reinterpret_cast<float*>(DSl + MM_TILE);   // [6][64]: m, 1/omega, gbar, kappa, kbar.y, kbar.t
-    const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
-    const int warp = (tid >> 5) & 3;      // key group (16 keys); query group in the dQ product
-    const int cg = tid >> 7;              // column group (64 output columns)
-    const int bh = blockIdx.x;
-    const int j0 = blockIdx.y * 64;
-    const size_t base = (size_t)bh * n;
-    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
-    mm_load_bf16<D>(Ks, k, kvbase + j0, min(64, n - j0));
-    mm_load_bf16<D>(Vs, v, kvbase + j0, min(64, n - j0));
-    // ldmatrix lane offsets: (rows +8 by bit 3, columns +8 by bit 4) and (columns +8 by bit 3, rows +8 by bit 4)
-    const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
-    const int offA = (l7 + 8 * b3) * LDB + 8 * b4;     // A operand, or B^T-stored operand read with .trans
-    const int offB = (l7 + 8 * b4) * LDB + 8 * b3;     // B operand stored [n][k], or A^T-stored operand read with .trans
-    const int kr0 = 16 * warp;
-    float adk[8][4] = {}, adv[8][4] = {};
-    const int it0 = max(j0, first) / 64, it1 = (n + 63) / 64;
-    for (int it = it0; it < it1; ++it) {
-        const int i0 = it * 64;
-        const int nrow = min(64, n - i0);
-        __syncthreads();
-        mm_load_bf16<D>(Qs, q, base + i0, nrow);
-        mm_load_split<D>(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
-        mm_load_split<D>(Yh, Yl, yvec, LLA_F32, base + i0, nrow, first - i0);
-        mm_load_split<D>(Th, Tl, tvec, LLA_F32, base + i0, nrow, first - i0);
-        for (int idx = tid; idx < 6 * 64; idx += MM_THREADS) {
-            const int w = idx >> 6, r = idx & 63, gi = i0 + r;
-            rs[idx] = (gi < n && gi >= first) ? rowsc[(base + gi) * BW_ROWSC + w] : 0.f;
-        }
-        __syncthreads();
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-            const int ih = 32 * half;
-            float sT[4][4] = {}, eT[4][4] = {}, fT[4][4] = {}, gT[4][4] = {};
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                uint32_t ak[4], av[4];
-                ldsm4(ak, Ks + kr0 * LDB + 16 * ks + offA);
-                ldsm4(av, Vs + kr0 * LDB + 16 * ks + offA);
-#pragma unroll
-                for (int nbp = 0; nbp < 2; ++nbp) {
-                    const int o = (ih + 16 * nbp) * LDB + 16 * ks + offB;
-                    uint32_t b[4];
-                    ldsm4(b, Qs + o);
-                    mma_bf16(sT[2 * nbp], ak, b[0], b[1]);
-                    mma_bf16(sT[2 * nbp + 1], ak, b[2], b[3]);
-                    ldsm4(b, Yh + o);
-                    mma_bf16(eT[2 * nbp], ak, b[0], b[1]);
-                    mma_bf16(eT[2 * nbp + 1], ak, b[2], b[3]);
-                    ldsm4(b, Yl + o);
-                    mma_bf16(eT[2 * nbp], ak, b[0], b[1]);
-                    mma_bf16(eT[2 * nbp + 1], ak, b[2], b[3]);
-                    ldsm4(b, Th + o);
-                    mma_bf16(fT[2 * nbp], ak, b[0], b[1]);
-                    mma_bf16(fT[2 * nbp + 1], ak, b[2], b[3]);
-                    ldsm4(b, Tl + o);
-                    mma_bf16(fT[2 * nbp], ak, b[0], b[1]);
-                    mma_bf16(fT[2 * nbp + 1], ak, b[2], b[3]);
-                    ldsm4(b, Gh + o);
-                    mma_bf16(gT[2 * nbp], av, b[0], b[1]);
-                    mma_bf16(gT[2 * nbp + 1], av, b[2], b[3]);
-                    ldsm4(b, Gl + o);
-                    mma_bf16(gT[2 * nbp], av, b[0], b[1]);
-                    mma_bf16(gT[2 * nbp + 1], av, b[2], b[3]);
-                }
-            }
-            // pair coefficients in place: sT <- a, eT <- scale dL/ds, fT <- p (f - gamma + gbar)
-#pragma unroll
-            for (int nb = 0; nb < 4; ++nb) {
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    const int il = ih + 8 * nb + 2 * t4 + (x & 1), gi = i0 + il;
-                    const int gj = j0 + kr0 + g + 8 * (x >> 1);
-                    const float iom = rs[64 + il];
-                    const float p = (iom > 0.f && gj <= gi) ? __expf(fmaf(scale, sT[nb][x], -rs[il])) * iom : 0.f;
-                    const float gbar = rs[128 + il], kappa = rs[192 + il];
-                    const float ev = eT[nb][x] - rs[256 + il], fv = fT[nb][x] - rs[320 + il], gam = gT[nb][x];
-                    sT[nb][x] = p * (1.f - ev);
-                    eT[nb][x] = scale * p * (gam * (1.f - ev) + (gbar + fv) * ev - fv - kappa);
-                    fT[nb][x] = p * (fv - gam + gbar);
-                }
-            }
-#pragma unroll
-            for (int ks2 = 0; ks2 < 2; ++ks2) {
-                // A fragments (rows = this warp's keys, k = 16 queries) of a, -a, ds, p1 as hi and lo
-                uint32_t ah[4], al[4], nh[4], nl[4], dh[4], dl[4], ph[4], pl[4];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int nb = 2 * ks2 + (r >> 1), x = 2 * (r & 1);
-                    split_pack(sT[nb][x], sT[nb][x + 1], ah[r], al[r]);
-                    nh[r] = ah[r] ^ 0x80008000u;
-                    nl[r] = al[r] ^ 0x80008000u;
-                    split_pack(eT[nb][x], eT[nb][x + 1], dh[r], dl[r]);
-                    split_pack(fT[nb][x], fT[nb][x + 1], ph[r], pl[r]);
-                    const int row = kr0 + g + 8 * (r & 1), col = ih + 8 * nb + 2 * t4;
-                    if (cg == 0) {
-                        *reinterpret_cast<uint32_t*>(DSh + row * LDB + col) = dh[r];
-                        *reinterpret_cast<uint32_t*>(DSl + row * LDB + col) = dl[r];
-                    }
-                }
-#pragma unroll
-                for (int ncp = 0; ncp < 4; ++ncp) {
-                    const int o = (ih + 16 * ks2) * LDB + 64 * cg + 16 * ncp + offA;
-                    uint32_t b[4], c[4];
-                    ldsm4t(b, Gh + o);
-                    ldsm4t(c, Gl + o);
-                    mma_bf16(adv[2 * ncp], ah, b[0], b[1]);  mma_bf16(adv[2 * ncp + 1], ah, b[2], b[3]);
-                    mma_bf16(adv[2 * ncp], al, b[0], b[1]);  mma_bf16(adv[2 * ncp + 1], al, b[2], b[3]);
-                    mma_bf16(adv[2 * ncp], ah, c[0], c[1]);  mma_bf16(adv[2 * ncp + 1], ah, c[2], c[3]);
-                    ldsm4t(b, Qs + o);
-                    mma_bf16(adk[2 * ncp], dh, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], dh, b[2], b[3]);
-                    mma_bf16(adk[2 * ncp], dl, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], dl, b[2], b[3]);
-                    ldsm4t(b, Yh + o);
-                    ldsm4t(c, Yl + o);
-                    mma_bf16(adk[2 * ncp], ph, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], ph, b[2], b[3]);
-                    mma_bf16(adk[2 * ncp], pl, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], pl, b[2], b[3]);
-                    mma_bf16(adk[2 * ncp], ph, c[0], c[1]);  mma_bf16(adk[2 * ncp + 1], ph, c[2], c[3]);
-                    ldsm4t(b, Th + o);
-                    ldsm4t(c, Tl + o);
-                    mma_bf16(adk[2 * ncp], nh, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], nh, b[2], b[3]);
-                    mma_bf16(adk[2 * ncp], nl, b[0], b[1]);  mma_bf16(adk[2 * ncp + 1], nl, b[2], b[3]);
-                    mma_bf16(adk[2 * ncp], nh, c[0], c[1]);  mma_bf16(adk[2 * ncp + 1], nh, c[2], c[3]);
-                }
-            }
-        }
-        __syncthreads();
-        // dQ rows 16 warp .. +15 of the tile: sum over the block's 64 keys of (scale dL/ds) k_j
-        float adq[8][4] = {};
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-            uint32_t ah[4], al[4];
-            ldsm4t(ah, DSh + 16 * ks * LDB + 16 * warp + offB);
-            ldsm4t(al, DSl + 16 * ks * LDB + 16 * warp + offB);
-#pragma unroll
-            for (int ncp = 0; ncp < 4; ++ncp) {
-                uint32_t b[4];
-                ldsm4t(b, Ks + 16 * ks * LDB + 64 * cg + 16 * ncp + offA);
-                mma_bf16(adq[2 * ncp], ah, b[0], b[1]);  mma_bf16(adq[2 * ncp + 1], ah, b[2], b[3]);
-                mma_bf16(adq[2 * ncp], al, b[0], b[1]);  mma_bf16(adq[2 * ncp + 1], al, b[2], b[3]);
-            }
-        }
-#pragma unroll
-        for (int nb = 0; nb < 8; ++nb)
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int gi = i0 + 16 * warp + g + 8 * (x >> 1);
-                if (gi < n && gi >= first) atomicAdd(dq + (base + gi) * D + 64 * cg + 8 * nb + 2 * t4 + (x & 1), adq[nb][x]);
-            }
-    }
-#pragma unroll
-    for (int nb = 0; nb < 8; ++nb)
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-            const int gj = j0 + kr0 + g + 8 * (x >> 1);
-            if (gj >= n) continue;
-            const size_t e = (kvbase + gj) * D + 64 * cg + 8 * nb + 2 * t4 + (x & 1);
-            atomicAdd(dk + e, adk[nb][x]);
-            atomicAdd(dv + e, adv[nb][x]);
-        }
-}
-
-// The moments kernel on the tensor cores (d = 64): a warp owns 16 of the tile's 64 query rows; S = Q K^T
-// and Gamma = G V^T accumulate in registers, p and p gamma are packed straight into A fragments (hi + lo)
-// and multiply the key tile again for kbar and sum_j p gamma k.
-template <int D>
-__global__ void __launch_bounds__(MmCfg<D>::THREADS, D == 64 ? 2 : 1)
-bwd_moments_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-                       const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
-                       const float* __restrict__ stats, float* __restrict__ kbar, float* __restrict__ hvec,
-                       float* __restrict__ rowsc, int n, int first, float scale, int H, int kv_group) {
-    constexpr int LDB = MmCfg<D>::LDB, MM_TILE = MmCfg<D>::TILE, KS = MmCfg<D>::KS;
-    extern __shared__ __align__(16) unsigned char mm_smem[];
-    __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(mm_smem);
-    __nv_bfloat16* Gh = Qs + MM_TILE;
-    __nv_bfloat16* Gl = Gh + MM_TILE;
-    __nv_bfloat16* Ks = Gl + MM_TILE;
-    __nv_bfloat16* Vs = Ks + MM_TILE;
-    const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
-    const int warp = (tid >> 5) & 3;      // query group (16 rows)
-    const int cg = tid >> 7;              // column group (64 output columns)
-    const int tile = gridDim.y - 1 - blockIdx.y;
-    const int bh = blockIdx.x;
-    const int i0 = tile * 64;
-    if (i0 + 64 <= first) return;
-    const size_t base = (size_t)bh * n;
-    const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
-    const int nrow = min(64, n - i0);
-    mm_load_bf16<D>(Qs, q, base + i0, nrow);
-    mm_load_split<D>(Gh, Gl, dout, dout_dtype, base + i0, nrow, 0);
-    const int l7 = lane & 7, b3 = (lane >> 3) & 1, b4 = lane >> 4;
-    const int offA = (l7 + 8 * b3) * LDB + 8 * b4;
-    const int offB = (l7 + 8 * b4) * LDB + 8 * b3;
-    const int r0 = 16 * warp;
-    float mrow[2], iom[2], gb[2] = {0.f, 0.f};
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int gi = i0 + r0 + g + 8 * h;
-        const bool okr = gi < n && gi >= first;
-        mrow[h] = okr ? stats[(base + gi) * 3 + 0] : 0.f;
-        iom[h] = okr ? 1.f / stats[(base + gi) * 3 + 1] : 0.f;
-    }
-    float akb[8][4] = {}, ah[8][4] = {};
-    const int jt_end = (min(n, i0 + 64) + 63) / 64;
-    for (int jt = 0; jt < jt_end; ++jt) {
-        const int j0 = jt * 64;
-        __syncthreads();
-        mm_load_bf16<D>(Ks, k, kvbase + j0, min(64, n - j0));
-        mm_load_bf16<D>(Vs, v, kvbase + j0, min(64, n - j0));
-        __syncthreads();
-        float s[8][4] = {}, gm[8][4] = {};
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            uint32_t aq[4], agh[4], agl[4];
-            ldsm4(aq, Qs + r0 * LDB + 16 * ks + offA);
-            ldsm4(agh, Gh + r0 * LDB + 16 * ks + offA);
-            ldsm4(agl, Gl + r0 * LDB + 16 * ks + offA);
-#pragma unroll
-            for (int nbp = 0; nbp < 4; ++nbp) {
-                uint32_t b[4];
-                ldsm4(b, Ks + 16 * nbp * LDB + 16 * ks + offB);
-                mma_bf16(s[2 * nbp], aq, b[0], b[1]);
-                mma_bf16(s[2 * nbp + 1], aq, b[2], b[3]);
-                ldsm4(b, Vs + 16 * nbp * LDB + 16 * ks + offB);
-                mma_bf16(gm[2 * nbp], agh, b[0], b[1]);
-                mma_bf16(gm[2 * nbp + 1], agh, b[2], b[3]);
-                mma_bf16(gm[2 * nbp], agl, b[0], b[1]);
-                mma_bf16(gm[2 * nbp + 1], agl, b[2], b[3]);
-            }
-        }
-        // s <- p, gm <- p gamma
-#pragma unroll
-        for (int nb = 0; nb < 8; ++nb)
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int h = x >> 1, gi = i0 + r0 + g + 8 * h, gj = j0 + 8 * nb + 2 * t4 + (x & 1);
-                const float p = (gj <= gi && iom[h] > 0.f) ? __expf(fmaf(scale, s[nb][x], -mrow[h])) * iom[h] : 0.f;
-                s[nb][x] = p;
-                gm[nb][x] *= p;
-                gb[h] += gm[nb][x];
-            }
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-            uint32_t ph[4], pl[4], gh[4], gl[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const int nb = 2 * ks + (r >> 1), x = 2 * (r & 1);
-                split_pack(s[nb][x], s[nb][x + 1], ph[r], pl[r]);
-                split_pack(gm[nb][x], gm[nb][x + 1], gh[r], gl[r]);
-            }
-#pragma unroll
-            for (int ncp = 0; ncp < 4; ++ncp) {
-                uint32_t b[4];
-                ldsm4t(b, Ks + 16 * ks * LDB + 64 * cg + 16 * ncp + offA);
-                mma_bf16(akb[2 * ncp], ph, b[0], b[1]);  mma_bf16(akb[2 * ncp + 1], ph, b[2], b[3]);
-                mma_bf16(akb[2 * ncp], pl, b[0], b[1]);  mma_bf16(akb[2 * ncp + 1], pl, b[2], b[3]);
-                mma_bf16(ah[2 * ncp], gh, b[0], b[1]);   mma_bf16(ah[2 * ncp + 1], gh, b[2], b[3]);
-                mma_bf16(ah[2 * ncp], gl, b[0], b[1]);   mma_bf16(ah[2 * ncp + 1], gl, b[2], b[3]);
-            }
-        }
-    }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        gb[h] += __shfl_xor_sync(0xffffffffu, gb[h], 1);
-        gb[h] += __shfl_xor_sync(0xffffffffu, gb[h], 2);
-        const int gi = i0 + r0 + g + 8 * h;
-        if (gi >= n || gi < first) continue;
-        if (t4 == 0 && cg == 0) rowsc[(base + gi) * BW_ROWSC + 2] = gb[h];
-#pragma unroll
-        for (int nb = 0; nb < 8; ++nb) {
-            const float kb0 = akb[nb][2 * h], kb1 = akb[nb][2 * h + 1];
-            const size_t e = (base + gi) * D + 64 * cg + 8 * nb + 2 * t4;
-            *reinterpret_cast<float2*>(kbar + e) = make_float2(kb0, kb1);
-            *reinterpret_cast<float2*>(hvec + e) = make_float2(ah[nb][2 * h] - gb[h] * kb0, ah[nb][2 * h + 1] - gb[h] * kb1);
         }
     }
 }
@@ -933,11 +612,12 @@ size_t head_smem_bytes(int lcap) {
     return sizeof(double) * ((size_t)D * (D + 1) + 7 * D + 4 * lcap) + sizeof(__nv_bfloat16) * (size_t)lcap * D;
 }
 
-// workspace: kbar, h, t, y as [rows][D] fp32, then the scalar records
-size_t ws_floats(long long rows, int d, long long heads) {
-    (void)heads;
-    return (size_t)rows * (4 * (size_t)d + BW_ROWSC);
-}
+// workspace: kbar, h, t, y as [rows][D] fp32, the scalar records, then the tensor-core kernels' bf16 operand arrays
+// (y and -t as hi and lo; the upstream gradient's hi and lo, used when it comes in fp32)
+size_t ws_floats(long long rows, int d) { return (size_t)rows * (4 * (size_t)d + BW_ROWSC); }
+size_t ws_fp32_bytes(long long rows, int d) { return (ws_floats(rows, d) * sizeof(float) + 255) & ~(size_t)255; }
+size_t ws_pair_bytes(long long rows, int d) { return ((size_t)rows * d * 2 + 255) & ~(size_t)255; }      // one bf16 array
+size_t ws_own_bytes(long long rows, int d) { return ws_fp32_bytes(rows, d) + 6 * ws_pair_bytes(rows, d); }
 
 template <int D>
 int launch_t(const BackwardArgs& a) {
@@ -947,20 +627,21 @@ int launch_t(const BackwardArgs& a) {
     const int first = max(0, min(a.n, a.head_rows - 1));      // rows [0, first) are solved directly
     const int kvg = a.kv_group > 0 ? a.kv_group : 1;
     const long long kvrows = rows / kvg;                       // rows of k, v, dk, dv
-    if (a.workspace_bytes < ws_floats(rows, D, BH) * sizeof(float) || !a.workspace) return LLA_ERR_WORKSPACE;
+    if (a.workspace_bytes < ws_own_bytes(rows, D) || !a.workspace) return LLA_ERR_WORKSPACE;
     if (first > 2 * D) return LLA_ERR_UNSUPPORTED;
     float* kbar = static_cast<float*>(a.workspace);
     float* hvec = kbar + rows * D;
     float* tvec = hvec + rows * D;
     float* yvec = tvec + rows * D;
     float* rowsc = yvec + rows * D;
+    char* pairs = static_cast<char*>(a.workspace) + ws_fp32_bytes(rows, D);
+    const size_t pb = ws_pair_bytes(rows, D);
+    const bool tensor = !a.cuda_core_pairs;
     const auto* q = static_cast<const __nv_bfloat16*>(a.q);
     const auto* k = static_cast<const __nv_bfloat16*>(a.k);
     const auto* v = static_cast<const __nv_bfloat16*>(a.v);
     const size_t head_smem = head_smem_bytes<D>(first);
     if (head_smem > 227u * 1024u) return LLA_ERR_UNSUPPORTED;
-    LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::MOMENTS_SMEM));
-    LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::PAIRS_SMEM));
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_head_rows_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem));
     LLA_CUDA_TRY(cudaMemsetAsync(a.dk, 0, sizeof(float) * kvrows * D, a.stream));
     LLA_CUDA_TRY(cudaMemsetAsync(a.dv, 0, sizeof(float) * kvrows * D, a.stream));
@@ -979,18 +660,35 @@ int launch_t(const BackwardArgs& a) {
         if (forked) LLA_CUDA_TRY(cudaEventRecord(a.join, hs));
     }
     if (first < a.n) {
-        const dim3 gm(BH, (a.n + C::BI - 1) / C::BI);
-        if (!a.cuda_core_pairs) {
-            using M = MmCfg<D>;
-            const dim3 gm(BH, (a.n + 63) / 64);
-            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::MOMENTS_SMEM));
-            bwd_moments_mma_kernel<D><<<gm, M::THREADS, M::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
-                                                                               rowsc, a.n, first, a.scale, a.H, kvg);
+        BwdTensorArgs t = {};
+        Pairs16 p16 = {};
+        if (tensor) {
+            t.q = a.q; t.k = a.k; t.v = a.v;
+            t.yh = pairs; t.yl = pairs + pb; t.tnh = pairs + 2 * pb; t.tnl = pairs + 3 * pb;
+            p16.yh = reinterpret_cast<uint32_t*>(pairs); p16.yl = reinterpret_cast<uint32_t*>(pairs + pb);
+            p16.tnh = reinterpret_cast<uint32_t*>(pairs + 2 * pb); p16.tnl = reinterpret_cast<uint32_t*>(pairs + 3 * pb);
+            if (a.dout_dtype == LLA_F32) {
+                t.gh = pairs + 4 * pb; t.gl = pairs + 5 * pb;
+                const size_t quads = (size_t)rows * D / 4;
+                bwd_split_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, a.stream>>>(
+                    static_cast<const float*>(a.dout), reinterpret_cast<uint2*>(pairs + 4 * pb), reinterpret_cast<uint2*>(pairs + 5 * pb), quads);
+                LLA_CUDA_TRY(cudaGetLastError());
+            } else {
+                t.gh = a.dout; t.gl = nullptr;
+            }
+            t.rowsc = rowsc; t.stats = a.stats; t.yvec = yvec; t.tvec = tvec;
+            t.kbar = kbar; t.hvec = hvec; t.dq = a.dq; t.dk = a.dk; t.dv = a.dv;
+            t.B = a.B; t.H = a.H; t.n = a.n; t.d = D; t.first = first; t.kv_group = kvg;
+            t.scale = a.scale; t.status = a.status; t.stream = a.stream;
+            const int rc = launch_backward_tensor(t, 0);
+            if (rc != LLA_OK) return rc;
         } else {
+            const dim3 gm(BH, (a.n + C::BI - 1) / C::BI);
+            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::MOMENTS_SMEM));
             bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
                                                                               rowsc, a.n, first, a.scale, a.H, kvg);
+            LLA_CUDA_TRY(cudaGetLastError());
         }
-        LLA_CUDA_TRY(cudaGetLastError());
         // C_i t_i = h_i for the iterative rows: the forward's tensor-core CG with h as right-hand side
         ForwardArgs f = {};
         f.q = a.q; f.k = a.k; f.v = a.v; f.out = nullptr;
@@ -1002,9 +700,9 @@ int launch_t(const BackwardArgs& a) {
         f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg;
         f.rhs = hvec; f.sol = tvec;
         f.set_contiguous();
-        // what the workspace holds beyond this pass's own vectors serves the solve (the fp16 copy of k; for
+        // what the workspace holds beyond this pass's own arrays serves the solve (the fp16 copy of k; for
         // d = 128 the row-state slots), so that the backward pass allocates nothing
-        const size_t own = (ws_floats(rows, D, BH) * sizeof(float) + 255) & ~(size_t)255;
+        const size_t own = ws_own_bytes(rows, D);
         if (a.workspace_bytes > own) {
             f.workspace = static_cast<char*>(a.workspace) + own;
             f.workspace_bytes = a.workspace_bytes - own;
@@ -1014,21 +712,20 @@ int launch_t(const BackwardArgs& a) {
         const int rc = launch_forward_tensor(f);
         if (rc != LLA_OK) return rc;
         bwd_rowprep_kernel<D><<<(unsigned)((rows + 7) / 8), BW_THREADS, 0, a.stream>>>(
-            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, a.n, first, rows, a.dlambda);
+            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, a.n, first, rows, a.dlambda, p16);
         LLA_CUDA_TRY(cudaGetLastError());
-    }
-    {
-        const dim3 gp(BH, (a.n + BW_BJ - 1) / BW_BJ);
-        if (!a.cuda_core_pairs) {
-            using M = MmCfg<D>;
-            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::PAIRS_SMEM));
-            bwd_pairs_mma_kernel<D><<<gp, M::THREADS, M::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc, a.dq,
-                                                                     a.dk, a.dv, a.n, first, a.scale, a.H, kvg);
+        if (tensor) {
+            int rc2 = launch_backward_tensor(t, 1);
+            if (rc2 != LLA_OK) return rc2;
+            rc2 = launch_backward_tensor(t, 2);
+            if (rc2 != LLA_OK) return rc2;
         } else {
+            const dim3 gp(BH, (a.n + BW_BJ - 1) / BW_BJ);
+            LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_pairs_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::PAIRS_SMEM));
             bwd_pairs_kernel<D><<<gp, BW_THREADS, C::PAIRS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, yvec, tvec, rowsc,
                                                                           a.dq, a.dk, a.dv, a.n, first, a.scale, a.H, kvg);
+            LLA_CUDA_TRY(cudaGetLastError());
         }
-        LLA_CUDA_TRY(cudaGetLastError());
     }
     if (forked) LLA_CUDA_TRY(cudaStreamWaitEvent(a.stream, a.join, 0));
     return LLA_OK;
@@ -1037,8 +734,7 @@ int launch_t(const BackwardArgs& a) {
 }  // namespace
 
 size_t backward_workspace_bytes(int B, int H, int n, int d) {
-    const size_t own = (ws_floats((long long)B * H * n, d, (long long)B * H) * sizeof(float) + 255) & ~(size_t)255;
-    return own + forward_tensor_workspace_bytes(B, H, n, d);
+    return ws_own_bytes((long long)B * H * n, d) + forward_tensor_workspace_bytes(B, H, n, d);
 }
 
 int launch_backward(const BackwardArgs& a) {

@@ -1,0 +1,662 @@
+// Backward pass of causal local linear attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 inputs,
+// d = dv in {64, 128}: the pair sums of the paper's backward appendix in the centred form that lla_backward.cu
+// derives (same symbols).  Three kernels share one skeleton -- TMA brings 128B-swizzled bf16 tiles, one warp issues
+// the MMAs, eight warps (two threads per TMEM lane) turn score tiles into coefficient tiles:
+//
+//   bwd_qtile_tc_kernel<D, 0>   per 128-row query tile, over its key blocks of 64:
+//                                 S = Q K^T, Gamma = G V^T  ->  p, p gamma  ->  kbar += P K, sum_j p gamma k += (P Gamma) K
+//   bwd_qtile_tc_kernel<D, 1>   the same loop with S, E = Y K^T, F = T K^T, Gamma  ->  scale dL/ds  ->  dQ += DS K
+//                                 (a query tile owns its rows of dQ: plain stores, the same bits on every run)
+//   bwd_ktile_tc_kernel<D>      per 128-key tile, over the later query rows in steps of 64, everything transposed
+//                               (keys on the TMEM lanes):  S^T = K Q^T, E^T = K Y^T, F^T = K T^T, Gamma^T = V G^T  ->
+//                               a^T, (scale dL/ds)^T, (p (f - gamma + gbar))^T  ->  dV += A^T G,  dK += DS^T Q + P1^T Y - A^T T
+//
+// Every product of a score tile is an SS MMA of the forward kernel's shape (128 x 64 x d, both operands K-major);
+// every product of a coefficient tile takes the coefficients from TMEM, where the compute threads leave them in
+// the columns the scores came from, and the other operand MN-major from the tile TMA delivered.  The fp32
+// operands (y, t, g and the coefficient tiles) enter as bf16 pairs hi + lo and a product keeps the three leading
+// terms, which gives fp32-like accuracy; q, k, v are exact.  y, -t and g come as bf16 arrays written by the row
+// preparation kernel (-t, so that "- A^T T" is an accumulation like the others).  In the dQ kernel y sits in TMEM
+// (the tile's five other stationary operands fill the shared memory at d = 128).
+//
+// Score tiles are single-buffered: 4 x 64 columns plus the accumulators take all 512 TMEM columns at d = 128.
+// All waits are bounded; a wait that expires sets LLA_STATUS_TIMEOUT and the block leaves through the common exit.
+#include "lla_sm100.cuh"
+
+namespace lla {
+namespace {
+
+using namespace sm100;
+
+constexpr int BT_COMPUTE = 256;       // compute threads (warps 0..7)
+constexpr int BT_THREADS = 320;       // + TMA warp (8) + MMA warp (9)
+constexpr int BT_TMEM_COLS = 512;
+constexpr float BT_LOG2E = 1.4426950408889634f;
+
+constexpr uint32_t BT_IDESC_SS = make_idesc(128, 64, 0, 0);       // score tiles: [128 x 64], both operands K-major
+
+struct BtParams {
+    int n, first, H, kv_group;
+    int has_glo;          // the upstream gradient has a lo half (fp32 dout)
+    float scale;
+    const float* stats;   // [rows][3] saved by the forward
+    const float* rowsc;   // [rows][8] per-row scalars (see bwd_rowprep_kernel)
+    const float* yvec;    // [rows][D] fp32
+    const float* tvec;    // [rows][D] fp32
+    float* rowsc_w;       // moments kernel: gbar goes to slot 2
+    float* kbar;
+    float* hvec;
+    float* dq;
+    float* dk;
+    float* dv;
+    int* status;
+    long long wait_clocks;
+};
+
+// ------------------------------------------------------------------------------------------------
+// dK, dV: one block per (head, 128-key tile)
+// ------------------------------------------------------------------------------------------------
+template <int D>
+struct KtCfg {
+    static constexpr int KSUB = D / 64;
+    static constexpr int T128 = KSUB * 16384;      // a 128-row operand tile
+    static constexpr int T64 = KSUB * 8192;        // a 64-row operand tile
+    static constexpr int NST = D == 64 ? 2 : 1;    // stages of the query-side ring
+    static constexpr int SM_K = 0, SM_V = T128, SM_ST = 2 * T128;
+    static constexpr int ST_Q = 0, ST_YH = T64, ST_YL = 2 * T64, ST_TH = 3 * T64, ST_TL = 4 * T64, ST_GH = 5 * T64, ST_GL = 6 * T64;
+    static constexpr int ST_RS = 7 * T64;          // 64 row records of 8 floats
+    static constexpr int STAGE = 7 * T64 + 2048;
+    static constexpr int SM_BAR = SM_ST + NST * STAGE;
+    static constexpr int SM_MISC = SM_BAR + 128;
+    static constexpr int SM_ALLOC = SM_MISC + 64 + 1024;
+    static constexpr uint32_t IDESC_TS = make_idesc(128, D, 0, 1);      // accumulators: A from TMEM, B MN-major, N = D
+    // TMEM columns
+    static constexpr int C_S = 0, C_E = 64, C_F = 128, C_G = 192, C_DK = 256, C_DV = 256 + D;
+};
+static_assert(KtCfg<64>::SM_ALLOC <= 227 * 1024 && KtCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
+enum { KB_KV = 0, KB_FULL = 1, KB_EMPTY = 3, KB_SFULL = 5, KB_PREADY = 6, KB_ACCFULL = 7, KB_EXIT = 8, KB_COUNT = 9 };
+
+template <int D>
+__global__ void __launch_bounds__(BT_THREADS, 1)
+bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                    const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmYh,
+                    const __grid_constant__ CUtensorMap tmYl, const __grid_constant__ CUtensorMap tmTh,
+                    const __grid_constant__ CUtensorMap tmTl, const __grid_constant__ CUtensorMap tmGh,
+                    const __grid_constant__ CUtensorMap tmGl, const __grid_constant__ CUtensorMap tmRS, const BtParams prm) {
+    using Cfg = KtCfg<D>;
+    constexpr int KSUB = Cfg::KSUB, NST = Cfg::NST, STAGE = Cfg::STAGE, T64 = Cfg::T64;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + Cfg::SM_BAR;
+    auto bar = [&](int i) { return bars + 8u * i; };
+    volatile int* misc = reinterpret_cast<volatile int*>(smem + Cfg::SM_MISC);     // [0] tmem base, [2] abort
+    volatile int* abort_flag = misc + 2;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.x;
+    const int kvu = kv_unit(bh, prm.H, prm.kv_group);
+    const int n = prm.n;
+    const int j0 = blockIdx.y * 128;          // key tile 0 sees the most query rows and starts first (heads fastest)
+    const int it0 = max(j0, prm.first) / 64, it1 = (n + 63) / 64;     // query steps of 64 rows
+    const int nstep = it1 - it0;
+    const long long wcap = prm.wait_clocks;
+    if (nstep <= 0) return;
+
+    if (tid == 0) {
+        mbar_init(bar(KB_KV), 1);
+        for (int s = 0; s < NST; ++s) {
+            mbar_init(bar(KB_FULL + s), 1);
+            mbar_init(bar(KB_EMPTY + s), 1);
+        }
+        mbar_init(bar(KB_SFULL), 1);
+        mbar_init(bar(KB_PREADY), BT_COMPUTE / 32);
+        mbar_init(bar(KB_ACCFULL), 1);
+        mbar_init(bar(KB_EXIT), 1);
+        misc[2] = 0;
+        fence_barrier_init();
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(sbase + Cfg::SM_MISC), "r"(BT_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)misc[0];
+
+    if (warp == 8) {
+        // ================================ TMA producer ================================
+        if (lane == 0) {
+            mbar_expect_tx(bar(KB_KV), 2 * Cfg::T128);
+            for (int sub = 0; sub < KSUB; ++sub) {
+                tma_load_3d(sbase + Cfg::SM_K + sub * 16384, &tmK, bar(KB_KV), 64 * sub, j0, kvu);
+                tma_load_3d(sbase + Cfg::SM_V + sub * 16384, &tmV, bar(KB_KV), 64 * sub, j0, kvu);
+            }
+            int issued = 0;
+            for (int g = 0; g < nstep; ++g) {
+                const int s = g % NST, i0 = 64 * (it0 + g);
+                if (!mbar_wait(bar(KB_EMPTY + s), ((g / NST) & 1) ^ 1, abort_flag, wcap)) break;
+                const uint32_t st = sbase + Cfg::SM_ST + s * STAGE, fb = bar(KB_FULL + s);
+                mbar_expect_tx(fb, (6 + (prm.has_glo ? 1 : 0)) * T64 + 2048);
+                for (int sub = 0; sub < KSUB; ++sub) {
+                    tma_load_3d(st + Cfg::ST_Q + sub * 8192, &tmQ, fb, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_YH + sub * 8192, &tmYh, fb, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_YL + sub * 8192, &tmYl, fb, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_TH + sub * 8192, &tmTh, fb, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_TL + sub * 8192, &tmTl, fb, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_GH + sub * 8192, &tmGh, fb, 64 * sub, i0, bh);
+                    if (prm.has_glo) tma_load_3d(st + Cfg::ST_GL + sub * 8192, &tmGl, fb, 64 * sub, i0, bh);
+                }
+                tma_load_3d(st + Cfg::ST_RS, &tmRS, fb, 0, i0, bh);
+                issued = g + 1;
+            }
+            if (*abort_flag) {      // an aborted block: what was issued must have landed before the block exits
+                (void)mbar_wait_landed(bar(KB_KV), 0, wcap);
+                for (int g = max(0, issued - NST); g < issued; ++g) (void)mbar_wait_landed(bar(KB_FULL + g % NST), (g / NST) & 1, wcap);
+            }
+        }
+    } else if (warp == 9) {
+        // ================================ MMA issuer ================================
+        const uint32_t el = elect_one();
+        const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
+        const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
+        bool ok = mbar_wait(bar(KB_KV), 0, abort_flag, wcap);
+        const uint64_t kdesc = make_desc(sb_u + Cfg::SM_K), vdesc = make_desc(sb_u + Cfg::SM_V);
+        for (int g = 0; g < nstep && ok; ++g) {
+            const int s = g % NST;
+            if (!mbar_wait(bar(KB_FULL + s), (g / NST) & 1, abort_flag, wcap)) break;
+            tc_fence_after();
+            const uint32_t st = sb_u + Cfg::SM_ST + s * STAGE;
+            auto score = [&](uint32_t col, uint64_t adesc, int off, uint32_t acc) {
+                const uint64_t bdesc = make_desc(st + off);
+#pragma unroll
+                for (int sub = 0; sub < KSUB; ++sub)
+                    mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
+            };
+            score(Cfg::C_S, kdesc, Cfg::ST_Q, 0);
+            score(Cfg::C_E, kdesc, Cfg::ST_YH, 0);
+            score(Cfg::C_E, kdesc, Cfg::ST_YL, 1);
+            score(Cfg::C_F, kdesc, Cfg::ST_TH, 0);
+            score(Cfg::C_F, kdesc, Cfg::ST_TL, 1);
+            score(Cfg::C_G, vdesc, Cfg::ST_GH, 0);
+            if (prm.has_glo) score(Cfg::C_G, vdesc, Cfg::ST_GL, 1);
+            tc_commit_el(el, bar(KB_SFULL));
+            if (!mbar_wait(bar(KB_PREADY), g & 1, abort_flag, wcap)) break;
+            tc_fence_after();
+            // coefficient tiles (hi + lo pairs) sit where the scores were: a^T in S, ds^T in E, p1^T in F
+            auto bd = [&](int off) { return make_desc(st + off, 8192); };
+            const uint32_t acc = g > 0;
+            mma_ts_hilo_k64(el, tm_u + Cfg::C_DV, tm_u + Cfg::C_S, bd(Cfg::ST_GH), Cfg::IDESC_TS, acc);
+            if (prm.has_glo) mma_ts_hi_k64(el, tm_u + Cfg::C_DV, tm_u + Cfg::C_S, bd(Cfg::ST_GL), Cfg::IDESC_TS, 1);
+            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_E, bd(Cfg::ST_Q), Cfg::IDESC_TS, acc);
+            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YH), Cfg::IDESC_TS, 1);
+            mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YL), Cfg::IDESC_TS, 1);
+            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TH), Cfg::IDESC_TS, 1);
+            mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TL), Cfg::IDESC_TS, 1);
+            tc_commit_el(el, bar(KB_EMPTY + s));
+            if (g == nstep - 1) tc_commit_el(el, bar(KB_ACCFULL));
+        }
+        if (*abort_flag) {      // an aborted block: the MMAs issued above must be done before TMEM and shared memory go
+            tc_commit_el(el, bar(KB_EXIT));
+            (void)mbar_wait_landed(bar(KB_EXIT), 0, wcap);
+        }
+    } else {
+        // ================================ compute warps ================================
+        const int quad = warp & 3, half = warp >> 2;
+        const int lrow = quad * 32 + lane;            // key inside the tile == TMEM lane
+        const int gj = j0 + lrow;
+        const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
+        const float c1 = prm.scale * BT_LOG2E, scale = prm.scale;
+        bool ok = true;
+        for (int g = 0; g < nstep; ++g) {
+            const int s = g % NST, i0 = 64 * (it0 + g);
+            if (!mbar_wait(bar(KB_FULL + s), (g / NST) & 1, abort_flag, wcap)) { ok = false; break; }      // the row records
+            if (!mbar_wait(bar(KB_SFULL), g & 1, abort_flag, wcap)) { ok = false; break; }
+            tc_fence_after();
+            const float4* rs = reinterpret_cast<const float4*>(smem + Cfg::SM_ST + s * STAGE + Cfg::ST_RS);
+#pragma unroll 1
+            for (int chunk = 0; chunk < 2; ++chunk) {
+                const int colbase = 32 * half + 16 * chunk;      // 16 query rows = one 16-element step of the products
+                uint32_t sv[16], ev[16], fv[16], gv[16];
+                tmem_ld16(tm_lane + Cfg::C_S + colbase, sv);
+                tmem_ld16(tm_lane + Cfg::C_E + colbase, ev);
+                tmem_ld16(tm_lane + Cfg::C_F + colbase, fv);
+                tmem_ld16(tm_lane + Cfg::C_G + colbase, gv);
+                tc_wait_ld();
+                uint32_t pa[16], pd[16], pp[16];
+#pragma unroll
+                for (int e2 = 0; e2 < 8; ++e2) {
+                    float a[2], ds[2], p1[2];
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        const int e = 2 * e2 + x, col = colbase + e, gi = i0 + col;
+                        const float4 r0 = rs[2 * col], r1 = rs[2 * col + 1];     // (m, 1/omega, gbar, kappa), (kbar.y, kbar.t, -m log2 e, -)
+                        const bool valid = gj <= gi && gi < n && r0.y > 0.f;
+                        const float p = valid ? ex2f(fmaf(__uint_as_float(sv[e]), c1, r1.z)) * r0.y : 0.f;
+                        const float evv = __uint_as_float(ev[e]) - r1.x;
+                        const float fvv = -__uint_as_float(fv[e]) - r1.y;      // the tile holds (-t) . k
+                        const float gam = __uint_as_float(gv[e]);
+                        const float ome = 1.f - evv;
+                        a[x] = valid ? p * ome : 0.f;
+                        ds[x] = valid ? scale * p * (gam * ome + (r0.z + fvv) * evv - fvv - r0.w) : 0.f;
+                        p1[x] = valid ? p * (fvv - gam + r0.z) : 0.f;
+                    }
+                    pa[e2] = split_bf16x2(a[0], a[1], pa[8 + e2]);
+                    pd[e2] = split_bf16x2(ds[0], ds[1], pd[8 + e2]);
+                    pp[e2] = split_bf16x2(p1[0], p1[1], pp[8 + e2]);
+                }
+                tmem_st16(tm_lane + Cfg::C_S + colbase, pa);
+                tmem_st16(tm_lane + Cfg::C_E + colbase, pd);
+                tmem_st16(tm_lane + Cfg::C_F + colbase, pp);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(KB_PREADY));
+        }
+        if (ok && mbar_wait(bar(KB_ACCFULL), 0, abort_flag, wcap)) {
+            tc_fence_after();
+            // (added, not stored: the directly-solved rows add their share from another stream, grouped heads theirs)
+            const size_t rowoff = ((size_t)kvu * n + gj) * D + half * (D / 2);
+#pragma unroll 1
+            for (int cb = 0; cb < D / 2; cb += 32) {
+                uint32_t v[32];
+                tmem_ld32(tm_lane + Cfg::C_DK + half * (D / 2) + cb, v);
+                tc_wait_ld();
+                if (gj < n)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) atomicAdd(prm.dk + rowoff + cb + e, __uint_as_float(v[e]));
+                tmem_ld32(tm_lane + Cfg::C_DV + half * (D / 2) + cb, v);
+                tc_wait_ld();
+                if (gj < n)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) atomicAdd(prm.dv + rowoff + cb + e, __uint_as_float(v[e]));
+            }
+        }
+    }
+    // ================================ common exit ================================
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BT_TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && *abort_flag && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Query-tile kernels: MODE 0 = moments (kbar, gbar, h), MODE 1 = dQ
+// ------------------------------------------------------------------------------------------------
+template <int D>
+struct QtCfg {
+    static constexpr int KSUB = D / 64;
+    static constexpr int T128 = KSUB * 16384, T64 = KSUB * 8192;
+    static constexpr int SM_Q = 0, SM_GH = T128, SM_GL = 2 * T128, SM_TH = 3 * T128, SM_TL = 4 * T128;
+    static constexpr int SM_KV = 5 * T128;         // stage 0: K block, V block.  A second stage: see stage_base()
+    static constexpr int STAGE = 2 * T64;
+    static constexpr int NST_FIXED = D == 64 ? 3 : 1;      // stages at SM_KV
+    static constexpr int SM_RED = SM_KV + NST_FIXED * STAGE;        // 2 x 128 floats
+    static constexpr int SM_BAR = SM_RED + 1024;
+    static constexpr int SM_MISC = SM_BAR + 128;
+    static constexpr int SM_ALLOC = SM_MISC + 64 + 1024;
+    static constexpr uint32_t IDESC_TS = make_idesc(128, D, 0, 1);
+    // TMEM columns.  MODE 1: S, E, F, Gamma, dQ, then y as bf16 pairs (hi D / 2 columns, lo D / 2 columns)
+    static constexpr int C_S = 0, C_E = 64, C_F = 128, C_G1 = 192, C_DQ = 256, C_Y = 384;
+    // MODE 0: S, Gamma, kbar, sum p gamma k
+    static constexpr int C_G0 = 64, C_KB = 128, C_H = 128 + D;
+};
+static_assert(QtCfg<64>::SM_ALLOC <= 227 * 1024 && QtCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
+enum { QB_QFULL = 0, QB_YREADY = 1, QB_FULL = 2, QB_EMPTY = 5, QB_SFULL = 8, QB_PREADY = 9, QB_ACCFULL = 10, QB_EXIT = 11, QB_COUNT = 12 };
+
+template <int D, int MODE>
+__global__ void __launch_bounds__(BT_THREADS, 1)
+bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmGh,
+                    const __grid_constant__ CUtensorMap tmGl, const __grid_constant__ CUtensorMap tmTh,
+                    const __grid_constant__ CUtensorMap tmTl, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const BtParams prm) {
+    using Cfg = QtCfg<D>;
+    constexpr int KSUB = Cfg::KSUB, STAGE = Cfg::STAGE, T64 = Cfg::T64, T128 = Cfg::T128;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + Cfg::SM_BAR;
+    auto bar = [&](int i) { return bars + 8u * i; };
+    volatile int* misc = reinterpret_cast<volatile int*>(smem + Cfg::SM_MISC);
+    volatile int* abort_flag = misc + 2;
+    float* red = reinterpret_cast<float*>(smem + Cfg::SM_RED);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.x;
+    const int kvu = kv_unit(bh, prm.H, prm.kv_group);
+    const int n = prm.n;
+    const int tile = gridDim.y - 1 - blockIdx.y;      // longest tiles first, heads fastest
+    const int i0 = tile * 128;
+    if (i0 + 128 <= prm.first) return;                // every row of the tile is solved directly
+    const int nblk = (min(n, i0 + 128) + 63) / 64;
+    const long long wcap = prm.wait_clocks;
+    // Stages of the K/V ring.  d = 128: the tiles that stay for the whole block leave room for one stage; where the
+    // upstream gradient has no lo half (bf16), that half's tile is a second one.  The moments kernel has no T tiles.
+    const int nst = D == 64 ? 3 : (MODE == 0 ? 3 : (prm.has_glo ? 1 : 2));
+    auto stage_base = [&](int s) -> uint32_t {
+        if (D == 64) return Cfg::SM_KV + s * STAGE;
+        if (MODE == 0) return s == 0 ? Cfg::SM_KV : (s == 1 ? Cfg::SM_TH : Cfg::SM_TL);
+        return s == 0 ? Cfg::SM_KV : Cfg::SM_GL;
+    };
+    static_assert(D == 64 || QtCfg<D>::STAGE == QtCfg<D>::T128, "a d = 128 stage takes the place of one stationary tile");
+
+    if (tid == 0) {
+        mbar_init(bar(QB_QFULL), 1);
+        mbar_init(bar(QB_YREADY), BT_COMPUTE / 32);
+        for (int s = 0; s < 3; ++s) {
+            mbar_init(bar(QB_FULL + s), 1);
+            mbar_init(bar(QB_EMPTY + s), 1);
+        }
+        mbar_init(bar(QB_SFULL), 1);
+        mbar_init(bar(QB_PREADY), BT_COMPUTE / 32);
+        mbar_init(bar(QB_ACCFULL), 1);
+        mbar_init(bar(QB_EXIT), 1);
+        misc[2] = 0;
+        fence_barrier_init();
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(sbase + Cfg::SM_MISC), "r"(BT_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)misc[0];
+
+    if (warp == 8) {
+        // ================================ TMA producer ================================
+        if (lane == 0) {
+            const int ntile = (MODE == 1 ? 4 : 2) + (prm.has_glo ? 1 : 0);
+            mbar_expect_tx(bar(QB_QFULL), ntile * T128);
+            for (int sub = 0; sub < KSUB; ++sub) {
+                tma_load_3d(sbase + Cfg::SM_Q + sub * 16384, &tmQ, bar(QB_QFULL), 64 * sub, i0, bh);
+                tma_load_3d(sbase + Cfg::SM_GH + sub * 16384, &tmGh, bar(QB_QFULL), 64 * sub, i0, bh);
+                if (prm.has_glo) tma_load_3d(sbase + Cfg::SM_GL + sub * 16384, &tmGl, bar(QB_QFULL), 64 * sub, i0, bh);
+                if (MODE == 1) {
+                    tma_load_3d(sbase + Cfg::SM_TH + sub * 16384, &tmTh, bar(QB_QFULL), 64 * sub, i0, bh);
+                    tma_load_3d(sbase + Cfg::SM_TL + sub * 16384, &tmTl, bar(QB_QFULL), 64 * sub, i0, bh);
+                }
+            }
+            int issued = 0;
+            for (int c = 0; c < nblk; ++c) {
+                const int s = c % nst;
+                if (!mbar_wait(bar(QB_EMPTY + s), ((c / nst) & 1) ^ 1, abort_flag, wcap)) break;
+                const uint32_t st = sbase + stage_base(s), fb = bar(QB_FULL + s);
+                mbar_expect_tx(fb, STAGE);
+                for (int sub = 0; sub < KSUB; ++sub) {
+                    tma_load_3d(st + sub * 8192, &tmK, fb, 64 * sub, 64 * c, kvu);
+                    tma_load_3d(st + T64 + sub * 8192, &tmV, fb, 64 * sub, 64 * c, kvu);
+                }
+                issued = c + 1;
+            }
+            if (*abort_flag) {
+                (void)mbar_wait_landed(bar(QB_QFULL), 0, wcap);
+                for (int c = max(0, issued - nst); c < issued; ++c) (void)mbar_wait_landed(bar(QB_FULL + c % nst), (c / nst) & 1, wcap);
+            }
+        }
+    } else if (warp == 9) {
+        // ================================ MMA issuer ================================
+        const uint32_t el = elect_one();
+        const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
+        const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
+        bool ok = mbar_wait(bar(QB_QFULL), 0, abort_flag, wcap);
+        if (MODE == 1) ok = ok && mbar_wait(bar(QB_YREADY), 0, abort_flag, wcap);
+        tc_fence_after();
+        for (int c = 0; c < nblk && ok; ++c) {
+            const int s = c % nst;
+            if (!mbar_wait(bar(QB_FULL + s), (c / nst) & 1, abort_flag, wcap)) break;
+            tc_fence_after();
+            const uint32_t st = sb_u + stage_base(s);
+            const uint64_t kdesc = make_desc(st), vdesc = make_desc(st + T64);
+            auto score = [&](uint32_t col, int aoff, uint64_t bdesc, uint32_t acc) {
+                const uint64_t adesc = make_desc(sb_u + aoff);
+#pragma unroll
+                for (int sub = 0; sub < KSUB; ++sub)
+                    mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
+            };
+            score(Cfg::C_S, Cfg::SM_Q, kdesc, 0);
+            if (MODE == 1) {
+                // E = Y K^T with y (hi, then lo) from TMEM: D / 16 steps of 8 columns each
+#pragma unroll
+                for (int part = 0; part < 2; ++part)
+#pragma unroll
+                    for (int sub = 0; sub < KSUB; ++sub)
+                        mma_ts_kmajor_k64(el, tm_u + Cfg::C_E, tm_u + Cfg::C_Y + part * (D / 2) + 32 * sub, kdesc + sub * (8192 >> 4),
+                                          BT_IDESC_SS, (part | sub) > 0);
+                score(Cfg::C_F, Cfg::SM_TH, kdesc, 0);
+                score(Cfg::C_F, Cfg::SM_TL, kdesc, 1);
+            }
+            const uint32_t cg = MODE == 1 ? Cfg::C_G1 : Cfg::C_G0;
+            score(cg, Cfg::SM_GH, vdesc, 0);
+            if (prm.has_glo) score(cg, Cfg::SM_GL, vdesc, 1);
+            tc_commit_el(el, bar(QB_SFULL));
+            if (!mbar_wait(bar(QB_PREADY), c & 1, abort_flag, wcap)) break;
+            tc_fence_after();
+            const uint64_t kmn = make_desc(st, 8192);       // the K block read MN-major, N = D
+            if (MODE == 1) {
+                mma_ts_hilo_k64(el, tm_u + Cfg::C_DQ, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
+            } else {
+                mma_ts_hilo_k64(el, tm_u + Cfg::C_KB, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
+                mma_ts_hilo_k64(el, tm_u + Cfg::C_H, tm_u + Cfg::C_G0, kmn, Cfg::IDESC_TS, c > 0);
+            }
+            tc_commit_el(el, bar(QB_EMPTY + s));
+            if (c == nblk - 1) tc_commit_el(el, bar(QB_ACCFULL));
+        }
+        if (*abort_flag) {
+            tc_commit_el(el, bar(QB_EXIT));
+            (void)mbar_wait_landed(bar(QB_EXIT), 0, wcap);
+        }
+    } else {
+        // ================================ compute warps ================================
+        const int quad = warp & 3, half = warp >> 2;
+        const int lrow = quad * 32 + lane;            // query row inside the tile == TMEM lane
+        const int gi = i0 + lrow;
+        const bool okr = gi < n && gi >= prm.first;
+        const size_t row = (size_t)bh * n + gi;
+        const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
+        const float c1 = prm.scale * BT_LOG2E, scale = prm.scale;
+        float nm2 = 0.f, iom = 0.f, gbar = 0.f, kappa = 0.f, ky = 0.f, kt = 0.f;
+        if (okr) {
+            if (MODE == 1) {
+                const float4 r0 = *reinterpret_cast<const float4*>(prm.rowsc + row * 8);
+                const float4 r1 = *reinterpret_cast<const float4*>(prm.rowsc + row * 8 + 4);
+                iom = r0.y; gbar = r0.z; kappa = r0.w; ky = r1.x; kt = r1.y; nm2 = r1.z;
+            } else {
+                nm2 = -prm.stats[row * 3 + 0] * BT_LOG2E;
+                iom = 1.f / prm.stats[row * 3 + 1];
+            }
+        }
+        if (MODE == 1) {
+            // this thread's half of y_i -> bf16 pairs in TMEM: 16-element steps of 8 columns, hi block then lo block
+            constexpr int NW = D / 4;      // packed words per half row and part
+            uint32_t yh[NW], yl[NW];
+#pragma unroll
+            for (int e = 0; e < NW; e += 2) {
+                float4 y4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (okr) y4 = *reinterpret_cast<const float4*>(prm.yvec + row * D + half * (D / 2) + 2 * e);
+                yh[e] = split_bf16x2(y4.x, y4.y, yl[e]);
+                yh[e + 1] = split_bf16x2(y4.z, y4.w, yl[e + 1]);
+            }
+            if constexpr (NW == 16) {
+                tmem_st16(tm_lane + Cfg::C_Y + half * NW, yh);
+                tmem_st16(tm_lane + Cfg::C_Y + D / 2 + half * NW, yl);
+            } else {
+                tmem_st32(tm_lane + Cfg::C_Y + half * NW, yh);
+                tmem_st32(tm_lane + Cfg::C_Y + D / 2 + half * NW, yl);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(QB_YREADY));
+        }
+        float gb = 0.f;
+        bool ok = true;
+        for (int c = 0; c < nblk; ++c) {
+            if (!mbar_wait(bar(QB_SFULL), c & 1, abort_flag, wcap)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int chunk = 0; chunk < 2; ++chunk) {
+                const int colbase = 32 * half + 16 * chunk;      // 16 keys = one 16-element step of the products
+                const int jlim = (okr ? gi + 1 : 0) - (64 * c + colbase);      // keys e < jlim of this chunk are visible
+                if (MODE == 1) {
+                    uint32_t sv[16], ev[16], fv[16], gv[16], pd[16];
+                    tmem_ld16(tm_lane + Cfg::C_S + colbase, sv);
+                    tmem_ld16(tm_lane + Cfg::C_E + colbase, ev);
+                    tmem_ld16(tm_lane + Cfg::C_F + colbase, fv);
+                    tmem_ld16(tm_lane + Cfg::C_G1 + colbase, gv);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int e2 = 0; e2 < 8; ++e2) {
+                        float ds[2];
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            const int e = 2 * e2 + x;
+                            const bool valid = e < jlim;
+                            const float p = valid ? ex2f(fmaf(__uint_as_float(sv[e]), c1, nm2)) * iom : 0.f;
+                            const float evv = __uint_as_float(ev[e]) - ky;
+                            const float fvv = -__uint_as_float(fv[e]) - kt;      // the tile holds (-t) . k
+                            const float gam = __uint_as_float(gv[e]);
+                            ds[x] = valid ? scale * p * (gam * (1.f - evv) + (gbar + fvv) * evv - fvv - kappa) : 0.f;
+                        }
+                        pd[e2] = split_bf16x2(ds[0], ds[1], pd[8 + e2]);
+                    }
+                    tmem_st16(tm_lane + Cfg::C_S + colbase, pd);
+                } else {
+                    uint32_t sv[16], gv[16], pp[16], pg[16];
+                    tmem_ld16(tm_lane + Cfg::C_S + colbase, sv);
+                    tmem_ld16(tm_lane + Cfg::C_G0 + colbase, gv);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int e2 = 0; e2 < 8; ++e2) {
+                        float p[2], q[2];
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            const int e = 2 * e2 + x;
+                            const bool valid = e < jlim;
+                            p[x] = valid ? ex2f(fmaf(__uint_as_float(sv[e]), c1, nm2)) * iom : 0.f;
+                            q[x] = valid ? p[x] * __uint_as_float(gv[e]) : 0.f;
+                            gb += q[x];
+                        }
+                        pp[e2] = split_bf16x2(p[0], p[1], pp[8 + e2]);
+                        pg[e2] = split_bf16x2(q[0], q[1], pg[8 + e2]);
+                    }
+                    tmem_st16(tm_lane + Cfg::C_S + colbase, pp);
+                    tmem_st16(tm_lane + Cfg::C_G0 + colbase, pg);
+                }
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(QB_PREADY));
+        }
+        if (MODE == 0) {      // gbar: the two halves of a row meet (all compute threads take part, aborted or not)
+            red[half * 128 + lrow] = gb;
+            named_sync_compute();
+            gb = red[lrow] + red[128 + lrow];
+        }
+        if (ok && mbar_wait(bar(QB_ACCFULL), 0, abort_flag, wcap)) {
+            tc_fence_after();
+            const size_t e0 = row * D + half * (D / 2);
+            if (MODE == 0 && okr && half == 0) prm.rowsc_w[row * 8 + 2] = gb;
+#pragma unroll 1
+            for (int cb = 0; cb < D / 2; cb += 32) {
+                uint32_t v[32];
+                if (MODE == 1) {
+                    tmem_ld32(tm_lane + Cfg::C_DQ + half * (D / 2) + cb, v);
+                    tc_wait_ld();
+                    if (okr)
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            const float4 t4 = *reinterpret_cast<const float4*>(prm.tvec + e0 + cb + e);
+                            *reinterpret_cast<float4*>(prm.dq + e0 + cb + e) =
+                                make_float4(__uint_as_float(v[e]) + t4.x, __uint_as_float(v[e + 1]) + t4.y,
+                                            __uint_as_float(v[e + 2]) + t4.z, __uint_as_float(v[e + 3]) + t4.w);
+                        }
+                } else {
+                    uint32_t h[32];
+                    tmem_ld32(tm_lane + Cfg::C_KB + half * (D / 2) + cb, v);
+                    tmem_ld32(tm_lane + Cfg::C_H + half * (D / 2) + cb, h);
+                    tc_wait_ld();
+                    if (okr)
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            const float k0 = __uint_as_float(v[e]), k1 = __uint_as_float(v[e + 1]), k2 = __uint_as_float(v[e + 2]),
+                                        k3 = __uint_as_float(v[e + 3]);
+                            *reinterpret_cast<float4*>(prm.kbar + e0 + cb + e) = make_float4(k0, k1, k2, k3);
+                            *reinterpret_cast<float4*>(prm.hvec + e0 + cb + e) =
+                                make_float4(__uint_as_float(h[e]) - gb * k0, __uint_as_float(h[e + 1]) - gb * k1,
+                                            __uint_as_float(h[e + 2]) - gb * k2, __uint_as_float(h[e + 3]) - gb * k3);
+                        }
+                }
+            }
+        }
+    }
+    // ================================ common exit ================================
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BT_TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && *abort_flag && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+}
+
+template <int D>
+int launch_t(const BwdTensorArgs& a, int which) {
+    const int BH = a.B * a.H, kvg = a.kv_group > 0 ? a.kv_group : 1, KVU = BH / kvg;
+    BtParams p = {};
+    p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.has_glo = a.gl != nullptr; p.scale = a.scale;
+    p.stats = a.stats; p.rowsc = a.rowsc; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
+    p.kbar = a.kbar; p.hvec = a.hvec; p.dq = a.dq; p.dk = a.dk; p.dv = a.dv; p.status = a.status;
+    p.wait_clocks = kWaitClocks;
+    const void* gl = a.gl ? a.gl : a.gh;        // a valid map either way; never loaded without a lo half
+    if (which == 2) {
+        using Cfg = KtCfg<D>;
+        CUtensorMap mK, mV, mQ, mYh, mYl, mTh, mTl, mGh, mGl, mRS;
+        bool ok = make_map_bf16(&mK, a.k, KVU, a.n, D, 128) && make_map_bf16(&mV, a.v, KVU, a.n, D, 128) &&
+                  make_map_bf16(&mQ, a.q, BH, a.n, D, 64) && make_map_bf16(&mYh, a.yh, BH, a.n, D, 64) &&
+                  make_map_bf16(&mYl, a.yl, BH, a.n, D, 64) && make_map_bf16(&mTh, a.tnh, BH, a.n, D, 64) &&
+                  make_map_bf16(&mTl, a.tnl, BH, a.n, D, 64) && make_map_bf16(&mGh, a.gh, BH, a.n, D, 64) &&
+                  make_map_bf16(&mGl, gl, BH, a.n, D, 64) && make_map_f32_rows(&mRS, a.rowsc, BH, a.n, 8, 64);
+        if (!ok) return LLA_ERR_CUDA;
+        LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_ktile_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
+        const dim3 grid(BH, (a.n + 127) / 128);
+        bwd_ktile_tc_kernel<D><<<grid, BT_THREADS, Cfg::SM_ALLOC, a.stream>>>(mK, mV, mQ, mYh, mYl, mTh, mTl, mGh, mGl, mRS, p);
+        LLA_CUDA_TRY(cudaGetLastError());
+        return LLA_OK;
+    }
+    using Cfg = QtCfg<D>;
+    CUtensorMap mQ, mGh, mGl, mTh, mTl, mK, mV;
+    const void* th = which == 1 ? a.tnh : a.q;      // the moments kernel loads no T tiles
+    const void* tl = which == 1 ? a.tnl : a.q;
+    bool ok = make_map_bf16(&mQ, a.q, BH, a.n, D, 128) && make_map_bf16(&mGh, a.gh, BH, a.n, D, 128) &&
+              make_map_bf16(&mGl, gl, BH, a.n, D, 128) && make_map_bf16(&mTh, th, BH, a.n, D, 128) &&
+              make_map_bf16(&mTl, tl, BH, a.n, D, 128) && make_map_bf16(&mK, a.k, KVU, a.n, D, 64) &&
+              make_map_bf16(&mV, a.v, KVU, a.n, D, 64);
+    if (!ok) return LLA_ERR_CUDA;
+    const dim3 grid(BH, (a.n + 127) / 128);
+    if (which == 0) {
+        LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_qtile_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
+        bwd_qtile_tc_kernel<D, 0><<<grid, BT_THREADS, Cfg::SM_ALLOC, a.stream>>>(mQ, mGh, mGl, mTh, mTl, mK, mV, p);
+    } else {
+        LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_qtile_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
+        bwd_qtile_tc_kernel<D, 1><<<grid, BT_THREADS, Cfg::SM_ALLOC, a.stream>>>(mQ, mGh, mGl, mTh, mTl, mK, mV, p);
+    }
+    LLA_CUDA_TRY(cudaGetLastError());
+    return LLA_OK;
+}
+
+}  // namespace
+
+int launch_backward_tensor(const BwdTensorArgs& a, int which) {
+    if (a.d == 64) return launch_t<64>(a, which);
+    if (a.d == 128) return launch_t<128>(a, which);
+    return LLA_ERR_UNSUPPORTED;
+}
+
+}  // namespace lla

@@ -154,6 +154,24 @@ struct BackwardArgs {
     cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
     cudaEvent_t fork, join;
 };
+// The tensor-core kernels of the backward pass (lla_backward_tensor.cu).  Every array is contiguous [B, H (or the
+// key/value heads), n, d]; gh/gl, yh/yl, tnh/tnl are the upstream gradient, y and -t as bf16 pairs hi + lo (gl may
+// be null: a bf16 gradient has no lo half); rowsc holds eight floats per row: m, 1/omega (0: row not handled here),
+// gbar, kappa, kbar.y, kbar.t, -m log2(e), unused.
+struct BwdTensorArgs {
+    const void *q, *k, *v;
+    const void *gh, *gl, *yh, *yl, *tnh, *tnl;
+    float* rowsc;
+    const float* stats;
+    const float* yvec;
+    const float* tvec;
+    float *kbar, *hvec, *dq, *dk, *dv;
+    int B, H, n, d, first, kv_group;
+    float scale;
+    int* status;
+    cudaStream_t stream;
+};
+int launch_backward_tensor(const BwdTensorArgs& a, int which);   // which: 0 = kbar, gbar, h; 1 = dQ; 2 = dK and dV
 size_t backward_workspace_bytes(int B, int H, int n, int d);
 int launch_backward(const BackwardArgs& a);
 

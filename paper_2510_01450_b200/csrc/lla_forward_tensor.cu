@@ -102,95 +102,8 @@ enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + TC_NST_MAX, B_VFULL = B
        B_COUNT = B_MFULL + 1 };
 static_assert(B_COUNT * 8 <= 256, "barrier area too small");
 
-// MMA issue.  The whole MMA warp runs these convergently and the instructions are predicated on the
-// elected lane (el != 0): issuing from a divergent single-thread branch instead costs ~100 clocks
-// per instruction (operands have to be moved into uniform registers one by one), three times the
-// execution time of a 128x64x16 MMA.
-// D[tmem] (+)= A[smem] * B[smem] over 64 elements of K (4 instructions, both operands K-major:
-// +32 bytes = 2 descriptor units per step).  acc0 = 0 overwrites D with the first product.
-__device__ __forceinline__ void mma_ss_k64(uint32_t el, uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
-        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "add.u64 a1, %2, 2; add.u64 a2, %2, 4; add.u64 a3, %2, 6;\n\t"
-        "add.u64 b1, %3, 2; add.u64 b2, %3, 4; add.u64 b3, %3, 6;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
-        "setp.ne.b32 p, 1, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, p;\n\t}"
-        ::"r"(el), "r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
-}
-// D[tmem] (+)= (U_hi + U_lo)[tmem] * B[smem] over 64 keys: per 16-key step the hi operand sits at
-// a + 16*step and the lo operand 8 columns further; B is MN-major (+2048 bytes = 128 units per step).
-__device__ __forceinline__ void mma_ts_hilo_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a0l, a1, a1l, a2, a2l, a3, a3l;\n\t"
-        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "add.u32 a0l, %2, 8; add.u32 a1, %2, 16; add.u32 a1l, %2, 24; add.u32 a2, %2, 32;\n\t"
-        "add.u32 a2l, %2, 40; add.u32 a3, %2, 48; add.u32 a3l, %2, 56;\n\t"
-        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
-        "setp.ne.b32 p, 1, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a0l], %3, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1l], b1, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2l], b2, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3l], b3, %4, p;\n\t}"
-        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
-}
-// D[tmem] (+)= U[tmem] * B[smem] over 64 keys with U a single 16-bit operand: the compute threads leave the
-// 16-key steps 0, 1 at columns a, a + 8 and the steps 2, 3 at a + 32, a + 40 (each 32-key pass writes into
-// the columns it read its scores from).
-__device__ __forceinline__ void mma_ts_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
-        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "add.u32 a1, %2, 8; add.u32 a2, %2, 32; add.u32 a3, %2, 40;\n\t"
-        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
-        "setp.ne.b32 p, 1, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
-        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
-}
-// The same with the four 16-element steps of the TMEM operand in consecutive groups of 8 columns.
-__device__ __forceinline__ void mma_ts_k64c(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
-        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "add.u32 a1, %2, 8; add.u32 a2, %2, 16; add.u32 a3, %2, 24;\n\t"
-        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
-        "setp.ne.b32 p, 1, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
-        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
-}
-// Shared-memory matrix descriptors (128-byte swizzle, tile base 1024-byte aligned).
-//   K-major:  rows of 128 bytes, 8-row groups 1024 bytes apart; a 16-element K step is +32 bytes.
-//   MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements; 8-row groups
-//             1024 bytes apart; a 16-element K step is +2048 bytes.
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_bytes = 16) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);         // start address
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;    // leading byte offset: distance between the 64-wide
-                                                         // column groups of an MN-major operand wider than 64
-    d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset
-    d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
-    d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
-    return d;
-}
-
 constexpr uint32_t IDESC_SS = make_idesc(TC_BR, TC_BC, 0, 0);   // S/A: A, B K-major; ACC uses make_idesc(128, D, 0, 1)
 constexpr uint32_t IDESC_SS16 = make_idesc(TC_BR, TC_BC, 0, 0, /*f16=*/1);   // the same products with both operands fp16
-
-// byte offset of the 16-byte chunk `chunk` (8 bf16) of row `row` in a swizzled 128 x 64 bf16 tile
-__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
 struct TcParams {
     int n, nq, causal, head_rows, max_iters, first_tile;   // n keys; nq query rows at positions n - nq .. n - 1

@@ -116,6 +116,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t* r) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(addr) : "memory");
 }
+// 16 consecutive TMEM columns of this thread's lane -> registers
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(addr) : "memory");
+}
 __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -182,6 +191,126 @@ constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn, int f16 = 0) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// tcgen05.mma issue and shared-memory matrix descriptors
+// ------------------------------------------------------------------------------------------------
+// MMA issue.  The whole MMA warp runs these convergently and the instructions are predicated on the
+// elected lane (el != 0): issuing from a divergent single-thread branch instead costs ~100 clocks
+// per instruction (operands have to be moved into uniform registers one by one), three times the
+// execution time of a 128x64x16 MMA.
+// D[tmem] (+)= A[smem] * B[smem] over 64 elements of K (4 instructions, both operands K-major:
+// +32 bytes = 2 descriptor units per step).  acc0 = 0 overwrites D with the first product.
+__device__ __forceinline__ void mma_ss_k64(uint32_t el, uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u64 a1, %2, 2; add.u64 a2, %2, 4; add.u64 a3, %2, 6;\n\t"
+        "add.u64 b1, %3, 2; add.u64 b2, %3, 4; add.u64 b3, %3, 6;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// D[tmem] (+)= (U_hi + U_lo)[tmem] * B[smem] over 64 keys: per 16-key step the hi operand sits at
+// a + 16*step and the lo operand 8 columns further; B is MN-major (+2048 bytes = 128 units per step).
+__device__ __forceinline__ void mma_ts_hilo_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a0l, a1, a1l, a2, a2l, a3, a3l;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a0l, %2, 8; add.u32 a1, %2, 16; add.u32 a1l, %2, 24; add.u32 a2, %2, 32;\n\t"
+        "add.u32 a2l, %2, 40; add.u32 a3, %2, 48; add.u32 a3l, %2, 56;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a0l], %3, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1l], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2l], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3l], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// D[tmem] (+)= U[tmem] * B[smem] over 64 keys with U a single 16-bit operand: the compute threads leave the
+// 16-key steps 0, 1 at columns a, a + 8 and the steps 2, 3 at a + 32, a + 40 (each 32-key pass writes into
+// the columns it read its scores from).
+__device__ __forceinline__ void mma_ts_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a1, %2, 8; add.u32 a2, %2, 32; add.u32 a3, %2, 40;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// The same with the four 16-element steps of the TMEM operand in consecutive groups of 8 columns.
+__device__ __forceinline__ void mma_ts_k64c(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a1, %2, 8; add.u32 a2, %2, 16; add.u32 a3, %2, 24;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// D[tmem] (+)= U_hi[tmem] * B[smem] over 64 keys: only the hi halves of the operand pairs laid out as for
+// mma_ts_hilo_k64 (16 columns per 16-key step), B MN-major.
+__device__ __forceinline__ void mma_ts_hi_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a1, %2, 16; add.u32 a2, %2, 32; add.u32 a3, %2, 48;\n\t"
+        "add.u64 b1, %3, 128; add.u64 b2, %3, 256; add.u64 b3, %3, 384;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem] over 64 elements of K with B K-major (a 64-row tile as TMA leaves it): the
+// operand in TMEM holds its four 16-element steps in consecutive groups of 8 columns, B advances 32 bytes a step.
+__device__ __forceinline__ void mma_ts_kmajor_k64(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "add.u32 a1, %2, 8; add.u32 a2, %2, 16; add.u32 a3, %2, 24;\n\t"
+        "add.u64 b1, %3, 2; add.u64 b2, %3, 4; add.u64 b3, %3, 6;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, p;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0) : "memory");
+}
+// Shared-memory matrix descriptors (128-byte swizzle, tile base 1024-byte aligned).
+//   K-major:  rows of 128 bytes, 8-row groups 1024 bytes apart; a 16-element K step is +32 bytes.
+//   MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements; 8-row groups
+//             1024 bytes apart; a 16-element K step is +2048 bytes.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_bytes = 16) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);         // start address
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;    // leading byte offset: distance between the 64-wide
+                                                         // column groups of an MN-major operand wider than 64
+    d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset
+    d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
+    return d;
+}
+
+// byte offset of the 16-byte chunk `chunk` (8 bf16) of row `row` in a swizzled 128 x 64 bf16 tile
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+// ------------------------------------------------------------------------------------------------
 // Host: tensor-map encoding through the driver entry point (no link-time dependency on libcuda)
 // ------------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -244,6 +373,20 @@ inline bool make_map_16bit_4d(CUtensorMap* map, const void* base, int batches, i
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return enc(map, dtype, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// fp32 [outer][rows][cols] records (cols * 4 a multiple of 16 bytes), box = all columns x box_rows rows, no swizzle:
+// rows past the end of an `outer` unit arrive as zeros.
+inline bool make_map_f32_rows(CUtensorMap* map, const void* base, int outer, int rows, int cols, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)outer};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)rows * cols * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)cols, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace sm100
