@@ -360,10 +360,11 @@ int lla_decode_default_splits(int B, int H, int Lmax);
  *               bytes, 256-byte aligned (required; LLA_ERR_WORKSPACE otherwise)
  * All pointers 16-byte aligned; no output may alias an input.  Work is enqueued on `stream`; the call
  * does not synchronise and keeps no pointer.
- * Reproducibility: dk and dv of a key tile accumulate in registers in a fixed order, but dq (every key tile adds
- * its share to the query rows), the directly-solved rows' shares of dk and dv, and, with grouped heads, all of dk
- * and dv are summed with fp32 atomic adds, whose order varies from run to run: those outputs agree between runs
- * to rounding (about 1e-6 relative), not bit for bit.
+ * Reproducibility: dq is bit-identical from run to run (each query tile owns its rows and stores them; with
+ * impl = LLA_IMPL_SIMT the key tiles add their shares atomically instead and it is not).  dk and dv are summed
+ * with fp32 atomic adds -- the key tiles', the directly-solved rows' and, with grouped heads, every query head's
+ * share -- whose order varies: those two outputs agree between runs to rounding (about 1e-6 relative), not bit
+ * for bit.
  */
 typedef struct lla_backward_params {
     const void *q, *k, *v, *out, *dout;
