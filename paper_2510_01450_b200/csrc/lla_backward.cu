@@ -214,7 +214,14 @@ __device__ __forceinline__ void split_pack(float x0, float x1, uint32_t& hi, uin
 }
 struct Pairs16 {
     uint32_t *yh, *yl, *tnh, *tnl;      // two bf16 per word
+    float* pairsc;                      // [heads][npair][8]: the scalars of two rows per record (BwdTensorArgs::pairsc)
+    int npair;
 };
+// row i's four scalars go to slots s, 2 + s, 4 + s, 6 + s of record i / 2 (s = i & 1)
+__device__ __forceinline__ void store_pair_record(const Pairs16& p16, long long head, int i, float nm2, float ky, float gk, float kk) {
+    float* rp = p16.pairsc + ((size_t)head * p16.npair + (i >> 1)) * 8 + (i & 1);
+    rp[0] = nm2; rp[2] = ky; rp[4] = gk; rp[6] = kk;
+}
 template <int D>
 __global__ void __launch_bounds__(BW_THREADS)
 bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__ out, int out_dtype,
@@ -232,7 +239,7 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
                 const size_t w = ((size_t)row * D + c) >> 1;
                 p16.yh[w] = 0; p16.yl[w] = 0; p16.tnh[w] = 0; p16.tnl[w] = 0;
             }
-            if (lane < BW_ROWSC) rowsc[row * BW_ROWSC + lane] = 0.f;
+            if (lane == 0) store_pair_record(p16, row / n, i, -1e30f, 0.f, 0.f, 0.f);
         }
         return;
     }
@@ -276,8 +283,11 @@ bwd_rowprep_kernel(const __nv_bfloat16* __restrict__ q, const void* __restrict__
         rs[3] = go + kt - qt;      // kappa = g.o + t.(kbar - q)
         rs[4] = ky;
         rs[5] = kt;
-        rs[6] = -m * 1.4426950408889634f;
-        rs[7] = 0.f;
+        if (p16.yh) {
+            const float kappa = go + kt - qt;
+            store_pair_record(p16, row / n, i, -(m * 1.4426950408889634f + log2f(omega)), ky, rs[2] - kt, kt - kappa);
+            if (i == n - 1 && (n & 1)) store_pair_record(p16, row / n, n, -1e30f, 0.f, 0.f, 0.f);      // the record's unused half
+        }
         // dL/d(lambda_i): lambda enters C as (e^{-m} / omega) lambda I and dL = t^T dC y
         if (dlambda) dlambda[row] = __expf(-m) / omega * ty;
     }
@@ -615,9 +625,12 @@ size_t head_smem_bytes(int lcap) {
 // workspace: kbar, h, t, y as [rows][D] fp32, the scalar records, then the tensor-core kernels' bf16 operand arrays
 // (y and -t as hi and lo; the upstream gradient's hi and lo, used when it comes in fp32)
 size_t ws_floats(long long rows, int d) { return (size_t)rows * (4 * (size_t)d + BW_ROWSC); }
-size_t ws_fp32_bytes(long long rows, int d) { return (ws_floats(rows, d) * sizeof(float) + 255) & ~(size_t)255; }
+size_t ws_pairsc_floats(long long heads, int n) { return (size_t)heads * ((n + 1) / 2) * 8; }      // two rows per record
+size_t ws_fp32_bytes(long long rows, int d, long long heads) {
+    return ((ws_floats(rows, d) + ws_pairsc_floats(heads, (int)(rows / heads))) * sizeof(float) + 255) & ~(size_t)255;
+}
 size_t ws_pair_bytes(long long rows, int d) { return ((size_t)rows * d * 2 + 255) & ~(size_t)255; }      // one bf16 array
-size_t ws_own_bytes(long long rows, int d) { return ws_fp32_bytes(rows, d) + 6 * ws_pair_bytes(rows, d); }
+size_t ws_own_bytes(long long rows, int d, long long heads) { return ws_fp32_bytes(rows, d, heads) + 6 * ws_pair_bytes(rows, d); }
 
 template <int D>
 int launch_t(const BackwardArgs& a) {
@@ -627,14 +640,15 @@ int launch_t(const BackwardArgs& a) {
     const int first = max(0, min(a.n, a.head_rows - 1));      // rows [0, first) are solved directly
     const int kvg = a.kv_group > 0 ? a.kv_group : 1;
     const long long kvrows = rows / kvg;                       // rows of k, v, dk, dv
-    if (a.workspace_bytes < ws_own_bytes(rows, D) || !a.workspace) return LLA_ERR_WORKSPACE;
+    if (a.workspace_bytes < ws_own_bytes(rows, D, BH) || !a.workspace) return LLA_ERR_WORKSPACE;
     if (first > 2 * D) return LLA_ERR_UNSUPPORTED;
     float* kbar = static_cast<float*>(a.workspace);
     float* hvec = kbar + rows * D;
     float* tvec = hvec + rows * D;
     float* yvec = tvec + rows * D;
     float* rowsc = yvec + rows * D;
-    char* pairs = static_cast<char*>(a.workspace) + ws_fp32_bytes(rows, D);
+    float* pairsc = rowsc + rows * BW_ROWSC;
+    char* pairs = static_cast<char*>(a.workspace) + ws_fp32_bytes(rows, D, BH);
     const size_t pb = ws_pair_bytes(rows, D);
     const bool tensor = !a.cuda_core_pairs;
     const auto* q = static_cast<const __nv_bfloat16*>(a.q);
@@ -667,6 +681,7 @@ int launch_t(const BackwardArgs& a) {
             t.yh = pairs; t.yl = pairs + pb; t.tnh = pairs + 2 * pb; t.tnl = pairs + 3 * pb;
             p16.yh = reinterpret_cast<uint32_t*>(pairs); p16.yl = reinterpret_cast<uint32_t*>(pairs + pb);
             p16.tnh = reinterpret_cast<uint32_t*>(pairs + 2 * pb); p16.tnl = reinterpret_cast<uint32_t*>(pairs + 3 * pb);
+            p16.pairsc = pairsc; p16.npair = (a.n + 1) / 2;
             if (a.dout_dtype == LLA_F32) {
                 t.gh = pairs + 4 * pb; t.gl = pairs + 5 * pb;
                 const size_t quads = (size_t)rows * D / 4;
@@ -676,7 +691,7 @@ int launch_t(const BackwardArgs& a) {
             } else {
                 t.gh = a.dout; t.gl = nullptr;
             }
-            t.rowsc = rowsc; t.stats = a.stats; t.yvec = yvec; t.tvec = tvec;
+            t.rowsc = rowsc; t.pairsc = pairsc; t.stats = a.stats; t.yvec = yvec; t.tvec = tvec;
             t.kbar = kbar; t.hvec = hvec; t.dq = a.dq; t.dk = a.dk; t.dv = a.dv;
             t.B = a.B; t.H = a.H; t.n = a.n; t.d = D; t.first = first; t.kv_group = kvg;
             t.scale = a.scale; t.status = a.status; t.stream = a.stream;
@@ -702,7 +717,7 @@ int launch_t(const BackwardArgs& a) {
         f.set_contiguous();
         // what the workspace holds beyond this pass's own arrays serves the solve (the fp16 copy of k; for
         // d = 128 the row-state slots), so that the backward pass allocates nothing
-        const size_t own = ws_own_bytes(rows, D);
+        const size_t own = ws_own_bytes(rows, D, BH);
         if (a.workspace_bytes > own) {
             f.workspace = static_cast<char*>(a.workspace) + own;
             f.workspace_bytes = a.workspace_bytes - own;
@@ -734,7 +749,7 @@ int launch_t(const BackwardArgs& a) {
 }  // namespace
 
 size_t backward_workspace_bytes(int B, int H, int n, int d) {
-    return ws_own_bytes((long long)B * H * n, d) + forward_tensor_workspace_bytes(B, H, n, d);
+    return ws_own_bytes((long long)B * H * n, d, (long long)B * H) + forward_tensor_workspace_bytes(B, H, n, d);
 }
 
 int launch_backward(const BackwardArgs& a) {

@@ -19,7 +19,10 @@
 // preparation kernel (-t, so that "- A^T T" is an accumulation like the others).  In the dQ kernel y sits in TMEM
 // (the tile's five other stationary operands fill the shared memory at d = 128).
 //
-// Score tiles are single-buffered: 4 x 64 columns plus the accumulators take all 512 TMEM columns at d = 128.
+// Score tiles are single-buffered (4 x 64 columns plus the accumulators take all 512 TMEM columns at d = 128), so
+// a step is pipelined inside itself: the MMA warp commits the score products in two groups and the compute threads
+// hand the coefficient tiles back in two groups, so that each side works on one group while the other side is busy
+// with the other.
 // All waits are bounded; a wait that expires sets LLA_STATUS_TIMEOUT and the block leaves through the common exit.
 #include "lla_sm100.cuh"
 
@@ -40,7 +43,8 @@ struct BtParams {
     int has_glo;          // the upstream gradient has a lo half (fp32 dout)
     float scale;
     const float* stats;   // [rows][3] saved by the forward
-    const float* rowsc;   // [rows][8] per-row scalars (see bwd_rowprep_kernel)
+    const float* pairsc;  // [heads][npair][8] per-row scalars, two rows per record (see bwd_rowprep_kernel)
+    int npair;            // records per head: ceil(n / 2)
     const float* yvec;    // [rows][D] fp32
     const float* tvec;    // [rows][D] fp32
     float* rowsc_w;       // moments kernel: gbar goes to slot 2
@@ -64,8 +68,8 @@ struct KtCfg {
     static constexpr int NST = D == 64 ? 2 : 1;    // stages of the query-side ring
     static constexpr int SM_K = 0, SM_V = T128, SM_ST = 2 * T128;
     static constexpr int ST_Q = 0, ST_YH = T64, ST_YL = 2 * T64, ST_TH = 3 * T64, ST_TL = 4 * T64, ST_GH = 5 * T64, ST_GL = 6 * T64;
-    static constexpr int ST_RS = 7 * T64;          // 64 row records of 8 floats
-    static constexpr int STAGE = 7 * T64 + 2048;
+    static constexpr int ST_RS = 7 * T64;          // 32 records of 8 floats: the scalars of the step's 64 rows, two rows each
+    static constexpr int STAGE = 7 * T64 + 1024;
     static constexpr int SM_BAR = SM_ST + NST * STAGE;
     static constexpr int SM_MISC = SM_BAR + 128;
     static constexpr int SM_ALLOC = SM_MISC + 64 + 1024;
@@ -74,7 +78,27 @@ struct KtCfg {
     static constexpr int C_S = 0, C_E = 64, C_F = 128, C_G = 192, C_DK = 256, C_DV = 256 + D;
 };
 static_assert(KtCfg<64>::SM_ALLOC <= 227 * 1024 && KtCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
-enum { KB_KV = 0, KB_FULL = 1, KB_EMPTY = 3, KB_SFULL = 5, KB_PREADY = 6, KB_ACCFULL = 7, KB_EXIT = 8, KB_COUNT = 9 };
+enum { KB_KV = 0, KB_FULL = 1, KB_EMPTY = 3, KB_SF1 = 5, KB_SF2 = 6, KB_PRA = 7, KB_PRB = 8, KB_ACCFULL = 9, KB_EXIT = 10, KB_COUNT = 11 };
+
+// one MMA with the A operand in TMEM, predicated on the elected lane
+__device__ __forceinline__ void mma_ts1(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t}"
+        ::"r"(el), "r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+// bf16 pair of two packed fp32 values: returns the hi word, writes the lo word
+__device__ __forceinline__ uint32_t split2(uint64_t v, uint32_t& lo) {
+    float a, b;
+    upk2(v, a, b);
+    return split_bf16x2(a, b, lo);
+}
+__device__ __forceinline__ uint64_t pku(uint32_t a, uint32_t b) { return pk2(__uint_as_float(a), __uint_as_float(b)); }
+__device__ __forceinline__ uint64_t ex2_2(uint64_t t) {
+    float a, b;
+    upk2(t, a, b);
+    return pk2(ex2f(a), ex2f(b));
+}
 
 template <int D>
 __global__ void __launch_bounds__(BT_THREADS, 1)
@@ -108,8 +132,10 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             mbar_init(bar(KB_FULL + s), 1);
             mbar_init(bar(KB_EMPTY + s), 1);
         }
-        mbar_init(bar(KB_SFULL), 1);
-        mbar_init(bar(KB_PREADY), BT_COMPUTE / 32);
+        mbar_init(bar(KB_SF1), 1);
+        mbar_init(bar(KB_SF2), 1);
+        mbar_init(bar(KB_PRA), BT_COMPUTE / 32);
+        mbar_init(bar(KB_PRB), BT_COMPUTE / 32);
         mbar_init(bar(KB_ACCFULL), 1);
         mbar_init(bar(KB_EXIT), 1);
         misc[2] = 0;
@@ -138,7 +164,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const int s = g % NST, i0 = 64 * (it0 + g);
                 if (!mbar_wait(bar(KB_EMPTY + s), ((g / NST) & 1) ^ 1, abort_flag, wcap)) break;
                 const uint32_t st = sbase + Cfg::SM_ST + s * STAGE, fb = bar(KB_FULL + s);
-                mbar_expect_tx(fb, (6 + (prm.has_glo ? 1 : 0)) * T64 + 2048);
+                mbar_expect_tx(fb, (6 + (prm.has_glo ? 1 : 0)) * T64 + 1024);
                 for (int sub = 0; sub < KSUB; ++sub) {
                     tma_load_3d(st + Cfg::ST_Q + sub * 8192, &tmQ, fb, 64 * sub, i0, bh);
                     tma_load_3d(st + Cfg::ST_YH + sub * 8192, &tmYh, fb, 64 * sub, i0, bh);
@@ -148,7 +174,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     tma_load_3d(st + Cfg::ST_GH + sub * 8192, &tmGh, fb, 64 * sub, i0, bh);
                     if (prm.has_glo) tma_load_3d(st + Cfg::ST_GL + sub * 8192, &tmGl, fb, 64 * sub, i0, bh);
                 }
-                tma_load_3d(st + Cfg::ST_RS, &tmRS, fb, 0, i0, bh);
+                tma_load_3d(st + Cfg::ST_RS, &tmRS, fb, 0, i0 / 2, bh);
                 issued = g + 1;
             }
             if (*abort_flag) {      // an aborted block: what was issued must have landed before the block exits
@@ -174,26 +200,30 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 for (int sub = 0; sub < KSUB; ++sub)
                     mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
             };
+            // group 1: what a^T needs; group 2: the rest
             score(Cfg::C_S, kdesc, Cfg::ST_Q, 0);
             score(Cfg::C_E, kdesc, Cfg::ST_YH, 0);
             score(Cfg::C_E, kdesc, Cfg::ST_YL, 1);
+            tc_commit_el(el, bar(KB_SF1));
             score(Cfg::C_F, kdesc, Cfg::ST_TH, 0);
             score(Cfg::C_F, kdesc, Cfg::ST_TL, 1);
             score(Cfg::C_G, vdesc, Cfg::ST_GH, 0);
             if (prm.has_glo) score(Cfg::C_G, vdesc, Cfg::ST_GL, 1);
-            tc_commit_el(el, bar(KB_SFULL));
-            if (!mbar_wait(bar(KB_PREADY), g & 1, abort_flag, wcap)) break;
-            tc_fence_after();
-            // coefficient tiles (hi + lo pairs) sit where the scores were: a^T in S, ds^T in E, p1^T in F
+            tc_commit_el(el, bar(KB_SF2));
+            // coefficient tiles (hi + lo pairs) sit where the scores were: a^T in S, then ds^T in E and p1^T in F
             auto bd = [&](int off) { return make_desc(st + off, 8192); };
             const uint32_t acc = g > 0;
+            if (!mbar_wait(bar(KB_PRA), g & 1, abort_flag, wcap)) break;
+            tc_fence_after();
             mma_ts_hilo_k64(el, tm_u + Cfg::C_DV, tm_u + Cfg::C_S, bd(Cfg::ST_GH), Cfg::IDESC_TS, acc);
             if (prm.has_glo) mma_ts_hi_k64(el, tm_u + Cfg::C_DV, tm_u + Cfg::C_S, bd(Cfg::ST_GL), Cfg::IDESC_TS, 1);
-            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_E, bd(Cfg::ST_Q), Cfg::IDESC_TS, acc);
+            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TH), Cfg::IDESC_TS, acc);
+            mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TL), Cfg::IDESC_TS, 1);
+            if (!mbar_wait(bar(KB_PRB), g & 1, abort_flag, wcap)) break;
+            tc_fence_after();
+            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_E, bd(Cfg::ST_Q), Cfg::IDESC_TS, 1);
             mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YH), Cfg::IDESC_TS, 1);
             mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YL), Cfg::IDESC_TS, 1);
-            mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TH), Cfg::IDESC_TS, 1);
-            mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TL), Cfg::IDESC_TS, 1);
             tc_commit_el(el, bar(KB_EMPTY + s));
             if (g == nstep - 1) tc_commit_el(el, bar(KB_ACCFULL));
         }
@@ -207,53 +237,74 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int lrow = quad * 32 + lane;            // key inside the tile == TMEM lane
         const int gj = j0 + lrow;
         const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
-        const float c1 = prm.scale * BT_LOG2E, scale = prm.scale;
+        const float c1 = prm.scale * BT_LOG2E;
+        const uint64_t c1c1 = pk2(c1, c1), one2 = pk2(1.f, 1.f), sc2 = pk2(prm.scale, prm.scale);
         bool ok = true;
         for (int g = 0; g < nstep; ++g) {
             const int s = g % NST, i0 = 64 * (it0 + g);
             if (!mbar_wait(bar(KB_FULL + s), (g / NST) & 1, abort_flag, wcap)) { ok = false; break; }      // the row records
-            if (!mbar_wait(bar(KB_SFULL), g & 1, abort_flag, wcap)) { ok = false; break; }
+            if (!mbar_wait(bar(KB_SF1), g & 1, abort_flag, wcap)) { ok = false; break; }
             tc_fence_after();
-            const float4* rs = reinterpret_cast<const float4*>(smem + Cfg::SM_ST + s * STAGE + Cfg::ST_RS);
-#pragma unroll 1
-            for (int chunk = 0; chunk < 2; ++chunk) {
-                const int colbase = 32 * half + 16 * chunk;      // 16 query rows = one 16-element step of the products
-                uint32_t sv[16], ev[16], fv[16], gv[16];
-                tmem_ld16(tm_lane + Cfg::C_S + colbase, sv);
-                tmem_ld16(tm_lane + Cfg::C_E + colbase, ev);
-                tmem_ld16(tm_lane + Cfg::C_F + colbase, fv);
-                tmem_ld16(tm_lane + Cfg::C_G + colbase, gv);
+            // records of this thread's 32 query rows (16 pairs): (nm2, nm2, kbar.y, kbar.y), (gk, gk, kk, kk)
+            const float4* rsp = reinterpret_cast<const float4*>(smem + Cfg::SM_ST + s * STAGE + Cfg::ST_RS) + 32 * half;
+            const uint32_t col0 = 32 * half;
+            uint64_t p2[16], e2v[16];
+            {
+                // a = p (1 - e) from S and E: p = 2^(c1 s + nm2) carries 1 / omega; rows switched off have nm2 = -1e30
+                uint32_t sv[32], ev[32], pa[32];
+                tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
+                tmem_ld32(tm_lane + Cfg::C_E + col0, ev);
                 tc_wait_ld();
-                uint32_t pa[16], pd[16], pp[16];
+                if (i0 < j0 + 128 || i0 + 64 > n) {      // a diagonal or last step: hide the pairs with j > i or i >= n
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int gi = i0 + (int)col0 + e;
+                        if (gj > gi || gi >= n) sv[e] = __float_as_uint(-1e30f);
+                    }
+                }
+#pragma unroll
+                for (int e2 = 0; e2 < 16; ++e2) {
+                    const float4 ra = rsp[2 * e2];
+                    const uint64_t p = ex2_2(fma2(pku(sv[2 * e2], sv[2 * e2 + 1]), c1c1, pk2(ra.x, ra.y)));
+                    const uint64_t evv = sub2(pku(ev[2 * e2], ev[2 * e2 + 1]), pk2(ra.z, ra.w));
+                    const int ks = e2 >> 3, e = e2 & 7;
+                    pa[ks * 16 + e] = split2(mul2(p, sub2(one2, evv)), pa[ks * 16 + 8 + e]);
+                    p2[e2] = p;
+                    e2v[e2] = evv;
+                }
+                tmem_st32(tm_lane + Cfg::C_S + col0, pa);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(KB_PRA));
+            }
+            if (!mbar_wait(bar(KB_SF2), g & 1, abort_flag, wcap)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int chunk = 0; chunk < 2; ++chunk) {
+                // with u = gbar - f (the F tile holds (-t) . k, so u = gk - F with gk = gbar - kbar.t):
+                //   p1 = p (u - gamma),  ds = scale p (gamma (1 - e) + u e + F + kk),  kk = kbar.t - kappa
+                uint32_t fv[16], gv[16], pd[16], pp[16];
+                tmem_ld16(tm_lane + Cfg::C_F + col0 + 16 * chunk, fv);
+                tmem_ld16(tm_lane + Cfg::C_G + col0 + 16 * chunk, gv);
+                tc_wait_ld();
 #pragma unroll
                 for (int e2 = 0; e2 < 8; ++e2) {
-                    float a[2], ds[2], p1[2];
-#pragma unroll
-                    for (int x = 0; x < 2; ++x) {
-                        const int e = 2 * e2 + x, col = colbase + e, gi = i0 + col;
-                        const float4 r0 = rs[2 * col], r1 = rs[2 * col + 1];     // (m, 1/omega, gbar, kappa), (kbar.y, kbar.t, -m log2 e, -)
-                        const bool valid = gj <= gi && gi < n && r0.y > 0.f;
-                        const float p = valid ? ex2f(fmaf(__uint_as_float(sv[e]), c1, r1.z)) * r0.y : 0.f;
-                        const float evv = __uint_as_float(ev[e]) - r1.x;
-                        const float fvv = -__uint_as_float(fv[e]) - r1.y;      // the tile holds (-t) . k
-                        const float gam = __uint_as_float(gv[e]);
-                        const float ome = 1.f - evv;
-                        a[x] = valid ? p * ome : 0.f;
-                        ds[x] = valid ? scale * p * (gam * ome + (r0.z + fvv) * evv - fvv - r0.w) : 0.f;
-                        p1[x] = valid ? p * (fvv - gam + r0.z) : 0.f;
-                    }
-                    pa[e2] = split_bf16x2(a[0], a[1], pa[8 + e2]);
-                    pd[e2] = split_bf16x2(ds[0], ds[1], pd[8 + e2]);
-                    pp[e2] = split_bf16x2(p1[0], p1[1], pp[8 + e2]);
+                    const int idx = 8 * chunk + e2;
+                    const float4 rb = rsp[2 * idx + 1];
+                    const uint64_t f2 = pku(fv[2 * e2], fv[2 * e2 + 1]), g2 = pku(gv[2 * e2], gv[2 * e2 + 1]);
+                    const uint64_t u = sub2(pk2(rb.x, rb.y), f2);
+                    const uint64_t inner = fma2(g2, sub2(one2, e2v[idx]), fma2(u, e2v[idx], add2(f2, pk2(rb.z, rb.w))));
+                    pd[e2] = split2(mul2(mul2(p2[idx], sc2), inner), pd[8 + e2]);
+                    pp[e2] = split2(mul2(p2[idx], sub2(u, g2)), pp[8 + e2]);
                 }
-                tmem_st16(tm_lane + Cfg::C_S + colbase, pa);
-                tmem_st16(tm_lane + Cfg::C_E + colbase, pd);
-                tmem_st16(tm_lane + Cfg::C_F + colbase, pp);
+                tmem_st16(tm_lane + Cfg::C_E + col0 + 16 * chunk, pd);
+                tmem_st16(tm_lane + Cfg::C_F + col0 + 16 * chunk, pp);
             }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(KB_PREADY));
+            if (lane == 0) mbar_arrive(bar(KB_PRB));
         }
         if (ok && mbar_wait(bar(KB_ACCFULL), 0, abort_flag, wcap)) {
             tc_fence_after();
@@ -307,7 +358,8 @@ struct QtCfg {
     static constexpr int C_G0 = 64, C_KB = 128, C_H = 128 + D;
 };
 static_assert(QtCfg<64>::SM_ALLOC <= 227 * 1024 && QtCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
-enum { QB_QFULL = 0, QB_YREADY = 1, QB_FULL = 2, QB_EMPTY = 5, QB_SFULL = 8, QB_PREADY = 9, QB_ACCFULL = 10, QB_EXIT = 11, QB_COUNT = 12 };
+enum { QB_QFULL = 0, QB_YREADY = 1, QB_FULL = 2, QB_EMPTY = 5, QB_SF1 = 8, QB_SF2 = 9, QB_PRA = 10, QB_PRB = 11, QB_ACCFULL = 12,
+       QB_EXIT = 13, QB_COUNT = 14 };
 
 template <int D, int MODE>
 __global__ void __launch_bounds__(BT_THREADS, 1)
@@ -351,8 +403,10 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_init(bar(QB_FULL + s), 1);
             mbar_init(bar(QB_EMPTY + s), 1);
         }
-        mbar_init(bar(QB_SFULL), 1);
-        mbar_init(bar(QB_PREADY), BT_COMPUTE / 32);
+        mbar_init(bar(QB_SF1), 1);
+        mbar_init(bar(QB_SF2), 1);
+        mbar_init(bar(QB_PRA), BT_COMPUTE / 32);
+        mbar_init(bar(QB_PRB), BT_COMPUTE / 32);
         mbar_init(bar(QB_ACCFULL), 1);
         mbar_init(bar(QB_EXIT), 1);
         misc[2] = 0;
@@ -419,7 +473,9 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int sub = 0; sub < KSUB; ++sub)
                     mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
             };
+            const uint64_t kmn = make_desc(st, 8192);       // the K block read MN-major, N = D
             score(Cfg::C_S, Cfg::SM_Q, kdesc, 0);
+            tc_commit_el(el, bar(QB_SF1));      // the weights can be formed while the other products run
             if (MODE == 1) {
                 // E = Y K^T with y (hi, then lo) from TMEM: D / 16 steps of 8 columns each
 #pragma unroll
@@ -434,16 +490,16 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const uint32_t cg = MODE == 1 ? Cfg::C_G1 : Cfg::C_G0;
             score(cg, Cfg::SM_GH, vdesc, 0);
             if (prm.has_glo) score(cg, Cfg::SM_GL, vdesc, 1);
-            tc_commit_el(el, bar(QB_SFULL));
-            if (!mbar_wait(bar(QB_PREADY), c & 1, abort_flag, wcap)) break;
-            tc_fence_after();
-            const uint64_t kmn = make_desc(st, 8192);       // the K block read MN-major, N = D
-            if (MODE == 1) {
-                mma_ts_hilo_k64(el, tm_u + Cfg::C_DQ, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
-            } else {
+            tc_commit_el(el, bar(QB_SF2));
+            if (MODE == 0) {
+                if (!mbar_wait(bar(QB_PRA), c & 1, abort_flag, wcap)) break;
+                tc_fence_after();
                 mma_ts_hilo_k64(el, tm_u + Cfg::C_KB, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
-                mma_ts_hilo_k64(el, tm_u + Cfg::C_H, tm_u + Cfg::C_G0, kmn, Cfg::IDESC_TS, c > 0);
             }
+            if (!mbar_wait(bar(QB_PRB), c & 1, abort_flag, wcap)) break;
+            tc_fence_after();
+            if (MODE == 1) mma_ts_hilo_k64(el, tm_u + Cfg::C_DQ, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
+            else mma_ts_hilo_k64(el, tm_u + Cfg::C_H, tm_u + Cfg::C_G0, kmn, Cfg::IDESC_TS, c > 0);
             tc_commit_el(el, bar(QB_EMPTY + s));
             if (c == nblk - 1) tc_commit_el(el, bar(QB_ACCFULL));
         }
@@ -459,18 +515,20 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const bool okr = gi < n && gi >= prm.first;
         const size_t row = (size_t)bh * n + gi;
         const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
-        const float c1 = prm.scale * BT_LOG2E, scale = prm.scale;
-        float nm2 = 0.f, iom = 0.f, gbar = 0.f, kappa = 0.f, ky = 0.f, kt = 0.f;
+        const float c1 = prm.scale * BT_LOG2E;
+        // per-row scalars (see bwd_rowprep_kernel): p = 2^(c1 s + nm2) carries 1 / omega; a row that is switched off
+        // has nm2 = -1e30 and no weight
+        float nm2 = -1e30f, ky = 0.f, gk = 0.f, kk = 0.f;
         if (okr) {
             if (MODE == 1) {
-                const float4 r0 = *reinterpret_cast<const float4*>(prm.rowsc + row * 8);
-                const float4 r1 = *reinterpret_cast<const float4*>(prm.rowsc + row * 8 + 4);
-                iom = r0.y; gbar = r0.z; kappa = r0.w; ky = r1.x; kt = r1.y; nm2 = r1.z;
+                const float* rp = prm.pairsc + ((size_t)bh * prm.npair + (gi >> 1)) * 8 + (gi & 1);
+                nm2 = rp[0]; ky = rp[2]; gk = rp[4]; kk = rp[6];
             } else {
-                nm2 = -prm.stats[row * 3 + 0] * BT_LOG2E;
-                iom = 1.f / prm.stats[row * 3 + 1];
+                nm2 = -(prm.stats[row * 3 + 0] * BT_LOG2E + log2f(prm.stats[row * 3 + 1]));
             }
         }
+        const uint64_t c1c1 = pk2(c1, c1), nm22 = pk2(nm2, nm2), one2 = pk2(1.f, 1.f), sc2 = pk2(prm.scale, prm.scale);
+        const uint64_t ky2 = pk2(ky, ky), gk2 = pk2(gk, gk), kk2 = pk2(kk, kk);
         if (MODE == 1) {
             // this thread's half of y_i -> bf16 pairs in TMEM: 16-element steps of 8 columns, hi block then lo block
             constexpr int NW = D / 4;      // packed words per half row and part
@@ -494,65 +552,84 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(QB_YREADY));
         }
-        float gb = 0.f;
+        uint64_t gb2 = pk2(0.f, 0.f);
         bool ok = true;
         for (int c = 0; c < nblk; ++c) {
-            if (!mbar_wait(bar(QB_SFULL), c & 1, abort_flag, wcap)) { ok = false; break; }
+            if (!mbar_wait(bar(QB_SF1), c & 1, abort_flag, wcap)) { ok = false; break; }
             tc_fence_after();
-#pragma unroll 1
+            const uint32_t col0 = 32 * half;      // this thread's 32 keys of the block
+            uint64_t p2[16];
+            {
+                uint32_t sv[32];
+                tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
+                tc_wait_ld();
+                const int jlim = gi + 1 - (64 * c + (int)col0);      // keys e < jlim are visible
+                if (jlim < 32) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (e >= jlim) sv[e] = __float_as_uint(-1e30f);
+                }
+#pragma unroll
+                for (int e2 = 0; e2 < 16; ++e2) p2[e2] = ex2_2(fma2(pku(sv[2 * e2], sv[2 * e2 + 1]), c1c1, nm22));
+                if (MODE == 0) {      // P over S, ready for kbar += P K while Gamma is still being formed
+                    uint32_t pp[32];
+#pragma unroll
+                    for (int e2 = 0; e2 < 16; ++e2) {
+                        const int ks = e2 >> 3, e = e2 & 7;
+                        pp[ks * 16 + e] = split2(p2[e2], pp[ks * 16 + 8 + e]);
+                    }
+                    tmem_st32(tm_lane + Cfg::C_S + col0, pp);
+                    tc_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(QB_PRA));
+                }
+            }
+            if (!mbar_wait(bar(QB_SF2), c & 1, abort_flag, wcap)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
             for (int chunk = 0; chunk < 2; ++chunk) {
-                const int colbase = 32 * half + 16 * chunk;      // 16 keys = one 16-element step of the products
-                const int jlim = (okr ? gi + 1 : 0) - (64 * c + colbase);      // keys e < jlim of this chunk are visible
+                const uint32_t colbase = col0 + 16 * chunk;      // 16 keys = one 16-element step of the products
                 if (MODE == 1) {
-                    uint32_t sv[16], ev[16], fv[16], gv[16], pd[16];
-                    tmem_ld16(tm_lane + Cfg::C_S + colbase, sv);
+                    // with u = gbar - f (the F tile holds (-t) . k, so u = gk - F with gk = gbar - kbar.t):
+                    //   ds = scale p (gamma (1 - e) + u e + F + kk),  kk = kbar.t - kappa
+                    uint32_t ev[16], fv[16], gv[16], pd[16];
                     tmem_ld16(tm_lane + Cfg::C_E + colbase, ev);
                     tmem_ld16(tm_lane + Cfg::C_F + colbase, fv);
                     tmem_ld16(tm_lane + Cfg::C_G1 + colbase, gv);
                     tc_wait_ld();
 #pragma unroll
                     for (int e2 = 0; e2 < 8; ++e2) {
-                        float ds[2];
-#pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            const int e = 2 * e2 + x;
-                            const bool valid = e < jlim;
-                            const float p = valid ? ex2f(fmaf(__uint_as_float(sv[e]), c1, nm2)) * iom : 0.f;
-                            const float evv = __uint_as_float(ev[e]) - ky;
-                            const float fvv = -__uint_as_float(fv[e]) - kt;      // the tile holds (-t) . k
-                            const float gam = __uint_as_float(gv[e]);
-                            ds[x] = valid ? scale * p * (gam * (1.f - evv) + (gbar + fvv) * evv - fvv - kappa) : 0.f;
-                        }
-                        pd[e2] = split_bf16x2(ds[0], ds[1], pd[8 + e2]);
+                        const uint64_t f2 = pku(fv[2 * e2], fv[2 * e2 + 1]), g2 = pku(gv[2 * e2], gv[2 * e2 + 1]);
+                        const uint64_t evv = sub2(pku(ev[2 * e2], ev[2 * e2 + 1]), ky2);
+                        const uint64_t u = sub2(gk2, f2);
+                        const uint64_t inner = fma2(g2, sub2(one2, evv), fma2(u, evv, add2(f2, kk2)));
+                        pd[e2] = split2(mul2(mul2(p2[8 * chunk + e2], sc2), inner), pd[8 + e2]);
                     }
                     tmem_st16(tm_lane + Cfg::C_S + colbase, pd);
                 } else {
-                    uint32_t sv[16], gv[16], pp[16], pg[16];
-                    tmem_ld16(tm_lane + Cfg::C_S + colbase, sv);
+                    uint32_t gv[16], pg[16];
                     tmem_ld16(tm_lane + Cfg::C_G0 + colbase, gv);
                     tc_wait_ld();
 #pragma unroll
                     for (int e2 = 0; e2 < 8; ++e2) {
-                        float p[2], q[2];
-#pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            const int e = 2 * e2 + x;
-                            const bool valid = e < jlim;
-                            p[x] = valid ? ex2f(fmaf(__uint_as_float(sv[e]), c1, nm2)) * iom : 0.f;
-                            q[x] = valid ? p[x] * __uint_as_float(gv[e]) : 0.f;
-                            gb += q[x];
-                        }
-                        pp[e2] = split_bf16x2(p[0], p[1], pp[8 + e2]);
-                        pg[e2] = split_bf16x2(q[0], q[1], pg[8 + e2]);
+                        const uint64_t q2 = mul2(p2[8 * chunk + e2], pku(gv[2 * e2], gv[2 * e2 + 1]));
+                        gb2 = add2(gb2, q2);
+                        pg[e2] = split2(q2, pg[8 + e2]);
                     }
-                    tmem_st16(tm_lane + Cfg::C_S + colbase, pp);
                     tmem_st16(tm_lane + Cfg::C_G0 + colbase, pg);
                 }
             }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(QB_PREADY));
+            if (lane == 0) mbar_arrive(bar(QB_PRB));
+        }
+        float gb;
+        {
+            float g0, g1;
+            upk2(gb2, g0, g1);
+            gb = g0 + g1;
         }
         if (MODE == 0) {      // gbar: the two halves of a row meet (all compute threads take part, aborted or not)
             red[half * 128 + lrow] = gb;
@@ -611,7 +688,7 @@ int launch_t(const BwdTensorArgs& a, int which) {
     const int BH = a.B * a.H, kvg = a.kv_group > 0 ? a.kv_group : 1, KVU = BH / kvg;
     BtParams p = {};
     p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.has_glo = a.gl != nullptr; p.scale = a.scale;
-    p.stats = a.stats; p.rowsc = a.rowsc; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
+    p.stats = a.stats; p.pairsc = a.pairsc; p.npair = (a.n + 1) / 2; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
     p.kbar = a.kbar; p.hvec = a.hvec; p.dq = a.dq; p.dk = a.dk; p.dv = a.dv; p.status = a.status;
     p.wait_clocks = kWaitClocks;
     const void* gl = a.gl ? a.gl : a.gh;        // a valid map either way; never loaded without a lo half
@@ -622,7 +699,7 @@ int launch_t(const BwdTensorArgs& a, int which) {
                   make_map_bf16(&mQ, a.q, BH, a.n, D, 64) && make_map_bf16(&mYh, a.yh, BH, a.n, D, 64) &&
                   make_map_bf16(&mYl, a.yl, BH, a.n, D, 64) && make_map_bf16(&mTh, a.tnh, BH, a.n, D, 64) &&
                   make_map_bf16(&mTl, a.tnl, BH, a.n, D, 64) && make_map_bf16(&mGh, a.gh, BH, a.n, D, 64) &&
-                  make_map_bf16(&mGl, gl, BH, a.n, D, 64) && make_map_f32_rows(&mRS, a.rowsc, BH, a.n, 8, 64);
+                  make_map_bf16(&mGl, gl, BH, a.n, D, 64) && make_map_f32_rows(&mRS, a.pairsc, BH, (a.n + 1) / 2, 8, 32);
         if (!ok) return LLA_ERR_CUDA;
         LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_ktile_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
         const dim3 grid(BH, (a.n + 127) / 128);

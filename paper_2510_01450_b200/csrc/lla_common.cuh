@@ -156,12 +156,15 @@ struct BackwardArgs {
 };
 // The tensor-core kernels of the backward pass (lla_backward_tensor.cu).  Every array is contiguous [B, H (or the
 // key/value heads), n, d]; gh/gl, yh/yl, tnh/tnl are the upstream gradient, y and -t as bf16 pairs hi + lo (gl may
-// be null: a bf16 gradient has no lo half); rowsc holds eight floats per row: m, 1/omega (0: row not handled here),
-// gbar, kappa, kbar.y, kbar.t, -m log2(e), unused.
+// be null: a bf16 gradient has no lo half); rowsc is the per-row record of the CUDA-core kernels, of which the
+// moments kernel fills gbar (slot 2); pairsc [heads][ceil(n / 2)][8] holds the scalars of two consecutive rows a, b
+// per record: (nm2_a, nm2_b, ky_a, ky_b, gk_a, gk_b, kk_a, kk_b) with nm2 = -(m log2 e + log2 omega) (-1e30: the row
+// is not handled by these kernels), ky = kbar.y, gk = gbar - kbar.t, kk = kbar.t - kappa.
 struct BwdTensorArgs {
     const void *q, *k, *v;
     const void *gh, *gl, *yh, *yl, *tnh, *tnl;
     float* rowsc;
+    const float* pairsc;
     const float* stats;
     const float* yvec;
     const float* tvec;

@@ -150,10 +150,10 @@ def test_validation_of_the_position_options(lib):
     assert bwd(workspace=0x10010) == 3             # not 256-byte aligned
     assert bwd(kv_heads=3) == 1
     assert bwd(impl=7) == 1
-    # the pass's own fp32 vectors and row records, six bf16 operand arrays (y, -t and the upstream gradient as hi + lo
+    # the pass's own fp32 vectors and row records (8 + 4 floats a row), six bf16 operand arrays (y, -t and the upstream gradient as hi + lo
     # pairs), then the scratch of the forward's CG kernel that it runs: fp16 copy of k + a status word, Gram sums and
     # preconditioner matrices per block of 128 keys (2 blocks, 4 heads)
-    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == (4 * 4 * 256 * (4 * 64 + 8) + 6 * 4 * 256 * 64 * 2
+    assert binding.lla_backward_workspace_bytes(1, 4, 256, 64) == (4 * 4 * 256 * (4 * 64 + 8 + 4) + 6 * 4 * 256 * 64 * 2
                                                                   + 4 * 256 * 64 * 2 + 256
                                                                   + 4 * 2 * (64 * 64 + 64) * 4 + 4 * 2 * 64 * 64 * 2)
 
