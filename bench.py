@@ -408,13 +408,16 @@ def run_ours(args):
     if rank == 0 and not args.no_decode:
         decode, cl = bench_decode(L, torch, peaks, head.sp, head.stream, local)
         samplers.append(cl)
-    backward3 = None
+    backward3 = backward4 = None
     if rank == 0 and not args.no_backward:
         bw_obj = leg_objs.get(2) or Prefill(L, torch, inputs.CONFIGS[2], local)
         backward, cl = bench_backward(L, torch, peaks, bw_obj, local)
         samplers.append(cl)
-        if 3 in leg_objs:      # the n = 4096 workload as well, where the pair kernel dominates the pass
+        if 3 in leg_objs:      # the n = 4096 workload as well, where the pair kernels dominate the pass
             backward3, cl = bench_backward(L, torch, peaks, leg_objs[3], local, steps=10, nsets=2)
+            samplers.append(cl)
+        if head.w.name == inputs.CONFIGS[HEADLINE].name:      # and the headline workload (d = 128)
+            backward4, cl = bench_backward(L, torch, peaks, head, local, steps=4, warmup=3, nsets=2)
             samplers.append(cl)
 
     tokens_step = w.B * w.n
@@ -446,6 +449,8 @@ def run_ours(args):
         line["backward"] = backward
     if backward3 is not None:
         line["backward_cfg3"] = backward3
+    if backward4 is not None:
+        line["backward_cfg4"] = backward4
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"], parity[f"cfg{args.workload}"] = cpu_baseline(head, 15.0)
@@ -494,7 +499,7 @@ def bench_decode(L, torch, peaks, sp, stream, local, steps=30, warmup=5):
 
 
 def bench_backward(L, torch, peaks, pre, local, steps=20, warmup=3, nsets=4):
-    """Backward pass (gradients with respect to q, k, v) on the n=1024, d=64 prefill workload: the forward
+    """Backward pass (gradients with respect to q, k, v) on the prefill workload of `pre`: the forward
     runs once per input set outside the timed region to save rho, stats and the fp32 output; the timed steps
     are lla_backward_ex alone, rotating over nsets sets of inputs and saved tensors (together larger than L2)."""
     w, sp, stream = pre.w, pre.sp, pre.stream
@@ -542,7 +547,7 @@ def bench_backward(L, torch, peaks, pre, local, steps=20, warmup=3, nsets=4):
             "tflops": flops / (ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "cg_mean_iters": float(it[it >= 0].mean()) if (it >= 0).any() else 0.0,
-            "algorithmic_flops_per_step": flops, "gpu_launches_per_step": 5,
+            "algorithmic_flops_per_step": flops, "gpu_launches_per_step": 8,
             "sm_mhz": c["sm_mhz"], "ms_x_mhz": ms * c["sm_mhz"] if c["sm_mhz"] else None,
             "l2": f"inputs and saved tensors rotate over {nsets} sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)",
             "inputs": "bf16 q, k, v; fp32 upstream gradient, forward output, rho, stats; fp32 gradients"}, clk
