@@ -73,7 +73,9 @@ enum {
     LLA_STATUS_BAD_PIVOT = 1,    /* directly-solved rows whose Cholesky met a pivot <= 0 */
     LLA_STATUS_TIMEOUT = 2,      /* bounded waits that expired (0 in a healthy run) */
     LLA_STATUS_ITER_SUM = 3,     /* low 31 bits of the sum over CG rows of iterations executed */
-    LLA_STATUS_WORDS = 4
+    LLA_STATUS_BOUNDS = 4,       /* debug build only (liblla_debug.so): stores skipped because their index was out of range */
+    LLA_STATUS_BOUNDS_SITE = 5,  /* debug build only: id of the first such store (0: none) */
+    LLA_STATUS_WORDS = 8
 };
 
 /*

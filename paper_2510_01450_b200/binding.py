@@ -8,17 +8,19 @@ call raises, telling how to build it.
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 
 _PKG = Path(__file__).resolve().parent
-_LIB_PATH = _PKG / "liblla.so"
+# LLA_LIBRARY selects another build of the same library (the bounds-checking debug build, liblla_debug.so)
+_LIB_PATH = Path(os.environ["LLA_LIBRARY"]) if os.environ.get("LLA_LIBRARY") else _PKG / "liblla.so"
 _lib = None
 
 LLA_BF16, LLA_F32 = 0, 1
 LLA_IMPL_AUTO, LLA_IMPL_SIMT, LLA_IMPL_TENSOR = 0, 1, 2
-LLA_STATUS_WORDS = 4
+LLA_STATUS_WORDS = 8
 LLA_PHASE_ALL, LLA_PHASE_DIRECT, LLA_PHASE_ITERATIVE = 0, 1, 2
-STATUS_ROWS_AT_CAP, STATUS_BAD_PIVOT, STATUS_TIMEOUT, STATUS_ITER_SUM = 0, 1, 2, 3
+STATUS_ROWS_AT_CAP, STATUS_BAD_PIVOT, STATUS_TIMEOUT, STATUS_ITER_SUM, STATUS_BOUNDS, STATUS_BOUNDS_SITE = 0, 1, 2, 3, 4, 5
 LLA_RIDGE_DEFINITION, LLA_RIDGE_PRINTED = 0, 1
 LLA_CG_PRECISE_ALL, LLA_CG_PRECISE_NONE = -1, -2
 LLA_DEBUG_NO_LOADS = 1

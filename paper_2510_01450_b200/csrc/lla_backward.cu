@@ -220,6 +220,7 @@ struct Pairs16 {
 // row i's four scalars go to slots s, 2 + s, 4 + s, 6 + s of record i / 2 (s = i & 1)
 __device__ __forceinline__ void store_pair_record(const Pairs16& p16, long long head, int i, float nm2, float ky, float gk, float kk) {
     float* rp = p16.pairsc + ((size_t)head * p16.npair + (i >> 1)) * 8 + (i & 1);
+    if (!LLA_IN_BOUNDS(i >> 1, p16.npair, nullptr, 601)) return;
     rp[0] = nm2; rp[2] = ky; rp[4] = gk; rp[6] = kk;
 }
 template <int D>
@@ -478,6 +479,7 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int bh = blockIdx.x;
     const int i = gridDim.y - 1 - blockIdx.y;       // rows with the most keys first
     const int L = i + 1;
+    if (!LLA_IN_BOUNDS(L, lcap + 1, status, 602)) return;      // (debug build: the keys must fit the arrays sized for lcap)
     const size_t base = (size_t)bh * n;
     const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
     for (int c = tid; c < D; c += HB_THREADS) {

@@ -310,17 +310,18 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             tc_fence_after();
             // (added, not stored: the directly-solved rows add their share from another stream, grouped heads theirs)
             const size_t rowoff = ((size_t)kvu * n + gj) * D + half * (D / 2);
+            const bool inb = gj >= n || LLA_IN_BOUNDS((size_t)kvu * n + gj, (size_t)(gridDim.x / prm.kv_group) * n, prm.status, 702);
 #pragma unroll 1
             for (int cb = 0; cb < D / 2; cb += 32) {
                 uint32_t v[32];
                 tmem_ld32(tm_lane + Cfg::C_DK + half * (D / 2) + cb, v);
                 tc_wait_ld();
-                if (gj < n)
+                if (gj < n && inb)
 #pragma unroll
                     for (int e = 0; e < 32; ++e) atomicAdd(prm.dk + rowoff + cb + e, __uint_as_float(v[e]));
                 tmem_ld32(tm_lane + Cfg::C_DV + half * (D / 2) + cb, v);
                 tc_wait_ld();
-                if (gj < n)
+                if (gj < n && inb)
 #pragma unroll
                     for (int e = 0; e < 32; ++e) atomicAdd(prm.dv + rowoff + cb + e, __uint_as_float(v[e]));
             }
@@ -512,8 +513,8 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int quad = warp & 3, half = warp >> 2;
         const int lrow = quad * 32 + lane;            // query row inside the tile == TMEM lane
         const int gi = i0 + lrow;
-        const bool okr = gi < n && gi >= prm.first;
         const size_t row = (size_t)bh * n + gi;
+        const bool okr = gi < n && gi >= prm.first && LLA_IN_BOUNDS(row, (size_t)gridDim.x * n, prm.status, 701);
         const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
         const float c1 = prm.scale * BT_LOG2E;
         // per-row scalars (see bwd_rowprep_kernel): p = 2^(c1 s + nm2) carries 1 / omega; a row that is switched off

@@ -12,6 +12,27 @@ namespace lla {
 // ---------------------------------------------------------------------------------------------
 // Launch arguments handed from the C-ABI layer to the kernel launchers (plain pointers + sizes).
 // ---------------------------------------------------------------------------------------------
+// Debug build (-DLLA_DEBUG_BOUNDS, liblla_debug.so): the kernels' global stores check their row or record index
+// against the extent that the launch geometry implies; a failed check counts in LLA_STATUS_BOUNDS, leaves the id
+// of the first failing site in LLA_STATUS_BOUNDS_SITE and skips the store (no trap, the context stays usable).
+// In the product build the macro is the constant `true`.
+// ---------------------------------------------------------------------------------------------
+#ifdef LLA_DEBUG_BOUNDS
+__device__ __forceinline__ bool in_bounds(unsigned long long idx, unsigned long long limit, int* status, int site) {
+    if (idx < limit) return true;
+    if (status) {
+        atomicAdd(status + LLA_STATUS_BOUNDS, 1);
+        atomicCAS(status + LLA_STATUS_BOUNDS_SITE, 0, site);
+    }
+    return false;
+}
+#define LLA_IN_BOUNDS(idx, limit, status, site) \
+    ::lla::in_bounds((unsigned long long)(idx), (unsigned long long)(limit), (status), (site))
+#else
+#define LLA_IN_BOUNDS(idx, limit, status, site) true
+#endif
+
+// ---------------------------------------------------------------------------------------------
 // (batch, query head) unit -> (batch, key/value head) unit when `group` query heads share one K/V head
 __host__ __device__ __forceinline__ int kv_unit(int bh, int H, int group) {
     return group <= 1 ? bh : (bh / H) * (H / group) + (bh % H) / group;

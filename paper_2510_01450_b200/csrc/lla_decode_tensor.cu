@@ -519,6 +519,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (prm.splits > 1 || prm.defer) {
         // partial record for the solve kernel: M, N, a, c, omega, m (same layout as the SIMT path)
+        if (!LLA_IN_BOUNDS((size_t)bh * prm.splits + part, (size_t)gridDim.y * prm.splits, prm.status, 501)) return;
         float* dst = prm.parts + ((size_t)bh * prm.splits + part) * (2 * 64 * 64 + 2 * 64 + 4);
         if (warp < 4) {
             float* rowp = dst + (size_t)tid * 64;                 // tid < 64: M rows; 64..127: N rows

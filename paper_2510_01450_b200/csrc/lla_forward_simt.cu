@@ -269,6 +269,7 @@ forward_simt_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const 
     if (row_ok) {
         const float inv_den = 1.f / den;
         const size_t rowi = (size_t)bh * nq + row;
+        if (!LLA_IN_BOUNDS(rowi, (size_t)gridDim.x * nq, status, 301)) return;
         TOut* orow = out + so.at(bh / H, bh % H, row);
 #pragma unroll
         for (int g = 0; g < NGV; ++g) {

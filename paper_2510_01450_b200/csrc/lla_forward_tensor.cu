@@ -943,7 +943,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // ---- output sweep ----
         float gfac = 1.f;
         if (ok && prm.sol) {
-            if (row_ok) {
+            if (row_ok && LLA_IN_BOUNDS((size_t)bh * nq + row, (size_t)gridDim.x * nq, prm.status, 101)) {
                 const size_t rowi = (size_t)bh * nq + row;
 #pragma unroll
                 for (int e = 0; e < NCOL; ++e) prm.sol[rowi * D + c0 + e] = xs[(c0 + e) * TC_BR + lrow];
@@ -983,7 +983,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 float o[NCOL];
                 acc_load(o);
                 den = pair_sum(part);
-                if (row_ok) {
+                if (row_ok && LLA_IN_BOUNDS((size_t)bh * nq + row, (size_t)gridDim.x * nq, prm.status, 102)) {
                     const float inv_den = 1.f / den;
                     const size_t rowi = (size_t)bh * nq + row;
                     TOut* orow = out + prm.so.at(bh / prm.H, bh % prm.H, row) + c0;

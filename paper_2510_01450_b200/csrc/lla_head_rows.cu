@@ -125,6 +125,8 @@ head_rows_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn
         if (L > lcap) return;               // long caches go through the moment kernel
     }
     const size_t row = lens ? (size_t)bh : (size_t)bh * nq + i;      // row of the contiguous per-row outputs (rho, stats, ...)
+    // (debug build: the keys must fit the shared-memory arrays sized for lcap, the row the per-row outputs)
+    if (!LLA_IN_BOUNDS(L, lcap + 1, status, 201) || !LLA_IN_BOUNDS(row, (size_t)gridDim.x * (lens ? 1 : nq), status, 202)) return;
     // prefill: q, k, v and out are addressed through their strides; decode keeps its contiguous / paged layout
     const TIn* qrow = lens ? q + row * D : q + sq.at(bh / H, bh % H, i);
     // (decode over a paged cache: the at most lcap <= page_size keys of a directly-solved unit sit in its first page)

@@ -42,7 +42,7 @@ def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IM
     grads = [torch.full(shape, float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
     nbytes = L.lla_backward_workspace_bytes(w.B, w.H, w.n, w.d)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
     L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, *grads, w.B, w.H, w.n, w.d, w.scale, w.lam,
                       out_dtype=LLA_DT[out_dtype], dout_dtype=LLA_DT[dout_dtype], device_status=status,
                       workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), impl=impl, **kw)
