@@ -29,8 +29,10 @@ import numpy as np
 import torch
 
 
-def _forward_rows(Q, K, V, rows, scale, lam, causal):
-    """o_i for the given row indices of one head, from the definition (float64 tensors)."""
+def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0):
+    """o_i for the given row indices of one head, from the definition (float64 tensors).  window > 0 (causal only):
+    row i sees its last `window` positions, keys max(0, i - window + 1) .. i (the sliding window that the paper's
+    discussion section suggests; the sums of Eq. "query_specific" then run over those keys)."""
     n = K.shape[0]
     d = K.shape[1]
     L = int(rows.max()) + 1 if causal else n
@@ -39,6 +41,8 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal):
     s = scale * (Qr @ Kl.T)                                        # scores, Section 3.1
     if causal:
         mask = torch.arange(L)[None, :] <= rows[:, None]           # row i sees keys j <= i
+        if window > 0:
+            mask = mask & (torch.arange(L)[None, :] > rows[:, None] - window)
     else:
         mask = torch.ones(len(rows), L, dtype=torch.bool)
     m = torch.where(mask, s, torch.full_like(s, -torch.inf)).max(dim=1).values.detach()
@@ -52,7 +56,7 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal):
     return (c @ Vl) / c.sum(dim=1, keepdim=True)                   # Eq. "lla"
 
 
-def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False):
+def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, window=0):
     """Gradients of sum_i <g_i, o_i> with respect to q, k, v.
 
     q, k: [B, H, n, d]; v, g: [B, H, n, dv]; numpy arrays (any float dtype; widened to float64).
@@ -73,7 +77,8 @@ def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False):
             lam_rows = torch.full((n,), float(lam), dtype=torch.float64, requires_grad=True)
             for r0 in range(0, n, chunk):
                 rows = torch.arange(r0, min(n, r0 + chunk))
-                o = _forward_rows(Q, K, V, rows, float(scale), lam_rows if want_dlambda else float(lam), bool(causal))
+                o = _forward_rows(Q, K, V, rows, float(scale), lam_rows if want_dlambda else float(lam), bool(causal),
+                                  int(window))
                 (o * G[rows]).sum().backward()
             dq[b, h], dk[b, h], dv[b, h] = Q.grad.numpy(), K.grad.numpy(), V.grad.numpy()
             if want_dlambda:
@@ -81,7 +86,7 @@ def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False):
     return (dq, dk, dv, dlam) if want_dlambda else (dq, dk, dv)
 
 
-def forward(q, k, v, scale, lam, causal=True, chunk=32):
+def forward(q, k, v, scale, lam, causal=True, chunk=32, window=0):
     """The forward values the gradient above differentiates (used by the pins to tie this module's
     forward to the C oracle's)."""
     q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
@@ -94,5 +99,5 @@ def forward(q, k, v, scale, lam, causal=True, chunk=32):
                 for r0 in range(0, n, chunk):
                     rows = torch.arange(r0, min(n, r0 + chunk))
                     out[b, h, r0:r0 + len(rows)] = _forward_rows(Q, K, V, rows, float(scale), float(lam),
-                                                                 bool(causal)).numpy()
+                                                                 bool(causal), int(window)).numpy()
     return out

@@ -7,6 +7,8 @@ by mathematics, none of it by the CUDA path.
   (d) lambda -> infinity: the gradient tends to the textbook softmax-attention gradient, error ~ 1/lambda
   (e) a single token: o_0 = v_0 for every lambda > 0, so dQ = dK = 0 and dV = g
   (f) the hand-derived formulas of the paper's backward appendix, evaluated literally in numpy
+  (g) sliding window: the windowed forward is the C oracle's forward of each row's own key range, and the windowed
+      gradient is the finite difference of that
 """
 import numpy as np
 import pytest
@@ -144,3 +146,44 @@ def test_ridge_gradient_by_finite_differences_of_c_oracle():
         assert abs(num - dlam[0, 0, i]) <= 1e-6 * max(1.0, abs(num)), i
     # the first row's output is v_0 for every positive ridge: no dependence on lambda
     assert abs(dlam[0, 0, 0]) <= 1e-12
+
+
+def _windowed_forward_by_c_oracle(q, k, v, scale, lam, window):
+    """Row i of a sliding-window forward is the last row of a plain causal forward over keys i - window + 1 .. i
+    alone (the C oracle knows no window): the definition of the window, evaluated row by row."""
+    B, H, n, _ = q.shape
+    out = np.zeros(v.shape)
+    for i in range(n):
+        lo = max(0, i - window + 1)
+        sl = slice(lo, i + 1)
+        qq = np.repeat(q[:, :, i:i + 1], i + 1 - lo, axis=2)          # only the last row's query matters
+        out[:, :, i] = fwd_c.forward(qq, k[:, :, sl], v[:, :, sl], scale, lam)[:, :, -1]
+    return out
+
+
+def test_sliding_window_forward_and_finite_differences():
+    n, d, dv, scale, lam, window = 9, 3, 2, 0.6, 5e-2, 4
+    q, k, v, g = _inputs(8, n, d, dv)
+    ref = _windowed_forward_by_c_oracle(q, k, v, scale, lam, window)
+    assert np.abs(bwd.forward(q, k, v, scale, lam, window=window) - ref).max() <= 1e-9 * np.abs(ref).max()
+    assert np.abs(bwd.forward(q, k, v, scale, lam, window=n) - bwd.forward(q, k, v, scale, lam)).max() == 0.0
+    dq, dk, dv_ = bwd.backward(q, k, v, g, scale, lam, window=window)
+    full = bwd.backward(q, k, v, g, scale, lam)
+    assert np.abs(dk - full[1]).max() > 1e-3          # the window changes the gradient (the pin below is not vacuous)
+
+    def loss(q_, k_, v_):
+        return float((_windowed_forward_by_c_oracle(q_, k_, v_, scale, lam, window) * g).sum())
+
+    eps = 1e-5
+    for name, x, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv_)):
+        num = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps
+            xm[idx] -= eps
+            ap = {"q": q, "k": k, "v": v, name: xp}
+            am = {"q": q, "k": k, "v": v, name: xm}
+            num[idx] = (loss(ap["q"], ap["k"], ap["v"]) - loss(am["q"], am["k"], am["v"])) / (2 * eps)
+        assert np.abs(num - grad).max() <= 2e-7 * max(1.0, np.abs(grad).max()), name
