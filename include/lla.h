@@ -353,8 +353,8 @@ int lla_decode_default_splits(int B, int H, int Lmax);
  *               taken from it; a bf16 `out` limits the accuracy of dq and dk to its rounding
  *   dout      : [B, H, n, d] g, dout_dtype (LLA_BF16 or LLA_F32)
  *   rho, stats: [B, H, n, d] and [B, H, n, 3] fp32, written by lla_forward_ex for the same inputs,
- *               scale, lambda and head_rows (a plain causal forward: no window, q_rows = n, the ridge of
- *               the definition; the call cannot tell and would return the gradient of that forward)
+ *               scale, lambda, head_rows and window (a causal forward with q_rows = n and the ridge of the
+ *               definition; the call cannot tell and would return the gradient of that forward)
  *   dq, dk, dv: [B, H, n, d] fp32 on the device, overwritten
  *   max_iters, tol, head_rows : as in lla_forward_params (0 = defaults)
  *   device_status : optional int[LLA_STATUS_WORDS], zeroed by the call
@@ -390,6 +390,8 @@ typedef struct lla_backward_params {
     int impl;     /* LLA_IMPL_AUTO: moments and pair kernels on the tensor cores; LLA_IMPL_SIMT: on the CUDA cores */
     int kv_heads; /* as in lla_forward_params: k, v, dk, dv are [B, kv_heads, n, d]; a key/value head's gradient
                      sums over the query heads that read it */
+    int window;   /* as in lla_forward_params: the forward being differentiated ran with this causal sliding window
+                     (0: none).  At least head_rows, and not with impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED otherwise */
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -388,6 +388,10 @@ int lla_backward_ex(const lla_backward_params* p) {
     a.dlambda = p->dlambda;
     if (p->kv_heads < 0 || (p->kv_heads > 0 && p->H % p->kv_heads != 0)) return LLA_ERR_INVALID_ARG;
     a.kv_group = p->kv_heads > 0 ? p->H / p->kv_heads : 1;
+    if (p->window < 0) return LLA_ERR_INVALID_ARG;
+    // as in the forward, the window must leave the directly-solved rows whole; the CUDA-core kernels know no window
+    if (p->window > 0 && (p->window < a.head_rows || a.cuda_core_pairs)) return LLA_ERR_UNSUPPORTED;
+    a.window = p->window;
     SideStream* side = side_stream();
     std::unique_lock<std::mutex> side_lock;
     if (side) {

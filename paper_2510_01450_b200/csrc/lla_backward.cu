@@ -695,7 +695,7 @@ int launch_t(const BackwardArgs& a) {
             }
             t.rowsc = rowsc; t.pairsc = pairsc; t.stats = a.stats; t.yvec = yvec; t.tvec = tvec;
             t.kbar = kbar; t.hvec = hvec; t.dq = a.dq; t.dk = a.dk; t.dv = a.dv;
-            t.B = a.B; t.H = a.H; t.n = a.n; t.d = D; t.first = first; t.kv_group = kvg;
+            t.B = a.B; t.H = a.H; t.n = a.n; t.d = D; t.first = first; t.kv_group = kvg; t.window = a.window;
             t.scale = a.scale; t.status = a.status; t.stream = a.stream;
             const int rc = launch_backward_tensor(t, 0);
             if (rc != LLA_OK) return rc;
@@ -714,7 +714,7 @@ int launch_t(const BackwardArgs& a) {
         f.scale = a.scale; f.lambda = a.lambda; f.causal = 1;
         f.max_iters = a.max_iters; f.tol = a.tol; f.head_rows = a.head_rows;
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
-        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg;
+        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg; f.window = a.window;
         f.rhs = hvec; f.sol = tvec;
         f.set_contiguous();
         // what the workspace holds beyond this pass's own arrays serves the solve (the fp16 copy of k; for

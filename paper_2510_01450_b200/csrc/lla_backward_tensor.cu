@@ -40,6 +40,7 @@ constexpr uint32_t BT_IDESC_SS = make_idesc(128, 64, 0, 0);       // score tiles
 
 struct BtParams {
     int n, first, H, kv_group;
+    int window;           // causal sliding window (0: none): a row sees its last `window` positions
     int has_glo;          // the upstream gradient has a lo half (fp32 dout)
     float scale;
     const float* stats;   // [rows][3] saved by the forward
@@ -121,7 +122,11 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int kvu = kv_unit(bh, prm.H, prm.kv_group);
     const int n = prm.n;
     const int j0 = blockIdx.y * 128;          // key tile 0 sees the most query rows and starts first (heads fastest)
-    const int it0 = max(j0, prm.first) / 64, it1 = (n + 63) / 64;     // query steps of 64 rows
+    // query steps of 64 rows: from the tile's first key (or the first row these kernels handle) to the last row that
+    // still sees a key of the tile
+    const int W = prm.window;
+    const int last_row = W > 0 ? min(n - 1, j0 + 127 + W - 1) : n - 1;
+    const int it0 = max(j0, prm.first) / 64, it1 = last_row / 64 + 1;
     const int nstep = it1 - it0;
     const long long wcap = prm.wait_clocks;
     if (nstep <= 0) return;
@@ -255,11 +260,13 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
                 tmem_ld32(tm_lane + Cfg::C_E + col0, ev);
                 tc_wait_ld();
-                if (i0 < j0 + 128 || i0 + 64 > n) {      // a diagonal or last step: hide the pairs with j > i or i >= n
+                if (i0 < j0 + 128 || i0 + 64 > n || (W > 0 && i0 + 63 - j0 >= W)) {
+                    // a diagonal or last step, or one that reaches past the window: hide the pairs with j > i, i >= n
+                    // or i - j >= window
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const int gi = i0 + (int)col0 + e;
-                        if (gj > gi || gi >= n) sv[e] = __float_as_uint(-1e30f);
+                        if (gj > gi || gi >= n || (W > 0 && gi - gj >= W)) sv[e] = __float_as_uint(-1e30f);
                     }
                 }
 #pragma unroll
@@ -385,7 +392,11 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int tile = gridDim.y - 1 - blockIdx.y;      // longest tiles first, heads fastest
     const int i0 = tile * 128;
     if (i0 + 128 <= prm.first) return;                // every row of the tile is solved directly
-    const int nblk = (min(n, i0 + 128) + 63) / 64;
+    // key blocks [cbeg, cend): with a sliding window the loop starts at the block of the first row's first visible key
+    const int W = prm.window;
+    const int cend = (min(n, i0 + 128) + 63) / 64;
+    const int cbeg = W > 0 ? max(0, i0 + 1 - W) / 64 : 0;
+    const int nblk = cend - cbeg;
     const long long wcap = prm.wait_clocks;
     // Stages of the K/V ring.  d = 128: the tiles that stay for the whole block leave room for one stage; where the
     // upstream gradient has no lo half (bf16), that half's tile is a second one.  The moments kernel has no T tiles.
@@ -444,8 +455,8 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const uint32_t st = sbase + stage_base(s), fb = bar(QB_FULL + s);
                 mbar_expect_tx(fb, STAGE);
                 for (int sub = 0; sub < KSUB; ++sub) {
-                    tma_load_3d(st + sub * 8192, &tmK, fb, 64 * sub, 64 * c, kvu);
-                    tma_load_3d(st + T64 + sub * 8192, &tmV, fb, 64 * sub, 64 * c, kvu);
+                    tma_load_3d(st + sub * 8192, &tmK, fb, 64 * sub, 64 * (cbeg + c), kvu);
+                    tma_load_3d(st + T64 + sub * 8192, &tmV, fb, 64 * sub, 64 * (cbeg + c), kvu);
                 }
                 issued = c + 1;
             }
@@ -564,11 +575,13 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 uint32_t sv[32];
                 tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
                 tc_wait_ld();
-                const int jlim = gi + 1 - (64 * c + (int)col0);      // keys e < jlim are visible
-                if (jlim < 32) {
+                const int key0 = 64 * (cbeg + c) + (int)col0;
+                const int jlim = gi + 1 - key0;                           // keys jfirst <= e < jlim are visible
+                const int jfirst = W > 0 ? gi + 1 - W - key0 : 0;
+                if (jlim < 32 || jfirst > 0) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
-                        if (e >= jlim) sv[e] = __float_as_uint(-1e30f);
+                        if (e >= jlim || e < jfirst) sv[e] = __float_as_uint(-1e30f);
                 }
 #pragma unroll
                 for (int e2 = 0; e2 < 16; ++e2) p2[e2] = ex2_2(fma2(pku(sv[2 * e2], sv[2 * e2 + 1]), c1c1, nm22));
@@ -688,7 +701,7 @@ template <int D>
 int launch_t(const BwdTensorArgs& a, int which) {
     const int BH = a.B * a.H, kvg = a.kv_group > 0 ? a.kv_group : 1, KVU = BH / kvg;
     BtParams p = {};
-    p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.has_glo = a.gl != nullptr; p.scale = a.scale;
+    p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.window = a.window; p.has_glo = a.gl != nullptr; p.scale = a.scale;
     p.stats = a.stats; p.pairsc = a.pairsc; p.npair = (a.n + 1) / 2; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
     p.kbar = a.kbar; p.hvec = a.hvec; p.dq = a.dq; p.dk = a.dk; p.dv = a.dv; p.status = a.status;
     p.wait_clocks = kWaitClocks;

@@ -172,6 +172,7 @@ struct BackwardArgs {
     cudaStream_t stream;
     int kv_group;               // query heads per key/value head (k, v, dk, dv are [B, H / kv_group, n, d])
     int cuda_core_pairs;        // 1: pair kernel on the CUDA cores even where the tensor-core one exists
+    int window;                 // causal sliding window of the forward being differentiated (0: none)
     cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
     cudaEvent_t fork, join;
 };
@@ -191,6 +192,7 @@ struct BwdTensorArgs {
     const float* tvec;
     float *kbar, *hvec, *dq, *dk, *dv;
     int B, H, n, d, first, kv_group;
+    int window;     // causal sliding window (0: none)
     float scale;
     int* status;
     cudaStream_t stream;

@@ -30,7 +30,7 @@ def grad_err(got, ref):
     return diff / np.maximum(rn, max(0.1 * float(np.median(rn)), 1e-4))
 
 
-def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IMPL_AUTO, **kw):
+def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IMPL_AUTO, window=0, **kw):
     dq_, dk_, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
     dg = dev(g, dout_dtype)
     shape = (w.B, w.H, w.n, w.d)
@@ -38,14 +38,14 @@ def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IM
     rho = torch.empty(shape, dtype=torch.float32, device="cuda")
     stats = torch.empty((w.B, w.H, w.n, 3), dtype=torch.float32, device="cuda")
     L.lla_forward_ex(dq_, dk_, dv_, out, w.B, w.H, w.n, w.d, w.d, w.scale, w.lam, in_dtype=L.LLA_BF16,
-                     out_dtype=LLA_DT[out_dtype], rho=rho, stats=stats, stream=stream_ptr())
+                     out_dtype=LLA_DT[out_dtype], rho=rho, stats=stats, stream=stream_ptr(), window=window)
     grads = [torch.full(shape, float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
     nbytes = L.lla_backward_workspace_bytes(w.B, w.H, w.n, w.d)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
     L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, *grads, w.B, w.H, w.n, w.d, w.scale, w.lam,
                       out_dtype=LLA_DT[out_dtype], dout_dtype=LLA_DT[dout_dtype], device_status=status,
-                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), impl=impl, **kw)
+                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), impl=impl, window=window, **kw)
     torch.cuda.synchronize()
     st = status.cpu().numpy()
     assert st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
@@ -151,6 +151,23 @@ def test_backward_grouped_kv_heads(backward_oracle, d, impl):
         assert err.max() <= TOL, (name, float(err.max()))
 
 
+@pytest.mark.parametrize("d,n,window", [(64, 700, 200), (64, 520, 96), (128, 600, 256)])
+def test_backward_sliding_window(backward_oracle, d, n, window):
+    # the gradient of the forward with a causal sliding window (the variant the paper's discussion suggests): the
+    # query tiles start at the block of their first visible key, the key tiles stop at their last viewer
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=n, d=d, dv=d, seed=290 + d)
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam, window=window)
+    got = run_backward(w, q, k, v, g, window=window)
+    for name, a, b in zip(("dq", "dk", "dv"), got, ref):
+        assert np.isfinite(a).all(), name
+        err = grad_err(a, b)
+        assert err.max() <= TOL, (name, float(err.max()), int(err.argmax()))
+    full = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
+    assert grad_err(got[1], full[1]).max() > 10 * TOL        # (the window matters at these sizes)
+
+
 def test_backward_dq_is_bit_identical_between_runs():
     # dq comes from plain stores of the query tile that owns the rows (and of one block per directly-solved row), so
     # two runs give the same bits; dk and dv are summed atomically and only agree to rounding
@@ -162,6 +179,16 @@ def test_backward_dq_is_bit_identical_between_runs():
     assert np.array_equal(a[0], b[0])
     for x, y in zip(a[1:], b[1:]):
         assert np.abs(x - y).max() <= 1e-5 * np.abs(x).max()
+
+
+def test_backward_window_argument_checks():
+    ok = 0x1000
+    ws = torch.empty(L.lla_backward_workspace_bytes(1, 1, 256, 64), dtype=torch.uint8, device="cuda")
+    for kw in (dict(window=50), dict(window=128, impl=L.LLA_IMPL_SIMT)):      # below head_rows; CUDA-core kernels
+        with pytest.raises(L.LlaError) as e:
+            L.lla_backward_ex(ok, ok, ok, ok, ok, ok, ok, ok, ok, ok, 1, 1, 256, 64, 0.125, 1e-3, workspace=ws,
+                              workspace_bytes=ws.numel(), **kw)
+        assert e.value.status == 2
 
 
 def test_backward_argument_checks():
