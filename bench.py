@@ -541,12 +541,24 @@ def bench_backward(L, torch, peaks, pre, local, steps=20, warmup=3, nsets=4):
         e1.record(stream)
         torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
+    # the same steps with the extra solve preconditioned (optional mode, as in the forward)
+    step(0, iters=iters, cg_precondition=1)
+    torch.cuda.synchronize()
+    it_pc = iters.cpu().numpy().reshape(-1, w.n).astype(np.float64)
+    e0.record(stream)
+    for i in range(steps):
+        step(warmup + i, cg_precondition=1)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_pc = e0.elapsed_time(e1) / steps
     set_bytes = sum(t.numel() * t.element_size() for t in saved[0])
     c = clk.summary()
     return {"workload": w.name, "ms_per_step": ms, "tokens_per_s": w.B * w.n / (ms * 1e-3),
             "tflops": flops / (ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "cg_mean_iters": float(it[it >= 0].mean()) if (it >= 0).any() else 0.0,
+            "preconditioned": {"ms_per_step": ms_pc, "cg_mean_iters": float(it_pc[it_pc >= 0].mean()) if (it_pc >= 0).any() else 0.0,
+                               "note": "optional mode (lla_backward_params.cg_precondition = 1)"},
             "algorithmic_flops_per_step": flops, "gpu_launches_per_step": 8,
             "sm_mhz": c["sm_mhz"], "ms_x_mhz": ms * c["sm_mhz"] if c["sm_mhz"] else None,
             "l2": f"inputs and saved tensors rotate over {nsets} sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)",

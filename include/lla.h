@@ -363,10 +363,11 @@ int lla_decode_default_splits(int B, int H, int Lmax);
  * All pointers 16-byte aligned; no output may alias an input.  Work is enqueued on `stream`; the call
  * does not synchronise and keeps no pointer.
  * Reproducibility: dq is bit-identical from run to run (each query tile owns its rows and stores them; with
- * impl = LLA_IMPL_SIMT the key tiles add their shares atomically instead and it is not).  dk and dv are summed
- * with fp32 atomic adds -- the key tiles', the directly-solved rows' and, with grouped heads, every query head's
- * share -- whose order varies: those two outputs agree between runs to rounding (about 1e-6 relative), not bit
- * for bit.
+ * impl = LLA_IMPL_SIMT the key tiles add their shares atomically instead and it is not).  So are the rows of dk and
+ * dv from position 128 * ceil((head_rows - 1) / 128) on, unless heads are grouped: a key tile owns and stores them.
+ * The earlier rows also receive the directly-solved query rows' shares, and with grouped heads every row receives
+ * one share per query head of its group; those are summed with fp32 atomic adds, whose order varies, and agree
+ * between runs to rounding (about 1e-6 relative), not bit for bit.
  */
 typedef struct lla_backward_params {
     const void *q, *k, *v, *out, *dout;
@@ -392,6 +393,8 @@ typedef struct lla_backward_params {
                      sums over the query heads that read it */
     int window;   /* as in lla_forward_params: the forward being differentiated ran with this causal sliding window
                      (0: none).  At least head_rows, and not with impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED otherwise */
+    int cg_precondition; /* as in lla_forward_params: 1 = the extra solve runs the preconditioned conjugate gradients
+                     (about half the iterations; same result within the tolerance) */
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -392,6 +392,8 @@ int lla_backward_ex(const lla_backward_params* p) {
     // as in the forward, the window must leave the directly-solved rows whole; the CUDA-core kernels know no window
     if (p->window > 0 && (p->window < a.head_rows || a.cuda_core_pairs)) return LLA_ERR_UNSUPPORTED;
     a.window = p->window;
+    if (p->cg_precondition != 0 && p->cg_precondition != 1) return LLA_ERR_INVALID_ARG;
+    a.precondition = p->cg_precondition;
     SideStream* side = side_stream();
     std::unique_lock<std::mutex> side_lock;
     if (side) {

@@ -315,22 +315,31 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
         if (ok && mbar_wait(bar(KB_ACCFULL), 0, abort_flag, wcap)) {
             tc_fence_after();
-            // (added, not stored: the directly-solved rows add their share from another stream, grouped heads theirs)
+            // Key rows below `first` also get the directly-solved rows' shares (from another stream), and with grouped
+            // heads every query head of the group adds into the same rows: those are added atomically.  Any other
+            // row is this block's alone and is stored.
+            const bool plain = prm.kv_group == 1 && j0 >= prm.first;
             const size_t rowoff = ((size_t)kvu * n + gj) * D + half * (D / 2);
-            const bool inb = gj >= n || LLA_IN_BOUNDS((size_t)kvu * n + gj, (size_t)(gridDim.x / prm.kv_group) * n, prm.status, 702);
+            const bool inb = gj < n && LLA_IN_BOUNDS((size_t)kvu * n + gj, (size_t)(gridDim.x / prm.kv_group) * n, prm.status, 702);
 #pragma unroll 1
-            for (int cb = 0; cb < D / 2; cb += 32) {
-                uint32_t v[32];
-                tmem_ld32(tm_lane + Cfg::C_DK + half * (D / 2) + cb, v);
-                tc_wait_ld();
-                if (gj < n && inb)
+            for (int part = 0; part < 2; ++part) {
+                float* dst = (part == 0 ? prm.dk : prm.dv) + rowoff;
+#pragma unroll 1
+                for (int cb = 0; cb < D / 2; cb += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tm_lane + (part == 0 ? Cfg::C_DK : Cfg::C_DV) + half * (D / 2) + cb, v);
+                    tc_wait_ld();
+                    if (!inb) continue;
+                    if (plain) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) atomicAdd(prm.dk + rowoff + cb + e, __uint_as_float(v[e]));
-                tmem_ld32(tm_lane + Cfg::C_DV + half * (D / 2) + cb, v);
-                tc_wait_ld();
-                if (gj < n && inb)
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<float4*>(dst + cb + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                                                                   __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) atomicAdd(prm.dv + rowoff + cb + e, __uint_as_float(v[e]));
+                        for (int e = 0; e < 32; ++e) atomicAdd(dst + cb + e, __uint_as_float(v[e]));
+                    }
+                }
             }
         }
     }

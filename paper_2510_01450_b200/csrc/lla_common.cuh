@@ -173,6 +173,7 @@ struct BackwardArgs {
     int kv_group;               // query heads per key/value head (k, v, dk, dv are [B, H / kv_group, n, d])
     int cuda_core_pairs;        // 1: pair kernel on the CUDA cores even where the tensor-core one exists
     int window;                 // causal sliding window of the forward being differentiated (0: none)
+    int precondition;           // 1: the extra solve runs the preconditioned CG (as ForwardArgs::precondition)
     cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
     cudaEvent_t fork, join;
 };

@@ -168,6 +168,20 @@ def test_backward_sliding_window(backward_oracle, d, n, window):
     assert grad_err(got[1], full[1]).max() > 10 * TOL        # (the window matters at these sizes)
 
 
+def test_backward_with_preconditioned_solve(backward_oracle):
+    w = inputs.CONFIGS[2].shrink(B=1, H=2, n=640, seed=295)
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
+    its = [torch.full((w.B, w.H, w.n), -1, dtype=torch.int32, device="cuda") for _ in range(2)]
+    plain = run_backward(w, q, k, v, g, iters=its[0])
+    got = run_backward(w, q, k, v, g, iters=its[1], cg_precondition=1)
+    for name, a, b in zip(("dq", "dk", "dv"), got, ref):
+        assert grad_err(a, b).max() <= TOL, name
+    a, b = (t.cpu().numpy().ravel() for t in its)
+    assert b[b >= 0].mean() < 0.75 * a[a >= 0].mean()        # fewer iterations of the extra solve
+
+
 def test_backward_dq_is_bit_identical_between_runs():
     # dq comes from plain stores of the query tile that owns the rows (and of one block per directly-solved row), so
     # two runs give the same bits; dk and dv are summed atomically and only agree to rounding
