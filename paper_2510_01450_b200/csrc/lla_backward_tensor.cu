@@ -79,7 +79,11 @@ struct KtCfg {
     static constexpr int C_S = 0, C_E = 64, C_F = 128, C_G = 192, C_DK = 256, C_DV = 256 + D;
 };
 static_assert(KtCfg<64>::SM_ALLOC <= 227 * 1024 && KtCfg<128>::SM_ALLOC <= 227 * 1024, "shared memory budget");
-enum { KB_KV = 0, KB_FULL = 1, KB_EMPTY = 3, KB_SF1 = 5, KB_SF2 = 6, KB_PRA = 7, KB_PRB = 8, KB_ACCFULL = 9, KB_EXIT = 10, KB_COUNT = 11 };
+// A stage of the query-side ring is loaded and released in two halves: A = the T and G tiles (read last by the
+// products of a^T), B = the Q and Y tiles and the row records (read last by the products of ds^T and p1^T).
+enum { KB_KV = 0, KB_FULL_A = 1, KB_FULL_B = 3, KB_EMPTY_A = 5, KB_EMPTY_B = 7, KB_SF_SE = 9, KB_SF_FG = 10, KB_PRA = 11, KB_PRB = 12,
+       KB_ACCFULL = 13, KB_EXIT = 14, KB_COUNT = 15 };
+static_assert(KB_COUNT * 8 <= 128, "barrier area too small");
 
 // one MMA with the A operand in TMEM, predicated on the elected lane
 __device__ __forceinline__ void mma_ts1(uint32_t el, uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
@@ -134,11 +138,13 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (tid == 0) {
         mbar_init(bar(KB_KV), 1);
         for (int s = 0; s < NST; ++s) {
-            mbar_init(bar(KB_FULL + s), 1);
-            mbar_init(bar(KB_EMPTY + s), 1);
+            mbar_init(bar(KB_FULL_A + s), 1);
+            mbar_init(bar(KB_FULL_B + s), 1);
+            mbar_init(bar(KB_EMPTY_A + s), 1);
+            mbar_init(bar(KB_EMPTY_B + s), 1);
         }
-        mbar_init(bar(KB_SF1), 1);
-        mbar_init(bar(KB_SF2), 1);
+        mbar_init(bar(KB_SF_SE), 1);
+        mbar_init(bar(KB_SF_FG), 1);
         mbar_init(bar(KB_PRA), BT_COMPUTE / 32);
         mbar_init(bar(KB_PRB), BT_COMPUTE / 32);
         mbar_init(bar(KB_ACCFULL), 1);
@@ -164,27 +170,35 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 tma_load_3d(sbase + Cfg::SM_K + sub * 16384, &tmK, bar(KB_KV), 64 * sub, j0, kvu);
                 tma_load_3d(sbase + Cfg::SM_V + sub * 16384, &tmV, bar(KB_KV), 64 * sub, j0, kvu);
             }
-            int issued = 0;
+            int issued_a = 0, issued_b = 0;
             for (int g = 0; g < nstep; ++g) {
                 const int s = g % NST, i0 = 64 * (it0 + g);
-                if (!mbar_wait(bar(KB_EMPTY + s), ((g / NST) & 1) ^ 1, abort_flag, wcap)) break;
-                const uint32_t st = sbase + Cfg::SM_ST + s * STAGE, fb = bar(KB_FULL + s);
-                mbar_expect_tx(fb, (6 + (prm.has_glo ? 1 : 0)) * T64 + 1024);
+                const uint32_t st = sbase + Cfg::SM_ST + s * STAGE;
+                if (!mbar_wait(bar(KB_EMPTY_A + s), ((g / NST) & 1) ^ 1, abort_flag, wcap)) break;
+                const uint32_t fa = bar(KB_FULL_A + s);
+                mbar_expect_tx(fa, (3 + (prm.has_glo ? 1 : 0)) * T64);
+                for (int sub = 0; sub < KSUB; ++sub) {
+                    tma_load_3d(st + Cfg::ST_TH + sub * 8192, &tmTh, fa, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_TL + sub * 8192, &tmTl, fa, 64 * sub, i0, bh);
+                    tma_load_3d(st + Cfg::ST_GH + sub * 8192, &tmGh, fa, 64 * sub, i0, bh);
+                    if (prm.has_glo) tma_load_3d(st + Cfg::ST_GL + sub * 8192, &tmGl, fa, 64 * sub, i0, bh);
+                }
+                issued_a = g + 1;
+                if (!mbar_wait(bar(KB_EMPTY_B + s), ((g / NST) & 1) ^ 1, abort_flag, wcap)) break;
+                const uint32_t fb = bar(KB_FULL_B + s);
+                mbar_expect_tx(fb, 3 * T64 + 1024);
                 for (int sub = 0; sub < KSUB; ++sub) {
                     tma_load_3d(st + Cfg::ST_Q + sub * 8192, &tmQ, fb, 64 * sub, i0, bh);
                     tma_load_3d(st + Cfg::ST_YH + sub * 8192, &tmYh, fb, 64 * sub, i0, bh);
                     tma_load_3d(st + Cfg::ST_YL + sub * 8192, &tmYl, fb, 64 * sub, i0, bh);
-                    tma_load_3d(st + Cfg::ST_TH + sub * 8192, &tmTh, fb, 64 * sub, i0, bh);
-                    tma_load_3d(st + Cfg::ST_TL + sub * 8192, &tmTl, fb, 64 * sub, i0, bh);
-                    tma_load_3d(st + Cfg::ST_GH + sub * 8192, &tmGh, fb, 64 * sub, i0, bh);
-                    if (prm.has_glo) tma_load_3d(st + Cfg::ST_GL + sub * 8192, &tmGl, fb, 64 * sub, i0, bh);
                 }
                 tma_load_3d(st + Cfg::ST_RS, &tmRS, fb, 0, i0 / 2, bh);
-                issued = g + 1;
+                issued_b = g + 1;
             }
             if (*abort_flag) {      // an aborted block: what was issued must have landed before the block exits
                 (void)mbar_wait_landed(bar(KB_KV), 0, wcap);
-                for (int g = max(0, issued - NST); g < issued; ++g) (void)mbar_wait_landed(bar(KB_FULL + g % NST), (g / NST) & 1, wcap);
+                for (int g = max(0, issued_a - NST); g < issued_a; ++g) (void)mbar_wait_landed(bar(KB_FULL_A + g % NST), (g / NST) & 1, wcap);
+                for (int g = max(0, issued_b - NST); g < issued_b; ++g) (void)mbar_wait_landed(bar(KB_FULL_B + g % NST), (g / NST) & 1, wcap);
             }
         }
     } else if (warp == 9) {
@@ -196,8 +210,6 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint64_t kdesc = make_desc(sb_u + Cfg::SM_K), vdesc = make_desc(sb_u + Cfg::SM_V);
         for (int g = 0; g < nstep && ok; ++g) {
             const int s = g % NST;
-            if (!mbar_wait(bar(KB_FULL + s), (g / NST) & 1, abort_flag, wcap)) break;
-            tc_fence_after();
             const uint32_t st = sb_u + Cfg::SM_ST + s * STAGE;
             auto score = [&](uint32_t col, uint64_t adesc, int off, uint32_t acc) {
                 const uint64_t bdesc = make_desc(st + off);
@@ -205,16 +217,34 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 for (int sub = 0; sub < KSUB; ++sub)
                     mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
             };
-            // group 1: what a^T needs; group 2: the rest
-            score(Cfg::C_S, kdesc, Cfg::ST_Q, 0);
-            score(Cfg::C_E, kdesc, Cfg::ST_YH, 0);
-            score(Cfg::C_E, kdesc, Cfg::ST_YL, 1);
-            tc_commit_el(el, bar(KB_SF1));
-            score(Cfg::C_F, kdesc, Cfg::ST_TH, 0);
-            score(Cfg::C_F, kdesc, Cfg::ST_TL, 1);
-            score(Cfg::C_G, vdesc, Cfg::ST_GH, 0);
-            if (prm.has_glo) score(Cfg::C_G, vdesc, Cfg::ST_GL, 1);
-            tc_commit_el(el, bar(KB_SF2));
+            // Two groups of score products: (S, E), which a^T needs, and (F, Gamma).  With two stages (S, E) go
+            // first, so that a^T is formed while (F, Gamma) run.  With one stage (d = 128) the order is reversed: half A
+            // of the stage was released first by the previous step and lands first, and the wait for half B hides
+            // behind the products of half A.
+            auto group_se = [&]() -> bool {
+                if (!mbar_wait(bar(KB_FULL_B + s), (g / NST) & 1, abort_flag, wcap)) return false;
+                tc_fence_after();
+                score(Cfg::C_S, kdesc, Cfg::ST_Q, 0);
+                score(Cfg::C_E, kdesc, Cfg::ST_YH, 0);
+                score(Cfg::C_E, kdesc, Cfg::ST_YL, 1);
+                tc_commit_el(el, bar(KB_SF_SE));
+                return true;
+            };
+            auto group_fg = [&]() -> bool {
+                if (!mbar_wait(bar(KB_FULL_A + s), (g / NST) & 1, abort_flag, wcap)) return false;
+                tc_fence_after();
+                score(Cfg::C_F, kdesc, Cfg::ST_TH, 0);
+                score(Cfg::C_F, kdesc, Cfg::ST_TL, 1);
+                score(Cfg::C_G, vdesc, Cfg::ST_GH, 0);
+                if (prm.has_glo) score(Cfg::C_G, vdesc, Cfg::ST_GL, 1);
+                tc_commit_el(el, bar(KB_SF_FG));
+                return true;
+            };
+            if (NST > 1) {
+                if (!group_se() || !group_fg()) break;
+            } else {
+                if (!group_fg() || !group_se()) break;
+            }
             // coefficient tiles (hi + lo pairs) sit where the scores were: a^T in S, then ds^T in E and p1^T in F
             auto bd = [&](int off) { return make_desc(st + off, 8192); };
             const uint32_t acc = g > 0;
@@ -224,12 +254,13 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             if (prm.has_glo) mma_ts_hi_k64(el, tm_u + Cfg::C_DV, tm_u + Cfg::C_S, bd(Cfg::ST_GL), Cfg::IDESC_TS, 1);
             mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TH), Cfg::IDESC_TS, acc);
             mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_S, bd(Cfg::ST_TL), Cfg::IDESC_TS, 1);
+            tc_commit_el(el, bar(KB_EMPTY_A + s));
             if (!mbar_wait(bar(KB_PRB), g & 1, abort_flag, wcap)) break;
             tc_fence_after();
             mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_E, bd(Cfg::ST_Q), Cfg::IDESC_TS, 1);
             mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YH), Cfg::IDESC_TS, 1);
             mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YL), Cfg::IDESC_TS, 1);
-            tc_commit_el(el, bar(KB_EMPTY + s));
+            tc_commit_el(el, bar(KB_EMPTY_B + s));
             if (g == nstep - 1) tc_commit_el(el, bar(KB_ACCFULL));
         }
         if (*abort_flag) {      // an aborted block: the MMAs issued above must be done before TMEM and shared memory go
@@ -247,8 +278,8 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         bool ok = true;
         for (int g = 0; g < nstep; ++g) {
             const int s = g % NST, i0 = 64 * (it0 + g);
-            if (!mbar_wait(bar(KB_FULL + s), (g / NST) & 1, abort_flag, wcap)) { ok = false; break; }      // the row records
-            if (!mbar_wait(bar(KB_SF1), g & 1, abort_flag, wcap)) { ok = false; break; }
+            if (!mbar_wait(bar(KB_FULL_B + s), (g / NST) & 1, abort_flag, wcap)) { ok = false; break; }      // the row records
+            if (!mbar_wait(bar(KB_SF_SE), g & 1, abort_flag, wcap)) { ok = false; break; }
             tc_fence_after();
             // records of this thread's 32 query rows (16 pairs): (nm2, nm2, kbar.y, kbar.y), (gk, gk, kk, kk)
             const float4* rsp = reinterpret_cast<const float4*>(smem + Cfg::SM_ST + s * STAGE + Cfg::ST_RS) + 32 * half;
@@ -285,7 +316,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(KB_PRA));
             }
-            if (!mbar_wait(bar(KB_SF2), g & 1, abort_flag, wcap)) { ok = false; break; }
+            if (!mbar_wait(bar(KB_SF_FG), g & 1, abort_flag, wcap)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll
             for (int chunk = 0; chunk < 2; ++chunk) {
@@ -363,7 +394,7 @@ struct QtCfg {
     static constexpr int SM_Q = 0, SM_GH = T128, SM_GL = 2 * T128, SM_TH = 3 * T128, SM_TL = 4 * T128;
     static constexpr int SM_KV = 5 * T128;         // stage 0: K block, V block.  A second stage: see stage_base()
     static constexpr int STAGE = 2 * T64;
-    static constexpr int NST_FIXED = D == 64 ? 3 : 1;      // stages at SM_KV
+    static constexpr int NST_FIXED = D == 64 ? 3 : 2;      // stages at SM_KV
     static constexpr int SM_RED = SM_KV + NST_FIXED * STAGE;        // 2 x 128 floats
     static constexpr int SM_BAR = SM_RED + 1024;
     static constexpr int SM_MISC = SM_BAR + 128;
@@ -407,13 +438,13 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int cbeg = W > 0 ? max(0, i0 + 1 - W) / 64 : 0;
     const int nblk = cend - cbeg;
     const long long wcap = prm.wait_clocks;
-    // Stages of the K/V ring.  d = 128: the tiles that stay for the whole block leave room for one stage; where the
-    // upstream gradient has no lo half (bf16), that half's tile is a second one.  The moments kernel has no T tiles.
-    const int nst = D == 64 ? 3 : (MODE == 0 ? 3 : (prm.has_glo ? 1 : 2));
+    // Stages of the K/V ring.  d = 128: the tiles that stay for the whole block leave room for two stages; a third one
+    // takes the place of a tile that is not loaded (the upstream gradient's lo half when it comes in bf16; the T tiles
+    // in the moments kernel).
+    const int nst = D == 64 ? 3 : (MODE == 0 ? 3 : (prm.has_glo ? 2 : 3));
     auto stage_base = [&](int s) -> uint32_t {
-        if (D == 64) return Cfg::SM_KV + s * STAGE;
-        if (MODE == 0) return s == 0 ? Cfg::SM_KV : (s == 1 ? Cfg::SM_TH : Cfg::SM_TL);
-        return s == 0 ? Cfg::SM_KV : Cfg::SM_GL;
+        if (D == 64 || s < 2) return Cfg::SM_KV + s * STAGE;
+        return MODE == 0 ? Cfg::SM_TH : Cfg::SM_GL;
     };
     static_assert(D == 64 || QtCfg<D>::STAGE == QtCfg<D>::T128, "a d = 128 stage takes the place of one stationary tile");
 
