@@ -716,6 +716,7 @@ int launch_t(const BackwardArgs& a) {
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
         f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg; f.window = a.window;
         f.rhs = hvec; f.sol = tvec;
+        f.kbar_in = kbar; f.stats_in = a.stats;      // kbar from the moments kernel, shift and omega as the forward saved them
         f.precondition = a.precondition;      // optional: the extra solve preconditioned (the matrices come from the pre-pass below)
         f.set_contiguous();
         // what the workspace holds beyond this pass's own arrays serves the solve (the fp16 copy of k; for

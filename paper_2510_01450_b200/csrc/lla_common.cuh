@@ -101,6 +101,8 @@ struct ForwardArgs {
     int window = 0;             // causal sliding window: a row sees its last `window` positions (0: all)
     const float* rhs = nullptr; // tensor-core kernel only: solve C_i x_i = rhs_i (centred system) for the
     float* sol = nullptr;       // iterative rows and write x_i [B, H, nq, d] instead of the output
+    const float* kbar_in = nullptr;     // with rhs / sol, optional: kbar_i [B, H, nq, d] and the saved stats [B, H, nq, 3] of
+    const float* stats_in = nullptr;    // the forward; given both, the kernel skips the sweep that recomputes them
     // layouts of q [B, H, nq, d], k [B, H / kv_group, n, d], v [.., dv] and out [B, H, nq, dv]; zero = not set: the
     // launchers that build a ForwardArgs themselves call set_contiguous()
     Strides sq = {0, 0, 0}, sk = {0, 0, 0}, sv = {0, 0, 0}, so = {0, 0, 0};

@@ -32,6 +32,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <type_traits>
 #include <mutex>
 
 #include "lla_sm100.cuh"
@@ -121,6 +122,8 @@ struct TcParams {
     int window;          // causal sliding window (0: none): a row sees its last `window` positions
     const float* rhs;    // solve mode: right-hand sides h_i [B, H, nq, D]; the CG then solves C_i x = h_i ...
     float* sol;          // ... and x_i is written here instead of running the output sweep
+    const float* kbar_in;    // solve mode, optional: kbar_i [B, H, nq, D] and the forward's saved stats [B, H, nq, 3] (the
+    const float* stats_in;   // shift and omega): given both, the statistics sweep that would recompute them is skipped
     int* iters;
     int* status;
     float* scratch;      // D = 128: per-SM slots for x, kbar, r (TcCfg::SCRATCH_FLOATS_PER_SM each)
@@ -133,8 +136,10 @@ struct TcParams {
     unsigned short order[TC_ORDER_MAX];
 };
 
-// PC: preconditioned CG compiled in (an instance of its own, so that the plain path carries none of its code)
-template <int D, typename TOut, bool PC>
+// PC: preconditioned CG compiled in (an instance of its own, so that the plain path carries none of its code).
+// GIVEN: solve mode with kbar and the saved row statistics supplied (fp32 output type only), likewise an instance
+// of its own: the statistics sweep is compiled out.
+template <int D, typename TOut, bool PC, bool GIVEN = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmK16,
@@ -756,7 +761,13 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         {
             float part = 0.f;
             mx2 = 0.f;
-            for (int attempt = 0; attempt < 2 && ok; ++attempt) {
+            // (solve mode with the row statistics given: nothing to sweep for)
+            constexpr bool given = GIVEN;
+            if (given && row_ok) {
+                mx2 = prm.stats_in[((size_t)bh * nq + row) * 3 + 0] * 1.4426950408889634f;
+                tmax = mx2;
+            }
+            for (int attempt = 0; attempt < 2 && ok && !given; ++attempt) {
                 smax = -INFINITY;
                 start_sweep(SW_STATS);
                 part = sweep(SW_STATS);
@@ -769,8 +780,18 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             if (ok) {
                 float acc[NCOL];
-                acc_load(acc);
-                omega = pair_sum(part);
+                if (given) {
+                    omega = row_ok ? prm.stats_in[((size_t)bh * nq + row) * 3 + 1] : 1.f;
+#pragma unroll
+                    for (int col = 0; col < NCOL; col += 4) {
+                        float4 kb4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (row_ok) kb4 = *reinterpret_cast<const float4*>(prm.kbar_in + ((size_t)bh * nq + row) * D + c0 + col);
+                        acc[col] = kb4.x * omega; acc[col + 1] = kb4.y * omega; acc[col + 2] = kb4.z * omega; acc[col + 3] = kb4.w * omega;
+                    }
+                } else {
+                    acc_load(acc);
+                    omega = pair_sum(part);
+                }
                 inv_omega = 1.f / omega;
                 const float lam_i = (prm.lambda_rows && row < nq) ? prm.lambda_rows[(size_t)bh * nq + row] : prm.lambda;
                 // ridge in the frame of the shift: lambda e^{-shift} by the definition; the printed algorithm adds
@@ -1141,7 +1162,7 @@ int launch_t(const ForwardArgs& a) {
     prm.scale = a.scale; prm.lambda = a.lambda; prm.tol = a.tol;
     prm.lambda_rows = a.lambda_rows; prm.ridge_mode = a.ridge_mode;
     prm.block_mask = a.block_mask; prm.block_mask_stride = a.block_mask_stride;
-    prm.rhs = a.rhs; prm.sol = a.sol;
+    prm.rhs = a.rhs; prm.sol = a.sol; prm.kbar_in = a.kbar_in; prm.stats_in = a.stats_in;
     prm.H = a.H; prm.kv_group = a.kv_group > 0 ? a.kv_group : 1;
     prm.so = a.so;
     prm.rho = a.rho; prm.stats = a.stats; prm.iters = a.iters; prm.status = a.status;
@@ -1185,6 +1206,9 @@ int launch_t(const ForwardArgs& a) {
         precond = true;
     }
     auto kern = precond ? forward_tc_kernel<D, TOut, true> : forward_tc_kernel<D, TOut, false>;
+    if constexpr (std::is_same<TOut, float>::value) {
+        if (a.sol && a.kbar_in && a.stats_in) kern = precond ? forward_tc_kernel<D, TOut, true, true> : forward_tc_kernel<D, TOut, false, true>;
+    }
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
     dim3 grid(BH, tiles);
     kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, mk16, mm, (TOut*)a.out, prm);
