@@ -416,7 +416,7 @@ def run_ours(args):
         if 3 in leg_objs:      # the n = 4096 workload as well, where the pair kernels dominate the pass
             backward3, cl = bench_backward(L, torch, peaks, leg_objs[3], local, steps=10, nsets=2)
             samplers.append(cl)
-        if head.w.name == inputs.CONFIGS[HEADLINE].name:      # and the headline workload (d = 128)
+        if head.w.name.startswith(inputs.CONFIGS[HEADLINE].name):      # and the headline workload (d = 128; also with --heads)
             backward4, cl = bench_backward(L, torch, peaks, head, local, steps=4, warmup=3, nsets=2)
             samplers.append(cl)
 
