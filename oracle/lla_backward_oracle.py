@@ -86,6 +86,24 @@ def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, 
     return (dq, dk, dv, dlam) if want_dlambda else (dq, dk, dv)
 
 
+def backward_rows(q, k, v, g, scale, lam, rows, window=0):
+    """The share of the gradient that the given query rows of ONE head contribute (causal): q, k [n, d]; v, g [n, dv];
+    rows a sequence of row indices.  Returns (dq_rows [len(rows), d], dk [n, d], dv [n, dv]) for the loss
+    sum_{i in rows} <g_i, o_i>: dq_rows are the full gradient's rows (a query enters its own row only), dk and dv its
+    shares from these rows -- complete for every key that no other row sees, e.g. the last m keys when rows are the
+    last m rows.  Same definition and operations as backward(), one row at a time (sizes the full-size tests need)."""
+    q, k, v, g = (np.asarray(a, dtype=np.float64) for a in (q, k, v, g))
+    Q = torch.tensor(q, requires_grad=True)
+    K = torch.tensor(k, requires_grad=True)
+    V = torch.tensor(v, requires_grad=True)
+    G = torch.tensor(g)
+    for i in rows:
+        r = torch.tensor([int(i)])
+        o = _forward_rows(Q, K, V, r, float(scale), float(lam), True, int(window))
+        (o * G[r]).sum().backward()
+    return Q.grad.numpy()[np.asarray(list(rows), dtype=np.int64)], K.grad.numpy(), V.grad.numpy()
+
+
 def forward(q, k, v, scale, lam, causal=True, chunk=32, window=0):
     """The forward values the gradient above differentiates (used by the pins to tie this module's
     forward to the C oracle's)."""

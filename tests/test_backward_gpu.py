@@ -168,6 +168,60 @@ def test_backward_sliding_window(backward_oracle, d, n, window):
     assert grad_err(got[1], full[1]).max() > 10 * TOL        # (the window matters at these sizes)
 
 
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_backward_full_size_sampled(backward_oracle, cfg):
+    # the n = 4096 and n = 16384 workloads at full size, in the launch configuration bench.py times.  The oracle
+    # cannot form whole gradients there; it checks what it can compute row by row -- dq on sampled rows, and dk, dv of
+    # the last keys (which only the last rows see) -- and two identities hold at any size: sum_j dV_j = sum_i g_i
+    # (the coefficients of a row sum to one) and <dV, V> = <g, o> (the output is linear in the values).
+    w = inputs.CONFIGS[cfg]
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    dq_, dk_, dv_, dg = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16"), dev(g, "f32")
+    shape = (w.B, w.H, w.n, w.d)
+    out, rho = (torch.empty(shape, dtype=torch.float32, device="cuda") for _ in range(2))
+    stats = torch.empty((w.B, w.H, w.n, 3), dtype=torch.float32, device="cuda")
+    fws = torch.empty(max(L.lla_forward_workspace_bytes(w.B, w.H, w.n, w.d, w.d), 256), dtype=torch.uint8, device="cuda")
+    L.lla_forward_ex(dq_, dk_, dv_, out, w.B, w.H, w.n, w.d, w.d, w.scale, w.lam, out_dtype=L.LLA_F32, rho=rho, stats=stats,
+                     workspace=fws, workspace_bytes=fws.numel(), stream=stream_ptr())
+    grads = [torch.full(shape, float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+    nbytes = L.lla_backward_workspace_bytes(w.B, w.H, w.n, w.d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, *grads, w.B, w.H, w.n, w.d, w.scale, w.lam, device_status=status,
+                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr())
+    torch.cuda.synchronize()
+    st = status.cpu().numpy()
+    assert st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0 and st[L.STATUS_ROWS_AT_CAP] == 0
+    gq, gk, gv = (t.cpu().numpy().astype(np.float64) for t in grads)
+    o = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(gq).all() and np.isfinite(gk).all() and np.isfinite(gv).all()
+    # identities, per head
+    sum_dv, sum_g = gv.sum(axis=2), g.astype(np.float64).sum(axis=2)
+    assert np.abs(sum_dv - sum_g).max() <= 1e-3 * np.abs(g).sum(axis=2).max()
+    lhs = (gv * v.astype(np.float64)).sum(axis=(2, 3))
+    rhs = (g.astype(np.float64) * o).sum(axis=(2, 3))
+    scale_ = np.sqrt((g.astype(np.float64) ** 2).sum(axis=(2, 3)) * (o ** 2).sum(axis=(2, 3)))
+    assert np.abs(lhs - rhs).max() <= 1e-3 * scale_.max()
+    # sampled rows and the last keys of two heads
+    rng = np.random.default_rng(300 + cfg)
+    m = 6
+    for b, h in ((0, 0), (w.B - 1, w.H - 1)):
+        first = w.d + w.d // 2 - 1
+        rows = np.concatenate([[first, first + 1, 2 * w.d, 4 * w.d + 3], rng.integers(first, w.n - m, size=6),
+                               np.arange(w.n - m, w.n)])
+        rq, rk, rv = backward_oracle.backward_rows(q[b, h], k[b, h], v[b, h], g[b, h], w.scale, w.lam, rows)
+        med = np.median(np.linalg.norm(gq[b, h], axis=1))
+        err = np.linalg.norm(gq[b, h][rows] - rq, axis=1) / np.maximum(np.linalg.norm(rq, axis=1), 0.1 * med)
+        assert err.max() <= TOL, ("dq", b, h, float(err.max()), int(rows[err.argmax()]))
+        # only the last m rows see the last m keys: drop the other sampled rows' shares by recomputing with those rows alone
+        _, tk, tv = backward_oracle.backward_rows(q[b, h], k[b, h], v[b, h], g[b, h], w.scale, w.lam, np.arange(w.n - m, w.n))
+        for name, got, ref in (("dk", gk[b, h], tk), ("dv", gv[b, h], tv)):
+            medk = np.median(np.linalg.norm(got, axis=1))
+            e = np.linalg.norm(got[w.n - m:] - ref[w.n - m:], axis=1) / np.maximum(np.linalg.norm(ref[w.n - m:], axis=1), 0.1 * medk)
+            assert e.max() <= TOL, (name, b, h, float(e.max()))
+
+
 def test_backward_with_preconditioned_solve(backward_oracle):
     w = inputs.CONFIGS[2].shrink(B=1, H=2, n=640, seed=295)
     q, k, v = inputs.make_prefill(w)

@@ -187,3 +187,20 @@ def test_sliding_window_forward_and_finite_differences():
             am = {"q": q, "k": k, "v": v, name: xm}
             num[idx] = (loss(ap["q"], ap["k"], ap["v"]) - loss(am["q"], am["k"], am["v"])) / (2 * eps)
         assert np.abs(num - grad).max() <= 2e-7 * max(1.0, np.abs(grad).max()), name
+
+
+def test_row_shares_add_up_to_the_gradient():
+    # backward_rows (one row at a time, for the full-size tests) against backward on a small case: all rows' shares
+    # sum to the gradient, and the last m rows alone give the complete dk, dv of the last m keys
+    n, d, dv, scale, lam = 24, 5, 3, 0.5, 2e-2
+    q, k, v, g = _inputs(9, n, d, dv)
+    dq, dk, dv_ = (x[0, 0] for x in bwd.backward(q, k, v, g, scale, lam))
+    rq, rk, rv = bwd.backward_rows(q[0, 0], k[0, 0], v[0, 0], g[0, 0], scale, lam, range(n))
+    for a, b in ((rq, dq), (rk, dk), (rv, dv_)):
+        assert np.abs(a - b).max() <= 1e-12 * max(1.0, np.abs(b).max())
+    m = 5
+    rq, rk, rv = bwd.backward_rows(q[0, 0], k[0, 0], v[0, 0], g[0, 0], scale, lam, range(n - m, n))
+    assert np.abs(rq - dq[n - m:]).max() <= 1e-12 * np.abs(dq).max()
+    assert np.abs(rk[n - m:] - dk[n - m:]).max() <= 1e-12 * np.abs(dk).max()
+    assert np.abs(rv[n - m:] - dv_[n - m:]).max() <= 1e-12 * np.abs(dv_).max()
+    assert np.abs(rk[:n - m] - dk[:n - m]).max() > 1e-3      # (the earlier keys also hear from the other rows)
