@@ -29,10 +29,11 @@ import numpy as np
 import torch
 
 
-def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0):
+def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0, visible=None):
     """o_i for the given row indices of one head, from the definition (float64 tensors).  window > 0 (causal only):
     row i sees its last `window` positions, keys max(0, i - window + 1) .. i (the sliding window that the paper's
-    discussion section suggests; the sums of Eq. "query_specific" then run over those keys)."""
+    discussion section suggests; the sums of Eq. "query_specific" then run over those keys).  visible (optional, bool
+    [n, n]): row i sees key j only where visible[i, j] as well (sparse attention: the same sums over fewer keys)."""
     n = K.shape[0]
     d = K.shape[1]
     L = int(rows.max()) + 1 if causal else n
@@ -45,6 +46,8 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0):
             mask = mask & (torch.arange(L)[None, :] > rows[:, None] - window)
     else:
         mask = torch.ones(len(rows), L, dtype=torch.bool)
+    if visible is not None:
+        mask = mask & torch.as_tensor(np.asarray(visible)[rows.numpy()][:, :L])
     m = torch.where(mask, s, torch.full_like(s, -torch.inf)).max(dim=1).values.detach()
     w = torch.where(mask, torch.exp(s - m[:, None]), torch.zeros_like(s))
     lam_i = (lam[rows] if torch.is_tensor(lam) else lam) * torch.exp(-m)    # one ridge per row when lam is a tensor
@@ -56,10 +59,11 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0):
     return (c @ Vl) / c.sum(dim=1, keepdim=True)                   # Eq. "lla"
 
 
-def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, window=0):
+def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, window=0, visible=None):
     """Gradients of sum_i <g_i, o_i> with respect to q, k, v.
 
     q, k: [B, H, n, d]; v, g: [B, H, n, dv]; numpy arrays (any float dtype; widened to float64).
+    visible: optional bool [n, n] or [B * H, n, n] (row, key) visibility on top of causality (see _forward_rows).
     Returns (dq, dk, dv) as float64 numpy arrays of the inputs' shapes; with want_dlambda also
     dlambda [B, H, n], the derivative with respect to a ridge of its own per query row (the paper's
     learnable per-token regularisation, Appendix on the regularisation), each evaluated at lam.
@@ -77,8 +81,9 @@ def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, 
             lam_rows = torch.full((n,), float(lam), dtype=torch.float64, requires_grad=True)
             for r0 in range(0, n, chunk):
                 rows = torch.arange(r0, min(n, r0 + chunk))
+                vis = None if visible is None else (visible if np.ndim(visible) == 2 else visible[b * H + h])
                 o = _forward_rows(Q, K, V, rows, float(scale), lam_rows if want_dlambda else float(lam), bool(causal),
-                                  int(window))
+                                  int(window), vis)
                 (o * G[rows]).sum().backward()
             dq[b, h], dk[b, h], dv[b, h] = Q.grad.numpy(), K.grad.numpy(), V.grad.numpy()
             if want_dlambda:
@@ -104,7 +109,7 @@ def backward_rows(q, k, v, g, scale, lam, rows, window=0):
     return Q.grad.numpy()[np.asarray(list(rows), dtype=np.int64)], K.grad.numpy(), V.grad.numpy()
 
 
-def forward(q, k, v, scale, lam, causal=True, chunk=32, window=0):
+def forward(q, k, v, scale, lam, causal=True, chunk=32, window=0, visible=None):
     """The forward values the gradient above differentiates (used by the pins to tie this module's
     forward to the C oracle's)."""
     q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
@@ -116,6 +121,7 @@ def forward(q, k, v, scale, lam, causal=True, chunk=32, window=0):
                 Q, K, V = (torch.tensor(a[b, h]) for a in (q, k, v))
                 for r0 in range(0, n, chunk):
                     rows = torch.arange(r0, min(n, r0 + chunk))
+                    vis = None if visible is None else (visible if np.ndim(visible) == 2 else visible[b * H + h])
                     out[b, h, r0:r0 + len(rows)] = _forward_rows(Q, K, V, rows, float(scale), float(lam),
-                                                                 bool(causal), int(window)).numpy()
+                                                                 bool(causal), int(window), vis).numpy()
     return out

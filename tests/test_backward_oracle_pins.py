@@ -9,6 +9,8 @@ by mathematics, none of it by the CUDA path.
   (f) the hand-derived formulas of the paper's backward appendix, evaluated literally in numpy
   (g) sliding window: the windowed forward is the C oracle's forward of each row's own key range, and the windowed
       gradient is the finite difference of that
+  (h) sparse visibility: the same with an arbitrary set of visible keys per row (the C oracle's decode entry point
+      on exactly those keys)
 """
 import numpy as np
 import pytest
@@ -204,3 +206,46 @@ def test_row_shares_add_up_to_the_gradient():
     assert np.abs(rk[n - m:] - dk[n - m:]).max() <= 1e-12 * np.abs(dk).max()
     assert np.abs(rv[n - m:] - dv_[n - m:]).max() <= 1e-12 * np.abs(dv_).max()
     assert np.abs(rk[:n - m] - dk[:n - m]).max() > 1e-3      # (the earlier keys also hear from the other rows)
+
+
+def _sparse_forward_by_c_oracle(q, k, v, scale, lam, visible):
+    """Row i of a forward with a visibility matrix is a single query over exactly its visible keys: the C oracle's
+    decode entry point, which knows no mask, on those keys."""
+    B, H, n, d = q.shape
+    out = np.zeros(v.shape)
+    for i in range(n):
+        idx = np.nonzero(visible[i, :i + 1])[0]
+        kc = np.zeros((B, H, n, d))
+        vc = np.zeros((B, H, n, v.shape[3]))
+        kc[:, :, :len(idx)] = k[:, :, idx]
+        vc[:, :, :len(idx)] = v[:, :, idx]
+        out[:, :, i] = fwd_c.decode(q[:, :, i], kc, vc, np.full(B, len(idx), dtype=np.int32), scale, lam)
+    return out
+
+
+def test_sparse_visibility_forward_and_finite_differences():
+    n, d, dv, scale, lam = 9, 3, 2, 0.6, 5e-2
+    q, k, v, g = _inputs(10, n, d, dv)
+    rng = np.random.default_rng(11)
+    visible = rng.random((n, n)) < 0.6
+    visible[np.arange(n), np.arange(n)] = True           # every row keeps its own key
+    ref = _sparse_forward_by_c_oracle(q, k, v, scale, lam, visible)
+    assert np.abs(bwd.forward(q, k, v, scale, lam, visible=visible) - ref).max() <= 1e-9 * np.abs(ref).max()
+    dq, dk, dv_ = bwd.backward(q, k, v, g, scale, lam, visible=visible)
+
+    def loss(q_, k_, v_):
+        return float((_sparse_forward_by_c_oracle(q_, k_, v_, scale, lam, visible) * g).sum())
+
+    eps = 1e-5
+    for name, x, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv_)):
+        num = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps
+            xm[idx] -= eps
+            ap = {"q": q, "k": k, "v": v, name: xp}
+            am = {"q": q, "k": k, "v": v, name: xm}
+            num[idx] = (loss(ap["q"], ap["k"], ap["v"]) - loss(am["q"], am["k"], am["v"])) / (2 * eps)
+        assert np.abs(num - grad).max() <= 2e-7 * max(1.0, np.abs(grad).max()), name
