@@ -395,6 +395,10 @@ typedef struct lla_backward_params {
                      (0: none).  At least head_rows, and not with impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED otherwise */
     int cg_precondition; /* as in lla_forward_params: 1 = the extra solve runs the preconditioned conjugate gradients
                      (about half the iterations; same result within the tolerance) */
+    const unsigned char *block_mask; /* as in lla_forward_params: the forward being differentiated ran with this block
+                     mask (same layout, same always-attended blocks; NULL = dense).  Not with a window, n > 65536 or
+                     impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED */
+    long long block_mask_stride;
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -394,6 +394,9 @@ int lla_backward_ex(const lla_backward_params* p) {
     a.window = p->window;
     if (p->cg_precondition != 0 && p->cg_precondition != 1) return LLA_ERR_INVALID_ARG;
     a.precondition = p->cg_precondition;
+    // block sparsity: under the forward's conditions, and in the tensor-core kernels only
+    if (p->block_mask && (a.cuda_core_pairs || a.window > 0 || p->n > 65536 || p->block_mask_stride < 0)) return LLA_ERR_UNSUPPORTED;
+    a.block_mask = p->block_mask; a.block_mask_stride = p->block_mask_stride;
     SideStream* side = side_stream();
     std::unique_lock<std::mutex> side_lock;
     if (side) {

@@ -41,6 +41,9 @@ constexpr uint32_t BT_IDESC_SS = make_idesc(128, 64, 0, 0);       // score tiles
 struct BtParams {
     int n, first, H, kv_group;
     int window;           // causal sliding window (0: none): a row sees its last `window` positions
+    int head_rows;        // block sparsity: the key blocks that start below this position are always attended
+    const unsigned char* block_mask;   // optional [query tiles of 128][key blocks of 64] (+ unit * block_mask_stride), as in the forward
+    long long block_mask_stride;
     int has_glo;          // the upstream gradient has a lo half (fp32 dout)
     float scale;
     const float* stats;   // [rows][3] saved by the forward
@@ -134,6 +137,22 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int nstep = it1 - it0;
     const long long wcap = prm.wait_clocks;
     if (nstep <= 0) return;
+    // Block sparsity (the forward's rule): query tile t = rows 128 t .. 128 t + 127 attends to key block c = keys
+    // 64 c .. 64 c + 63 if the mask says so, if the block starts below head_rows or if it is a diagonal block of the
+    // tile.  This tile's keys are the blocks 2 J and 2 J + 1 (TMEM lanes 0..63 and 64..127): bit 0 and bit 1 of the
+    // result.  A step (64 query rows) with neither is skipped by every role; g counts the steps taken.
+    const unsigned char* bmask = prm.block_mask ? prm.block_mask + (size_t)bh * prm.block_mask_stride : nullptr;
+    const int nblk_all = (n + 63) / 64;
+    auto blocks_on = [&](int i0) -> int {
+        if (!bmask) return 3;
+        const int t = i0 >> 7, c0 = (int)(2 * blockIdx.y);
+        int r = 0;
+        for (int x = 0; x < 2; ++x) {
+            const int c = c0 + x;
+            if (c < nblk_all && (bmask[(size_t)t * nblk_all + c] != 0 || c * 64 < prm.head_rows || c * 64 + 63 >= 128 * t)) r |= 1 << x;
+        }
+        return r;
+    };
 
     if (tid == 0) {
         mbar_init(bar(KB_KV), 1);
@@ -171,8 +190,10 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 tma_load_3d(sbase + Cfg::SM_V + sub * 16384, &tmV, bar(KB_KV), 64 * sub, j0, kvu);
             }
             int issued_a = 0, issued_b = 0;
-            for (int g = 0; g < nstep; ++g) {
-                const int s = g % NST, i0 = 64 * (it0 + g);
+            for (int it = it0, g = 0; it < it1; ++it) {
+                const int i0 = 64 * it;
+                if (!blocks_on(i0)) continue;
+                const int s = g % NST;
                 const uint32_t st = sbase + Cfg::SM_ST + s * STAGE;
                 if (!mbar_wait(bar(KB_EMPTY_A + s), ((g / NST) & 1) ^ 1, abort_flag, wcap)) break;
                 const uint32_t fa = bar(KB_FULL_A + s);
@@ -193,7 +214,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     tma_load_3d(st + Cfg::ST_YL + sub * 8192, &tmYl, fb, 64 * sub, i0, bh);
                 }
                 tma_load_3d(st + Cfg::ST_RS, &tmRS, fb, 0, i0 / 2, bh);
-                issued_b = g + 1;
+                issued_b = ++g;
             }
             if (*abort_flag) {      // an aborted block: what was issued must have landed before the block exits
                 (void)mbar_wait_landed(bar(KB_KV), 0, wcap);
@@ -208,7 +229,8 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t tm_u = __shfl_sync(0xffffffffu, tmem, 0);
         bool ok = mbar_wait(bar(KB_KV), 0, abort_flag, wcap);
         const uint64_t kdesc = make_desc(sb_u + Cfg::SM_K), vdesc = make_desc(sb_u + Cfg::SM_V);
-        for (int g = 0; g < nstep && ok; ++g) {
+        for (int it = it0, g = 0; it < it1 && ok; ++it) {
+            if (!blocks_on(64 * it)) continue;
             const int s = g % NST;
             const uint32_t st = sb_u + Cfg::SM_ST + s * STAGE;
             auto score = [&](uint32_t col, uint64_t adesc, int off, uint32_t acc) {
@@ -261,8 +283,9 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             mma_ts_hilo_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YH), Cfg::IDESC_TS, 1);
             mma_ts_hi_k64(el, tm_u + Cfg::C_DK, tm_u + Cfg::C_F, bd(Cfg::ST_YL), Cfg::IDESC_TS, 1);
             tc_commit_el(el, bar(KB_EMPTY_B + s));
-            if (g == nstep - 1) tc_commit_el(el, bar(KB_ACCFULL));
+            ++g;
         }
+        tc_commit_el(el, bar(KB_ACCFULL));      // the last step's products (the diagonal steps are always taken)
         if (*abort_flag) {      // an aborted block: the MMAs issued above must be done before TMEM and shared memory go
             tc_commit_el(el, bar(KB_EXIT));
             (void)mbar_wait_landed(bar(KB_EXIT), 0, wcap);
@@ -276,8 +299,12 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const float c1 = prm.scale * BT_LOG2E;
         const uint64_t c1c1 = pk2(c1, c1), one2 = pk2(1.f, 1.f), sc2 = pk2(prm.scale, prm.scale);
         bool ok = true;
-        for (int g = 0; g < nstep; ++g) {
-            const int s = g % NST, i0 = 64 * (it0 + g);
+        for (int it = it0, g = 0; it < it1; ++it) {
+            const int i0 = 64 * it;
+            const int on = blocks_on(i0);
+            if (!on) continue;
+            const bool lane_on = (on >> (lrow >> 6)) & 1;      // this lane's key block is attended by the step's query tile
+            const int s = g % NST;
             if (!mbar_wait(bar(KB_FULL_B + s), (g / NST) & 1, abort_flag, wcap)) { ok = false; break; }      // the row records
             if (!mbar_wait(bar(KB_SF_SE), g & 1, abort_flag, wcap)) { ok = false; break; }
             tc_fence_after();
@@ -291,13 +318,13 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
                 tmem_ld32(tm_lane + Cfg::C_E + col0, ev);
                 tc_wait_ld();
-                if (i0 < j0 + 128 || i0 + 64 > n || (W > 0 && i0 + 63 - j0 >= W)) {
-                    // a diagonal or last step, or one that reaches past the window: hide the pairs with j > i, i >= n
-                    // or i - j >= window
+                if (i0 < j0 + 128 || i0 + 64 > n || (W > 0 && i0 + 63 - j0 >= W) || on != 3) {
+                    // a diagonal or last step, one that reaches past the window or one with a key block left out: hide
+                    // the pairs with j > i, i >= n or i - j >= window, and the lanes of the block that is not attended
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const int gi = i0 + (int)col0 + e;
-                        if (gj > gi || gi >= n || (W > 0 && gi - gj >= W)) sv[e] = __float_as_uint(-1e30f);
+                        if (gj > gi || gi >= n || (W > 0 && gi - gj >= W) || !lane_on) sv[e] = __float_as_uint(-1e30f);
                     }
                 }
 #pragma unroll
@@ -343,6 +370,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(KB_PRB));
+            ++g;
         }
         if (ok && mbar_wait(bar(KB_ACCFULL), 0, abort_flag, wcap)) {
             tc_fence_after();
@@ -398,7 +426,8 @@ struct QtCfg {
     static constexpr int SM_RED = SM_KV + NST_FIXED * STAGE;        // 2 x 128 floats
     static constexpr int SM_BAR = SM_RED + 1024;
     static constexpr int SM_MISC = SM_BAR + 128;
-    static constexpr int SM_ALLOC = SM_MISC + 64 + 1024;
+    static constexpr int SM_BITS = SM_MISC + 64;      // block sparsity: one bit per key block of the tile (n <= 65536)
+    static constexpr int SM_ALLOC = SM_BITS + 128 + 1024;
     static constexpr uint32_t IDESC_TS = make_idesc(128, D, 0, 1);
     // TMEM columns.  MODE 1: S, E, F, Gamma, dQ, then y as bf16 pairs (hi D / 2 columns, lo D / 2 columns)
     static constexpr int C_S = 0, C_E = 64, C_F = 128, C_G1 = 192, C_DQ = 256, C_Y = 384;
@@ -436,8 +465,22 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int W = prm.window;
     const int cend = (min(n, i0 + 128) + 63) / 64;
     const int cbeg = W > 0 ? max(0, i0 + 1 - W) / 64 : 0;
-    const int nblk = cend - cbeg;
     const long long wcap = prm.wait_clocks;
+    // Block sparsity: the loops visit only the key blocks that the mask lists for this query tile, plus the ones that
+    // are always attended (the forward's rule): the blocks of the first head_rows keys and the tile's diagonal blocks.
+    // Every role walks the blocks in order and skips the same ones; c counts the blocks visited.
+    const bool sparse = prm.block_mask != nullptr;
+    uint32_t* bits = reinterpret_cast<uint32_t*>(smem + Cfg::SM_BITS);
+    if (sparse && tid < 32) {
+        const unsigned char* mrow = prm.block_mask + (size_t)bh * prm.block_mask_stride + (size_t)tile * ((n + 63) / 64);
+        uint32_t word = 0;
+        for (int b = 0; b < 32; ++b) {
+            const int cb = 32 * tid + b;
+            if (cb < cend && (mrow[cb] != 0 || cb * 64 < prm.head_rows || cb * 64 + 63 >= i0)) word |= 1u << b;
+        }
+        bits[tid] = word;
+    }
+    auto block_on = [&](int cb) { return !sparse || ((bits[cb >> 5] >> (cb & 31)) & 1u) != 0; };
     // Stages of the K/V ring.  d = 128: the tiles that stay for the whole block leave room for two stages; a third one
     // takes the place of a tile that is not loaded (the upstream gradient's lo half when it comes in bf16; the T tiles
     // in the moments kernel).
@@ -489,16 +532,17 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
             int issued = 0;
-            for (int c = 0; c < nblk; ++c) {
+            for (int cb = cbeg, c = 0; cb < cend; ++cb) {
+                if (!block_on(cb)) continue;
                 const int s = c % nst;
                 if (!mbar_wait(bar(QB_EMPTY + s), ((c / nst) & 1) ^ 1, abort_flag, wcap)) break;
                 const uint32_t st = sbase + stage_base(s), fb = bar(QB_FULL + s);
                 mbar_expect_tx(fb, STAGE);
                 for (int sub = 0; sub < KSUB; ++sub) {
-                    tma_load_3d(st + sub * 8192, &tmK, fb, 64 * sub, 64 * (cbeg + c), kvu);
-                    tma_load_3d(st + T64 + sub * 8192, &tmV, fb, 64 * sub, 64 * (cbeg + c), kvu);
+                    tma_load_3d(st + sub * 8192, &tmK, fb, 64 * sub, 64 * cb, kvu);
+                    tma_load_3d(st + T64 + sub * 8192, &tmV, fb, 64 * sub, 64 * cb, kvu);
                 }
-                issued = c + 1;
+                issued = ++c;
             }
             if (*abort_flag) {
                 (void)mbar_wait_landed(bar(QB_QFULL), 0, wcap);
@@ -513,7 +557,8 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         bool ok = mbar_wait(bar(QB_QFULL), 0, abort_flag, wcap);
         if (MODE == 1) ok = ok && mbar_wait(bar(QB_YREADY), 0, abort_flag, wcap);
         tc_fence_after();
-        for (int c = 0; c < nblk && ok; ++c) {
+        for (int cb = cbeg, c = 0; cb < cend && ok; ++cb) {
+            if (!block_on(cb)) continue;
             const int s = c % nst;
             if (!mbar_wait(bar(QB_FULL + s), (c / nst) & 1, abort_flag, wcap)) break;
             tc_fence_after();
@@ -553,8 +598,9 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (MODE == 1) mma_ts_hilo_k64(el, tm_u + Cfg::C_DQ, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
             else mma_ts_hilo_k64(el, tm_u + Cfg::C_H, tm_u + Cfg::C_G0, kmn, Cfg::IDESC_TS, c > 0);
             tc_commit_el(el, bar(QB_EMPTY + s));
-            if (c == nblk - 1) tc_commit_el(el, bar(QB_ACCFULL));
+            ++c;
         }
+        tc_commit_el(el, bar(QB_ACCFULL));      // the last block's products (at least the diagonal blocks were visited)
         if (*abort_flag) {
             tc_commit_el(el, bar(QB_EXIT));
             (void)mbar_wait_landed(bar(QB_EXIT), 0, wcap);
@@ -606,7 +652,8 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         uint64_t gb2 = pk2(0.f, 0.f);
         bool ok = true;
-        for (int c = 0; c < nblk; ++c) {
+        for (int cb = cbeg, c = 0; cb < cend; ++cb) {
+            if (!block_on(cb)) continue;
             if (!mbar_wait(bar(QB_SF1), c & 1, abort_flag, wcap)) { ok = false; break; }
             tc_fence_after();
             const uint32_t col0 = 32 * half;      // this thread's 32 keys of the block
@@ -615,7 +662,7 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 uint32_t sv[32];
                 tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
                 tc_wait_ld();
-                const int key0 = 64 * (cbeg + c) + (int)col0;
+                const int key0 = 64 * cb + (int)col0;
                 const int jlim = gi + 1 - key0;                           // keys jfirst <= e < jlim are visible
                 const int jfirst = W > 0 ? gi + 1 - W - key0 : 0;
                 if (jlim < 32 || jfirst > 0) {
@@ -678,6 +725,7 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(QB_PRB));
+            ++c;
         }
         float gb;
         {
@@ -741,7 +789,8 @@ template <int D>
 int launch_t(const BwdTensorArgs& a, int which) {
     const int BH = a.B * a.H, kvg = a.kv_group > 0 ? a.kv_group : 1, KVU = BH / kvg;
     BtParams p = {};
-    p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.window = a.window; p.has_glo = a.gl != nullptr; p.scale = a.scale;
+    p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.window = a.window;
+    p.head_rows = a.head_rows; p.block_mask = a.block_mask; p.block_mask_stride = a.block_mask_stride; p.has_glo = a.gl != nullptr; p.scale = a.scale;
     p.stats = a.stats; p.pairsc = a.pairsc; p.npair = (a.n + 1) / 2; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
     p.kbar = a.kbar; p.hvec = a.hvec; p.dq = a.dq; p.dk = a.dk; p.dv = a.dv; p.status = a.status;
     p.wait_clocks = kWaitClocks;

@@ -176,6 +176,8 @@ struct BackwardArgs {
     int cuda_core_pairs;        // 1: pair kernel on the CUDA cores even where the tensor-core one exists
     int window;                 // causal sliding window of the forward being differentiated (0: none)
     int precondition;           // 1: the extra solve runs the preconditioned CG (as ForwardArgs::precondition)
+    const unsigned char* block_mask;    // block sparsity of the forward being differentiated (as ForwardArgs::block_mask)
+    long long block_mask_stride;
     cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
     cudaEvent_t fork, join;
 };
@@ -196,6 +198,9 @@ struct BwdTensorArgs {
     float *kbar, *hvec, *dq, *dk, *dv;
     int B, H, n, d, first, kv_group;
     int window;     // causal sliding window (0: none)
+    int head_rows;  // with block_mask: key blocks that start below this position are always attended
+    const unsigned char* block_mask;    // optional, as ForwardArgs::block_mask
+    long long block_mask_stride;
     float scale;
     int* status;
     cudaStream_t stream;

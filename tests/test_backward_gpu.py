@@ -30,7 +30,8 @@ def grad_err(got, ref):
     return diff / np.maximum(rn, max(0.1 * float(np.median(rn)), 1e-4))
 
 
-def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IMPL_AUTO, window=0, **kw):
+def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IMPL_AUTO, window=0, block_mask=None,
+                 block_mask_stride=0, **kw):
     dq_, dk_, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
     dg = dev(g, dout_dtype)
     shape = (w.B, w.H, w.n, w.d)
@@ -38,14 +39,16 @@ def run_backward(w, q, k, v, g, out_dtype="f32", dout_dtype="f32", impl=L.LLA_IM
     rho = torch.empty(shape, dtype=torch.float32, device="cuda")
     stats = torch.empty((w.B, w.H, w.n, 3), dtype=torch.float32, device="cuda")
     L.lla_forward_ex(dq_, dk_, dv_, out, w.B, w.H, w.n, w.d, w.d, w.scale, w.lam, in_dtype=L.LLA_BF16,
-                     out_dtype=LLA_DT[out_dtype], rho=rho, stats=stats, stream=stream_ptr(), window=window)
+                     out_dtype=LLA_DT[out_dtype], rho=rho, stats=stats, stream=stream_ptr(), window=window,
+                     block_mask=block_mask, block_mask_stride=block_mask_stride)
     grads = [torch.full(shape, float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
     nbytes = L.lla_backward_workspace_bytes(w.B, w.H, w.n, w.d)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
     L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, *grads, w.B, w.H, w.n, w.d, w.scale, w.lam,
                       out_dtype=LLA_DT[out_dtype], dout_dtype=LLA_DT[dout_dtype], device_status=status,
-                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), impl=impl, window=window, **kw)
+                      workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), impl=impl, window=window,
+                      block_mask=block_mask, block_mask_stride=block_mask_stride, **kw)
     torch.cuda.synchronize()
     st = status.cpu().numpy()
     assert st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
@@ -220,6 +223,37 @@ def test_backward_full_size_sampled(backward_oracle, cfg):
             medk = np.median(np.linalg.norm(got, axis=1))
             e = np.linalg.norm(got[w.n - m:] - ref[w.n - m:], axis=1) / np.maximum(np.linalg.norm(ref[w.n - m:], axis=1), 0.1 * medk)
             assert e.max() <= TOL, (name, b, h, float(e.max()))
+
+
+@pytest.mark.parametrize("d,n,per_head", [(64, 700, True), (64, 1024, False), (128, 600, True)])
+def test_backward_block_sparse(backward_oracle, d, n, per_head):
+    # the gradient of the block-sparse forward: a random mask over [query tiles of 128] x [key blocks of 64] (about
+    # 40 % kept), the blocks of the first head_rows keys and each tile's diagonal blocks attended whatever it says.
+    # The oracle gets the resulting row-by-key visibility.
+    B, H = 1, 2
+    w = inputs.CONFIGS[2].shrink(B=B, H=H, n=n, d=d, dv=d, seed=310 + d)
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    tiles, blocks = (n + 127) // 128, (n + 63) // 64
+    rng = np.random.default_rng(17)
+    units = B * H if per_head else 1
+    mask = (rng.random((units, tiles, blocks)) < 0.4).astype(np.uint8)
+    head_rows = d + d // 2
+    visible = np.zeros((B * H, n, n), dtype=bool)
+    for u in range(B * H):
+        for t in range(tiles):
+            for c in range(blocks):
+                if mask[u if per_head else 0, t, c] or c * 64 < head_rows or c * 64 + 63 >= t * 128:
+                    visible[u, t * 128:(t + 1) * 128, c * 64:(c + 1) * 64] = True
+    ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam, visible=visible)
+    got = run_backward(w, q, k, v, g, block_mask=torch.from_numpy(mask).cuda(),
+                       block_mask_stride=tiles * blocks if per_head else 0)
+    for name, a, b in zip(("dq", "dk", "dv"), got, ref):
+        assert np.isfinite(a).all(), name
+        err = grad_err(a, b)
+        assert err.max() <= TOL, (name, float(err.max()), int(err.argmax()))
+    dense = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
+    assert grad_err(got[1], dense[1]).max() > 10 * TOL        # (the mask matters)
 
 
 def test_backward_with_preconditioned_solve(backward_oracle):
