@@ -45,7 +45,7 @@ using namespace sm100;
 constexpr int TC_BR = 128;           // query rows per block (TMEM lanes)
 constexpr int TC_BC = 64;            // keys per block
 constexpr int TC_COMPUTE = 256;      // compute threads (warps 0..7)
-constexpr int TC_THREADS = 352;      // + TMA warp + two MMA warps
+constexpr int TC_THREADS = 352;      // + TMA warp + two MMA warps (d = 128: 384, with an idle warp that completes the third warpgroup)
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_NBUF = 3;           // S/A/U buffers in TMEM (128 columns each)
 constexpr int TC_ACC_COL = TC_NBUF * 128;   // ACC columns [384, 384 + D)
@@ -140,7 +140,7 @@ struct TcParams {
 // GIVEN: solve mode with kbar and the saved row statistics supplied (fp32 output type only), likewise an instance
 // of its own: the statistics sweep is compiled out.
 template <int D, typename TOut, bool PC, bool GIVEN = false>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(D == 128 ? 384 : TC_THREADS, 1)
 forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmK16,
                   const __grid_constant__ CUtensorMap tmM, TOut* __restrict__ out, const TcParams prm) {
@@ -252,7 +252,13 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     tc_fence_after();
     const uint32_t tmem = (uint32_t)misc[0];
 
+    // Register hand-over between the warpgroups: the copy- and MMA-issuing warps need few registers and give theirs
+    // up, the compute warps take them (168 a thread at launch, the most that twelve warps can have).
+    auto regs_give = [&]() { if constexpr (D == 128) asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory"); };
+    auto regs_take = [&]() { if constexpr (D == 128) asm volatile("setmaxnreg.inc.sync.aligned.u32 216;" ::: "memory"); };
+
     if (warp == 8) {
+        regs_give();
         // ================================ TMA producer ================================
         // K blocks stream through the ring continuously: once a sweep's blocks are issued the first
         // blocks of the next sweep are prefetched without waiting to learn what kind of sweep it is
@@ -337,6 +343,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
     } else if (warp == 9) {
+        regs_give();
         // ================================ MMA issuer 1: S = Q K^T, A = P K^T ================================
         // All 32 lanes run the loop convergently; the MMAs and commits are predicated on one lane.
         // tcgen05.mma issue is throttled to the execution rate, so the time an issuing warp spends
@@ -390,6 +397,7 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             (void)mbar_wait_landed(bar(B_EXIT + 0), 0, wcap);
         }
     } else if (warp == 10) {
+        regs_give();
         // ================================ MMA issuer 2: ACC += U B ================================
         const uint32_t el = elect_one();
         const uint32_t sb_u = __shfl_sync(0xffffffffu, sbase, 0);
@@ -418,7 +426,10 @@ forward_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tc_commit_el(el, bar(B_EXIT + 1));
             (void)mbar_wait_landed(bar(B_EXIT + 1), 0, wcap);
         }
+    } else if (warp == 11) {
+        regs_give();
     } else {
+        regs_take();
         // ================================ compute warps ================================
         const int quad = warp & 3, half = warp >> 2;
         const int lrow = quad * 32 + lane;                 // row inside the tile == TMEM lane
@@ -1211,7 +1222,7 @@ int launch_t(const ForwardArgs& a) {
     }
     LLA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
     dim3 grid(BH, tiles);
-    kern<<<grid, TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, mk16, mm, (TOut*)a.out, prm);
+    kern<<<grid, D == 128 ? 384 : TC_THREADS, Cfg::SM_ALLOC, a.stream>>>(mq, mk, mv, mk16, mm, (TOut*)a.out, prm);
     LLA_CUDA_TRY(cudaGetLastError());
     return LLA_OK;
 }
