@@ -38,7 +38,7 @@ L2_BYTES = 126e6
 NCU_TRAFFIC = {
     2: (12.68e6, "profiles/forward_tc_kernel_cfg2.md"),
     3: (4 * 17.06e6, "profiles/forward_tc_kernel_cfg3.md (8 of 32 units captured, x 4)"),
-    4: (8 * (34.26e6 + 4.23e6), "profiles/forward_tc_kernel_cfg4.md (2 of 16 heads captured, x 8)"),
+    4: (8 * (33.67e6 + 2.58e6), "profiles/forward_tc_kernel_cfg4.md (2 of 16 heads captured, x 8)"),
 }
 NCU_DECODE_TRAFFIC = (1.188e9 + 24.2e6 + 34.3e6, "profiles/decode_tc_kernel_cfg5.md")   # streaming read + record write, solve read
 
