@@ -29,16 +29,18 @@ import numpy as np
 import torch
 
 
-def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0, visible=None):
+def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0, visible=None, q_offset=0):
     """o_i for the given row indices of one head, from the definition (float64 tensors).  window > 0 (causal only):
     row i sees its last `window` positions, keys max(0, i - window + 1) .. i (the sliding window that the paper's
     discussion section suggests; the sums of Eq. "query_specific" then run over those keys).  visible (optional, bool
-    [n, n]): row i sees key j only where visible[i, j] as well (sparse attention: the same sums over fewer keys)."""
+    [n, n]): row i sees key j only where visible[i, j] as well (sparse attention: the same sums over fewer keys).
+    q_offset: Q holds only the queries of positions q_offset .. n - 1 (a chunk of queries against a longer key
+    sequence); `rows` are positions."""
     n = K.shape[0]
     d = K.shape[1]
     L = int(rows.max()) + 1 if causal else n
     Kl, Vl = K[:L], V[:L]
-    Qr = Q[rows]
+    Qr = Q[rows - q_offset]
     s = scale * (Qr @ Kl.T)                                        # scores, Section 3.1
     if causal:
         mask = torch.arange(L)[None, :] <= rows[:, None]           # row i sees keys j <= i
@@ -62,16 +64,20 @@ def _forward_rows(Q, K, V, rows, scale, lam, causal, window=0, visible=None):
 def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, window=0, visible=None):
     """Gradients of sum_i <g_i, o_i> with respect to q, k, v.
 
-    q, k: [B, H, n, d]; v, g: [B, H, n, dv]; numpy arrays (any float dtype; widened to float64).
+    k: [B, H, n, d]; v: [B, H, n, dv]; q: [B, H, nq, d] and g: [B, H, nq, dv] with nq <= n: the queries (and their
+    upstream gradients) of the last nq positions, a chunk of queries against a longer key sequence; nq = n is the
+    whole sequence.  numpy arrays (any float dtype; widened to float64).
     visible: optional bool [n, n] or [B * H, n, n] (row, key) visibility on top of causality (see _forward_rows).
     Returns (dq, dk, dv) as float64 numpy arrays of the inputs' shapes; with want_dlambda also
     dlambda [B, H, n], the derivative with respect to a ridge of its own per query row (the paper's
     learnable per-token regularisation, Appendix on the regularisation), each evaluated at lam.
     """
     q, k, v, g = (np.asarray(a, dtype=np.float64) for a in (q, k, v, g))
-    B, H, n, _ = q.shape
+    B, H, nq, _ = q.shape
+    n = k.shape[2]
+    off = n - nq              # the queries are the last nq positions (causal); nq = n is the whole sequence
     dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
-    dlam = np.zeros((B, H, n))
+    dlam = np.zeros((B, H, nq))
     for b in range(B):
         for h in range(H):
             Q = torch.tensor(q[b, h], requires_grad=True)
@@ -79,15 +85,15 @@ def backward(q, k, v, g, scale, lam, causal=True, chunk=32, want_dlambda=False, 
             V = torch.tensor(v[b, h], requires_grad=True)
             G = torch.tensor(g[b, h])
             lam_rows = torch.full((n,), float(lam), dtype=torch.float64, requires_grad=True)
-            for r0 in range(0, n, chunk):
+            for r0 in range(off, n, chunk):
                 rows = torch.arange(r0, min(n, r0 + chunk))
                 vis = None if visible is None else (visible if np.ndim(visible) == 2 else visible[b * H + h])
                 o = _forward_rows(Q, K, V, rows, float(scale), lam_rows if want_dlambda else float(lam), bool(causal),
-                                  int(window), vis)
-                (o * G[rows]).sum().backward()
+                                  int(window), vis, off)
+                (o * G[rows - off]).sum().backward()
             dq[b, h], dk[b, h], dv[b, h] = Q.grad.numpy(), K.grad.numpy(), V.grad.numpy()
             if want_dlambda:
-                dlam[b, h] = lam_rows.grad.numpy()
+                dlam[b, h] = lam_rows.grad.numpy()[off:]
     return (dq, dk, dv, dlam) if want_dlambda else (dq, dk, dv)
 
 

@@ -249,3 +249,18 @@ def test_sparse_visibility_forward_and_finite_differences():
             am = {"q": q, "k": k, "v": v, name: xm}
             num[idx] = (loss(ap["q"], ap["k"], ap["v"]) - loss(am["q"], am["k"], am["v"])) / (2 * eps)
         assert np.abs(num - grad).max() <= 2e-7 * max(1.0, np.abs(grad).max()), name
+
+
+def test_chunk_of_queries_is_the_full_gradient_with_zero_upstream_elsewhere():
+    # the last nq queries against all n keys: the loss of the whole sequence with g = 0 on the earlier rows
+    n, nq, d, dv, scale, lam = 20, 7, 4, 3, 0.5, 3e-2
+    q, k, v, g = _inputs(12, n, d, dv)
+    g0 = g.copy()
+    g0[:, :, :n - nq] = 0.0
+    fq, fk, fv = bwd.backward(q, k, v, g0, scale, lam)
+    cq, ck, cv = bwd.backward(q[:, :, n - nq:], k, v, g[:, :, n - nq:], scale, lam)
+    assert cq.shape == (1, 1, nq, d)
+    assert np.abs(cq - fq[:, :, n - nq:]).max() <= 1e-12 * np.abs(fq).max()
+    assert np.abs(ck - fk).max() <= 1e-12 * np.abs(fk).max()
+    assert np.abs(cv - fv).max() <= 1e-12 * np.abs(fv).max()
+    assert np.abs(fq[:, :, :n - nq]).max() == 0.0
