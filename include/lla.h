@@ -399,6 +399,9 @@ typedef struct lla_backward_params {
                      mask (same layout, same always-attended blocks; NULL = dense).  Not with a window, n > 65536 or
                      impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED */
     long long block_mask_stride;
+    int q_rows;   /* as in lla_forward_params: the forward being differentiated had only the queries of the last q_rows
+                     positions (0 = n); q, out, dout, rho, stats, dq, iters and dlambda are then [B, H, q_rows, ..],
+                     k, v, dk, dv keep n rows.  Not with a block mask or impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED */
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -397,6 +397,10 @@ int lla_backward_ex(const lla_backward_params* p) {
     // block sparsity: under the forward's conditions, and in the tensor-core kernels only
     if (p->block_mask && (a.cuda_core_pairs || a.window > 0 || p->n > 65536 || p->block_mask_stride < 0)) return LLA_ERR_UNSUPPORTED;
     a.block_mask = p->block_mask; a.block_mask_stride = p->block_mask_stride;
+    // a chunk of queries against the whole key sequence: tensor-core kernels only, and not with a block mask
+    if (p->q_rows < 0 || p->q_rows > p->n) return LLA_ERR_INVALID_ARG;
+    a.nq = p->q_rows > 0 ? p->q_rows : p->n;
+    if (a.nq != p->n && (a.cuda_core_pairs || p->block_mask)) return LLA_ERR_UNSUPPORTED;
     SideStream* side = side_stream();
     std::unique_lock<std::mutex> side_lock;
     if (side) {

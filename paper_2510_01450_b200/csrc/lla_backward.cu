@@ -460,7 +460,8 @@ __global__ void __launch_bounds__(HB_THREADS, D == 64 ? 4 : 1)
 bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const void* __restrict__ dout, int dout_dtype,
                      float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv, int n, int lcap,
-                     double scale, double lambda, int* __restrict__ status, float* __restrict__ dlambda, int H, int kv_group) {
+                     double scale, double lambda, int* __restrict__ status, float* __restrict__ dlambda, int H, int kv_group,
+                     int nq) {
     constexpr int LDS = D + 1;
     extern __shared__ __align__(16) double hb_smem[];
     double* S = hb_smem;                  // D x (D + 1)
@@ -478,9 +479,9 @@ bwd_head_rows_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x;
     const int i = gridDim.y - 1 - blockIdx.y;       // rows with the most keys first
-    const int L = i + 1;
+    const int L = (n - nq) + i + 1;                 // query row i sits at position n - nq + i
     if (!LLA_IN_BOUNDS(L, lcap + 1, status, 602)) return;      // (debug build: the keys must fit the arrays sized for lcap)
-    const size_t base = (size_t)bh * n;
+    const size_t base = (size_t)bh * nq;            // rows of q, dout, dq, dlambda
     const size_t kvbase = (size_t)kv_unit(bh, H, kv_group) * n;     // grouped heads: the key/value head's rows
     for (int c = tid; c < D; c += HB_THREADS) {
         qd[c] = (double)__bfloat162float(q[(base + i) * D + c]);
@@ -637,13 +638,14 @@ size_t ws_own_bytes(long long rows, int d, long long heads) { return ws_fp32_byt
 template <int D>
 int launch_t(const BackwardArgs& a) {
     using C = BwCfg<D>;
-    const long long rows = (long long)a.B * a.H * a.n;
+    const int nq = a.nq > 0 ? a.nq : a.n, off = a.n - nq;      // the queries are the positions off .. n - 1
+    const long long rows = (long long)a.B * a.H * nq;          // rows of q, out, dout, rho, stats, dq
     const int BH = a.B * a.H;
-    const int first = max(0, min(a.n, a.head_rows - 1));      // rows [0, first) are solved directly
+    const int first = max(0, min(nq, a.head_rows - 1 - off));  // query rows [0, first) see fewer than head_rows keys: solved directly
     const int kvg = a.kv_group > 0 ? a.kv_group : 1;
-    const long long kvrows = rows / kvg;                       // rows of k, v, dk, dv
+    const long long kvrows = (long long)a.B * a.H * a.n / kvg; // rows of k, v, dk, dv
     if (a.workspace_bytes < ws_own_bytes(rows, D, BH) || !a.workspace) return LLA_ERR_WORKSPACE;
-    if (first > 2 * D) return LLA_ERR_UNSUPPORTED;
+    if (first > 0 && off + first > 2 * D) return LLA_ERR_UNSUPPORTED;      // (head_rows beyond 2 d + 1)
     float* kbar = static_cast<float*>(a.workspace);
     float* hvec = kbar + rows * D;
     float* tvec = hvec + rows * D;
@@ -656,7 +658,8 @@ int launch_t(const BackwardArgs& a) {
     const auto* q = static_cast<const __nv_bfloat16*>(a.q);
     const auto* k = static_cast<const __nv_bfloat16*>(a.k);
     const auto* v = static_cast<const __nv_bfloat16*>(a.v);
-    const size_t head_smem = head_smem_bytes<D>(first);
+    const int lcap = first > 0 ? off + first : 0;              // most keys a directly-solved row sees
+    const size_t head_smem = head_smem_bytes<D>(lcap);
     if (head_smem > 227u * 1024u) return LLA_ERR_UNSUPPORTED;
     LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_head_rows_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem));
     LLA_CUDA_TRY(cudaMemsetAsync(a.dk, 0, sizeof(float) * kvrows * D, a.stream));
@@ -671,11 +674,11 @@ int launch_t(const BackwardArgs& a) {
     if (first > 0) {
         const dim3 gh(BH, first);
         bwd_head_rows_kernel<D><<<gh, HB_THREADS, head_smem, hs>>>(
-            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, first, (double)a.scale, (double)a.lambda, a.status, a.dlambda, a.H, kvg);
+            q, k, v, a.dout, a.dout_dtype, a.dq, a.dk, a.dv, a.n, lcap, (double)a.scale, (double)a.lambda, a.status, a.dlambda, a.H, kvg, nq);
         LLA_CUDA_TRY(cudaGetLastError());
         if (forked) LLA_CUDA_TRY(cudaEventRecord(a.join, hs));
     }
-    if (first < a.n) {
+    if (first < nq) {
         BwdTensorArgs t = {};
         Pairs16 p16 = {};
         if (tensor) {
@@ -683,7 +686,7 @@ int launch_t(const BackwardArgs& a) {
             t.yh = pairs; t.yl = pairs + pb; t.tnh = pairs + 2 * pb; t.tnl = pairs + 3 * pb;
             p16.yh = reinterpret_cast<uint32_t*>(pairs); p16.yl = reinterpret_cast<uint32_t*>(pairs + pb);
             p16.tnh = reinterpret_cast<uint32_t*>(pairs + 2 * pb); p16.tnl = reinterpret_cast<uint32_t*>(pairs + 3 * pb);
-            p16.pairsc = pairsc; p16.npair = (a.n + 1) / 2;
+            p16.pairsc = pairsc; p16.npair = (nq + 1) / 2;
             if (a.dout_dtype == LLA_F32) {
                 t.gh = pairs + 4 * pb; t.gl = pairs + 5 * pb;
                 const size_t quads = (size_t)rows * D / 4;
@@ -695,12 +698,13 @@ int launch_t(const BackwardArgs& a) {
             }
             t.rowsc = rowsc; t.pairsc = pairsc; t.stats = a.stats; t.yvec = yvec; t.tvec = tvec;
             t.kbar = kbar; t.hvec = hvec; t.dq = a.dq; t.dk = a.dk; t.dv = a.dv;
-            t.B = a.B; t.H = a.H; t.n = a.n; t.d = D; t.first = first; t.kv_group = kvg; t.window = a.window;
+            t.B = a.B; t.H = a.H; t.n = a.n; t.nq = nq; t.d = D; t.first = first; t.kv_group = kvg; t.window = a.window;
             t.head_rows = a.head_rows; t.block_mask = a.block_mask; t.block_mask_stride = a.block_mask_stride;
             t.scale = a.scale; t.status = a.status; t.stream = a.stream;
             const int rc = launch_backward_tensor(t, 0);
             if (rc != LLA_OK) return rc;
         } else {
+            if (nq != a.n) return LLA_ERR_UNSUPPORTED;      // the CUDA-core kernels take whole sequences only
             const dim3 gm(BH, (a.n + C::BI - 1) / C::BI);
             LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_moments_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::MOMENTS_SMEM));
             bwd_moments_kernel<D><<<gm, BW_THREADS, C::MOMENTS_SMEM, a.stream>>>(q, k, v, a.dout, a.dout_dtype, a.stats, kbar, hvec,
@@ -715,7 +719,7 @@ int launch_t(const BackwardArgs& a) {
         f.scale = a.scale; f.lambda = a.lambda; f.causal = 1;
         f.max_iters = a.max_iters; f.tol = a.tol; f.head_rows = a.head_rows;
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
-        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = a.n; f.kv_group = kvg; f.window = a.window;
+        f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = nq; f.kv_group = kvg; f.window = a.window;
         f.block_mask = a.block_mask; f.block_mask_stride = a.block_mask_stride;
         f.rhs = hvec; f.sol = tvec;
         f.kbar_in = kbar; f.stats_in = a.stats;      // kbar from the moments kernel, shift and omega as the forward saved them
@@ -733,7 +737,7 @@ int launch_t(const BackwardArgs& a) {
         const int rc = launch_forward_tensor(f);
         if (rc != LLA_OK) return rc;
         bwd_rowprep_kernel<D><<<(unsigned)((rows + 7) / 8), BW_THREADS, 0, a.stream>>>(
-            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, a.n, first, rows, a.dlambda, p16);
+            q, a.out, a.out_dtype, a.dout, a.dout_dtype, a.rho, a.stats, kbar, tvec, yvec, rowsc, a.dq, nq, first, rows, a.dlambda, p16);
         LLA_CUDA_TRY(cudaGetLastError());
         if (tensor) {
             int rc2 = launch_backward_tensor(t, 1);

@@ -39,7 +39,8 @@ constexpr float BT_LOG2E = 1.4426950408889634f;
 constexpr uint32_t BT_IDESC_SS = make_idesc(128, 64, 0, 0);       // score tiles: [128 x 64], both operands K-major
 
 struct BtParams {
-    int n, first, H, kv_group;
+    int n, first, H, kv_group;      // n keys; first: the query rows [0, first) are not handled here
+    int nq;               // query rows: the positions n - nq .. n - 1 (a chunk of queries; nq = n: the whole sequence)
     int window;           // causal sliding window (0: none): a row sees its last `window` positions
     int head_rows;        // block sparsity: the key blocks that start below this position are always attended
     const unsigned char* block_mask;   // optional [query tiles of 128][key blocks of 64] (+ unit * block_mask_stride), as in the forward
@@ -127,13 +128,13 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x;
     const int kvu = kv_unit(bh, prm.H, prm.kv_group);
-    const int n = prm.n;
+    const int n = prm.n, nq = prm.nq, off = n - nq;      // query row i sits at position off + i
     const int j0 = blockIdx.y * 128;          // key tile 0 sees the most query rows and starts first (heads fastest)
-    // query steps of 64 rows: from the tile's first key (or the first row these kernels handle) to the last row that
-    // still sees a key of the tile
+    // query steps of 64 rows: from the first row that sees the tile's first key (or the first row these kernels
+    // handle) to the last row that still sees a key of the tile
     const int W = prm.window;
-    const int last_row = W > 0 ? min(n - 1, j0 + 127 + W - 1) : n - 1;
-    const int it0 = max(j0, prm.first) / 64, it1 = last_row / 64 + 1;
+    const int last_row = W > 0 ? min(nq - 1, j0 + 127 + W - 1 - off) : nq - 1;
+    const int it0 = max(max(j0 - off, 0), prm.first) / 64, it1 = last_row < 0 ? 0 : last_row / 64 + 1;
     const int nstep = it1 - it0;
     const long long wcap = prm.wait_clocks;
     if (nstep <= 0) return;
@@ -149,7 +150,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         int r = 0;
         for (int x = 0; x < 2; ++x) {
             const int c = c0 + x;
-            if (c < nblk_all && (bmask[(size_t)t * nblk_all + c] != 0 || c * 64 < prm.head_rows || c * 64 + 63 >= 128 * t)) r |= 1 << x;
+            if (c < nblk_all && (bmask[(size_t)t * nblk_all + c] != 0 || c * 64 < prm.head_rows || c * 64 + 63 >= off + 128 * t)) r |= 1 << x;
         }
         return r;
     };
@@ -318,13 +319,14 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
                 tmem_ld32(tm_lane + Cfg::C_E + col0, ev);
                 tc_wait_ld();
-                if (i0 < j0 + 128 || i0 + 64 > n || (W > 0 && i0 + 63 - j0 >= W) || on != 3) {
+                if (off + i0 < j0 + 128 || i0 + 64 > nq || (W > 0 && off + i0 + 63 - j0 >= W) || on != 3) {
                     // a diagonal or last step, one that reaches past the window or one with a key block left out: hide
-                    // the pairs with j > i, i >= n or i - j >= window, and the lanes of the block that is not attended
+                    // the pairs with j > position, row >= nq or position - j >= window, and the lanes of the block that
+                    // is not attended
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
-                        const int gi = i0 + (int)col0 + e;
-                        if (gj > gi || gi >= n || (W > 0 && gi - gj >= W) || !lane_on) sv[e] = __float_as_uint(-1e30f);
+                        const int gi = i0 + (int)col0 + e, pos = off + gi;
+                        if (gj > pos || gi >= nq || (W > 0 && pos - gj >= W) || !lane_on) sv[e] = __float_as_uint(-1e30f);
                     }
                 }
 #pragma unroll
@@ -377,7 +379,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // Key rows below `first` also get the directly-solved rows' shares (from another stream), and with grouped
             // heads every query head of the group adds into the same rows: those are added atomically.  Any other
             // row is this block's alone and is stored.
-            const bool plain = prm.kv_group == 1 && j0 >= prm.first;
+            const bool plain = prm.kv_group == 1 && (prm.first == 0 || j0 >= off + prm.first);
             const size_t rowoff = ((size_t)kvu * n + gj) * D + half * (D / 2);
             const bool inb = gj < n && LLA_IN_BOUNDS((size_t)kvu * n + gj, (size_t)(gridDim.x / prm.kv_group) * n, prm.status, 702);
 #pragma unroll 1
@@ -457,14 +459,14 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x;
     const int kvu = kv_unit(bh, prm.H, prm.kv_group);
-    const int n = prm.n;
+    const int n = prm.n, nq = prm.nq, off = n - nq;      // query row i sits at position off + i
     const int tile = gridDim.y - 1 - blockIdx.y;      // longest tiles first, heads fastest
     const int i0 = tile * 128;
     if (i0 + 128 <= prm.first) return;                // every row of the tile is solved directly
     // key blocks [cbeg, cend): with a sliding window the loop starts at the block of the first row's first visible key
     const int W = prm.window;
-    const int cend = (min(n, i0 + 128) + 63) / 64;
-    const int cbeg = W > 0 ? max(0, i0 + 1 - W) / 64 : 0;
+    const int cend = (off + min(nq, i0 + 128) + 63) / 64;
+    const int cbeg = W > 0 ? max(0, off + i0 + 1 - W) / 64 : 0;
     const long long wcap = prm.wait_clocks;
     // Block sparsity: the loops visit only the key blocks that the mask lists for this query tile, plus the ones that
     // are always attended (the forward's rule): the blocks of the first head_rows keys and the tile's diagonal blocks.
@@ -476,7 +478,7 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         uint32_t word = 0;
         for (int b = 0; b < 32; ++b) {
             const int cb = 32 * tid + b;
-            if (cb < cend && (mrow[cb] != 0 || cb * 64 < prm.head_rows || cb * 64 + 63 >= i0)) word |= 1u << b;
+            if (cb < cend && (mrow[cb] != 0 || cb * 64 < prm.head_rows || cb * 64 + 63 >= off + i0)) word |= 1u << b;
         }
         bits[tid] = word;
     }
@@ -610,8 +612,8 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int quad = warp & 3, half = warp >> 2;
         const int lrow = quad * 32 + lane;            // query row inside the tile == TMEM lane
         const int gi = i0 + lrow;
-        const size_t row = (size_t)bh * n + gi;
-        const bool okr = gi < n && gi >= prm.first && LLA_IN_BOUNDS(row, (size_t)gridDim.x * n, prm.status, 701);
+        const size_t row = (size_t)bh * nq + gi;
+        const bool okr = gi < nq && gi >= prm.first && LLA_IN_BOUNDS(row, (size_t)gridDim.x * nq, prm.status, 701);
         const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
         const float c1 = prm.scale * BT_LOG2E;
         // per-row scalars (see bwd_rowprep_kernel): p = 2^(c1 s + nm2) carries 1 / omega; a row that is switched off
@@ -663,8 +665,8 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tmem_ld32(tm_lane + Cfg::C_S + col0, sv);
                 tc_wait_ld();
                 const int key0 = 64 * cb + (int)col0;
-                const int jlim = gi + 1 - key0;                           // keys jfirst <= e < jlim are visible
-                const int jfirst = W > 0 ? gi + 1 - W - key0 : 0;
+                const int jlim = off + gi + 1 - key0;                     // keys jfirst <= e < jlim are visible
+                const int jfirst = W > 0 ? off + gi + 1 - W - key0 : 0;
                 if (jlim < 32 || jfirst > 0) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
@@ -789,9 +791,9 @@ template <int D>
 int launch_t(const BwdTensorArgs& a, int which) {
     const int BH = a.B * a.H, kvg = a.kv_group > 0 ? a.kv_group : 1, KVU = BH / kvg;
     BtParams p = {};
-    p.n = a.n; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.window = a.window;
+    p.n = a.n; p.nq = a.nq; p.first = a.first; p.H = a.H; p.kv_group = kvg; p.window = a.window;
     p.head_rows = a.head_rows; p.block_mask = a.block_mask; p.block_mask_stride = a.block_mask_stride; p.has_glo = a.gl != nullptr; p.scale = a.scale;
-    p.stats = a.stats; p.pairsc = a.pairsc; p.npair = (a.n + 1) / 2; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
+    p.stats = a.stats; p.pairsc = a.pairsc; p.npair = (a.nq + 1) / 2; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
     p.kbar = a.kbar; p.hvec = a.hvec; p.dq = a.dq; p.dk = a.dk; p.dv = a.dv; p.status = a.status;
     p.wait_clocks = kWaitClocks;
     const void* gl = a.gl ? a.gl : a.gh;        // a valid map either way; never loaded without a lo half
@@ -799,10 +801,10 @@ int launch_t(const BwdTensorArgs& a, int which) {
         using Cfg = KtCfg<D>;
         CUtensorMap mK, mV, mQ, mYh, mYl, mTh, mTl, mGh, mGl, mRS;
         bool ok = make_map_bf16(&mK, a.k, KVU, a.n, D, 128) && make_map_bf16(&mV, a.v, KVU, a.n, D, 128) &&
-                  make_map_bf16(&mQ, a.q, BH, a.n, D, 64) && make_map_bf16(&mYh, a.yh, BH, a.n, D, 64) &&
-                  make_map_bf16(&mYl, a.yl, BH, a.n, D, 64) && make_map_bf16(&mTh, a.tnh, BH, a.n, D, 64) &&
-                  make_map_bf16(&mTl, a.tnl, BH, a.n, D, 64) && make_map_bf16(&mGh, a.gh, BH, a.n, D, 64) &&
-                  make_map_bf16(&mGl, gl, BH, a.n, D, 64) && make_map_f32_rows(&mRS, a.pairsc, BH, (a.n + 1) / 2, 8, 32);
+                  make_map_bf16(&mQ, a.q, BH, a.nq, D, 64) && make_map_bf16(&mYh, a.yh, BH, a.nq, D, 64) &&
+                  make_map_bf16(&mYl, a.yl, BH, a.nq, D, 64) && make_map_bf16(&mTh, a.tnh, BH, a.nq, D, 64) &&
+                  make_map_bf16(&mTl, a.tnl, BH, a.nq, D, 64) && make_map_bf16(&mGh, a.gh, BH, a.nq, D, 64) &&
+                  make_map_bf16(&mGl, gl, BH, a.nq, D, 64) && make_map_f32_rows(&mRS, a.pairsc, BH, (a.nq + 1) / 2, 8, 32);
         if (!ok) return LLA_ERR_CUDA;
         LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_ktile_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
         const dim3 grid(BH, (a.n + 127) / 128);
@@ -814,12 +816,12 @@ int launch_t(const BwdTensorArgs& a, int which) {
     CUtensorMap mQ, mGh, mGl, mTh, mTl, mK, mV;
     const void* th = which == 1 ? a.tnh : a.q;      // the moments kernel loads no T tiles
     const void* tl = which == 1 ? a.tnl : a.q;
-    bool ok = make_map_bf16(&mQ, a.q, BH, a.n, D, 128) && make_map_bf16(&mGh, a.gh, BH, a.n, D, 128) &&
-              make_map_bf16(&mGl, gl, BH, a.n, D, 128) && make_map_bf16(&mTh, th, BH, a.n, D, 128) &&
-              make_map_bf16(&mTl, tl, BH, a.n, D, 128) && make_map_bf16(&mK, a.k, KVU, a.n, D, 64) &&
+    bool ok = make_map_bf16(&mQ, a.q, BH, a.nq, D, 128) && make_map_bf16(&mGh, a.gh, BH, a.nq, D, 128) &&
+              make_map_bf16(&mGl, gl, BH, a.nq, D, 128) && make_map_bf16(&mTh, th, BH, a.nq, D, 128) &&
+              make_map_bf16(&mTl, tl, BH, a.nq, D, 128) && make_map_bf16(&mK, a.k, KVU, a.n, D, 64) &&
               make_map_bf16(&mV, a.v, KVU, a.n, D, 64);
     if (!ok) return LLA_ERR_CUDA;
-    const dim3 grid(BH, (a.n + 127) / 128);
+    const dim3 grid(BH, (a.nq + 127) / 128);
     if (which == 0) {
         LLA_CUDA_TRY(cudaFuncSetAttribute(bwd_qtile_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SM_ALLOC));
         bwd_qtile_tc_kernel<D, 0><<<grid, BT_THREADS, Cfg::SM_ALLOC, a.stream>>>(mQ, mGh, mGl, mTh, mTl, mK, mV, p);

@@ -174,6 +174,8 @@ struct BackwardArgs {
     cudaStream_t stream;
     int kv_group;               // query heads per key/value head (k, v, dk, dv are [B, H / kv_group, n, d])
     int cuda_core_pairs;        // 1: pair kernel on the CUDA cores even where the tensor-core one exists
+    int nq;                     // query rows of the forward being differentiated (0 = n): q, out, dout, rho, stats, dq are
+                                // [B, H, nq, ..] for the positions n - nq .. n - 1
     int window;                 // causal sliding window of the forward being differentiated (0: none)
     int precondition;           // 1: the extra solve runs the preconditioned CG (as ForwardArgs::precondition)
     const unsigned char* block_mask;    // block sparsity of the forward being differentiated (as ForwardArgs::block_mask)
@@ -197,6 +199,7 @@ struct BwdTensorArgs {
     const float* tvec;
     float *kbar, *hvec, *dq, *dk, *dv;
     int B, H, n, d, first, kv_group;
+    int nq;         // query rows (the positions n - nq .. n - 1); the row arrays are [B, H, nq, ..]
     int window;     // causal sliding window (0: none)
     int head_rows;  // with block_mask: key blocks that start below this position are always attended
     const unsigned char* block_mask;    // optional, as ForwardArgs::block_mask

@@ -256,6 +256,51 @@ def test_backward_block_sparse(backward_oracle, d, n, per_head):
     assert grad_err(got[1], dense[1]).max() > 10 * TOL        # (the mask matters)
 
 
+@pytest.mark.parametrize("d,n,nq,window,Hkv", [(64, 700, 300, 0, 0), (64, 300, 260, 0, 0), (128, 640, 200, 0, 0),
+                                                (64, 900, 500, 256, 2)])
+def test_backward_chunk_of_queries(backward_oracle, d, n, nq, window, Hkv):
+    # the gradient of a forward that had only the queries of the last nq positions (q_rows): dq has nq rows, dk and dv
+    # all n.  Cases: the chunk starts beyond the directly-solved positions; it starts among them (some of its rows
+    # are solved directly); d = 128; with a sliding window and grouped key/value heads on top.
+    B, H = 1, 2
+    w = inputs.CONFIGS[2].shrink(B=B, H=H, n=n, d=d, dv=d, seed=320 + d + nq)
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    off = n - nq
+    qc, gc = q[:, :, off:], g[:, :, off:]
+    if Hkv:
+        grp = H // Hkv
+        k, v = k[:, :Hkv], v[:, :Hkv]
+        rq, rk, rv = backward_oracle.backward(qc, np.repeat(k, grp, axis=1), np.repeat(v, grp, axis=1), gc, w.scale, w.lam,
+                                              window=window)
+        rk = rk.reshape(B, Hkv, grp, n, d).sum(axis=2)
+        rv = rv.reshape(B, Hkv, grp, n, d).sum(axis=2)
+    else:
+        rq, rk, rv = backward_oracle.backward(qc, k, v, gc, w.scale, w.lam, window=window)
+    dq_, dk_, dv_, dg = dev(qc, "bf16"), dev(k, "bf16"), dev(v, "bf16"), dev(gc, "f32")
+    out = torch.empty((B, H, nq, d), dtype=torch.float32, device="cuda")
+    rho = torch.empty((B, H, nq, d), dtype=torch.float32, device="cuda")
+    stats = torch.empty((B, H, nq, 3), dtype=torch.float32, device="cuda")
+    L.lla_forward_ex(dq_, dk_, dv_, out, B, H, n, d, d, w.scale, w.lam, out_dtype=L.LLA_F32, rho=rho, stats=stats,
+                     q_rows=nq, window=window, kv_heads=Hkv, stream=stream_ptr())
+    gq = torch.full((B, H, nq, d), float("nan"), dtype=torch.float32, device="cuda")
+    gk = torch.full(k.shape, float("nan"), dtype=torch.float32, device="cuda")
+    gv = torch.full(v.shape, float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = L.lla_backward_workspace_bytes(B, H, n, d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+    L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, gq, gk, gv, B, H, n, d, w.scale, w.lam, device_status=status,
+                      workspace=ws, workspace_bytes=nbytes, q_rows=nq, window=window, kv_heads=Hkv, stream=stream_ptr())
+    torch.cuda.synchronize()
+    st = status.cpu().numpy()
+    assert st[L.STATUS_BAD_PIVOT] == 0 and st[L.STATUS_TIMEOUT] == 0
+    for name, a, r in (("dq", gq, rq), ("dk", gk, rk), ("dv", gv, rv)):
+        a = a.cpu().numpy().astype(np.float64)
+        assert np.isfinite(a).all(), name
+        err = grad_err(a, r)
+        assert err.max() <= TOL, (name, float(err.max()), int(err.argmax()))
+
+
 def test_backward_with_preconditioned_solve(backward_oracle):
     w = inputs.CONFIGS[2].shrink(B=1, H=2, n=640, seed=295)
     q, k, v = inputs.make_prefill(w)
