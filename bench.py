@@ -440,7 +440,8 @@ def run_ours(args):
                 "ms_per_step": 1e3 * e2e_s / e2e_steps,
                 "note": "lla_forward_host on pinned buffers; the host link carries "
                         f"{(h2d + pout.numel() * 2) / 1e6:.0f} MB per step"},
-        "gpu_launches": 2 * args.steps,
+        # per step: the fp16 copy of k, the iterative-rows kernel, the direct-rows kernel
+        "gpu_launches": 3 * args.steps,
     }
     line.update(legs)
     if decode is not None:
