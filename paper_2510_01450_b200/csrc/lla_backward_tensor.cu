@@ -559,22 +559,44 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         bool ok = mbar_wait(bar(QB_QFULL), 0, abort_flag, wcap);
         if (MODE == 1) ok = ok && mbar_wait(bar(QB_YREADY), 0, abort_flag, wcap);
         tc_fence_after();
-        for (int cb = cbeg, c = 0; cb < cend && ok; ++cb) {
-            if (!block_on(cb)) continue;
-            const int s = c % nst;
-            if (!mbar_wait(bar(QB_FULL + s), (c / nst) & 1, abort_flag, wcap)) break;
-            tc_fence_after();
-            const uint32_t st = sb_u + stage_base(s);
-            const uint64_t kdesc = make_desc(st), vdesc = make_desc(st + T64);
-            auto score = [&](uint32_t col, int aoff, uint64_t bdesc, uint32_t acc) {
-                const uint64_t adesc = make_desc(sb_u + aoff);
+        auto next_block = [&](int cb) { while (cb < cend && !block_on(cb)) ++cb; return cb; };
+        auto score = [&](uint32_t st, uint32_t col, int aoff, bool v_tile, uint32_t acc) {
+            const uint64_t adesc = make_desc(sb_u + aoff), bdesc = make_desc(st + (v_tile ? T64 : 0));
 #pragma unroll
-                for (int sub = 0; sub < KSUB; ++sub)
-                    mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
-            };
+            for (int sub = 0; sub < KSUB; ++sub)
+                mma_ss_k64(el, tm_u + col, adesc + sub * (16384 >> 4), bdesc + sub * (8192 >> 4), BT_IDESC_SS, acc | (sub > 0));
+        };
+        // S = Q K^T of visited block number c (waits for its stage); the weights can be formed as soon as it is done
+        auto issue_s = [&](int c) -> bool {
+            const int s = c % nst;
+            if (!mbar_wait(bar(QB_FULL + s), (c / nst) & 1, abort_flag, wcap)) return false;
+            tc_fence_after();
+            score(sb_u + stage_base(s), Cfg::C_S, Cfg::SM_Q, false, 0);
+            tc_commit_el(el, bar(QB_SF1));
+            return true;
+        };
+        auto issue_g = [&](int c) {
+            const uint32_t st = sb_u + stage_base(c % nst), cg = MODE == 1 ? Cfg::C_G1 : Cfg::C_G0;
+            score(st, cg, Cfg::SM_GH, true, 0);
+            if (prm.has_glo) score(st, cg, Cfg::SM_GL, true, 1);
+        };
+        // The score products of the next block are issued as early as the columns they overwrite allow: S as soon as
+        // the compute warps have read the current S (they signal it on PRA: with the weights stored in the moments
+        // kernel, after the read in the dQ kernel, whose coefficient tile goes to the E columns), Gamma in the moments
+        // kernel right after the product that read the current one.  The tensor pipe runs its instructions in order,
+        // so a product issued after the one that reads a tile may overwrite that tile.
+        int cb = next_block(cbeg);
+        ok = ok && cb < cend && issue_s(0);
+        if (ok && MODE == 0) {
+            issue_g(0);
+            tc_commit_el(el, bar(QB_SF2));
+        }
+        for (int c = 0; ok && cb < cend; ++c) {
+            const int s = c % nst;
+            const uint32_t st = sb_u + stage_base(s);
+            const uint64_t kdesc = make_desc(st);
             const uint64_t kmn = make_desc(st, 8192);       // the K block read MN-major, N = D
-            score(Cfg::C_S, Cfg::SM_Q, kdesc, 0);
-            tc_commit_el(el, bar(QB_SF1));      // the weights can be formed while the other products run
+            const int nb = next_block(cb + 1);
             if (MODE == 1) {
                 // E = Y K^T with y (hi, then lo) from TMEM: D / 16 steps of 8 columns each
 #pragma unroll
@@ -583,24 +605,33 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     for (int sub = 0; sub < KSUB; ++sub)
                         mma_ts_kmajor_k64(el, tm_u + Cfg::C_E, tm_u + Cfg::C_Y + part * (D / 2) + 32 * sub, kdesc + sub * (8192 >> 4),
                                           BT_IDESC_SS, (part | sub) > 0);
-                score(Cfg::C_F, Cfg::SM_TH, kdesc, 0);
-                score(Cfg::C_F, Cfg::SM_TL, kdesc, 1);
-            }
-            const uint32_t cg = MODE == 1 ? Cfg::C_G1 : Cfg::C_G0;
-            score(cg, Cfg::SM_GH, vdesc, 0);
-            if (prm.has_glo) score(cg, Cfg::SM_GL, vdesc, 1);
-            tc_commit_el(el, bar(QB_SF2));
-            if (MODE == 0) {
+                score(st, Cfg::C_F, Cfg::SM_TH, false, 0);
+                score(st, Cfg::C_F, Cfg::SM_TL, false, 1);
+                issue_g(c);
+                tc_commit_el(el, bar(QB_SF2));
+                if (nb < cend) {
+                    if (!mbar_wait(bar(QB_PRA), c & 1, abort_flag, wcap)) break;      // S of this block has been read
+                    if (!issue_s(c + 1)) break;
+                }
+                if (!mbar_wait(bar(QB_PRB), c & 1, abort_flag, wcap)) break;
+                tc_fence_after();
+                mma_ts_hilo_k64(el, tm_u + Cfg::C_DQ, tm_u + Cfg::C_E, kmn, Cfg::IDESC_TS, c > 0);
+                tc_commit_el(el, bar(QB_EMPTY + s));
+            } else {
                 if (!mbar_wait(bar(QB_PRA), c & 1, abort_flag, wcap)) break;
                 tc_fence_after();
                 mma_ts_hilo_k64(el, tm_u + Cfg::C_KB, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
+                if (nb < cend && !issue_s(c + 1)) break;
+                if (!mbar_wait(bar(QB_PRB), c & 1, abort_flag, wcap)) break;
+                tc_fence_after();
+                mma_ts_hilo_k64(el, tm_u + Cfg::C_H, tm_u + Cfg::C_G0, kmn, Cfg::IDESC_TS, c > 0);
+                tc_commit_el(el, bar(QB_EMPTY + s));
+                if (nb < cend) {
+                    issue_g(c + 1);
+                    tc_commit_el(el, bar(QB_SF2));
+                }
             }
-            if (!mbar_wait(bar(QB_PRB), c & 1, abort_flag, wcap)) break;
-            tc_fence_after();
-            if (MODE == 1) mma_ts_hilo_k64(el, tm_u + Cfg::C_DQ, tm_u + Cfg::C_S, kmn, Cfg::IDESC_TS, c > 0);
-            else mma_ts_hilo_k64(el, tm_u + Cfg::C_H, tm_u + Cfg::C_G0, kmn, Cfg::IDESC_TS, c > 0);
-            tc_commit_el(el, bar(QB_EMPTY + s));
-            ++c;
+            cb = nb;
         }
         tc_commit_el(el, bar(QB_ACCFULL));      // the last block's products (at least the diagonal blocks were visited)
         if (*abort_flag) {
@@ -674,6 +705,11 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
 #pragma unroll
                 for (int e2 = 0; e2 < 16; ++e2) p2[e2] = ex2_2(fma2(pku(sv[2 * e2], sv[2 * e2 + 1]), c1c1, nm22));
+                if (MODE == 1) {      // S has been read: the next block's S may take its place
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(QB_PRA));
+                }
                 if (MODE == 0) {      // P over S, ready for kbar += P K while Gamma is still being formed
                     uint32_t pp[32];
 #pragma unroll
@@ -709,7 +745,7 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const uint64_t inner = fma2(g2, sub2(one2, evv), fma2(u, evv, add2(f2, kk2)));
                         pd[e2] = split2(mul2(mul2(p2[8 * chunk + e2], sc2), inner), pd[8 + e2]);
                     }
-                    tmem_st16(tm_lane + Cfg::C_S + colbase, pd);
+                    tmem_st16(tm_lane + Cfg::C_E + colbase, pd);      // over the E columns this thread has just read
                 } else {
                     uint32_t gv[16], pg[16];
                     tmem_ld16(tm_lane + Cfg::C_G0 + colbase, gv);
