@@ -402,6 +402,10 @@ typedef struct lla_backward_params {
     int q_rows;   /* as in lla_forward_params: the forward being differentiated had only the queries of the last q_rows
                      positions (0 = n); q, out, dout, rho, stats, dq, iters and dlambda are then [B, H, q_rows, ..],
                      k, v, dk, dv keep n rows.  Not with a block mask or impl = LLA_IMPL_SIMT: LLA_ERR_UNSUPPORTED */
+    long long debug_wait_clocks; /* as in lla_forward_params, for the solve and the tensor-core kernels of this pass */
+    int debug_flags;             /* LLA_DEBUG_NO_LOADS: their copy-issuing warps issue nothing, every bounded wait
+                                    expires with nothing in flight, the blocks leave without results and
+                                    device_status[LLA_STATUS_TIMEOUT] counts them; the call still returns LLA_OK */
 } lla_backward_params;
 
 int lla_backward_ex(const lla_backward_params *p);

@@ -45,6 +45,7 @@ class BackwardParams(ctypes.Structure):
         ("stream", ctypes.c_void_p), ("iters", ctypes.c_void_p), ("dlambda", ctypes.c_void_p), ("impl", ctypes.c_int), ("kv_heads", ctypes.c_int),
         ("window", ctypes.c_int), ("cg_precondition", ctypes.c_int),
         ("block_mask", ctypes.c_void_p), ("block_mask_stride", ctypes.c_longlong), ("q_rows", ctypes.c_int),
+        ("debug_wait_clocks", ctypes.c_longlong), ("debug_flags", ctypes.c_int),
     ]
 
 
@@ -228,9 +229,10 @@ def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, i
 def lla_backward_ex(q, k, v, out, dout, rho, stats, dq, dk, dv, B, H, n, d, scale, lam, out_dtype=LLA_F32,
                     dout_dtype=LLA_F32, max_iters=0, tol=0.0, head_rows=0, device_status=None, workspace=None,
                     workspace_bytes=0, stream=0, impl=LLA_IMPL_AUTO, iters=None, dlambda=None, kv_heads=0, window=0,
-                    cg_precondition=0, block_mask=None, block_mask_stride=0, q_rows=0):
+                    cg_precondition=0, block_mask=None, block_mask_stride=0, q_rows=0, debug_wait_clocks=0, debug_flags=0):
     p = BackwardParams()
     p.q_rows = q_rows
+    p.debug_wait_clocks, p.debug_flags = debug_wait_clocks, debug_flags
     p.kv_heads, p.window, p.cg_precondition = kv_heads, window, cg_precondition
     p.block_mask, p.block_mask_stride = _p(block_mask), block_mask_stride
     p.impl, p.iters, p.dlambda = impl, _p(iters), _p(dlambda)

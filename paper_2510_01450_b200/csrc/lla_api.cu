@@ -401,6 +401,9 @@ int lla_backward_ex(const lla_backward_params* p) {
     if (p->q_rows < 0 || p->q_rows > p->n) return LLA_ERR_INVALID_ARG;
     a.nq = p->q_rows > 0 ? p->q_rows : p->n;
     if (a.nq != p->n && (a.cuda_core_pairs || p->block_mask)) return LLA_ERR_UNSUPPORTED;
+    if (p->debug_wait_clocks < 0 || (p->debug_flags & ~LLA_DEBUG_NO_LOADS)) return LLA_ERR_INVALID_ARG;
+    a.wait_clocks = p->debug_wait_clocks;
+    a.no_loads = (p->debug_flags & LLA_DEBUG_NO_LOADS) ? 1 : 0;
     SideStream* side = side_stream();
     std::unique_lock<std::mutex> side_lock;
     if (side) {

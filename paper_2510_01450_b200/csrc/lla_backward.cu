@@ -700,6 +700,7 @@ int launch_t(const BackwardArgs& a) {
             t.kbar = kbar; t.hvec = hvec; t.dq = a.dq; t.dk = a.dk; t.dv = a.dv;
             t.B = a.B; t.H = a.H; t.n = a.n; t.nq = nq; t.d = D; t.first = first; t.kv_group = kvg; t.window = a.window;
             t.head_rows = a.head_rows; t.block_mask = a.block_mask; t.block_mask_stride = a.block_mask_stride;
+            t.wait_clocks = a.wait_clocks; t.no_loads = a.no_loads;
             t.scale = a.scale; t.status = a.status; t.stream = a.stream;
             const int rc = launch_backward_tensor(t, 0);
             if (rc != LLA_OK) return rc;
@@ -721,6 +722,7 @@ int launch_t(const BackwardArgs& a) {
         f.status = a.status; f.iters = a.iters; f.stream = a.stream;
         f.ridge_mode = LLA_RIDGE_DEFINITION; f.nq = nq; f.kv_group = kvg; f.window = a.window;
         f.block_mask = a.block_mask; f.block_mask_stride = a.block_mask_stride;
+        f.wait_clocks = a.wait_clocks; f.no_loads = a.no_loads;
         f.rhs = hvec; f.sol = tvec;
         f.kbar_in = kbar; f.stats_in = a.stats;      // kbar from the moments kernel, shift and omega as the forward saved them
         f.precondition = a.precondition;      // optional: the extra solve preconditioned (the matrices come from the pre-pass below)

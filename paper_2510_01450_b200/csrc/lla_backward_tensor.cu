@@ -59,7 +59,8 @@ struct BtParams {
     float* dk;
     float* dv;
     int* status;
-    long long wait_clocks;
+    long long wait_clocks;    // cap of every bounded wait, in SM clocks
+    int no_loads;             // test aid: the TMA warp issues no copy at all, so that every wait expires with nothing in flight
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -184,7 +185,7 @@ bwd_ktile_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
     if (warp == 8) {
         // ================================ TMA producer ================================
-        if (lane == 0) {
+        if (lane == 0 && !prm.no_loads) {
             mbar_expect_tx(bar(KB_KV), 2 * Cfg::T128);
             for (int sub = 0; sub < KSUB; ++sub) {
                 tma_load_3d(sbase + Cfg::SM_K + sub * 16384, &tmK, bar(KB_KV), 64 * sub, j0, kvu);
@@ -521,7 +522,7 @@ bwd_qtile_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     if (warp == 8) {
         // ================================ TMA producer ================================
-        if (lane == 0) {
+        if (lane == 0 && !prm.no_loads) {
             const int ntile = (MODE == 1 ? 4 : 2) + (prm.has_glo ? 1 : 0);
             mbar_expect_tx(bar(QB_QFULL), ntile * T128);
             for (int sub = 0; sub < KSUB; ++sub) {
@@ -831,7 +832,8 @@ int launch_t(const BwdTensorArgs& a, int which) {
     p.head_rows = a.head_rows; p.block_mask = a.block_mask; p.block_mask_stride = a.block_mask_stride; p.has_glo = a.gl != nullptr; p.scale = a.scale;
     p.stats = a.stats; p.pairsc = a.pairsc; p.npair = (a.nq + 1) / 2; p.yvec = a.yvec; p.tvec = a.tvec; p.rowsc_w = a.rowsc;
     p.kbar = a.kbar; p.hvec = a.hvec; p.dq = a.dq; p.dk = a.dk; p.dv = a.dv; p.status = a.status;
-    p.wait_clocks = kWaitClocks;
+    p.wait_clocks = a.wait_clocks > 0 ? a.wait_clocks : kWaitClocks;
+    p.no_loads = a.no_loads;
     const void* gl = a.gl ? a.gl : a.gh;        // a valid map either way; never loaded without a lo half
     if (which == 2) {
         using Cfg = KtCfg<D>;

@@ -178,6 +178,8 @@ struct BackwardArgs {
                                 // [B, H, nq, ..] for the positions n - nq .. n - 1
     int window;                 // causal sliding window of the forward being differentiated (0: none)
     int precondition;           // 1: the extra solve runs the preconditioned CG (as ForwardArgs::precondition)
+    long long wait_clocks;      // as ForwardArgs::wait_clocks / no_loads, for the solve and the tensor-core kernels
+    int no_loads;
     const unsigned char* block_mask;    // block sparsity of the forward being differentiated (as ForwardArgs::block_mask)
     long long block_mask_stride;
     cudaStream_t side_stream;   // optional: the directly-solved rows run here, forked from and joined to `stream`
@@ -201,6 +203,8 @@ struct BwdTensorArgs {
     int B, H, n, d, first, kv_group;
     int nq;         // query rows (the positions n - nq .. n - 1); the row arrays are [B, H, nq, ..]
     int window;     // causal sliding window (0: none)
+    long long wait_clocks;  // cap of the kernels' bounded waits in SM clocks (0: default) and a test aid: issue no copy at
+    int no_loads;           // all (lla_backward_params.debug_*)
     int head_rows;  // with block_mask: key blocks that start below this position are always attended
     const unsigned char* block_mask;    // optional, as ForwardArgs::block_mask
     long long block_mask_stride;

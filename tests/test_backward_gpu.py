@@ -301,6 +301,42 @@ def test_backward_chunk_of_queries(backward_oracle, d, n, nq, window, Hkv):
         assert err.max() <= TOL, (name, float(err.max()), int(err.argmax()))
 
 
+def test_backward_bounded_waits_run_out_and_the_context_stays_usable(backward_oracle):
+    # Failure detection without a fault, as in the forward: the copy-issuing warps of the solve and of the three
+    # tensor-core kernels issue nothing, so every bounded wait runs out (cap 2^20 clocks) with no copy or MMA in
+    # flight; the blocks release their tensor memory and leave, the status words count them, the call returns
+    # normally, and the next calls on the same context are correct.
+    w = inputs.CONFIGS[2].shrink(B=1, H=1, n=256, seed=330)
+    q, k, v = inputs.make_prefill(w)
+    g = inputs.make_upstream_grad(w)
+    ref = backward_oracle.backward(q, k, v, g, w.scale, w.lam)
+    dq_, dk_, dv_, dg = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16"), dev(g, "f32")
+    shape = (1, 1, w.n, w.d)
+    out, rho = (torch.empty(shape, dtype=torch.float32, device="cuda") for _ in range(2))
+    stats = torch.empty((1, 1, w.n, 3), dtype=torch.float32, device="cuda")
+    L.lla_forward_ex(dq_, dk_, dv_, out, 1, 1, w.n, w.d, w.d, w.scale, w.lam, out_dtype=L.LLA_F32, rho=rho, stats=stats,
+                     stream=stream_ptr())
+    nbytes = L.lla_backward_workspace_bytes(1, 1, w.n, w.d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+
+    def run(**kw):
+        grads = [torch.full(shape, float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+        L.lla_backward_ex(dq_, dk_, dv_, out, dg, rho, stats, *grads, 1, 1, w.n, w.d, w.scale, w.lam, device_status=status,
+                          workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), **kw)
+        torch.cuda.synchronize()
+        return [t.cpu().numpy().astype(np.float64) for t in grads], status.cpu().tolist()
+
+    _, st = run(debug_wait_clocks=1 << 20, debug_flags=L.LLA_DEBUG_NO_LOADS)
+    # two query tiles in each of the moments, solve and dQ kernels, two key tiles in the dK/dV kernel
+    assert st[L.STATUS_TIMEOUT] == 8
+    for _ in range(2):
+        grads, st = run()
+        assert st[L.STATUS_TIMEOUT] == 0
+        for name, a, b in zip(("dq", "dk", "dv"), grads, ref):
+            assert grad_err(a, b).max() <= TOL, name
+
+
 def test_backward_with_preconditioned_solve(backward_oracle):
     w = inputs.CONFIGS[2].shrink(B=1, H=2, n=640, seed=295)
     q, k, v = inputs.make_prefill(w)
