@@ -47,7 +47,7 @@ constexpr int SMD_FIN = 8 * (64 * 65 + 3 * 64) + 4 * 64 * 65 + 8 * (128 + 24);
 constexpr int SMD_ALLOC = (SMD_TOTAL > SMD_FIN ? SMD_TOTAL : SMD_FIN) + 1024;
 
 enum { DB_KVFULL = 0, DB_KVEMPTY = DB_KVFULL + DT_NST, DB_BFULL = DB_KVEMPTY + DT_NST, DB_BFREE = DB_BFULL + 2,
-       DB_DFULL = DB_BFREE + 2, DB_PASS = DB_DFULL + 1, DB_COUNT = DB_PASS + 1 };
+       DB_DFULL = DB_BFREE + 2, DB_PASS = DB_DFULL + 1, DB_EXIT = DB_PASS + 1, DB_COUNT = DB_EXIT + 1 };
 static_assert(DB_COUNT * 8 <= 128, "barrier area too small");
 
 // A = [K^T ; V^T]: MN-major, 128B swizzle; the V tile (second group of 64 rows of M) lies 8192 bytes
@@ -233,6 +233,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int b = 0; b < 2; ++b) { mbar_init(bar(DB_BFULL + b), DT_COMPUTE / 32); mbar_init(bar(DB_BFREE + b), 1); }
         mbar_init(bar(DB_DFULL), 1);
         mbar_init(bar(DB_PASS), DT_COMPUTE / 32);
+        mbar_init(bar(DB_EXIT), 1);
         misc[1] = 0;
         misc[2] = 0;      // set by the compute warps when the pass has to be repeated
         fence_barrier_init();
@@ -258,11 +259,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group;
             const int kvh = (bh / prm.H) * hkv + kvl;
             const int* table = prm.paged.table ? prm.paged.table + (size_t)(bh / prm.H) * prm.paged.max_pages : nullptr;
+            int issued = 0;      // tiles whose copies have been issued
             for (int g = 0, pass = 0; pass < 2; ++pass) {
               bool okp = true;
               for (int t = 0; t < ntile; ++t, ++g) {      // g: running tile count over both passes (ring position)
                 const uint32_t s = g % DT_NST;
                 if (!mbar_wait(bar(DB_KVEMPTY + s), ((g / DT_NST) & 1) ^ 1, abort_flag)) { okp = false; break; }
+                issued = g + 1;
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
                 int unit = kvh, jrow = kstart + jbeg + t * DT_BK;
@@ -276,6 +279,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
               }
               // a second pass only if the compute warps ask for it
               if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag) || misc[2] == 0) break;
+            }
+            if (*abort_flag) {      // an aborted block: the copies issued above must have landed before the block exits
+                for (int g = max(0, issued - DT_NST); g < issued; ++g)
+                    (void)mbar_wait_landed(bar(DB_KVFULL + g % DT_NST), (g / DT_NST) & 1);
             }
         }
     } else if (warp == 5) {
@@ -295,6 +302,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
             }
             if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag) || misc[2] == 0) break;
+        }
+        if (*abort_flag) {      // an aborted block: the MMAs issued above must be done before TMEM and shared memory go
+            tc_commit_el(el, bar(DB_EXIT));
+            (void)mbar_wait_landed(bar(DB_EXIT), 0);
         }
     } else {
         // ================================ compute warps ================================
@@ -510,8 +521,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     const bool aborted = *abort_flag != 0;
     if (aborted) {
-        for (int i = 0; i < 64; ++i) __nanosleep(1000);
-        if (tid == 0 && prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+        // (the TMA and MMA warps have waited above for what they had issued)
+        if (tid == 0) {
+            if (prm.status) atomicAdd(prm.status + LLA_STATUS_TIMEOUT, 1);
+            if (prm.splits > 1 || prm.defer) {
+                // no record of this part: poison its weight and maximum, so that the solve kernel emits NaN for the
+                // unit instead of reading whatever an earlier call left in the record buffer
+                float* dst = prm.parts + ((size_t)bh * prm.splits + part) * (2 * 64 * 64 + 2 * 64 + 4);
+                dst[2 * 64 * 64 + 128] = __int_as_float(0x7fc00000);
+                dst[2 * 64 * 64 + 129] = __int_as_float(0x7fc00000);
+            }
+        }
         return;
     }
     const float omega_tot = s_omega[0] + s_omega[1] + s_omega[2] + s_omega[3];
