@@ -262,6 +262,10 @@ typedef struct lla_decode_params {
     int page_size, max_pages, num_pages;
     int window;     /* sliding window: 0 = the query sees all lens[b] cached keys; W > 0 = only the last
                        min(W, lens[b]) of them (positions lens[b] - W .. lens[b] - 1).  Not with a paged cache */
+    long long debug_wait_clocks; /* as in lla_forward_params, for the tensor-core streaming kernel (bf16, d = 64) */
+    int debug_flags;             /* LLA_DEBUG_NO_LOADS: its copy-issuing warp issues nothing, every bounded wait expires
+                                    with nothing in flight, device_status[LLA_STATUS_TIMEOUT] counts the blocks and
+                                    their units' outputs are NaN (the record of a block that gave up is poisoned) */
 } lla_decode_params;
 
 int lla_decode_ex(const lla_decode_params *p);

@@ -87,6 +87,7 @@ class DecodeParams(ctypes.Structure):
         ("stream", ctypes.c_void_p), ("lambda_units", ctypes.c_void_p), ("ridge_mode", ctypes.c_int),
         ("kv_heads", ctypes.c_int), ("block_table", ctypes.c_void_p), ("page_size", ctypes.c_int),
         ("max_pages", ctypes.c_int), ("num_pages", ctypes.c_int), ("window", ctypes.c_int),
+        ("debug_wait_clocks", ctypes.c_longlong), ("debug_flags", ctypes.c_int),
     ]
 
 
@@ -212,9 +213,10 @@ def lla_forward_ex(q, k, v, out, B, H, n, d, dv, scale, lam, causal=1, in_dtype=
 def lla_decode_ex(q, kcache, vcache, lens, out, B, H, Lmax, d, dv, scale, lam, in_dtype=LLA_BF16,
                   out_dtype=LLA_BF16, splits=0, impl=LLA_IMPL_AUTO, device_status=None, workspace=None,
                   workspace_bytes=0, stream=0, lambda_units=None, ridge_mode=LLA_RIDGE_DEFINITION, kv_heads=0, block_table=None,
-                  page_size=0, max_pages=0, num_pages=0, window=0):
+                  page_size=0, max_pages=0, num_pages=0, window=0, debug_wait_clocks=0, debug_flags=0):
     p = DecodeParams()
     p.window = window
+    p.debug_wait_clocks, p.debug_flags = debug_wait_clocks, debug_flags
     p.kv_heads = kv_heads
     p.block_table, p.page_size, p.max_pages, p.num_pages = _p(block_table), page_size, max_pages, num_pages
     p.q, p.kcache, p.vcache, p.lens, p.out = _p(q), _p(kcache), _p(vcache), _p(lens), _p(out)

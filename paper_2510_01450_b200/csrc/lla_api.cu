@@ -295,6 +295,9 @@ int lla_decode_ex(const lla_decode_params* p) {
     }
     if (p->window < 0 || (p->window > 0 && p->block_table)) return LLA_ERR_INVALID_ARG;
     a.window = p->window;
+    if (p->debug_wait_clocks < 0 || (p->debug_flags & ~LLA_DEBUG_NO_LOADS)) return LLA_ERR_INVALID_ARG;
+    a.wait_clocks = p->debug_wait_clocks;
+    a.no_loads = (p->debug_flags & LLA_DEBUG_NO_LOADS) ? 1 : 0;
     if (a.status) LLA_CUDA_TRY(cudaMemsetAsync(a.status, 0, sizeof(int) * LLA_STATUS_WORDS, a.stream));
     // The units with short caches go to the direct kernel, which writes rows of `out` nobody else writes and
     // returns at once for every other unit: it runs on the side stream beside the streaming kernel instead of

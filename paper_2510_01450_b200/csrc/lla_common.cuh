@@ -145,6 +145,8 @@ struct DecodeArgs {
     int kv_group = 1;           // query heads per key/value head: caches are [B, H / kv_group, Lmax, d]
     PagedKv paged = {nullptr, 0, 0, 0};
     int window = 0;             // sliding window: only the last `window` cached keys are visible (0: all)
+    long long wait_clocks = 0;  // tensor-core kernel: cap of its bounded waits in SM clocks (0: default) and a test aid:
+    int no_loads = 0;           // issue no copy at all (lla_decode_params.debug_*)
 };
 
 // Backward pass (backward appendix): gradients of a scalar loss with respect to q, k, v given

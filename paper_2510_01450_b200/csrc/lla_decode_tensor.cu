@@ -185,6 +185,8 @@ struct DtParams {
     int ridge_mode;
     int kv_group;        // query heads per key/value head
     int window;          // sliding window (0: none)
+    long long wait_clocks;   // cap of every bounded wait, in SM clocks
+    int no_loads;        // test aid: the TMA warp issues no copy at all, so that every wait expires with nothing in flight
     PagedKv paged;       // table != nullptr: the tensor maps cover [num_pages * kv heads][page_size][64]
 };
 
@@ -200,6 +202,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     volatile int* misc = reinterpret_cast<volatile int*>(smem + SMD_MISC);   // [0] tmem base, [1] abort
     volatile int* abort_flag = misc + 1;
     volatile float* tmax = reinterpret_cast<volatile float*>(smem + SMD_MISC + 16);   // 2 x 4 warp maxima
+    const long long wcap = prm.wait_clocks;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int part = blockIdx.x;
@@ -253,7 +256,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (warp == 4) {
         // ================================ TMA producer ================================
-        if (lane == 0) {
+        if (lane == 0 && !prm.no_loads) {
             // K/V unit and row of a tile in the tensor map: (batch, key/value head) and the key index, or for a
             // paged cache (page, key/value head) and the row inside the page (a tile never straddles a page)
             const int hkv = prm.H / prm.kv_group, kvl = (bh % prm.H) / prm.kv_group;
@@ -264,7 +267,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
               bool okp = true;
               for (int t = 0; t < ntile; ++t, ++g) {      // g: running tile count over both passes (ring position)
                 const uint32_t s = g % DT_NST;
-                if (!mbar_wait(bar(DB_KVEMPTY + s), ((g / DT_NST) & 1) ^ 1, abort_flag)) { okp = false; break; }
+                if (!mbar_wait(bar(DB_KVEMPTY + s), ((g / DT_NST) & 1) ^ 1, abort_flag, wcap)) { okp = false; break; }
                 issued = g + 1;
                 const uint32_t dst = sbase + SMD_KV + s * 16384;
                 mbar_expect_tx(bar(DB_KVFULL + s), 16384);
@@ -278,11 +281,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tma_load_3d(dst + 8192, &tmV, bar(DB_KVFULL + s), 0, jrow, unit);
               }
               // a second pass only if the compute warps ask for it
-              if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag) || misc[2] == 0) break;
+              if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag, wcap) || misc[2] == 0) break;
             }
             if (*abort_flag) {      // an aborted block: the copies issued above must have landed before the block exits
                 for (int g = max(0, issued - DT_NST); g < issued; ++g)
-                    (void)mbar_wait_landed(bar(DB_KVFULL + g % DT_NST), (g / DT_NST) & 1);
+                    (void)mbar_wait_landed(bar(DB_KVFULL + g % DT_NST), (g / DT_NST) & 1, wcap);
             }
         }
     } else if (warp == 5) {
@@ -292,8 +295,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             bool okp = true;
             for (int t = 0; t < ntile; ++t, ++g) {
                 const uint32_t s = g % DT_NST, b = g & 1;
-                if (!mbar_wait(bar(DB_KVFULL + s), (g / DT_NST) & 1, abort_flag)) { okp = false; break; }
-                if (!mbar_wait(bar(DB_BFULL + b), (g >> 1) & 1, abort_flag)) { okp = false; break; }
+                if (!mbar_wait(bar(DB_KVFULL + s), (g / DT_NST) & 1, abort_flag, wcap)) { okp = false; break; }
+                if (!mbar_wait(bar(DB_BFULL + b), (g >> 1) & 1, abort_flag, wcap)) { okp = false; break; }
                 tc_fence_after();
                 const uint32_t bsm = sbase + SMD_B + b * 2 * DT_BTILE;
                 mma_tile(el, tmem, make_desc_a(sbase + SMD_KV + s * 16384), make_desc_b(bsm), t > 0);     // t == 0 overwrites
@@ -301,11 +304,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tc_commit_el(el, bar(DB_BFREE + b));
                 if (t == ntile - 1) tc_commit_el(el, bar(DB_DFULL));
             }
-            if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag) || misc[2] == 0) break;
+            if (!okp || pass == 1 || ntile == 0 || !mbar_wait(bar(DB_PASS), 0, abort_flag, wcap) || misc[2] == 0) break;
         }
         if (*abort_flag) {      // an aborted block: the MMAs issued above must be done before TMEM and shared memory go
             tc_commit_el(el, bar(DB_EXIT));
-            (void)mbar_wait_landed(bar(DB_EXIT), 0);
+            (void)mbar_wait_landed(bar(DB_EXIT), 0, wcap);
         }
     } else {
         // ================================ compute warps ================================
@@ -333,7 +336,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         //  buffer and barrier phase)
         auto stage_load = [&](int g) -> bool {
             const uint32_t s = g % DT_NST;
-            if (!mbar_wait(bar(DB_KVFULL + s), (g / DT_NST) & 1, abort_flag)) return false;
+            if (!mbar_wait(bar(DB_KVFULL + s), (g / DT_NST) & 1, abort_flag, wcap)) return false;
             uint8_t* ktile = smem + SMD_KV + s * 16384;
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -407,7 +410,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const uint32_t b = g & 1;
                 const bool more = t + 1 < ntile;
                 // wait until the MMA of the tile two before has released this B buffer (long done in steady state)
-                if (!mbar_wait(bar(DB_BFREE + b), ((g >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bar(DB_BFREE + b), ((g >> 1) & 1) ^ 1, abort_flag, wcap)) { ok = false; break; }
                 // B rows of tile t: w * [k | 1] as bf16 hi + lo, eight features at a time straight into the
                 // operand tiles, so the stores drain while the rest of the iteration runs
                 uint8_t* bhi = smem + SMD_B + b * 2 * DT_BTILE;
@@ -481,7 +484,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (tid == 0) s_mref = m_ref;
     bool d_ok = true;
     if (warp < 4 && ntile > 0) {
-        d_ok = mbar_wait(bar(DB_DFULL), d_parity, abort_flag);
+        d_ok = mbar_wait(bar(DB_DFULL), d_parity, abort_flag, wcap);
         tc_fence_after();
     }
     // moments -> registers (lane f: row f of M plus a[f]; lane 64+f: row f of N plus c[f])
@@ -733,6 +736,7 @@ int launch_t(const DecodeArgs& a) {
     prm.B = a.B; prm.H = a.H; prm.Lmax = a.Lmax; prm.splits = splits; prm.head_rows = a.head_rows;
     prm.scale = a.scale; prm.lambda = a.lambda; prm.lens = a.lens;
     prm.lambda_units = a.lambda_units; prm.ridge_mode = a.ridge_mode; prm.kv_group = kvg; prm.paged = a.paged; prm.window = a.window;
+    prm.wait_clocks = a.wait_clocks > 0 ? a.wait_clocks : kWaitClocks; prm.no_loads = a.no_loads;
     prm.parts = (float*)a.workspace; prm.status = a.status;
     prm.defer = have_ws ? 1 : 0;      // with a record buffer the solve runs as its own kernel
     auto kern = decode_tc_kernel<TOut>;

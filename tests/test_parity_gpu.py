@@ -320,6 +320,36 @@ def test_bounded_waits_run_out_and_the_context_stays_usable(oracle):
         assert row_err(got, ref).max() <= TOL_BF16
 
 
+@pytest.mark.parametrize("splits", [1, 3])
+def test_decode_bounded_waits_run_out_and_the_context_stays_usable(oracle, splits):
+    # the same for the decode's streaming kernel: no copy is issued, every block's waits run out, the blocks leave
+    # (their records poisoned, so the solve kernel emits NaN rather than what an earlier call left in the workspace),
+    # the time-outs are counted, and the next call is correct
+    w = inputs.CONFIGS[5].shrink(B=2, H=2, n=700, len_min=200, len_max=700, seed=340)
+    q, kc, vc, lens = inputs.make_decode(w)
+    ref = oracle.decode(q, kc, vc, lens, w.scale, w.lam)
+    dq, dk, dv_ = dev(q, "bf16"), dev(kc, "bf16"), dev(vc, "bf16")
+    dl = torch.from_numpy(lens).cuda()
+    nbytes = L.lla_decode_workspace_bytes(w.B, w.H, w.n, w.d, w.dv, L.LLA_BF16, splits)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(L.LLA_STATUS_WORDS, dtype=torch.int32, device="cuda")
+
+    def run(**kw):
+        out = torch.full((w.B, w.H, w.dv), 7.0, dtype=torch.float32, device="cuda")
+        L.lla_decode_ex(dq, dk, dv_, dl, out, w.B, w.H, w.n, w.d, w.dv, w.scale, w.lam, out_dtype=L.LLA_F32, splits=splits,
+                        device_status=status, workspace=ws, workspace_bytes=nbytes, stream=stream_ptr(), **kw)
+        torch.cuda.synchronize()
+        return out.cpu().numpy(), status.cpu().tolist()
+
+    good, st = run()                                   # leaves valid records of these units in the workspace
+    assert st[L.STATUS_TIMEOUT] == 0 and row_err(good, ref).max() <= TOL_BF16
+    got, st = run(debug_wait_clocks=1 << 20, debug_flags=L.LLA_DEBUG_NO_LOADS)
+    assert w.B * w.H <= st[L.STATUS_TIMEOUT] <= w.B * w.H * splits      # every part that has keys (a short cache's last parts are empty)
+    assert np.isnan(got).all()
+    got, st = run()
+    assert st[L.STATUS_TIMEOUT] == 0 and row_err(got, ref).max() <= TOL_BF16
+
+
 def test_host_buffer_forward_from_two_threads(oracle):
     # two host threads, each with its own stream and its own problem, in the chunked host-buffer form at the same
     # time: the library's worker streams and events are shared per device, so the calls must not mix them up
