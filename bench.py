@@ -557,6 +557,10 @@ def bench_backward(L, torch, peaks, pre, local, steps=20, warmup=3, nsets=4):
     return {"workload": w.name, "ms_per_step": ms, "tokens_per_s": w.B * w.n / (ms * 1e-3),
             "tflops": flops / (ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                         "kernel": "the whole pass (eight launches: solve, dK/dV, dQ, moments, direct rows, ...; profiles/backward_cfg3.md)",
+                         "peak_source": f"{peaks['source']} burst bf16 (MEASURED_PEAKS.json)"},
             "cg_mean_iters": float(it[it >= 0].mean()) if (it >= 0).any() else 0.0,
             "preconditioned": {"ms_per_step": ms_pc, "cg_mean_iters": float(it_pc[it_pc >= 0].mean()) if (it_pc >= 0).any() else 0.0,
                                "note": "optional mode (lla_backward_params.cg_precondition = 1)"},
